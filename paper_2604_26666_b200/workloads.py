@@ -1,0 +1,171 @@
+"""Seeded synthetic inputs and the shape table of the benchmark configurations.
+
+This module holds NO arithmetic of the method (no product, no epilogue): it
+only names shapes and draws random BF16 tensors on the CPU.  Both the CUDA
+path and the CPU oracle are fed from here, so that they see the same bits.
+
+The shapes stand in for the workloads of the paper's evaluation (Section 5.1
+"Benchmark problems": square, batched and large-K matrix products; Section 5.2:
+the linear layers of the MiniGPT block and of the Llama-3-8B decoder block),
+at the sizes and value distributions the benchmark configurations state.
+None of the original benchmark files or model weights is used.
+
+Recipe (identical for every case): draw FP32 values from a
+``torch.Generator(device="cpu")`` seeded with the case's seed, in the order
+X/A, W/B, bias, residual; scale in FP32; round once to BF16 (nearest even).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Optional
+
+import torch
+
+
+@dataclass(frozen=True)
+class Case:
+    """One GEMM-family problem.  ``N`` is the number of OUTPUT columns; the
+    weight has ``2 * N`` columns for SILU_GATE (gate first, then up)."""
+
+    name: str
+    op: str  # "gemm" | "gemm_batched" | "gemm_splitk" | "linear"
+    M: int
+    N: int
+    K: int
+    batch: int = 1
+    epilogue: str = "NONE"
+    layout: str = "KN"  # "KN": B[K x N] (torch.matmul);  "NK": W[N x K] (nn.Linear.weight)
+    out: str = "bf16"  # "bf16" | "f32"
+    has_bias: bool = False
+    has_residual: bool = False
+    seed: int = 0
+    x_dist: str = "normal"  # "normal" | "uniform"  (uniform = U(-1, 1))
+    w_dist: str = "normal"
+    x_scale: float = 1.0
+    w_scale: float = 1.0
+    config: int = 0  # 1-based index of the benchmark configuration this case belongs to
+
+    @property
+    def n_weight_cols(self) -> int:
+        return 2 * self.N if self.epilogue == "SILU_GATE" else self.N
+
+    @property
+    def flops(self) -> float:
+        """2 * batch * M * (weight columns) * K -- the accounting of the paper's
+        Section 5.2 throughput figures (epilogue work is not counted)."""
+        return 2.0 * self.batch * self.M * self.n_weight_cols * self.K
+
+    @property
+    def out_bytes_per_elem(self) -> int:
+        return 4 if self.out == "f32" else 2
+
+    @property
+    def algorithmic_bytes(self) -> float:
+        """Each operand read once plus the output written once."""
+        b = self.batch * (self.M * self.K + self.K * self.n_weight_cols) * 2
+        b += self.batch * self.M * self.N * self.out_bytes_per_elem
+        if self.has_bias:
+            b += self.N * 2
+        if self.has_residual:
+            b += self.batch * self.M * self.N * 2
+        return float(b)
+
+
+def _k_inv_sqrt(k: int) -> float:
+    return float(k) ** -0.5
+
+
+def benchmark_cases(layout_linear: str = "NK") -> list[Case]:
+    """The thirteen shapes of the five benchmark configurations."""
+    c: list[Case] = []
+    # config 1: C = ReLU(A.B + bias), 512^3, U(-1,1) operands, N(0,1) bias, seed 0
+    c.append(Case("c1_512_bias_relu", "linear", 512, 512, 512, epilogue="BIAS_RELU", layout="KN",
+                  has_bias=True, seed=0, x_dist="uniform", w_dist="uniform", config=1))
+    # config 2: square GEMMs, operands N(0,1)/sqrt(K), seed 1
+    for n in (4096, 8192):
+        c.append(Case(f"c2_square_{n}", "gemm", n, n, n, layout="KN", seed=1,
+                      x_scale=_k_inv_sqrt(n), w_scale=_k_inv_sqrt(n), config=2))
+    # config 3: batched GEMM + large-K FP32-output split-K GEMM, seed 2
+    c.append(Case("c3_batched_128x512x512x1024", "gemm_batched", 512, 512, 1024, batch=128, layout="KN",
+                  seed=2, config=3))
+    c.append(Case("c3_splitk_256x256x131072", "gemm_splitk", 256, 256, 131072, layout="KN", out="f32",
+                  seed=2, x_dist="uniform", w_dist="uniform", config=3))
+    # config 4: GPT-style block linears, 16384 tokens, d_model 768, MLP 3072, seed 3
+    L = layout_linear
+    c.append(Case("c4_qkv", "linear", 16384, 2304, 768, epilogue="BIAS", layout=L, has_bias=True,
+                  seed=3, w_scale=0.02, config=4))
+    c.append(Case("c4_out_proj", "linear", 16384, 768, 768, epilogue="BIAS_RESIDUAL", layout=L,
+                  has_bias=True, has_residual=True, seed=3, w_scale=0.02, config=4))
+    c.append(Case("c4_mlp_up_gelu", "linear", 16384, 3072, 768, epilogue="BIAS_GELU_TANH", layout=L,
+                  has_bias=True, seed=3, w_scale=0.02, config=4))
+    c.append(Case("c4_mlp_down", "linear", 16384, 768, 3072, epilogue="BIAS_RESIDUAL", layout=L,
+                  has_bias=True, has_residual=True, seed=3, w_scale=0.02, config=4))
+    # config 5: Llama-3-8B-shaped linears, 8192 tokens, hidden 4096, MLP 14336, seed 4
+    c.append(Case("c5_qkv", "linear", 8192, 6144, 4096, epilogue="NONE", layout=L, seed=4,
+                  w_scale=0.02, config=5))
+    c.append(Case("c5_o_proj", "linear", 8192, 4096, 4096, epilogue="BIAS_RESIDUAL", layout=L,
+                  has_residual=True, seed=4, w_scale=0.02, config=5))
+    c.append(Case("c5_gate_up_silu", "linear", 8192, 14336, 4096, epilogue="SILU_GATE", layout=L,
+                  seed=4, w_scale=0.02, config=5))
+    c.append(Case("c5_down", "linear", 8192, 4096, 14336, epilogue="BIAS_RESIDUAL", layout=L,
+                  has_residual=True, seed=4, w_scale=0.02, config=5))
+    return c
+
+
+def case_by_name(name: str, layout_linear: str = "NK") -> Case:
+    for cs in benchmark_cases(layout_linear):
+        if cs.name == name:
+            return cs
+    raise KeyError(name)
+
+
+def _draw(gen: torch.Generator, shape, dist: str, scale: float) -> torch.Tensor:
+    if dist == "normal":
+        t = torch.randn(shape, generator=gen, dtype=torch.float32)
+    elif dist == "uniform":
+        t = torch.rand(shape, generator=gen, dtype=torch.float32) * 2.0 - 1.0
+    else:
+        raise ValueError(dist)
+    if scale != 1.0:
+        t = t * scale
+    return t.to(torch.bfloat16)
+
+
+@dataclass
+class Inputs:
+    X: torch.Tensor  # bf16 [M,K] or [batch,M,K]
+    W: torch.Tensor  # bf16 [K,Nw] / [Nw,K] (or batched)
+    bias: Optional[torch.Tensor] = None  # bf16 [N]
+    residual: Optional[torch.Tensor] = None  # bf16 [M,N] (or batched)
+    extra: dict = field(default_factory=dict)
+
+
+def make_inputs(case: Case, gen: Optional[torch.Generator] = None, pin: bool = False) -> Inputs:
+    """Draw the case's inputs on the CPU (BF16).  ``gen`` lets a caller continue
+    one generator across the cases of a configuration; by default a fresh
+    generator seeded with ``case.seed`` is used."""
+    if gen is None:
+        gen = torch.Generator(device="cpu")
+        gen.manual_seed(case.seed)
+    b = (case.batch,) if case.batch > 1 else ()
+    Nw = case.n_weight_cols
+    X = _draw(gen, b + (case.M, case.K), case.x_dist, case.x_scale)
+    wshape = (case.K, Nw) if case.layout == "KN" else (Nw, case.K)
+    W = _draw(gen, b + wshape, case.w_dist, case.w_scale)
+    bias = _draw(gen, (case.N,), "normal", 1.0) if case.has_bias else None
+    residual = _draw(gen, b + (case.M, case.N), "normal", 1.0) if case.has_residual else None
+    ins = Inputs(X, W, bias, residual)
+    if pin:
+        for f in ("X", "W", "bias", "residual"):
+            t = getattr(ins, f)
+            if t is not None:
+                setattr(ins, f, t.pin_memory())
+    return ins
+
+
+def bits(t: torch.Tensor):
+    """BF16 tensor (CPU) -> numpy uint16 view of its bit patterns (no copy)."""
+    import numpy as np
+
+    assert t.dtype == torch.bfloat16 and t.device.type == "cpu"
+    return t.view(torch.int16).numpy().view(np.uint16)
