@@ -1,0 +1,222 @@
+/*
+ * libfact -- fused-epilogue BF16 GEMMs for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The library computes the GEMM family of the paper's evaluation: the three
+ * matrix-product problems of Section 5.1 "Benchmark problems" (Problem 1: one
+ * square product, data-parallel tiles; Problem 3: a batch of independent
+ * products; Problem 6: a product with a very long K, cut along K) and the
+ * linear layers that Section 5.2 fuses with their element-wise successors
+ * (MiniGPT pattern p2: Linear + GELU, Linear + standard epilogue; Llama
+ * pattern p2: SiLU(gate) x up, down projection).
+ *
+ * Conventions shared by every entry point
+ *   - All matrix pointers are DEVICE pointers on the handle's device.  Only
+ *     the handle, the status/size out-parameters, config structs and file
+ *     paths are host memory.
+ *   - Matrices are row-major.  Leading dimensions (ld*) and batch strides are
+ *     in ELEMENTS.  Inputs are BF16; products are accumulated in FP32; the
+ *     output is BF16 (round to nearest even, once, after the epilogue) or
+ *     FP32.
+ *   - Operand loads go through TMA, hence: every operand base pointer (A/X,
+ *     B/W) must be 16-byte aligned and its leading dimension and batch stride
+ *     a multiple of 8 elements.  Output and residual rows are written/read in
+ *     16-byte vectors when the pointer is 16-byte aligned and the leading
+ *     dimension a multiple of 8 (BF16) / 4 (FP32) elements; otherwise element
+ *     by element (slower, still correct).  M, N, K themselves are arbitrary.
+ *   - Ownership: the caller owns every buffer and the stream.  The library
+ *     never allocates or frees device memory on a call path; split-K scratch
+ *     is a caller-provided workspace sized by fact_workspace_bytes.  The handle
+ *     owns a small device status word, a cache of encoded tensor maps and the
+ *     tuner's table.
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and return; results are valid
+ *     in stream order.
+ *   - Errors: a status code is returned; argument errors are detected before
+ *     anything is launched and leave the outputs untouched.  There is no CPU
+ *     fallback and no library GEMM fallback: on a device that is not sm_100
+ *     fact_create fails with FACT_ERR_ARCH.
+ *   - A handle must not be used from two host threads at once.
+ *   - M == 0 or N == 0 (or batch == 0) is a successful no-op.  K == 0 applies
+ *     the epilogue to a zero accumulator.
+ */
+#ifndef FACT_H_
+#define FACT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fact_handle_s* fact_handle_t;
+
+typedef enum {
+  FACT_OK = 0,
+  FACT_ERR_INVALID_ARG = 1,         /* null pointer, negative size, bad enum, inconsistent arguments */
+  FACT_ERR_BAD_ALIGNMENT = 2,       /* operand pointer / leading dimension breaks the 16-byte TMA rule */
+  FACT_ERR_UNSUPPORTED = 3,         /* a config the kernels cannot run (tile shape, smem/TMEM budget) */
+  FACT_ERR_ARCH = 4,                /* device is not sm_100 */
+  FACT_ERR_WORKSPACE_TOO_SMALL = 5, /* split-K needs more scratch than was passed */
+  FACT_ERR_CUDA = 6,                /* a CUDA runtime/driver call failed */
+  FACT_ERR_DEVICE_TIMEOUT = 7       /* a bounded device-side wait expired (reported by fact_device_status) */
+} fact_status_t;
+
+/* Element-wise work fused into the GEMM epilogue (computed in FP32 on the
+ * accumulator, before the single rounding to the output type):
+ *   NONE            y = acc                                   (Section 5.1 problems)
+ *   BIAS            y = acc + bias[n]
+ *   BIAS_RELU       y = max(acc + bias[n], 0)
+ *   BIAS_GELU_TANH  z = acc + bias[n];  y = 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
+ *                                                             (Section 5.2, MiniGPT p2 GEMM 1)
+ *   SILU_GATE       y = silu(acc[m, n]) * acc[m, N_out + n],  silu(g) = g / (1 + exp(-g))
+ *                   W carries 2*N_out columns: gate columns first, then up columns
+ *                                                             (Section 5.2, Llama p2 GEMM 1)
+ *   BIAS_RESIDUAL   y = acc + bias[n] + R[m, n]   (bias may be NULL)
+ *                                                             (GEMM 2 of both blocks + the residual add) */
+typedef enum {
+  FACT_EPI_NONE = 0,
+  FACT_EPI_BIAS = 1,
+  FACT_EPI_BIAS_RELU = 2,
+  FACT_EPI_BIAS_GELU_TANH = 3,
+  FACT_EPI_SILU_GATE = 4,
+  FACT_EPI_BIAS_RESIDUAL = 5
+} fact_epilogue_t;
+
+typedef enum { FACT_OUT_BF16 = 0, FACT_OUT_F32 = 1 } fact_out_t;
+
+/* Storage of the second operand. */
+typedef enum {
+  FACT_B_KN = 0, /* B[K x N], N contiguous  (torch.matmul(A, B))      */
+  FACT_B_NK = 1  /* W[N x K], K contiguous  (torch.nn.Linear.weight)  */
+} fact_blayout_t;
+
+/* Which entry point a workspace / tuning query is about. */
+typedef enum { FACT_OP_GEMM = 0, FACT_OP_GEMM_BATCHED = 1, FACT_OP_GEMM_SPLITK = 2, FACT_OP_LINEAR = 3 } fact_op_t;
+
+/* One kernel configuration.  A zero field means "let the library choose".
+ *   tile_m       128 (one CTA per tile) or 256 (a 2-CTA cluster per tile; then cta_group must be 2)
+ *   tile_n       accumulator columns per tile, a multiple of 16 in [32, 256] (FACT_B_KN: multiple of 64;
+ *                SILU_GATE: multiple of 32, half gate + half up)
+ *   tile_k       64 (one 128-byte swizzle row of BF16)
+ *   stages       depth of the shared-memory ring, 2..8, limited by 227 KB
+ *   cta_group    1 or 2
+ *   raster_group number of M-tiles walked before moving to the next N-tile (L2 reuse), >= 1
+ *   split_k      number of K slices, >= 1 (> 1 needs a workspace)
+ *   store_mode   0 = library default, 1 = direct register stores, 2 = shared-memory staged stores */
+typedef struct {
+  int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode;
+} fact_config_t;
+
+/* Create / destroy a handle bound to CUDA device `device`.  fact_create makes
+ * that device current, checks for sm_100, allocates the 4-byte device status
+ * word and resolves the driver's tensor-map encoder.  These two calls are the
+ * only ones that allocate or free device memory. */
+fact_status_t fact_create(fact_handle_t* handle, int device);
+fact_status_t fact_destroy(fact_handle_t handle);
+
+/* Static, never NULL. */
+const char* fact_status_string(fact_status_t status);
+
+/* Scratch bytes the given problem needs with `cfg` (NULL = the library's own
+ * choice, the same one the compute call will make with cfg == NULL).  0 when
+ * no K split is used.  N is the number of OUTPUT columns; `epilogue` matters
+ * because SILU_GATE partials are twice as wide. */
+fact_status_t fact_workspace_bytes(fact_handle_t handle, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                                   fact_epilogue_t epilogue, fact_blayout_t b_layout, fact_out_t out_type,
+                                   const fact_config_t* cfg, size_t* bytes);
+
+/* C[M x N] = A[M x K] . B          (Section 5.1, Problem 1: data-parallel tiles)
+ * A: BF16 [M x K], lda.  B: BF16, [K x N] (FACT_B_KN, ldb >= N) or [N x K]
+ * (FACT_B_NK, ldb >= K).  C: BF16 or FP32 [M x N], ldc.  The library may
+ * still split K when cfg (or its own choice) says so; then `workspace` must
+ * hold fact_workspace_bytes(...) bytes, else it may be NULL/0. */
+fact_status_t fact_gemm(fact_handle_t handle, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                        const void* B, int64_t ldb, fact_blayout_t b_layout, void* C, int64_t ldc,
+                        fact_out_t out_type, const fact_config_t* cfg, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/* C[b] = A[b] . B[b] for b in [0, batch)      (Section 5.1, Problem 3: batched)
+ * Batch b of an operand starts stride* elements after batch b-1. */
+fact_status_t fact_gemm_batched(fact_handle_t handle, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
+                                int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                                fact_blayout_t b_layout, void* C, int64_t ldc, int64_t strideC, fact_out_t out_type,
+                                const fact_config_t* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* C = A . B with K cut into `splits` contiguous slices (0 = library's choice)
+ *                                              (Section 5.1, Problem 6: long K)
+ * Each (tile, slice) writes an FP32 partial to the workspace; a second kernel
+ * adds the partials of every element in ascending slice order and stores C.
+ * Slice boundaries and the order of additions depend only on (M, N, K, config),
+ * so repeated calls return bit-identical results. */
+fact_status_t fact_gemm_splitk(fact_handle_t handle, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                               const void* B, int64_t ldb, fact_blayout_t b_layout, void* C, int64_t ldc,
+                               fact_out_t out_type, int splits, const fact_config_t* cfg, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream);
+
+/* Y[M x N_out] = epilogue(X[M x K] . W)        (Section 5.2: fused linear layers)
+ * W: FACT_B_NK [Nw x K] (nn.Linear weight) or FACT_B_KN [K x Nw]; Nw = N_out,
+ * or 2*N_out for SILU_GATE.  bias: BF16 [N_out]; required by BIAS, BIAS_RELU,
+ * BIAS_GELU_TANH, optional for BIAS_RESIDUAL, must be NULL otherwise.
+ * residual: BF16 [M x N_out] with ldr; required by BIAS_RESIDUAL, must be NULL
+ * otherwise.  Y may alias residual only if pointer and leading dimension are
+ * identical. */
+fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                          const void* W, int64_t ldw, fact_blayout_t w_layout, const void* bias,
+                          const void* residual, int64_t ldr, void* Y, int64_t ldy, fact_out_t out_type,
+                          fact_epilogue_t epilogue, const fact_config_t* cfg, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream);
+
+/* The configuration the library would run for this problem when cfg == NULL
+ * (its tuned entry if fact_tune / fact_tune_cache_load provided one, else a
+ * heuristic).  The paper's counterpart is the lookup in its pattern table
+ * (Section 3; Section 4.2, Action 6). */
+fact_status_t fact_get_config(fact_handle_t handle, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                              fact_epilogue_t epilogue, fact_blayout_t b_layout, fact_out_t out_type,
+                              fact_config_t* cfg_out);
+
+/* On-device tile-configuration search for one problem (Section 4.2, Action 5
+ * "auto-tuning": sweep tile shapes, pipeline depth, cluster size and grid
+ * schedule, time every feasible candidate, keep the best).  Runs on the given
+ * device buffers (outputs are overwritten), times each feasible candidate with
+ * CUDA events (`warmup` + `iters` launches; 0 = 5 and 20, the paper's
+ * protocol in Section 5.1), synchronises the stream, stores the winner in the
+ * handle's table and returns it.  Candidates over the shared-memory or TMEM
+ * budget are skipped on the host and never launched.  `workspace` must be
+ * large enough for every split-K candidate the search is allowed to try:
+ * candidates that need more are skipped. */
+fact_status_t fact_tune(fact_handle_t handle, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                        const void* A, int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                        fact_blayout_t b_layout, const void* bias, const void* residual, int64_t ldr,
+                        int64_t strideR, void* C, int64_t ldc, int64_t strideC, fact_out_t out_type,
+                        fact_epilogue_t epilogue, void* workspace, size_t workspace_bytes, int warmup, int iters,
+                        void* cuda_stream, fact_config_t* best, double* best_ms, int* n_tried);
+
+/* Persist / restore the tuner's table as a text file (one line per problem
+ * key; host path).  Loading merges into the handle's table. */
+fact_status_t fact_tune_cache_save(fact_handle_t handle, const char* path);
+fact_status_t fact_tune_cache_load(fact_handle_t handle, const char* path);
+
+/* Synchronise `cuda_stream`, read the device status word into *status
+ * (FACT_OK or FACT_ERR_DEVICE_TIMEOUT) and clear it.  Every device-side wait
+ * in the kernels is bounded; a wait that expires records the timeout, the
+ * kernel releases its tensor memory and returns, and the output of that call
+ * is undefined. */
+fact_status_t fact_device_status(fact_handle_t handle, void* cuda_stream, int* status);
+
+/* Number of kernels this handle has launched so far (for benchmark reports). */
+int64_t fact_launch_count(fact_handle_t handle);
+
+/* Text of the most recent CUDA runtime/driver failure seen through this handle
+ * (the call that returned FACT_ERR_CUDA), "" if none.  Owned by the handle;
+ * valid until the next failing call or fact_destroy. */
+const char* fact_last_error(fact_handle_t handle);
+
+/* Device properties the handle saw (any pointer may be NULL). */
+fact_status_t fact_device_info(fact_handle_t handle, int* sm_count, int* max_smem_per_block, int* cc_major,
+                               int* cc_minor);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FACT_H_ */

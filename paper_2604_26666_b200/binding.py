@@ -1,0 +1,322 @@
+"""ctypes binding of libfact: argument marshalling only.
+
+Every step of the computation runs in the CUDA library; PyTorch is used for
+device memory (tensors, the split-K workspace) and for the current stream.
+There is no fallback: if ``libfact.so`` has not been built, or the device is
+not sm_100, the calls raise.
+
+The raw C entry points are available under their C names on ``lib()``
+(``lib().fact_gemm`` ...); ``Handle`` wraps them for torch tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int64, c_size_t, c_void_p
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libfact.so"
+
+OK = 0
+STATUS_NAMES = {
+    0: "FACT_OK", 1: "FACT_ERR_INVALID_ARG", 2: "FACT_ERR_BAD_ALIGNMENT", 3: "FACT_ERR_UNSUPPORTED",
+    4: "FACT_ERR_ARCH", 5: "FACT_ERR_WORKSPACE_TOO_SMALL", 6: "FACT_ERR_CUDA", 7: "FACT_ERR_DEVICE_TIMEOUT",
+}
+EPILOGUES = {"NONE": 0, "BIAS": 1, "BIAS_RELU": 2, "BIAS_GELU_TANH": 3, "SILU_GATE": 4, "BIAS_RESIDUAL": 5}
+LAYOUTS = {"KN": 0, "NK": 1}
+OUT_TYPES = {torch.bfloat16: 0, torch.float32: 1, "bf16": 0, "f32": 1}
+OPS = {"gemm": 0, "gemm_batched": 1, "gemm_splitk": 2, "linear": 3}
+
+# every symbol include/fact.h declares
+EXPORTED = [
+    "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
+    "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
+    "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
+]
+
+
+class FactError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)}")
+
+
+class Config(Structure):
+    """Mirror of fact_config_t; zero fields mean "library's choice"."""
+
+    _fields_ = [(n, c_int) for n in
+                ("tile_m", "tile_n", "tile_k", "stages", "cta_group", "raster_group", "split_k", "store_mode")]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+    def __repr__(self):
+        return "Config(" + ", ".join(f"{k}={v}" for k, v in self.as_dict().items()) + ")"
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libfact.so (built in-tree by ``python -m paper_2604_26666_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_26666_b200.build` "
+                           "(there is no fallback path)")
+    L = ctypes.CDLL(str(LIB_PATH))
+    i64, vp, sz = c_int64, c_void_p, c_size_t
+    cfgp = POINTER(Config)
+    L.fact_create.argtypes = [POINTER(vp), c_int]
+    L.fact_destroy.argtypes = [vp]
+    L.fact_status_string.argtypes = [c_int]
+    L.fact_status_string.restype = c_char_p
+    L.fact_workspace_bytes.argtypes = [vp, c_int, i64, i64, i64, i64, c_int, c_int, c_int, cfgp, POINTER(sz)]
+    L.fact_gemm.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, cfgp, vp, sz, vp]
+    L.fact_gemm_batched.argtypes = [vp, i64, i64, i64, i64, vp, i64, i64, vp, i64, i64, c_int, vp, i64, i64, c_int,
+                                    cfgp, vp, sz, vp]
+    L.fact_gemm_splitk.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, c_int, cfgp, vp, sz, vp]
+    L.fact_linear.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, vp, i64, vp, i64, c_int, c_int, cfgp,
+                              vp, sz, vp]
+    L.fact_get_config.argtypes = [vp, c_int, i64, i64, i64, i64, c_int, c_int, c_int, cfgp]
+    L.fact_tune.argtypes = [vp, c_int, i64, i64, i64, i64, vp, i64, i64, vp, i64, i64, c_int, vp, vp, i64, i64, vp,
+                            i64, i64, c_int, c_int, vp, sz, c_int, c_int, vp, cfgp, POINTER(c_double), POINTER(c_int)]
+    L.fact_tune_cache_save.argtypes = [vp, c_char_p]
+    L.fact_tune_cache_load.argtypes = [vp, c_char_p]
+    L.fact_device_status.argtypes = [vp, vp, POINTER(c_int)]
+    L.fact_launch_count.argtypes = [vp]
+    L.fact_launch_count.restype = i64
+    L.fact_device_info.argtypes = [vp, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
+    L.fact_last_error.argtypes = [vp]
+    L.fact_last_error.restype = c_char_p
+    for name in EXPORTED:
+        fn = getattr(L, name)
+        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error"):
+            fn.restype = c_int
+    _lib = L
+    return L
+
+
+def _check(code: int, where: str, handle=None):
+    if code != OK:
+        if code == 6 and handle is not None:
+            where += " [" + (lib().fact_last_error(handle) or b"").decode() + "]"
+        raise FactError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _need(t: torch.Tensor, name: str, dtype, ndim):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if t.ndim != ndim:
+        raise ValueError(f"{name} must have {ndim} dimensions")
+    if t.shape[-1] > 1 and t.stride(-1) != 1:
+        raise ValueError(f"{name}: innermost dimension must be contiguous")
+
+
+def _ld(t: torch.Tensor) -> int:
+    """Leading dimension of the last two dims; a one-row matrix may carry any stride."""
+    return int(t.stride(-2)) if t.shape[-2] > 1 else max(int(t.shape[-1]), int(t.stride(-2)))
+
+
+class Handle:
+    """A libfact handle on one CUDA device, plus a grow-only torch workspace."""
+
+    def __init__(self, device: int = 0):
+        self._h = c_void_p()
+        self.device = int(device)
+        _check(lib().fact_create(byref(self._h), self.device), "fact_create")
+        self._ws: Optional[torch.Tensor] = None
+
+    def close(self):
+        if self._h:
+            lib().fact_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers ------------------------------------------------------------------------------
+    def _stream(self, stream) -> c_void_p:
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        return c_void_p(s.cuda_stream)
+
+    def _cfg(self, cfg):
+        if cfg is None:
+            return None
+        if isinstance(cfg, Config):
+            return byref(cfg)
+        c = Config(**{k: int(v) for k, v in dict(cfg).items()})
+        return byref(c)
+
+    def workspace(self, nbytes: int) -> Optional[torch.Tensor]:
+        if nbytes <= 0:
+            return None
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty(nbytes, dtype=torch.uint8, device=f"cuda:{self.device}")
+        return self._ws
+
+    def workspace_bytes(self, op, batch, M, N, K, epilogue="NONE", layout="KN", out_dtype=torch.bfloat16, cfg=None,
+                        splits=0) -> int:
+        n = c_size_t(0)
+        c = self._cfg_with_splits(cfg, splits)
+        _check(lib().fact_workspace_bytes(self._h, OPS[op], batch, M, N, K, EPILOGUES[epilogue], LAYOUTS[layout],
+                                          OUT_TYPES[out_dtype], c, byref(n)), "fact_workspace_bytes")
+        return int(n.value)
+
+    def _cfg_with_splits(self, cfg, splits):
+        if not splits:
+            return self._cfg(cfg)
+        d = cfg.as_dict() if isinstance(cfg, Config) else dict(cfg or {})
+        d["split_k"] = int(splits)
+        return self._cfg(d)
+
+    def get_config(self, op, batch, M, N, K, epilogue="NONE", layout="KN", out_dtype=torch.bfloat16) -> Config:
+        c = Config()
+        _check(lib().fact_get_config(self._h, OPS[op], batch, M, N, K, EPILOGUES[epilogue], LAYOUTS[layout],
+                                     OUT_TYPES[out_dtype], byref(c)), "fact_get_config")
+        return c
+
+    def device_status(self, stream=None) -> int:
+        v = c_int(0)
+        _check(lib().fact_device_status(self._h, self._stream(stream), byref(v)), "fact_device_status")
+        return int(v.value)
+
+    def launch_count(self) -> int:
+        return int(lib().fact_launch_count(self._h))
+
+    def device_info(self) -> dict:
+        a, b, c, d = c_int(), c_int(), c_int(), c_int()
+        _check(lib().fact_device_info(self._h, byref(a), byref(b), byref(c), byref(d)), "fact_device_info")
+        return {"sm_count": a.value, "max_smem_per_block": b.value, "cc": (c.value, d.value)}
+
+    def tune_cache_save(self, path: str):
+        _check(lib().fact_tune_cache_save(self._h, str(path).encode()), "fact_tune_cache_save")
+
+    def tune_cache_load(self, path: str):
+        _check(lib().fact_tune_cache_load(self._h, str(path).encode()), "fact_tune_cache_load")
+
+    # -- compute ------------------------------------------------------------------------------
+    def gemm(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
+        """C = A @ B  (fact_gemm).  layout "KN": B is [K, N]; "NK": B is [N, K]."""
+        _need(A, "A", torch.bfloat16, 2)
+        _need(B, "B", torch.bfloat16, 2)
+        M, K = A.shape
+        N = B.shape[1] if layout == "KN" else B.shape[0]
+        if (B.shape[0] if layout == "KN" else B.shape[1]) != K:
+            raise ValueError("inner dimensions differ")
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+        _need(out, "out", out.dtype, 2)
+        c = self._cfg(cfg)
+        nws = self.workspace_bytes("gemm", 1, M, N, K, "NONE", layout, out.dtype, cfg)
+        ws = self.workspace(nws)
+        _check(lib().fact_gemm(self._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
+                               _ld(out), OUT_TYPES[out.dtype], c, _ptr(ws), nws, self._stream(stream)), "fact_gemm", self._h)
+        return out
+
+    def gemm_batched(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
+        """C[b] = A[b] @ B[b]  (fact_gemm_batched)."""
+        _need(A, "A", torch.bfloat16, 3)
+        _need(B, "B", torch.bfloat16, 3)
+        batch, M, K = A.shape
+        N = B.shape[2] if layout == "KN" else B.shape[1]
+        if B.shape[0] != batch or (B.shape[1] if layout == "KN" else B.shape[2]) != K:
+            raise ValueError("shapes differ")
+        if out is None:
+            out = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
+        _need(out, "out", out.dtype, 3)
+        nws = self.workspace_bytes("gemm_batched", batch, M, N, K, "NONE", layout, out.dtype, cfg)
+        ws = self.workspace(nws)
+        _check(lib().fact_gemm_batched(self._h, batch, M, N, K, _ptr(A), _ld(A), A.stride(0), _ptr(B), _ld(B),
+                                       B.stride(0), LAYOUTS[layout], _ptr(out), _ld(out), out.stride(0),
+                                       OUT_TYPES[out.dtype], self._cfg(cfg), _ptr(ws), nws, self._stream(stream)),
+               "fact_gemm_batched", self._h)
+        return out
+
+    def gemm_splitk(self, A, B, layout="KN", out=None, out_dtype=torch.float32, splits=0, cfg=None, stream=None):
+        """C = A @ B with K cut into slices and a fixed-order reduction  (fact_gemm_splitk)."""
+        _need(A, "A", torch.bfloat16, 2)
+        _need(B, "B", torch.bfloat16, 2)
+        M, K = A.shape
+        N = B.shape[1] if layout == "KN" else B.shape[0]
+        if (B.shape[0] if layout == "KN" else B.shape[1]) != K:
+            raise ValueError("inner dimensions differ")
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+        _need(out, "out", out.dtype, 2)
+        nws = self.workspace_bytes("gemm_splitk", 1, M, N, K, "NONE", layout, out.dtype, cfg, splits)
+        ws = self.workspace(nws)
+        _check(lib().fact_gemm_splitk(self._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
+                                      _ld(out), OUT_TYPES[out.dtype], int(splits), self._cfg(cfg), _ptr(ws), nws,
+                                      self._stream(stream)), "fact_gemm_splitk", self._h)
+        return out
+
+    def linear(self, X, W, bias=None, residual=None, epilogue="NONE", layout="NK", out=None,
+               out_dtype=torch.bfloat16, cfg=None, stream=None):
+        """Y = epilogue(X @ W)  (fact_linear).  layout "NK": W is [Nw, K] (nn.Linear weight); "KN": [K, Nw].
+        For SILU_GATE W carries 2*N_out columns (gate first, then up)."""
+        _need(X, "X", torch.bfloat16, 2)
+        _need(W, "W", torch.bfloat16, 2)
+        M, K = X.shape
+        Nw = W.shape[1] if layout == "KN" else W.shape[0]
+        if (W.shape[0] if layout == "KN" else W.shape[1]) != K:
+            raise ValueError("inner dimensions differ")
+        if epilogue == "SILU_GATE":
+            if Nw % 2:
+                raise ValueError("SILU_GATE needs an even number of weight columns")
+            N = Nw // 2
+        else:
+            N = Nw
+        if bias is not None:
+            _need(bias, "bias", torch.bfloat16, 1)
+            if bias.shape[0] != N:
+                raise ValueError("bias must have N_out entries")
+        if residual is not None:
+            _need(residual, "residual", torch.bfloat16, 2)
+            if tuple(residual.shape) != (M, N):
+                raise ValueError("residual must be [M, N_out]")
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype, device=X.device)
+        _need(out, "out", out.dtype, 2)
+        nws = self.workspace_bytes("linear", 1, M, N, K, epilogue, layout, out.dtype, cfg)
+        ws = self.workspace(nws)
+        _check(lib().fact_linear(self._h, M, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W), LAYOUTS[layout], _ptr(bias),
+                                 _ptr(residual), _ld(residual) if residual is not None else 0, _ptr(out), _ld(out),
+                                 OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg), _ptr(ws), nws,
+                                 self._stream(stream)), "fact_linear", self._h)
+        return out
+
+    def tune(self, op, A, B, layout="KN", bias=None, residual=None, epilogue="NONE", out=None,
+             out_dtype=torch.bfloat16, workspace_bytes=256 << 20, warmup=0, iters=0, stream=None):
+        """Search tile configurations for this problem on the device (fact_tune).
+        Returns (Config, best_ms, n_tried)."""
+        batched = A.ndim == 3
+        batch = A.shape[0] if batched else 1
+        M, K = A.shape[-2:]
+        Nw = B.shape[-1] if layout == "KN" else B.shape[-2]
+        N = Nw // 2 if epilogue == "SILU_GATE" else Nw
+        if out is None:
+            out = torch.empty(((batch, M, N) if batched else (M, N)), dtype=out_dtype, device=A.device)
+        ws = self.workspace(workspace_bytes)
+        best, ms, n = Config(), c_double(0.0), c_int(0)
+        _check(lib().fact_tune(self._h, OPS[op], batch, M, N, K, _ptr(A), _ld(A), A.stride(0) if batched else 0,
+                               _ptr(B), _ld(B), B.stride(0) if batched else 0, LAYOUTS[layout], _ptr(bias),
+                               _ptr(residual), _ld(residual) if residual is not None else 0,
+                               residual.stride(0) if (residual is not None and batched) else 0, _ptr(out), _ld(out),
+                               out.stride(0) if batched else 0, OUT_TYPES[out.dtype], EPILOGUES[epilogue], _ptr(ws),
+                               ws.numel() if ws is not None else 0, warmup, iters, self._stream(stream), byref(best),
+                               byref(ms), byref(n)), "fact_tune", self._h)
+        return best, float(ms.value), int(n.value)

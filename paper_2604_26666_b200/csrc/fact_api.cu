@@ -1,0 +1,732 @@
+// Host side of libfact: argument validation, configuration choice, tensor-map
+// encoding, kernel launch, the tile-configuration tuner and its table.
+// Declarations and per-call contracts are in include/fact.h.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "fact.h"
+#include "gemm_kernel.cuh"
+
+namespace {
+
+using namespace fact;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kSmemBudget = 226 * 1024;  // opt-in shared memory per CTA on sm_100 (227 KB) minus 1 KB for static data
+constexpr int kSmemSlack = 1024;         // room to align the stage ring to 1024 bytes
+constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
+
+// Key of the tuner's table: everything that changes which configuration is best.
+typedef std::tuple<int, int, int, int, long long, long long, long long, long long> TuneKey;
+
+struct Problem {
+  fact_op_t op;
+  long long batch, M, N_out, K;
+  const void* A;
+  long long lda, strideA;
+  const void* B;
+  long long ldb, strideB;
+  fact_blayout_t layout;
+  const void* bias;
+  const void* R;
+  long long ldr, strideR;
+  void* C;
+  long long ldc, strideC;
+  fact_out_t out;
+  fact_epilogue_t epi;
+  long long Nw() const { return epi == FACT_EPI_SILU_GATE ? 2 * N_out : N_out; }
+};
+
+struct Plan {
+  fact_config_t cfg;
+  int smem_bytes;
+  int grid;
+  size_t ws_bytes;
+  GemmParams p;
+};
+
+}  // namespace
+
+struct fact_handle_s {
+  int device = 0;
+  int sm_count = 0;
+  int max_smem = 0;
+  int cc_major = 0, cc_minor = 0;
+  int* d_status = nullptr;
+  EncodeTiledFn encode = nullptr;
+  long long launches = 0;
+  std::map<TuneKey, fact_config_t> table;
+  unsigned configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
+  std::string last_error;        // text of the most recent CUDA failure
+};
+
+namespace {
+
+TuneKey make_key(const Problem& q) {
+  return TuneKey((int)q.op, (int)q.epi, (int)q.layout, (int)q.out, q.batch, q.M, q.N_out, q.K);
+}
+
+fact_status_t cuda_fail(fact_handle_t h, const char* where, cudaError_t e) {
+  h->last_error = std::string(where) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
+  cudaGetLastError();
+  return FACT_ERR_CUDA;
+}
+
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
+uint32_t pow2_at_least(uint32_t x) {
+  uint32_t r = 32;
+  while (r < x) r <<= 1;
+  return r;
+}
+
+// Per-CTA bytes of one pipeline stage.
+int stage_bytes_for(int tile_n, int cta_group) { return (int)kStageBytesA + (tile_n / cta_group) * kTileK * 2; }
+
+int max_stages_for(int tile_n, int cta_group) {
+  int s = (kSmemBudget - kSmemSlack) / stage_bytes_for(tile_n, cta_group);
+  return std::min(s, kMaxStages);
+}
+
+// Is (tile_n, cta_group) runnable for this problem's layout / epilogue?
+bool tile_ok(const Problem& q, int tile_n, int cg) {
+  if (cg != 1 && cg != 2) return false;
+  if (tile_n < 32 || tile_n > 256 || tile_n % 32) return false;
+  const bool gate = q.epi == FACT_EPI_SILU_GATE;
+  const int per_cta = tile_n / cg;
+  if (cg == 2 && tile_n % 64) return false;
+  if (gate && tile_n % 64) return false;
+  if (q.layout == FACT_B_KN) {
+    if (per_cta % 64) return false;
+    if (gate && (tile_n / 2) % 64) return false;
+  }
+  return true;
+}
+
+// Fill every zero field of `cfg`.  Returns FACT_ERR_UNSUPPORTED for a combination the kernels cannot run.
+fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_config_t* user, int splits_override,
+                             fact_config_t* out) {
+  fact_config_t c;
+  memset(&c, 0, sizeof c);
+  if (user) c = *user;
+  else {
+    auto it = h->table.find(make_key(q));
+    if (it != h->table.end()) c = it->second;
+  }
+  if (splits_override > 0) c.split_k = splits_override;
+  if (c.tile_k != 0 && c.tile_k != kTileK) return FACT_ERR_UNSUPPORTED;
+  c.tile_k = kTileK;
+  if (c.cta_group == 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
+  if (c.tile_m == 0) c.tile_m = 128 * c.cta_group;
+  if (c.tile_m != 128 * c.cta_group) return FACT_ERR_UNSUPPORTED;
+  const long long Nw = q.Nw();
+  if (c.tile_n == 0) {
+    // widest tile that does not overshoot the problem, in the granularity the layout allows
+    const int gran = (q.layout == FACT_B_KN ? 64 : 32) * c.cta_group * (q.epi == FACT_EPI_SILU_GATE ? 2 : 1);
+    const long long cover = q.epi == FACT_EPI_SILU_GATE ? 2 * std::min<long long>(q.N_out, 128) : std::min<long long>(Nw, 256);
+    c.tile_n = std::max(gran, std::min(256, round_up((int)cover, gran)));
+    while (c.tile_n > gran && !tile_ok(q, c.tile_n, c.cta_group)) c.tile_n -= gran;
+  }
+  if (!tile_ok(q, c.tile_n, c.cta_group)) return FACT_ERR_UNSUPPORTED;
+  const int smax = max_stages_for(c.tile_n, c.cta_group);
+  if (c.stages == 0) c.stages = smax;
+  if (c.stages < 2 || c.stages > smax) return FACT_ERR_UNSUPPORTED;
+  if (c.raster_group == 0) c.raster_group = 8;
+  if (c.raster_group < 1) return FACT_ERR_INVALID_ARG;
+  const int k_blocks = (int)((q.K + kTileK - 1) / kTileK);
+  if (c.split_k == 0) {
+    c.split_k = 1;
+    if (q.op == FACT_OP_GEMM_SPLITK) {
+      const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
+      const long long tiles = q.batch * ((q.M + c.tile_m - 1) / c.tile_m) * ((q.N_out + out_cols - 1) / out_cols);
+      const long long slots = h->sm_count / c.cta_group;
+      long long s = tiles > 0 ? slots / tiles : 1;
+      s = std::min<long long>(s, k_blocks / 4);  // at least four k-blocks per slice
+      c.split_k = (int)std::max<long long>(1, s);
+    }
+  }
+  if (c.split_k < 1) return FACT_ERR_INVALID_ARG;
+  c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
+  if (c.store_mode == 0) c.store_mode = 1;
+  if (c.store_mode != 1) return FACT_ERR_UNSUPPORTED;
+  *out = c;
+  return FACT_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+fact_status_t validate(const Problem& q) {
+  if (q.batch < 0 || q.M < 0 || q.N_out < 0 || q.K < 0) return FACT_ERR_INVALID_ARG;
+  if (q.epi < FACT_EPI_NONE || q.epi > FACT_EPI_BIAS_RESIDUAL) return FACT_ERR_INVALID_ARG;
+  if (q.layout != FACT_B_KN && q.layout != FACT_B_NK) return FACT_ERR_INVALID_ARG;
+  if (q.out != FACT_OUT_BF16 && q.out != FACT_OUT_F32) return FACT_ERR_INVALID_ARG;
+  if (q.batch == 0 || q.M == 0 || q.N_out == 0) return FACT_OK;
+  if (q.M > 0x7fffffffLL - 512 || q.Nw() > 0x7fffffffLL - 512 || q.K > 0x7fffffffLL - 512 || q.batch > 65535 * 16)
+    return FACT_ERR_INVALID_ARG;
+  if (!q.C) return FACT_ERR_INVALID_ARG;
+  const bool needs_bias = q.epi == FACT_EPI_BIAS || q.epi == FACT_EPI_BIAS_RELU || q.epi == FACT_EPI_BIAS_GELU_TANH;
+  if (needs_bias && !q.bias) return FACT_ERR_INVALID_ARG;
+  if ((q.epi == FACT_EPI_NONE || q.epi == FACT_EPI_SILU_GATE) && q.bias) return FACT_ERR_INVALID_ARG;
+  if (q.epi == FACT_EPI_BIAS_RESIDUAL) {
+    if (!q.R || q.ldr < q.N_out) return FACT_ERR_INVALID_ARG;
+    if (q.R == q.C && q.ldr != q.ldc) return FACT_ERR_INVALID_ARG;
+    if (q.R == q.C && q.out != FACT_OUT_BF16) return FACT_ERR_INVALID_ARG;
+  } else if (q.R) {
+    return FACT_ERR_INVALID_ARG;
+  }
+  if (q.ldc < q.N_out) return FACT_ERR_INVALID_ARG;
+  if (q.K > 0) {
+    if (!q.A || !q.B) return FACT_ERR_INVALID_ARG;
+    if (q.lda < q.K) return FACT_ERR_INVALID_ARG;
+    if (q.ldb < (q.layout == FACT_B_KN ? q.Nw() : q.K)) return FACT_ERR_INVALID_ARG;
+    if (!aligned16(q.A) || !aligned16(q.B)) return FACT_ERR_BAD_ALIGNMENT;
+    if (q.lda % 8 || q.ldb % 8) return FACT_ERR_BAD_ALIGNMENT;
+    if (q.batch > 1) {
+      if (q.strideA % 8 || q.strideB % 8) return FACT_ERR_BAD_ALIGNMENT;
+      if (q.strideA < 0 || q.strideB < 0 || q.strideC < 0) return FACT_ERR_INVALID_ARG;
+    }
+  }
+  return FACT_OK;
+}
+
+size_t workspace_for(const Problem& q, const fact_config_t& c) {
+  if (c.split_k <= 1) return 0;
+  const long long ws_ld = round_up((int)q.Nw(), 4);
+  return (size_t)c.split_k * (size_t)q.batch * (size_t)q.M * (size_t)ws_ld * sizeof(float);
+}
+
+uint64_t smem_desc_template(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // 64-bit shared-memory matrix descriptor without the start address:
+  // [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4, [46,48) version 1 (sm_100),
+  // [61,64) layout type 2 = 128-byte swizzle
+  return ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) | ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* user, int splits_override,
+                        Plan* plan) {
+  fact_status_t st = resolve_config(h, q, user, splits_override, &plan->cfg);
+  if (st != FACT_OK) return st;
+  const fact_config_t& c = plan->cfg;
+  GemmParams& p = plan->p;
+  memset(&p, 0, sizeof p);
+  const int cg = c.cta_group;
+  const bool gate = q.epi == FACT_EPI_SILU_GATE;
+  p.M = (int)q.M;
+  p.N_out = (int)q.N_out;
+  p.Nw = (int)q.Nw();
+  p.K = (int)q.K;
+  p.batch = (int)q.batch;
+  p.tile_n = c.tile_n;
+  p.out_cols = gate ? c.tile_n / 2 : c.tile_n;
+  p.tiles_m = (int)((q.M + c.tile_m - 1) / c.tile_m);
+  p.tiles_n = (int)((q.N_out + p.out_cols - 1) / p.out_cols);
+  p.k_blocks = (int)((q.K + kTileK - 1) / kTileK);
+  p.split_k = c.split_k;
+  p.raster_group = std::min(c.raster_group, std::max(1, p.tiles_m));
+  p.stages = c.stages;
+  const long long units = (long long)p.batch * p.tiles_m * p.tiles_n * p.split_k;
+  if (units > 0x7fffffffLL) return FACT_ERR_UNSUPPORTED;
+  p.total_units = (int)units;
+  const int per_cta = c.tile_n / cg;
+  p.b_kn = q.layout == FACT_B_KN;
+  p.gate = gate;
+  if (p.b_kn) {
+    p.b_box_n = 64;
+    p.b_loads = per_cta / 64;
+  } else if (gate && cg == 1) {
+    p.b_box_n = c.tile_n / 2;
+    p.b_loads = 2;
+  } else {
+    p.b_box_n = per_cta;
+    p.b_loads = 1;
+  }
+  p.b_box_bytes = (uint32_t)p.b_box_n * kTileK * 2;
+  p.stage_bytes = (uint32_t)stage_bytes_for(c.tile_n, cg);
+  p.tx_bytes = p.stage_bytes * (uint32_t)cg;
+  // A and W[N x K]: K-major, rows of 128 bytes, 8-row swizzle atoms 1024 bytes apart; 16 K-elements = 32 bytes.
+  p.a_desc = smem_desc_template(16, 1024);
+  p.a_k_step = 32 >> 4;
+  if (p.b_kn) {
+    // B[K x N]: N-major.  One TMA box = 64 k-rows of 64 n (128 bytes): 8-k groups are 1024 bytes apart
+    // (stride offset), successive 64-n chunks one box (8192 bytes) apart (leading offset); 16 k = 2048 bytes.
+    p.b_desc = smem_desc_template(kTileK * 128, 1024);
+    p.b_k_step = (kUmmaK * 128) >> 4;
+  } else {
+    p.b_desc = p.a_desc;
+    p.b_k_step = p.a_k_step;
+  }
+  // instruction descriptor: D = F32 (1 @ bit 4), A = B = BF16 (1 @ bits 7, 10), A K-major, B major-ness @ bit 16,
+  // N >> 3 @ bit 17, M >> 4 @ bit 24
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_kn << 16) | ((uint32_t)(c.tile_n >> 3) << 17) |
+            ((uint32_t)((kTileM * cg) >> 4) << 24);
+  p.tmem_cols = pow2_at_least((uint32_t)(2 * c.tile_n));
+  p.C = q.C;
+  p.ldc = q.ldc;
+  p.strideC = q.strideC;
+  p.out_f32 = q.out == FACT_OUT_F32;
+  const int c_elems16 = p.out_f32 ? 4 : 8;
+  p.c_vec = aligned16(q.C) && (q.ldc % c_elems16 == 0) && (q.batch <= 1 || q.strideC % c_elems16 == 0);
+  p.bias = reinterpret_cast<const __nv_bfloat16*>(q.bias);
+  p.bias_vec = q.bias && aligned16(q.bias);
+  p.R = reinterpret_cast<const __nv_bfloat16*>(q.R);
+  p.ldr = q.ldr;
+  p.strideR = q.strideR;
+  p.r_vec = q.R && aligned16(q.R) && (q.ldr % 8 == 0) && (q.batch <= 1 || q.strideR % 8 == 0);
+  p.ws_ld = round_up(p.Nw, 4);
+  p.ws_batch_stride = (long long)p.M * p.ws_ld;
+  p.ws_split_stride = p.ws_batch_stride * p.batch;
+  p.status = h->d_status;
+  plan->ws_bytes = workspace_for(q, c);
+  plan->smem_bytes = std::max(c.stages * (int)p.stage_bytes + kSmemSlack, kMinSmemRequest);
+  if (plan->smem_bytes > kSmemBudget || kSmemBudget + 1024 > h->max_smem) return FACT_ERR_UNSUPPORTED;
+  const int slots = std::max(1, h->sm_count / cg);
+  plan->grid = (int)std::min<long long>(slots, units) * cg;
+  return FACT_OK;
+}
+
+fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                         uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1) {
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
+  cuuint32_t box[3] = {box0, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    h->last_error = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
+    return FACT_ERR_CUDA;
+  }
+  return FACT_OK;
+}
+
+template <int CG, int EPI>
+fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap& tmA,
+                              const CUtensorMap& tmB, cudaStream_t stream) {
+  auto kern = fact_gemm_kernel<CG, EPI>;
+  if (!(h->configured_mask & (1u << slot))) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+    h->configured_mask |= (1u << slot);
+  }
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3((unsigned)plan.grid, 1, 1);
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = (size_t)plan.smem_bytes;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (CG == 2) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+  }
+  cudaError_t e = cudaLaunchKernelEx(&lc, kern, tmA, tmB, plan.p);
+  if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx", e);
+  h->launches++;
+  return FACT_OK;
+}
+
+template <int CG>
+fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                         cudaStream_t stream) {
+  const int base = (CG - 1) * 8;
+  switch (epi) {
+    case kEpiNone: return launch_instance<CG, kEpiNone>(h, base + 0, plan, tmA, tmB, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias>(h, base + 1, plan, tmA, tmB, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu>(h, base + 2, plan, tmA, tmB, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh>(h, base + 3, plan, tmA, tmB, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate>(h, base + 4, plan, tmA, tmB, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual>(h, base + 5, plan, tmA, tmB, stream);
+    case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tmA, tmB, stream);
+    default: return FACT_ERR_INVALID_ARG;
+  }
+}
+
+fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan, int splits, const float* ws,
+                            cudaStream_t stream) {
+  ReduceParams r;
+  memset(&r, 0, sizeof r);
+  r.ws = ws;
+  r.ws_ld = plan.p.ws_ld;
+  r.ws_batch_stride = plan.p.ws_batch_stride;
+  r.ws_split_stride = plan.p.ws_split_stride;
+  r.splits = splits;
+  r.M = plan.p.M;
+  r.N_out = plan.p.N_out;
+  r.batch = plan.p.batch;
+  r.epi = (int)q.epi;
+  r.C = q.C;
+  r.ldc = q.ldc;
+  r.strideC = q.strideC;
+  r.out_f32 = q.out == FACT_OUT_F32;
+  r.bias = reinterpret_cast<const __nv_bfloat16*>(q.bias);
+  r.R = reinterpret_cast<const __nv_bfloat16*>(q.R);
+  r.ldr = q.ldr;
+  r.strideR = q.strideR;
+  const long long total = (long long)r.batch * r.M * ((r.N_out + 3) / 4);
+  const int blocks = (int)std::min<long long>((total + 255) / 256, (long long)h->sm_count * 8);
+  fact_splitk_reduce_kernel<<<std::max(1, blocks), 256, 0, stream>>>(r);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(h, "split-K reduce launch", e);
+  h->launches++;
+  return FACT_OK;
+}
+
+fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, int splits_override, void* ws,
+                  size_t ws_bytes, void* stream_v) {
+  if (!h) return FACT_ERR_INVALID_ARG;
+  fact_status_t st = validate(q);
+  if (st != FACT_OK) return st;
+  if (q.batch == 0 || q.M == 0 || q.N_out == 0) return FACT_OK;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+  Plan plan;
+  st = make_plan(h, q, user, splits_override, &plan);
+  if (st != FACT_OK) return st;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+
+  if (q.K == 0) {  // empty sum: the epilogue of a zero accumulator
+    st = launch_reduce(h, q, plan, 0, reinterpret_cast<const float*>(q.C), stream);
+  } else {
+    const bool split = plan.cfg.split_k > 1;
+    if (split) {
+      if (!ws || ws_bytes < plan.ws_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
+      if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
+      plan.p.ws = reinterpret_cast<float*>(ws);
+    }
+    CUtensorMap tmA, tmB;
+    const uint64_t batch_dim = (uint64_t)q.batch;
+    const uint64_t sA = q.batch > 1 ? (uint64_t)q.strideA : (uint64_t)q.lda * (uint64_t)q.M;
+    st = encode_map(h, &tmA, q.A, (uint64_t)q.K, (uint64_t)q.M, batch_dim, (uint64_t)q.lda, std::max<uint64_t>(sA, 8),
+                    kTileK, kTileM);
+    if (st != FACT_OK) return st;
+    if (q.layout == FACT_B_KN) {
+      const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.K;
+      st = encode_map(h, &tmB, q.B, (uint64_t)q.Nw(), (uint64_t)q.K, batch_dim, (uint64_t)q.ldb,
+                      std::max<uint64_t>(sB, 8), 64, kTileK);
+    } else {
+      const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.Nw();
+      st = encode_map(h, &tmB, q.B, (uint64_t)q.K, (uint64_t)q.Nw(), batch_dim, (uint64_t)q.ldb,
+                      std::max<uint64_t>(sB, 8), kTileK, (uint32_t)plan.p.b_box_n);
+    }
+    if (st != FACT_OK) return st;
+    const int epi = split ? (int)kEpiPartial : (int)q.epi;
+    if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tmA, tmB, stream);
+    else st = launch_epi<1>(h, epi, plan, tmA, tmB, stream);
+    if (st == FACT_OK && split) st = launch_reduce(h, q, plan, plan.cfg.split_k, plan.p.ws, stream);
+  }
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
+}
+
+Problem make_problem(fact_op_t op, long long batch, long long M, long long N, long long K, const void* A,
+                     long long lda, long long sA, const void* B, long long ldb, long long sB, fact_blayout_t layout,
+                     const void* bias, const void* R, long long ldr, long long sR, void* C, long long ldc,
+                     long long sC, fact_out_t out, fact_epilogue_t epi) {
+  Problem q;
+  q.op = op;
+  q.batch = batch;
+  q.M = M;
+  q.N_out = N;
+  q.K = K;
+  q.A = A;
+  q.lda = lda;
+  q.strideA = sA;
+  q.B = B;
+  q.ldb = ldb;
+  q.strideB = sB;
+  q.layout = layout;
+  q.bias = bias;
+  q.R = R;
+  q.ldr = ldr;
+  q.strideR = sR;
+  q.C = C;
+  q.ldc = ldc;
+  q.strideC = sC;
+  q.out = out;
+  q.epi = epi;
+  return q;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fact_status_string(fact_status_t s) {
+  switch (s) {
+    case FACT_OK: return "FACT_OK";
+    case FACT_ERR_INVALID_ARG: return "FACT_ERR_INVALID_ARG";
+    case FACT_ERR_BAD_ALIGNMENT: return "FACT_ERR_BAD_ALIGNMENT";
+    case FACT_ERR_UNSUPPORTED: return "FACT_ERR_UNSUPPORTED";
+    case FACT_ERR_ARCH: return "FACT_ERR_ARCH";
+    case FACT_ERR_WORKSPACE_TOO_SMALL: return "FACT_ERR_WORKSPACE_TOO_SMALL";
+    case FACT_ERR_CUDA: return "FACT_ERR_CUDA";
+    case FACT_ERR_DEVICE_TIMEOUT: return "FACT_ERR_DEVICE_TIMEOUT";
+    default: return "FACT_ERR_UNKNOWN";
+  }
+}
+
+fact_status_t fact_create(fact_handle_t* handle, int device) {
+  if (!handle) return FACT_ERR_INVALID_ARG;
+  *handle = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) {
+    cudaGetLastError();
+    return FACT_ERR_CUDA;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) return FACT_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FACT_ERR_CUDA;
+  if (prop.major != 10) return FACT_ERR_ARCH;
+  fact_handle_s* h = new fact_handle_s();
+  h->device = device;
+  h->sm_count = prop.multiProcessorCount;
+  h->max_smem = (int)prop.sharedMemPerBlockOptin;
+  h->cc_major = prop.major;
+  h->cc_minor = prop.minor;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete h;
+    return FACT_ERR_CUDA;
+  }
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess || cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) {
+    delete h;
+    return FACT_ERR_CUDA;
+  }
+  *handle = h;
+  return FACT_OK;
+}
+
+fact_status_t fact_destroy(fact_handle_t h) {
+  if (!h) return FACT_OK;
+  if (h->d_status) cudaFree(h->d_status);
+  delete h;
+  return FACT_OK;
+}
+
+fact_status_t fact_device_info(fact_handle_t h, int* sm_count, int* max_smem, int* cc_major, int* cc_minor) {
+  if (!h) return FACT_ERR_INVALID_ARG;
+  if (sm_count) *sm_count = h->sm_count;
+  if (max_smem) *max_smem = h->max_smem;
+  if (cc_major) *cc_major = h->cc_major;
+  if (cc_minor) *cc_minor = h->cc_minor;
+  return FACT_OK;
+}
+
+int64_t fact_launch_count(fact_handle_t h) { return h ? h->launches : 0; }
+
+const char* fact_last_error(fact_handle_t h) { return h ? h->last_error.c_str() : ""; }
+
+fact_status_t fact_device_status(fact_handle_t h, void* stream, int* status) {
+  if (!h || !status) return FACT_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return FACT_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
+  if (v != 0 && cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) return FACT_ERR_CUDA;
+  *status = v;
+  return FACT_OK;
+}
+
+static Problem shape_only(fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K, fact_epilogue_t epi,
+                          fact_blayout_t layout, fact_out_t out) {
+  return make_problem(op, batch, M, N, K, nullptr, K, 0, nullptr, 0, 0, layout, nullptr, nullptr, 0, 0, nullptr, N, 0,
+                      out, epi);
+}
+
+fact_status_t fact_get_config(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                              fact_epilogue_t epi, fact_blayout_t layout, fact_out_t out, fact_config_t* cfg_out) {
+  if (!h || !cfg_out || batch < 0 || M < 0 || N < 0 || K < 0) return FACT_ERR_INVALID_ARG;
+  Problem q = shape_only(op, batch, M, N, K, epi, layout, out);
+  return resolve_config(h, q, nullptr, 0, cfg_out);
+}
+
+fact_status_t fact_workspace_bytes(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                                   fact_epilogue_t epi, fact_blayout_t layout, fact_out_t out,
+                                   const fact_config_t* cfg, size_t* bytes) {
+  if (!h || !bytes || batch < 0 || M < 0 || N < 0 || K < 0) return FACT_ERR_INVALID_ARG;
+  Problem q = shape_only(op, batch, M, N, K, epi, layout, out);
+  fact_config_t c;
+  fact_status_t st = resolve_config(h, q, cfg, 0, &c);
+  if (st != FACT_OK) return st;
+  *bytes = workspace_for(q, c);
+  return FACT_OK;
+}
+
+fact_status_t fact_gemm(fact_handle_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const void* B,
+                        int64_t ldb, fact_blayout_t layout, void* C, int64_t ldc, fact_out_t out,
+                        const fact_config_t* cfg, void* ws, size_t ws_bytes, void* stream) {
+  Problem q = make_problem(FACT_OP_GEMM, 1, M, N, K, A, lda, 0, B, ldb, 0, layout, nullptr, nullptr, 0, 0, C, ldc, 0,
+                           out, FACT_EPI_NONE);
+  return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_gemm_batched(fact_handle_t h, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
+                                int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                                fact_blayout_t layout, void* C, int64_t ldc, int64_t strideC, fact_out_t out,
+                                const fact_config_t* cfg, void* ws, size_t ws_bytes, void* stream) {
+  Problem q = make_problem(FACT_OP_GEMM_BATCHED, batch, M, N, K, A, lda, strideA, B, ldb, strideB, layout, nullptr,
+                           nullptr, 0, 0, C, ldc, strideC, out, FACT_EPI_NONE);
+  return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_gemm_splitk(fact_handle_t h, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                               const void* B, int64_t ldb, fact_blayout_t layout, void* C, int64_t ldc,
+                               fact_out_t out, int splits, const fact_config_t* cfg, void* ws, size_t ws_bytes,
+                               void* stream) {
+  if (splits < 0) return FACT_ERR_INVALID_ARG;
+  Problem q = make_problem(FACT_OP_GEMM_SPLITK, 1, M, N, K, A, lda, 0, B, ldb, 0, layout, nullptr, nullptr, 0, 0, C,
+                           ldc, 0, out, FACT_EPI_NONE);
+  return run(h, q, cfg, splits, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_linear(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                          const void* W, int64_t ldw, fact_blayout_t layout, const void* bias, const void* residual,
+                          int64_t ldr, void* Y, int64_t ldy, fact_out_t out, fact_epilogue_t epi,
+                          const fact_config_t* cfg, void* ws, size_t ws_bytes, void* stream) {
+  Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, 0, layout, bias, residual, ldr, 0, Y,
+                           ldy, 0, out, epi);
+  return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
+                        int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                        fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, int64_t strideR,
+                        void* C, int64_t ldc, int64_t strideC, fact_out_t out, fact_epilogue_t epi, void* ws,
+                        size_t ws_bytes, int warmup, int iters, void* stream_v, fact_config_t* best, double* best_ms,
+                        int* n_tried) {
+  if (!h || !best) return FACT_ERR_INVALID_ARG;
+  Problem q = make_problem(op, batch, M, N, K, A, lda, strideA, B, ldb, strideB, layout, bias, residual, ldr, strideR,
+                           C, ldc, strideC, out, epi);
+  fact_status_t st = validate(q);
+  if (st != FACT_OK) return st;
+  if (q.batch == 0 || q.M == 0 || q.N_out == 0 || q.K == 0) return resolve_config(h, q, nullptr, 0, best);
+  if (warmup <= 0) warmup = 5;
+  if (iters <= 0) iters = 20;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return FACT_ERR_CUDA;
+
+  // Candidate axes: pair size, tile width, ring depth, raster group, K slices.
+  std::vector<fact_config_t> cands;
+  const int k_blocks = (int)((K + kTileK - 1) / kTileK);
+  for (int cg = 1; cg <= 2; ++cg) {
+    for (int tn : {64, 96, 128, 160, 192, 224, 256}) {
+      if (!tile_ok(q, tn, cg)) continue;
+      const int out_cols = epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
+      if (out_cols >= 2 * N && tn > 64) continue;  // more than half the tile would be padding
+      const int smax = max_stages_for(tn, cg);
+      const long long tiles = batch * ((M + 128 * cg - 1) / (128 * cg)) * ((N + out_cols - 1) / out_cols);
+      std::vector<int> splits = {1};
+      const long long slots = h->sm_count / cg;
+      if (op == FACT_OP_GEMM_SPLITK || tiles * 2 <= slots) {
+        for (long long s : {slots / std::max<long long>(tiles, 1), slots / std::max<long long>(tiles, 1) / 2,
+                            2 * slots / std::max<long long>(tiles, 1)}) {
+          s = std::min<long long>(s, k_blocks / 2);
+          if (s > 1 && std::find(splits.begin(), splits.end(), (int)s) == splits.end()) splits.push_back((int)s);
+        }
+      }
+      for (int stg : {smax, std::max(2, smax - 1)}) {
+        for (int rg : {4, 16}) {
+          for (int sp : splits) {
+            fact_config_t c = {128 * cg, tn, kTileK, stg, cg, rg, sp, 1};
+            cands.push_back(c);
+            if (stg == 2 && smax == 2) break;
+          }
+        }
+        if (smax <= 2) break;
+      }
+    }
+  }
+  double best_t = 1e30;
+  fact_config_t best_c;
+  memset(&best_c, 0, sizeof best_c);
+  int tried = 0;
+  for (const fact_config_t& c : cands) {
+    Plan plan;
+    if (make_plan(h, q, &c, 0, &plan) != FACT_OK) continue;  // over budget: never launched
+    if (plan.ws_bytes > ws_bytes) continue;
+    bool ok = true;
+    for (int i = 0; i < warmup && ok; ++i) ok = run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
+    if (!ok) continue;
+    cudaEventRecord(e0, stream);
+    for (int i = 0; i < iters && ok; ++i) ok = run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
+    cudaEventRecord(e1, stream);
+    int dev_status = 0;
+    if (fact_device_status(h, stream_v, &dev_status) != FACT_OK || dev_status != 0 || !ok) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) continue;
+    ++tried;
+    const double t = (double)ms / iters;
+    if (t < best_t) {
+      best_t = t;
+      best_c = plan.cfg;
+    }
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (n_tried) *n_tried = tried;
+  if (tried == 0) return FACT_ERR_UNSUPPORTED;
+  h->table[make_key(q)] = best_c;
+  *best = best_c;
+  if (best_ms) *best_ms = best_t;
+  return FACT_OK;
+}
+
+fact_status_t fact_tune_cache_save(fact_handle_t h, const char* path) {
+  if (!h || !path) return FACT_ERR_INVALID_ARG;
+  FILE* f = fopen(path, "w");
+  if (!f) return FACT_ERR_INVALID_ARG;
+  fprintf(f, "# libfact tuner table v1: op epilogue layout out batch M N K | tile_m tile_n tile_k stages cta_group raster_group split_k store_mode\n");
+  for (const auto& kv : h->table) {
+    const TuneKey& k = kv.first;
+    const fact_config_t& c = kv.second;
+    fprintf(f, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d\n", std::get<0>(k), std::get<1>(k),
+            std::get<2>(k), std::get<3>(k), std::get<4>(k), std::get<5>(k), std::get<6>(k), std::get<7>(k), c.tile_m,
+            c.tile_n, c.tile_k, c.stages, c.cta_group, c.raster_group, c.split_k, c.store_mode);
+  }
+  fclose(f);
+  return FACT_OK;
+}
+
+fact_status_t fact_tune_cache_load(fact_handle_t h, const char* path) {
+  if (!h || !path) return FACT_ERR_INVALID_ARG;
+  FILE* f = fopen(path, "r");
+  if (!f) return FACT_ERR_INVALID_ARG;
+  char line[512];
+  while (fgets(line, sizeof line, f)) {
+    if (line[0] == '#' || line[0] == '\n') continue;
+    int op, epi, lay, out;
+    long long b, M, N, K;
+    fact_config_t c;
+    if (sscanf(line, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d", &op, &epi, &lay, &out, &b, &M, &N, &K,
+               &c.tile_m, &c.tile_n, &c.tile_k, &c.stages, &c.cta_group, &c.raster_group, &c.split_k,
+               &c.store_mode) != 16)
+      continue;
+    h->table[TuneKey(op, epi, lay, out, b, M, N, K)] = c;
+  }
+  fclose(f);
+  return FACT_OK;
+}
+
+}  // extern "C"

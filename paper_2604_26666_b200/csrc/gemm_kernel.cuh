@@ -1,0 +1,533 @@
+// The persistent, warp-specialised BF16 GEMM kernel for sm_100a and the
+// split-K reduction kernel.
+//
+// One CTA (or a 2-CTA cluster when CG == 2) walks a static list of work units
+// (batch, m-tile, n-tile, k-slice).  Three roles run concurrently:
+//   warp 0     TMA producer: fills a ring of shared-memory stages with 128B-swizzled
+//              A (128 x 64) and B (tile_n x 64) tiles, signalling `full` mbarriers
+//   warp 1     MMA issuer: one thread issues tcgen05.mma (UMMA K = 16, four per stage)
+//              into one of two FP32 accumulators in tensor memory, releasing stages
+//              through tcgen05.commit -> `empty`, and publishing a finished accumulator
+//              through tcgen05.commit -> `acc_full`
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (one output row per thread), apply
+//              the fused element-wise operation in FP32, round once, store; then hand
+//              the accumulator back (`acc_empty`) so the next tile's main loop overlaps
+// Every mbarrier wait is bounded in time; an expired wait records
+// FACT_ERR_DEVICE_TIMEOUT in the status word, all roles leave their loops, tensor
+// memory is released and the kernel returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ptx.cuh"
+
+namespace fact {
+
+constexpr int kMaxStages = 8;
+constexpr int kTileM = 128;       // rows per CTA (= TMEM lanes)
+constexpr int kTileK = 64;        // BF16 elements per 128-byte swizzle row
+constexpr int kUmmaK = 16;        // K of one tcgen05.mma.kind::f16
+constexpr int kThreads = 192;     // 6 warps: producer, MMA, 4 x epilogue
+constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+// Epilogue selector of the kernel: the public enum plus the split-K partial store.
+enum : int {
+  kEpiNone = 0,
+  kEpiBias = 1,
+  kEpiBiasRelu = 2,
+  kEpiBiasGeluTanh = 3,
+  kEpiSiluGate = 4,
+  kEpiBiasResidual = 5,
+  kEpiPartial = 6  // raw FP32 accumulator to the split-K workspace
+};
+constexpr int kDeviceTimeoutCode = 7;  // FACT_ERR_DEVICE_TIMEOUT
+
+struct GemmParams {
+  // problem
+  int M, N_out, Nw, K, batch;
+  // tiling and schedule
+  int tile_n;        // accumulator columns per tile (UMMA N)
+  int out_cols;      // output columns per tile: tile_n, or tile_n / 2 for SILU_GATE
+  int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
+  int total_units;   // batch * tiles_m * tiles_n * split_k
+  // B operand loads issued by ONE CTA per stage
+  int b_loads;       // number of TMA boxes
+  int b_box_n;       // accumulator columns covered by one box
+  int b_kn;          // 1: B is [K x N] (N contiguous), 0: W is [N x K]
+  int gate;          // 1: SILU_GATE column pairing
+  uint32_t b_box_bytes;
+  uint32_t stage_bytes;  // A + B bytes of one CTA's stage
+  uint32_t tx_bytes;     // bytes the `full` barrier expects (both CTAs' stages when CG == 2)
+  // UMMA descriptors: everything but the start address; K advance in 16-byte units
+  uint64_t a_desc, b_desc;
+  uint32_t a_k_step, b_k_step;
+  uint32_t idesc;
+  uint32_t tmem_cols;
+  // epilogue operands
+  void* C;
+  long long ldc, strideC;
+  int out_f32, c_vec;
+  const __nv_bfloat16* bias;
+  int bias_vec;
+  const __nv_bfloat16* R;
+  long long ldr, strideR;
+  int r_vec;
+  // split-K partials: ws[split][batch][M][ws_ld] FP32
+  float* ws;
+  long long ws_ld, ws_batch_stride, ws_split_stride;
+  int* status;
+};
+
+struct WorkUnit {
+  int b, tm, tn, kb_begin, kb_end, split;
+};
+
+__device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
+  WorkUnit w;
+  w.split = u % p.split_k;
+  int t = u / p.split_k;
+  const int per_batch = p.tiles_m * p.tiles_n;
+  w.b = t / per_batch;
+  int r = t - w.b * per_batch;
+  // grouped raster: walk `raster_group` m-tiles, then step to the next n-tile
+  const int group_sz = p.raster_group * p.tiles_n;
+  const int g = r / group_sz;
+  const int first_m = g * p.raster_group;
+  const int gm = min(p.raster_group, p.tiles_m - first_m);
+  const int in = r - g * group_sz;
+  w.tm = first_m + in % gm;
+  w.tn = in / gm;
+  w.kb_begin = (int)(((long long)w.split * p.k_blocks) / p.split_k);
+  w.kb_end = (int)(((long long)(w.split + 1) * p.k_blocks) / p.split_k);
+  return w;
+}
+
+// Bounded mbarrier wait.  Returns false if the wait was abandoned.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = ptx::globaltimer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, kDeviceTimeoutCode);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float (&f)[8]) {
+  f[0] = __uint_as_float(q.x << 16);
+  f[1] = __uint_as_float(q.x & 0xffff0000u);
+  f[2] = __uint_as_float(q.y << 16);
+  f[3] = __uint_as_float(q.y & 0xffff0000u);
+  f[4] = __uint_as_float(q.z << 16);
+  f[5] = __uint_as_float(q.z & 0xffff0000u);
+  f[6] = __uint_as_float(q.w << 16);
+  f[7] = __uint_as_float(q.w & 0xffff0000u);
+}
+
+// 8 consecutive BF16 values starting at ptr[0]; entries >= nvalid read as 0.
+__device__ __forceinline__ void load_bf16x8(const __nv_bfloat16* ptr, int nvalid, bool vec, float (&f)[8]) {
+  if (vec && nvalid >= 8) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(ptr));
+    unpack_bf16x8(q, f);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = (j < nvalid) ? __bfloat162float(ptr[j]) : 0.f;
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void store_bf16x8(__nv_bfloat16* dst, const float (&y)[8], int nvalid, bool vec) {
+  if (vec && nvalid >= 8) {
+    uint4 q;
+    q.x = pack_bf16x2(y[0], y[1]);
+    q.y = pack_bf16x2(y[2], y[3]);
+    q.z = pack_bf16x2(y[4], y[5]);
+    q.w = pack_bf16x2(y[6], y[7]);
+    *reinterpret_cast<uint4*>(dst) = q;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < nvalid) dst[j] = __float2bfloat16_rn(y[j]);
+  }
+}
+
+__device__ __forceinline__ void store_f32x8(float* dst, const float (&y)[8], int nvalid, bool vec) {
+  if (vec && nvalid >= 8) {
+    *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < nvalid) dst[j] = y[j];
+  }
+}
+
+__device__ __forceinline__ float gelu_tanh_f32(float z) {
+  // 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
+  const float u = 0.7978845608028654f * fmaf(0.044715f * z * z, z, z);
+  return 0.5f * z * (1.f + ptx::tanh_approx(u));
+}
+__device__ __forceinline__ float silu_f32(float g) { return __fdividef(g, 1.f + __expf(-g)); }
+
+// The fused element-wise operation on 8 consecutive output columns.
+template <int EPI>
+__device__ __forceinline__ void apply_epilogue8(const uint32_t* acc, const uint32_t* acc_up, const float (&bias)[8],
+                                                const float (&res)[8], float (&y)[8]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float a = __uint_as_float(acc[j]);
+    if constexpr (EPI == kEpiNone || EPI == kEpiPartial) {
+      y[j] = a;
+    } else if constexpr (EPI == kEpiBias) {
+      y[j] = a + bias[j];
+    } else if constexpr (EPI == kEpiBiasRelu) {
+      y[j] = fmaxf(a + bias[j], 0.f);
+    } else if constexpr (EPI == kEpiBiasGeluTanh) {
+      y[j] = gelu_tanh_f32(a + bias[j]);
+    } else if constexpr (EPI == kEpiSiluGate) {
+      y[j] = silu_f32(a) * __uint_as_float(acc_up[j]);
+    } else {  // kEpiBiasResidual
+      y[j] = a + bias[j] + res[j];
+    }
+  }
+}
+
+template <int CG, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+    fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_mem[2 * kMaxStages + 4];
+  __shared__ uint32_t tmem_holder;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = ptx::smem_u32(bar_mem);
+  auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
+  auto accf_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + b); };
+  auto acce_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kMaxStages; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(accf_bar(b), 1);
+      ptx::mbar_init(acce_bar(b), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
+    }
+    abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc<CG>(ptx::smem_u32(&tmem_holder), p.tmem_cols);
+    ptx::tmem_relinquish<CG>();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {  // the peer's barriers must exist before anything arrives on them
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_holder);
+
+  const int unit0 = (int)(blockIdx.x / CG);
+  const int unit_stride = (int)(gridDim.x / CG);
+  volatile int* abort_p = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+        const WorkUnit w = decode_unit(p, u);
+        const int m0 = (w.tm * CG + (int)cta_rank) * kTileM;
+        // first accumulator column this CTA's B boxes feed
+        const int col0 = (CG == 2) ? (int)cta_rank * (p.tile_n / 2) : 0;
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!wait_bar(empty_bar(stage), phase ^ 1u, abort_p, p.status)) {
+            ok = false;
+            break;
+          }
+          const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
+          const uint32_t sb = sa + kStageBytesA;
+          uint32_t fb = full_bar(stage);
+          if constexpr (CG == 2) {
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
+            fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
+            ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
+          } else {
+            ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
+            ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+          }
+          for (int i = 0; i < p.b_loads; ++i) {
+            const int col = col0 + i * p.b_box_n;  // accumulator column of this box
+            int n;
+            if (p.gate) {
+              const int half = p.tile_n >> 1;
+              n = (col < half) ? (w.tn * half + col) : (p.N_out + w.tn * half + (col - half));
+            } else {
+              n = w.tn * p.tile_n + col;
+            }
+            const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
+            if constexpr (CG == 2) {
+              if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n, kb * kTileK, w.b);
+              else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n, w.b);
+            } else {
+              if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n, kb * kTileK, w.b);
+              else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n, w.b);
+            }
+          }
+          if (++stage == p.stages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      // Drain: wait until every stage this CTA filled has been released, so that no
+      // commit arrival is still on its way to this CTA's barriers when it exits.
+      for (int s = 0; ok && s < p.stages; ++s) {
+        if (!wait_bar(empty_bar(stage), phase ^ 1u, abort_p, p.status)) ok = false;
+        if (++stage == p.stages) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0 && cta_rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+        const WorkUnit w = decode_unit(p, u);
+        if (!wait_bar(acce_bar(acc), acc_phase ^ 1u, abort_p, p.status)) {
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tile_n);
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!wait_bar(full_bar(stage), phase, abort_p, p.status)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
+          const uint32_t sb = sa + kStageBytesA;
+          const uint64_t adesc = p.a_desc | (uint64_t)((sa >> 4) & 0x3fffu);
+          const uint64_t bdesc = p.b_desc | (uint64_t)((sb >> 4) & 0x3fffu);
+#pragma unroll
+          for (int k = 0; k < kTileK / kUmmaK; ++k) {
+            ptx::umma_bf16<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
+                               p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+          }
+          // release the stage (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (CG == 2) ptx::umma_commit_pair(empty_bar(stage), 0x3);
+          else ptx::umma_commit<CG>(empty_bar(stage));
+          if (++stage == p.stages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (!ok) break;
+        if constexpr (CG == 2) ptx::umma_commit_pair(accf_bar(acc), 0x3);
+        else ptx::umma_commit<CG>(accf_bar(acc));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;  // the TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    const bool c_vec = p.c_vec != 0;
+    for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+      const WorkUnit w = decode_unit(p, u);
+      if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+        ok = false;
+        break;
+      }
+      ptx::tc_fence_after();
+      const int row = (w.tm * CG + (int)cta_rank) * kTileM + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+      const int n_tile0 = w.tn * p.out_cols;
+      // destination row
+      char* c_row;
+      if constexpr (EPI == kEpiPartial) {
+        c_row = reinterpret_cast<char*>(p.ws + (long long)w.split * p.ws_split_stride +
+                                        (long long)w.b * p.ws_batch_stride + (long long)row * p.ws_ld);
+      } else {
+        const long long off = (long long)w.b * p.strideC + (long long)row * p.ldc;
+        c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
+      }
+      const __nv_bfloat16* r_row = nullptr;
+      if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
+
+      for (int c = 0; c < p.out_cols; c += 32) {
+        const int n0 = n_tile0 + c;
+        if (n0 >= p.N_out) break;  // uniform across the warp
+        uint32_t v[32];
+        uint32_t vu[32];
+        ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
+        if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
+        ptx::tmem_wait_ld();
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int n = n0 + g * 8;
+          const int nvalid = min(8, p.N_out - n);
+          float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          float y[8];
+          if (nvalid > 0) {
+            if constexpr (EPI == kEpiBias || EPI == kEpiBiasRelu || EPI == kEpiBiasGeluTanh ||
+                          EPI == kEpiBiasResidual) {
+              if (p.bias != nullptr) load_bf16x8(p.bias + n, nvalid, p.bias_vec != 0, bias);
+            }
+            if constexpr (EPI == kEpiBiasResidual) {
+              if (row_ok) load_bf16x8(r_row + n, nvalid, p.r_vec != 0, res);
+            }
+            apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
+            if (row_ok) {
+              if (EPI == kEpiPartial || p.out_f32) store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid,
+                                                                 EPI == kEpiPartial || c_vec);
+              else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
+            }
+          }
+        }
+      }
+      // hand the accumulator back to the MMA issuer (of the leader CTA)
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(acce_bar(acc), 0));
+        else ptx::mbar_arrive(acce_bar(acc));
+      }
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  if (*abort_p) {
+    // a wait expired somewhere: give copies that may still be in flight time to land
+    const unsigned long long t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 200000ull) {
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {  // neither CTA may free tensor memory or exit while its peer still uses it
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc<CG>(tmem_base, p.tmem_cols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K reduction: adds the S partials of every output element in ascending slice order,
+// applies the epilogue and stores.  One thread per 4 consecutive output columns.
+struct ReduceParams {
+  const float* ws;
+  long long ws_ld, ws_batch_stride, ws_split_stride;
+  int splits;
+  int M, N_out, batch;
+  int epi;
+  void* C;
+  long long ldc, strideC;
+  int out_f32;
+  const __nv_bfloat16* bias;
+  const __nv_bfloat16* R;
+  long long ldr, strideR;
+};
+
+__device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, float bias, float res) {
+  switch (epi) {
+    case kEpiBias: return a + bias;
+    case kEpiBiasRelu: return fmaxf(a + bias, 0.f);
+    case kEpiBiasGeluTanh: return gelu_tanh_f32(a + bias);
+    case kEpiSiluGate: return silu_f32(a) * up;
+    case kEpiBiasResidual: return a + bias + res;
+    default: return a;
+  }
+}
+
+__global__ void __launch_bounds__(256) fact_splitk_reduce_kernel(const ReduceParams p) {
+  const long long groups_per_row = (p.N_out + 3) / 4;
+  const long long total = (long long)p.batch * p.M * groups_per_row;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int gcol = (int)(i % groups_per_row);
+    const long long rm = i / groups_per_row;
+    const int m = (int)(rm % p.M);
+    const int b = (int)(rm / p.M);
+    const int n = gcol * 4;
+    const int nvalid = min(4, p.N_out - n);
+    float a[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
+    const float* src = p.ws + (long long)b * p.ws_batch_stride + (long long)m * p.ws_ld + n;
+    const bool gate = p.epi == kEpiSiluGate;
+    const bool up_vec = (p.N_out & 3) == 0;
+    for (int s = 0; s < p.splits; ++s) {  // ascending slice order: deterministic
+      const float* ps = src + (long long)s * p.ws_split_stride;
+      const float4 v = *reinterpret_cast<const float4*>(ps);  // ws_ld is a multiple of 4: in-bounds padding
+      a[0] += v.x; a[1] += v.y; a[2] += v.z; a[3] += v.w;
+      if (gate) {
+        if (up_vec) {
+          const float4 t = *reinterpret_cast<const float4*>(ps + p.N_out);
+          up[0] += t.x; up[1] += t.y; up[2] += t.z; up[3] += t.w;
+        } else {
+          for (int j = 0; j < nvalid; ++j) up[j] += ps[p.N_out + j];
+        }
+      }
+    }
+    for (int j = 0; j < nvalid; ++j) {
+      const float bias = p.bias ? __bfloat162float(p.bias[n + j]) : 0.f;
+      const float res =
+          (p.epi == kEpiBiasResidual) ? __bfloat162float(p.R[(long long)b * p.strideR + (long long)m * p.ldr + n + j]) : 0.f;
+      const float y = reduce_epilogue(p.epi, a[j], up[j], bias, res);
+      const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n + j;
+      if (p.out_f32) reinterpret_cast<float*>(p.C)[off] = y;
+      else reinterpret_cast<__nv_bfloat16*>(p.C)[off] = __float2bfloat16_rn(y);
+    }
+  }
+}
+
+}  // namespace fact

@@ -1,0 +1,220 @@
+"""GPU parity tests: libfact (through the C ABI binding) against the FP64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_26666_b200 import workloads as wl
+from tests.helpers import check_case, gates, oracle_for, run_gpu, small_int_inputs, to_f64
+
+pytestmark = pytest.mark.gpu
+
+ALL_EPI = ["NONE", "BIAS", "BIAS_RELU", "BIAS_GELU_TANH", "SILU_GATE", "BIAS_RESIDUAL"]
+
+
+@pytest.fixture(scope="module")
+def h():
+    from paper_2604_26666_b200.binding import Handle
+    hd = Handle(0)
+    yield hd
+    hd.close()
+
+
+def mk(name, M, N, K, op="linear", epilogue="NONE", layout="KN", out="bf16", batch=1, seed=5, **kw):
+    has_bias = epilogue in ("BIAS", "BIAS_RELU", "BIAS_GELU_TANH", "BIAS_RESIDUAL")
+    has_res = epilogue == "BIAS_RESIDUAL"
+    return wl.Case(name, op, M, N, K, batch=batch, epilogue=epilogue, layout=layout, out=out, has_bias=has_bias,
+                   has_residual=has_res, seed=seed, **kw)
+
+
+def bit_exact(h, case, ins, cfg=None, splits=0):
+    got = run_gpu(h, ins, case, cfg=cfg, splits=splits)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    ref = oracle_for(ins, case)
+    if case.out == "bf16":
+        want = np.vectorize(oracle.round_bf16, otypes=[np.uint16])(ref)
+        gotb = wl.bits(got.cpu().contiguous())
+        bad = np.argwhere(gotb != want)
+    else:
+        bad = np.argwhere(got.cpu().double().numpy() != ref)
+    assert len(bad) == 0, f"{case.name}: {len(bad)} of {ref.size} elements differ, first at {bad[:5].tolist()}"
+
+
+# ------------------------------------------------------------------ exact pins
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+def test_identity_is_bit_exact(h, layout):
+    g = torch.Generator().manual_seed(1)
+    M, K = 200, 256
+    X = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    W = torch.eye(K).to(torch.bfloat16)
+    case = mk("identity", M, K, K, layout=layout)
+    got = run_gpu(h, wl.Inputs(X, W), case)
+    assert torch.equal(got.cpu(), X)
+
+
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("K", [64, 512, 768, 3072, 4096])
+def test_all_ones_gives_K(h, layout, K):
+    M, N = 130, 192
+    X = torch.ones(M, K, dtype=torch.bfloat16)
+    W = torch.ones((K, N) if layout == "KN" else (N, K), dtype=torch.bfloat16)
+    got = run_gpu(h, wl.Inputs(X, W), mk("ones", M, N, K, layout=layout, out="f32"))
+    assert (got.cpu() == float(K)).all()
+
+
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+def test_positional_probe(h, layout):
+    # C[i, j] = (i % 7 + 1) * (j % 5 + 1) through a single k: locates any row/column/swizzle mix-up
+    M, N, K = 256, 256, 128
+    for k0 in (0, 5, 17, 63, 64, 127):
+        A = torch.zeros(M, K)
+        B = torch.zeros(K, N)
+        A[:, k0] = (torch.arange(M) % 7 + 1).float()
+        B[k0, :] = (torch.arange(N) % 5 + 1).float()
+        W = B if layout == "KN" else B.t().contiguous()
+        case = mk("probe", M, N, K, layout=layout, out="f32")
+        got = run_gpu(h, wl.Inputs(A.to(torch.bfloat16), W.to(torch.bfloat16)), case).cpu()
+        want = torch.outer(torch.arange(M) % 7 + 1, torch.arange(N) % 5 + 1).float()
+        assert torch.equal(got, want), f"k0={k0}: {(got != want).sum().item()} wrong"
+
+
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("out", ["bf16", "f32"])
+def test_small_integers_bit_exact(h, layout, out):
+    case = mk("ints", 300, 320, 1000 if layout == "NK" else 1000, layout=layout, out=out)
+    bit_exact(h, case, small_int_inputs(case, 7))
+
+
+# ------------------------------------------------------------------ epilogues, layouts, tails
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("epi", ALL_EPI)
+@pytest.mark.parametrize("out", ["bf16", "f32"])
+def test_epilogues_ragged(h, layout, epi, out):
+    # 3 m-tiles with a tail, 2 n-tiles with a tail, K not a multiple of 64
+    case = mk(f"rag_{epi}", 300, 328, 520, epilogue=epi, layout=layout, out=out, w_scale=0.05)
+    check_case(h, case)
+
+
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("epi", ["BIAS_RELU", "SILU_GATE", "BIAS_RESIDUAL"])
+def test_epilogue_exact_on_integers(h, layout, epi):
+    # ReLU / residual on integer data are exact; SiLU is compared through the gate
+    case = mk(f"int_{epi}", 140, 136, 200, epilogue=epi, layout=layout, out="f32")
+    ins = small_int_inputs(case, 9, lo=-2, hi=2)
+    if epi == "SILU_GATE":
+        check_case(h, case, ins=ins)
+    else:
+        bit_exact(h, case, ins)
+
+
+@pytest.mark.parametrize("tile_n", [32, 64, 96, 128, 192, 256])
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+def test_tile_widths(h, tile_n, layout):
+    if layout == "KN" and tile_n % 64:
+        pytest.skip("N-major B tiles are whole 64-column boxes")
+    case = mk(f"tn{tile_n}", 260, 520, 384, epilogue="BIAS", layout=layout)
+    check_case(h, case, cfg={"tile_n": tile_n})
+
+
+@pytest.mark.parametrize("stages", [2, 3, 4, 6])
+def test_stage_counts(h, stages):
+    case = mk(f"st{stages}", 256, 256, 2048, layout="NK")
+    check_case(h, case, cfg={"tile_n": 128, "stages": stages})
+
+
+def test_unaligned_output_and_odd_sizes(h):
+    # N odd: rows of C are not 16-byte aligned -> element-wise stores
+    for (M, N, K) in [(1, 1, 8), (5, 7, 24), (129, 33, 72), (64, 250, 136)]:
+        case = mk(f"odd_{M}_{N}_{K}", M, N, K, epilogue="BIAS_RESIDUAL", layout="NK")
+        check_case(h, case)
+
+
+def test_strided_operands(h):
+    g = torch.Generator().manual_seed(3)
+    M, N, K = 150, 200, 264
+    Xbig = torch.randn(M, K + 24, generator=g).to(torch.bfloat16)
+    Wbig = (torch.randn(N, K + 8, generator=g) * 0.1).to(torch.bfloat16)
+    Cbig = torch.zeros(M, N + 16, dtype=torch.bfloat16, device="cuda")
+    out = Cbig[:, :N]
+    h.linear(Xbig.cuda()[:, :K], Wbig.cuda()[:, :K], layout="NK", out=out)
+    torch.cuda.synchronize()
+    ref = oracle.linear(wl.bits(Xbig)[:, :K], wl.bits(Wbig)[:, :K], layout="NK")
+    c, t = gates(ref, to_f64(out), "bf16", "NONE")
+    assert c <= 1 and t <= 1
+    assert (Cbig[:, N:] == 0).all(), "wrote outside the N columns"
+
+
+# ------------------------------------------------------------------ batched and split-K
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+def test_batched(h, layout):
+    case = mk("batched", 136, 200, 264, op="gemm_batched", batch=5, layout=layout)
+    check_case(h, case)
+
+
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("splits", [0, 2, 7, 16])
+def test_splitk_parity_and_determinism(h, layout, splits):
+    case = mk("splitk", 256, 256, 8192 + 64, op="gemm_splitk", layout=layout, out="f32",
+              x_dist="uniform", w_dist="uniform")
+    ins = wl.make_inputs(case)
+    check_case(h, case, splits=splits, ins=ins)
+    a = run_gpu(h, ins, case, splits=splits).clone()
+    for _ in range(3):
+        b = run_gpu(h, ins, case, splits=splits)
+        assert torch.equal(a, b), "split-K result changed between runs"
+
+
+def test_splitk_exact_on_integers_for_any_split(h):
+    case = mk("splitk_int", 200, 136, 4096, op="gemm_splitk", layout="KN", out="f32")
+    ins = small_int_inputs(case, 11)
+    for s in (1, 3, 8, 64):
+        bit_exact(h, case, ins, splits=s)
+
+
+def test_splitk_with_epilogue_through_linear(h):
+    for epi in ("BIAS_GELU_TANH", "SILU_GATE", "BIAS_RESIDUAL"):
+        case = mk(f"lin_split_{epi}", 200, 264, 2048, epilogue=epi, layout="NK", w_scale=0.05)
+        check_case(h, case, cfg={"split_k": 5})
+
+
+# ------------------------------------------------------------------ degenerate sizes
+def test_empty_and_k_zero(h):
+    dev = "cuda:0"
+    A = torch.zeros(0, 64, dtype=torch.bfloat16, device=dev)
+    B = torch.zeros(64, 32, dtype=torch.bfloat16, device=dev)
+    assert h.gemm(A, B).shape == (0, 32)
+    # K == 0: the epilogue of a zero accumulator
+    X = torch.zeros(10, 0, dtype=torch.bfloat16, device=dev)
+    W = torch.zeros(24, 0, dtype=torch.bfloat16, device=dev)
+    bias = torch.arange(24, dtype=torch.float32).to(torch.bfloat16).to(dev)
+    y = h.linear(X, W, bias=bias, epilogue="BIAS_RELU", layout="NK")
+    assert torch.equal(y.cpu(), bias.cpu().expand(10, 24))
+
+
+# ------------------------------------------------------------------ host-side error paths
+def test_error_codes(h):
+    from paper_2604_26666_b200.binding import FactError
+    dev = "cuda:0"
+    A = torch.zeros(64, 72, dtype=torch.bfloat16, device=dev)
+    B = torch.zeros(72, 64, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(FactError) as e:
+        h.gemm(A[:, 1:65], B[:64])  # operand pointer not 16-byte aligned
+    assert e.value.code == 2
+    with pytest.raises(FactError) as e:
+        h.linear(A, B, epilogue="BIAS", layout="KN")  # missing bias
+    assert e.value.code == 1
+    with pytest.raises(FactError) as e:
+        h.gemm(A, B, cfg={"tile_n": 48})  # not a multiple of 32
+    assert e.value.code == 3
+    with pytest.raises(FactError) as e:
+        h.gemm(A, B, cfg={"tile_n": 256, "stages": 8})  # over the shared-memory budget
+    assert e.value.code == 3
+    # split-K without enough workspace, through the raw C entry point
+    from ctypes import c_void_p
+    from paper_2604_26666_b200.binding import lib
+    C = torch.zeros(64, 64, dtype=torch.float32, device=dev)
+    rc = lib().fact_gemm_splitk(h._h, 64, 64, 72, c_void_p(A.data_ptr()), 72, c_void_p(B.data_ptr()), 64, 0,
+                                c_void_p(C.data_ptr()), 64, 1, 2, None, None, 0, None)
+    assert rc == 5
+    assert (C == 0).all()
