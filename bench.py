@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of libfact on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-shapes]
+
+One "step" is one pass over the square-GEMM configuration (C = A.B at 4096^3
+and 8192^3, BF16 in, FP32 accumulate, BF16 out, operands N(0,1)/sqrt(K),
+seed 1).  The headline value is whole-job TFLOP/s (2 M N K per product,
+epilogue work not counted) with inputs resident in HBM; `e2e` repeats it with
+pinned-host inputs copied in and the result copied out inside the timed region.
+`shapes` adds, for every shape of the five configurations, its own time,
+TFLOP/s, GB/s and roofline fraction, next to a cuBLAS (torch.matmul) side
+reference that is never on the product path.
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU (the
+path shards by rows / batch entries with no exchange step): weak scaling, value
+= all ranks' FLOPs / max-over-ranks time.
+
+`--impl reference` times the FP64 CPU oracle on the host cores on a bounded row
+slab of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "TFLOP/s & % of dense BF16 tensor peak per fused-epilogue GEMM shape"
+WORKLOAD = "config 2: square BF16 GEMM 4096^3 + 8192^3, N(0,1)/sqrt(K), seed 1"
+L2_FLUSH_BYTES = 512 << 20
+
+# DRAM traffic per launch of the dominant kernel (8192^3), from the ncu capture summarised in
+# profiles/ (None until a capture exists).
+DOMINANT_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        # keep the samples taken under load (clock above idle), else all
+        busy = [c for c in sm if c > 0.5 * (max(mx) if mx else 1)] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_time_case(case, ins, target_seconds: float):
+    """Time the oracle (as it stands) on a leading row slab of `case` sized for about `target_seconds`.
+    Returns (tflops, rows, seconds, threads)."""
+    import numpy as np
+
+    import oracle
+    from paper_2604_26666_b200 import workloads as wl
+
+    xb, wb = wl.bits(ins.X), wl.bits(ins.W)
+    bias = None if ins.bias is None else wl.bits(ins.bias)
+    res = None if ins.residual is None else wl.bits(ins.residual)
+    if case.batch > 1:
+        xb, wb = xb[:1], wb[:1]
+        res = None if res is None else res[:1]
+    flops_per_row = 2.0 * case.n_weight_cols * case.K
+
+    def run(rows):
+        idx = np.arange(rows, dtype=np.int64)
+        t0 = time.perf_counter()
+        oracle.linear(xb, wb, layout=case.layout, epilogue=case.epilogue, bias=bias, residual=res, rows=idx)
+        return time.perf_counter() - t0
+
+    probe_rows = min(case.M, 64)
+    t_probe = run(probe_rows)
+    rate = probe_rows * flops_per_row / max(t_probe, 1e-9)
+    rows = int(max(probe_rows, min(case.M, target_seconds * rate / flops_per_row)))
+    rows = max(8, rows // 8 * 8) if case.M >= 8 else case.M
+    t = run(rows)
+    return rows * flops_per_row / t / 1e12, rows, t, oracle.max_threads()
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on the host cores, bounded row slabs of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2604_26666_b200 import workloads as wl
+
+    cases = [c for c in wl.benchmark_cases() if c.config == 2]
+    per_step_budget = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    inputs = [wl.make_inputs(c) for c in cases]
+    times, flops, samples, threads = [], [], [], 1
+    for it in range(args.warmup + args.steps):
+        t_step, f_step, desc = 0.0, 0.0, []
+        for c, ins in zip(cases, inputs):
+            tf, rows, secs, threads = oracle_time_case(c, ins, per_step_budget / len(cases))
+            t_step += secs
+            f_step += tf * 1e12 * secs
+            desc.append(f"{c.name}: first {rows} of {c.M} rows")
+        if it >= args.warmup:
+            times.append(t_step)
+            flops.append(f_step)
+            samples = desc
+    value = sum(flops) / sum(times) / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "each step is a bounded leading-row slab of every GEMM"},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+                         "sample": "; ".join(samples)},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ product arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="fact", choices=["fact", "reference"])
+    ap.add_argument("--no-shapes", action="store_true", help="skip the per-shape table")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+    from paper_2604_26666_b200.binding import Handle
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    h = Handle(local_rank)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def flush_l2():
+        flush_buf.fill_(1)
+
+    tune_table = os.path.join(ROOT, "paper_2604_26666_b200", "tuned_b200.txt")
+    if os.path.exists(tune_table):
+        h.tune_cache_load(tune_table)
+
+    # ---------------------------------------------------------------- headline: config 2
+    cases = [c for c in wl.benchmark_cases() if c.config == 2]
+    host_inputs = [wl.make_inputs(c, pin=True) for c in cases]
+    dev_inputs = [(i.X.to(dev), i.W.to(dev)) for i in host_inputs]
+    outs = [torch.empty((c.M, c.N), dtype=torch.bfloat16, device=dev) for c in cases]
+    step_flops = sum(c.flops for c in cases)
+    dom = max(range(len(cases)), key=lambda i: cases[i].flops)
+
+    if args.tune:
+        for c, (X, W), o in zip(cases, dev_inputs, outs):
+            h.tune("gemm", X, W, layout=c.layout, out=o)
+
+    def step(events=None):
+        for i, (c, (X, W), o) in enumerate(zip(cases, dev_inputs, outs)):
+            if events is not None and i == dom:
+                events[0].record(stream)
+            h.gemm(X, W, layout=c.layout, out=o)
+            if events is not None and i == dom:
+                events[1].record(stream)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = h.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+           torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for s in range(args.steps):
+        flush_l2()  # untimed: between timed iterations the L2 is overwritten by a 512 MB fill
+        ev[s][0].record(stream)
+        step(events=(ev[s][2], ev[s][3]))
+        ev[s][1].record(stream)
+    barrier()
+    launches = h.launch_count() - launches0
+    step_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    dom_ms = [e[2].elapsed_time(e[3]) for e in ev]
+    total_ms = sum(step_ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    assert h.device_status() == 0, "a device-side wait timed out during the timed region"
+    value = world * step_flops * args.steps / (total_ms * 1e-3) / 1e12
+    dom_case = cases[dom]
+    dom_avg_ms = sum(dom_ms) / len(dom_ms)
+    achieved = dom_case.flops / (dom_avg_ms * 1e-3) / 1e12
+
+    # ---------------------------------------------------------------- end to end: host buffers in, host result out
+    h2d = sum(i.X.numel() * 2 + i.W.numel() * 2 for i in host_inputs)
+    d2h = sum(o.numel() * 2 for o in outs)
+    host_outs = [torch.empty((c.M, c.N), dtype=torch.bfloat16).pin_memory() for c in cases]
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        for c, hi, (X, W), o, ho in zip(cases, host_inputs, dev_inputs, outs, host_outs):
+            X.copy_(hi.X, non_blocking=True)
+            W.copy_(hi.W, non_blocking=True)
+            h.gemm(X, W, layout=c.layout, out=o)
+            ho.copy_(o, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * step_flops * e2e_steps / (e2e_ms * 1e-3) / 1e12
+    clocks = sampler.stop()
+    del host_outs
+
+    # ---------------------------------------------------------------- every shape of the five configurations
+    shapes = []
+    if not args.no_shapes and rank == 0:
+        shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
+
+    # ---------------------------------------------------------------- CPU baseline (oracle) on rank 0
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tf, rows, secs, threads = oracle_time_case(dom_case, host_inputs[dom], 15.0)
+        cpu = {"value": tf, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+               "sample": f"first {rows} of {dom_case.M} rows of the {dom_case.M}^3 GEMM, {secs:.1f} s "
+                         f"(cost is linear in M)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "b_layout": "KN (row-major B)", "timing": "CUDA events per step",
+                       "l2": "512 MB fill between timed steps (untimed); step footprint 480 MB > L2",
+                       "parallelism": f"dp{world} (independent replicas of the workload, no collective)"},
+            "pct_of_peak": {"burst_measured": 100 * value / world / peaks["bf16_tflops"],
+                            "sustained_measured": 100 * value / world / peaks["bf16_tflops_sustained"],
+                            "nominal_2250": 100 * value / world / 2250.0, "peaks": peaks["source"]},
+            "roofline": {"bound": "tensor", "kernel": f"fact_gemm_kernel on {dom_case.name}", "achieved": achieved,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                         "peak_source": peaks["source"] + " (burst)", "launch_ms": dom_avg_ms,
+                         "traffic": DOMINANT_TRAFFIC_BYTES},
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "cpu_baseline": cpu,
+            "shapes": shapes,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    h.close()
+    return 0
+
+
+def per_shape_table(h, dev, stream, flush_l2, peaks, tune):
+    """Time every benchmark shape alone (5 warm-up + 20 timed launches, L2 overwritten between launches)."""
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    rows = []
+    for case in wl.benchmark_cases():
+        ins = wl.make_inputs(case)
+        X, W = ins.X.to(dev), ins.W.to(dev)
+        bias = None if ins.bias is None else ins.bias.to(dev)
+        res = None if ins.residual is None else ins.residual.to(dev)
+        odt = torch.float32 if case.out == "f32" else torch.bfloat16
+        oshape = (case.batch, case.M, case.N) if case.batch > 1 else (case.M, case.N)
+        out = torch.empty(oshape, dtype=odt, device=dev)
+
+        def call():
+            if case.op == "gemm":
+                h.gemm(X, W, layout=case.layout, out=out)
+            elif case.op == "gemm_batched":
+                h.gemm_batched(X, W, layout=case.layout, out=out)
+            elif case.op == "gemm_splitk":
+                h.gemm_splitk(X, W, layout=case.layout, out=out)
+            else:
+                h.linear(X, W, bias=bias, residual=res, epilogue=case.epilogue, layout=case.layout, out=out)
+
+        def side():
+            # cuBLAS through torch: the bare product only, as a side reference
+            if case.batch > 1:
+                torch.bmm(X, W if case.layout == "KN" else W.transpose(1, 2))
+            else:
+                torch.matmul(X, W if case.layout == "KN" else W.t())
+
+        if tune:
+            h.tune(case.op, X, W, layout=case.layout, bias=bias, residual=res, epilogue=case.epilogue, out=out)
+
+        def time_it(fn, warm=5, iters=20, cold=True):
+            for _ in range(warm):
+                fn()
+            ts = []
+            for _ in range(iters):
+                if cold:
+                    flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                ts.append((a, b))
+            torch.cuda.synchronize(dev)
+            return sorted(x.elapsed_time(y) for x, y in ts)
+
+        t = time_it(call)
+        t_hot = time_it(call, cold=False)
+        t_side = time_it(side, iters=10)
+        med = t[len(t) // 2]
+        t_tensor = case.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        bound = "tensor" if t_tensor >= t_hbm else "hbm"
+        cfg = h.get_config(case.op, case.batch, case.M, case.N, case.K, case.epilogue, case.layout, odt).as_dict()
+        rows.append({
+            "name": case.name, "config": case.config, "op": case.op, "epilogue": case.epilogue,
+            "layout": case.layout, "batch": case.batch, "M": case.M, "N": case.N, "K": case.K, "out": case.out,
+            "us_median": med * 1e3, "us_min": t[0] * 1e3, "us_hot_l2_median": t_hot[len(t_hot) // 2] * 1e3,
+            "tflops": case.flops / (med * 1e-3) / 1e12, "gbs": case.algorithmic_bytes / (med * 1e-3) / 1e9,
+            "pct_of_bf16_peak_burst": 100 * case.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "bound": bound, "roofline_us": max(t_tensor, t_hbm) * 1e3,
+            "roofline_frac": max(t_tensor, t_hbm) / med,
+            "cublas_matmul_only_us": t_side[len(t_side) // 2] * 1e3, "tile": cfg,
+        })
+        del X, W, out
+    return rows
+
+
+if __name__ == "__main__":
+    sys.exit(main())

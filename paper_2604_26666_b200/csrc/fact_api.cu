@@ -127,7 +127,11 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (splits_override > 0) c.split_k = splits_override;
   if (c.tile_k != 0 && c.tile_k != kTileK) return FACT_ERR_UNSUPPORTED;
   c.tile_k = kTileK;
-  if (c.cta_group == 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
+  if (c.cta_group == 0) {
+    // A 2-CTA pair halves each CTA's B traffic; it pays once a 256-row tile is mostly full.
+    if (c.tile_m != 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
+    else c.cta_group = (q.M > 192 && q.Nw() >= 128 && (c.tile_n == 0 || tile_ok(q, c.tile_n, 2))) ? 2 : 1;
+  }
   if (c.tile_m == 0) c.tile_m = 128 * c.cta_group;
   if (c.tile_m != 128 * c.cta_group) return FACT_ERR_UNSUPPORTED;
   const long long Nw = q.Nw();

@@ -399,9 +399,21 @@ __global__ void __launch_bounds__(kThreads, 1)
       const __nv_bfloat16* r_row = nullptr;
       if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
 
-      for (int c = 0; c < p.out_cols; c += 32) {
-        const int n0 = n_tile0 + c;
-        if (n0 >= p.N_out) break;  // uniform across the warp
+      // A split-K partial stores every accumulator column; a gated accumulator holds the gate
+      // columns in its first half and the up columns (N_out further right in W) in its second.
+      const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
+      for (int c = 0; c < acc_cols; c += 32) {
+        int n0 = n_tile0 + c;
+        int n_limit = p.N_out;
+        if (EPI == kEpiPartial && p.gate) {
+          const int half = p.tile_n >> 1;
+          const int g0 = w.tn * half + (c < half ? c : c - half);
+          if (g0 >= p.N_out) continue;  // uniform across the warp
+          n0 = (c < half) ? g0 : p.N_out + g0;
+          n_limit = (c < half) ? p.N_out : 2 * p.N_out;
+        } else if (n0 >= p.N_out) {
+          break;  // uniform across the warp
+        }
         uint32_t v[32];
         uint32_t vu[32];
         ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
@@ -410,7 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int n = n0 + g * 8;
-          const int nvalid = min(8, p.N_out - n);
+          const int nvalid = min(8, n_limit - n);
           float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
           float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
           float y[8];
@@ -424,8 +436,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
             apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
             if (row_ok) {
-              if (EPI == kEpiPartial || p.out_f32) store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid,
-                                                                 EPI == kEpiPartial || c_vec);
+              if (EPI == kEpiPartial || p.out_f32)
+                store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid,
+                            EPI == kEpiPartial ? ((n & 3) == 0) : c_vec);
               else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
             }
           }
