@@ -186,6 +186,10 @@ def main():
     ap.add_argument("--no-shapes", action="store_true", help="skip the per-shape table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
+    ap.add_argument("--shape", default=None,
+                    help="time only this benchmark shape (a name from the `shapes` table, or `all`): "
+                         "--warmup/--steps launches, no side reference; the small command used for profiling")
+    ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -227,6 +231,14 @@ def main():
     tune_table = os.path.join(ROOT, "paper_2604_26666_b200", "tuned_b200.txt")
     if os.path.exists(tune_table):
         h.tune_cache_load(tune_table)
+
+    if args.shape is not None:
+        names = None if args.shape == "all" else args.shape.split(",")
+        rows = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup,
+                               iters=args.steps, side_ref=False, layout=args.layout)
+        print(json.dumps({"shapes": rows, "gpu_launches": h.launch_count()}))
+        h.close()
+        return 0
 
     # ---------------------------------------------------------------- headline: config 2
     cases = [c for c in wl.benchmark_cases() if c.config == 2]
@@ -350,14 +362,16 @@ def main():
     return 0
 
 
-def per_shape_table(h, dev, stream, flush_l2, peaks, tune):
+def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, iters=20, side_ref=True, layout="NK"):
     """Time every benchmark shape alone (5 warm-up + 20 timed launches, L2 overwritten between launches)."""
     import torch
 
     from paper_2604_26666_b200 import workloads as wl
 
     rows = []
-    for case in wl.benchmark_cases():
+    for case in wl.benchmark_cases(layout):
+        if names is not None and case.name not in names:
+            continue
         ins = wl.make_inputs(case)
         X, W = ins.X.to(dev), ins.W.to(dev)
         bias = None if ins.bias is None else ins.bias.to(dev)
@@ -386,7 +400,7 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune):
         if tune:
             h.tune(case.op, X, W, layout=case.layout, bias=bias, residual=res, epilogue=case.epilogue, out=out)
 
-        def time_it(fn, warm=5, iters=20, cold=True):
+        def time_it(fn, warm=warm, iters=iters, cold=True):
             for _ in range(warm):
                 fn()
             ts = []
@@ -402,8 +416,8 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune):
             return sorted(x.elapsed_time(y) for x, y in ts)
 
         t = time_it(call)
-        t_hot = time_it(call, cold=False)
-        t_side = time_it(side, iters=10)
+        t_hot = time_it(call, cold=False) if side_ref else t
+        t_side = time_it(side, iters=10) if side_ref else [0.0]
         med = t[len(t) // 2]
         t_tensor = case.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
         t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3

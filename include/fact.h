@@ -207,6 +207,13 @@ fact_status_t fact_device_status(fact_handle_t handle, void* cuda_stream, int* s
 /* Number of kernels this handle has launched so far (for benchmark reports). */
 int64_t fact_launch_count(fact_handle_t handle);
 
+/* Diagnostic: synchronise `cuda_stream` and return how many SM clock cycles and
+ * how many nanoseconds the first CTA of the most recent GEMM kernel launch spent
+ * between its start and its end.  cycles / nanoseconds is the SM clock (GHz)
+ * that launch really ran at, which a power-limited part does not keep constant. */
+fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, int64_t* sm_cycles,
+                                     int64_t* nanoseconds);
+
 /* Text of the most recent CUDA runtime/driver failure seen through this handle
  * (the call that returned FACT_ERR_CUDA), "" if none.  Owned by the handle;
  * valid until the next failing call or fact_destroy. */

@@ -7,6 +7,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <string>
@@ -70,6 +71,7 @@ struct fact_handle_s {
   std::map<TuneKey, fact_config_t> table;
   unsigned configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
+  int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
 };
 
 namespace {
@@ -292,6 +294,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.ws_batch_stride = (long long)p.M * p.ws_ld;
   p.ws_split_stride = p.ws_batch_stride * p.batch;
   p.status = h->d_status;
+  p.debug = h->debug_flags;
   plan->ws_bytes = workspace_for(q, c);
   plan->smem_bytes = std::max(c.stages * (int)p.stage_bytes + kSmemSlack, kMinSmemRequest);
   if (plan->smem_bytes > kSmemBudget || kSmemBudget + 1024 > h->max_smem) return FACT_ERR_UNSUPPORTED;
@@ -505,6 +508,7 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
   h->max_smem = (int)prop.sharedMemPerBlockOptin;
   h->cc_major = prop.major;
   h->cc_minor = prop.minor;
+  if (const char* dbg = getenv("FACT_DEBUG_FLAGS")) h->debug_flags = atoi(dbg);
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -513,7 +517,8 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
     return FACT_ERR_CUDA;
   }
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess || cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) {
+  if (cudaMalloc(&h->d_status, 8 * sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->d_status, 0, 8 * sizeof(int)) != cudaSuccess) {
     delete h;
     return FACT_ERR_CUDA;
   }
@@ -538,6 +543,16 @@ fact_status_t fact_device_info(fact_handle_t h, int* sm_count, int* max_smem, in
 }
 
 int64_t fact_launch_count(fact_handle_t h) { return h ? h->launches : 0; }
+
+fact_status_t fact_last_kernel_clock(fact_handle_t h, void* stream, int64_t* sm_cycles, int64_t* nanoseconds) {
+  if (!h || !sm_cycles || !nanoseconds) return FACT_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return FACT_ERR_CUDA;
+  long long v[2] = {0, 0};
+  if (cudaMemcpy(v, h->d_status + 2, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
+  *sm_cycles = v[0];
+  *nanoseconds = v[1];
+  return FACT_OK;
+}
 
 const char* fact_last_error(fact_handle_t h) { return h ? h->last_error.c_str() : ""; }
 

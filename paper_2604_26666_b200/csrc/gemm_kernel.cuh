@@ -3,8 +3,8 @@
 //
 // One CTA (or a 2-CTA cluster when CG == 2) walks a static list of work units
 // (batch, m-tile, n-tile, k-slice).  Three roles run concurrently:
-//   warp 0     TMA producer: fills a ring of shared-memory stages with 128B-swizzled
-//              A (128 x 64) and B (tile_n x 64) tiles, signalling `full` mbarriers
+//   warps 0, 6 TMA producers (A tiles / B tiles): fill a ring of shared-memory stages with
+//              128B-swizzled A (128 x 64) and B (tile_n x 64) tiles, signalling `full` mbarriers
 //   warp 1     MMA issuer: one thread issues tcgen05.mma (UMMA K = 16, four per stage)
 //              into one of two FP32 accumulators in tensor memory, releasing stages
 //              through tcgen05.commit -> `empty`, and publishing a finished accumulator
@@ -29,7 +29,8 @@ constexpr int kMaxStages = 8;
 constexpr int kTileM = 128;       // rows per CTA (= TMEM lanes)
 constexpr int kTileK = 64;        // BF16 elements per 128-byte swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma.kind::f16
-constexpr int kThreads = 192;     // 6 warps: producer, MMA, 4 x epilogue
+constexpr int kThreads = 224;     // 7 warps: A producer, MMA, 4 x epilogue, B producer
+constexpr int kProducerBWarp = 6;
 constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
@@ -79,6 +80,9 @@ struct GemmParams {
   float* ws;
   long long ws_ld, ws_batch_stride, ws_split_stride;
   int* status;
+  // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
+  // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
+  int debug;
 };
 
 struct WorkUnit {
@@ -217,7 +221,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   __shared__ uint32_t tmem_holder;
   __shared__ int abort_flag;
 
-  const int warp = threadIdx.x >> 5;
+  // The warp index is made provably warp-uniform (a shuffle result), and the producer / MMA roles
+  // run their loops with all 32 lanes converged, electing one lane only for the instruction that
+  // must be issued once.  Loop state then lives in uniform registers; running the whole loop in a
+  // single divergent lane instead costs ~80 cycles per tcgen05/TMA instruction and starves the
+  // tensor pipe.
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -256,53 +265,79 @@ __global__ void __launch_bounds__(kThreads, 1)
   ptx::tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_holder);
 
+  // CTA 0 stamps the SM cycle counter and the nanosecond timer around its work (status[2..5]):
+  // their ratio is the SM clock this launch really ran at.
+  long long t_clk0 = 0;
+  unsigned long long t_ns0 = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    t_clk0 = clock64();
+    t_ns0 = ptx::globaltimer_ns();
+  }
   const int unit0 = (int)(blockIdx.x / CG);
   const int unit_stride = (int)(gridDim.x / CG);
   volatile int* abort_p = &abort_flag;
+  // a bounded wait whose verdict is warp-uniform
+  auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+    return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_p, p.status)) != 0;
+  };
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+  if (warp == 0 || warp == kProducerBWarp) {
+    // ------------------------------------------------------------ TMA producers
+    // Warp 0 loads the A tiles (and posts the expected byte count), warp 6 the B boxes.
+    const bool do_a = warp == 0;
+    if (!(p.debug & 1)) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
         const WorkUnit w = decode_unit(p, u);
         const int m0 = (w.tm * CG + (int)cta_rank) * kTileM;
-        // first accumulator column this CTA's B boxes feed
+        // first accumulator column this CTA's B boxes feed, and the W column of every box
         const int col0 = (CG == 2) ? (int)cta_rank * (p.tile_n / 2) : 0;
+        int n_box[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int col = col0 + i * p.b_box_n;
+          if (p.gate) {
+            const int half = p.tile_n >> 1;
+            n_box[i] = (col < half) ? (w.tn * half + col) : (p.N_out + w.tn * half + (col - half));
+          } else {
+            n_box[i] = w.tn * p.tile_n + col;
+          }
+        }
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
-          if (!wait_bar(empty_bar(stage), phase ^ 1u, abort_p, p.status)) {
+          if (!wait_all(empty_bar(stage), phase ^ 1u)) {
             ok = false;
             break;
           }
           const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
           const uint32_t sb = sa + kStageBytesA;
           uint32_t fb = full_bar(stage);
-          if constexpr (CG == 2) {
-            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-            fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
-            ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
-          } else {
-            ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-            ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
-          }
-          for (int i = 0; i < p.b_loads; ++i) {
-            const int col = col0 + i * p.b_box_n;  // accumulator column of this box
-            int n;
-            if (p.gate) {
-              const int half = p.tile_n >> 1;
-              n = (col < half) ? (w.tn * half + col) : (p.N_out + w.tn * half + (col - half));
+          if (ptx::elect_one()) {
+            if (do_a) {
+              if constexpr (CG == 2) {
+                if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
+                fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
+                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
+              } else {
+                ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
+                ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+              }
             } else {
-              n = w.tn * p.tile_n + col;
-            }
-            const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
-            if constexpr (CG == 2) {
-              if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n, kb * kTileK, w.b);
-              else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n, w.b);
-            } else {
-              if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n, kb * kTileK, w.b);
-              else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n, w.b);
+              if constexpr (CG == 2) fb = ptx::mapa(fb, 0);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                if (i < p.b_loads) {
+                  const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
+                  if constexpr (CG == 2) {
+                    if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n_box[i], kb * kTileK, w.b);
+                    else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n_box[i], w.b);
+                  } else {
+                    if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n_box[i], kb * kTileK, w.b);
+                    else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n_box[i], w.b);
+                  }
+                }
+              }
             }
           }
           if (++stage == p.stages) {
@@ -313,8 +348,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
       // Drain: wait until every stage this CTA filled has been released, so that no
       // commit arrival is still on its way to this CTA's barriers when it exits.
-      for (int s = 0; ok && s < p.stages; ++s) {
-        if (!wait_bar(empty_bar(stage), phase ^ 1u, abort_p, p.status)) ok = false;
+      for (int s = 0; ok && do_a && s < p.stages; ++s) {
+        if (!wait_all(empty_bar(stage), phase ^ 1u)) ok = false;
         if (++stage == p.stages) {
           stage = 0;
           phase ^= 1u;
@@ -324,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0 && cta_rank == 0) {
+    if (cta_rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -332,14 +367,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
         const WorkUnit w = decode_unit(p, u);
-        if (!wait_bar(acce_bar(acc), acc_phase ^ 1u, abort_p, p.status)) {
+        if (!wait_all(acce_bar(acc), acc_phase ^ 1u)) {
           ok = false;
           break;
         }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tile_n);
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
-          if (!wait_bar(full_bar(stage), phase, abort_p, p.status)) {
+          if (!(p.debug & 1) && !wait_all(full_bar(stage), phase)) {
             ok = false;
             break;
           }
@@ -348,22 +383,28 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint32_t sb = sa + kStageBytesA;
           const uint64_t adesc = p.a_desc | (uint64_t)((sa >> 4) & 0x3fffu);
           const uint64_t bdesc = p.b_desc | (uint64_t)((sb >> 4) & 0x3fffu);
+          if (ptx::elect_one()) {
+            if (!(p.debug & 2)) {
 #pragma unroll
-          for (int k = 0; k < kTileK / kUmmaK; ++k) {
-            ptx::umma_bf16<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
-                               p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+              for (int k = 0; k < kTileK / kUmmaK; ++k) {
+                ptx::umma_bf16<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
+                                   p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+              }
+            }
+            // release the stage (in both CTAs of a pair) once these MMAs have read it
+            if constexpr (CG == 2) ptx::umma_commit_pair(empty_bar(stage), 0x3);
+            else ptx::umma_commit<CG>(empty_bar(stage));
           }
-          // release the stage (in both CTAs of a pair) once these MMAs have read it
-          if constexpr (CG == 2) ptx::umma_commit_pair(empty_bar(stage), 0x3);
-          else ptx::umma_commit<CG>(empty_bar(stage));
           if (++stage == p.stages) {
             stage = 0;
             phase ^= 1u;
           }
         }
         if (!ok) break;
-        if constexpr (CG == 2) ptx::umma_commit_pair(accf_bar(acc), 0x3);
-        else ptx::umma_commit<CG>(accf_bar(acc));
+        if (ptx::elect_one()) {
+          if constexpr (CG == 2) ptx::umma_commit_pair(accf_bar(acc), 0x3);
+          else ptx::umma_commit<CG>(accf_bar(acc));
+        }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -435,7 +476,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               if (row_ok) load_bf16x8(r_row + n, nvalid, p.r_vec != 0, res);
             }
             apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
-            if (row_ok) {
+            if (row_ok && !(p.debug & 4)) {
               if (EPI == kEpiPartial || p.out_f32)
                 store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid,
                             EPI == kEpiPartial ? ((n & 3) == 0) : c_vec);
@@ -465,6 +506,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    long long* stamp = reinterpret_cast<long long*>(p.status + 2);
+    stamp[0] = clock64() - t_clk0;
+    stamp[1] = (long long)(ptx::globaltimer_ns() - t_ns0);
+  }
   if constexpr (CG == 2) {  // neither CTA may free tensor memory or exit while its peer still uses it
     ptx::cluster_arrive();
     ptx::cluster_wait();
