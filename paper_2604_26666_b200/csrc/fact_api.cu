@@ -97,9 +97,12 @@ uint32_t pow2_at_least(uint32_t x) {
 int stage_bytes_for(int tile_n, int cta_group) { return (int)kStageBytesA + (tile_n / cta_group) * kTileK * 2; }
 
 int max_stages_for(int tile_n, int cta_group) {
-  int s = (kSmemBudget - kSmemSlack) / stage_bytes_for(tile_n, cta_group);
+  int s = (kSmemBudget - kSmemSlack - (int)kEpiSmemBytes) / stage_bytes_for(tile_n, cta_group);
   return std::min(s, kMaxStages);
 }
+
+long long ws_ld_for(const Problem& q) { return round_up((int)q.N_out, 4); }
+int ws_planes_for(const Problem& q) { return q.epi == FACT_EPI_SILU_GATE ? 2 : 1; }
 
 // Is (tile_n, cta_group) runnable for this problem's layout / epilogue?
 bool tile_ok(const Problem& q, int tile_n, int cg) {
@@ -164,8 +167,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   }
   if (c.split_k < 1) return FACT_ERR_INVALID_ARG;
   c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
-  if (c.store_mode == 0) c.store_mode = 1;
-  if (c.store_mode != 1) return FACT_ERR_UNSUPPORTED;
+  if (c.store_mode < 0 || c.store_mode > 2) return FACT_ERR_INVALID_ARG;
   *out = c;
   return FACT_OK;
 }
@@ -208,8 +210,8 @@ fact_status_t validate(const Problem& q) {
 
 size_t workspace_for(const Problem& q, const fact_config_t& c) {
   if (c.split_k <= 1) return 0;
-  const long long ws_ld = round_up((int)q.Nw(), 4);
-  return (size_t)c.split_k * (size_t)q.batch * (size_t)q.M * (size_t)ws_ld * sizeof(float);
+  return (size_t)c.split_k * (size_t)q.batch * (size_t)ws_planes_for(q) * (size_t)q.M * (size_t)ws_ld_for(q) *
+         sizeof(float);
 }
 
 uint64_t smem_desc_template(uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -290,27 +292,39 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.ldr = q.ldr;
   p.strideR = q.strideR;
   p.r_vec = q.R && aligned16(q.R) && (q.ldr % 8 == 0) && (q.batch <= 1 || q.strideR % 8 == 0);
-  p.ws_ld = round_up(p.Nw, 4);
-  p.ws_batch_stride = (long long)p.M * p.ws_ld;
-  p.ws_split_stride = p.ws_batch_stride * p.batch;
+  p.ws_ld = ws_ld_for(q);
+  p.ws_planes = ws_planes_for(q);
+  // Staged TMA stores need a 16-byte aligned output whose rows are 16-byte multiples, whole 128-byte chunks per
+  // tile, and (for a residual) a BF16 output; anything else is stored directly from registers.
+  const int chunk_cols = p.out_f32 ? 32 : 64;
+  const bool can_stage = p.c_vec && (p.out_cols % chunk_cols == 0) &&
+                         !(p.out_f32 && q.epi == FACT_EPI_BIAS_RESIDUAL);
+  if (c.store_mode == 2 && !can_stage) return FACT_ERR_UNSUPPORTED;
+  p.store_tma = (c.store_mode == 1) ? 0 : (can_stage ? 1 : 0);
+  p.r_tma = p.store_tma && q.epi == FACT_EPI_BIAS_RESIDUAL && p.r_vec;
+  plan->cfg.store_mode = p.store_tma ? 2 : 1;
   p.status = h->d_status;
   p.debug = h->debug_flags;
   plan->ws_bytes = workspace_for(q, c);
-  plan->smem_bytes = std::max(c.stages * (int)p.stage_bytes + kSmemSlack, kMinSmemRequest);
+  plan->smem_bytes = std::max(c.stages * (int)p.stage_bytes + kSmemSlack + (int)kEpiSmemBytes, kMinSmemRequest);
   if (plan->smem_bytes > kSmemBudget || kSmemBudget + 1024 > h->max_smem) return FACT_ERR_UNSUPPORTED;
   const int slots = std::max(1, h->sm_count / cg);
   plan->grid = (int)std::min<long long>(slots, units) * cg;
   return FACT_OK;
 }
 
+// A rank-3 tensor map (inner, rows, batch) with a (box0 x box1 x 1) box and 128-byte swizzle.
 fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
-                         uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1) {
+                         uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1,
+                         bool f32 = false) {
+  const uint64_t esz = f32 ? 4 : 2;
   cuuint64_t dims[3] = {d0, d1, d2};
-  cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
+  cuuint64_t strides[2] = {stride1_elems * esz, stride2_elems * esz};
   cuuint32_t box[3] = {box0, box1, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  CUresult r = h->encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     h->last_error = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string((int)r);
@@ -320,8 +334,8 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
 }
 
 template <int CG, int EPI>
-fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap& tmA,
-                              const CUtensorMap& tmB, cudaStream_t stream) {
+fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
+                              cudaStream_t stream) {
   auto kern = fact_gemm_kernel<CG, EPI>;
   if (!(h->configured_mask & (1u << slot))) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -343,24 +357,23 @@ fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const
     lc.attrs = attr;
     lc.numAttrs = 1;
   }
-  cudaError_t e = cudaLaunchKernelEx(&lc, kern, tmA, tmB, plan.p);
+  cudaError_t e = cudaLaunchKernelEx(&lc, kern, tm[0], tm[1], tm[2], tm[3], plan.p);
   if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx", e);
   h->launches++;
   return FACT_OK;
 }
 
 template <int CG>
-fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                         cudaStream_t stream) {
+fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
   const int base = (CG - 1) * 8;
   switch (epi) {
-    case kEpiNone: return launch_instance<CG, kEpiNone>(h, base + 0, plan, tmA, tmB, stream);
-    case kEpiBias: return launch_instance<CG, kEpiBias>(h, base + 1, plan, tmA, tmB, stream);
-    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu>(h, base + 2, plan, tmA, tmB, stream);
-    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh>(h, base + 3, plan, tmA, tmB, stream);
-    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate>(h, base + 4, plan, tmA, tmB, stream);
-    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual>(h, base + 5, plan, tmA, tmB, stream);
-    case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tmA, tmB, stream);
+    case kEpiNone: return launch_instance<CG, kEpiNone>(h, base + 0, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias>(h, base + 1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu>(h, base + 2, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh>(h, base + 3, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate>(h, base + 4, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual>(h, base + 5, plan, tm, stream);
+    case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tm, stream);
     default: return FACT_ERR_INVALID_ARG;
   }
 }
@@ -371,8 +384,7 @@ fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan,
   memset(&r, 0, sizeof r);
   r.ws = ws;
   r.ws_ld = plan.p.ws_ld;
-  r.ws_batch_stride = plan.p.ws_batch_stride;
-  r.ws_split_stride = plan.p.ws_split_stride;
+  r.planes = plan.p.ws_planes;
   r.splits = splits;
   r.M = plan.p.M;
   r.N_out = plan.p.N_out;
@@ -416,9 +428,13 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     if (split) {
       if (!ws || ws_bytes < plan.ws_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
       if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
-      plan.p.ws = reinterpret_cast<float*>(ws);
+      plan.p.store_tma = 1;  // partials always go through the staged path: the workspace layout is the library's
+      plan.p.r_tma = 0;
     }
-    CUtensorMap tmA, tmB;
+    CUtensorMap tm[4];  // A, B, output (or split-K workspace), residual
+    CUtensorMap& tmA = tm[0];
+    CUtensorMap& tmB = tm[1];
+    memset(tm, 0, sizeof tm);
     const uint64_t batch_dim = (uint64_t)q.batch;
     const uint64_t sA = q.batch > 1 ? (uint64_t)q.strideA : (uint64_t)q.lda * (uint64_t)q.M;
     st = encode_map(h, &tmA, q.A, (uint64_t)q.K, (uint64_t)q.M, batch_dim, (uint64_t)q.lda, std::max<uint64_t>(sA, 8),
@@ -434,10 +450,30 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
                       std::max<uint64_t>(sB, 8), kTileK, (uint32_t)plan.p.b_box_n);
     }
     if (st != FACT_OK) return st;
+    if (split) {
+      // FP32 partial planes: (ws_ld, M, splits * batch * planes), stored 32 columns x 32 rows at a time
+      const uint64_t planes = (uint64_t)plan.cfg.split_k * q.batch * plan.p.ws_planes;
+      st = encode_map(h, &tm[2], ws, (uint64_t)plan.p.ws_ld, (uint64_t)q.M, planes, (uint64_t)plan.p.ws_ld,
+                      (uint64_t)plan.p.ws_ld * (uint64_t)q.M, 32, 32, true);
+      if (st != FACT_OK) return st;
+    } else if (plan.p.store_tma) {
+      const bool f32 = q.out == FACT_OUT_F32;
+      const uint64_t sC = q.batch > 1 ? (uint64_t)q.strideC : (uint64_t)q.ldc * (uint64_t)q.M;
+      st = encode_map(h, &tm[2], q.C, (uint64_t)q.N_out, (uint64_t)q.M, batch_dim, (uint64_t)q.ldc,
+                      std::max<uint64_t>(sC, 8), f32 ? 32 : 64, 32, f32);
+      if (st != FACT_OK) return st;
+      if (plan.p.r_tma) {
+        const uint64_t sR = q.batch > 1 ? (uint64_t)q.strideR : (uint64_t)q.ldr * (uint64_t)q.M;
+        st = encode_map(h, &tm[3], q.R, (uint64_t)q.N_out, (uint64_t)q.M, batch_dim, (uint64_t)q.ldr,
+                        std::max<uint64_t>(sR, 8), 64, 32, false);
+        if (st != FACT_OK) return st;
+      }
+    }
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
-    if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tmA, tmB, stream);
-    else st = launch_epi<1>(h, epi, plan, tmA, tmB, stream);
-    if (st == FACT_OK && split) st = launch_reduce(h, q, plan, plan.cfg.split_k, plan.p.ws, stream);
+    if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
+    else st = launch_epi<1>(h, epi, plan, tm, stream);
+    if (st == FACT_OK && split)
+      st = launch_reduce(h, q, plan, plan.cfg.split_k, reinterpret_cast<const float*>(ws), stream);
   }
   if (dev != h->device) cudaSetDevice(dev);
   return st;

@@ -2,16 +2,19 @@
 // split-K reduction kernel.
 //
 // One CTA (or a 2-CTA cluster when CG == 2) walks a static list of work units
-// (batch, m-tile, n-tile, k-slice).  Three roles run concurrently:
+// (batch, m-tile, n-tile, k-slice).  Roles run concurrently:
 //   warps 0, 6 TMA producers (A tiles / B tiles): fill a ring of shared-memory stages with
 //              128B-swizzled A (128 x 64) and B (tile_n x 64) tiles, signalling `full` mbarriers
-//   warp 1     MMA issuer: one thread issues tcgen05.mma (UMMA K = 16, four per stage)
-//              into one of two FP32 accumulators in tensor memory, releasing stages
-//              through tcgen05.commit -> `empty`, and publishing a finished accumulator
-//              through tcgen05.commit -> `acc_full`
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (one output row per thread), apply
-//              the fused element-wise operation in FP32, round once, store; then hand
-//              the accumulator back (`acc_empty`) so the next tile's main loop overlaps
+//   warp 1     MMA issuer: issues tcgen05.mma (UMMA K = 16, four per stage) into one of two
+//              FP32 accumulators in tensor memory, releasing stages through
+//              tcgen05.commit -> `empty`, and publishing a finished accumulator through
+//              tcgen05.commit -> `acc_full`
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (one output row per thread), apply the
+//              fused element-wise operation in FP32, round once, and store -- either through
+//              128-byte-swizzled shared-memory staging and TMA tensor stores (residual tiles
+//              arrive the same way, by TMA loads), or directly from registers when the output
+//              is not 16-byte aligned; then hand the accumulator back (`acc_empty`) so the
+//              next tile's main loop overlaps
 // Every mbarrier wait is bounded in time; an expired wait records
 // FACT_ERR_DEVICE_TIMEOUT in the status word, all roles leave their loops, tensor
 // memory is released and the kernel returns.
@@ -33,6 +36,13 @@ constexpr int kThreads = 224;     // 7 warps: A producer, MMA, 4 x epilogue, B p
 constexpr int kProducerBWarp = 6;
 constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+// Epilogue staging in shared memory, per epilogue warp: three 32-row x 128-byte buffers that
+// rotate (residual tile in, result tile out) and 256 FP32 bias values.
+constexpr int kEpiBufs = 3;
+constexpr uint32_t kEpiBufBytes = 32 * 128;
+constexpr uint32_t kEpiBiasBytes = 256 * 4;
+constexpr uint32_t kEpiSmemBytes = 4 * (kEpiBufs * kEpiBufBytes + kEpiBiasBytes);
 
 // Epilogue selector of the kernel: the public enum plus the split-K partial store.
 enum : int {
@@ -71,14 +81,17 @@ struct GemmParams {
   void* C;
   long long ldc, strideC;
   int out_f32, c_vec;
+  int store_tma;  // 1: staged shared memory + TMA tensor stores (tmC); 0: direct register stores
+  int r_tma;      // 1: residual tiles come in by TMA (tmR); 0: direct loads
   const __nv_bfloat16* bias;
   int bias_vec;
   const __nv_bfloat16* R;
   long long ldr, strideR;
   int r_vec;
-  // split-K partials: ws[split][batch][M][ws_ld] FP32
-  float* ws;
-  long long ws_ld, ws_batch_stride, ws_split_stride;
+  // split-K partials, FP32: ws[(split * batch + b) * ws_planes + plane][M][ws_ld];
+  // plane 1 holds the "up" columns of a gated accumulator
+  int ws_planes;
+  long long ws_ld;
   int* status;
   // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
   // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
@@ -189,6 +202,11 @@ __device__ __forceinline__ float gelu_tanh_f32(float z) {
 }
 __device__ __forceinline__ float silu_f32(float g) { return __fdividef(g, 1.f + __expf(-g)); }
 
+template <int EPI>
+constexpr bool epi_has_bias() {
+  return EPI == kEpiBias || EPI == kEpiBiasRelu || EPI == kEpiBiasGeluTanh || EPI == kEpiBiasResidual;
+}
+
 // The fused element-wise operation on 8 consecutive output columns.
 template <int EPI>
 __device__ __forceinline__ void apply_epilogue8(const uint32_t* acc, const uint32_t* acc_up, const float (&bias)[8],
@@ -215,9 +233,10 @@ __device__ __forceinline__ void apply_epilogue8(const uint32_t* acc, const uint3
 template <int CG, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
                      const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_mem[2 * kMaxStages + 4];
+  __shared__ __align__(8) uint64_t bar_mem[2 * kMaxStages + 4 + 4 * kEpiBufs];
   __shared__ uint32_t tmem_holder;
   __shared__ int abort_flag;
 
@@ -235,6 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
   auto accf_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + b); };
   auto acce_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 2 + b); };
+  auto res_bar = [&](int q, int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 4 + q * kEpiBufs + b); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
@@ -245,6 +265,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       ptx::mbar_init(accf_bar(b), 1);
       ptx::mbar_init(acce_bar(b), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
     }
+    for (int q = 0; q < 4; ++q)
+      for (int b = 0; b < kEpiBufs; ++b) ptx::mbar_init(res_bar(q, b), 1);
     abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -416,84 +438,212 @@ __global__ void __launch_bounds__(kThreads, 1)
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    const bool c_vec = p.c_vec != 0;
-    for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
-      const WorkUnit w = decode_unit(p, u);
-      if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
-        ok = false;
-        break;
-      }
-      ptx::tc_fence_after();
-      const int row = (w.tm * CG + (int)cta_rank) * kTileM + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
-      const int n_tile0 = w.tn * p.out_cols;
-      // destination row
-      char* c_row;
-      if constexpr (EPI == kEpiPartial) {
-        c_row = reinterpret_cast<char*>(p.ws + (long long)w.split * p.ws_split_stride +
-                                        (long long)w.b * p.ws_batch_stride + (long long)row * p.ws_ld);
-      } else {
-        const long long off = (long long)w.b * p.strideC + (long long)row * p.ldc;
-        c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
-      }
-      const __nv_bfloat16* r_row = nullptr;
-      if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
-
-      // A split-K partial stores every accumulator column; a gated accumulator holds the gate
-      // columns in its first half and the up columns (N_out further right in W) in its second.
-      const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
-      for (int c = 0; c < acc_cols; c += 32) {
-        int n0 = n_tile0 + c;
-        int n_limit = p.N_out;
-        if (EPI == kEpiPartial && p.gate) {
-          const int half = p.tile_n >> 1;
-          const int g0 = w.tn * half + (c < half ? c : c - half);
-          if (g0 >= p.N_out) continue;  // uniform across the warp
-          n0 = (c < half) ? g0 : p.N_out + g0;
-          n_limit = (c < half) ? p.N_out : 2 * p.N_out;
-        } else if (n0 >= p.N_out) {
-          break;  // uniform across the warp
+    if (p.store_tma) {
+      // ---- staged: registers -> swizzled shared memory -> TMA tensor store, 32 rows x 128 bytes at a time
+      const uint32_t epi_base = smem_base + (uint32_t)p.stages * p.stage_bytes;
+      const uint32_t stg0 = epi_base + (uint32_t)q * (kEpiBufs * kEpiBufBytes);
+      const uint32_t bias_s = epi_base + 4u * kEpiBufs * kEpiBufBytes + (uint32_t)q * kEpiBiasBytes;
+      const bool f32 = (EPI == kEpiPartial) || (p.out_f32 != 0);
+      const int chunk_cols = f32 ? 32 : 64;               // 128 bytes of output per row
+      const bool use_r = (EPI == kEpiBiasResidual) && p.r_tma;
+      const uint32_t my_row = (uint32_t)lane * 128u;      // this thread's row inside a staging buffer
+      const uint32_t swz = (uint32_t)(lane & 7);          // 128-byte swizzle: 16-byte chunk j lives at j ^ (row & 7)
+      uint32_t gc = 0;                                    // chunks issued so far: buffer = gc % kEpiBufs
+      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+        const WorkUnit w = decode_unit(p, u);
+        const int row0 = (w.tm * CG + (int)cta_rank) * kTileM + q * 32;
+        const int n_tile0 = w.tn * p.out_cols;
+        const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
+        // The coordinates of chunk `ci`: first column, plane / batch coordinate, whether it exists.
+        auto chunk_coord = [&](int ci, int& n, int& z) -> bool {
+          const int c = ci * chunk_cols;
+          if (EPI == kEpiPartial) {
+            int plane = 0;
+            if (p.gate) {
+              const int half = p.tile_n >> 1;
+              plane = c >= half;
+              n = w.tn * half + (c - plane * half);
+            } else {
+              n = w.tn * p.tile_n + c;
+            }
+            z = (w.split * p.batch + w.b) * p.ws_planes + plane;
+          } else {
+            n = n_tile0 + c;
+            z = w.b;
+          }
+          return c < acc_cols && n < p.N_out;
+        };
+        auto issue_residual = [&](int ci, uint32_t g) {
+          int n, z;
+          if (chunk_coord(ci, n, z) && lane == 0) {
+            ptx::bulk_wait_group_read<1>();  // the store that last read this buffer is done with it
+            const uint32_t rb = res_bar(q, (int)(g % kEpiBufs));
+            ptx::mbar_arrive_expect_tx(rb, kEpiBufBytes);
+            ptx::tma_load_3d(stg0 + (g % kEpiBufs) * kEpiBufBytes, &tmR, rb, n, row0, z);
+          }
+        };
+        // this tile's bias slice, as FP32, into the warp's own shared-memory copy
+        if constexpr (epi_has_bias<EPI>()) {
+          __syncwarp();
+          float bv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          const int nb = n_tile0 + lane * 8;
+          if (p.bias != nullptr && lane * 8 < p.out_cols && nb < p.N_out)
+            load_bf16x8(p.bias + nb, min(8, p.N_out - nb), p.bias_vec != 0, bv);
+          ptx::st_shared_v4(bias_s + (uint32_t)lane * 32u, __float_as_uint(bv[0]), __float_as_uint(bv[1]),
+                            __float_as_uint(bv[2]), __float_as_uint(bv[3]));
+          ptx::st_shared_v4(bias_s + (uint32_t)lane * 32u + 16u, __float_as_uint(bv[4]), __float_as_uint(bv[5]),
+                            __float_as_uint(bv[6]), __float_as_uint(bv[7]));
+          __syncwarp();
         }
-        uint32_t v[32];
-        uint32_t vu[32];
-        ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
-        if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
-        ptx::tmem_wait_ld();
+        if (use_r) issue_residual(0, gc);
+        if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+        const int n_chunks = acc_cols / chunk_cols;
+        for (int ci = 0; ci < n_chunks; ++ci) {
+          int n_chunk, z;
+          if (!chunk_coord(ci, n_chunk, z)) continue;  // uniform across the warp
+          const uint32_t buf = stg0 + (gc % kEpiBufs) * kEpiBufBytes;
+          if (use_r) {
+            if (ci + 1 < n_chunks) issue_residual(ci + 1, gc + 1);
+            if (!wait_bar(res_bar(q, (int)(gc % kEpiBufs)), (gc / kEpiBufs) & 1u, abort_p, p.status)) {
+              ok = false;
+              break;
+            }
+          } else {
+            if (lane == 0) ptx::bulk_wait_group_read<kEpiBufs - 1>();
+            __syncwarp();
+          }
+#pragma unroll 1
+          for (int piece = 0; piece * 32 < chunk_cols; ++piece) {
+            const int c = ci * chunk_cols + piece * 32;  // accumulator column of this 32-wide piece
+            uint32_t v[32];
+            uint32_t vu[32];
+            ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
+            if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
+            ptx::tmem_wait_ld();
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const int n = n0 + g * 8;
-          const int nvalid = min(8, n_limit - n);
-          float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          float y[8];
-          if (nvalid > 0) {
-            if constexpr (EPI == kEpiBias || EPI == kEpiBiasRelu || EPI == kEpiBiasGeluTanh ||
-                          EPI == kEpiBiasResidual) {
-              if (p.bias != nullptr) load_bf16x8(p.bias + n, nvalid, p.bias_vec != 0, bias);
+            for (int g = 0; g < 4; ++g) {
+              float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+              float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+              float y[8];
+              if constexpr (epi_has_bias<EPI>()) {
+                const uint4 b0 = ptx::ld_shared_v4(bias_s + (uint32_t)(c + g * 8) * 4u);
+                const uint4 b1 = ptx::ld_shared_v4(bias_s + (uint32_t)(c + g * 8) * 4u + 16u);
+                bias[0] = __uint_as_float(b0.x); bias[1] = __uint_as_float(b0.y);
+                bias[2] = __uint_as_float(b0.z); bias[3] = __uint_as_float(b0.w);
+                bias[4] = __uint_as_float(b1.x); bias[5] = __uint_as_float(b1.y);
+                bias[6] = __uint_as_float(b1.z); bias[7] = __uint_as_float(b1.w);
+              }
+              if (f32) {
+                apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
+                const uint32_t j0 = (uint32_t)(2 * g), j1 = j0 + 1u;
+                ptx::st_shared_v4(buf + my_row + ((j0 ^ swz) << 4), __float_as_uint(y[0]), __float_as_uint(y[1]),
+                                  __float_as_uint(y[2]), __float_as_uint(y[3]));
+                ptx::st_shared_v4(buf + my_row + ((j1 ^ swz) << 4), __float_as_uint(y[4]), __float_as_uint(y[5]),
+                                  __float_as_uint(y[6]), __float_as_uint(y[7]));
+              } else {
+                const uint32_t j = (uint32_t)(piece * 4 + g);
+                const uint32_t addr = buf + my_row + ((j ^ swz) << 4);
+                if constexpr (EPI == kEpiBiasResidual) {
+                  if (use_r) {
+                    const uint4 rq = ptx::ld_shared_v4(addr);
+                    unpack_bf16x8(rq, res);
+                  } else {
+                    const int row = row0 + lane;
+                    const int n = n_chunk + piece * 32 + g * 8;
+                    if (row < p.M && n < p.N_out)
+                      load_bf16x8(p.R + (long long)z * p.strideR + (long long)row * p.ldr + n, min(8, p.N_out - n),
+                                  p.r_vec != 0, res);
+                  }
+                }
+                apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
+                ptx::st_shared_v4(addr, pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]),
+                                  pack_bf16x2(y[6], y[7]));
+              }
             }
-            if constexpr (EPI == kEpiBiasResidual) {
-              if (row_ok) load_bf16x8(r_row + n, nvalid, p.r_vec != 0, res);
-            }
-            apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
-            if (row_ok && !(p.debug & 4)) {
-              if (EPI == kEpiPartial || p.out_f32)
-                store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid,
-                            EPI == kEpiPartial ? ((n & 3) == 0) : c_vec);
-              else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (row0 < p.M && !(p.debug & 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
+            ptx::bulk_commit_group();
+          }
+          ++gc;
+        }
+        if (!ok) break;
+        // hand the accumulator back to the MMA issuer (of the leader CTA)
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(acce_bar(acc), 0));
+          else ptx::mbar_arrive(acce_bar(acc));
+        }
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+      if (lane == 0) ptx::bulk_wait_group<0>();  // every store has left shared memory and reached global memory
+      __syncwarp();
+    } else {
+      // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
+      const bool c_vec = p.c_vec != 0;
+      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+        const WorkUnit w = decode_unit(p, u);
+        if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        const int row = (w.tm * CG + (int)cta_rank) * kTileM + q * 32 + lane;
+        const bool row_ok = row < p.M;
+        const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+        const int n_tile0 = w.tn * p.out_cols;
+        const long long off = (long long)w.b * p.strideC + (long long)row * p.ldc;
+        char* c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
+        const __nv_bfloat16* r_row = nullptr;
+        if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
+        for (int c = 0; c < p.out_cols; c += 32) {
+          const int n0 = n_tile0 + c;
+          if (n0 >= p.N_out) break;  // uniform across the warp
+          uint32_t v[32];
+          uint32_t vu[32];
+          ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
+          if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int n = n0 + g * 8;
+            const int nvalid = min(8, p.N_out - n);
+            float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float y[8];
+            if (nvalid > 0) {
+              if constexpr (epi_has_bias<EPI>()) {
+                if (p.bias != nullptr) load_bf16x8(p.bias + n, nvalid, p.bias_vec != 0, bias);
+              }
+              if constexpr (EPI == kEpiBiasResidual) {
+                if (row_ok) load_bf16x8(r_row + n, nvalid, p.r_vec != 0, res);
+              }
+              apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
+              if (row_ok && !(p.debug & 4)) {
+                if (p.out_f32) store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid, c_vec);
+                else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
+              }
             }
           }
         }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(acce_bar(acc), 0));
+          else ptx::mbar_arrive(acce_bar(acc));
+        }
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
       }
-      // hand the accumulator back to the MMA issuer (of the leader CTA)
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(acce_bar(acc), 0));
-        else ptx::mbar_arrive(acce_bar(acc));
-      }
-      acc ^= 1;
-      if (acc == 0) acc_phase ^= 1u;
     }
   }
 
@@ -525,8 +675,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 // Split-K reduction: adds the S partials of every output element in ascending slice order,
 // applies the epilogue and stores.  One thread per 4 consecutive output columns.
 struct ReduceParams {
-  const float* ws;
-  long long ws_ld, ws_batch_stride, ws_split_stride;
+  const float* ws;  // ws[(split * batch + b) * planes + plane][M][ws_ld]
+  long long ws_ld;
+  int planes;
   int splits;
   int M, N_out, batch;
   int epi;
@@ -552,6 +703,7 @@ __device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, flo
 __global__ void __launch_bounds__(256) fact_splitk_reduce_kernel(const ReduceParams p) {
   const long long groups_per_row = (p.N_out + 3) / 4;
   const long long total = (long long)p.batch * p.M * groups_per_row;
+  const long long plane_stride = (long long)p.M * p.ws_ld;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int gcol = (int)(i % groups_per_row);
@@ -561,20 +713,14 @@ __global__ void __launch_bounds__(256) fact_splitk_reduce_kernel(const ReducePar
     const int n = gcol * 4;
     const int nvalid = min(4, p.N_out - n);
     float a[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
-    const float* src = p.ws + (long long)b * p.ws_batch_stride + (long long)m * p.ws_ld + n;
     const bool gate = p.epi == kEpiSiluGate;
-    const bool up_vec = (p.N_out & 3) == 0;
     for (int s = 0; s < p.splits; ++s) {  // ascending slice order: deterministic
-      const float* ps = src + (long long)s * p.ws_split_stride;
-      const float4 v = *reinterpret_cast<const float4*>(ps);  // ws_ld is a multiple of 4: in-bounds padding
+      const float* ps = p.ws + ((long long)(s * p.batch + b) * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
+      const float4 v = *reinterpret_cast<const float4*>(ps);  // ws_ld is a multiple of 4: padding is in bounds
       a[0] += v.x; a[1] += v.y; a[2] += v.z; a[3] += v.w;
       if (gate) {
-        if (up_vec) {
-          const float4 t = *reinterpret_cast<const float4*>(ps + p.N_out);
-          up[0] += t.x; up[1] += t.y; up[2] += t.z; up[3] += t.w;
-        } else {
-          for (int j = 0; j < nvalid; ++j) up[j] += ps[p.N_out + j];
-        }
+        const float4 t = *reinterpret_cast<const float4*>(ps + plane_stride);
+        up[0] += t.x; up[1] += t.y; up[2] += t.z; up[3] += t.w;
       }
     }
     for (int j = 0; j < nvalid; ++j) {
