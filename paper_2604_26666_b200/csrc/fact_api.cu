@@ -25,8 +25,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kSmemBudget = 226 * 1024;  // opt-in shared memory per CTA on sm_100 (227 KB) minus 1 KB for static data
-constexpr int kSmemSlack = 1024;         // room to align the stage ring to 1024 bytes
+constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the whole 227 KB opt-in limit (no static
+                                         // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
 
 // Key of the tuner's table: everything that changes which configuration is best.
@@ -96,9 +96,18 @@ uint32_t pow2_at_least(uint32_t x) {
 // Per-CTA bytes of one pipeline stage.
 int stage_bytes_for(int tile_n, int cta_group) { return (int)kStageBytesA + (tile_n / cta_group) * kTileK * 2; }
 
-int max_stages_for(int tile_n, int cta_group) {
-  int s = (kSmemBudget - kSmemSlack - (int)kEpiSmemBytes) / stage_bytes_for(tile_n, cta_group);
-  return std::min(s, kMaxStages);
+// Staging buffers per epilogue warp: a residual tile that arrives by TMA wants a second buffer to prefetch
+// into, but only short main loops (small K) have no slack to hide that load behind.
+int epi_bufs_for(const Problem& q) { return (q.epi == FACT_EPI_BIAS_RESIDUAL && q.K <= 2048) ? 2 : 1; }
+
+int smem_bytes_for(const Problem& q, int tile_n, int cta_group, int stages) {
+  return stages * stage_bytes_for(tile_n, cta_group) + (int)epi_smem_bytes(epi_bufs_for(q)) + (int)kCtrlSmemBytes;
+}
+
+int max_stages_for(const Problem& q, int tile_n, int cta_group) {
+  int s = kMaxStages;
+  while (s > 0 && smem_bytes_for(q, tile_n, cta_group, s) > kSmemBudget) --s;
+  return s;
 }
 
 long long ws_ld_for(const Problem& q) { return round_up((int)q.N_out, 4); }
@@ -148,7 +157,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     while (c.tile_n > gran && !tile_ok(q, c.tile_n, c.cta_group)) c.tile_n -= gran;
   }
   if (!tile_ok(q, c.tile_n, c.cta_group)) return FACT_ERR_UNSUPPORTED;
-  const int smax = max_stages_for(c.tile_n, c.cta_group);
+  const int smax = max_stages_for(q, c.tile_n, c.cta_group);
   if (c.stages == 0) c.stages = smax;
   if (c.stages < 2 || c.stages > smax) return FACT_ERR_UNSUPPORTED;
   if (c.raster_group == 0) c.raster_group = 8;
@@ -306,8 +315,9 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.status = h->d_status;
   p.debug = h->debug_flags;
   plan->ws_bytes = workspace_for(q, c);
-  plan->smem_bytes = std::max(c.stages * (int)p.stage_bytes + kSmemSlack + (int)kEpiSmemBytes, kMinSmemRequest);
-  if (plan->smem_bytes > kSmemBudget || kSmemBudget + 1024 > h->max_smem) return FACT_ERR_UNSUPPORTED;
+  p.epi_bufs = epi_bufs_for(q);
+  plan->smem_bytes = std::max(smem_bytes_for(q, c.tile_n, cg, c.stages), kMinSmemRequest);
+  if (plan->smem_bytes > kSmemBudget || kSmemBudget > h->max_smem) return FACT_ERR_UNSUPPORTED;
   const int slots = std::max(1, h->sm_count / cg);
   plan->grid = (int)std::min<long long>(slots, units) * cg;
   return FACT_OK;
@@ -690,7 +700,7 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
       if (!tile_ok(q, tn, cg)) continue;
       const int out_cols = epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
       if (out_cols >= 2 * N && tn > 64) continue;  // more than half the tile would be padding
-      const int smax = max_stages_for(tn, cg);
+      const int smax = max_stages_for(q, tn, cg);
       const long long tiles = batch * ((M + 128 * cg - 1) / (128 * cg)) * ((N + out_cols - 1) / out_cols);
       std::vector<int> splits = {1};
       const long long slots = h->sm_count / cg;

@@ -32,17 +32,22 @@ constexpr int kMaxStages = 8;
 constexpr int kTileM = 128;       // rows per CTA (= TMEM lanes)
 constexpr int kTileK = 64;        // BF16 elements per 128-byte swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma.kind::f16
-constexpr int kThreads = 224;     // 7 warps: A producer, MMA, 4 x epilogue, B producer
+constexpr int kThreads = 352;     // 11 warps: A producer, MMA, 4 x epilogue, B producer, 4 x epilogue
 constexpr int kProducerBWarp = 6;
+constexpr int kEpiSetBWarp0 = 7;  // warps 7..10 share the TMEM lane quarters of warps 2..5 (quarter = warp % 4)
 constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
-// Epilogue staging in shared memory, per epilogue warp: three 32-row x 128-byte buffers that
-// rotate (residual tile in, result tile out) and 256 FP32 bias values.
-constexpr int kEpiBufs = 3;
+// Epilogue staging in shared memory, per epilogue warp: one or two 32-row x 128-byte buffers
+// (residual tile in, result tile out) and the BF16 bias values of the 128 columns the warp owns.
+constexpr int kEpiWarps = 8;
+constexpr int kEpiMaxBufs = 2;
 constexpr uint32_t kEpiBufBytes = 32 * 128;
-constexpr uint32_t kEpiBiasBytes = 256 * 4;
-constexpr uint32_t kEpiSmemBytes = 4 * (kEpiBufs * kEpiBufBytes + kEpiBiasBytes);
+constexpr uint32_t kEpiBiasBytes = 128 * 2;
+constexpr uint32_t epi_smem_bytes(int bufs) { return kEpiWarps * ((uint32_t)bufs * kEpiBufBytes + kEpiBiasBytes); }
+// Shared-memory layout (dynamic, 1024-byte aligned): [stage ring][epilogue staging][bias][mbarriers, flags]
+constexpr int kNumBarriers = 2 * kMaxStages + 4 + kEpiWarps * kEpiMaxBufs;
+constexpr uint32_t kCtrlSmemBytes = kNumBarriers * 8 + 16;
 
 // Epilogue selector of the kernel: the public enum plus the split-K partial store.
 enum : int {
@@ -82,6 +87,7 @@ struct GemmParams {
   long long ldc, strideC;
   int out_f32, c_vec;
   int store_tma;  // 1: staged shared memory + TMA tensor stores (tmC); 0: direct register stores
+  int epi_bufs;   // staging buffers per epilogue warp (1 or 2)
   int r_tma;      // 1: residual tiles come in by TMA (tmR); 0: direct loads
   const __nv_bfloat16* bias;
   int bias_vec;
@@ -230,15 +236,50 @@ __device__ __forceinline__ void apply_epilogue8(const uint32_t* acc, const uint3
   }
 }
 
+// The fused element-wise operation on two adjacent output columns, as packed FP32 pairs
+// (add/mul/fma.f32x2 halve the instruction count of the epilogue, which is issue-bound).
+template <int EPI>
+__device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uint64_t bias, uint64_t res) {
+  if constexpr (EPI == kEpiNone || EPI == kEpiPartial) {
+    return acc;
+  } else if constexpr (EPI == kEpiBias) {
+    return ptx::add_f32x2(acc, bias);
+  } else if constexpr (EPI == kEpiBiasRelu) {
+    uint32_t lo, hi;
+    ptx::unpack_f32x2(ptx::add_f32x2(acc, bias), lo, hi);
+    return ptx::pack_f32x2(__float_as_uint(fmaxf(__uint_as_float(lo), 0.f)),
+                           __float_as_uint(fmaxf(__uint_as_float(hi), 0.f)));
+  } else if constexpr (EPI == kEpiBiasGeluTanh) {
+    // z (k0 + k1 z^2) = sqrt(2/pi) (z + 0.044715 z^3);  0.5 z (1 + tanh u) = h + h tanh u with h = 0.5 z
+    const uint64_t k0 = ptx::pack_f32x2(__float_as_uint(0.7978845608028654f), __float_as_uint(0.7978845608028654f));
+    const uint64_t k1 = ptx::pack_f32x2(__float_as_uint(0.7978845608028654f * 0.044715f),
+                                        __float_as_uint(0.7978845608028654f * 0.044715f));
+    const uint64_t half2 = ptx::pack_f32x2(__float_as_uint(0.5f), __float_as_uint(0.5f));
+    const uint64_t z = ptx::add_f32x2(acc, bias);
+    const uint64_t u = ptx::mul_f32x2(ptx::fma_f32x2(ptx::mul_f32x2(z, z), k1, k0), z);
+    uint32_t ulo, uhi;
+    ptx::unpack_f32x2(u, ulo, uhi);
+    const uint64_t t = ptx::pack_f32x2(__float_as_uint(ptx::tanh_approx(__uint_as_float(ulo))),
+                                       __float_as_uint(ptx::tanh_approx(__uint_as_float(uhi))));
+    const uint64_t h = ptx::mul_f32x2(z, half2);
+    return ptx::fma_f32x2(h, t, h);
+  } else if constexpr (EPI == kEpiSiluGate) {
+    uint32_t glo, ghi;
+    ptx::unpack_f32x2(acc, glo, ghi);
+    const uint64_t s = ptx::pack_f32x2(__float_as_uint(silu_f32(__uint_as_float(glo))),
+                                       __float_as_uint(silu_f32(__uint_as_float(ghi))));
+    return ptx::mul_f32x2(s, up);
+  } else {  // kEpiBiasResidual
+    return ptx::add_f32x2(ptx::add_f32x2(acc, bias), res);
+  }
+}
+
 template <int CG, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
                      const GemmParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_mem[2 * kMaxStages + 4 + 4 * kEpiBufs];
-  __shared__ uint32_t tmem_holder;
-  __shared__ int abort_flag;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
 
   // The warp index is made provably warp-uniform (a shuffle result), and the producer / MMA roles
   // run their loops with all 32 lanes converged, electing one lane only for the instruction that
@@ -248,13 +289,24 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
-  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = ptx::smem_u32(bar_mem);
+  const uint32_t smem_base = ptx::smem_u32(smem_raw);
+  if (smem_base & 1023u) {  // the swizzled tiles need a 1024-byte aligned ring: refuse to run otherwise
+    if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+    return;
+  }
+  const uint32_t epi_base = smem_base + (uint32_t)p.stages * p.stage_bytes;
+  const uint32_t bias_base = epi_base + (uint32_t)(kEpiWarps * p.epi_bufs) * kEpiBufBytes;
+  const uint32_t bar_base = bias_base + kEpiWarps * kEpiBiasBytes;
+  const uint32_t ctrl_off = bar_base - smem_base + kNumBarriers * 8;
+  volatile uint32_t* tmem_holder_p = reinterpret_cast<volatile uint32_t*>(smem_raw + ctrl_off);
+  volatile int* abort_p = reinterpret_cast<volatile int*>(smem_raw + ctrl_off + 4);
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
   auto accf_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + b); };
   auto acce_bar = [&](int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 2 + b); };
-  auto res_bar = [&](int q, int b) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 4 + q * kEpiBufs + b); };
+  auto res_bar = [&](int e, int b) {
+    return bar_base + 8u * (uint32_t)(2 * kMaxStages + 4 + e * kEpiMaxBufs + b);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
@@ -263,11 +315,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(accf_bar(b), 1);
-      ptx::mbar_init(acce_bar(b), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
+      ptx::mbar_init(acce_bar(b), kEpiWarps * CG);  // one arrival per epilogue warp of every CTA of the group
     }
-    for (int q = 0; q < 4; ++q)
-      for (int b = 0; b < kEpiBufs; ++b) ptx::mbar_init(res_bar(q, b), 1);
-    abort_flag = 0;
+    for (int e = 0; e < kEpiWarps; ++e)
+      for (int b = 0; b < kEpiMaxBufs; ++b) ptx::mbar_init(res_bar(e, b), 1);
+    *abort_p = 0;
     ptx::fence_mbar_init();
   }
   if (warp == 0 && lane == 0) {
@@ -275,7 +327,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::prefetch_tensormap(&tmB);
   }
   if (warp == 1) {
-    ptx::tmem_alloc<CG>(ptx::smem_u32(&tmem_holder), p.tmem_cols);
+    ptx::tmem_alloc<CG>(smem_base + ctrl_off, p.tmem_cols);
     ptx::tmem_relinquish<CG>();
   }
   ptx::tc_fence_before();
@@ -285,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::cluster_wait();
   }
   ptx::tc_fence_after();
-  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_holder);
+  const uint32_t tmem_base = *tmem_holder_p;
 
   // CTA 0 stamps the SM cycle counter and the nanosecond timer around its work (status[2..5]):
   // their ratio is the SM clock this launch really ran at.
@@ -297,7 +349,6 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   const int unit0 = (int)(blockIdx.x / CG);
   const int unit_stride = (int)(gridDim.x / CG);
-  volatile int* abort_p = &abort_flag;
   // a bounded wait whose verdict is warp-uniform
   auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
     return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_p, p.status)) != 0;
@@ -433,36 +484,41 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;  // the TMEM lane quarter this warp may read
+    // ------------------------------------------------------------ epilogue warps (2..5 and 7..10)
+    // Two warps share each TMEM lane quarter; they take alternate 128-byte column chunks of the tile.
+    const int q = warp & 3;                            // the TMEM lane quarter this warp may read
+    const int half = warp >= kEpiSetBWarp0 ? 1 : 0;    // which of the two warps of the quarter
+    const int e = half * 4 + q;                        // this warp's staging slot
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
     if (p.store_tma) {
       // ---- staged: registers -> swizzled shared memory -> TMA tensor store, 32 rows x 128 bytes at a time
-      const uint32_t epi_base = smem_base + (uint32_t)p.stages * p.stage_bytes;
-      const uint32_t stg0 = epi_base + (uint32_t)q * (kEpiBufs * kEpiBufBytes);
-      const uint32_t bias_s = epi_base + 4u * kEpiBufs * kEpiBufBytes + (uint32_t)q * kEpiBiasBytes;
+      const int bufs = p.epi_bufs;
+      const uint32_t stg0 = epi_base + (uint32_t)(e * bufs) * kEpiBufBytes;
+      const uint32_t bias_s = bias_base + (uint32_t)e * kEpiBiasBytes;
       const bool f32 = (EPI == kEpiPartial) || (p.out_f32 != 0);
       const int chunk_cols = f32 ? 32 : 64;               // 128 bytes of output per row
       const bool use_r = (EPI == kEpiBiasResidual) && p.r_tma;
       const uint32_t my_row = (uint32_t)lane * 128u;      // this thread's row inside a staging buffer
       const uint32_t swz = (uint32_t)(lane & 7);          // 128-byte swizzle: 16-byte chunk j lives at j ^ (row & 7)
-      uint32_t gc = 0;                                    // chunks issued so far: buffer = gc % kEpiBufs
+      uint32_t gc = 0;      // chunks this warp has stored so far: buffer = gc % bufs
+      uint32_t r_next = 0;  // residual loads have been issued for every chunk counter below this
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
         const WorkUnit w = decode_unit(p, u);
         const int row0 = (w.tm * CG + (int)cta_rank) * kTileM + q * 32;
         const int n_tile0 = w.tn * p.out_cols;
         const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
+        const int n_chunks = acc_cols / chunk_cols;
         // The coordinates of chunk `ci`: first column, plane / batch coordinate, whether it exists.
         auto chunk_coord = [&](int ci, int& n, int& z) -> bool {
           const int c = ci * chunk_cols;
           if (EPI == kEpiPartial) {
             int plane = 0;
             if (p.gate) {
-              const int half = p.tile_n >> 1;
-              plane = c >= half;
-              n = w.tn * half + (c - plane * half);
+              const int hw = p.tile_n >> 1;
+              plane = c >= hw;
+              n = w.tn * hw + (c - plane * hw);
             } else {
               n = w.tn * p.tile_n + c;
             }
@@ -471,107 +527,144 @@ __global__ void __launch_bounds__(kThreads, 1)
             n = n_tile0 + c;
             z = w.b;
           }
-          return c < acc_cols && n < p.N_out;
+          return ci < n_chunks && n < p.N_out;
         };
-        auto issue_residual = [&](int ci, uint32_t g) {
+        // Start the TMA load of the residual tile of chunk `ci` into the buffer of chunk counter `g`.
+        auto issue_residual = [&](int ci, uint32_t g) -> bool {
           int n, z;
-          if (chunk_coord(ci, n, z) && lane == 0) {
-            ptx::bulk_wait_group_read<1>();  // the store that last read this buffer is done with it
-            const uint32_t rb = res_bar(q, (int)(g % kEpiBufs));
+          if (!chunk_coord(ci, n, z)) return false;
+          if (lane == 0) {
+            // the store that last read this buffer must be done with it
+            if (bufs == 1) ptx::bulk_wait_group_read<0>();
+            else ptx::bulk_wait_group_read<1>();
+            const uint32_t rb = res_bar(e, (int)(g % bufs));
             ptx::mbar_arrive_expect_tx(rb, kEpiBufBytes);
-            ptx::tma_load_3d(stg0 + (g % kEpiBufs) * kEpiBufBytes, &tmR, rb, n, row0, z);
+            ptx::tma_load_3d(stg0 + (g % bufs) * kEpiBufBytes, &tmR, rb, n, row0, z);
           }
+          return true;
         };
-        // this tile's bias slice, as FP32, into the warp's own shared-memory copy
+        // the bias values of this warp's own chunks, as BF16, into the warp's shared-memory slice
         if constexpr (epi_has_bias<EPI>()) {
           __syncwarp();
-          float bv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          const int nb = n_tile0 + lane * 8;
-          if (p.bias != nullptr && lane * 8 < p.out_cols && nb < p.N_out)
-            load_bf16x8(p.bias + nb, min(8, p.N_out - nb), p.bias_vec != 0, bv);
-          ptx::st_shared_v4(bias_s + (uint32_t)lane * 32u, __float_as_uint(bv[0]), __float_as_uint(bv[1]),
-                            __float_as_uint(bv[2]), __float_as_uint(bv[3]));
-          ptx::st_shared_v4(bias_s + (uint32_t)lane * 32u + 16u, __float_as_uint(bv[4]), __float_as_uint(bv[5]),
-                            __float_as_uint(bv[6]), __float_as_uint(bv[7]));
+          if (lane < 16) {
+            const int local = lane * 8;                      // index among the warp's 128 columns
+            const int ci = 2 * (local / chunk_cols) + half;  // the chunk that column belongs to
+            const int nb = n_tile0 + ci * chunk_cols + (local % chunk_cols);
+            float bv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (p.bias != nullptr && ci < n_chunks && nb < p.N_out)
+              load_bf16x8(p.bias + nb, min(8, p.N_out - nb), p.bias_vec != 0, bv);
+            ptx::st_shared_v4(bias_s + (uint32_t)lane * 16u, pack_bf16x2(bv[0], bv[1]), pack_bf16x2(bv[2], bv[3]),
+                              pack_bf16x2(bv[4], bv[5]), pack_bf16x2(bv[6], bv[7]));
+          }
           __syncwarp();
         }
-        if (use_r) issue_residual(0, gc);
+        if (use_r && r_next <= gc && issue_residual(half, gc)) r_next = gc + 1;
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
           ok = false;
           break;
         }
         ptx::tc_fence_after();
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
-        const int n_chunks = acc_cols / chunk_cols;
-        for (int ci = 0; ci < n_chunks; ++ci) {
+        for (int ci = half; ci < n_chunks; ci += 2) {
           int n_chunk, z;
           if (!chunk_coord(ci, n_chunk, z)) continue;  // uniform across the warp
-          const uint32_t buf = stg0 + (gc % kEpiBufs) * kEpiBufBytes;
+          const uint32_t buf = stg0 + (gc % bufs) * kEpiBufBytes;
+          const int c0 = ci * chunk_cols;  // first accumulator column of the chunk
+          const int pieces = chunk_cols / 32;
+          // Start the TMEM loads; compute the whole chunk into packed registers; only then claim the staging
+          // buffer (the TMA store that last read it has had the time of the math to finish) and write it.
+          uint32_t v0[32];
+          uint32_t v1[32];
+          uint32_t outw[32];  // the chunk's 128 bytes per row: 64 BF16 or 32 FP32 values
+          ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c0, v0);
+          if constexpr (EPI == kEpiSiluGate) {
+            ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c0), v1);
+          } else {
+            if (pieces == 2) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(c0 + 32), v1);
+          }
           if (use_r) {
-            if (ci + 1 < n_chunks) issue_residual(ci + 1, gc + 1);
-            if (!wait_bar(res_bar(q, (int)(gc % kEpiBufs)), (gc / kEpiBufs) & 1u, abort_p, p.status)) {
+            if (r_next <= gc && issue_residual(ci, gc)) r_next = gc + 1;
+            if (!wait_bar(res_bar(e, (int)(gc % bufs)), (gc / bufs) & 1u, abort_p, p.status)) {
               ok = false;
               break;
             }
-          } else {
-            if (lane == 0) ptx::bulk_wait_group_read<kEpiBufs - 1>();
-            __syncwarp();
           }
-#pragma unroll 1
-          for (int piece = 0; piece * 32 < chunk_cols; ++piece) {
-            const int c = ci * chunk_cols + piece * 32;  // accumulator column of this 32-wide piece
-            uint32_t v[32];
-            uint32_t vu[32];
-            ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
-            if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
-            ptx::tmem_wait_ld();
+          ptx::tmem_wait_ld();
+          // one 32-column piece: fused operation on packed FP32 pairs, rounding, into outw
+          auto do_piece = [&](int piece, const uint32_t (&a)[32], const uint32_t (&up)[32]) {
+            const int local0 = (ci >> 1) * chunk_cols + piece * 32;  // index among the warp's 128 columns
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-              float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-              float res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-              float y[8];
+              uint32_t bw[4] = {0u, 0u, 0u, 0u};  // 8 BF16 bias values
+              uint32_t rw[4] = {0u, 0u, 0u, 0u};  // 8 BF16 residual values
               if constexpr (epi_has_bias<EPI>()) {
-                const uint4 b0 = ptx::ld_shared_v4(bias_s + (uint32_t)(c + g * 8) * 4u);
-                const uint4 b1 = ptx::ld_shared_v4(bias_s + (uint32_t)(c + g * 8) * 4u + 16u);
-                bias[0] = __uint_as_float(b0.x); bias[1] = __uint_as_float(b0.y);
-                bias[2] = __uint_as_float(b0.z); bias[3] = __uint_as_float(b0.w);
-                bias[4] = __uint_as_float(b1.x); bias[5] = __uint_as_float(b1.y);
-                bias[6] = __uint_as_float(b1.z); bias[7] = __uint_as_float(b1.w);
+                const uint4 bq = ptx::ld_shared_v4(bias_s + (uint32_t)(local0 + g * 8) * 2u);
+                bw[0] = bq.x; bw[1] = bq.y; bw[2] = bq.z; bw[3] = bq.w;
               }
-              if (f32) {
-                apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
-                const uint32_t j0 = (uint32_t)(2 * g), j1 = j0 + 1u;
-                ptx::st_shared_v4(buf + my_row + ((j0 ^ swz) << 4), __float_as_uint(y[0]), __float_as_uint(y[1]),
-                                  __float_as_uint(y[2]), __float_as_uint(y[3]));
-                ptx::st_shared_v4(buf + my_row + ((j1 ^ swz) << 4), __float_as_uint(y[4]), __float_as_uint(y[5]),
-                                  __float_as_uint(y[6]), __float_as_uint(y[7]));
-              } else {
-                const uint32_t j = (uint32_t)(piece * 4 + g);
-                const uint32_t addr = buf + my_row + ((j ^ swz) << 4);
-                if constexpr (EPI == kEpiBiasResidual) {
-                  if (use_r) {
-                    const uint4 rq = ptx::ld_shared_v4(addr);
-                    unpack_bf16x8(rq, res);
-                  } else {
-                    const int row = row0 + lane;
-                    const int n = n_chunk + piece * 32 + g * 8;
-                    if (row < p.M && n < p.N_out)
-                      load_bf16x8(p.R + (long long)z * p.strideR + (long long)row * p.ldr + n, min(8, p.N_out - n),
-                                  p.r_vec != 0, res);
+              if constexpr (EPI == kEpiBiasResidual) {
+                if (use_r) {
+                  const uint32_t j = (uint32_t)(piece * 4 + g);
+                  const uint4 rq = ptx::ld_shared_v4(buf + my_row + ((j ^ swz) << 4));
+                  rw[0] = rq.x; rw[1] = rq.y; rw[2] = rq.z; rw[3] = rq.w;
+                } else {
+                  const int row = row0 + lane;
+                  const int n = n_chunk + piece * 32 + g * 8;
+                  if (row < p.M && n < p.N_out) {
+                    float rf[8];
+                    load_bf16x8(p.R + (long long)z * p.strideR + (long long)row * p.ldr + n, min(8, p.N_out - n),
+                                p.r_vec != 0, rf);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) rw[t] = pack_bf16x2(rf[2 * t], rf[2 * t + 1]);  // exact: BF16 values
                   }
                 }
-                apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
-                ptx::st_shared_v4(addr, pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]),
-                                  pack_bf16x2(y[6], y[7]));
+              }
+#pragma unroll
+              for (int t = 0; t < 4; ++t) {
+                const uint64_t y2 = epilogue_pair<EPI>(ptx::pack_f32x2(a[g * 8 + 2 * t], a[g * 8 + 2 * t + 1]),
+                                                       ptx::pack_f32x2(up[g * 8 + 2 * t], up[g * 8 + 2 * t + 1]),
+                                                       ptx::bf16x2_to_f32x2(bw[t]), ptx::bf16x2_to_f32x2(rw[t]));
+                uint32_t lo, hi;
+                ptx::unpack_f32x2(y2, lo, hi);
+                if (f32) {
+                  outw[g * 8 + 2 * t] = lo;
+                  outw[g * 8 + 2 * t + 1] = hi;
+                } else {
+                  outw[piece * 16 + g * 4 + t] = pack_bf16x2(__uint_as_float(lo), __uint_as_float(hi));
+                }
               }
             }
+          };
+          if constexpr (EPI == kEpiSiluGate) {
+            do_piece(0, v0, v1);
+            if (pieces == 2) {
+              ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(c0 + 32), v0);
+              ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c0 + 32), v1);
+              ptx::tmem_wait_ld();
+              do_piece(1, v0, v1);
+            }
+          } else {
+            do_piece(0, v0, v0);
+            if (pieces == 2) do_piece(1, v1, v1);
           }
+          if (!use_r) {
+            if (lane == 0) {
+              if (bufs == 1) ptx::bulk_wait_group_read<0>();
+              else ptx::bulk_wait_group_read<1>();
+            }
+            __syncwarp();
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            ptx::st_shared_v4(buf + my_row + (((uint32_t)j ^ swz) << 4), outw[4 * j], outw[4 * j + 1],
+                              outw[4 * j + 2], outw[4 * j + 3]);
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
             if (row0 < p.M && !(p.debug & 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
             ptx::bulk_commit_group();
           }
+          // with two buffers the next residual tile can start now: its buffer's last store is one chunk old
+          if (use_r && bufs == 2 && issue_residual(ci + 2, gc + 1)) r_next = gc + 2;
           ++gc;
         }
         if (!ok) break;
@@ -605,7 +698,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         char* c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
         const __nv_bfloat16* r_row = nullptr;
         if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
-        for (int c = 0; c < p.out_cols; c += 32) {
+        for (int c = half * 32; c < p.out_cols; c += 64) {  // the two warps of a quarter alternate 32-column pieces
           const int n0 = n_tile0 + c;
           if (n0 >= p.N_out) break;  // uniform across the warp
           uint32_t v[32];
