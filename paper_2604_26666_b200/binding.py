@@ -133,11 +133,15 @@ def _ld(t: torch.Tensor) -> int:
 class Handle:
     """A libfact handle on one CUDA device, plus a grow-only torch workspace."""
 
-    def __init__(self, device: int = 0):
+    def __init__(self, device: int = 0, load_table: bool = True):
         self._h = c_void_p()
         self.device = int(device)
         _check(lib().fact_create(byref(self._h), self.device), "fact_create")
         self._ws: Optional[torch.Tensor] = None
+        self._ws_cache: dict = {}
+        table = _PKG / "tuned_b200.txt"
+        if load_table and table.exists():  # the tuner's table for the benchmark shapes, measured on a B200
+            self.tune_cache_load(str(table))
 
     def close(self):
         if self._h:
@@ -172,10 +176,19 @@ class Handle:
 
     def workspace_bytes(self, op, batch, M, N, K, epilogue="NONE", layout="KN", out_dtype=torch.bfloat16, cfg=None,
                         splits=0) -> int:
+        if cfg is None or isinstance(cfg, Config):
+            ckey = None if cfg is None else tuple(cfg.as_dict().values())
+        else:
+            ckey = tuple(sorted(dict(cfg).items()))
+        key = (op, batch, M, N, K, epilogue, layout, out_dtype, ckey, splits)
+        hit = self._ws_cache.get(key)
+        if hit is not None:
+            return hit
         n = c_size_t(0)
         c = self._cfg_with_splits(cfg, splits)
         _check(lib().fact_workspace_bytes(self._h, OPS[op], batch, M, N, K, EPILOGUES[epilogue], LAYOUTS[layout],
                                           OUT_TYPES[out_dtype], c, byref(n)), "fact_workspace_bytes")
+        self._ws_cache[key] = int(n.value)
         return int(n.value)
 
     def _cfg_with_splits(self, cfg, splits):
@@ -215,6 +228,7 @@ class Handle:
 
     def tune_cache_load(self, path: str):
         _check(lib().fact_tune_cache_load(self._h, str(path).encode()), "fact_tune_cache_load")
+        self._ws_cache.clear()  # the library's own choices may have changed
 
     # -- compute ------------------------------------------------------------------------------
     def gemm(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
@@ -320,6 +334,7 @@ class Handle:
             out = torch.empty(((batch, M, N) if batched else (M, N)), dtype=out_dtype, device=A.device)
         ws = self.workspace(workspace_bytes)
         best, ms, n = Config(), c_double(0.0), c_int(0)
+        self._ws_cache.clear()
         _check(lib().fact_tune(self._h, OPS[op], batch, M, N, K, _ptr(A), _ld(A), A.stride(0) if batched else 0,
                                _ptr(B), _ld(B), B.stride(0) if batched else 0, LAYOUTS[layout], _ptr(bias),
                                _ptr(residual), _ld(residual) if residual is not None else 0,

@@ -1,0 +1,57 @@
+"""Run the on-device tile-configuration tuner over the benchmark shapes and
+write the table that `Handle` loads by default.
+
+    python -m paper_2604_26666_b200.tune [--out PATH] [--layout NK|KN|both] [--shapes a,b,...]
+
+The counterpart of the paper's auto-tuning action (Section 4.2, Action 5): every
+feasible candidate is timed on the device (5 warm-up + 20 timed launches, the
+protocol of Section 5.1) and the fastest is kept per problem key.
+"""
+from __future__ import annotations
+
+import argparse
+import sys
+from pathlib import Path
+
+import torch
+
+from . import workloads as wl
+from .binding import Handle
+
+DEFAULT_TABLE = Path(__file__).resolve().parent / "tuned_b200.txt"
+
+
+def tune_case(h: Handle, case: wl.Case, dev: str = "cuda:0"):
+    ins = wl.make_inputs(case)
+    X, W = ins.X.to(dev), ins.W.to(dev)
+    bias = None if ins.bias is None else ins.bias.to(dev)
+    res = None if ins.residual is None else ins.residual.to(dev)
+    odt = torch.float32 if case.out == "f32" else torch.bfloat16
+    return h.tune(case.op, X, W, layout=case.layout, bias=bias, residual=res, epilogue=case.epilogue, out_dtype=odt)
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default=str(DEFAULT_TABLE))
+    ap.add_argument("--layout", default="both", choices=["NK", "KN", "both"])
+    ap.add_argument("--shapes", default=None)
+    args = ap.parse_args(argv)
+    h = Handle(0, load_table=False)
+    names = None if args.shapes is None else set(args.shapes.split(","))
+    seen = set()
+    for layout in (["NK", "KN"] if args.layout == "both" else [args.layout]):
+        for case in wl.benchmark_cases(layout):
+            key = (case.name, case.layout)
+            if key in seen or (names is not None and case.name not in names):
+                continue
+            seen.add(key)
+            cfg, ms, n = tune_case(h, case)
+            print(f"{case.name:32s} {case.layout} best {ms * 1e3:9.1f} us  {case.flops / ms / 1e9:8.1f} TFLOP/s  "
+                  f"of {n:3d} candidates: {cfg}", flush=True)
+    h.tune_cache_save(args.out)
+    print("wrote", args.out)
+    h.close()
+
+
+if __name__ == "__main__":
+    sys.exit(main())
