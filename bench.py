@@ -202,18 +202,12 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
+    from paper_2604_26666_b200 import dist_util
 
-        dist = dist_mod
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    rank, world, local_rank = dist_util.env_ranks()
     dev = torch.device(f"cuda:{local_rank}")
     torch.cuda.set_device(dev)
+    dist = dist_util.init("nccl", dev)
     h = Handle(local_rank)
     peaks = load_peaks()
     stream = torch.cuda.current_stream(dev)
@@ -228,10 +222,7 @@ def main():
     def flush_l2():
         flush_buf.fill_(1)
 
-    tune_table = os.path.join(ROOT, "paper_2604_26666_b200", "tuned_b200.txt")
-    if os.path.exists(tune_table):
-        h.tune_cache_load(tune_table)
-
+    # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
         rows = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup,
@@ -278,11 +269,7 @@ def main():
     launches = h.launch_count() - launches0
     step_ms = [e[0].elapsed_time(e[1]) for e in ev]
     dom_ms = [e[2].elapsed_time(e[3]) for e in ev]
-    total_ms = sum(step_ms)
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = dist_util.max_over_ranks(sum(step_ms), dist, dev)
     assert h.device_status() == 0, "a device-side wait timed out during the timed region"
     value = world * step_flops * args.steps / (total_ms * 1e-3) / 1e12
     dom_case = cases[dom]
@@ -310,11 +297,7 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1), dist, dev)
     e2e_value = world * step_flops * e2e_steps / (e2e_ms * 1e-3) / 1e12
     clocks = sampler.stop()
     del host_outs

@@ -1,0 +1,115 @@
+"""Parity of the five benchmark configurations at their full sizes, in the launch
+configuration bench.py times (the handle's tuned table / default choice).
+
+The small configuration (config 1) and the batched / split-K shapes are compared
+element by element.  For the large shapes the oracle computes a stratified sample of
+output rows (first/last rows, tile borders, random rows: every column of each), and a
+Freivalds-style product check covers every element of the linear epilogues:
+    Y x  ==  X (W x) + (bias . x) + R x        for random +-1 vectors x, in FP64.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_26666_b200 import workloads as wl
+from tests.helpers import check_case, gates, oracle_for, run_gpu, stratified_rows, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def h():
+    from paper_2604_26666_b200.binding import Handle
+    hd = Handle(0)
+    yield hd
+    hd.close()
+
+
+CASES = {c.name: c for c in wl.benchmark_cases("NK")}
+CASES_KN = {c.name: c for c in wl.benchmark_cases("KN")}
+
+
+def test_config1_elementwise(h):
+    check_case(h, CASES["c1_512_bias_relu"])
+
+
+def test_config3_batched_elementwise(h):
+    # 128 x (512 x 512 x 1024): 34 GFLOP of oracle work
+    check_case(h, CASES["c3_batched_128x512x512x1024"])
+
+
+def test_config3_splitk_elementwise_and_deterministic(h):
+    case = CASES["c3_splitk_256x256x131072"]
+    ins = wl.make_inputs(case)
+    got = run_gpu(h, ins, case)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    ref = oracle_for(ins, case)
+    g = to_f64(got)
+    c, t = gates(ref, g, "f32", "NONE")
+    assert c <= 1.0 and t <= 1.0, (c, t)
+    # the componentwise backward-error scale: |err| / sum_k |a||b| stays at FP32 accumulation level
+    absx = ins.X.float().abs().double().numpy()
+    absw = ins.W.float().abs().double().numpy()
+    scale = absx @ absw
+    assert (np.abs(g - ref) / scale).max() < 1e-6
+    # pure relative error is undefined next to zero: count how many elements a plain 2e-3 bound would flag
+    rel_viol = int((np.abs(g - ref) > 2e-3 * np.abs(ref)).sum())
+    assert rel_viol <= 16, rel_viol
+    again = run_gpu(h, ins, case)
+    assert torch.equal(got, again), "split-K output is not reproducible"
+
+
+def freivalds(ins, case, got, n_vec=2, seed=0):
+    """max over vectors of |Y x - (X (W x) + bias.x + R x)| / scale, in FP64."""
+    rng = np.random.default_rng(seed)
+    X = ins.X.float().double().numpy()
+    W = ins.W.float().double().numpy()
+    Wkn = W if case.layout == "KN" else W.T  # [K, N]
+    Y = to_f64(got)
+    worst = 0.0
+    for _ in range(n_vec):
+        x = rng.choice([-1.0, 1.0], size=case.N)
+        want = X @ (Wkn @ x)
+        if ins.bias is not None:
+            want = want + float(ins.bias.float().double().numpy() @ x)
+        if ins.residual is not None:
+            want = want + ins.residual.float().double().numpy() @ x
+        have = Y @ x
+        # each of the N terms carries a BF16 rounding error of at most 2^-9 |y|; they add like a random walk
+        scale = 2.0 ** -9 * np.sqrt(case.N) * (np.sqrt(np.mean(Y * Y)) + 1e-30)
+        worst = max(worst, float(np.abs(have - want).max() / scale))
+    return worst
+
+
+LINEAR_SAMPLED = ["c2_square_4096", "c2_square_8192", "c4_qkv", "c4_out_proj", "c4_mlp_up_gelu", "c4_mlp_down",
+                  "c5_qkv", "c5_o_proj", "c5_gate_up_silu", "c5_down"]
+
+
+@pytest.mark.parametrize("name", LINEAR_SAMPLED)
+def test_full_size_sampled_rows(h, name):
+    case = (CASES_KN if name.startswith("c2") else CASES)[name]
+    ins = wl.make_inputs(case)
+    got = run_gpu(h, ins, case)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    n_rows = 48 if case.flops > 5e11 else 96
+    rows = stratified_rows(case.M, n_rows, seed=case.seed, tile=256)
+    ref = oracle_for(ins, case, rows=rows)
+    g = to_f64(got)[rows]
+    assert np.isfinite(to_f64(got)).all()
+    c, t = gates(ref, g, case.out, case.epilogue)
+    assert c <= 1.0, f"{name}: contract gate ratio {c:.3f}"
+    assert t <= 1.0, f"{name}: tight gate ratio {t:.3f}"
+    if case.epilogue in ("NONE", "BIAS", "BIAS_RESIDUAL"):
+        f = freivalds(ins, case, got)
+        assert f < 6.0, f"{name}: Freivalds residual {f:.2f} x the rounding scale"
+
+
+@pytest.mark.parametrize("name", ["c4_qkv", "c4_mlp_down", "c5_o_proj"])
+def test_full_size_kn_layout(h, name):
+    """The same linears with the weight stored [K x N]."""
+    case = CASES_KN[name]
+    rows = stratified_rows(case.M, 32, seed=1, tile=256)
+    check_case(h, case, rows=rows)
