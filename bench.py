@@ -87,7 +87,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             parts = [x.strip() for x in ln.split(",")]
@@ -96,15 +96,17 @@ class ClockSampler:
             try:
                 sm.append(float(parts[0]))
                 mx.append(float(parts[1]))
+                pw.append(float(parts[2]))
             except ValueError:
                 continue
             for nm, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
-        # keep the samples taken under load (clock above idle), else all
-        busy = [c for c in sm if c > 0.5 * (max(mx) if mx else 1)] or sm
+        # "under load" = the samples drawing at least half of the largest power seen
+        busy = [c for c, w in zip(sm, pw) if w >= 0.5 * max(pw)] if pw else sm
         return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "samples_under_load": len(busy),
+                "power_w_max": max(pw) if pw else None}
 
 
 # ------------------------------------------------------------------------------------------ reference arm
@@ -251,11 +253,11 @@ def main():
             if events is not None and i == dom:
                 events[1].record(stream)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = h.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
            torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -271,6 +273,7 @@ def main():
     dom_ms = [e[2].elapsed_time(e[3]) for e in ev]
     total_ms = dist_util.max_over_ranks(sum(step_ms), dist, dev)
     assert h.device_status() == 0, "a device-side wait timed out during the timed region"
+    k_cycles, k_ns = h.last_kernel_clock()  # the dominant launch is the last one of a step
     value = world * step_flops * args.steps / (total_ms * 1e-3) / 1e12
     dom_case = cases[dom]
     dom_avg_ms = sum(dom_ms) / len(dom_ms)
@@ -299,13 +302,13 @@ def main():
     barrier()
     e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1), dist, dev)
     e2e_value = world * step_flops * e2e_steps / (e2e_ms * 1e-3) / 1e12
-    clocks = sampler.stop()
     del host_outs
 
     # ---------------------------------------------------------------- every shape of the five configurations
     shapes = []
     if not args.no_shapes and rank == 0:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
+    clocks = sampler.stop()  # sampled from the first warm-up step to the end of the per-shape table
 
     # ---------------------------------------------------------------- CPU baseline (oracle) on rank 0
     cpu = None
@@ -334,7 +337,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches,
-            "clocks": clocks,
+            "clocks": dict(clocks, sm_mhz_in_dominant_kernel=(1e3 * k_cycles / k_ns if k_ns else None)),
             "cpu_baseline": cpu,
             "shapes": shapes,
         }
