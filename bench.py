@@ -38,9 +38,9 @@ METRIC = "TFLOP/s & % of dense BF16 tensor peak per fused-epilogue GEMM shape"
 WORKLOAD = "config 2: square BF16 GEMM 4096^3 + 8192^3, N(0,1)/sqrt(K), seed 1"
 L2_FLUSH_BYTES = 512 << 20
 
-# DRAM traffic per launch of the dominant kernel (8192^3), from the ncu capture summarised in
-# profiles/ (None until a capture exists).
-DOMINANT_TRAFFIC_BYTES = None
+# DRAM traffic per launch of the dominant kernel (8192^3): dram__bytes_read.sum + dram__bytes_write.sum of the
+# ncu capture summarised in profiles/fact_gemm_kernel_c2_square_8192.md (1.0745 GB + 127.15 MB).
+DOMINANT_TRAFFIC_BYTES = 1.2017e9
 
 
 def load_peaks():
@@ -333,7 +333,7 @@ def main():
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                          "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                          "peak_source": peaks["source"] + " (burst)", "launch_ms": dom_avg_ms,
-                         "traffic": DOMINANT_TRAFFIC_BYTES},
+                         "traffic": DOMINANT_TRAFFIC_BYTES, "algorithmic_bytes": dom_case.algorithmic_bytes},
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches,
