@@ -432,8 +432,8 @@ fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan,
   r.ldr = q.ldr;
   r.strideR = q.strideR;
   const long long total = (long long)r.batch * r.M * ((r.N_out + 3) / 4);
-  const int blocks = (int)std::min<long long>((total + 255) / 256, (long long)h->sm_count * 8);
-  fact_splitk_reduce_kernel<<<std::max(1, blocks), 256, 0, stream>>>(r);
+  const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)h->sm_count * 16);
+  fact_splitk_reduce_kernel<<<std::max(1, blocks), 128, 0, stream>>>(r);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(h, "split-K reduce launch", e);
   h->launches++;

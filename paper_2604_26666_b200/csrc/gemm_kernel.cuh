@@ -793,7 +793,7 @@ __device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, flo
   }
 }
 
-__global__ void __launch_bounds__(256) fact_splitk_reduce_kernel(const ReduceParams p) {
+__global__ void __launch_bounds__(128) fact_splitk_reduce_kernel(const ReduceParams p) {
   const long long groups_per_row = (p.N_out + 3) / 4;
   const long long total = (long long)p.batch * p.M * groups_per_row;
   const long long plane_stride = (long long)p.M * p.ws_ld;
@@ -807,13 +807,28 @@ __global__ void __launch_bounds__(256) fact_splitk_reduce_kernel(const ReducePar
     const int nvalid = min(4, p.N_out - n);
     float a[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
     const bool gate = p.epi == kEpiSiluGate;
-    for (int s = 0; s < p.splits; ++s) {  // ascending slice order: deterministic
-      const float* ps = p.ws + ((long long)(s * p.batch + b) * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
-      const float4 v = *reinterpret_cast<const float4*>(ps);  // ws_ld is a multiple of 4: padding is in bounds
-      a[0] += v.x; a[1] += v.y; a[2] += v.z; a[3] += v.w;
-      if (gate) {
-        const float4 t = *reinterpret_cast<const float4*>(ps + plane_stride);
-        up[0] += t.x; up[1] += t.y; up[2] += t.z; up[3] += t.w;
+    const float* base = p.ws + ((long long)b * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
+    const long long slice_stride = (long long)p.batch * p.planes * plane_stride;
+    // Loads of eight slices are issued together, then added in ascending slice order: the order of the
+    // additions (and so the result) depends only on the number of slices.
+    for (int s0 = 0; s0 < p.splits; s0 += 8) {
+      float4 v[8], t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (s0 + i < p.splits) {
+          const float* ps = base + (long long)(s0 + i) * slice_stride;
+          v[i] = __ldcg(reinterpret_cast<const float4*>(ps));  // ws_ld is a multiple of 4: padding is in bounds
+          if (gate) t[i] = __ldcg(reinterpret_cast<const float4*>(ps + plane_stride));
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (s0 + i < p.splits) {
+          a[0] += v[i].x; a[1] += v[i].y; a[2] += v[i].z; a[3] += v[i].w;
+          if (gate) {
+            up[0] += t[i].x; up[1] += t[i].y; up[2] += t[i].z; up[3] += t[i].w;
+          }
+        }
       }
     }
     for (int j = 0; j < nvalid; ++j) {
