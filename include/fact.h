@@ -154,6 +154,41 @@ fact_status_t fact_gemm_splitk(fact_handle_t handle, int64_t M, int64_t N, int64
                                fact_out_t out_type, int splits, const fact_config_t* cfg, void* workspace,
                                size_t workspace_bytes, void* cuda_stream);
 
+/* fact_gemm_splitk for callers that must not allocate device memory.  (The paper has no counterpart
+ * of this entry point; it exists for integration, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region whose device memory
+ * is owned by a pool or arena that forbids side allocations, in a latency-critical loop that may not
+ * take the allocator's locks or implicit synchronisation, or in a process that has handed all of its
+ * memory budget to someone else.  Such a caller can create neither a handle (fact_create allocates
+ * the status word) nor a split-K workspace.  This call needs neither: it takes no handle, and its
+ * scratch is a fixed 16 MiB array that is part of the library's device image (so every GPU that loads
+ * the library carries those 16 MiB until the process exits).
+ *
+ * Computes C[M x N] = A[M x K] . B exactly like fact_gemm_splitk (same kernels, same fixed-order
+ * reduction, same argument rules for A, B, C, leading dimensions, b_layout, out_type; `splits` = 0
+ * lets the library choose), on CUDA device `device`, enqueued on `cuda_stream`.  The caller still
+ * owns and passes the inputs and the output.  It calls no cudaMalloc / cudaFree and no allocating
+ * library routine.
+ *
+ * Limits and rules:
+ *   - the FP32 partial planes, splits * M * round_up(N, 4) * 4 bytes, must fit in 16 MiB; a larger
+ *     problem (or split count) is refused with FACT_ERR_WORKSPACE_TOO_SMALL and nothing is launched
+ *     -- pass fewer splits, or use fact_gemm_splitk with your own workspace;
+ *   - the first call on a device resolves the device addresses of the static arrays and a few device
+ *     properties (it makes `device` current for the duration of the call); make that first call
+ *     outside any stream capture;
+ *   - all calls on a device share the one scratch array and it keeps whatever the last call left in
+ *     it.  Nothing in it has to start at zero (every partial that is read is written first by the
+ *     same call), but two calls that overlap on the GPU -- different streams, or different host
+ *     threads -- race on it and both results are garbage: keep calls on one device in one stream
+ *     order;
+ *   - a device-side wait that expires is recorded in a status word that is likewise static and
+ *     per device; this entry point does not report it (there is no handle to ask). */
+fact_status_t fact_gemm_splitk_static(int device, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                      const void* B, int64_t ldb, fact_blayout_t b_layout, void* C, int64_t ldc,
+                                      fact_out_t out_type, int splits, void* cuda_stream);
+
 /* Y[M x N_out] = epilogue(X[M x K] . W)        (Section 5.2: fused linear layers)
  * W: FACT_B_NK [Nw x K] (nn.Linear weight) or FACT_B_KN [K x Nw]; Nw = N_out,
  * or 2*N_out for SILU_GATE.  bias: BF16 [N_out]; required by BIAS, BIAS_RELU,

@@ -35,7 +35,7 @@ EXPORTED = [
     "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
     "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
-    "fact_last_kernel_clock",
+    "fact_last_kernel_clock", "fact_gemm_splitk_static",
 ]
 
 
@@ -81,6 +81,7 @@ def lib() -> ctypes.CDLL:
     L.fact_gemm_batched.argtypes = [vp, i64, i64, i64, i64, vp, i64, i64, vp, i64, i64, c_int, vp, i64, i64, c_int,
                                     cfgp, vp, sz, vp]
     L.fact_gemm_splitk.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, c_int, cfgp, vp, sz, vp]
+    L.fact_gemm_splitk_static.argtypes = [c_int, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, c_int, vp]
     L.fact_linear.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, vp, i64, vp, i64, c_int, c_int, cfgp,
                               vp, sz, vp]
     L.fact_get_config.argtypes = [vp, c_int, i64, i64, i64, i64, c_int, c_int, c_int, cfgp]
@@ -128,6 +129,23 @@ def _need(t: torch.Tensor, name: str, dtype, ndim):
 def _ld(t: torch.Tensor) -> int:
     """Leading dimension of the last two dims; a one-row matrix may carry any stride."""
     return int(t.stride(-2)) if t.shape[-2] > 1 else max(int(t.shape[-1]), int(t.stride(-2)))
+
+
+def gemm_splitk_static(A, B, out, layout="KN", splits=0, device=None, stream=None):
+    """C = A @ B through fact_gemm_splitk_static: no handle, no workspace, no device allocation inside the
+    library (its split-K scratch is a fixed 16 MiB array inside the library image).  For callers that may
+    not call cudaMalloc; `out` must be preallocated by the caller.  Calls on one device must not overlap."""
+    _need(A, "A", torch.bfloat16, 2)
+    _need(B, "B", torch.bfloat16, 2)
+    _need(out, "out", out.dtype, 2)
+    M, K = A.shape
+    N = B.shape[1] if layout == "KN" else B.shape[0]
+    dev = A.device.index if device is None else int(device)
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    _check(lib().fact_gemm_splitk_static(dev, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
+                                         _ld(out), OUT_TYPES[out.dtype], int(splits), c_void_p(s.cuda_stream)),
+           "fact_gemm_splitk_static")
+    return out
 
 
 class Handle:

@@ -17,6 +17,14 @@
 #include "fact.h"
 #include "gemm_kernel.cuh"
 
+// Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
+// device image, so that entry point never has to allocate.  Every GPU that loads the library holds these
+// 16 MiB until the process exits.  In host code these names are only stand-ins for the device symbols; the
+// device addresses the kernels get come from cudaGetSymbolAddress (see static_setup below).
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static __device__ __align__(256) int g_static_status[8];
+
 namespace {
 
 using namespace fact;
@@ -853,6 +861,85 @@ fact_status_t fact_tune_cache_load(fact_handle_t h, const char* path) {
   }
   fclose(f);
   return FACT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free split-K GEMM.  One host-side state per device, filled on the first call for that device.
+namespace {
+constexpr int kMaxStaticDevices = 64;
+struct StaticDeviceState {
+  bool ready = false;
+  void* scratch = nullptr;  // device address of g_static_scratch on this device
+  fact_handle_s handle;     // host-side bookkeeping only; its status word is g_static_status on this device
+};
+StaticDeviceState g_static_state[kMaxStaticDevices];
+
+// Resolve, with `device` current, the device addresses of the static arrays and the few device facts the
+// planner needs.  Nothing here allocates device memory.
+fact_status_t static_setup(int device, StaticDeviceState* st) {
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FACT_ERR_CUDA;
+  if (prop.major != 10) return FACT_ERR_ARCH;
+  void* scratch = nullptr;
+  void* status = nullptr;
+  if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) {
+    cudaGetLastError();
+    return FACT_ERR_CUDA;
+  }
+  if (cudaGetSymbolAddress(&status, g_static_status) != cudaSuccess || !status) {
+    cudaGetLastError();
+    return FACT_ERR_CUDA;
+  }
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return FACT_ERR_CUDA;
+  }
+  fact_handle_s& h = st->handle;
+  h.device = device;
+  h.sm_count = prop.multiProcessorCount;
+  h.max_smem = (int)prop.sharedMemPerBlockOptin;
+  h.cc_major = prop.major;
+  h.cc_minor = prop.minor;
+  h.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  h.d_status = reinterpret_cast<int*>(status);
+  st->scratch = scratch;
+  st->ready = true;
+  return FACT_OK;
+}
+}  // namespace
+
+fact_status_t fact_gemm_splitk_static(int device, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                      const void* B, int64_t ldb, fact_blayout_t layout, void* C, int64_t ldc,
+                                      fact_out_t out, int splits, void* stream) {
+  if (device < 0 || device >= kMaxStaticDevices || splits < 0) return FACT_ERR_INVALID_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) {
+    cudaGetLastError();
+    return FACT_ERR_CUDA;
+  }
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) return FACT_ERR_CUDA;
+  StaticDeviceState* st = &g_static_state[device];
+  fact_status_t rc = FACT_OK;
+  if (!st->ready) rc = static_setup(device, st);  // first call on this device, with this device current
+  if (rc == FACT_OK) {
+    Problem q = make_problem(FACT_OP_GEMM_SPLITK, 1, M, N, K, A, lda, 0, B, ldb, 0, layout, nullptr, nullptr, 0, 0, C,
+                             ldc, 0, out, FACT_EPI_NONE);
+    rc = validate(q);
+    if (rc == FACT_OK && M > 0 && N > 0) {
+      Plan plan;
+      rc = make_plan(&st->handle, q, nullptr, splits, &plan);
+      // the partial planes of this problem must fit the fixed scratch: refuse, never spill elsewhere
+      if (rc == FACT_OK && plan.ws_bytes > kStaticScratchBytes) rc = FACT_ERR_WORKSPACE_TOO_SMALL;
+      if (rc == FACT_OK) rc = run(&st->handle, q, nullptr, splits, st->scratch, kStaticScratchBytes, stream);
+    }
+  }
+  if (prev != device) cudaSetDevice(prev);
+  return rc;
 }
 
 }  // extern "C"
