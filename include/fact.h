@@ -249,6 +249,14 @@ int64_t fact_launch_count(fact_handle_t handle);
 fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, int64_t* sm_cycles,
                                      int64_t* nanoseconds);
 
+/* Diagnostic: where the first CTA of the most recent GEMM launch spent its SM cycles.  Only filled when
+ * the process was started with FACT_DEBUG_FLAGS=256 (the counters cost a few clock reads per tile);
+ * otherwise counters[2..7] keep older values.  counters[0] cycles from start to end, [1] the same span
+ * in nanoseconds, [2] MMA issuer waiting for a free accumulator (epilogue too slow), [3] MMA issuer waiting
+ * for operand stages (loads too slow), [4] one epilogue warp busy from "accumulator ready" to "accumulator
+ * released", [5] that warp waiting for an accumulator, [6] tiles that CTA processed, [7] unused. */
+fact_status_t fact_last_kernel_profile(fact_handle_t handle, void* cuda_stream, int64_t counters[8]);
+
 /* Text of the most recent CUDA runtime/driver failure seen through this handle
  * (the call that returned FACT_ERR_CUDA), "" if none.  Owned by the handle;
  * valid until the next failing call or fact_destroy. */

@@ -35,7 +35,7 @@ EXPORTED = [
     "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
     "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
-    "fact_last_kernel_clock", "fact_gemm_splitk_static",
+    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile",
 ]
 
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
     L.fact_launch_count.restype = i64
     L.fact_device_info.argtypes = [vp, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
     L.fact_last_kernel_clock.argtypes = [vp, vp, POINTER(i64), POINTER(i64)]
+    L.fact_last_kernel_profile.argtypes = [vp, vp, POINTER(i64)]
     L.fact_last_error.argtypes = [vp]
     L.fact_last_error.restype = c_char_p
     for name in EXPORTED:
@@ -232,6 +233,12 @@ class Handle:
         c, n = c_int64(0), c_int64(0)
         _check(lib().fact_last_kernel_clock(self._h, self._stream(stream), byref(c), byref(n)), "fact_last_kernel_clock")
         return int(c.value), int(n.value)
+
+    def last_kernel_profile(self, stream=None):
+        """The eight cycle counters of fact_last_kernel_profile (needs FACT_DEBUG_FLAGS=256)."""
+        arr = (c_int64 * 8)()
+        _check(lib().fact_last_kernel_profile(self._h, self._stream(stream), arr), "fact_last_kernel_profile")
+        return [int(x) for x in arr]
 
     def launch_count(self) -> int:
         return int(lib().fact_launch_count(self._h))

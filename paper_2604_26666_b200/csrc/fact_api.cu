@@ -23,7 +23,7 @@
 // device addresses the kernels get come from cudaGetSymbolAddress (see static_setup below).
 constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-static __device__ __align__(256) int g_static_status[8];
+static __device__ __align__(256) int g_static_status[32];
 
 namespace {
 
@@ -439,7 +439,7 @@ fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan,
   r.R = reinterpret_cast<const __nv_bfloat16*>(q.R);
   r.ldr = q.ldr;
   r.strideR = q.strideR;
-  const long long total = (long long)r.batch * r.M * ((r.N_out + 3) / 4);
+  const long long total = 4LL * r.batch * r.M * ((r.N_out + 3) / 4);  // four threads per group of 4 columns
   const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)h->sm_count * 16);
   fact_splitk_reduce_kernel<<<std::max(1, blocks), 128, 0, stream>>>(r);
   cudaError_t e = cudaGetLastError();
@@ -471,6 +471,9 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
       plan.p.store_tma = 1;  // partials always go through the staged path: the workspace layout is the library's
       plan.p.r_tma = 0;
+      plan.p.ws = reinterpret_cast<const float*>(ws);
+      plan.p.fused_reduce = 1;  // the grid never exceeds the SM count, so the barrier in the kernel's tail is safe
+      plan.p.reduce_epi = (int)q.epi;
     }
     CUtensorMap tm[4];  // A, B, output (or split-K workspace), residual
     CUtensorMap& tmA = tm[0];
@@ -513,7 +516,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
     if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
     else st = launch_epi<1>(h, epi, plan, tm, stream);
-    if (st == FACT_OK && split)
+    if (st == FACT_OK && split && !plan.p.fused_reduce)
       st = launch_reduce(h, q, plan, plan.cfg.split_k, reinterpret_cast<const float*>(ws), stream);
   }
   if (dev != h->device) cudaSetDevice(dev);
@@ -594,8 +597,8 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
     return FACT_ERR_CUDA;
   }
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&h->d_status, 8 * sizeof(int)) != cudaSuccess ||
-      cudaMemset(h->d_status, 0, 8 * sizeof(int)) != cudaSuccess) {
+  if (cudaMalloc(&h->d_status, 32 * sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->d_status, 0, 32 * sizeof(int)) != cudaSuccess) {
     delete h;
     return FACT_ERR_CUDA;
   }
@@ -628,6 +631,15 @@ fact_status_t fact_last_kernel_clock(fact_handle_t h, void* stream, int64_t* sm_
   if (cudaMemcpy(v, h->d_status + 2, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
   *sm_cycles = v[0];
   *nanoseconds = v[1];
+  return FACT_OK;
+}
+
+fact_status_t fact_last_kernel_profile(fact_handle_t h, void* stream, int64_t counters[8]) {
+  if (!h || !counters) return FACT_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return FACT_ERR_CUDA;
+  long long v[8];
+  if (cudaMemcpy(v, h->d_status + 2, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
+  for (int i = 0; i < 8; ++i) counters[i] = v[i];
   return FACT_OK;
 }
 

@@ -98,7 +98,10 @@ struct GemmParams {
   // plane 1 holds the "up" columns of a gated accumulator
   int ws_planes;
   long long ws_ld;
-  int* status;
+  const float* ws;    // the partial planes, for the reduction in the kernel's tail
+  int fused_reduce;   // 1: after a grid-wide barrier every CTA reduces its share of the output (split-K only)
+  int reduce_epi;     // the epilogue the reduction applies
+  int* status;        // [0] error word, [2..17] clock / profile counters, [24], [25] grid-barrier counters
   // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
   // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
   int debug;
@@ -236,6 +239,125 @@ __device__ __forceinline__ void apply_epilogue8(const uint32_t* acc, const uint3
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Split-K reduction: adds the S partials of every output element in ascending slice order,
+// applies the epilogue and stores.  One thread per 4 consecutive output columns.  The same routine
+// serves the tail of the GEMM kernel (all CTAs, after a grid-wide barrier) and a stand-alone kernel.
+struct ReduceParams {
+  const float* ws;  // ws[(split * batch + b) * planes + plane][M][ws_ld]
+  long long ws_ld;
+  int planes;
+  int splits;
+  int M, N_out, batch;
+  int epi;
+  void* C;
+  long long ldc, strideC;
+  int out_f32;
+  const __nv_bfloat16* bias;
+  const __nv_bfloat16* R;
+  long long ldr, strideR;
+};
+
+__device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, float bias, float res) {
+  switch (epi) {
+    case kEpiBias: return a + bias;
+    case kEpiBiasRelu: return fmaxf(a + bias, 0.f);
+    case kEpiBiasGeluTanh: return gelu_tanh_f32(a + bias);
+    case kEpiSiluGate: return silu_f32(a) * up;
+    case kEpiBiasResidual: return a + bias + res;
+    default: return a;
+  }
+}
+
+constexpr int kReduceBatch = 8;  // loads in flight per thread and round trip (32 slices)
+
+// Four adjacent lanes share one group of 4 output columns: lane q of the quad adds slices q, q+4, q+8, ...
+// in ascending order, then the four sums are combined as (s0 + s1) + (s2 + s3).  The order of every
+// addition depends only on the number of slices, so the result is reproducible bit for bit.
+// `first` and `stride` count threads and must be multiples of 32 (whole warps walk the loop together).
+__device__ __forceinline__ void reduce_groups(const ReduceParams& p, long long first, long long stride) {
+  const long long groups_per_row = (p.N_out + 3) / 4;
+  const long long total = (long long)p.batch * p.M * groups_per_row;
+  const long long plane_stride = (long long)p.M * p.ws_ld;
+  const long long slice_stride = (long long)p.batch * p.planes * plane_stride;
+  const bool gate = p.epi == kEpiSiluGate;
+  const long long warp_first = first & ~31LL;
+  const int lane = (int)(first & 31);
+  const int sub = lane & 3;
+  for (long long t0 = warp_first; t0 < total * 4; t0 += stride) {  // uniform trip count within a warp
+    const long long i = (t0 + lane) >> 2;                           // the quad's group
+    const bool valid = i < total;
+    const long long ii = valid ? i : 0;
+    int gcol, m, b;
+    if (total < 0x7fffffffLL) {  // 32-bit index arithmetic: 64-bit division costs hundreds of cycles
+      const unsigned iu = (unsigned)ii, gpr = (unsigned)groups_per_row;
+      const unsigned rmu = iu / gpr;
+      gcol = (int)(iu - rmu * gpr);
+      b = (int)(rmu / (unsigned)p.M);
+      m = (int)(rmu - (unsigned)b * (unsigned)p.M);
+    } else {
+      gcol = (int)(ii % groups_per_row);
+      const long long rm = ii / groups_per_row;
+      m = (int)(rm % p.M);
+      b = (int)(rm / p.M);
+    }
+    const int n = gcol * 4;
+    const int nvalid = min(4, p.N_out - n);
+    float a[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
+    const float* base = p.ws + ((long long)b * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
+    if (valid) {
+      for (int s0 = sub; s0 < p.splits; s0 += 4 * kReduceBatch) {  // this lane's slices, a batch of loads at a time
+        float4 v[kReduceBatch], t[kReduceBatch];
+#pragma unroll
+        for (int i8 = 0; i8 < kReduceBatch; ++i8) {
+          const int sl = s0 + 4 * i8;
+          if (sl < p.splits) {
+            const float* ps = base + (long long)sl * slice_stride;
+            v[i8] = __ldcg(reinterpret_cast<const float4*>(ps));  // ws_ld is a multiple of 4: padding is in bounds
+            if (gate) t[i8] = __ldcg(reinterpret_cast<const float4*>(ps + plane_stride));
+          }
+        }
+#pragma unroll
+        for (int i8 = 0; i8 < kReduceBatch; ++i8) {
+          if (s0 + 4 * i8 < p.splits) {
+            a[0] += v[i8].x; a[1] += v[i8].y; a[2] += v[i8].z; a[3] += v[i8].w;
+            if (gate) {
+              up[0] += t[i8].x; up[1] += t[i8].y; up[2] += t[i8].z; up[3] += t[i8].w;
+            }
+          }
+        }
+      }
+    }
+    // (s0 + s1) + (s2 + s3): every lane of the quad ends with the same total
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      a[j] += __shfl_xor_sync(0xffffffffu, a[j], 1);
+      a[j] += __shfl_xor_sync(0xffffffffu, a[j], 2);
+      if (gate) {
+        up[j] += __shfl_xor_sync(0xffffffffu, up[j], 1);
+        up[j] += __shfl_xor_sync(0xffffffffu, up[j], 2);
+      }
+    }
+    // lane `sub` of the quad finishes column n + sub
+    if (valid && sub < nvalid) {
+      const int j = sub;
+      const float av = sub == 0 ? a[0] : sub == 1 ? a[1] : sub == 2 ? a[2] : a[3];
+      const float uv = sub == 0 ? up[0] : sub == 1 ? up[1] : sub == 2 ? up[2] : up[3];
+      const float bias = p.bias ? __bfloat162float(p.bias[n + j]) : 0.f;
+      const float res =
+          (p.epi == kEpiBiasResidual) ? __bfloat162float(p.R[(long long)b * p.strideR + (long long)m * p.ldr + n + j]) : 0.f;
+      const float y = reduce_epilogue(p.epi, av, uv, bias, res);
+      const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n + j;
+      if (p.out_f32) reinterpret_cast<float*>(p.C)[off] = y;
+      else reinterpret_cast<__nv_bfloat16*>(p.C)[off] = __float2bfloat16_rn(y);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(128) fact_splitk_reduce_kernel(const ReduceParams p) {
+  reduce_groups(p, blockIdx.x * (long long)blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+}
+
 // The fused element-wise operation on two adjacent output columns, as packed FP32 pairs
 // (add/mul/fma.f32x2 halve the instruction count of the epilogue, which is issue-bound).
 template <int EPI>
@@ -347,6 +469,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     t_clk0 = clock64();
     t_ns0 = ptx::globaltimer_ns();
   }
+  // With debug bit 256 the first CTA also counts where its cycles go (status[2..]: see fact_last_kernel_profile).
+  const bool prof = (p.debug & 256) && blockIdx.x == 0;
   const int unit0 = (int)(blockIdx.x / CG);
   const int unit_stride = (int)(gridDim.x / CG);
   // a bounded wait whose verdict is warp-uniform
@@ -438,19 +562,24 @@ __global__ void __launch_bounds__(kThreads, 1)
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      long long prof_acc_wait = 0, prof_full_wait = 0;
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
         const WorkUnit w = decode_unit(p, u);
+        long long t0 = prof ? clock64() : 0;
         if (!wait_all(acce_bar(acc), acc_phase ^ 1u)) {
           ok = false;
           break;
         }
+        if (prof) prof_acc_wait += clock64() - t0;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tile_n);
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (prof) t0 = clock64();
           if (!(p.debug & 1) && !wait_all(full_bar(stage), phase)) {
             ok = false;
             break;
           }
+          if (prof) prof_full_wait += clock64() - t0;
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
           const uint32_t sb = sa + kStageBytesA;
@@ -481,6 +610,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
+      if (prof && lane == 0) {
+        long long* c = reinterpret_cast<long long*>(p.status + 2);
+        c[2] = prof_acc_wait;
+        c[3] = prof_full_wait;
+      }
     }
     __syncwarp();
   } else {
@@ -502,6 +636,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const bool use_r = (EPI == kEpiBiasResidual) && p.r_tma;
       const uint32_t my_row = (uint32_t)lane * 128u;      // this thread's row inside a staging buffer
       const uint32_t swz = (uint32_t)(lane & 7);          // 128-byte swizzle: 16-byte chunk j lives at j ^ (row & 7)
+      long long prof_epi_busy = 0, prof_epi_wait = 0, prof_tiles = 0;
       uint32_t gc = 0;      // chunks this warp has stored so far: buffer = gc % bufs
       uint32_t r_next = 0;  // residual loads have been issued for every chunk counter below this
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
@@ -559,10 +694,13 @@ __global__ void __launch_bounds__(kThreads, 1)
           __syncwarp();
         }
         if (use_r && r_next <= gc && issue_residual(half, gc)) r_next = gc + 1;
+        long long tw = prof ? clock64() : 0;
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
           ok = false;
           break;
         }
+        const long long tb = prof ? clock64() : 0;
+        if (prof) prof_epi_wait += tb - tw;
         ptx::tc_fence_after();
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
         for (int ci = half; ci < n_chunks; ci += 2) {
@@ -675,10 +813,23 @@ __global__ void __launch_bounds__(kThreads, 1)
           if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(acce_bar(acc), 0));
           else ptx::mbar_arrive(acce_bar(acc));
         }
+        if (prof) {
+          prof_epi_busy += clock64() - tb;
+          ++prof_tiles;
+        }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
-      if (lane == 0) ptx::bulk_wait_group<0>();  // every store has left shared memory and reached global memory
+      if (prof && e == 0 && lane == 0) {
+        long long* c = reinterpret_cast<long long*>(p.status + 2);
+        c[4] = prof_epi_busy;
+        c[5] = prof_epi_wait;
+        c[6] = prof_tiles;
+      }
+      if (lane == 0) {
+        ptx::bulk_wait_group<0>();  // every store has left shared memory and reached global memory
+        asm volatile("fence.proxy.async;" ::: "memory");  // ... and is ordered before generic-proxy traffic that follows
+      }
       __syncwarp();
     } else {
       // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
@@ -740,6 +891,60 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   }
 
+  // ------------------------------------------------------------ split-K: reduce in the tail
+  if constexpr (EPI == kEpiPartial) {
+    if (p.fused_reduce) {
+      // Every CTA's partial stores are complete (the epilogue warps waited for their bulk groups).  A
+      // grid-wide barrier -- all CTAs are resident: at most one per SM and never more CTAs than SMs --
+      // then every thread of the grid reduces its share of the output in ascending slice order.
+      __syncthreads();
+      volatile int* arrived = p.status + 24;
+      int* leaving = p.status + 25;
+      if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(p.status + 24, 1);
+        const unsigned long long t0 = ptx::globaltimer_ns();
+        while (*arrived < (int)gridDim.x) {
+          if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {  // bounded: give up, flag, skip the reduction
+            *abort_p = 1;
+            atomicExch(p.status, kDeviceTimeoutCode);
+            break;
+          }
+        }
+        __threadfence();
+      }
+      __syncthreads();
+      if (prof && threadIdx.x == 0) reinterpret_cast<long long*>(p.status + 2)[7] = clock64() - t_clk0;
+      if (!*abort_p) {
+        ReduceParams r;
+        r.ws = p.ws;
+        r.ws_ld = p.ws_ld;
+        r.planes = p.ws_planes;
+        r.splits = p.split_k;
+        r.M = p.M;
+        r.N_out = p.N_out;
+        r.batch = p.batch;
+        r.epi = p.reduce_epi;
+        r.C = p.C;
+        r.ldc = p.ldc;
+        r.strideC = p.strideC;
+        r.out_f32 = p.out_f32;
+        r.bias = p.bias;
+        r.R = p.R;
+        r.ldr = p.ldr;
+        r.strideR = p.strideR;
+        reduce_groups(r, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+      }
+      __syncthreads();
+      // the last CTA to leave resets both counters for the next launch
+      if (threadIdx.x == 0 && atomicAdd(leaving, 1) == (int)gridDim.x - 1) {
+        *arrived = 0;
+        *leaving = 0;
+        __threadfence();
+      }
+    }
+  }
+
   // ------------------------------------------------------------ teardown
   if (*abort_p) {
     // a wait expired somewhere: give copies that may still be in flight time to land
@@ -761,85 +966,6 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc<CG>(tmem_base, p.tmem_cols);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Split-K reduction: adds the S partials of every output element in ascending slice order,
-// applies the epilogue and stores.  One thread per 4 consecutive output columns.
-struct ReduceParams {
-  const float* ws;  // ws[(split * batch + b) * planes + plane][M][ws_ld]
-  long long ws_ld;
-  int planes;
-  int splits;
-  int M, N_out, batch;
-  int epi;
-  void* C;
-  long long ldc, strideC;
-  int out_f32;
-  const __nv_bfloat16* bias;
-  const __nv_bfloat16* R;
-  long long ldr, strideR;
-};
-
-__device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, float bias, float res) {
-  switch (epi) {
-    case kEpiBias: return a + bias;
-    case kEpiBiasRelu: return fmaxf(a + bias, 0.f);
-    case kEpiBiasGeluTanh: return gelu_tanh_f32(a + bias);
-    case kEpiSiluGate: return silu_f32(a) * up;
-    case kEpiBiasResidual: return a + bias + res;
-    default: return a;
-  }
-}
-
-__global__ void __launch_bounds__(128) fact_splitk_reduce_kernel(const ReduceParams p) {
-  const long long groups_per_row = (p.N_out + 3) / 4;
-  const long long total = (long long)p.batch * p.M * groups_per_row;
-  const long long plane_stride = (long long)p.M * p.ws_ld;
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
-       i += (long long)gridDim.x * blockDim.x) {
-    const int gcol = (int)(i % groups_per_row);
-    const long long rm = i / groups_per_row;
-    const int m = (int)(rm % p.M);
-    const int b = (int)(rm / p.M);
-    const int n = gcol * 4;
-    const int nvalid = min(4, p.N_out - n);
-    float a[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
-    const bool gate = p.epi == kEpiSiluGate;
-    const float* base = p.ws + ((long long)b * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
-    const long long slice_stride = (long long)p.batch * p.planes * plane_stride;
-    // Loads of eight slices are issued together, then added in ascending slice order: the order of the
-    // additions (and so the result) depends only on the number of slices.
-    for (int s0 = 0; s0 < p.splits; s0 += 8) {
-      float4 v[8], t[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (s0 + i < p.splits) {
-          const float* ps = base + (long long)(s0 + i) * slice_stride;
-          v[i] = __ldcg(reinterpret_cast<const float4*>(ps));  // ws_ld is a multiple of 4: padding is in bounds
-          if (gate) t[i] = __ldcg(reinterpret_cast<const float4*>(ps + plane_stride));
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (s0 + i < p.splits) {
-          a[0] += v[i].x; a[1] += v[i].y; a[2] += v[i].z; a[3] += v[i].w;
-          if (gate) {
-            up[0] += t[i].x; up[1] += t[i].y; up[2] += t[i].z; up[3] += t[i].w;
-          }
-        }
-      }
-    }
-    for (int j = 0; j < nvalid; ++j) {
-      const float bias = p.bias ? __bfloat162float(p.bias[n + j]) : 0.f;
-      const float res =
-          (p.epi == kEpiBiasResidual) ? __bfloat162float(p.R[(long long)b * p.strideR + (long long)m * p.ldr + n + j]) : 0.f;
-      const float y = reduce_epilogue(p.epi, a[j], up[j], bias, res);
-      const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n + j;
-      if (p.out_f32) reinterpret_cast<float*>(p.C)[off] = y;
-      else reinterpret_cast<__nv_bfloat16*>(p.C)[off] = __float2bfloat16_rn(y);
-    }
   }
 }
 
