@@ -145,10 +145,14 @@ fact_status_t fact_gemm_batched(fact_handle_t handle, int64_t batch, int64_t M, 
 
 /* C = A . B with K cut into `splits` contiguous slices (0 = library's choice)
  *                                              (Section 5.1, Problem 6: long K)
- * Each (tile, slice) writes an FP32 partial to the workspace; a second kernel
- * adds the partials of every element in ascending slice order and stores C.
- * Slice boundaries and the order of additions depend only on (M, N, K, config),
- * so repeated calls return bit-identical results. */
+ * Each (tile, slice) CTA writes an FP32 partial to the workspace.  After a grid-wide barrier in the
+ * tail of the same kernel (the grid never exceeds the SM count, so all CTAs are resident; the wait is
+ * bounded like every other device wait) all threads share out the output and add the partials of
+ * each element in a fixed order: four sums over slices q, q+4, q+8, ... (ascending, q = 0..3), combined
+ * as (s0 + s1) + (s2 + s3); then the epilogue and the store.  Slice boundaries and the order of every
+ * addition depend only on (M, N, K, config), so repeated calls return bit-identical results.  Split-K
+ * calls through one handle must be stream-ordered with respect to each other (they share the handle's
+ * barrier counters), and must not share a workspace while they overlap. */
 fact_status_t fact_gemm_splitk(fact_handle_t handle, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                const void* B, int64_t ldb, fact_blayout_t b_layout, void* C, int64_t ldc,
                                fact_out_t out_type, int splits, const fact_config_t* cfg, void* workspace,
