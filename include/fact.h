@@ -258,7 +258,8 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * otherwise counters[2..7] keep older values.  counters[0] cycles from start to end, [1] the same span
  * in nanoseconds, [2] MMA issuer waiting for a free accumulator (epilogue too slow), [3] MMA issuer waiting
  * for operand stages (loads too slow), [4] one epilogue warp busy from "accumulator ready" to "accumulator
- * released", [5] that warp waiting for an accumulator, [6] tiles that CTA processed, [7] unused. */
+ * released", [5] that warp waiting for an accumulator, [6] tiles that CTA processed, [7] cycles from kernel
+ * entry until the first operand stage was ready (the prologue). */
 fact_status_t fact_last_kernel_profile(fact_handle_t handle, void* cuda_stream, int64_t counters[8]);
 
 /* Text of the most recent CUDA runtime/driver failure seen through this handle

@@ -68,6 +68,7 @@ struct GemmParams {
   int tile_n;        // accumulator columns per tile (UMMA N)
   int out_cols;      // output columns per tile: tile_n, or tile_n / 2 for SILU_GATE
   int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
+  int k_base, k_rem;  // k_blocks = split_k * k_base + k_rem: slice s covers k_base (+1 if s < k_rem) k-blocks
   int total_units;   // batch * tiles_m * tiles_n * split_k
   // B operand loads issued by ONE CTA per stage
   int b_loads;       // number of TMA boxes
@@ -112,22 +113,37 @@ struct WorkUnit {
 };
 
 __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
+  // 32-bit unsigned arithmetic only, and no division at all on the common paths (one slice, one batch):
+  // this runs once per tile in every role, on the critical path of short-K tiles.
   WorkUnit w;
-  w.split = u % p.split_k;
-  int t = u / p.split_k;
-  const int per_batch = p.tiles_m * p.tiles_n;
-  w.b = t / per_batch;
-  int r = t - w.b * per_batch;
+  unsigned t = (unsigned)u;
+  if (p.split_k > 1) {
+    w.split = (int)(t % (unsigned)p.split_k);
+    t /= (unsigned)p.split_k;
+    // slices differ by at most one k-block: the first `k_rem` slices take `k_base + 1`
+    const int lead = min(w.split, p.k_rem);
+    w.kb_begin = w.split * p.k_base + lead;
+    w.kb_end = w.kb_begin + p.k_base + (w.split < p.k_rem ? 1 : 0);
+  } else {
+    w.split = 0;
+    w.kb_begin = 0;
+    w.kb_end = p.k_blocks;
+  }
+  unsigned r = t;
+  w.b = 0;
+  if (p.batch > 1) {
+    const unsigned per_batch = (unsigned)(p.tiles_m * p.tiles_n);
+    w.b = (int)(t / per_batch);
+    r = t - (unsigned)w.b * per_batch;
+  }
   // grouped raster: walk `raster_group` m-tiles, then step to the next n-tile
-  const int group_sz = p.raster_group * p.tiles_n;
-  const int g = r / group_sz;
-  const int first_m = g * p.raster_group;
-  const int gm = min(p.raster_group, p.tiles_m - first_m);
-  const int in = r - g * group_sz;
-  w.tm = first_m + in % gm;
-  w.tn = in / gm;
-  w.kb_begin = (int)(((long long)w.split * p.k_blocks) / p.split_k);
-  w.kb_end = (int)(((long long)(w.split + 1) * p.k_blocks) / p.split_k);
+  const unsigned group_sz = (unsigned)(p.raster_group * p.tiles_n);
+  const unsigned g = r / group_sz;
+  const int first_m = (int)g * p.raster_group;
+  const unsigned gm = (unsigned)min(p.raster_group, p.tiles_m - first_m);
+  const unsigned in = r - g * group_sz;
+  w.tn = (int)(in / gm);
+  w.tm = first_m + (int)(in - (unsigned)w.tn * gm);
   return w;
 }
 
@@ -402,6 +418,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
                      const GemmParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const long long t_entry = clock64();
 
   // The warp index is made provably warp-uniform (a shuffle result), and the producer / MMA roles
   // run their loops with all 32 lanes converged, electing one lane only for the instruction that
@@ -430,18 +447,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     return bar_base + 8u * (uint32_t)(2 * kMaxStages + 4 + e * kEpiMaxBufs + b);
   };
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kMaxStages; ++s) {
-      ptx::mbar_init(full_bar(s), 1);
-      ptx::mbar_init(empty_bar(s), 1);
-    }
-    for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(accf_bar(b), 1);
-      ptx::mbar_init(acce_bar(b), kEpiWarps * CG);  // one arrival per epilogue warp of every CTA of the group
-    }
-    for (int e = 0; e < kEpiWarps; ++e)
-      for (int b = 0; b < kEpiMaxBufs; ++b) ptx::mbar_init(res_bar(e, b), 1);
-    *abort_p = 0;
+  // One thread per mbarrier: serial initialisation by a single thread costs about a thousand cycles of prologue.
+  if (threadIdx.x < kNumBarriers) {
+    const int i = (int)threadIdx.x;
+    uint32_t count = 1;                                                                  // full / empty / acc_full / residual
+    if (i >= 2 * kMaxStages + 2 && i < 2 * kMaxStages + 4) count = kEpiWarps * CG;       // acc_empty: one arrival per
+    ptx::mbar_init(bar_base + 8u * (uint32_t)i, count);                                  // epilogue warp of the group
+    if (i == 0) *abort_p = 0;
     ptx::fence_mbar_init();
   }
   if (warp == 0 && lane == 0) {
@@ -449,6 +461,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::prefetch_tensormap(&tmB);
   }
   if (warp == 1) {
+    __syncwarp();  // lanes 0..3 of this warp initialised barriers above: reconverge for the warp-wide allocation
     ptx::tmem_alloc<CG>(smem_base + ctrl_off, p.tmem_cols);
     ptx::tmem_relinquish<CG>();
   }
@@ -562,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      long long prof_acc_wait = 0, prof_full_wait = 0;
+      long long prof_acc_wait = 0, prof_full_wait = 0, prof_first_full = 0;
       for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
         const WorkUnit w = decode_unit(p, u);
         long long t0 = prof ? clock64() : 0;
@@ -579,7 +592,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             ok = false;
             break;
           }
-          if (prof) prof_full_wait += clock64() - t0;
+          if (prof) {
+            const long long now = clock64();
+            prof_full_wait += now - t0;
+            if (prof_first_full == 0) prof_first_full = now - t_entry;
+          }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
           const uint32_t sb = sa + kStageBytesA;
@@ -614,6 +631,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         long long* c = reinterpret_cast<long long*>(p.status + 2);
         c[2] = prof_acc_wait;
         c[3] = prof_full_wait;
+        c[7] = prof_first_full;  // cycles from kernel entry to the first operand stage being ready
       }
     }
     __syncwarp();
@@ -827,8 +845,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         c[6] = prof_tiles;
       }
       if (lane == 0) {
-        ptx::bulk_wait_group<0>();  // every store has left shared memory and reached global memory
-        asm volatile("fence.proxy.async;" ::: "memory");  // ... and is ordered before generic-proxy traffic that follows
+        if (EPI == kEpiPartial) {
+          ptx::bulk_wait_group<0>();  // the reduction in the tail reads these partials: wait until they are in global
+          asm volatile("fence.proxy.async;" ::: "memory");  // memory, and order them before generic-proxy traffic
+        } else {
+          ptx::bulk_wait_group_read<0>();  // shared memory may go once every store has read it; the writes complete
+        }                                  // with the grid
       }
       __syncwarp();
     } else {
