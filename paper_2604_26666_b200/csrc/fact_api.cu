@@ -282,6 +282,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.tiles_n = (int)((q.N_out + p.out_cols - 1) / p.out_cols);
   p.k_blocks = (int)((q.K + kTileK - 1) / kTileK);
   p.split_k = c.split_k;
+  p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
   p.k_base = p.k_blocks / std::max(1, c.split_k);
   p.k_rem = p.k_blocks % std::max(1, c.split_k);
   p.raster_group = std::min(c.raster_group, std::max(1, p.tiles_m));

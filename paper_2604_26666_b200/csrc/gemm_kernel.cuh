@@ -68,6 +68,7 @@ struct GemmParams {
   int tile_n;        // accumulator columns per tile (UMMA N)
   int out_cols;      // output columns per tile: tile_n, or tile_n / 2 for SILU_GATE
   int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
+  int k_serpentine;   // 1: every second tile of a CTA walks K downwards (L2 reuse between waves)
   int k_base, k_rem;  // k_blocks = split_k * k_base + k_rem: slice s covers k_base (+1 if s < k_rem) k-blocks
   int total_units;   // batch * tiles_m * tiles_n * split_k
   // B operand loads issued by ONE CTA per stage
@@ -499,8 +500,13 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
+      int wave = 0;
+      for (int u = unit0; ok && u < p.total_units; u += unit_stride, ++wave) {
         const WorkUnit w = decode_unit(p, u);
+        // Odd waves walk K downwards: the wave before ended at the top of K, so the operand slabs both waves
+        // share (same m-tiles of A, or same n-tiles of B) are met while they are still in L2.  The sum of an
+        // output element is then taken in descending k in those tiles, still fixed by (shape, config).
+        const bool k_down = (wave & 1) && p.k_serpentine;
         const int m0 = (w.tm * CG + (int)cta_rank) * kTileM;
         // first accumulator column this CTA's B boxes feed, and the W column of every box
         const int col0 = (CG == 2) ? (int)cta_rank * (p.tile_n / 2) : 0;
@@ -515,7 +521,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             n_box[i] = w.tn * p.tile_n + col;
           }
         }
-        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+        for (int kbi = w.kb_begin; kbi < w.kb_end; ++kbi) {
+          const int kb = k_down ? (w.kb_end - 1 - (kbi - w.kb_begin)) : kbi;
           if (!wait_all(empty_bar(stage), phase ^ 1u)) {
             ok = false;
             break;
