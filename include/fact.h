@@ -101,7 +101,9 @@ typedef enum { FACT_OP_GEMM = 0, FACT_OP_GEMM_BATCHED = 1, FACT_OP_GEMM_SPLITK =
  *   tile_k       64 (one 128-byte swizzle row of BF16)
  *   stages       depth of the shared-memory ring, 2..8, limited by 227 KB
  *   cta_group    1 or 2
- *   raster_group number of M-tiles walked before moving to the next N-tile (L2 reuse), >= 1
+ *   raster_group G > 0: the scheduler walks groups of G m-tiles (their slab of A/X stays in L2 while the
+ *                n-tiles stream by); G < 0: groups of |G| n-tiles (a slab of B/W stays); 0: the library's
+ *                traffic model chooses
  *   split_k      number of K slices, >= 1 (> 1 needs a workspace)
  *   store_mode   0 = library default, 1 = direct register stores, 2 = shared-memory staged stores */
 typedef struct {

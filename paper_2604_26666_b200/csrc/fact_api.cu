@@ -191,8 +191,23 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   const int smax = max_stages_for(q, c.tile_n, c.cta_group);
   if (c.stages == 0) c.stages = smax;
   if (c.stages < 2 || c.stages > smax) return FACT_ERR_UNSUPPORTED;
-  if (c.raster_group == 0) c.raster_group = 8;
-  if (c.raster_group < 1) return FACT_ERR_INVALID_ARG;
+  if (c.raster_group == 0) {
+    // Raster model.  With a group of G m-tiles the CTAs walk the n-tiles of that group; the group's slab of X
+    // (G * tile_m rows * K) is reused from L2 by every n-tile if it fits there, and W is streamed once per group:
+    // DRAM bytes = X + W * ceil(tiles_m / G).  Grouping n-tiles instead (a negative raster_group) keeps a slab
+    // of W resident and streams X once per group.  G is the largest group whose slab stays within a 32 MB share
+    // of L2; the direction with fewer modelled bytes wins.  (DRAM traffic is not the bound of these kernels, but
+    // on a power-limited part every extra gigabyte costs SM clock: 18 % of run time on the gate/up projection.)
+    const double slab_budget = 32.0 * 1024 * 1024;
+    const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
+    const long long tiles_m = (q.M + c.tile_m - 1) / c.tile_m, tiles_n = (q.N_out + out_cols - 1) / out_cols;
+    const double x_bytes = 2.0 * q.M * q.K, w_bytes = 2.0 * q.Nw() * q.K;
+    const long long gm = std::max<long long>(1, std::min<long long>(tiles_m, (long long)(slab_budget / (2.0 * c.tile_m * std::max<long long>(q.K, 1)))));
+    const long long gn = std::max<long long>(1, std::min<long long>(tiles_n, (long long)(slab_budget / (2.0 * c.tile_n * std::max<long long>(q.K, 1)))));
+    const double cost_m = x_bytes + w_bytes * (double)((tiles_m + gm - 1) / gm);
+    const double cost_n = w_bytes + x_bytes * (double)((tiles_n + gn - 1) / gn);
+    c.raster_group = (cost_n < cost_m * 0.95) ? -(int)gn : (int)gm;
+  }
   const int k_blocks = (int)((q.K + kTileK - 1) / kTileK);
   if (c.split_k == 0) {
     c.split_k = 1;
@@ -285,7 +300,9 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
   p.k_base = p.k_blocks / std::max(1, c.split_k);
   p.k_rem = p.k_blocks % std::max(1, c.split_k);
-  p.raster_group = std::min(c.raster_group, std::max(1, p.tiles_m));
+  p.raster_along_n = c.raster_group < 0;
+  p.raster_group = p.raster_along_n ? std::min(-c.raster_group, std::max(1, p.tiles_n))
+                                    : std::min(c.raster_group, std::max(1, p.tiles_m));
   p.stages = c.stages;
   const long long units = (long long)p.batch * p.tiles_m * p.tiles_n * p.split_k;
   if (units > 0x7fffffffLL) return FACT_ERR_UNSUPPORTED;
@@ -738,7 +755,7 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
   cudaEvent_t e0, e1;
   if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return FACT_ERR_CUDA;
 
-  // Candidate axes: pair size, tile width, ring depth, raster group, K slices.
+  // Candidate axes: pair size, tile width, ring depth, K slices.
   std::vector<fact_config_t> cands;
   const int k_blocks = (int)((K + kTileK - 1) / kTileK);
   for (int cg = 1; cg <= 2; ++cg) {
@@ -762,13 +779,13 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
       }
       std::vector<int> stage_opts = {smax};
       if (smax > 3) stage_opts.push_back(smax - 1);
+      // (the raster group is not swept: its effect is on DRAM traffic and, through power, on the clock, which a
+      // short timing run cannot resolve; the model in resolve_config chooses it)
       for (int stg : stage_opts)
-        for (int rg : {2, 8, 32})
-          for (int sp : splits) {
-            if (rg != 8 && (tiles <= slots || stg != smax)) continue;  // raster order only matters over several waves
-            fact_config_t c = {128 * cg, tn, kTileK, stg, cg, rg, sp, 0};
-            cands.push_back(c);
-          }
+        for (int sp : splits) {
+          fact_config_t c = {128 * cg, tn, kTileK, stg, cg, 0, sp, 0};
+          cands.push_back(c);
+        }
     }
   }
   // Time `c` over `n` launches; a negative result means the candidate failed.

@@ -68,6 +68,7 @@ struct GemmParams {
   int tile_n;        // accumulator columns per tile (UMMA N)
   int out_cols;      // output columns per tile: tile_n, or tile_n / 2 for SILU_GATE
   int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
+  int raster_along_n; // 1: the raster groups n-tiles (a slab of W stays in L2), 0: m-tiles (a slab of X)
   int k_serpentine;   // 1: every second tile of a CTA walks K downwards (L2 reuse between waves)
   int k_base, k_rem;  // k_blocks = split_k * k_base + k_rem: slice s covers k_base (+1 if s < k_rem) k-blocks
   int total_units;   // batch * tiles_m * tiles_n * split_k
@@ -137,14 +138,19 @@ __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
     w.b = (int)(t / per_batch);
     r = t - (unsigned)w.b * per_batch;
   }
-  // grouped raster: walk `raster_group` m-tiles, then step to the next n-tile
-  const unsigned group_sz = (unsigned)(p.raster_group * p.tiles_n);
+  // grouped raster: within a group of `raster_group` tiles of the grouped dimension, walk those tiles
+  // fastest and the other dimension slowest; then the next group
+  const int grouped = p.raster_along_n ? p.tiles_n : p.tiles_m;
+  const int other = p.raster_along_n ? p.tiles_m : p.tiles_n;
+  const unsigned group_sz = (unsigned)(p.raster_group * other);
   const unsigned g = r / group_sz;
-  const int first_m = (int)g * p.raster_group;
-  const unsigned gm = (unsigned)min(p.raster_group, p.tiles_m - first_m);
+  const int first = (int)g * p.raster_group;
+  const unsigned gsz = (unsigned)min(p.raster_group, grouped - first);
   const unsigned in = r - g * group_sz;
-  w.tn = (int)(in / gm);
-  w.tm = first_m + (int)(in - (unsigned)w.tn * gm);
+  const int o = (int)(in / gsz);
+  const int gi = first + (int)(in - (unsigned)o * gsz);
+  w.tm = p.raster_along_n ? o : gi;
+  w.tn = p.raster_along_n ? gi : o;
   return w;
 }
 
