@@ -245,6 +245,13 @@ fact_status_t fact_tune_cache_load(fact_handle_t handle, const char* path);
  * is undefined. */
 fact_status_t fact_device_status(fact_handle_t handle, void* cuda_stream, int* status);
 
+/* Self-test of the bounded-wait path, without faulting or hanging anything: launches one warp that waits on
+ * an mbarrier nothing will ever complete, with a limit of `limit_ms` milliseconds (0 < limit_ms <= 1000).
+ * The wait expires, the kernel records FACT_ERR_DEVICE_TIMEOUT in the handle's status word and returns
+ * normally; the call synchronises the stream and returns FACT_OK if that is what happened.  A following
+ * fact_device_status reports (and clears) the timeout; the context stays usable. */
+fact_status_t fact_selftest_wait_timeout(fact_handle_t handle, void* cuda_stream, double limit_ms);
+
 /* Number of kernels this handle has launched so far (for benchmark reports). */
 int64_t fact_launch_count(fact_handle_t handle);
 

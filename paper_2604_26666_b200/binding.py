@@ -35,7 +35,7 @@ EXPORTED = [
     "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
     "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
-    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile",
+    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
 ]
 
 
@@ -95,6 +95,7 @@ def lib() -> ctypes.CDLL:
     L.fact_device_info.argtypes = [vp, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
     L.fact_last_kernel_clock.argtypes = [vp, vp, POINTER(i64), POINTER(i64)]
     L.fact_last_kernel_profile.argtypes = [vp, vp, POINTER(i64)]
+    L.fact_selftest_wait_timeout.argtypes = [vp, vp, c_double]
     L.fact_last_error.argtypes = [vp]
     L.fact_last_error.restype = c_char_p
     for name in EXPORTED:
@@ -239,6 +240,11 @@ class Handle:
         arr = (c_int64 * 8)()
         _check(lib().fact_last_kernel_profile(self._h, self._stream(stream), arr), "fact_last_kernel_profile")
         return [int(x) for x in arr]
+
+    def selftest_wait_timeout(self, limit_ms: float = 5.0, stream=None):
+        """Run the bounded-wait self-test (fact_selftest_wait_timeout); raises unless the wait gave up cleanly."""
+        _check(lib().fact_selftest_wait_timeout(self._h, self._stream(stream), float(limit_ms)),
+               "fact_selftest_wait_timeout", self._h)
 
     def launch_count(self) -> int:
         return int(lib().fact_launch_count(self._h))

@@ -663,6 +663,20 @@ fact_status_t fact_last_kernel_profile(fact_handle_t h, void* stream, int64_t co
   return FACT_OK;
 }
 
+fact_status_t fact_selftest_wait_timeout(fact_handle_t h, void* stream, double limit_ms) {
+  if (!h || !(limit_ms > 0.0) || limit_ms > 1000.0) return FACT_ERR_INVALID_ARG;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  // d_status[30] receives "the wait gave up" (1) or "the wait returned" (0)
+  if (cudaMemsetAsync(h->d_status + 30, 0xff, sizeof(int), s) != cudaSuccess) return FACT_ERR_CUDA;
+  fact_wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(h->d_status, (unsigned long long)(limit_ms * 1e6), h->d_status + 30);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(h, "wait-timeout self-test launch", e);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return FACT_ERR_CUDA;
+  int gave_up = -1;
+  if (cudaMemcpy(&gave_up, h->d_status + 30, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
+  return gave_up == 1 ? FACT_OK : FACT_ERR_CUDA;
+}
+
 const char* fact_last_error(fact_handle_t h) { return h ? h->last_error.c_str() : ""; }
 
 fact_status_t fact_device_status(fact_handle_t h, void* stream, int* status) {

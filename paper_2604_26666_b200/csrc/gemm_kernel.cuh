@@ -155,7 +155,8 @@ __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
 }
 
 // Bounded mbarrier wait.  Returns false if the wait was abandoned.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                         unsigned long long limit_ns = kWaitLimitNs) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -165,7 +166,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
       const unsigned long long now = ptx::globaltimer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(status, kDeviceTimeoutCode);
         return false;
@@ -1002,6 +1003,21 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::tc_fence_after();
     ptx::tmem_dealloc<CG>(tmem_base, p.tmem_cols);
   }
+}
+
+// Self-test of the give-up path: one warp waits on an mbarrier that nothing will ever complete, with a short
+// limit.  The wait expires, the status word receives the timeout code, the kernel returns normally.
+__global__ void fact_wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns, int* gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  const bool ok = wait_bar(ptx::smem_u32(&bar), 0, &abort_flag, status, limit_ns);
+  if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
 }
 
 }  // namespace fact

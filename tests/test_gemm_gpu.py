@@ -218,3 +218,48 @@ def test_error_codes(h):
                                 c_void_p(C.data_ptr()), 64, 1, 2, None, None, 0, None)
     assert rc == 5
     assert (C == 0).all()
+
+
+# ------------------------------------------------------------------ bounded waits, tuner, raster direction
+def test_an_expired_device_wait_is_reported_and_the_context_survives(h):
+    """Nothing is hung or faulted: a warp waits on a barrier that is never completed, with a 5 ms limit."""
+    assert h.device_status() == 0
+    h.selftest_wait_timeout(5.0)
+    assert h.device_status() == 7  # FACT_ERR_DEVICE_TIMEOUT, reported once ...
+    assert h.device_status() == 0  # ... and cleared
+    case = mk("after_timeout", 200, 264, 520, epilogue="BIAS", layout="NK")
+    check_case(h, case)  # the handle and the context still work
+
+
+def test_raster_along_n_and_along_m_agree(h):
+    case = mk("raster", 1100, 1300, 264, layout="NK")
+    ins = wl.make_inputs(case)
+    outs = [run_gpu(h, ins, case, cfg={"raster_group": g, "tile_n": 128, "cta_group": 1}).clone() for g in (1, 3, -1, -4)]
+    for o in outs[1:]:
+        assert torch.equal(outs[0], o)  # the raster changes the order of tiles, never a value
+    check_case(h, case, cfg={"raster_group": -3}, ins=ins)
+
+
+def test_tuner_returns_a_runnable_config_and_the_table_round_trips(h, tmp_path):
+    case = mk("tune", 512, 384, 520, epilogue="BIAS_RELU", layout="NK")
+    ins = wl.make_inputs(case)
+    dev = "cuda:0"
+    X, W, b = ins.X.to(dev), ins.W.to(dev), ins.bias.to(dev)
+    cfg, ms, n = h.tune("linear", X, W, layout="NK", bias=b, epilogue="BIAS_RELU", warmup=2, iters=5)
+    assert n >= 4 and ms > 0
+    d = cfg.as_dict()
+    assert d["tile_m"] == 128 * d["cta_group"] and d["tile_n"] % 32 == 0 and d["stages"] >= 2
+    got = h.get_config("linear", 1, case.M, case.N, case.K, "BIAS_RELU", "NK").as_dict()
+    assert {k: got[k] for k in ("tile_n", "cta_group", "stages", "split_k")} == \
+           {k: d[k] for k in ("tile_n", "cta_group", "stages", "split_k")}
+    check_case(h, case, ins=ins)  # runs with the tuned entry
+    path = tmp_path / "table.txt"
+    h.tune_cache_save(str(path))
+    from paper_2604_26666_b200.binding import Handle
+    h2 = Handle(0, load_table=False)
+    before = h2.get_config("linear", 1, case.M, case.N, case.K, "BIAS_RELU", "NK").as_dict()
+    h2.tune_cache_load(str(path))
+    after = h2.get_config("linear", 1, case.M, case.N, case.K, "BIAS_RELU", "NK").as_dict()
+    assert {k: after[k] for k in ("tile_n", "cta_group", "stages")} == {k: d[k] for k in ("tile_n", "cta_group", "stages")}
+    assert isinstance(before, dict)
+    h2.close()
