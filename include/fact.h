@@ -208,6 +208,29 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
                           fact_epilogue_t epilogue, const fact_config_t* cfg, void* workspace,
                           size_t workspace_bytes, void* cuda_stream);
 
+/* O = softmax(scale * Q K^T + causal mask) V, fused           (Section 5.2, pattern p1: fused multi-head
+ * attention -- causal for the MiniGPT block; grouped queries, 32 query heads over 8 key/value heads of
+ * dimension 128, for the Llama block, where the paper first expands K/V with repeat_interleave: here the
+ * shared key/value heads are read in place)
+ * Q: BF16 [batch][seq_q][heads_q][head_dim], K and V: BF16 [batch][seq_kv][heads_kv][head_dim], O: BF16 like Q,
+ * each addressed by three strides in elements (batch, token, head; head_dim itself is contiguous), so the
+ * operands may be views into a fused QKV projection or stored heads-first.  Query head h uses key/value
+ * head h / (heads_q / heads_kv).  Scores and probabilities are FP32, P is rounded to BF16 for the second
+ * product, O is accumulated in FP32 and rounded once.  causal != 0 masks keys j > i and requires
+ * seq_q == seq_kv; scale <= 0 means 1 / sqrt(head_dim).
+ * Requirements: head_dim 64 or 128; heads_q a multiple of heads_kv; all four pointers 16-byte aligned and
+ * every stride a multiple of 8 elements (operands are read through TMA, O rows are written as 16-byte
+ * vectors).  Errors: FACT_ERR_UNSUPPORTED for another head_dim or causal with seq_q != seq_kv,
+ * FACT_ERR_BAD_ALIGNMENT, FACT_ERR_INVALID_ARG; nothing is launched on an error.  batch == 0 or
+ * seq_q == 0 is a successful no-op. */
+fact_status_t fact_attention(fact_handle_t handle, int64_t batch, int64_t seq_q, int64_t seq_kv, int64_t heads_q,
+                             int64_t heads_kv, int64_t head_dim, const void* Q, int64_t q_stride_batch,
+                             int64_t q_stride_token, int64_t q_stride_head, const void* K, int64_t k_stride_batch,
+                             int64_t k_stride_token, int64_t k_stride_head, const void* V, int64_t v_stride_batch,
+                             int64_t v_stride_token, int64_t v_stride_head, void* O, int64_t o_stride_batch,
+                             int64_t o_stride_token, int64_t o_stride_head, int causal, float scale,
+                             void* cuda_stream);
+
 /* The configuration the library would run for this problem when cfg == NULL
  * (its tuned entry if fact_tune / fact_tune_cache_load provided one, else a
  * heuristic).  The paper's counterpart is the lookup in its pattern table

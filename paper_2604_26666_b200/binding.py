@@ -35,7 +35,7 @@ EXPORTED = [
     "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
     "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
-    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
+    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout", "fact_attention",
 ]
 
 
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
                                     cfgp, vp, sz, vp]
     L.fact_gemm_splitk.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, c_int, cfgp, vp, sz, vp]
     L.fact_gemm_splitk_static.argtypes = [c_int, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, c_int, vp]
+    L.fact_attention.argtypes = [vp, i64, i64, i64, i64, i64, i64, vp, i64, i64, i64, vp, i64, i64, i64, vp, i64, i64, i64,
+                                 vp, i64, i64, i64, c_int, ctypes.c_float, vp]
     L.fact_linear.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, vp, i64, vp, i64, c_int, c_int, cfgp,
                               vp, sz, vp]
     L.fact_get_config.argtypes = [vp, c_int, i64, i64, i64, i64, c_int, c_int, c_int, cfgp]
@@ -244,7 +246,7 @@ class Handle:
     def selftest_wait_timeout(self, limit_ms: float = 5.0, stream=None):
         """Run the bounded-wait self-test (fact_selftest_wait_timeout); raises unless the wait gave up cleanly."""
         _check(lib().fact_selftest_wait_timeout(self._h, self._stream(stream), float(limit_ms)),
-               "fact_selftest_wait_timeout", self._h)
+               "fact_selftest_wait_timeout", "fact_attention", self._h)
 
     def launch_count(self) -> int:
         return int(lib().fact_launch_count(self._h))
@@ -350,6 +352,23 @@ class Handle:
                                  _ptr(residual), _ld(residual) if residual is not None else 0, _ptr(out), _ld(out),
                                  OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg), _ptr(ws), nws,
                                  self._stream(stream)), "fact_linear", self._h)
+        return out
+
+    def attention(self, q, k, v, causal=True, scale=0.0, out=None, stream=None):
+        """O = softmax(scale * Q K^T + causal mask) V  (fact_attention).
+        q: [B, Tq, Hq, D], k / v: [B, Tk, Hkv, D] BF16 CUDA tensors (any strides with contiguous head_dim, e.g.
+        slices of a fused QKV projection); returns [B, Tq, Hq, D]."""
+        for name, t in (("q", q), ("k", k), ("v", v)):
+            _need(t, name, torch.bfloat16, 4)
+        B, Tq, Hq, D = q.shape
+        _, Tk, Hkv, _ = k.shape
+        if out is None:
+            out = torch.empty((B, Tq, Hq, D), dtype=torch.bfloat16, device=q.device)
+        _need(out, "out", torch.bfloat16, 4)
+        st = lambda t: (int(t.stride(0)), int(t.stride(1)), int(t.stride(2)))
+        _check(lib().fact_attention(self._h, B, Tq, Tk, Hq, Hkv, D, _ptr(q), *st(q), _ptr(k), *st(k), _ptr(v), *st(v),
+                                    _ptr(out), *st(out), 1 if causal else 0, float(scale), self._stream(stream)),
+               "fact_attention", self._h)
         return out
 
     def tune(self, op, A, B, layout="KN", bias=None, residual=None, epilogue="NONE", out=None,

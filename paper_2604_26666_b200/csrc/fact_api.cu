@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -16,6 +17,7 @@
 
 #include "fact.h"
 #include "gemm_kernel.cuh"
+#include "attention_kernel.cuh"
 
 // Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
 // device image, so that entry point never has to allocate.  Every GPU that loads the library holds these
@@ -907,6 +909,99 @@ fact_status_t fact_tune_cache_load(fact_handle_t h, const char* path) {
   }
   fclose(f);
   return FACT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fused multi-head attention
+namespace {
+// Rank-4 BF16 tensor map over [B][T][H][D]-like storage, dims ordered (D, H, T, B), box 64 x 1 x 128 x 1.
+fact_status_t encode_map_bthd(fact_handle_t h, CUtensorMap* map, const void* base, long long D, long long H, long long T,
+                              long long B, long long stride_h, long long stride_t, long long stride_b) {
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2, (cuuint64_t)stride_b * 2};
+  cuuint32_t box[4] = {64, 1, (cuuint32_t)kAttnBlockQ, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    h->last_error = "cuTensorMapEncodeTiled (attention operand) failed with CUresult " + std::to_string((int)r);
+    return FACT_ERR_CUDA;
+  }
+  return FACT_OK;
+}
+}  // namespace
+
+fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int64_t seq_kv, int64_t heads_q,
+                             int64_t heads_kv, int64_t head_dim, const void* Q, int64_t q_sb, int64_t q_st,
+                             int64_t q_sh, const void* K, int64_t k_sb, int64_t k_st, int64_t k_sh, const void* V,
+                             int64_t v_sb, int64_t v_st, int64_t v_sh, void* O, int64_t o_sb, int64_t o_st,
+                             int64_t o_sh, int causal, float scale, void* stream_v) {
+  if (!h) return FACT_ERR_INVALID_ARG;
+  if (batch < 0 || seq_q < 0 || seq_kv < 0 || heads_q <= 0 || heads_kv <= 0 || heads_q % heads_kv) return FACT_ERR_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return FACT_ERR_UNSUPPORTED;
+  if (batch == 0 || seq_q == 0) return FACT_OK;
+  if (seq_kv == 0 || !Q || !K || !V || !O) return FACT_ERR_INVALID_ARG;
+  if (causal && seq_q != seq_kv) return FACT_ERR_UNSUPPORTED;
+  if (seq_q > 0x7fffff00LL || seq_kv > 0x7fffff00LL || batch * heads_q > 0x7fffffLL) return FACT_ERR_INVALID_ARG;
+  const int64_t strides[12] = {q_sb, q_st, q_sh, k_sb, k_st, k_sh, v_sb, v_st, v_sh, o_sb, o_st, o_sh};
+  for (int i = 0; i < 12; ++i)
+    if (strides[i] < 0) return FACT_ERR_INVALID_ARG;
+  // head_dim must be contiguous; every other stride a multiple of 8 elements (16 bytes), pointers 16-byte aligned
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return FACT_ERR_BAD_ALIGNMENT;
+  for (int i = 0; i < 12; ++i) {
+    const bool batch_stride = (i % 3) == 0;
+    if (strides[i] % 8) return FACT_ERR_BAD_ALIGNMENT;
+    if (!batch_stride && strides[i] < head_dim) return FACT_ERR_INVALID_ARG;
+  }
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  CUtensorMap tq, tk, tv;
+  auto bs = [&](int64_t s, int64_t fallback) { return (batch > 1 && s > 0) ? s : std::max<int64_t>(fallback, 8); };
+  fact_status_t st = encode_map_bthd(h, &tq, Q, head_dim, heads_q, seq_q, batch, q_sh, q_st, bs(q_sb, q_st * seq_q));
+  if (st == FACT_OK) st = encode_map_bthd(h, &tk, K, head_dim, heads_kv, seq_kv, batch, k_sh, k_st, bs(k_sb, k_st * seq_kv));
+  if (st == FACT_OK) st = encode_map_bthd(h, &tv, V, head_dim, heads_kv, seq_kv, batch, v_sh, v_st, bs(v_sb, v_st * seq_kv));
+  if (st == FACT_OK) {
+    AttnParams p;
+    memset(&p, 0, sizeof p);
+    p.B = (int)batch;
+    p.Tq = (int)seq_q;
+    p.Tk = (int)seq_kv;
+    p.Hq = (int)heads_q;
+    p.Hkv = (int)heads_kv;
+    p.D = (int)head_dim;
+    p.causal = causal != 0;
+    const double sc = scale > 0.f ? (double)scale : 1.0 / std::sqrt((double)head_dim);
+    p.scale_log2 = (float)(sc * 1.4426950408889634);
+    p.q_tiles = (int)((seq_q + kAttnBlockQ - 1) / kAttnBlockQ);
+    p.O = reinterpret_cast<__nv_bfloat16*>(O);
+    p.o_stride_b = o_sb;
+    p.o_stride_t = o_st;
+    p.o_stride_h = o_sh;
+    p.kmajor_desc = smem_desc_template(16, 1024);
+    p.v_desc = smem_desc_template(kAttnBlockK * 128, 1024);  // 64-column chunks of V are one 128-key tile apart
+    p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttnBlockK >> 3) << 17) | ((uint32_t)(kAttnBlockQ >> 4) << 24);
+    p.idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(head_dim >> 3) << 17) |
+                 ((uint32_t)(kAttnBlockQ >> 4) << 24);
+    p.status = h->d_status;
+    const long long ctas = (long long)p.q_tiles * heads_q * batch;
+    const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
+    if (!(h->configured_mask & (1u << 30))) {
+      cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e != cudaSuccess) st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
+      else h->configured_mask |= (1u << 30);
+    }
+    if (st == FACT_OK) {
+      fact_attention_kernel<<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, p);
+      cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
+      else h->launches++;
+    }
+  }
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -1,0 +1,155 @@
+"""GPU parity of fact_attention against the FP64 attention oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.attention import attention as oracle_attention
+from paper_2604_26666_b200 import workloads as wl
+from tests.helpers import gates, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def h():
+    from paper_2604_26666_b200.binding import Handle
+    hd = Handle(0)
+    yield hd
+    hd.close()
+
+
+def rnd(shape, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(shape, generator=g) * scale).to(torch.bfloat16)
+
+
+def attention_gates(q, k, v, causal, got, rows=None, scale=0.0):
+    """(contract ratio, tight ratio).  Contract: |err| <= 1e-2 + 1e-2 |ref| (BF16 output).
+    Tight: |err| <= 2^-8 |ref| + 2^-8 A with A = sum_j p_j |v_j| (the oracle run on |V|): the kernel rounds each
+    probability to BF16 (relative 2^-9) before the second product, so the weighted sum is off by at most 2^-9 A;
+    the row sum is taken from the unrounded probabilities (a normalisation mismatch of at most 2^-9 |ref|) and
+    the result is rounded once more to BF16 (2^-9 |ref|)."""
+    sc = None if scale <= 0 else scale
+    qb, kb, vb = wl.bits(q.contiguous()), wl.bits(k.contiguous()), wl.bits(v.contiguous())
+    ref = oracle_attention(qb, kb, vb, causal=causal, scale=sc, rows=rows)
+    absv = oracle_attention(qb, kb, vb & np.uint16(0x7FFF), causal=causal, scale=sc, rows=rows)
+    err = np.abs(got - ref)
+    contract = float((err / (1e-2 + 1e-2 * np.abs(ref))).max())
+    tight = float((err / (2.0 ** -8 * np.abs(ref) + 2.0 ** -8 * absv + 1e-30)).max())
+    return contract, tight
+
+
+def check(h, q, k, v, causal, rows=None, scale=0.0):
+    dev = "cuda:0"
+    out = h.attention(q.to(dev), k.to(dev), v.to(dev), causal=causal, scale=scale)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    got = to_f64(out)
+    if rows is not None:
+        got = got[:, rows]
+    assert np.isfinite(got).all()
+    c, t = attention_gates(q, k, v, causal, got, rows=rows, scale=scale)
+    assert c <= 1.0, f"contract gate ratio {c:.3f}"
+    assert t <= 1.0, f"tight gate ratio {t:.3f}"
+    return out
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("T", [128, 200, 513])
+def test_mha_small(h, causal, D, T):
+    B, H = 2, 3
+    check(h, rnd((B, T, H, D), 1), rnd((B, T, H, D), 2), rnd((B, T, H, D), 3), causal)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_grouped_queries(h, causal):
+    B, T, Hq, Hkv, D = 2, 300, 8, 2, 128
+    check(h, rnd((B, T, Hq, D), 4), rnd((B, T, Hkv, D), 5), rnd((B, T, Hkv, D), 6), causal)
+
+
+def test_cross_attention_lengths(h):
+    # non-causal with different query and key lengths, both ragged
+    B, H, D = 1, 2, 64
+    check(h, rnd((B, 77, H, D), 7), rnd((B, 391, H, D), 8), rnd((B, 391, H, D), 9), False)
+
+
+def test_views_into_a_fused_qkv_projection(h):
+    # Q, K, V are column slices of one [tokens, (Hq + 2 Hkv) D] matrix, as the QKV linear produces them
+    B, T, Hq, Hkv, D = 2, 260, 4, 2, 64
+    fused = rnd((B, T, (Hq + 2 * Hkv) * D), 10)
+    q = fused[..., : Hq * D].view(B, T, Hq, D)
+    k = fused[..., Hq * D: (Hq + Hkv) * D].view(B, T, Hkv, D)
+    v = fused[..., (Hq + Hkv) * D:].view(B, T, Hkv, D)
+    dev = "cuda:0"
+    fd = fused.to(dev)
+    qd = fd[..., : Hq * D].view(B, T, Hq, D)
+    kd = fd[..., Hq * D: (Hq + Hkv) * D].view(B, T, Hkv, D)
+    vd = fd[..., (Hq + Hkv) * D:].view(B, T, Hkv, D)
+    out = h.attention(qd, kd, vd, causal=True)
+    torch.cuda.synchronize()
+    c, t = attention_gates(q, k, v, True, to_f64(out))
+    assert c <= 1.0 and t <= 1.0, (c, t)
+
+
+def test_heads_first_storage(h):
+    # [B, H, T, D] storage viewed as [B, T, H, D]: the head stride is larger than the token stride
+    B, T, H, D = 1, 140, 3, 128
+    qs, ks, vs = (rnd((B, H, T, D), s) for s in (11, 12, 13))
+    dev = "cuda:0"
+    out_store = torch.empty((B, H, T, D), dtype=torch.bfloat16, device=dev)
+    h.attention(qs.to(dev).permute(0, 2, 1, 3), ks.to(dev).permute(0, 2, 1, 3), vs.to(dev).permute(0, 2, 1, 3),
+                causal=True, out=out_store.permute(0, 2, 1, 3))
+    torch.cuda.synchronize()
+    c, t = attention_gates(qs.permute(0, 2, 1, 3), ks.permute(0, 2, 1, 3), vs.permute(0, 2, 1, 3), True,
+                           to_f64(out_store.permute(0, 2, 1, 3)))
+    assert c <= 1.0 and t <= 1.0, (c, t)
+
+
+def test_closed_forms(h):
+    B, T, H, D = 1, 300, 2, 64
+    q, k = rnd((B, T, H, D), 14), rnd((B, T, H, D), 15)
+    row = rnd((D,), 16)
+    v = row.expand(B, T, H, D).contiguous()
+    out = check(h, q, k, v, True)
+    # weights sum to one: every output row is the common value row up to the rounding of P
+    assert (out.float().cpu() - row.float()).abs().max() <= 2.0 ** -7 * row.float().abs().max() + 1e-3
+    # first causal row sees only key 0: exact
+    v2 = rnd((B, T, H, D), 17)
+    out = check(h, q, k, v2, True)
+    assert torch.equal(out[:, 0].cpu(), v2[:, 0])
+
+
+def test_large_scores_do_not_overflow(h):
+    B, T, H, D = 1, 256, 1, 64
+    check(h, rnd((B, T, H, D), 18, 6.0), rnd((B, T, H, D), 19, 6.0), rnd((B, T, H, D), 20), True)
+
+
+@pytest.mark.parametrize("name", ["gpt", "llama"])
+def test_block_shapes_sampled_rows(h, name):
+    # the attention shapes of the two transformer blocks at the benchmark token counts
+    if name == "gpt":
+        B, T, Hq, Hkv, D = 16, 1024, 12, 12, 64
+    else:
+        B, T, Hq, Hkv, D = 4, 2048, 32, 8, 128
+    q, k, v = rnd((B, T, Hq, D), 21), rnd((B, T, Hkv, D), 22), rnd((B, T, Hkv, D), 23)
+    rows = np.array(sorted({0, 1, 127, 128, 129, T // 2, T - 129, T - 2, T - 1}), dtype=np.int64)
+    check(h, q, k, v, True, rows=rows)
+
+
+def test_error_codes(h):
+    from paper_2604_26666_b200.binding import FactError
+    dev = "cuda:0"
+    q = torch.zeros(1, 128, 2, 96, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(FactError) as e:
+        h.attention(q, q, q)
+    assert e.value.code == 3  # head_dim 96
+    q = torch.zeros(1, 128, 3, 64, dtype=torch.bfloat16, device=dev)
+    k = torch.zeros(1, 128, 2, 64, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(FactError) as e:
+        h.attention(q, k, k)
+    assert e.value.code == 1  # 3 query heads over 2 key/value heads
+    k = torch.zeros(1, 64, 3, 64, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(FactError) as e:
+        h.attention(q, k, k, causal=True)
+    assert e.value.code == 3  # causal with different lengths
