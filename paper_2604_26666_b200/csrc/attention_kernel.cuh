@@ -214,33 +214,39 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar(S_FREE + (j & 1)));
-      // mask and maximum
+      // Mask and maximum.  Only the block on the diagonal (or the ragged last one) needs the per-key mask; four
+      // independent chains keep the maximum and the sum from serialising on the instruction latency.
       const int key0 = j * kAttnBlockK;
       const int key_limit = min(p.Tk, p.causal ? t_row + 1 : p.Tk) - key0;  // keys [0, key_limit) of this block count
-      float mx = -INFINITY;
+      if (__any_sync(0xffffffffu, key_limit < kAttnBlockK)) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i >= key_limit) sraw[c][i] = 0xff800000u;  // -inf
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float sv = (c * 32 + i < key_limit) ? __uint_as_float(sraw[c][i]) * p.scale_log2 : -INFINITY;
-          sraw[c][i] = __float_as_uint(sv);
-          mx = fmaxf(mx, sv);
-        }
+        for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sraw[c][i]));
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;  // scale > 0
       const float m_new = fmaxf(m, mx);
       const float m_use = (m_new == -INFINITY) ? 0.f : m_new;  // a row with nothing visible yet
       const float alpha = ptx::ex2_approx(m - m_use);
-      float rowsum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pw[64];  // the row's 128 probabilities as BF16 pairs
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          const float p0 = ptx::ex2_approx(__uint_as_float(sraw[c][i]) - m_use);
-          const float p1 = ptx::ex2_approx(__uint_as_float(sraw[c][i + 1]) - m_use);
-          rowsum += p0 + p1;
+          // 2^(scale_log2 * s - m): one fused multiply-add and one ex2 per probability
+          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(sraw[c][i]), p.scale_log2, -m_use));
+          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(sraw[c][i + 1]), p.scale_log2, -m_use));
+          sum4[(i >> 1) & 3] += p0 + p1;
           pw[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
         }
-      l = l * alpha + rowsum;
+      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       m = m_new;
       // P's buffer and O are free once the previous block's second product has completed
       if (j > 0) {
