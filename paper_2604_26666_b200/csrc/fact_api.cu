@@ -975,7 +975,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.causal = causal != 0;
     const double sc = scale > 0.f ? (double)scale : 1.0 / std::sqrt((double)head_dim);
     p.scale_log2 = (float)(sc * 1.4426950408889634);
-    p.q_pairs = (int)((seq_q + 2 * kAttnBlockQ - 1) / (2 * kAttnBlockQ));
+    p.q_tiles = (int)((seq_q + kAttnBlockQ - 1) / kAttnBlockQ);
     p.O = reinterpret_cast<__nv_bfloat16*>(O);
     p.o_stride_b = o_sb;
     p.o_stride_t = o_st;
@@ -986,7 +986,8 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(head_dim >> 3) << 17) |
                  ((uint32_t)(kAttnBlockQ >> 4) << 24);
     p.status = h->d_status;
-    const long long ctas = (long long)p.q_pairs * heads_q * batch;
+    p.debug = h->debug_flags;
+    const long long ctas = (long long)p.q_tiles * heads_q * batch;
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
     if (!(h->configured_mask & (1u << 30))) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
