@@ -1,24 +1,30 @@
 // Fused multi-head attention forward for sm_100a: O = softmax(scale * Q K^T + causal mask) V, BF16 in and out,
 // FP32 scores / probabilities / accumulation, grouped queries (several query heads share one key/value head).
 //
-// One CTA owns 128 query positions of one (batch, query head) and walks the key/value sequence in blocks of 128
-// keys with the online-softmax recurrence (a reference maximum m and row sum l per row; the output accumulator is
-// rescaled by 2^(m_old - m_new) only when the block maximum exceeds m by more than 8, so probabilities stay below
-// 2^8 and the final division by l removes the stale reference exactly).  Roles:
-//   warp 0      TMA producer: the Q tile once, then K and V blocks into two three-stage rings
-//   warp 1      MMA issuer:
-//                 S(j)  = Q K_j^T      tcgen05.mma, M = 128, N = 128, K = head_dim, both operands from shared memory,
-//                                      into one of two score buffers in tensor memory
-//                 O    += P(j) V_j     tcgen05.mma, M = 128, N = head_dim, K = 128, A = P(j) read from tensor memory
-//   warps 2-9   softmax: two threads per query row (warps w and w + 4 share a lane quarter and split the block's
+// Persistent kernel: one CTA per SM walks a static list of work items (a tile of 128 query positions of one
+// (batch, query head)), heaviest first, and streams each tile's key/value sequence in blocks of 128 keys with the
+// online-softmax recurrence (a reference maximum m and row sum l per row; the output accumulator is rescaled by
+// 2^(m_old - m_new) only when the block maximum exceeds m by more than 8, so probabilities stay below 2^8 and the
+// final division by l removes the stale reference exactly).  All roles run ahead across tile boundaries, so the
+// loads, the first product and the Q copy of the next tile overlap the last blocks and the epilogue of this one.
+//   warp 8      TMA producer: K and V blocks into two three-stage rings; the next tile's Q into a staging buffer
+//   warp 9      MMA issuer, one block ahead with the first product:
+//                 Q                    tcgen05.cp from the staging buffer into tensor memory, once per tile
+//                 S(g)  = Q K^T        tcgen05.mma, M = 128, N = 128, K = head_dim, A = Q read from tensor memory
+//                                      (so the product reads only K from shared memory), into score buffer g & 1
+//                 O    += P(g) V       tcgen05.mma, M = 128, N = head_dim, K = 128, A = P(g) read from tensor memory
+//   warps 0-7   softmax: two threads per query row (warps w and w + 4 share a lane quarter and split the block's
 //               keys in halves): tcgen05.ld the scores, mask, maximum (exchanged between the two halves through
 //               shared memory), exponentials, row sum; rescale O in tensor memory when needed; tcgen05.st the BF16
-//               probabilities over the first 64 columns of the score buffer they came from; at the end O / l -> global
-// S(j+1) is issued before the softmax of block j starts, so the softmax warps never wait for the tensor pipe in
-// steady state and the pipe works on S(j+1) and O += P(j-1) V while they compute.  Tensor memory (512 columns):
-// S/P buffer 0 at 0, buffer 1 at 128, O at 256.  P(j) may overwrite S(j) because both threads of a row have read
-// their scores before either stores (the exchange of the maxima orders them), and S(j+2) is issued after
-// O += P(j) V on the same in-order pipe.  Every mbarrier wait is bounded, as in the GEMM kernel.
+//               probabilities over the first 64 columns of the score buffer they came from.  A finished tile's
+//               O is read, released and stored (O / l) inside the first block of the next tile, between storing
+//               that block's probabilities and announcing them, so the last product's latency is never waited for.
+// Tensor memory (512 columns): S/P buffer 0 at 0, buffer 1 at 128, O at 256, Q at 384 (two BF16 values per
+// column; one buffer is enough because the copy of the next tile's Q follows this tile's last first-product on
+// the in-order tensor pipe).  P(g) may overwrite S(g) because both threads of a row have read their scores
+// before either stores (the exchange of the maxima orders them), and S(g+2) is issued after O += P(g) V on the same
+// in-order pipe.  Every mbarrier wait is bounded, as in the GEMM kernel; the named barriers between the two warps
+// of a row are reached unconditionally, also by a warp whose wait gave up.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -30,33 +36,45 @@
 
 namespace fact {
 
-constexpr int kAttnThreads = 320;   // 10 warps
-constexpr int kAttnBlockQ = 128;    // query rows per CTA (= TMEM lanes)
+constexpr int kAttnThreads = 384;   // 12 warps: 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 spare
+constexpr int kAttnBlockQ = 128;    // query rows per tile (= TMEM lanes)
 constexpr int kAttnBlockK = 128;    // keys per block
 constexpr int kAttnStages = 3;      // K and V ring depth
 constexpr uint32_t kAttnChunkBytes = 128 * 128;  // one 64-column chunk of a 128-row tile, 128-byte rows
 constexpr float kAttnRescaleThreshold = 8.f;     // log2 units
+// Registers per thread after the warpgroups rebalance (setmaxnreg): the eight softmax warps take what the other four
+// give back.  A request for more than the CTA's pool holds would block forever, so the host checks before the
+// first launch that the kernel was compiled with at least kAttnRegsAtLaunch registers per thread.
+constexpr int kAttnRegsSoftmax = 208;
+constexpr int kAttnRegsOther = 80;
+constexpr int kAttnRegsAtLaunch = 168;
+static_assert(4 * kAttnRegsOther + 8 * kAttnRegsSoftmax <= 12 * kAttnRegsAtLaunch, "setmaxnreg requests exceed the pool");
 
 struct AttnParams {
   int B, Tq, Tk, Hq, Hkv, D;  // D = 64 or 128
   int causal;
   float scale_log2;           // softmax scale * log2(e)
   int q_tiles;                // ceil(Tq / 128)
+  int items;                  // B * Hq * q_tiles work items, ordered heaviest query tile first
   __nv_bfloat16* O;
   long long o_stride_b, o_stride_t, o_stride_h;  // in elements; head_dim is contiguous
-  uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (Q, K)
+  uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (K)
   uint64_t v_desc;            // UMMA descriptor template, V as an N-major operand
   uint32_t idesc_s, idesc_pv;
-  int* status;                // [0] error word, [2..17] eight 64-bit profile counters (debug bit 256)
+  int* status;                // [0] error word, [2..5] cycles and nanoseconds of the first CTA (debug bit 256)
   int debug;
 };
 
-// Shared-memory carve-up (dynamic, 1024-byte aligned): Q | K[stages] | V[stages] | exchange (2 x 2 x 128 floats) |
-// barriers and control words
+// Shared-memory carve-up (dynamic, 1024-byte aligned): K[stages] | V[stages] | Q staging | exchange (2 x 2 x 128
+// floats) | barriers and control words
 __host__ __device__ constexpr uint32_t attn_tile_bytes(int D) { return (uint32_t)(D / 64) * kAttnChunkBytes; }
 __host__ __device__ constexpr uint32_t attn_smem_bytes(int D) {
-  return attn_tile_bytes(D) * (1u + 2u * kAttnStages) + 2048u + 24u * 8u + 16u;
+  return attn_tile_bytes(D) * (2u * kAttnStages + 1u) + 2048u + 24u * 8u + 16u;
 }
+
+struct AttnTile {
+  int b, h, kvh, t0, nb;
+};
 
 __global__ void __launch_bounds__(kAttnThreads, 1)
     fact_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -69,50 +87,50 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
   }
-  // With debug bit 256 the first CTA counts where its cycles go: [0] CTA cycles, [1] CTA nanoseconds, [2] / [3]
-  // cycles warp 2 waited for scores / spent on them, [4] its blocks, [5] its rescales, [6] cycles the MMA warp
-  // waited for probabilities, [7] cycles from entry to the first scores.
   const bool prof = (p.debug & 256) && blockIdx.x == 0;
-  const bool trace = (p.debug & 512) && blockIdx.x == 0;
-  long long* prof_c = reinterpret_cast<long long*>(p.status + 2);
   const long long t_entry = prof ? clock64() : 0;
   const unsigned long long ns_entry = prof ? ptx::globaltimer_ns() : 0ull;
   const uint32_t tile_bytes = attn_tile_bytes(p.D);
-  const uint32_t q_s = smem_base;
-  const uint32_t k_s0 = q_s + tile_bytes;
+  const uint32_t k_s0 = smem_base;
   const uint32_t v_s0 = k_s0 + (uint32_t)kAttnStages * tile_bytes;
-  const uint32_t xch_off = (1u + 2u * kAttnStages) * tile_bytes;  // [parity][half][row] floats
+  const uint32_t q_stage = v_s0 + (uint32_t)kAttnStages * tile_bytes;
+  const uint32_t xch_off = (2u * kAttnStages + 1u) * tile_bytes;  // [parity][half][row] floats
   const uint32_t bar_base = smem_base + xch_off + 2048u;
   const uint32_t ctrl_off = xch_off + 2048u + 24u * 8u;
   float* xch = reinterpret_cast<float*>(smem_raw + xch_off);
   volatile uint32_t* tmem_holder_p = reinterpret_cast<volatile uint32_t*>(smem_raw + ctrl_off);
   volatile int* abort_p = reinterpret_cast<volatile int*>(smem_raw + ctrl_off + 4);
   enum {
-    Q_FULL = 0,
-    K_FULL = 1,
+    QS_FULL = 0,                      // the staging buffer holds a tile's Q (TMA bytes)
+    QS_EMPTY = 1,                     // its copy into tensor memory has completed
+    K_FULL = 2,
     V_FULL = K_FULL + kAttnStages,
     K_EMPTY = V_FULL + kAttnStages,
     V_EMPTY = K_EMPTY + kAttnStages,
-    S_FULL = V_EMPTY + kAttnStages,  // two: one per score buffer
-    P_FULL = S_FULL + 2,
-    PV_DONE = P_FULL + 1,
-    N_BARS = PV_DONE + 1
+    S_FULL = V_EMPTY + kAttnStages,   // two: one per score buffer
+    P_FULL = S_FULL + 2,              // two: a warp may finish block g + 1 before another has finished block g
+    PV_DONE = P_FULL + 2,
+    O_DONE = PV_DONE + 1,             // a tile's last product has completed (PV_DONE's one-bit phase cannot tell
+                                      // "two products behind" from "done", so the epilogue has its own barrier)
+    O_FREE = O_DONE + 1,              // the softmax warps have read a finished tile's O
+    N_BARS = O_FREE + 1
   };
   static_assert(N_BARS <= 24, "barrier area");
   auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
 
   if (threadIdx.x < N_BARS) {
     const int i = (int)threadIdx.x;
-    ptx::mbar_init(bar(i), i == P_FULL ? 8u : 1u);  // one arrival per softmax warp
+    const bool by_softmax = i == P_FULL || i == P_FULL + 1 || i == O_FREE;
+    ptx::mbar_init(bar(i), by_softmax ? 8u : 1u);  // one arrival per softmax warp
     if (i == 0) *abort_p = 0;
     ptx::fence_mbar_init();
   }
-  if (warp == 0 && lane == 0) {
+  if (warp == 8 && lane == 0) {
     ptx::prefetch_tensormap(&tmQ);
     ptx::prefetch_tensormap(&tmK);
     ptx::prefetch_tensormap(&tmV);
   }
-  if (warp == 1) {
+  if (warp == 9) {
     __syncwarp();
     ptx::tmem_alloc<1>(smem_base + ctrl_off, 512);
     ptx::tmem_relinquish<1>();
@@ -122,255 +140,334 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder_p;
   const uint32_t tmem_o = tmem_base + 256u;
+  const uint32_t tmem_q = tmem_base + 384u;
 
-  // this CTA's tile: heavy (late) query tiles of a causal problem are launched first
-  int t = (int)blockIdx.x;
-  const int qt_raw = t % p.q_tiles;
-  t /= p.q_tiles;
-  const int h = t % p.Hq;
-  const int b = t / p.Hq;
-  const int qt = p.causal ? (p.q_tiles - 1 - qt_raw) : qt_raw;
-  const int t0 = qt * kAttnBlockQ;
-  const int kvh = h / (p.Hq / p.Hkv);
+  // This CTA's work items: blockIdx.x, blockIdx.x + gridDim.x, ...  Items are numbered with the query tile as
+  // the slow index, heaviest first (the late tiles of a causal problem), so every CTA gets a similar mix and
+  // neighbouring CTAs work on query heads that share K and V.
+  const int n_items = ((int)blockIdx.x < p.items) ? (p.items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const int kv_blocks_all = (p.Tk + kAttnBlockK - 1) / kAttnBlockK;
-  const int nb = p.causal ? min(kv_blocks_all, qt + 1) : kv_blocks_all;
+  const int bh_count = p.B * p.Hq;
+  auto tile_of = [&](int n) -> AttnTile {
+    const int idx = (int)blockIdx.x + n * (int)gridDim.x;
+    const int qr = idx / bh_count;
+    const int bh = idx - qr * bh_count;
+    const int qt = p.causal ? (p.q_tiles - 1 - qr) : qr;
+    AttnTile t;
+    t.h = bh % p.Hq;
+    t.b = bh / p.Hq;
+    t.kvh = t.h / (p.Hq / p.Hkv);
+    t.t0 = qt * kAttnBlockQ;
+    t.nb = p.causal ? min(kv_blocks_all, qt + 1) : kv_blocks_all;
+    return t;
+  };
   const int chunks = p.D / 64;
   auto wait_all = [&](uint32_t br, uint32_t parity) -> bool {
-    return __all_sync(0xffffffffu, wait_bar(br, parity, abort_p, p.status)) != 0;
+    const bool was_aborted = *abort_p != 0;
+    const bool okw = __all_sync(0xffffffffu, wait_bar(br, parity, abort_p, p.status)) != 0;
+    if (!okw && !was_aborted && lane == 0 && (p.debug & 256))  // which wait gave up first: barrier index, warp, CTA
+      atomicCAS(reinterpret_cast<unsigned long long*>(p.status + 6), 0ull,
+                (unsigned long long)((br - bar_base) / 8u) | ((unsigned long long)warp << 8) |
+                    ((unsigned long long)blockIdx.x << 16) | (1ull << 40));
+    return okw;
   };
 
-  if (warp == 0) {
+  // The softmax warpgroups take the registers the third warpgroup gives back (see kAttnRegsSoftmax).
+  if (warp >= 8) {
+    ptx::setmaxnreg_dec<kAttnRegsOther>();
+  if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
-    if (ptx::elect_one()) {
-      ptx::mbar_arrive_expect_tx(bar(Q_FULL), tile_bytes);
-      for (int c = 0; c < chunks; ++c) ptx::tma_load_4d(q_s + c * kAttnChunkBytes, &tmQ, bar(Q_FULL), c * 64, h, t0, b);
-    }
+    auto load_q = [&](int n) {  // tile n's Q into the staging buffer
+      const AttnTile t = tile_of(n);
+      if (ptx::elect_one()) {
+        ptx::mbar_arrive_expect_tx(bar(QS_FULL), tile_bytes);
+        for (int c = 0; c < chunks; ++c)
+          ptx::tma_load_4d(q_stage + c * kAttnChunkBytes, &tmQ, bar(QS_FULL), c * 64, t.h, t.t0, t.b);
+      }
+    };
+    if (n_items > 0) load_q(0);
     int s = 0;
     uint32_t par = 1;  // an empty slot's first wait passes
-    for (int j = 0; j < nb; ++j) {
-      if (!wait_all(bar(K_EMPTY + s), par)) break;
-      if (ptx::elect_one()) {
-        ptx::mbar_arrive_expect_tx(bar(K_FULL + s), tile_bytes);
-        for (int c = 0; c < chunks; ++c)
-          ptx::tma_load_4d(k_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmK, bar(K_FULL + s), c * 64, kvh,
-                           j * kAttnBlockK, b);
-      }
-      if (!wait_all(bar(V_EMPTY + s), par)) break;
-      if (ptx::elect_one()) {
-        ptx::mbar_arrive_expect_tx(bar(V_FULL + s), tile_bytes);
-        for (int c = 0; c < chunks; ++c)
-          ptx::tma_load_4d(v_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmV, bar(V_FULL + s), c * 64, kvh,
-                           j * kAttnBlockK, b);
-      }
-      if (++s == kAttnStages) {
-        s = 0;
-        par ^= 1u;
+    bool ok = true;
+    for (int n = 0; ok && n < n_items; ++n) {
+      const AttnTile t = tile_of(n);
+      for (int j = 0; ok && j < t.nb; ++j) {
+        ok = wait_all(bar(K_EMPTY + s), par);
+        if (!ok) break;
+        if (ptx::elect_one()) {
+          ptx::mbar_arrive_expect_tx(bar(K_FULL + s), tile_bytes);
+          for (int c = 0; c < chunks; ++c)
+            ptx::tma_load_4d(k_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmK, bar(K_FULL + s), c * 64, t.kvh,
+                             j * kAttnBlockK, t.b);
+        }
+        ok = wait_all(bar(V_EMPTY + s), par);
+        if (!ok) break;
+        if (ptx::elect_one()) {
+          ptx::mbar_arrive_expect_tx(bar(V_FULL + s), tile_bytes);
+          for (int c = 0; c < chunks; ++c)
+            ptx::tma_load_4d(v_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmV, bar(V_FULL + s), c * 64, t.kvh,
+                             j * kAttnBlockK, t.b);
+        }
+        if (++s == kAttnStages) {
+          s = 0;
+          par ^= 1u;
+        }
+        // the next tile's Q follows this tile's first block, once this tile's Q has left the staging buffer
+        if (j == 0 && n + 1 < n_items) {
+          ok = wait_all(bar(QS_EMPTY), (uint32_t)n & 1u);
+          if (ok) load_q(n + 1);
+        }
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
+  } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    bool ok = wait_all(bar(Q_FULL), 0);
-    ptx::tc_fence_after();
-    int ks = 0, vs = 0;          // ring slots of the next K block to multiply and the next V block
+    int ks = 0, vs = 0;  // ring slots of the next K block to multiply and the next V block
     uint32_t kpar = 0, vpar = 0;
-    long long prof_p_wait = 0, prof_kv_wait = 0;
-    auto issue_s = [&](int j) -> bool {  // S(j) = Q K_j^T into score buffer j & 1; releases K_j when done
-      const long long tk = prof ? clock64() : 0;
+    int sn = 0, sj = 0, sg = 0;  // the next first product to issue: tile ordinal, block in the tile, global block
+    int s_nb = n_items > 0 ? tile_of(0).nb : 0;
+    auto issue_next_s = [&]() -> bool {  // S(sg) = Q K^T into score buffer sg & 1; releases the K block when done
+      if (sn >= n_items) return true;
+      if (sj == 0) {  // a new tile: its Q from the staging buffer into tensor memory, 16 elements of every row a copy
+        if (!wait_all(bar(QS_FULL), (uint32_t)sn & 1u)) return false;
+        ptx::tc_fence_after();
+        if (ptx::elect_one()) {
+          for (int kk = 0; kk < p.D / kUmmaK; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * kAttnChunkBytes + (uint32_t)(kk & 3) * 32u;
+            ptx::tmem_cp_128x256b(tmem_q + (uint32_t)kk * 8u, p.kmajor_desc | (uint64_t)(((q_stage + off) >> 4) & 0x3fffu));
+          }
+          ptx::umma_commit<1>(bar(QS_EMPTY));
+        }
+      }
       if (!wait_all(bar(K_FULL + ks), kpar)) return false;
-      if (prof) prof_kv_wait += clock64() - tk;
       ptx::tc_fence_after();
       if (ptx::elect_one()) {
         const uint32_t kaddr = k_s0 + (uint32_t)ks * tile_bytes;
-        const uint32_t d = tmem_base + (uint32_t)(j & 1) * 128u;
-        for (int kk = 0; kk < ((p.debug & 1) ? 0 : p.D / kUmmaK); ++kk) {
+        const uint32_t d = tmem_base + (uint32_t)(sg & 1) * 128u;
+        const uint32_t qa = tmem_q;
+        for (int kk = 0; kk < p.D / kUmmaK; ++kk) {
           const uint32_t off = (uint32_t)(kk >> 2) * kAttnChunkBytes + (uint32_t)(kk & 3) * 32u;
-          const uint64_t adesc = p.kmajor_desc | (uint64_t)(((q_s + off) >> 4) & 0x3fffu);
           const uint64_t bdesc = p.kmajor_desc | (uint64_t)(((kaddr + off) >> 4) & 0x3fffu);
-          ptx::umma_bf16<1>(d, adesc, bdesc, p.idesc_s, kk > 0 ? 1u : 0u);
+          ptx::umma_bf16_ts(d, qa + (uint32_t)kk * 8u, bdesc, p.idesc_s, kk > 0 ? 1u : 0u);  // 8 columns = 16 BF16
         }
-        ptx::umma_commit<1>(bar(S_FULL + (j & 1)));
+        ptx::umma_commit<1>(bar(S_FULL + (sg & 1)));
         ptx::umma_commit<1>(bar(K_EMPTY + ks));
       }
       if (++ks == kAttnStages) {
         ks = 0;
         kpar ^= 1u;
       }
+      ++sg;
+      if (++sj == s_nb) {
+        sj = 0;
+        ++sn;
+        s_nb = sn < n_items ? tile_of(sn).nb : 0;
+      }
       return true;
     };
-    if (ok && nb > 0) ok = issue_s(0);
-    for (int j = 0; ok && j < nb; ++j) {
-      // score buffer (j + 1) & 1 held P(j-1), which O += P(j-1) V (issued in the previous iteration) reads first
-      if (j + 1 < nb && !issue_s(j + 1)) break;
-      if (trace && lane == 0 && (j == 6 || j == 7)) prof_c[j == 6 ? 0 : 3] = clock64() - t_entry;
-      const long long tw = prof ? clock64() : 0;
-      if (!wait_all(bar(P_FULL), (uint32_t)j & 1u)) break;
-      const long long tv = prof ? clock64() : 0;
-      if (prof) prof_p_wait += tv - tw;
-      if (trace && lane == 0 && j == 6) prof_c[1] = clock64() - t_entry;
-      if (!wait_all(bar(V_FULL + vs), vpar)) break;
-      if (prof) prof_kv_wait += clock64() - tv;
-      ptx::tc_fence_after();
-      if (ptx::elect_one()) {  // O += P(j) V_j
-        const uint32_t vaddr = v_s0 + (uint32_t)vs * tile_bytes;
-        const uint32_t p_t = tmem_base + (uint32_t)(j & 1) * 128u;  // BF16 pairs: 8 columns per 16 keys
-        for (int kk = 0; kk < ((p.debug & 2) ? 0 : kAttnBlockK / kUmmaK); ++kk) {
-          const uint64_t bdesc = p.v_desc | (uint64_t)(((vaddr + (uint32_t)kk * 2048u) >> 4) & 0x3fffu);
-          ptx::umma_bf16_ts(tmem_o, p_t + (uint32_t)kk * 8u, bdesc, p.idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+    bool ok = issue_next_s();
+    int g = 0;
+    for (int n = 0; ok && n < n_items; ++n) {
+      const int nb = tile_of(n).nb;
+      for (int j = 0; ok && j < nb; ++j, ++g) {
+        // score buffer (g + 1) & 1 held P(g-1), which O += P(g-1) V (issued in the previous iteration) reads first
+        ok = issue_next_s();
+        if (!ok) break;
+        ok = wait_all(bar(P_FULL + (g & 1)), ((uint32_t)g >> 1) & 1u);
+        // the first block of a tile overwrites O: the previous tile's epilogue must have read it
+        if (ok && j == 0 && n > 0) ok = wait_all(bar(O_FREE), (uint32_t)(n - 1) & 1u);
+        if (ok) ok = wait_all(bar(V_FULL + vs), vpar);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        if (ptx::elect_one()) {  // O += P(g) V
+          const uint32_t vaddr = v_s0 + (uint32_t)vs * tile_bytes;
+          const uint32_t p_t = tmem_base + (uint32_t)(g & 1) * 128u;  // BF16 pairs: 8 columns per 16 keys
+          for (int kk = 0; kk < kAttnBlockK / kUmmaK; ++kk) {
+            const uint64_t bdesc = p.v_desc | (uint64_t)(((vaddr + (uint32_t)kk * 2048u) >> 4) & 0x3fffu);
+            ptx::umma_bf16_ts(tmem_o, p_t + (uint32_t)kk * 8u, bdesc, p.idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+          }
+          ptx::umma_commit<1>(bar(V_EMPTY + vs));
+          ptx::umma_commit<1>(bar(PV_DONE));
+          if (j == nb - 1) ptx::umma_commit<1>(bar(O_DONE));
         }
-        ptx::umma_commit<1>(bar(V_EMPTY + vs));
-        ptx::umma_commit<1>(bar(PV_DONE));
+        if (++vs == kAttnStages) {
+          vs = 0;
+          vpar ^= 1u;
+        }
       }
-      if (trace && lane == 0 && j == 6) prof_c[2] = clock64() - t_entry;
-      if (++vs == kAttnStages) {
-        vs = 0;
-        vpar ^= 1u;
-      }
-    }
-    if (prof && !trace && lane == 0) {
-      prof_c[6] = prof_p_wait;
-      prof_c[7] = prof_kv_wait;
     }
     __syncwarp();
+  }
   } else {
+    ptx::setmaxnreg_inc<kAttnRegsSoftmax>();
     // ------------------------------------------------------------ softmax warps: two threads per query row
-    const int half = (warp - 2) >> 2;  // which 64 keys of every block this thread owns
+    const int half = warp >> 2;        // which 64 keys of every block this thread owns
     const int q4 = warp & 3;           // the TMEM lane quarter this warp may access
     const int row = q4 * 32 + lane;
-    const int t_row = t0 + row;
     const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
     const uint32_t pair_bar = 1u + (uint32_t)q4;  // named barrier of this warp and its partner (warp +- 4)
     const int o_cols = p.D / 2;                   // output columns this thread rescales and stores
     const uint32_t o_addr = tmem_o + lane_addr + (uint32_t)(half * o_cols);
-    float m = -INFINITY;  // reference maximum of scale_log2 * score the exponentials are taken against
-    float l = 0.f;        // this thread's part of the running sum of 2^(scale_log2 * score - m)
-    bool ok = true;       // warp-uniform; a warp whose wait gave up keeps meeting its partner at the named barrier
-    long long prof_wait = 0, prof_busy = 0, prof_first = 0, prof_rescales = 0;
-    for (int j = 0; j < nb; ++j) {
-      const long long tw = prof ? clock64() : 0;
-      if (ok) ok = wait_all(bar(S_FULL + (j & 1)), ((uint32_t)j >> 1) & 1u);
-      const long long tb = prof ? clock64() : 0;
-      if (prof) {
-        prof_wait += tb - tw;
-        if (j == 0) prof_first = tb - t_entry;
+    bool ok = true;  // warp-uniform; a warp whose wait gave up keeps meeting its partner at the named barriers
+    long long prof_s_wait = 0, prof_epi = 0, prof_blocks = 0;
+    // A finished tile whose output has not been stored yet: this thread's part of the row sums, where its half
+    // row goes (null for a row past the end), and the tile's ordinal.
+    bool pend = false;
+    float pend_l = 0.f;
+    int pend_n = 0;
+    __nv_bfloat16* pend_row = nullptr;
+    // O / l -> global for the pending tile.  The row sum is the sum of the two halves', exchanged through the
+    // buffer `xbuf` that the latest exchange of maxima did not use; the second barrier keeps the next block's
+    // maxima from overwriting a sum not yet read.  O is read into registers and released before the stores, so the
+    // next tile's products may overwrite it while they drain.
+    auto finish_tile = [&](int xbuf) {
+      const long long te0 = prof ? clock64() : 0;
+      pend = false;
+      float* xl = xch + xbuf * 256;
+      xl[half * 128 + row] = pend_l;
+      ptx::named_bar_sync(pair_bar, 64);
+      const float lsum = pend_l + xl[(half ^ 1) * 128 + row];
+      ptx::named_bar_sync(pair_bar, 64);
+      if (ok) ok = wait_all(bar(O_DONE), (uint32_t)pend_n & 1u);
+      if (!ok) return;
+      ptx::tc_fence_after();
+      uint32_t o[2][32];
+      ptx::tmem_ld_32x32b_x32(o_addr, o[0]);
+      if (o_cols > 32) ptx::tmem_ld_32x32b_x32(o_addr + 32u, o[1]);
+      ptx::tmem_wait_ld();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar(O_FREE));
+      if (pend_row != nullptr) {
+        const float inv = (lsum > 0.f) ? __fdividef(1.f, lsum) : 0.f;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          if (c * 32 < o_cols) {
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {
+              uint4 qv;
+              qv.x = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 0]) * inv, __uint_as_float(o[c][gq * 8 + 1]) * inv);
+              qv.y = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 2]) * inv, __uint_as_float(o[c][gq * 8 + 3]) * inv);
+              qv.z = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 4]) * inv, __uint_as_float(o[c][gq * 8 + 5]) * inv);
+              qv.w = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 6]) * inv, __uint_as_float(o[c][gq * 8 + 7]) * inv);
+              *reinterpret_cast<uint4*>(pend_row + c * 32 + gq * 8) = qv;
+            }
+          }
+        }
       }
-      if (trace && warp == 2 && lane == 0 && (j == 6 || j == 7)) prof_c[j == 6 ? 4 : 6] = clock64() - t_entry;
-      const uint32_t buf = tmem_base + lane_addr + (uint32_t)(j & 1) * 128u;
-      uint32_t sraw[2][32];
-      float hm = -INFINITY;
-      if (ok) {
-        ptx::tc_fence_after();
-        ptx::tmem_ld_32x32b_x32(buf + (uint32_t)half * 64u, sraw[0]);
-        ptx::tmem_ld_32x32b_x32(buf + (uint32_t)half * 64u + 32u, sraw[1]);
-        ptx::tmem_wait_ld();
-        // Only the block on the diagonal (or the ragged last one) needs the per-key mask.
-        const int key_limit = min(p.Tk, p.causal ? t_row + 1 : p.Tk) - (j * kAttnBlockK + half * 64);
-        if (__any_sync(0xffffffffu, key_limit < 64)) {
+      if (prof) prof_epi += clock64() - te0;
+    };
+    int g = 0;  // global block counter
+    for (int n = 0; n < n_items; ++n) {
+      const AttnTile tile = tile_of(n);
+      const int nb = tile.nb;
+      const int t_row = tile.t0 + row;
+      float m = -INFINITY;  // reference maximum of scale_log2 * score the exponentials are taken against
+      float l = 0.f;        // this thread's part of the running sum of 2^(scale_log2 * score - m)
+      for (int j = 0; j < nb; ++j, ++g) {
+        const long long tc1 = prof ? clock64() : 0;
+        if (ok) ok = wait_all(bar(S_FULL + (g & 1)), ((uint32_t)g >> 1) & 1u);
+        if (prof) {
+          prof_s_wait += clock64() - tc1;
+          ++prof_blocks;
+        }
+        const uint32_t buf = tmem_base + lane_addr + (uint32_t)(g & 1) * 128u;
+        uint32_t sraw[2][32];
+        float hm = -INFINITY;
+        if (ok) {
+          ptx::tc_fence_after();
+          ptx::tmem_ld_32x32b_x32(buf + (uint32_t)half * 64u, sraw[0]);
+          ptx::tmem_ld_32x32b_x32(buf + (uint32_t)half * 64u + 32u, sraw[1]);
+          ptx::tmem_wait_ld();
+          // Only the block on the diagonal (or the ragged last one) needs the per-key mask.
+          const int key_limit = min(p.Tk, p.causal ? t_row + 1 : p.Tk) - (j * kAttnBlockK + half * 64);
+          if (__any_sync(0xffffffffu, key_limit < 64)) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i >= key_limit) sraw[c][i] = 0xff800000u;  // -inf
+          }
+          // four independent chains of three-input maxima
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int c = 0; c < 2; ++c)
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i >= key_limit) sraw[c][i] = 0xff800000u;  // -inf
+            for (int i = 0; i < 32; i += 2)
+              mx4[(i >> 1) & 3] = ptx::max3(mx4[(i >> 1) & 3], __uint_as_float(sraw[c][i]), __uint_as_float(sraw[c][i + 1]));
+          hm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         }
-        // four independent chains of three-input maxima
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        // the row maximum is the larger of the two halves'; passing the barrier also tells each thread that its
+        // partner has read its scores, so the probabilities may now overwrite them
+        float* xj = xch + (g & 1) * 256;
+        xj[half * 128 + row] = hm;
+        ptx::named_bar_sync(pair_bar, 64);
+        if (!ok) {
+          if (j == 0 && pend) finish_tile((g + 1) & 1);  // keeps the pair's barrier sequence identical
+          continue;
+        }
+        const float mx = fmaxf(hm, xj[(half ^ 1) * 128 + row]) * p.scale_log2;  // scale > 0
+        // Move the reference maximum only when this block exceeds it by more than the threshold (always from
+        // -inf); both threads of a row take the same decision from the same numbers.
+        if (__any_sync(0xffffffffu, mx > m + kAttnRescaleThreshold)) {
+          const float m_new = fmaxf(m, mx);
+          const float alpha = ptx::ex2_approx(m - ((m_new == -INFINITY) ? 0.f : m_new));
+          l *= alpha;
+          m = m_new;
+          if (j > 0) {
+            // O is rescaled between O += P(g-1) V, which must have completed, and O += P(g) V, which waits for P(g)
+            ok = wait_all(bar(PV_DONE), (uint32_t)(g - 1) & 1u);
+            if (!ok) continue;  // j > 0: no finished tile is pending here
+            ptx::tc_fence_after();
+            for (int c = 0; c < o_cols; c += 32) {
+              uint32_t o[32];
+              ptx::tmem_ld_32x32b_x32(o_addr + (uint32_t)c, o);
+              ptx::tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              ptx::tmem_st_32x32b_x32(o_addr + (uint32_t)c, o);
+            }
+          }
+        }
+        const float m_use = (m == -INFINITY) ? 0.f : m;  // a row with nothing visible yet
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pw[32];  // this thread's 64 probabilities as BF16 pairs
 #pragma unroll
         for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; i += 2)
-            mx4[(i >> 1) & 3] = ptx::max3(mx4[(i >> 1) & 3], __uint_as_float(sraw[c][i]), __uint_as_float(sraw[c][i + 1]));
-        hm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      }
-      // the row maximum is the larger of the two halves'; passing the barrier also tells each thread that its
-      // partner has read its scores, so the probabilities may now overwrite them
-      float* xj = xch + (j & 1) * 256;
-      xj[half * 128 + row] = hm;
-      ptx::named_bar_sync(pair_bar, 64);
-      if (!ok) continue;
-      const float mx = fmaxf(hm, xj[(half ^ 1) * 128 + row]) * p.scale_log2;  // scale > 0
-      // Move the reference maximum only when this block exceeds it by more than the threshold (always from -inf);
-      // both threads of a row take the same decision from the same numbers.
-      if (__any_sync(0xffffffffu, mx > m + kAttnRescaleThreshold)) {
-        const float m_new = fmaxf(m, mx);
-        const float alpha = ptx::ex2_approx(m - ((m_new == -INFINITY) ? 0.f : m_new));
-        l *= alpha;
-        m = m_new;
-        if (prof) ++prof_rescales;
-        if (j > 0) {
-          // O is rescaled between O += P(j-1) V, which must have completed, and O += P(j) V, which waits for P(j)
-          ok = wait_all(bar(PV_DONE), (uint32_t)(j - 1) & 1u);
-          if (!ok) continue;
-          ptx::tc_fence_after();
-          for (int c = 0; c < o_cols; c += 32) {
-            uint32_t o[32];
-            ptx::tmem_ld_32x32b_x32(o_addr + (uint32_t)c, o);
-            ptx::tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            ptx::tmem_st_32x32b_x32(o_addr + (uint32_t)c, o);
+          for (int i = 0; i < 32; i += 2) {
+            // 2^(scale_log2 * s - m): one fused multiply-add and one ex2 per probability
+            const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(sraw[c][i]), p.scale_log2, -m_use));
+            const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(sraw[c][i + 1]), p.scale_log2, -m_use));
+            sum4[(i >> 1) & 3] += p0 + p1;
+            pw[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
           }
-        }
+        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        // P(g) over the first 64 columns of S(g): lane = row, column c holds keys 2c and 2c + 1
+        ptx::tmem_st_32x32b_x32(buf + (uint32_t)half * 32u, pw);
+        ptx::tmem_wait_st();
+        // The previous tile's O: its last product was issued a whole block ago, and the first product that
+        // overwrites O waits for the probabilities announced below.
+        if (j == 0 && pend) finish_tile((g + 1) & 1);
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar(P_FULL + (g & 1)));
       }
-      const float m_use = (m == -INFINITY) ? 0.f : m;  // a row with nothing visible yet
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pw[32];  // this thread's 64 probabilities as BF16 pairs
-#pragma unroll
-      for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          // 2^(scale_log2 * s - m): one fused multiply-add and one ex2 per probability
-          float p0 = fmaf(__uint_as_float(sraw[c][i]), p.scale_log2, -m_use);
-          float p1 = fmaf(__uint_as_float(sraw[c][i + 1]), p.scale_log2, -m_use);
-          if (!(p.debug & 4)) {
-            p0 = ptx::ex2_approx(p0);
-            p1 = ptx::ex2_approx(p1);
-          }
-          sum4[(i >> 1) & 3] += p0 + p1;
-          pw[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
-        }
-      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      // P(j) over the first 64 columns of S(j): lane = row, column c holds keys 2c and 2c + 1
-      ptx::tmem_st_32x32b_x32(buf + (uint32_t)half * 32u, pw);
-      ptx::tmem_wait_st();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar(P_FULL));
-      if (prof) prof_busy += clock64() - tb;
-      if (trace && warp == 2 && lane == 0 && (j == 6 || j == 7)) prof_c[j == 6 ? 5 : 7] = clock64() - t_entry;
+      // this tile's output is finished inside the next tile's first block (or after the loop)
+      pend = true;
+      pend_l = l;
+      pend_n = n;
+      pend_row = (t_row < p.Tq) ? (p.O + (long long)tile.b * p.o_stride_b + (long long)t_row * p.o_stride_t +
+                                   (long long)tile.h * p.o_stride_h + half * o_cols)
+                                : nullptr;
     }
-    if (prof && !trace && warp == 2 && lane == 0) {
-      prof_c[2] = prof_wait;
-      prof_c[3] = prof_busy;
-      prof_c[4] = nb;
-      prof_c[5] = prof_rescales;
-    }
-    // the row sum is the sum of the two halves' (the exchange buffer of the parity the last block did not use)
-    float* xl = xch + (nb & 1) * 256;
-    xl[half * 128 + row] = l;
-    ptx::named_bar_sync(pair_bar, 64);
-    l += xl[(half ^ 1) * 128 + row];
-    // O / l -> global: each thread stores its half of the row's head_dim BF16 values
-    if (ok && nb > 0 && wait_all(bar(PV_DONE), (uint32_t)(nb - 1) & 1u)) {
-      ptx::tc_fence_after();
-      const float inv = (l > 0.f) ? __fdividef(1.f, l) : 0.f;
-      __nv_bfloat16* dst = p.O + (long long)b * p.o_stride_b + (long long)t_row * p.o_stride_t +
-                           (long long)h * p.o_stride_h + half * o_cols;
-      for (int c = 0; c < o_cols; c += 32) {
-        uint32_t o[32];
-        ptx::tmem_ld_32x32b_x32(o_addr + (uint32_t)c, o);
-        ptx::tmem_wait_ld();
-        if (t_row < p.Tq) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 qv;
-            qv.x = pack_bf16x2(__uint_as_float(o[g * 8 + 0]) * inv, __uint_as_float(o[g * 8 + 1]) * inv);
-            qv.y = pack_bf16x2(__uint_as_float(o[g * 8 + 2]) * inv, __uint_as_float(o[g * 8 + 3]) * inv);
-            qv.z = pack_bf16x2(__uint_as_float(o[g * 8 + 4]) * inv, __uint_as_float(o[g * 8 + 5]) * inv);
-            qv.w = pack_bf16x2(__uint_as_float(o[g * 8 + 6]) * inv, __uint_as_float(o[g * 8 + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + c + g * 8) = qv;
-          }
-        }
-      }
+    if (pend) finish_tile(g & 1);
+    if (prof && warp == 0 && lane == 0) {
+      long long* prof_c = reinterpret_cast<long long*>(p.status + 2);
+      prof_c[3] = prof_s_wait;
+      prof_c[4] = prof_blocks;
+      prof_c[6] = prof_epi;
+      prof_c[7] = n_items;
     }
   }
 
@@ -382,11 +479,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 9) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc<1>(tmem_base, 512);
   }
-  if (prof && !trace && threadIdx.x == 0) {
+  if (prof && threadIdx.x == 0) {
+    long long* prof_c = reinterpret_cast<long long*>(p.status + 2);
     prof_c[0] = clock64() - t_entry;
     prof_c[1] = (long long)(ptx::globaltimer_ns() - ns_entry);
   }

@@ -659,9 +659,13 @@ fact_status_t fact_last_kernel_clock(fact_handle_t h, void* stream, int64_t* sm_
 fact_status_t fact_last_kernel_profile(fact_handle_t h, void* stream, int64_t counters[8]) {
   if (!h || !counters) return FACT_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return FACT_ERR_CUDA;
-  long long v[8];
+  long long v[10];
   if (cudaMemcpy(v, h->d_status + 2, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
   for (int i = 0; i < 8; ++i) counters[i] = v[i];
+  if (h->debug_flags & 2048) {  // attention experiment: entry-to-first-scores and entry-to-last-block in [6], [7]
+    counters[6] = v[8];
+    counters[7] = v[9];
+  }
   return FACT_OK;
 }
 
@@ -987,12 +991,28 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
                  ((uint32_t)(kAttnBlockQ >> 4) << 24);
     p.status = h->d_status;
     p.debug = h->debug_flags;
-    const long long ctas = (long long)p.q_tiles * heads_q * batch;
+    const long long items = (long long)p.q_tiles * heads_q * batch;
+    if (items > 0x7fffffffLL) {
+      if (dev != h->device) cudaSetDevice(dev);
+      return FACT_ERR_UNSUPPORTED;
+    }
+    p.items = (int)items;
+    const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
     if (!(h->configured_mask & (1u << 30))) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-      if (e != cudaSuccess) st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
-      else h->configured_mask |= (1u << 30);
+      cudaFuncAttributes fa;
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel);
+      if (e != cudaSuccess) {
+        st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
+      } else if (fa.numRegs < kAttnRegsAtLaunch) {
+        // the kernel's register rebalancing would wait forever for registers the CTA does not own
+        h->last_error = "attention kernel compiled with " + std::to_string(fa.numRegs) + " registers per thread, needs " +
+                        std::to_string(kAttnRegsAtLaunch);
+        st = FACT_ERR_UNSUPPORTED;
+      } else {
+        h->configured_mask |= (1u << 30);
+      }
     }
     if (st == FACT_OK) {
       fact_attention_kernel<<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, p);

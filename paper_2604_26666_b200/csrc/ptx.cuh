@@ -206,6 +206,11 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, u
       "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Copy 128 rows x 32 bytes from shared memory (a K-major operand slice described like an MMA operand) into 8
+// columns of tensor memory, row r to lane r; ordered with the MMAs and commits this thread issues.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
 // Make `bar` (a shared::cluster address; a CTA-local address names this CTA) receive one
 // arrival once every tcgen05 operation this thread issued so far has completed.
 template <int CG>
@@ -259,6 +264,15 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// Give registers back to / take registers from the SM's pool; every warp of the warpgroup executes the same one.
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
 // max(a, b, c) in one instruction
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
