@@ -13,12 +13,14 @@
 //                 S(g)  = Q K^T        tcgen05.mma, M = 128, N = 128, K = head_dim, A = Q read from tensor memory
 //                                      (so the product reads only K from shared memory), into score buffer g & 1
 //                 O    += P(g) V       tcgen05.mma, M = 128, N = head_dim, K = 128, A = P(g) read from tensor memory
+//   warp 10     store warp: a finished tile's O / l from its staging buffer to global memory by TMA
 //   warps 0-7   softmax: two threads per query row (warps w and w + 4 share a lane quarter and split the block's
 //               keys in halves): tcgen05.ld the scores, mask, maximum (exchanged between the two halves through
 //               shared memory), exponentials, row sum; rescale O in tensor memory when needed; tcgen05.st the BF16
 //               probabilities over the first 64 columns of the score buffer they came from.  A finished tile's
-//               O is read, released and stored (O / l) inside the first block of the next tile, between storing
-//               that block's probabilities and announcing them, so the last product's latency is never waited for.
+//               O is read, released and written (O / l, BF16) to the staging buffer inside the first block of the
+//               next tile, between storing that block's probabilities and announcing them, so the last product's
+//               latency is never waited for.
 // Tensor memory (512 columns): S/P buffer 0 at 0, buffer 1 at 128, O at 256, Q at 384 (two BF16 values per
 // column; one buffer is enough because the copy of the next tile's Q follows this tile's last first-product on
 // the in-order tensor pipe).  P(g) may overwrite S(g) because both threads of a row have read their scores
@@ -39,7 +41,8 @@ namespace fact {
 constexpr int kAttnThreads = 384;   // 12 warps: 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 spare
 constexpr int kAttnBlockQ = 128;    // query rows per tile (= TMEM lanes)
 constexpr int kAttnBlockK = 128;    // keys per block
-constexpr int kAttnStages = 3;      // K and V ring depth
+constexpr int kAttnStagesK = 3;     // K ring depth: a K block is wanted one block before its V block
+constexpr int kAttnStagesV = 2;     // V ring depth
 constexpr uint32_t kAttnChunkBytes = 128 * 128;  // one 64-column chunk of a 128-row tile, 128-byte rows
 constexpr float kAttnRescaleThreshold = 8.f;     // log2 units
 // Registers per thread after the warpgroups rebalance (setmaxnreg): the eight softmax warps take what the other four
@@ -56,8 +59,6 @@ struct AttnParams {
   float scale_log2;           // softmax scale * log2(e)
   int q_tiles;                // ceil(Tq / 128)
   int items;                  // B * Hq * q_tiles work items, ordered heaviest query tile first
-  __nv_bfloat16* O;
-  long long o_stride_b, o_stride_t, o_stride_h;  // in elements; head_dim is contiguous
   uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (K)
   uint64_t v_desc;            // UMMA descriptor template, V as an N-major operand
   uint32_t idesc_s, idesc_pv;
@@ -65,11 +66,11 @@ struct AttnParams {
   int debug;
 };
 
-// Shared-memory carve-up (dynamic, 1024-byte aligned): K[stages] | V[stages] | Q staging | exchange (2 x 2 x 128
-// floats) | barriers and control words
+// Shared-memory carve-up (dynamic, 1024-byte aligned): K ring | V ring | Q staging | O staging | exchange (2 x 2 x
+// 128 floats) | barriers and control words
 __host__ __device__ constexpr uint32_t attn_tile_bytes(int D) { return (uint32_t)(D / 64) * kAttnChunkBytes; }
 __host__ __device__ constexpr uint32_t attn_smem_bytes(int D) {
-  return attn_tile_bytes(D) * (2u * kAttnStages + 1u) + 2048u + 24u * 8u + 16u;
+  return attn_tile_bytes(D) * (uint32_t)(kAttnStagesK + kAttnStagesV + 2) + 2048u + 24u * 8u + 16u;
 }
 
 struct AttnTile {
@@ -78,7 +79,8 @@ struct AttnTile {
 
 __global__ void __launch_bounds__(kAttnThreads, 1)
     fact_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                          const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+                          const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                          const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
@@ -92,9 +94,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const unsigned long long ns_entry = prof ? ptx::globaltimer_ns() : 0ull;
   const uint32_t tile_bytes = attn_tile_bytes(p.D);
   const uint32_t k_s0 = smem_base;
-  const uint32_t v_s0 = k_s0 + (uint32_t)kAttnStages * tile_bytes;
-  const uint32_t q_stage = v_s0 + (uint32_t)kAttnStages * tile_bytes;
-  const uint32_t xch_off = (2u * kAttnStages + 1u) * tile_bytes;  // [parity][half][row] floats
+  const uint32_t v_s0 = k_s0 + (uint32_t)kAttnStagesK * tile_bytes;
+  const uint32_t q_stage = v_s0 + (uint32_t)kAttnStagesV * tile_bytes;
+  const uint32_t o_stage = q_stage + tile_bytes;
+  const uint32_t xch_off = (uint32_t)(kAttnStagesK + kAttnStagesV + 2) * tile_bytes;  // [parity][half][row] floats
   const uint32_t bar_base = smem_base + xch_off + 2048u;
   const uint32_t ctrl_off = xch_off + 2048u + 24u * 8u;
   float* xch = reinterpret_cast<float*>(smem_raw + xch_off);
@@ -104,23 +107,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     QS_FULL = 0,                      // the staging buffer holds a tile's Q (TMA bytes)
     QS_EMPTY = 1,                     // its copy into tensor memory has completed
     K_FULL = 2,
-    V_FULL = K_FULL + kAttnStages,
-    K_EMPTY = V_FULL + kAttnStages,
-    V_EMPTY = K_EMPTY + kAttnStages,
-    S_FULL = V_EMPTY + kAttnStages,   // two: one per score buffer
+    V_FULL = K_FULL + kAttnStagesK,
+    K_EMPTY = V_FULL + kAttnStagesV,
+    V_EMPTY = K_EMPTY + kAttnStagesK,
+    S_FULL = V_EMPTY + kAttnStagesV,  // two: one per score buffer
     P_FULL = S_FULL + 2,              // two: a warp may finish block g + 1 before another has finished block g
     PV_DONE = P_FULL + 2,
     O_DONE = PV_DONE + 1,             // a tile's last product has completed (PV_DONE's one-bit phase cannot tell
                                       // "two products behind" from "done", so the epilogue has its own barrier)
     O_FREE = O_DONE + 1,              // the softmax warps have read a finished tile's O
-    N_BARS = O_FREE + 1
+    O_STAGED = O_FREE + 1,            // ... and written O / l into the staging buffer
+    OS_DONE = O_STAGED + 1,           // the store warp's TMA store has read the staging buffer
+    N_BARS = OS_DONE + 1
   };
   static_assert(N_BARS <= 24, "barrier area");
   auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
 
   if (threadIdx.x < N_BARS) {
     const int i = (int)threadIdx.x;
-    const bool by_softmax = i == P_FULL || i == P_FULL + 1 || i == O_FREE;
+    const bool by_softmax = i == P_FULL || i == P_FULL + 1 || i == O_FREE || i == O_STAGED;
     ptx::mbar_init(bar(i), by_softmax ? 8u : 1u);  // one arrival per softmax warp
     if (i == 0) *abort_p = 0;
     ptx::fence_mbar_init();
@@ -129,6 +134,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     ptx::prefetch_tensormap(&tmQ);
     ptx::prefetch_tensormap(&tmK);
     ptx::prefetch_tensormap(&tmV);
+    ptx::prefetch_tensormap(&tmO);
   }
   if (warp == 9) {
     __syncwarp();
@@ -186,31 +192,35 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       }
     };
     if (n_items > 0) load_q(0);
-    int s = 0;
-    uint32_t par = 1;  // an empty slot's first wait passes
+    int ks = 0, vs = 0;
+    uint32_t kpar = 1, vpar = 1;  // an empty slot's first wait passes
     bool ok = true;
     for (int n = 0; ok && n < n_items; ++n) {
       const AttnTile t = tile_of(n);
       for (int j = 0; ok && j < t.nb; ++j) {
-        ok = wait_all(bar(K_EMPTY + s), par);
+        ok = wait_all(bar(K_EMPTY + ks), kpar);
         if (!ok) break;
         if (ptx::elect_one()) {
-          ptx::mbar_arrive_expect_tx(bar(K_FULL + s), tile_bytes);
+          ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), tile_bytes);
           for (int c = 0; c < chunks; ++c)
-            ptx::tma_load_4d(k_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmK, bar(K_FULL + s), c * 64, t.kvh,
+            ptx::tma_load_4d(k_s0 + ks * tile_bytes + c * kAttnChunkBytes, &tmK, bar(K_FULL + ks), c * 64, t.kvh,
                              j * kAttnBlockK, t.b);
         }
-        ok = wait_all(bar(V_EMPTY + s), par);
+        if (++ks == kAttnStagesK) {
+          ks = 0;
+          kpar ^= 1u;
+        }
+        ok = wait_all(bar(V_EMPTY + vs), vpar);
         if (!ok) break;
         if (ptx::elect_one()) {
-          ptx::mbar_arrive_expect_tx(bar(V_FULL + s), tile_bytes);
+          ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), tile_bytes);
           for (int c = 0; c < chunks; ++c)
-            ptx::tma_load_4d(v_s0 + s * tile_bytes + c * kAttnChunkBytes, &tmV, bar(V_FULL + s), c * 64, t.kvh,
+            ptx::tma_load_4d(v_s0 + vs * tile_bytes + c * kAttnChunkBytes, &tmV, bar(V_FULL + vs), c * 64, t.kvh,
                              j * kAttnBlockK, t.b);
         }
-        if (++s == kAttnStages) {
-          s = 0;
-          par ^= 1u;
+        if (++vs == kAttnStagesV) {
+          vs = 0;
+          vpar ^= 1u;
         }
         // the next tile's Q follows this tile's first block, once this tile's Q has left the staging buffer
         if (j == 0 && n + 1 < n_items) {
@@ -253,7 +263,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         ptx::umma_commit<1>(bar(S_FULL + (sg & 1)));
         ptx::umma_commit<1>(bar(K_EMPTY + ks));
       }
-      if (++ks == kAttnStages) {
+      if (++ks == kAttnStagesK) {
         ks = 0;
         kpar ^= 1u;
       }
@@ -290,12 +300,29 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           ptx::umma_commit<1>(bar(PV_DONE));
           if (j == nb - 1) ptx::umma_commit<1>(bar(O_DONE));
         }
-        if (++vs == kAttnStages) {
+        if (++vs == kAttnStagesV) {
           vs = 0;
           vpar ^= 1u;
         }
       }
     }
+    __syncwarp();
+  } else if (warp == 10) {
+    // ------------------------------------------------------------ store warp: staged O tiles -> global by TMA
+    bool ok = true;
+    for (int n = 0; ok && n < n_items; ++n) {
+      ok = wait_all(bar(O_STAGED), (uint32_t)n & 1u);
+      if (!ok) break;
+      const AttnTile t = tile_of(n);
+      if (lane == 0) {  // bulk groups belong to the issuing thread
+        for (int c = 0; c < chunks; ++c) ptx::tma_store_4d(&tmO, o_stage + c * kAttnChunkBytes, c * 64, t.h, t.t0, t.b);
+        ptx::bulk_commit_group();
+        ptx::bulk_wait_group_read<0>();  // the staging buffer may be rewritten
+        ptx::mbar_arrive(bar(OS_DONE));
+      }
+      __syncwarp();
+    }
+    if (lane == 0) ptx::bulk_wait_group<0>();  // every store has reached global memory before the CTA exits
     __syncwarp();
   }
   } else {
@@ -310,16 +337,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const uint32_t o_addr = tmem_o + lane_addr + (uint32_t)(half * o_cols);
     bool ok = true;  // warp-uniform; a warp whose wait gave up keeps meeting its partner at the named barriers
     long long prof_s_wait = 0, prof_epi = 0, prof_blocks = 0;
-    // A finished tile whose output has not been stored yet: this thread's part of the row sums, where its half
-    // row goes (null for a row past the end), and the tile's ordinal.
+    // A finished tile whose output has not been stored yet: this thread's part of the row sums and the tile's ordinal.
     bool pend = false;
     float pend_l = 0.f;
     int pend_n = 0;
-    __nv_bfloat16* pend_row = nullptr;
-    // O / l -> global for the pending tile.  The row sum is the sum of the two halves', exchanged through the
-    // buffer `xbuf` that the latest exchange of maxima did not use; the second barrier keeps the next block's
-    // maxima from overwriting a sum not yet read.  O is read into registers and released before the stores, so the
-    // next tile's products may overwrite it while they drain.
+    // O / l of the pending tile -> staging buffer -> (store warp) global.  The row sum is the sum of the two
+    // halves', exchanged through the buffer `xbuf` that the latest exchange of maxima did not use; the second
+    // barrier keeps the next block's maxima from overwriting a sum not yet read.  O is read into registers and
+    // released first, so the next tile's products may overwrite it.
     auto finish_tile = [&](int xbuf) {
       const long long te0 = prof ? clock64() : 0;
       pend = false;
@@ -338,23 +363,34 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar(O_FREE));
-      if (pend_row != nullptr) {
+      // O / l as BF16 into the staging tile (128-byte rows of 64 columns, 16-byte pieces swizzled by the row like
+      // every other tile here), once the store of the tile before has read it
+      if (pend_n > 0) ok = wait_all(bar(OS_DONE), (uint32_t)(pend_n - 1) & 1u);
+      if (!ok) return;
+      {
         const float inv = (lsum > 0.f) ? __fdividef(1.f, lsum) : 0.f;
+        const int col0 = half * o_cols;  // this thread's first output column
+        const uint32_t dst = o_stage + (uint32_t)(col0 >> 6) * kAttnChunkBytes + (uint32_t)row * 128u;
+        const uint32_t piece0 = (uint32_t)(col0 & 63) >> 3;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           if (c * 32 < o_cols) {
 #pragma unroll
             for (int gq = 0; gq < 4; ++gq) {
-              uint4 qv;
-              qv.x = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 0]) * inv, __uint_as_float(o[c][gq * 8 + 1]) * inv);
-              qv.y = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 2]) * inv, __uint_as_float(o[c][gq * 8 + 3]) * inv);
-              qv.z = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 4]) * inv, __uint_as_float(o[c][gq * 8 + 5]) * inv);
-              qv.w = pack_bf16x2(__uint_as_float(o[c][gq * 8 + 6]) * inv, __uint_as_float(o[c][gq * 8 + 7]) * inv);
-              *reinterpret_cast<uint4*>(pend_row + c * 32 + gq * 8) = qv;
+              const uint32_t piece = piece0 + (uint32_t)(c * 4 + gq);
+              ptx::st_shared_v4(
+                  dst + ((piece ^ (uint32_t)(row & 7)) << 4),
+                  pack_bf16x2(__uint_as_float(o[c][gq * 8 + 0]) * inv, __uint_as_float(o[c][gq * 8 + 1]) * inv),
+                  pack_bf16x2(__uint_as_float(o[c][gq * 8 + 2]) * inv, __uint_as_float(o[c][gq * 8 + 3]) * inv),
+                  pack_bf16x2(__uint_as_float(o[c][gq * 8 + 4]) * inv, __uint_as_float(o[c][gq * 8 + 5]) * inv),
+                  pack_bf16x2(__uint_as_float(o[c][gq * 8 + 6]) * inv, __uint_as_float(o[c][gq * 8 + 7]) * inv));
             }
           }
         }
       }
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar(O_STAGED));
       if (prof) prof_epi += clock64() - te0;
     };
     int g = 0;  // global block counter
@@ -457,9 +493,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       pend = true;
       pend_l = l;
       pend_n = n;
-      pend_row = (t_row < p.Tq) ? (p.O + (long long)tile.b * p.o_stride_b + (long long)t_row * p.o_stride_t +
-                                   (long long)tile.h * p.o_stride_h + half * o_cols)
-                                : nullptr;
     }
     if (pend) finish_tile(g & 1);
     if (prof && warp == 0 && lane == 0) {

@@ -962,11 +962,12 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
   if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, to;
   auto bs = [&](int64_t s, int64_t fallback) { return (batch > 1 && s > 0) ? s : std::max<int64_t>(fallback, 8); };
   fact_status_t st = encode_map_bthd(h, &tq, Q, head_dim, heads_q, seq_q, batch, q_sh, q_st, bs(q_sb, q_st * seq_q));
   if (st == FACT_OK) st = encode_map_bthd(h, &tk, K, head_dim, heads_kv, seq_kv, batch, k_sh, k_st, bs(k_sb, k_st * seq_kv));
   if (st == FACT_OK) st = encode_map_bthd(h, &tv, V, head_dim, heads_kv, seq_kv, batch, v_sh, v_st, bs(v_sb, v_st * seq_kv));
+  if (st == FACT_OK) st = encode_map_bthd(h, &to, O, head_dim, heads_q, seq_q, batch, o_sh, o_st, bs(o_sb, o_st * seq_q));
   if (st == FACT_OK) {
     AttnParams p;
     memset(&p, 0, sizeof p);
@@ -980,10 +981,6 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     const double sc = scale > 0.f ? (double)scale : 1.0 / std::sqrt((double)head_dim);
     p.scale_log2 = (float)(sc * 1.4426950408889634);
     p.q_tiles = (int)((seq_q + kAttnBlockQ - 1) / kAttnBlockQ);
-    p.O = reinterpret_cast<__nv_bfloat16*>(O);
-    p.o_stride_b = o_sb;
-    p.o_stride_t = o_st;
-    p.o_stride_h = o_sh;
     p.kmajor_desc = smem_desc_template(16, 1024);
     p.v_desc = smem_desc_template(kAttnBlockK * 128, 1024);  // 64-column chunks of V are one 128-key tile apart
     p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttnBlockK >> 3) << 17) | ((uint32_t)(kAttnBlockQ >> 4) << 24);
@@ -1015,7 +1012,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      fact_attention_kernel<<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, p);
+      fact_attention_kernel<<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
       else h->launches++;
