@@ -190,7 +190,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, or `all`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, or `attention`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
@@ -228,9 +228,15 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        rows = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup,
-                               iters=args.steps, side_ref=False, layout=args.layout)
-        print(json.dumps({"shapes": rows, "gpu_launches": h.launch_count()}))
+        rows = [] if args.shape == "attention" else per_shape_table(
+            h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
+            side_ref=False, layout=args.layout)
+        if args.shape in ("all", "attention"):
+            att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
+        else:  # attention shapes can be named like the GEMM shapes
+            att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
+                                  names=names)
+        print(json.dumps({"shapes": rows, "attention": att, "gpu_launches": h.launch_count()}))
         h.close()
         return 0
 
@@ -319,6 +325,9 @@ def main():
     shapes = []
     if not args.no_shapes and rank == 0:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
+    attention = []
+    if not args.no_shapes and rank == 0:
+        attention = attention_table(h, dev, stream, flush_l2, peaks)
     clocks = sampler.stop()  # sampled from the first warm-up step to the end of the per-shape table
 
     # ---------------------------------------------------------------- CPU baseline (oracle) on rank 0
@@ -352,6 +361,7 @@ def main():
             "clocks": dict(clocks, sm_mhz_in_dominant_kernel=(1e3 * k_cycles / k_ns if k_ns else None)),
             "cpu_baseline": cpu,
             "shapes": shapes,
+            "attention": attention,
         }
         print(json.dumps(line))
     if dist is not None:
@@ -432,6 +442,63 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
             "cublas_matmul_only_us": t_side[len(t_side) // 2] * 1e3, "tile": cfg,
         })
         del X, W, out
+    return rows
+
+
+def attention_table(h, dev, stream, flush_l2, peaks, warm=5, iters=20, side_ref=True, names=None):
+    """Time the fused attention kernel on the transformer blocks' attention shapes (L2 overwritten between
+    launches); torch's scaled_dot_product_attention on the same tensors is a side reference."""
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    rows = []
+    for case in wl.attention_cases():
+        if names is not None and case.name not in names:
+            continue
+        q, k, v = wl.make_attention_inputs(case, dev)
+        out = torch.empty_like(q)
+
+        def call():
+            h.attention(q, k, v, causal=case.causal, out=out)
+
+        qt, kt, vt = (x.permute(0, 2, 1, 3) for x in (q, k, v))
+
+        def side():
+            torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=case.causal,
+                                                             enable_gqa=case.Hq != case.Hkv)
+
+        def time_it(fn, n):
+            for _ in range(warm):
+                fn()
+            ts = []
+            for _ in range(n):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                ts.append((a, b))
+            torch.cuda.synchronize(dev)
+            return sorted(x.elapsed_time(y) for x, y in ts)
+
+        t = time_it(call, iters)
+        med = t[len(t) // 2]
+        try:
+            ts = time_it(side, 10) if side_ref else [0.0]
+        except Exception:  # the side reference is optional
+            ts = [float("nan")]
+        t_tensor = case.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        rows.append({
+            "name": case.name, "B": case.B, "T": case.T, "heads_q": case.Hq, "heads_kv": case.Hkv,
+            "head_dim": case.D, "causal": case.causal, "us_median": med * 1e3, "us_min": t[0] * 1e3,
+            "tflops": case.flops / (med * 1e-3) / 1e12, "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+            "roofline_us": max(t_tensor, t_hbm) * 1e3, "roofline_frac": max(t_tensor, t_hbm) / med,
+            "torch_sdpa_us": ts[len(ts) // 2] * 1e3,
+        })
+        assert h.device_status() == 0
+        del q, k, v, out
     return rows
 
 

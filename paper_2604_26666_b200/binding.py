@@ -246,7 +246,7 @@ class Handle:
     def selftest_wait_timeout(self, limit_ms: float = 5.0, stream=None):
         """Run the bounded-wait self-test (fact_selftest_wait_timeout); raises unless the wait gave up cleanly."""
         _check(lib().fact_selftest_wait_timeout(self._h, self._stream(stream), float(limit_ms)),
-               "fact_selftest_wait_timeout", "fact_attention", self._h)
+               "fact_selftest_wait_timeout", self._h)
 
     def launch_count(self) -> int:
         return int(lib().fact_launch_count(self._h))

@@ -62,7 +62,9 @@ struct AttnParams {
   uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (K)
   uint64_t v_desc;            // UMMA descriptor template, V as an N-major operand
   uint32_t idesc_s, idesc_pv;
-  int* status;                // [0] error word, [2..5] cycles and nanoseconds of the first CTA (debug bit 256)
+  int* status;                // [0] error word; with debug bit 256 eight 64-bit counters of the first CTA from [2]:
+                              // cycles, nanoseconds, first wait that gave up, cycles warp 0 waited for scores, its
+                              // blocks, -, cycles it spent finishing tiles, its tiles
   int debug;
 };
 

@@ -659,13 +659,9 @@ fact_status_t fact_last_kernel_clock(fact_handle_t h, void* stream, int64_t* sm_
 fact_status_t fact_last_kernel_profile(fact_handle_t h, void* stream, int64_t counters[8]) {
   if (!h || !counters) return FACT_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return FACT_ERR_CUDA;
-  long long v[10];
+  long long v[8];
   if (cudaMemcpy(v, h->d_status + 2, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
   for (int i = 0; i < 8; ++i) counters[i] = v[i];
-  if (h->debug_flags & 2048) {  // attention experiment: entry-to-first-scores and entry-to-last-block in [6], [7]
-    counters[6] = v[8];
-    counters[7] = v[9];
-  }
   return FACT_OK;
 }
 

@@ -169,3 +169,54 @@ def bits(t: torch.Tensor):
 
     assert t.dtype == torch.bfloat16 and t.device.type == "cpu"
     return t.view(torch.int16).numpy().view(np.uint16)
+
+
+# ------------------------------------------------------------------------------------------------
+# Attention (the fused multi-head attention entry point; Section 5.2's transformer blocks)
+@dataclass(frozen=True)
+class AttentionCase:
+    """One attention problem: Q [B, T, Hq, D], K and V [B, T, Hkv, D], BF16."""
+    name: str
+    B: int
+    T: int
+    Hq: int
+    Hkv: int
+    D: int
+    causal: bool
+    seed: int
+
+    @property
+    def flops(self) -> float:
+        """Algorithmic FLOPs: two products of 2*D FLOPs per (query, visible key) pair."""
+        pairs = self.T * (self.T + 1) / 2 if self.causal else self.T * self.T
+        return 4.0 * self.D * pairs * self.B * self.Hq
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Q and O once, K and V once (BF16)."""
+        return 2 * self.B * self.T * self.D * (2 * self.Hq + 2 * self.Hkv)
+
+
+def attention_cases():
+    """The attention shapes of the two transformer blocks: GPT-2-like (12 heads of 64) and LLaMA-like (32 query
+    heads over 8 key/value heads of 128), at the benchmark's token counts (16 x 1024 and 4 x 2048 tokens) and at
+    the paper's (128 x 512 and 16 x 2048), causal and not."""
+    shapes = [("gpt2_16x1024", 16, 1024, 12, 12, 64), ("llama_4x2048", 4, 2048, 32, 8, 128),
+              ("gpt2_128x512", 128, 512, 12, 12, 64), ("llama_16x2048", 16, 2048, 32, 8, 128)]
+    out = []
+    for i, (name, B, T, Hq, Hkv, D) in enumerate(shapes):
+        for causal in (True, False):
+            out.append(AttentionCase(f"{name}_{'causal' if causal else 'full'}", B, T, Hq, Hkv, D, causal, 7000 + i))
+    return out
+
+
+def make_attention_inputs(case, device="cpu"):
+    """Seeded N(0, 1) BF16 Q, K, V (unit-variance activations, as after a layer norm and a projection)."""
+    import torch
+
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(case.seed)
+    q = torch.randn(case.B, case.T, case.Hq, case.D, generator=gen).to(torch.bfloat16)
+    k = torch.randn(case.B, case.T, case.Hkv, case.D, generator=gen).to(torch.bfloat16)
+    v = torch.randn(case.B, case.T, case.Hkv, case.D, generator=gen).to(torch.bfloat16)
+    return q.to(device), k.to(device), v.to(device)

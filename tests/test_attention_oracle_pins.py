@@ -74,3 +74,43 @@ def test_invariances():
     # the default scale is 1/sqrt(D): doubling Q and halving the scale changes nothing
     a = attention(bits(q * 2), bits(k), bits(v), causal=False, scale=0.5 / np.sqrt(D))
     assert np.allclose(a, base, rtol=1e-12, atol=1e-13)
+
+
+def test_brute_force_python_loops_on_a_tiny_case():
+    """The definition written out with scalar loops and math.exp: softmax(scale q.k + mask) v, grouped queries."""
+    import math
+
+    B, T, Hq, Hkv, D = 1, 5, 4, 2, 4
+    q, k, v = rnd((B, T, Hq, D), 14), rnd((B, T, Hkv, D), 15), rnd((B, T, Hkv, D), 16)
+    qf, kf, vf = (x.double().tolist() for x in (q, k, v))
+    for causal in (False, True):
+        got = attention(bits(q), bits(k), bits(v), causal=causal)
+        for h in range(Hq):
+            g = h // (Hq // Hkv)
+            for i in range(T):
+                keys = range(i + 1) if causal else range(T)
+                s = [sum(qf[0][i][h][d] * kf[0][j][g][d] for d in range(D)) / math.sqrt(D) for j in keys]
+                w = [math.exp(x - max(s)) for x in s]
+                for d in range(D):
+                    want = sum(wj * vf[0][j][g][d] for wj, j in zip(w, keys)) / sum(w)
+                    assert abs(got[0, i, h, d] - want) <= 1e-13 * max(1.0, abs(want))
+
+
+def test_key_set_split_and_merge():
+    """Attention over a key set equals the log-sum-exp weighted mix of attention over its two halves."""
+    B, T, H, D = 1, 10, 2, 8
+    q, k, v = rnd((B, T, H, D), 17), rnd((B, T, H, D), 18), rnd((B, T, H, D), 19)
+    full = attention(bits(q), bits(k), bits(v), causal=False)
+    a = attention(bits(q), bits(k[:, :4]), bits(v[:, :4]), causal=False)
+    b = attention(bits(q), bits(k[:, 4:]), bits(v[:, 4:]), causal=False)
+    qd, kd = q.double().numpy(), k.double().numpy()
+    s = np.einsum("bihd,bjhd->bihj", qd, kd) / np.sqrt(D)
+    za, zb = np.exp(s[..., :4]).sum(-1), np.exp(s[..., 4:]).sum(-1)  # partition sums of the halves
+    mix = (a * za[..., None] + b * zb[..., None]) / (za + zb)[..., None]
+    assert np.allclose(full, mix, rtol=1e-12, atol=1e-13)
+    # a key that the query scores hugely negative has weight ~ 0: the result equals attention without that key
+    far = k.clone()
+    far[:, -1] = -(q[:, 0] * 64)
+    near = attention(bits(q[:, :1]), bits(far), bits(v), causal=False)
+    drop = attention(bits(q[:, :1]), bits(k[:, :-1]), bits(v[:, :-1]), causal=False)
+    assert np.allclose(near, drop, rtol=1e-9, atol=1e-10)
