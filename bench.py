@@ -190,7 +190,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, `all`, or `attention`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention` or `blocks`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
@@ -228,15 +228,22 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        rows = [] if args.shape == "attention" else per_shape_table(
+        rows = [] if args.shape in ("attention", "blocks") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
             side_ref=False, layout=args.layout)
         if args.shape in ("all", "attention"):
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
+        elif args.shape == "blocks":
+            att = []
         else:  # attention shapes can be named like the GEMM shapes
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
                                   names=names)
-        print(json.dumps({"shapes": rows, "attention": att, "gpu_launches": h.launch_count()}))
+        blk = []
+        if args.shape == "all":
+            blk = block_table(h, dev, stream, flush_l2, peaks)
+        elif args.shape == "blocks":  # --warmup / --steps apply, no eager side reference: the form the ncu runs use
+            blk = block_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False)
+        print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "gpu_launches": h.launch_count()}))
         h.close()
         return 0
 
@@ -325,9 +332,10 @@ def main():
     shapes = []
     if not args.no_shapes and rank == 0:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
-    attention = []
+    attention, blocks = [], []
     if not args.no_shapes and rank == 0:
         attention = attention_table(h, dev, stream, flush_l2, peaks)
+        blocks = block_table(h, dev, stream, flush_l2, peaks)
     clocks = sampler.stop()  # sampled from the first warm-up step to the end of the per-shape table
 
     # ---------------------------------------------------------------- CPU baseline (oracle) on rank 0
@@ -362,6 +370,7 @@ def main():
             "cpu_baseline": cpu,
             "shapes": shapes,
             "attention": attention,
+            "blocks": blocks,
         }
         print(json.dumps(line))
     if dist is not None:
@@ -499,6 +508,92 @@ def attention_table(h, dev, stream, flush_l2, peaks, warm=5, iters=20, side_ref=
         })
         assert h.device_status() == 0
         del q, k, v, out
+    return rows
+
+
+def block_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=True):
+    """Time one forward pass of the paper's two transformer blocks through fact_block_forward (seven launches on one
+    stream; also replayed from a CUDA graph) next to the same block in PyTorch eager BF16 on this GPU."""
+    import torch
+    import torch.nn.functional as F
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    def time_it(fn, n):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(n):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            ts.append((a, b))
+        torch.cuda.synchronize(dev)
+        t = sorted(x.elapsed_time(y) for x, y in ts)
+        return t[len(t) // 2]
+
+    rows = []
+    for case in wl.block_cases():
+        x, w = wl.make_block_inputs(case, dev)
+        desc = h.block_desc(case.kind, case.B, case.T, case.Hq, case.Hkv, case.D, case.ffn, w)
+        y = torch.empty_like(x)
+        h.block_forward(desc, x, out=y)  # allocates the workspace, configures the kernels
+        launches0 = h.launch_count()
+        h.block_forward(desc, x, out=y)
+        launches = h.launch_count() - launches0
+        ms = time_it(lambda: h.block_forward(desc, x, out=y), iters)
+        ms_graph = None
+        try:
+            graph = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize(dev)
+            with torch.cuda.graph(graph, stream=torch.cuda.Stream(dev)):  # capture needs a side stream
+                h.block_forward(desc, x, out=y)
+            ms_graph = time_it(graph.replay, iters)
+        except Exception as e:  # the graph replay is an extra, the stream launch is the number
+            print(f"# graph capture of {case.name} failed: {e}", file=sys.stderr)
+        C, Hq, Hkv, D = case.hidden, case.Hq, case.Hkv, case.D
+
+        def eager():
+            norm = (lambda v, g, b: F.layer_norm(v, (C,), g, b, 1e-5)) if case.kind == "gpt" else \
+                   (lambda v, g, b: F.rms_norm(v, (C,), g, 1e-5))
+            n1 = norm(x, w["norm1_gamma"], w.get("norm1_beta"))
+            qkv = F.linear(n1, w["wqkv"], w.get("bqkv")).view(case.B, case.T, Hq + 2 * Hkv, D)
+            q, k, v = (t.transpose(1, 2) for t in (qkv[:, :, :Hq], qkv[:, :, Hq:Hq + Hkv], qkv[:, :, Hq + Hkv:]))
+            a = F.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=Hq != Hkv)
+            x1 = F.linear(a.transpose(1, 2).reshape(case.B * case.T, C), w["wo"], w.get("bo")) + x
+            n2 = norm(x1, w["norm2_gamma"], w.get("norm2_beta"))
+            if case.kind == "gpt":
+                hh = F.gelu(F.linear(n2, w["w1"], w["b1"]), approximate="tanh")
+            else:
+                gu = F.linear(n2, w["w1"])
+                hh = F.silu(gu[:, :case.ffn]) * gu[:, case.ffn:]
+            return F.linear(hh, w["w2"], w.get("b2")) + x1
+
+        ms_eager = None
+        if side_ref:
+            try:
+                ms_eager = time_it(eager, iters)
+            except Exception as e:
+                print(f"# eager reference of {case.name} failed: {e}", file=sys.stderr)
+        assert h.device_status() == 0
+        # the block's normalisation kernel alone: HBM-bound, one read and one write of the activation
+        nout = torch.empty_like(x)
+        kind = "layer" if case.kind == "gpt" else "rms"
+        ms_norm = time_it(lambda: h.norm(x, w["norm1_gamma"], w.get("norm1_beta"), kind=kind, out=nout), iters)
+        norm_bytes = 2 * x.numel() * 2
+        del nout
+        rows.append({
+            "norm_us": ms_norm * 1e3, "norm_gbs": norm_bytes / (ms_norm * 1e-3) / 1e9,
+            "norm_frac_of_hbm_peak": norm_bytes / (ms_norm * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "name": case.name, "kind": case.kind, "batch": case.B, "seq": case.T, "hidden": C, "heads_q": Hq,
+            "heads_kv": Hkv, "head_dim": D, "ffn": case.ffn, "ms": ms, "ms_cuda_graph": ms_graph,
+            "tflops": case.flops / (ms * 1e-3) / 1e12, "launches": launches, "torch_eager_bf16_ms": ms_eager,
+            "speedup_vs_torch_eager": (ms_eager / ms) if ms_eager else None,
+        })
+        del x, w, y, desc
+        torch.cuda.empty_cache()
     return rows
 
 

@@ -219,8 +219,7 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
  * product, O is accumulated in FP32 and rounded once.  causal != 0 masks keys j > i and requires
  * seq_q == seq_kv; scale <= 0 means 1 / sqrt(head_dim).
  * Requirements: head_dim 64 or 128; heads_q a multiple of heads_kv; all four pointers 16-byte aligned and
- * every stride a multiple of 8 elements (operands are read through TMA, O rows are written as 16-byte
- * vectors).  Errors: FACT_ERR_UNSUPPORTED for another head_dim or causal with seq_q != seq_kv,
+ * every stride a multiple of 8 elements (operands are read and O is written through TMA).  Errors: FACT_ERR_UNSUPPORTED for another head_dim or causal with seq_q != seq_kv,
  * FACT_ERR_BAD_ALIGNMENT, FACT_ERR_INVALID_ARG; nothing is launched on an error.  batch == 0 or
  * seq_q == 0 is a successful no-op. */
 fact_status_t fact_attention(fact_handle_t handle, int64_t batch, int64_t seq_q, int64_t seq_kv, int64_t heads_q,
@@ -230,6 +229,56 @@ fact_status_t fact_attention(fact_handle_t handle, int64_t batch, int64_t seq_q,
                              int64_t v_stride_token, int64_t v_stride_head, void* O, int64_t o_stride_batch,
                              int64_t o_stride_token, int64_t o_stride_head, int causal, float scale,
                              void* cuda_stream);
+
+/* Row normalisation of the transformer blocks (Section 5.2: the MiniGPT block is a pre-norm GPT block with
+ * layer norms, the Llama block uses RMS norms; the paper leaves them in the surrounding graph, they are here so
+ * that a whole block runs through this library):
+ *   FACT_NORM_LAYER:  Y[m,:] = (X[m,:] - mean) / sqrt(var + eps) * gamma + beta    (biased variance)
+ *   FACT_NORM_RMS:    Y[m,:] =  X[m,:] / sqrt(mean(X[m,:]^2) + eps) * gamma
+ * X, Y: BF16 [M x C] with leading dimensions ldx, ldy (elements); gamma: BF16 [C]; beta: BF16 [C] or NULL
+ * (must be NULL for FACT_NORM_RMS).  FP32 arithmetic, one rounding at the store.  C a multiple of 8 in
+ * [8, 8192]; pointers 16-byte aligned, ldx and ldy multiples of 8.  Y may alias X. */
+typedef enum { FACT_NORM_LAYER = 0, FACT_NORM_RMS = 1 } fact_norm_t;
+fact_status_t fact_norm(fact_handle_t handle, fact_norm_t kind, int64_t M, int64_t C, const void* X, int64_t ldx,
+                        const void* gamma, const void* beta, float eps, void* Y, int64_t ldy, void* cuda_stream);
+
+/* One pre-norm transformer block, forward, as a chain of this library's kernels on one stream (Section 5.2:
+ * the two Level-3 blocks the paper composes from its attention and MLP patterns):
+ *     n1  = norm1(x)
+ *     qkv = n1 . Wqkv^T (+ bqkv)                       [tokens x (heads_q + 2 heads_kv) head_dim], Q | K | V
+ *     a   = causal attention over the Q, K, V slices of qkv, read in place (grouped queries if heads_kv < heads_q)
+ *     x1  = a . Wo^T (+ bo) + x                        fused residual
+ *     n2  = norm2(x1)
+ *     h   = gelu_tanh(n2 . W1^T + b1)                  FACT_BLOCK_GPT:   W1 [ffn x hidden]
+ *         = silu(n2 . Wg^T) * (n2 . Wu^T)              FACT_BLOCK_LLAMA: W1 [2 ffn x hidden], gate rows first
+ *     y   = h . W2^T (+ b2) + x1                       fused residual
+ * FACT_BLOCK_GPT uses layer norms (gamma, beta) and biases; FACT_BLOCK_LLAMA uses RMS norms and no biases (the
+ * bias and beta pointers must be NULL).  The paper's block descriptions name no positional rotation of Q and K;
+ * none is applied.  All tensors BF16, row-major, dense: x, y [batch * seq x hidden]; weights [out x in] as
+ * torch.nn.Linear stores them; every intermediate is rounded to BF16 once, where it is stored.
+ * hidden must equal heads_q * head_dim; head_dim 64 or 128; hidden and ffn multiples of 8.
+ * `workspace` (device) holds the intermediates; fact_block_workspace_bytes gives its size.  y may alias x. */
+typedef enum { FACT_BLOCK_GPT = 0, FACT_BLOCK_LLAMA = 1 } fact_block_kind_t;
+typedef struct {
+  fact_block_kind_t kind;
+  int64_t batch, seq, hidden, heads_q, heads_kv, head_dim, ffn;
+  float eps;
+  const void *norm1_gamma, *norm1_beta; /* [hidden] */
+  const void *wqkv, *bqkv;              /* [(heads_q + 2 heads_kv) head_dim x hidden], [(heads_q + 2 heads_kv) head_dim] */
+  const void *wo, *bo;                  /* [hidden x hidden], [hidden] */
+  const void *norm2_gamma, *norm2_beta; /* [hidden] */
+  const void *w1, *b1;                  /* GPT [ffn x hidden], [ffn]; LLAMA [2 ffn x hidden] (gate | up), NULL */
+  const void *w2, *b2;                  /* [hidden x ffn], [hidden] */
+} fact_block_t;
+size_t fact_block_workspace_bytes(const fact_block_t* block);
+/* Where fact_block_forward keeps its intermediates, as byte offsets into the workspace (each dense, BF16,
+ * row-major [tokens x columns]): offsets[0] the norm output (n1, later overwritten by n2; hidden columns),
+ * [1] qkv ((heads_q + 2 heads_kv) head_dim columns), [2] a (hidden), [3] x1 (hidden), [4] h (ffn).  After a
+ * call they still hold that call's values, which lets a caller inspect or check every stage.  Returns
+ * FACT_ERR_INVALID_ARG for an inconsistent descriptor. */
+fact_status_t fact_block_workspace_offsets(const fact_block_t* block, size_t offsets[5]);
+fact_status_t fact_block_forward(fact_handle_t handle, const fact_block_t* block, const void* x, void* y,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* The configuration the library would run for this problem when cfg == NULL
  * (its tuned entry if fact_tune / fact_tune_cache_load provided one, else a

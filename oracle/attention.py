@@ -29,7 +29,12 @@ def _widen(bits: np.ndarray) -> np.ndarray:
 def attention(Q, K, V, *, causal: bool, scale: float | None = None, rows=None) -> np.ndarray:
     """Q: uint16 [B, Tq, Hq, D];  K, V: uint16 [B, Tk, Hkv, D];  returns float64 [B, Tq (or len(rows)), Hq, D].
     `rows`: optional query positions to compute (all batches and heads)."""
-    q, k, v = _widen(Q), _widen(K), _widen(V)
+    return attention_f64(_widen(Q), _widen(K), _widen(V), causal=causal, scale=scale, rows=rows)
+
+
+def attention_f64(q, k, v, *, causal: bool, scale: float | None = None, rows=None) -> np.ndarray:
+    """The same definition on float64 operands (used where attention is one stage of a longer float64 chain)."""
+    q, k, v = (np.asarray(t, dtype=np.float64) for t in (q, k, v))
     B, Tq, Hq, D = q.shape
     Bk, Tk, Hkv, Dk = k.shape
     if (Bk, Dk) != (B, D) or v.shape != k.shape or Hq % Hkv:

@@ -11,7 +11,7 @@ The raw C entry points are available under their C names on ``lib()``
 from __future__ import annotations
 
 import ctypes
-from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int64, c_size_t, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_int64, c_size_t, c_void_p
 from pathlib import Path
 from typing import Optional
 
@@ -35,8 +35,23 @@ EXPORTED = [
     "fact_create", "fact_destroy", "fact_status_string", "fact_workspace_bytes", "fact_gemm", "fact_gemm_batched",
     "fact_gemm_splitk", "fact_linear", "fact_get_config", "fact_tune", "fact_tune_cache_save",
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
-    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout", "fact_attention",
+    "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
+    "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
 ]
+
+
+NORMS = {"layer": 0, "rms": 1}
+BLOCK_KINDS = {"gpt": 0, "llama": 1}
+
+
+class Block(Structure):
+    """Mirror of fact_block_t."""
+
+    _fields_ = ([("kind", c_int)] +
+                [(n, c_int64) for n in ("batch", "seq", "hidden", "heads_q", "heads_kv", "head_dim", "ffn")] +
+                [("eps", c_float)] +
+                [(n, c_void_p) for n in ("norm1_gamma", "norm1_beta", "wqkv", "bqkv", "wo", "bo", "norm2_gamma",
+                                         "norm2_beta", "w1", "b1", "w2", "b2")])
 
 
 class FactError(RuntimeError):
@@ -100,9 +115,14 @@ def lib() -> ctypes.CDLL:
     L.fact_selftest_wait_timeout.argtypes = [vp, vp, c_double]
     L.fact_last_error.argtypes = [vp]
     L.fact_last_error.restype = c_char_p
+    L.fact_norm.argtypes = [vp, c_int, i64, i64, vp, i64, vp, vp, c_float, vp, i64, vp]
+    L.fact_block_workspace_bytes.argtypes = [POINTER(Block)]
+    L.fact_block_workspace_bytes.restype = sz
+    L.fact_block_workspace_offsets.argtypes = [POINTER(Block), POINTER(sz)]
+    L.fact_block_forward.argtypes = [vp, POINTER(Block), vp, vp, vp, sz, vp]
     for name in EXPORTED:
         fn = getattr(L, name)
-        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error"):
+        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
             fn.restype = c_int
     _lib = L
     return L
@@ -369,6 +389,62 @@ class Handle:
         _check(lib().fact_attention(self._h, B, Tq, Tk, Hq, Hkv, D, _ptr(q), *st(q), _ptr(k), *st(k), _ptr(v), *st(v),
                                     _ptr(out), *st(out), 1 if causal else 0, float(scale), self._stream(stream)),
                "fact_attention", self._h)
+        return out
+
+    def norm(self, x, gamma, beta=None, kind="layer", eps=1e-5, out=None, stream=None):
+        """Row normalisation (fact_norm): LayerNorm (kind="layer", gamma and beta) or RMSNorm (kind="rms", gamma).
+        x: [M, C] BF16 (rows may be strided); returns [M, C]."""
+        _need(x, "x", torch.bfloat16, 2)
+        M, C = x.shape
+        if out is None:
+            out = torch.empty((M, C), dtype=torch.bfloat16, device=x.device)
+        _check(lib().fact_norm(self._h, NORMS[kind], M, C, _ptr(x), _ld(x), _ptr(gamma), _ptr(beta), float(eps),
+                               _ptr(out), _ld(out), self._stream(stream)), "fact_norm", self._h)
+        return out
+
+    def block_desc(self, kind, batch, seq, heads_q, heads_kv, head_dim, ffn, weights, eps=1e-5):
+        """A fact_block_t for `weights`: a dict of contiguous BF16 CUDA tensors keyed like the struct's pointer
+        fields (absent or None = NULL).  The dict must outlive the calls that use the descriptor."""
+        b = Block()
+        b.kind = BLOCK_KINDS[kind]
+        b.batch, b.seq, b.hidden = batch, seq, heads_q * head_dim
+        b.heads_q, b.heads_kv, b.head_dim, b.ffn = heads_q, heads_kv, head_dim, ffn
+        b.eps = eps
+        for name in ("norm1_gamma", "norm1_beta", "wqkv", "bqkv", "wo", "bo", "norm2_gamma", "norm2_beta", "w1",
+                     "b1", "w2", "b2"):
+            t = weights.get(name)
+            if t is not None and not t.is_contiguous():
+                raise ValueError(f"{name} must be contiguous")
+            setattr(b, name, None if t is None else int(t.data_ptr()))
+        return b
+
+    def block_forward(self, desc, x, out=None, workspace=None, stream=None):
+        """One transformer block forward (fact_block_forward).  x: [batch * seq, hidden] BF16, contiguous."""
+        _need(x, "x", torch.bfloat16, 2)
+        if not x.is_contiguous():
+            raise ValueError("x must be contiguous")
+        if out is None:
+            out = torch.empty_like(x)
+        need = int(lib().fact_block_workspace_bytes(byref(desc)))
+        if workspace is None:
+            workspace = self.workspace(need)
+        _check(lib().fact_block_forward(self._h, byref(desc), _ptr(x), _ptr(out), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), self._stream(stream)),
+               "fact_block_forward", self._h)
+        return out
+
+    def block_intermediates(self, desc, workspace):
+        """Views of the intermediates a block_forward call left in `workspace` (fact_block_workspace_offsets):
+        dict n (= n2), qkv, a, x1, h, each [tokens, columns] BF16."""
+        off = (c_size_t * 5)()
+        _check(lib().fact_block_workspace_offsets(byref(desc), off), "fact_block_workspace_offsets")
+        tok = int(desc.batch * desc.seq)
+        cols = {"n": desc.hidden, "qkv": (desc.heads_q + 2 * desc.heads_kv) * desc.head_dim, "a": desc.hidden,
+                "x1": desc.hidden, "h": desc.ffn}
+        out = {}
+        for i, name in enumerate(("n", "qkv", "a", "x1", "h")):
+            nbytes = tok * int(cols[name]) * 2
+            out[name] = workspace[int(off[i]): int(off[i]) + nbytes].view(torch.bfloat16).view(tok, int(cols[name]))
         return out
 
     def tune(self, op, A, B, layout="KN", bias=None, residual=None, epilogue="NONE", out=None,

@@ -18,6 +18,7 @@
 #include "fact.h"
 #include "gemm_kernel.cuh"
 #include "attention_kernel.cuh"
+#include "norm_kernel.cuh"
 
 // Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
 // device image, so that entry point never has to allocate.  Every GPU that loads the library holds these
@@ -1016,6 +1017,139 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
   }
   if (dev != h->device) cudaSetDevice(dev);
   return st;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row normalisation and the whole-block chain
+fact_status_t fact_norm(fact_handle_t h, fact_norm_t kind, int64_t M, int64_t C, const void* X, int64_t ldx,
+                        const void* gamma, const void* beta, float eps, void* Y, int64_t ldy, void* stream_v) {
+  if (!h || M < 0 || (kind != FACT_NORM_LAYER && kind != FACT_NORM_RMS)) return FACT_ERR_INVALID_ARG;
+  if (C < 8 || C > 8192 || C % 8) return FACT_ERR_UNSUPPORTED;
+  if (M == 0) return FACT_OK;
+  if (!X || !Y || !gamma || (kind == FACT_NORM_RMS && beta) || !(eps >= 0.f)) return FACT_ERR_INVALID_ARG;
+  if (ldx < C || ldy < C || M > 0x7fffffffLL * kNormWarps) return FACT_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Y) || !aligned16(gamma) || (beta && !aligned16(beta)) || ldx % 8 || ldy % 8)
+    return FACT_ERR_BAD_ALIGNMENT;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  NormParams p;
+  p.X = reinterpret_cast<const __nv_bfloat16*>(X);
+  p.Y = reinterpret_cast<__nv_bfloat16*>(Y);
+  p.gamma = reinterpret_cast<const __nv_bfloat16*>(gamma);
+  p.beta = reinterpret_cast<const __nv_bfloat16*>(beta);
+  p.M = M;
+  p.C = (int)C;
+  p.ldx = ldx;
+  p.ldy = ldy;
+  p.eps = eps;
+  const unsigned grid = (unsigned)((M + kNormWarps - 1) / kNormWarps);
+  const int threads = kNormWarps * 32;
+  const bool rms = kind == FACT_NORM_RMS;
+  // a lane keeps ceil(C / 256) 16-byte chunks of its row in registers
+  if (C <= 1024) {
+    if (rms) fact_norm_kernel<4, true><<<grid, threads, 0, stream>>>(p);
+    else fact_norm_kernel<4, false><<<grid, threads, 0, stream>>>(p);
+  } else if (C <= 4096) {
+    if (rms) fact_norm_kernel<16, true><<<grid, threads, 0, stream>>>(p);
+    else fact_norm_kernel<16, false><<<grid, threads, 0, stream>>>(p);
+  } else {
+    if (rms) fact_norm_kernel<32, true><<<grid, threads, 0, stream>>>(p);
+    else fact_norm_kernel<32, false><<<grid, threads, 0, stream>>>(p);
+  }
+  fact_status_t st = FACT_OK;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) st = cuda_fail(h, "norm launch", e);
+  else h->launches++;
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
+}
+
+namespace {
+// Workspace carve-up of one block (element counts; every buffer starts on a 256-byte boundary).
+struct BlockLayout {
+  int64_t tokens, qkv_cols, h_cols;
+  size_t off_n, off_qkv, off_a, off_x1, off_h, total;
+};
+bool block_layout(const fact_block_t* b, BlockLayout* L) {
+  if (!b || (b->kind != FACT_BLOCK_GPT && b->kind != FACT_BLOCK_LLAMA)) return false;
+  if (b->batch < 0 || b->seq < 0 || b->hidden <= 0 || b->heads_q <= 0 || b->heads_kv <= 0 || b->ffn <= 0) return false;
+  if (b->heads_q % b->heads_kv || b->hidden != b->heads_q * b->head_dim || b->hidden % 8 || b->ffn % 8) return false;
+  if (b->batch > 0 && b->seq > 0x7fffffffLL / std::max<int64_t>(b->batch, 1)) return false;
+  L->tokens = b->batch * b->seq;
+  L->qkv_cols = (b->heads_q + 2 * b->heads_kv) * b->head_dim;
+  L->h_cols = b->ffn;
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  const size_t t = (size_t)L->tokens;
+  L->off_n = 0;
+  L->off_qkv = up(L->off_n + t * (size_t)b->hidden * 2);
+  L->off_a = up(L->off_qkv + t * (size_t)L->qkv_cols * 2);
+  L->off_x1 = up(L->off_a + t * (size_t)b->hidden * 2);
+  L->off_h = up(L->off_x1 + t * (size_t)b->hidden * 2);
+  L->total = up(L->off_h + t * (size_t)L->h_cols * 2);
+  return true;
+}
+}  // namespace
+
+size_t fact_block_workspace_bytes(const fact_block_t* b) {
+  BlockLayout L;
+  return block_layout(b, &L) ? L.total : 0;
+}
+
+fact_status_t fact_block_workspace_offsets(const fact_block_t* b, size_t offsets[5]) {
+  BlockLayout L;
+  if (!offsets || !block_layout(b, &L)) return FACT_ERR_INVALID_ARG;
+  offsets[0] = L.off_n;
+  offsets[1] = L.off_qkv;
+  offsets[2] = L.off_a;
+  offsets[3] = L.off_x1;
+  offsets[4] = L.off_h;
+  return FACT_OK;
+}
+
+fact_status_t fact_block_forward(fact_handle_t h, const fact_block_t* b, const void* x, void* y, void* ws,
+                                 size_t ws_bytes, void* stream) {
+  BlockLayout L;
+  if (!h || !block_layout(b, &L)) return FACT_ERR_INVALID_ARG;
+  if (b->head_dim != 64 && b->head_dim != 128) return FACT_ERR_UNSUPPORTED;
+  if (L.tokens == 0) return FACT_OK;
+  const bool llama = b->kind == FACT_BLOCK_LLAMA;
+  if (!x || !y || !b->norm1_gamma || !b->norm2_gamma || !b->wqkv || !b->wo || !b->w1 || !b->w2) return FACT_ERR_INVALID_ARG;
+  if (llama && (b->norm1_beta || b->norm2_beta || b->bqkv || b->bo || b->b1 || b->b2)) return FACT_ERR_INVALID_ARG;
+  if (!llama && !b->b1) return FACT_ERR_INVALID_ARG;  // the GELU epilogue carries the bias
+  if (!ws || ws_bytes < L.total) return FACT_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
+  uint8_t* w8 = reinterpret_cast<uint8_t*>(ws);
+  void* n = w8 + L.off_n;
+  __nv_bfloat16* qkv = reinterpret_cast<__nv_bfloat16*>(w8 + L.off_qkv);
+  void* a = w8 + L.off_a;
+  void* x1 = w8 + L.off_x1;
+  void* hbuf = w8 + L.off_h;
+  const int64_t T = L.tokens, C = b->hidden, D = b->head_dim, QC = L.qkv_cols;
+  const fact_norm_t nk = llama ? FACT_NORM_RMS : FACT_NORM_LAYER;
+  fact_status_t st = fact_norm(h, nk, T, C, x, C, b->norm1_gamma, b->norm1_beta, b->eps, n, C, stream);
+  if (st != FACT_OK) return st;
+  st = fact_linear(h, T, QC, C, n, C, b->wqkv, C, FACT_B_NK, b->bqkv, nullptr, 0, qkv, QC, FACT_OUT_BF16,
+                   b->bqkv ? FACT_EPI_BIAS : FACT_EPI_NONE, nullptr, nullptr, 0, stream);
+  if (st != FACT_OK) return st;
+  // Q, K, V are column ranges of qkv: token stride QC, head stride D, batch stride seq * QC
+  const __nv_bfloat16* qp = qkv;
+  const __nv_bfloat16* kp = qkv + b->heads_q * D;
+  const __nv_bfloat16* vp = kp + b->heads_kv * D;
+  st = fact_attention(h, b->batch, b->seq, b->seq, b->heads_q, b->heads_kv, D, qp, b->seq * QC, QC, D, kp, b->seq * QC,
+                      QC, D, vp, b->seq * QC, QC, D, a, b->seq * C, C, D, 1, 0.f, stream);
+  if (st != FACT_OK) return st;
+  st = fact_linear(h, T, C, C, a, C, b->wo, C, FACT_B_NK, b->bo, x, C, x1, C, FACT_OUT_BF16, FACT_EPI_BIAS_RESIDUAL,
+                   nullptr, nullptr, 0, stream);
+  if (st != FACT_OK) return st;
+  st = fact_norm(h, nk, T, C, x1, C, b->norm2_gamma, b->norm2_beta, b->eps, n, C, stream);
+  if (st != FACT_OK) return st;
+  st = fact_linear(h, T, b->ffn, C, n, C, b->w1, C, FACT_B_NK, b->b1, nullptr, 0, hbuf, b->ffn, FACT_OUT_BF16,
+                   llama ? FACT_EPI_SILU_GATE : FACT_EPI_BIAS_GELU_TANH, nullptr, nullptr, 0, stream);
+  if (st != FACT_OK) return st;
+  return fact_linear(h, T, C, b->ffn, hbuf, b->ffn, b->w2, b->ffn, FACT_B_NK, b->b2, x1, C, y, C, FACT_OUT_BF16,
+                     FACT_EPI_BIAS_RESIDUAL, nullptr, nullptr, 0, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

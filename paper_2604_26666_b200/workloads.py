@@ -220,3 +220,67 @@ def make_attention_inputs(case, device="cpu"):
     k = torch.randn(case.B, case.T, case.Hkv, case.D, generator=gen).to(torch.bfloat16)
     v = torch.randn(case.B, case.T, case.Hkv, case.D, generator=gen).to(torch.bfloat16)
     return q.to(device), k.to(device), v.to(device)
+
+
+# ------------------------------------------------------------------------------------------------
+# Whole transformer blocks (Section 5.2: the MiniGPT block at (128, 512, 768), the Llama-3-8B block at (16, 2048, 4096))
+@dataclass(frozen=True)
+class BlockCase:
+    """One pre-norm transformer block: x [B * T, Hq * D] BF16 and its weights."""
+    name: str
+    kind: str  # "gpt": layer norms, biases, GELU MLP;  "llama": RMS norms, no biases, SwiGLU, grouped queries
+    B: int
+    T: int
+    Hq: int
+    Hkv: int
+    D: int
+    ffn: int
+    seed: int
+
+    @property
+    def hidden(self) -> int:
+        return self.Hq * self.D
+
+    @property
+    def flops(self) -> float:
+        """Algorithmic FLOPs of the four linears and the causal attention (normalisations not counted)."""
+        tok, C = self.B * self.T, self.hidden
+        qc = (self.Hq + 2 * self.Hkv) * self.D
+        mlp = (2 if self.kind == "llama" else 1) * self.ffn * C + C * self.ffn
+        lin = 2.0 * tok * (qc * C + C * C + mlp)
+        att = 4.0 * self.D * (self.T * (self.T + 1) / 2) * self.B * self.Hq
+        return lin + att
+
+
+def block_cases():
+    """The paper's two block shapes."""
+    return [BlockCase("gpt_block_128x512x768", "gpt", 128, 512, 12, 12, 64, 3072, 7100),
+            BlockCase("llama_block_16x2048x4096", "llama", 16, 2048, 32, 8, 128, 14336, 7101)]
+
+
+BLOCK_WEIGHT_NAMES = ("norm1_gamma", "norm1_beta", "wqkv", "bqkv", "wo", "bo", "norm2_gamma", "norm2_beta", "w1", "b1",
+                      "w2", "b2")
+
+
+def make_block_inputs(case, device="cpu"):
+    """Seeded BF16 x ~ N(0, 1) and weights: linear weights N(0, 0.02^2) (the configurations' weight scale), norm
+    gains 1 + N(0, 0.1^2), norm offsets and biases N(0, 0.02^2); a Llama block has gains and weights only.
+    Returns (x, dict name -> tensor), drawn in the order of BLOCK_WEIGHT_NAMES after x."""
+    import torch
+
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(case.seed)
+    C, qc = case.hidden, (case.Hq + 2 * case.Hkv) * case.D
+    shapes = {"norm1_gamma": (C,), "norm1_beta": (C,), "wqkv": (qc, C), "bqkv": (qc,), "wo": (C, C), "bo": (C,),
+              "norm2_gamma": (C,), "norm2_beta": (C,), "w1": ((2 if case.kind == "llama" else 1) * case.ffn, C),
+              "b1": (case.ffn,), "w2": (C, case.ffn), "b2": (C,)}
+    x = torch.randn(case.B * case.T, C, generator=gen).to(torch.bfloat16).to(device)
+    w = {}
+    for name in BLOCK_WEIGHT_NAMES:
+        vector = len(shapes[name]) == 1
+        if case.kind == "llama" and vector and "gamma" not in name:
+            continue
+        t = torch.randn(*shapes[name], generator=gen)
+        t = 1.0 + 0.1 * t if "gamma" in name else 0.02 * t
+        w[name] = t.to(torch.bfloat16).to(device)
+    return x, w
