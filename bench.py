@@ -386,7 +386,7 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
     from paper_2604_26666_b200 import workloads as wl
 
     rows = []
-    for case in wl.benchmark_cases(layout):
+    for case in wl.benchmark_cases(layout) + wl.paper_cases():
         if names is not None and case.name not in names:
             continue
         ins = wl.make_inputs(case)

@@ -112,8 +112,18 @@ def benchmark_cases(layout_linear: str = "NK") -> list[Case]:
     return c
 
 
+def paper_cases() -> list[Case]:
+    """The paper's own Level-1 shapes where they differ from the benchmark configurations (Section 5.1): Problem 3,
+    a batch of 128 products 512 x 1024 . 1024 x 2048, and Problem 6, 256 x 524288 . 524288 x 256 with FP32 output.
+    (Problem 1, 4096^3, is configuration 2.)  config = 0 marks them as extras."""
+    return [Case("p3_batched_128x512x2048x1024", "gemm_batched", 512, 2048, 1024, batch=128, layout="KN", seed=12,
+                 config=0),
+            Case("p6_splitk_256x256x524288", "gemm_splitk", 256, 256, 524288, layout="KN", out="f32", seed=16,
+                 x_dist="uniform", w_dist="uniform", config=0)]
+
+
 def case_by_name(name: str, layout_linear: str = "NK") -> Case:
-    for cs in benchmark_cases(layout_linear):
+    for cs in benchmark_cases(layout_linear) + paper_cases():
         if cs.name == name:
             return cs
     raise KeyError(name)
