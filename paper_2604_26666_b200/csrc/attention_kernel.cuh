@@ -8,10 +8,12 @@
 // final division by l removes the stale reference exactly).  All roles run ahead across tile boundaries, so the
 // loads, the first product and the Q copy of the next tile overlap the last blocks and the epilogue of this one.
 //   warp 8      TMA producer: K and V blocks into two three-stage rings; the next tile's Q into a staging buffer
-//   warp 9      MMA issuer, one block ahead with the first product:
+//   warp 9      issuer of the first products, up to two blocks ahead of the softmax:
 //                 Q                    tcgen05.cp from the staging buffer into tensor memory, once per tile
 //                 S(g)  = Q K^T        tcgen05.mma, M = 128, N = 128, K = head_dim, A = Q read from tensor memory
-//                                      (so the product reads only K from shared memory), into score buffer g & 1
+//                                      (so the product reads only K from shared memory), into score buffer g & 1,
+//                                      once O += P(g-2) V has completed (P(g-2) lived in that buffer)
+//   warp 11     issuer of the second products:
 //                 O    += P(g) V       tcgen05.mma, M = 128, N = head_dim, K = 128, A = P(g) read from tensor memory
 //   warp 10     store warp: a finished tile's O / l from its staging buffer to global memory by TMA
 //   warps 0-7   softmax: two threads per query row (warps w and w + 4 share a lane quarter and split the block's
@@ -24,8 +26,8 @@
 // Tensor memory (512 columns): S/P buffer 0 at 0, buffer 1 at 128, O at 256, Q at 384 (two BF16 values per
 // column; one buffer is enough because the copy of the next tile's Q follows this tile's last first-product on
 // the in-order tensor pipe).  P(g) may overwrite S(g) because both threads of a row have read their scores
-// before either stores (the exchange of the maxima orders them), and S(g+2) is issued after O += P(g) V on the same
-// in-order pipe.  Every mbarrier wait is bounded, as in the GEMM kernel; the named barriers between the two warps
+// before either stores (the exchange of the maxima orders them), and S(g+2) is issued once O += P(g) V has
+// completed.  Every mbarrier wait is bounded, as in the GEMM kernel; the named barriers between the two warps
 // of a row are reached unconditionally, also by a warp whose wait gave up.
 #pragma once
 #include <cuda.h>
@@ -38,11 +40,12 @@
 
 namespace fact {
 
-constexpr int kAttnThreads = 384;   // 12 warps: 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 spare
+constexpr int kAttnThreads = 384;   // 12 warps: 0-7 softmax, 8 TMA producer, 9 and 11 MMA issuers, 10 store
 constexpr int kAttnBlockQ = 128;    // query rows per tile (= TMEM lanes)
 constexpr int kAttnBlockK = 128;    // keys per block
 constexpr int kAttnStagesK = 3;     // K ring depth: a K block is wanted one block before its V block
-constexpr int kAttnStagesV = 2;     // V ring depth
+constexpr int kAttnStagesV = 2;     // V ring depth (two: block g's V slot, g & 1, is released when O += P(g) V has completed,
+                                    // which is also the event the softmax warps wait for before rescaling O)
 constexpr uint32_t kAttnChunkBytes = 128 * 128;  // one 64-column chunk of a 128-row tile, 128-byte rows
 constexpr float kAttnRescaleThreshold = 8.f;     // log2 units
 // Registers per thread after the warpgroups rebalance (setmaxnreg): the eight softmax warps take what the other four
@@ -51,6 +54,7 @@ constexpr float kAttnRescaleThreshold = 8.f;     // log2 units
 constexpr int kAttnRegsSoftmax = 208;
 constexpr int kAttnRegsOther = 80;
 constexpr int kAttnRegsAtLaunch = 168;
+static_assert(kAttnStagesV == 2, "the softmax warps use V_EMPTY[g & 1] as \"O += P(g) V has completed\"");
 static_assert(4 * kAttnRegsOther + 8 * kAttnRegsSoftmax <= 12 * kAttnRegsAtLaunch, "setmaxnreg requests exceed the pool");
 
 struct AttnParams {
@@ -62,7 +66,9 @@ struct AttnParams {
   uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (K)
   uint64_t v_desc;            // UMMA descriptor template, V as an N-major operand
   uint32_t idesc_s, idesc_pv;
-  int* status;                // [0] error word; with debug bit 256 eight 64-bit counters of the first CTA from [2]:
+  int* status;                // (debug bits 8 / 16 / 64 / 128 switch off the softmax arithmetic / the K, V loads /
+                              // the first / the second product: experiments on where the time goes, results wrong)
+                              // [0] error word; with debug bit 256 eight 64-bit counters of the first CTA from [2]:
                               // cycles, nanoseconds, first wait that gave up, cycles warp 0 waited for scores, its
                               // blocks, -, cycles it spent finishing tiles, its tiles
   int debug;
@@ -79,6 +85,7 @@ struct AttnTile {
   int b, h, kvh, t0, nb;
 };
 
+template <int HD>  // head_dim: 64 or 128
 __global__ void __launch_bounds__(kAttnThreads, 1)
     fact_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -94,7 +101,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const bool prof = (p.debug & 256) && blockIdx.x == 0;
   const long long t_entry = prof ? clock64() : 0;
   const unsigned long long ns_entry = prof ? ptx::globaltimer_ns() : 0ull;
-  const uint32_t tile_bytes = attn_tile_bytes(p.D);
+  constexpr uint32_t tile_bytes = attn_tile_bytes(HD);
   const uint32_t k_s0 = smem_base;
   const uint32_t v_s0 = k_s0 + (uint32_t)kAttnStagesK * tile_bytes;
   const uint32_t q_stage = v_s0 + (uint32_t)kAttnStagesV * tile_bytes;
@@ -114,8 +121,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     V_EMPTY = K_EMPTY + kAttnStagesK,
     S_FULL = V_EMPTY + kAttnStagesV,  // two: one per score buffer
     P_FULL = S_FULL + 2,              // two: a warp may finish block g + 1 before another has finished block g
-    PV_DONE = P_FULL + 2,
-    O_DONE = PV_DONE + 1,             // a tile's last product has completed (PV_DONE's one-bit phase cannot tell
+    O_DONE = P_FULL + 2,              // a tile's last product has completed (the one-bit phase of V_EMPTY cannot tell
                                       // "two products behind" from "done", so the epilogue has its own barrier)
     O_FREE = O_DONE + 1,              // the softmax warps have read a finished tile's O
     O_STAGED = O_FREE + 1,            // ... and written O / l into the staging buffer
@@ -169,11 +175,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     t.nb = p.causal ? min(kv_blocks_all, qt + 1) : kv_blocks_all;
     return t;
   };
-  const int chunks = p.D / 64;
+  constexpr int chunks = HD / 64;
+  // A wait that is already satisfied costs one try_wait and a vote.  (The abort flag is read only on the slow
+  // path: a volatile generic load of shared memory costs about 170 cycles here, which on every wait of the MMA
+  // warp was most of its time.)
   auto wait_all = [&](uint32_t br, uint32_t parity) -> bool {
-    const bool was_aborted = *abort_p != 0;
+    if (__all_sync(0xffffffffu, ptx::mbar_try_wait(br, parity))) return true;
     const bool okw = __all_sync(0xffffffffu, wait_bar(br, parity, abort_p, p.status)) != 0;
-    if (!okw && !was_aborted && lane == 0 && (p.debug & 256))  // which wait gave up first: barrier index, warp, CTA
+    if (!okw && lane == 0 && (p.debug & 256))  // which wait gave up first: barrier index, warp, CTA
       atomicCAS(reinterpret_cast<unsigned long long*>(p.status + 6), 0ull,
                 (unsigned long long)((br - bar_base) / 8u) | ((unsigned long long)warp << 8) |
                     ((unsigned long long)blockIdx.x << 16) | (1ull << 40));
@@ -196,13 +205,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     if (n_items > 0) load_q(0);
     int ks = 0, vs = 0;
     uint32_t kpar = 1, vpar = 1;  // an empty slot's first wait passes
+    const bool skip_loads = (p.debug & 16) != 0;  // experiment switch: K and V are loaded once only
     bool ok = true;
     for (int n = 0; ok && n < n_items; ++n) {
       const AttnTile t = tile_of(n);
       for (int j = 0; ok && j < t.nb; ++j) {
         ok = wait_all(bar(K_EMPTY + ks), kpar);
         if (!ok) break;
-        if (ptx::elect_one()) {
+        if (skip_loads && n + j > 0) {
+          if (ptx::elect_one()) ptx::mbar_arrive(bar(K_FULL + ks));
+        } else if (ptx::elect_one()) {
           ptx::mbar_arrive_expect_tx(bar(K_FULL + ks), tile_bytes);
           for (int c = 0; c < chunks; ++c)
             ptx::tma_load_4d(k_s0 + ks * tile_bytes + c * kAttnChunkBytes, &tmK, bar(K_FULL + ks), c * 64, t.kvh,
@@ -214,7 +226,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         ok = wait_all(bar(V_EMPTY + vs), vpar);
         if (!ok) break;
-        if (ptx::elect_one()) {
+        if (skip_loads && n + j > 0) {
+          if (ptx::elect_one()) ptx::mbar_arrive(bar(V_FULL + vs));
+        } else if (ptx::elect_one()) {
           ptx::mbar_arrive_expect_tx(bar(V_FULL + vs), tile_bytes);
           for (int c = 0; c < chunks; ++c)
             ptx::tma_load_4d(v_s0 + vs * tile_bytes + c * kAttnChunkBytes, &tmV, bar(V_FULL + vs), c * 64, t.kvh,
@@ -233,78 +247,82 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     }
     __syncwarp();
   } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
-    int ks = 0, vs = 0;  // ring slots of the next K block to multiply and the next V block
-    uint32_t kpar = 0, vpar = 0;
-    int sn = 0, sj = 0, sg = 0;  // the next first product to issue: tile ordinal, block in the tile, global block
-    int s_nb = n_items > 0 ? tile_of(0).nb : 0;
-    auto issue_next_s = [&]() -> bool {  // S(sg) = Q K^T into score buffer sg & 1; releases the K block when done
-      if (sn >= n_items) return true;
-      if (sj == 0) {  // a new tile: its Q from the staging buffer into tensor memory, 16 elements of every row a copy
-        if (!wait_all(bar(QS_FULL), (uint32_t)sn & 1u)) return false;
-        ptx::tc_fence_after();
-        if (ptx::elect_one()) {
-          for (int kk = 0; kk < p.D / kUmmaK; ++kk) {
-            const uint32_t off = (uint32_t)(kk >> 2) * kAttnChunkBytes + (uint32_t)(kk & 3) * 32u;
-            ptx::tmem_cp_128x256b(tmem_q + (uint32_t)kk * 8u, p.kmajor_desc | (uint64_t)(((q_stage + off) >> 4) & 0x3fffu));
-          }
-          ptx::umma_commit<1>(bar(QS_EMPTY));
-        }
-      }
-      if (!wait_all(bar(K_FULL + ks), kpar)) return false;
+    // ------------------------------------------------------------ issuer of the first products, S(g) = Q K^T
+    // Two warps issue tensor-core work, one per kind of product: the queue behind the issuing thread is shallow,
+    // so a single issuer's waits and commits between two batches leave the pipe idle; with two, each one's
+    // bookkeeping hides behind the other's batch.  What in-order issue from one thread gave for free is now an
+    // explicit wait: S(g) overwrites the buffer that held P(g-2), so it follows the completion of O += P(g-2) V.
+    const bool skip_s = (p.debug & 64) != 0;  // experiment switch, 0 in normal use
+    int ks = 0;
+    uint32_t kpar = 0;
+    int g = 0;
+    bool ok = true;
+    for (int n = 0; ok && n < n_items; ++n) {
+      const int nb = tile_of(n).nb;
+      // a new tile: its Q from the staging buffer into tensor memory, 16 elements of every row a copy (the copy
+      // follows this thread's earlier products, the last readers of the previous tile's Q, on the in-order pipe)
+      ok = wait_all(bar(QS_FULL), (uint32_t)n & 1u);
+      if (!ok) break;
       ptx::tc_fence_after();
       if (ptx::elect_one()) {
-        const uint32_t kaddr = k_s0 + (uint32_t)ks * tile_bytes;
-        const uint32_t d = tmem_base + (uint32_t)(sg & 1) * 128u;
-        const uint32_t qa = tmem_q;
-        for (int kk = 0; kk < p.D / kUmmaK; ++kk) {
+#pragma unroll
+        for (int kk = 0; kk < HD / kUmmaK; ++kk) {
           const uint32_t off = (uint32_t)(kk >> 2) * kAttnChunkBytes + (uint32_t)(kk & 3) * 32u;
-          const uint64_t bdesc = p.kmajor_desc | (uint64_t)(((kaddr + off) >> 4) & 0x3fffu);
-          ptx::umma_bf16_ts(d, qa + (uint32_t)kk * 8u, bdesc, p.idesc_s, kk > 0 ? 1u : 0u);  // 8 columns = 16 BF16
+          ptx::tmem_cp_128x256b(tmem_q + (uint32_t)kk * 8u, p.kmajor_desc | (uint64_t)(((q_stage + off) >> 4) & 0x3fffu));
         }
-        ptx::umma_commit<1>(bar(S_FULL + (sg & 1)));
-        ptx::umma_commit<1>(bar(K_EMPTY + ks));
+        ptx::umma_commit<1>(bar(QS_EMPTY));
       }
-      if (++ks == kAttnStagesK) {
-        ks = 0;
-        kpar ^= 1u;
+      for (int j = 0; ok && j < nb; ++j, ++g) {
+        ok = wait_all(bar(K_FULL + ks), kpar);
+        if (ok && g >= 2) ok = wait_all(bar(V_EMPTY + (g & 1)), (((uint32_t)g >> 1) - 1u) & 1u);  // O += P(g-2) V done
+        if (!ok) break;
+        ptx::tc_fence_after();
+        if (ptx::elect_one()) {
+          const uint32_t kaddr = k_s0 + (uint32_t)ks * tile_bytes;
+          const uint32_t d = tmem_base + (uint32_t)(g & 1) * 128u;
+          // (shared-memory addresses stay below 2^18, so adding an offset never carries out of the 14-bit field)
+          const uint64_t kdesc0 = p.kmajor_desc | (uint64_t)((kaddr >> 4) & 0x3fffu);
+#pragma unroll
+          for (int kk = 0; kk < HD / kUmmaK; ++kk) {  // 16 elements of head_dim: 8 columns of Q, 32 bytes of a K row
+            const uint32_t off = (uint32_t)(kk >> 2) * kAttnChunkBytes + (uint32_t)(kk & 3) * 32u;
+            if (!skip_s) ptx::umma_bf16_ts(d, tmem_q + (uint32_t)kk * 8u, kdesc0 + (uint64_t)(off >> 4), p.idesc_s, kk > 0 ? 1u : 0u);
+          }
+          ptx::umma_commit<1>(bar(S_FULL + (g & 1)));
+          ptx::umma_commit<1>(bar(K_EMPTY + ks));
+        }
+        if (++ks == kAttnStagesK) {
+          ks = 0;
+          kpar ^= 1u;
+        }
       }
-      ++sg;
-      if (++sj == s_nb) {
-        sj = 0;
-        ++sn;
-        s_nb = sn < n_items ? tile_of(sn).nb : 0;
-      }
-      return true;
-    };
-    bool ok = issue_next_s();
+    }
+    __syncwarp();
+  } else if (warp == 11) {
+    // ------------------------------------------------------------ issuer of the second products, O += P(g) V
+    const bool skip_pv = (p.debug & 128) != 0;  // experiment switch, 0 in normal use
     int g = 0;
+    bool ok = true;
     for (int n = 0; ok && n < n_items; ++n) {
       const int nb = tile_of(n).nb;
       for (int j = 0; ok && j < nb; ++j, ++g) {
-        // score buffer (g + 1) & 1 held P(g-1), which O += P(g-1) V (issued in the previous iteration) reads first
-        ok = issue_next_s();
-        if (!ok) break;
-        ok = wait_all(bar(P_FULL + (g & 1)), ((uint32_t)g >> 1) & 1u);
+        const int vs = g & 1;
+        ok = wait_all(bar(P_FULL + vs), ((uint32_t)g >> 1) & 1u);
         // the first block of a tile overwrites O: the previous tile's epilogue must have read it
         if (ok && j == 0 && n > 0) ok = wait_all(bar(O_FREE), (uint32_t)(n - 1) & 1u);
-        if (ok) ok = wait_all(bar(V_FULL + vs), vpar);
+        if (ok) ok = wait_all(bar(V_FULL + vs), ((uint32_t)g >> 1) & 1u);
         if (!ok) break;
         ptx::tc_fence_after();
-        if (ptx::elect_one()) {  // O += P(g) V
+        if (ptx::elect_one()) {
           const uint32_t vaddr = v_s0 + (uint32_t)vs * tile_bytes;
-          const uint32_t p_t = tmem_base + (uint32_t)(g & 1) * 128u;  // BF16 pairs: 8 columns per 16 keys
-          for (int kk = 0; kk < kAttnBlockK / kUmmaK; ++kk) {
-            const uint64_t bdesc = p.v_desc | (uint64_t)(((vaddr + (uint32_t)kk * 2048u) >> 4) & 0x3fffu);
-            ptx::umma_bf16_ts(tmem_o, p_t + (uint32_t)kk * 8u, bdesc, p.idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
-          }
+          const uint32_t p_t = tmem_base + (uint32_t)vs * 128u;  // BF16 pairs: 8 columns per 16 keys
+          const uint64_t vdesc0 = p.v_desc | (uint64_t)((vaddr >> 4) & 0x3fffu);
+#pragma unroll
+          for (int kk = 0; kk < kAttnBlockK / kUmmaK; ++kk)  // 16 keys = 2048 bytes further on in V, 8 columns in P
+            if (!skip_pv)
+              ptx::umma_bf16_ts(tmem_o, p_t + (uint32_t)kk * 8u, vdesc0 + (uint64_t)(kk * 128), p.idesc_pv,
+                                (j > 0 || kk > 0) ? 1u : 0u);
           ptx::umma_commit<1>(bar(V_EMPTY + vs));
-          ptx::umma_commit<1>(bar(PV_DONE));
           if (j == nb - 1) ptx::umma_commit<1>(bar(O_DONE));
-        }
-        if (++vs == kAttnStagesV) {
-          vs = 0;
-          vpar ^= 1u;
         }
       }
     }
@@ -335,7 +353,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const int row = q4 * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
     const uint32_t pair_bar = 1u + (uint32_t)q4;  // named barrier of this warp and its partner (warp +- 4)
-    const int o_cols = p.D / 2;                   // output columns this thread rescales and stores
+    constexpr int o_cols = HD / 2;                // output columns this thread rescales and stores
     const uint32_t o_addr = tmem_o + lane_addr + (uint32_t)(half * o_cols);
     bool ok = true;  // warp-uniform; a warp whose wait gave up keeps meeting its partner at the named barriers
     long long prof_s_wait = 0, prof_epi = 0, prof_blocks = 0;
@@ -409,6 +427,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           prof_s_wait += clock64() - tc1;
           ++prof_blocks;
         }
+        if (p.debug & 8) {  // experiment switch: no softmax arithmetic, the barrier protocol only
+          ptx::named_bar_sync(pair_bar, 64);
+          if (j == 0 && pend) finish_tile((g + 1) & 1);
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(bar(P_FULL + (g & 1)));
+          continue;
+        }
         const uint32_t buf = tmem_base + lane_addr + (uint32_t)(g & 1) * 128u;
         uint32_t sraw[2][32];
         float hm = -INFINITY;
@@ -454,7 +480,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           m = m_new;
           if (j > 0) {
             // O is rescaled between O += P(g-1) V, which must have completed, and O += P(g) V, which waits for P(g)
-            ok = wait_all(bar(PV_DONE), (uint32_t)(g - 1) & 1u);
+            ok = wait_all(bar(V_EMPTY + ((g - 1) & 1)), ((uint32_t)(g - 1) >> 1) & 1u);
             if (!ok) continue;  // j > 0: no finished tile is pending here
             ptx::tc_fence_after();
             for (int c = 0; c < o_cols; c += 32) {

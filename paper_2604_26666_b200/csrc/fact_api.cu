@@ -994,9 +994,13 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
     if (!(h->configured_mask & (1u << 30))) {
-      cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-      cudaFuncAttributes fa;
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel);
+      cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      cudaFuncAttributes fa, fb;
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel<64>);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128>);
+      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
       if (e != cudaSuccess) {
         st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
       } else if (fa.numRegs < kAttnRegsAtLaunch) {
@@ -1009,7 +1013,8 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      fact_attention_kernel<<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      else fact_attention_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
       else h->launches++;
