@@ -175,26 +175,6 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
   }
 }
 
-// The same bounded wait as a tight poll (test_wait): lower wake-up latency, for a warp that has nothing else to do.
-__device__ __forceinline__ bool wait_bar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                              unsigned long long limit_ns = kWaitLimitNs) {
-  unsigned long long t0 = 0;
-  for (uint32_t it = 1;; ++it) {
-    if (ptx::mbar_test_wait(bar, parity)) return true;
-    if ((it & 4095u) == 0) {
-      if (*abort_flag) return false;
-      const unsigned long long now = ptx::globaltimer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > limit_ns) {
-        *abort_flag = 1;
-        atomicExch(status, kDeviceTimeoutCode);
-        return false;
-      }
-    }
-  }
-}
-
 __device__ __forceinline__ void unpack_bf16x8(const uint4& q, float (&f)[8]) {
   f[0] = __uint_as_float(q.x << 16);
   f[1] = __uint_as_float(q.x & 0xffff0000u);

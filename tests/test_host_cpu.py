@@ -89,3 +89,49 @@ def test_inputs_are_reproducible_and_scaled():
     assert torch.equal(a.X, b.X) and torch.equal(a.W, b.W)
     assert a.X.dtype == torch.bfloat16 and a.W.shape == (4096, 48)
     assert abs(float(a.X.float().std()) * 64.0 - 1.0) < 0.05  # N(0,1)/sqrt(4096)
+
+
+def test_block_workspace_layout_is_host_only_and_consistent():
+    """fact_block_workspace_bytes / _offsets need no GPU: sizes, order, alignment, rejection of bad descriptors."""
+    from ctypes import byref, c_size_t
+
+    from paper_2604_26666_b200 import binding
+
+    L = binding.lib()
+    b = binding.Block()
+    b.kind, b.batch, b.seq, b.hidden, b.heads_q, b.heads_kv, b.head_dim, b.ffn = 1, 16, 2048, 4096, 32, 8, 128, 14336
+    tok = 16 * 2048
+    off = (c_size_t * 5)()
+    assert L.fact_block_workspace_offsets(byref(b), off) == 0
+    o = [int(v) for v in off]
+    sizes = [tok * 4096 * 2, tok * 6144 * 2, tok * 4096 * 2, tok * 4096 * 2, tok * 14336 * 2]
+    assert o[0] == 0 and all(x % 256 == 0 for x in o)
+    for i in range(4):
+        assert o[i + 1] >= o[i] + sizes[i]  # buffers in order, no overlap
+    total = int(L.fact_block_workspace_bytes(byref(b)))
+    assert total >= o[4] + sizes[4] and total - (o[4] + sizes[4]) < 256
+    b.heads_kv = 5  # 32 query heads cannot share 5 key/value heads
+    assert int(L.fact_block_workspace_bytes(byref(b))) == 0
+    assert L.fact_block_workspace_offsets(byref(b), off) == 1  # FACT_ERR_INVALID_ARG
+    b.heads_kv, b.hidden = 8, 4000  # hidden != heads_q * head_dim
+    assert int(L.fact_block_workspace_bytes(byref(b))) == 0
+
+
+def test_attention_and_block_workloads():
+    cases = {c.name: c for c in wl.attention_cases()}
+    assert len(cases) == 8
+    c = cases["llama_4x2048_causal"]
+    assert c.flops == 4.0 * 128 * (2048 * 2049 / 2) * 4 * 32
+    assert cases["llama_4x2048_full"].algorithmic_bytes == 2 * 4 * 2048 * 128 * (2 * 32 + 2 * 8)
+    q, k, v = wl.make_attention_inputs(wl.AttentionCase("t", 1, 5, 4, 2, 8, True, 3))
+    assert q.shape == (1, 5, 4, 8) and k.shape == v.shape == (1, 5, 2, 8)
+    q2, _, _ = wl.make_attention_inputs(wl.AttentionCase("t", 1, 5, 4, 2, 8, True, 3))
+    assert (wl.bits(q) == wl.bits(q2)).all()
+    gpt, llama = wl.block_cases()
+    assert (gpt.B, gpt.T, gpt.hidden, gpt.ffn) == (128, 512, 768, 3072)
+    assert (llama.B, llama.T, llama.hidden, llama.Hq, llama.Hkv, llama.ffn) == (16, 2048, 4096, 32, 8, 14336)
+    x, w = wl.make_block_inputs(wl.BlockCase("t", "llama", 1, 4, 2, 1, 8, 16, 5))
+    assert sorted(w) == ["norm1_gamma", "norm2_gamma", "w1", "w2", "wo", "wqkv"] and w["w1"].shape == (32, 16)
+    x, w = wl.make_block_inputs(wl.BlockCase("t", "gpt", 1, 4, 2, 2, 8, 16, 5))
+    assert len(w) == 12 and w["w1"].shape == (16, 16) and w["bqkv"].shape == (48,)
+    assert [c.name for c in wl.paper_cases()] == ["p3_batched_128x512x2048x1024", "p6_splitk_256x256x524288"]
