@@ -133,7 +133,11 @@ def oracle_time_case(case, ins, target_seconds: float):
         oracle.linear(xb, wb, layout=case.layout, epilogue=case.epilogue, bias=bias, residual=res, rows=idx)
         return time.perf_counter() - t0
 
+    # two probes: the first call pays for thread start-up and cold caches and underestimates the rate
     probe_rows = min(case.M, 64)
+    t_probe = run(probe_rows)
+    rate = probe_rows * flops_per_row / max(t_probe, 1e-9)
+    probe_rows = int(max(probe_rows, min(case.M, 1.5 * rate / flops_per_row)))
     t_probe = run(probe_rows)
     rate = probe_rows * flops_per_row / max(t_probe, 1e-9)
     rows = int(max(probe_rows, min(case.M, target_seconds * rate / flops_per_row)))
