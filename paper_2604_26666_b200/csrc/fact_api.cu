@@ -144,10 +144,14 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
                              fact_config_t* out) {
   fact_config_t c;
   memset(&c, 0, sizeof c);
+  bool from_table = false;
   if (user) c = *user;
   else {
     auto it = h->table.find(make_key(q));
-    if (it != h->table.end()) c = it->second;
+    if (it != h->table.end()) {
+      c = it->second;
+      from_table = true;
+    }
   }
   if (splits_override > 0) c.split_k = splits_override;
   if (c.tile_k != 0 && c.tile_k != kTileK) return FACT_ERR_UNSUPPORTED;
@@ -193,6 +197,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (!tile_ok(q, c.tile_n, c.cta_group)) return FACT_ERR_UNSUPPORTED;
   const int smax = max_stages_for(q, c.tile_n, c.cta_group);
   if (c.stages == 0) c.stages = smax;
+  if (from_table && c.stages > smax) c.stages = smax;  // a table written when the other buffers were smaller
   if (c.stages < 2 || c.stages > smax) return FACT_ERR_UNSUPPORTED;
   if (c.raster_group == 0) {
     // Raster model.  With a group of G m-tiles the CTAs walk the n-tiles of that group; the group's slab of X

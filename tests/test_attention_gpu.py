@@ -137,6 +137,46 @@ def test_block_shapes_sampled_rows(h, name):
     check(h, q, k, v, True, rows=rows)
 
 
+@pytest.mark.parametrize("causal", [True, False])
+def test_many_ragged_tiles_per_cta(h, causal):
+    """960 work items over 148 persistent CTAs: every CTA walks several tiles, the last tile of each sequence is
+    ragged (333 = 2 * 128 + 77) and, when causal, the tiles of one CTA have different numbers of key blocks."""
+    B, T, Hq, Hkv, D = 40, 333, 8, 2, 64
+    q, k, v = rnd((B, T, Hq, D), 31), rnd((B, T, Hkv, D), 32), rnd((B, T, Hkv, D), 33)
+    check(h, q, k, v, causal)
+
+
+def test_long_sequence_sampled_rows(h):
+    # 8192 keys: 64 key blocks per tile; reference maxima move late in the row for some rows (scores scaled up)
+    B, T, Hq, Hkv, D = 1, 8192, 4, 1, 128
+    q, k, v = rnd((B, T, Hq, D), 34, 1.5), rnd((B, T, Hkv, D), 35, 1.5), rnd((B, T, Hkv, D), 36)
+    rows = np.array(sorted({0, 127, 128, 4095, 4096, 8000, 8191}), dtype=np.int64)
+    check(h, q, k, v, True, rows=rows)
+    check(h, q, k, v, False, rows=rows)
+
+
+def test_reference_that_keeps_rising(h):
+    """Keys sorted by growing norm: the row maximum rises block after block, so the output accumulator is
+    rescaled repeatedly (the rare path of the lazy rescaling) -- and once by a large step."""
+    B, T, H, D = 1, 1024, 2, 64
+    q = rnd((B, T, H, D), 37)
+    ramp = torch.linspace(0.2, 6.0, T).view(1, T, 1, 1)
+    k = (q.float() * ramp).to(torch.bfloat16)  # key j is query j scaled up: scores grow with j
+    k[:, 900:] = (k[:, 900:].float() * 3).to(torch.bfloat16)
+    v = rnd((B, T, H, D), 38)
+    check(h, q, k, v, True)
+    check(h, q, k, v, False)
+
+
+def test_repeated_calls_are_bitwise_identical(h):
+    B, T, Hq, Hkv, D = 3, 700, 8, 4, 128
+    q, k, v = rnd((B, T, Hq, D), 39).to("cuda:0"), rnd((B, T, Hkv, D), 40).to("cuda:0"), rnd((B, T, Hkv, D), 41).to("cuda:0")
+    a = h.attention(q, k, v, causal=True).clone()
+    for _ in range(3):
+        assert torch.equal(a, h.attention(q, k, v, causal=True))
+    assert h.device_status() == 0
+
+
 def test_error_codes(h):
     from paper_2604_26666_b200.binding import FactError
     dev = "cuda:0"
