@@ -104,7 +104,18 @@ typedef enum { FACT_OP_GEMM = 0, FACT_OP_GEMM_BATCHED = 1, FACT_OP_GEMM_SPLITK =
  *   raster_group G > 0: the scheduler walks groups of G m-tiles (their slab of A/X stays in L2 while the
  *                n-tiles stream by); G < 0: groups of |G| n-tiles (a slab of B/W stays); 0: the library's
  *                traffic model chooses
- *   split_k      number of K slices, >= 1 (> 1 needs a workspace)
+ *   split_k      number of K slices, >= 1 (> 1 needs a workspace); or a stream-K schedule (Section 4.2, Action 2:
+ *                the third grid-level policy): -1 cuts the tiles of the last, partial wave along K and deals their
+ *                k-blocks out evenly over all CTAs, so that every SM ends at the same time; -2 does so with the
+ *                partial wave plus one full wave (fewer pieces per tile when the partial wave is small).  The
+ *                tiles of the full waves before stay data-parallel with the fused epilogue.  A tile cut this way
+ *                is finished by the CTA that holds its first k-block: the CTAs with the other pieces park their
+ *                FP32 accumulators in the workspace (one tile per CTA, fact_workspace_bytes), the finishing CTA
+ *                adds them to its own in CTA order and applies the epilogue -- a fixed order, so results are
+ *                reproducible bit for bit, and bounded waits like everywhere else.  Where there is nothing to cut
+ *                (whole waves, K == 0, an output the staged store cannot write) the call is data-parallel.
+ *                Stream-K calls through one handle must be stream-ordered with respect to each other (they share
+ *                the handle's flags) and must not share a workspace while they overlap.
  *   store_mode   0 = library default, 1 = direct register stores, 2 = shared-memory staged stores */
 typedef struct {
   int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode;
@@ -323,6 +334,16 @@ fact_status_t fact_device_status(fact_handle_t handle, void* cuda_stream, int* s
  * normally; the call synchronises the stream and returns FACT_OK if that is what happened.  A following
  * fact_device_status reports (and clears) the timeout; the context stays usable. */
 fact_status_t fact_selftest_wait_timeout(fact_handle_t handle, void* cuda_stream, double limit_ms);
+
+/* Diagnostic, host arithmetic only (no device is touched): the stream-K schedule of one CTA group.  With
+ * `sk_tiles` tiles of `k_blocks` k-blocks each shared out over `groups` CTA groups, writes the pieces group
+ * `group` processes, in its order, as rows of five ints -- tile (index among the stream-K tiles), first k-block,
+ * one past the last k-block, role (0 whole tile; 1 the piece with the tile's first k-block, which finishes the
+ * tile; 2 a later piece, parked in the workspace), and for role 1 the number of following groups that hold the
+ * tile's other pieces -- and their number in *n_pieces (at most max_pieces rows are written).  The kernels walk
+ * exactly this schedule. */
+fact_status_t fact_stream_k_pieces(int groups, int64_t sk_tiles, int64_t k_blocks, int group, int max_pieces,
+                                   int32_t* pieces, int* n_pieces);
 
 /* Number of kernels this handle has launched so far (for benchmark reports). */
 int64_t fact_launch_count(fact_handle_t handle);

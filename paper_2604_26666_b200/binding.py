@@ -37,6 +37,7 @@ EXPORTED = [
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
+    "fact_stream_k_pieces",
 ]
 
 
@@ -120,6 +121,7 @@ def lib() -> ctypes.CDLL:
     L.fact_block_workspace_bytes.restype = sz
     L.fact_block_workspace_offsets.argtypes = [POINTER(Block), POINTER(sz)]
     L.fact_block_forward.argtypes = [vp, POINTER(Block), vp, vp, vp, sz, vp]
+    L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     for name in EXPORTED:
         fn = getattr(L, name)
         if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
@@ -153,6 +155,20 @@ def _need(t: torch.Tensor, name: str, dtype, ndim):
 def _ld(t: torch.Tensor) -> int:
     """Leading dimension of the last two dims; a one-row matrix may carry any stride."""
     return int(t.stride(-2)) if t.shape[-2] > 1 else max(int(t.shape[-1]), int(t.stride(-2)))
+
+
+def stream_k_pieces(groups: int, sk_tiles: int, k_blocks: int, group: int):
+    """The stream-K pieces of one CTA group (fact_stream_k_pieces; host arithmetic, no device needed):
+    a list of (tile, k_begin, k_end, role, peers)."""
+    cap = 8
+    while True:
+        buf = (ctypes.c_int32 * (5 * cap))()
+        n = c_int(0)
+        _check(lib().fact_stream_k_pieces(groups, sk_tiles, k_blocks, group, cap, buf, byref(n)),
+               "fact_stream_k_pieces")
+        if n.value <= cap:
+            return [tuple(buf[5 * i: 5 * i + 5]) for i in range(n.value)]
+        cap = n.value
 
 
 def gemm_splitk_static(A, B, out, layout="KN", splits=0, device=None, stream=None):

@@ -39,6 +39,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the whole 227 KB opt-in limit (no static
                                          // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
+constexpr int kStatusInts = 64;  // status word, clock / profile counters, grid-barrier counters; stream-K flags follow
 
 // Key of the tuner's table: everything that changes which configuration is best.
 typedef std::tuple<int, int, int, int, long long, long long, long long, long long> TuneKey;
@@ -83,6 +84,8 @@ struct fact_handle_s {
   unsigned configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
+  int* sk_flags() const { return d_status + kStatusInts; }  // stream-K flags: [SM][epilogue warp], 0 between launches
+  size_t status_ints() const { return (size_t)kStatusInts + (size_t)sm_count * kEpiWarps; }
 };
 
 namespace {
@@ -228,8 +231,8 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
       c.split_k = (int)std::max<long long>(1, s);
     }
   }
-  if (c.split_k < 1) return FACT_ERR_INVALID_ARG;
-  c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
+  if (c.split_k < -2) return FACT_ERR_INVALID_ARG;
+  if (c.split_k > 0) c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
   if (c.store_mode < 0 || c.store_mode > 2) return FACT_ERR_INVALID_ARG;
   *out = c;
   return FACT_OK;
@@ -271,7 +274,32 @@ fact_status_t validate(const Problem& q) {
   return FACT_OK;
 }
 
-size_t workspace_for(const Problem& q, const fact_config_t& c) {
+// Stream-K (split_k < 0): how many tiles at the end of the tile list are cut along K and shared out evenly over all
+// CTA groups.  -1: the tiles of the last, partial wave; -2: those plus one full wave (shorter runs of partial
+// pieces per tile when the partial wave is small).  0 when there is nothing to share (the tiles fill whole waves,
+// K is empty, or the run of a group would be shorter than one k-block): the call is then data-parallel.
+int sk_tiles_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
+  if (c.split_k >= 0 || q.K <= 0) return 0;
+  const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
+  // the pieces are parked and finished by the staged epilogue, which stores whole 128-byte chunks per tile
+  const bool f32 = q.out == FACT_OUT_F32;
+  if (out_cols % (f32 ? 32 : 64) != 0 || (f32 && q.epi == FACT_EPI_BIAS_RESIDUAL) || c.store_mode == 1) return 0;
+  const long long tiles = q.batch * ((q.M + c.tile_m - 1) / c.tile_m) * ((q.N_out + out_cols - 1) / out_cols);
+  const long long groups = std::max(1, h->sm_count / c.cta_group);
+  const long long k_blocks = (q.K + kTileK - 1) / kTileK;
+  long long sk = tiles % groups;
+  if (sk == 0) return 0;
+  if (c.split_k == -2 && tiles >= sk + groups) sk += groups;
+  if (sk * k_blocks < groups || sk * k_blocks > 0x3fffffffLL) return 0;
+  return (int)sk;
+}
+
+size_t workspace_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
+  if (c.split_k < 0) {  // stream-K: one FP32 accumulator tile per CTA
+    if (sk_tiles_for(h, q, c) == 0) return 0;
+    const size_t ctas = (size_t)std::max(1, h->sm_count / c.cta_group) * (size_t)c.cta_group;
+    return ctas * (size_t)kTileM * (size_t)c.tile_n * sizeof(float);
+  }
   if (c.split_k <= 1) return 0;
   return (size_t)c.split_k * (size_t)q.batch * (size_t)ws_planes_for(q) * (size_t)q.M * (size_t)ws_ld_for(q) *
          sizeof(float);
@@ -304,10 +332,11 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.tiles_m = (int)((q.M + c.tile_m - 1) / c.tile_m);
   p.tiles_n = (int)((q.N_out + p.out_cols - 1) / p.out_cols);
   p.k_blocks = (int)((q.K + kTileK - 1) / kTileK);
-  p.split_k = c.split_k;
+  const int slices = std::max(1, c.split_k);  // (stream-K, split_k < 0, cuts no tile into equal slices)
+  p.split_k = slices;
   p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
-  p.k_base = p.k_blocks / std::max(1, c.split_k);
-  p.k_rem = p.k_blocks % std::max(1, c.split_k);
+  p.k_base = p.k_blocks / slices;
+  p.k_rem = p.k_blocks % slices;
   p.raster_along_n = c.raster_group < 0;
   p.raster_group = p.raster_along_n ? std::min(-c.raster_group, std::max(1, p.tiles_n))
                                     : std::min(c.raster_group, std::max(1, p.tiles_m));
@@ -373,12 +402,28 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   plan->cfg.store_mode = p.store_tma ? 2 : 1;
   p.status = h->d_status;
   p.debug = h->debug_flags;
-  plan->ws_bytes = workspace_for(q, c);
+  plan->ws_bytes = workspace_for(h, q, c);
   p.epi_bufs = epi_bufs_for(q);
   plan->smem_bytes = std::max(smem_bytes_for(q, c.tile_n, cg, c.stages), kMinSmemRequest);
   if (plan->smem_bytes > kSmemBudget || kSmemBudget > h->max_smem) return FACT_ERR_UNSUPPORTED;
   const int slots = std::max(1, h->sm_count / cg);
   plan->grid = (int)std::min<long long>(slots, units) * cg;
+  if (c.split_k < 0) {
+    // Stream-K: the staged epilogue parks and finishes the pieces, so an output it cannot store is data-parallel.
+    const int sk = p.store_tma ? sk_tiles_for(h, q, c) : 0;
+    if (sk == 0) {
+      plan->cfg.split_k = 1;
+      plan->ws_bytes = 0;
+    } else {
+      const long long iters = (long long)sk * p.k_blocks;
+      p.sk_tiles = sk;
+      p.sk_first = p.total_units - sk;
+      p.total_units = p.sk_first;  // what is left for the data-parallel walk
+      p.sk_len = (int)(iters / slots);
+      p.sk_rem = (int)(iters % slots);
+      plan->grid = slots * cg;     // every group takes a run, whatever the number of tiles
+    }
+  }
   return FACT_OK;
 }
 
@@ -402,10 +447,10 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
   return FACT_OK;
 }
 
-template <int CG, int EPI>
+template <int CG, int EPI, bool SK = false>
 fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                               cudaStream_t stream) {
-  auto kern = fact_gemm_kernel<CG, EPI>;
+  auto kern = fact_gemm_kernel<CG, EPI, SK>;
   if (!(h->configured_mask & (1u << slot))) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
@@ -443,6 +488,21 @@ fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUten
     case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate>(h, base + 4, plan, tm, stream);
     case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual>(h, base + 5, plan, tm, stream);
     case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tm, stream);
+    default: return FACT_ERR_INVALID_ARG;
+  }
+}
+
+// The stream-K instantiations (every epilogue but the split-K partial store).
+template <int CG>
+fact_status_t launch_epi_sk(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  const int base = 16 + (CG - 1) * 8;
+  switch (epi) {
+    case kEpiNone: return launch_instance<CG, kEpiNone, true>(h, base + 0, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias, true>(h, base + 1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, true>(h, base + 2, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, true>(h, base + 3, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, true>(h, base + 4, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, true>(h, base + 5, plan, tm, stream);
     default: return FACT_ERR_INVALID_ARG;
   }
 }
@@ -490,10 +550,24 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
   if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
   if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
 
+  if (plan.cfg.split_k < 0 && (!ws || ws_bytes < plan.ws_bytes) && !user) {
+    // a tuned stream-K entry, but this caller brought no scratch: run the tiles data-parallel
+    fact_config_t dp = plan.cfg;
+    dp.split_k = 1;
+    st = make_plan(h, q, &dp, 0, &plan);
+    if (st != FACT_OK) return st;
+  }
   if (q.K == 0) {  // empty sum: the epilogue of a zero accumulator
     st = launch_reduce(h, q, plan, 0, reinterpret_cast<const float*>(q.C), stream);
   } else {
     const bool split = plan.cfg.split_k > 1;
+    const bool stream_k = plan.cfg.split_k < 0;
+    if (stream_k) {
+      if (!ws || ws_bytes < plan.ws_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
+      if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
+      plan.p.sk_ws = reinterpret_cast<float*>(ws);
+      plan.p.sk_flags = h->sk_flags();
+    }
     if (split) {
       if (!ws || ws_bytes < plan.ws_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
       if (!aligned16(ws)) return FACT_ERR_BAD_ALIGNMENT;
@@ -542,7 +616,9 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       }
     }
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
-    if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
+    if (stream_k) st = plan.cfg.cta_group == 2 ? launch_epi_sk<2>(h, epi, plan, tm, stream)
+                                               : launch_epi_sk<1>(h, epi, plan, tm, stream);
+    else if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
     else st = launch_epi<1>(h, epi, plan, tm, stream);
     if (st == FACT_OK && split && !plan.p.fused_reduce)
       st = launch_reduce(h, q, plan, plan.cfg.split_k, reinterpret_cast<const float*>(ws), stream);
@@ -625,8 +701,8 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
     return FACT_ERR_CUDA;
   }
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&h->d_status, 32 * sizeof(int)) != cudaSuccess ||
-      cudaMemset(h->d_status, 0, 32 * sizeof(int)) != cudaSuccess) {
+  if (cudaMalloc(&h->d_status, h->status_ints() * sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->d_status, 0, h->status_ints() * sizeof(int)) != cudaSuccess) {
     delete h;
     return FACT_ERR_CUDA;
   }
@@ -647,6 +723,32 @@ fact_status_t fact_device_info(fact_handle_t h, int* sm_count, int* max_smem, in
   if (max_smem) *max_smem = h->max_smem;
   if (cc_major) *cc_major = h->cc_major;
   if (cc_minor) *cc_minor = h->cc_minor;
+  return FACT_OK;
+}
+
+fact_status_t fact_stream_k_pieces(int groups, int64_t sk_tiles, int64_t k_blocks, int group, int max_pieces,
+                                   int32_t* pieces, int* n_pieces) {
+  if (groups < 1 || sk_tiles < 0 || k_blocks < 1 || group < 0 || group >= groups || max_pieces < 0 || !n_pieces ||
+      (max_pieces > 0 && !pieces) || sk_tiles * k_blocks > 0x3fffffffLL)
+    return FACT_ERR_INVALID_ARG;
+  const long long iters = sk_tiles * k_blocks;
+  const int len = (int)(iters / groups), rem = (int)(iters % groups);
+  int pos = sk_group_begin(len, rem, group);
+  const int end = sk_group_begin(len, rem, group + 1);
+  int n = 0;
+  while (pos < end) {
+    const SkPiece pc = sk_next_piece((int)k_blocks, len, rem, groups, group, pos, end);
+    if (n < max_pieces) {
+      int32_t* row = pieces + 5 * n;
+      row[0] = pc.tile;
+      row[1] = pc.k0;
+      row[2] = pc.k1;
+      row[3] = pc.role;
+      row[4] = pc.peers;
+    }
+    ++n;
+  }
+  *n_pieces = n;
   return FACT_OK;
 }
 
@@ -693,7 +795,11 @@ fact_status_t fact_device_status(fact_handle_t h, void* stream, int* status) {
   if (cudaStreamSynchronize(s) != cudaSuccess) return FACT_ERR_CUDA;
   int v = 0;
   if (cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FACT_ERR_CUDA;
-  if (v != 0 && cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) return FACT_ERR_CUDA;
+  // (a launch that gave up may have left stream-K flags and grid-barrier counters set: clear them with the word)
+  if (v != 0 && (cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess ||
+                 cudaMemset(h->d_status + 24, 0, 2 * sizeof(int)) != cudaSuccess ||
+                 cudaMemset(h->sk_flags(), 0, (size_t)h->sm_count * kEpiWarps * sizeof(int)) != cudaSuccess))
+    return FACT_ERR_CUDA;
   *status = v;
   return FACT_OK;
 }
@@ -719,7 +825,7 @@ fact_status_t fact_workspace_bytes(fact_handle_t h, fact_op_t op, int64_t batch,
   fact_config_t c;
   fact_status_t st = resolve_config(h, q, cfg, 0, &c);
   if (st != FACT_OK) return st;
-  *bytes = workspace_for(q, c);
+  *bytes = workspace_for(h, q, c);
   return FACT_OK;
 }
 
@@ -799,6 +905,11 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
           if (sp > 1 && std::find(splits.begin(), splits.end(), (int)sp) == splits.end()) splits.push_back((int)sp);
         }
       }
+      // stream-K, when the last wave is partial and short enough in waves for that to matter
+      if (tiles % slots != 0 && tiles <= 12 * slots) {
+        splits.push_back(-1);
+        if (tiles > slots) splits.push_back(-2);
+      }
       std::vector<int> stage_opts = {smax};
       if (smax > 3) stage_opts.push_back(smax - 1);
       // (the raster group is not swept: its effect is on DRAM traffic and, through power, on the clock, which a
@@ -832,7 +943,7 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
     h->table.erase(make_key(q));
     const fact_status_t rs = resolve_config(h, q, nullptr, 0, &ref_c);
     h->table = saved;
-    if (rs != FACT_OK || workspace_for(q, ref_c) > ws_bytes) {
+    if (rs != FACT_OK || workspace_for(h, q, ref_c) > ws_bytes) {
       cudaEventDestroy(e0);
       cudaEventDestroy(e1);
       return rs != FACT_OK ? rs : FACT_ERR_WORKSPACE_TOO_SMALL;

@@ -105,6 +105,13 @@ struct GemmParams {
   int fused_reduce;   // 1: after a grid-wide barrier every CTA reduces its share of the output (split-K only)
   int reduce_epi;     // the epilogue the reduction applies
   int* status;        // [0] error word, [2..17] clock / profile counters, [24], [25] grid-barrier counters
+  // stream-K (the SK instantiations only): the last `sk_tiles` tiles of the tile list are cut along K into one
+  // contiguous run of k-blocks per CTA group; see UnitWalk
+  int sk_tiles;       // 0: every tile is data-parallel
+  int sk_first;       // index of the first stream-K tile (= number of data-parallel tiles = total_units)
+  int sk_len, sk_rem; // group c owns k-block iterations [c * sk_len + min(c, sk_rem), + sk_len + (c < sk_rem))
+  float* sk_ws;       // one FP32 accumulator tile per CTA: [gridDim.x][tile_n / 32][8][128] float4
+  int* sk_flags;      // [gridDim.x][kEpiWarps]: 1 while that warp's share of the CTA's partial tile is ready
   // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
   // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
   int debug;
@@ -112,6 +119,9 @@ struct GemmParams {
 
 struct WorkUnit {
   int b, tm, tn, kb_begin, kb_end, split;
+  int wave;      // ordinal of this data-parallel unit within its CTA (0 for stream-K pieces)
+  int sk_role;   // 0: a whole tile; 1: the piece with the tile's first k-block (it finishes the tile); 2: a later piece
+  int sk_peers;  // role 1: how many following CTA groups hold the tile's other pieces
 };
 
 __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
@@ -152,6 +162,98 @@ __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
   w.tm = p.raster_along_n ? o : gi;
   w.tn = p.raster_along_n ? gi : o;
   return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stream-K partition (host and device share this arithmetic).  The k-block iterations of the stream-K tiles are
+// numbered tile by tile, `k_blocks` per tile, and dealt out in contiguous runs: group c owns
+// [sk_group_begin(c), sk_group_begin(c + 1)), runs differing by at most one iteration.
+__host__ __device__ inline int sk_group_begin(int len, int rem, int c) { return c * len + (c < rem ? c : rem); }
+
+struct SkPiece {
+  int tile;        // index among the stream-K tiles
+  int k0, k1;      // k-blocks [k0, k1) of that tile
+  int role;        // 0: the whole tile; 1: the piece with the tile's first k-block (it finishes the tile); 2: a later piece
+  int peers;       // role 1: how many following groups hold the tile's other pieces
+};
+
+// The next piece of `group`'s run, which currently stands at iteration `pos` and ends at `end`.
+__host__ __device__ inline SkPiece sk_next_piece(int k_blocks, int len, int rem, int groups, int group, int& pos,
+                                                 int end) {
+  SkPiece pc;
+  pc.tile = pos / k_blocks;
+  pc.k0 = pos - pc.tile * k_blocks;
+  const int left = end - pos;
+  pc.k1 = (k_blocks - pc.k0 < left) ? k_blocks : pc.k0 + left;
+  pc.role = pc.k0 > 0 ? 2 : (pc.k1 < k_blocks ? 1 : 0);
+  pc.peers = 0;
+  if (pc.role == 1) {
+    const int tile_end = (pc.tile + 1) * k_blocks;
+    int c2 = group + 1;
+    while (c2 < groups && sk_group_begin(len, rem, c2) < tile_end) ++c2;
+    pc.peers = c2 - group - 1;
+  }
+  pos += pc.k1 - pc.k0;
+  return pc;
+}
+
+// The sequence of work units of one CTA group.  Data-parallel kernels: units unit0, unit0 + stride, ...
+// Stream-K kernels: first the group's run of k-block iterations in the stream-K region -- a run covers the tail
+// of one tile, whole tiles, and the head of another, each a unit of its own -- then its data-parallel tiles.
+// A tile's pieces belong to consecutive groups; the group with the first k-block adds the others' FP32
+// partials (in group order) to its own accumulator and applies the epilogue.  Those others meet that piece first
+// of all their work and depend on nobody, so the wait for them cannot be circular.
+template <bool SK>
+struct UnitWalk {
+  int u, stride, wave;
+  int sk_pos, sk_end, group;
+  __device__ __forceinline__ UnitWalk(const GemmParams& p, int unit0, int unit_stride)
+      : u(unit0), stride(unit_stride), wave(0), sk_pos(0), sk_end(0), group(unit0) {
+    if constexpr (SK) {
+      sk_pos = sk_group_begin(p.sk_len, p.sk_rem, unit0);
+      sk_end = sk_group_begin(p.sk_len, p.sk_rem, unit0 + 1);
+    }
+  }
+  __device__ __forceinline__ bool next(const GemmParams& p, WorkUnit& w) {
+    if constexpr (SK) {
+      if (sk_pos < sk_end) {
+        const SkPiece pc = sk_next_piece(p.k_blocks, p.sk_len, p.sk_rem, stride, group, sk_pos, sk_end);
+        w = decode_unit(p, p.sk_first + pc.tile);
+        w.kb_begin = pc.k0;
+        w.kb_end = pc.k1;
+        w.wave = 0;
+        w.sk_role = pc.role;
+        w.sk_peers = pc.peers;
+        return true;
+      }
+    }
+    if (u >= p.total_units) return false;
+    w = decode_unit(p, u);
+    w.wave = wave++;
+    w.sk_role = 0;
+    w.sk_peers = 0;
+    u += stride;
+    return true;
+  }
+};
+
+// Bounded wait for a flag in global memory to become `want`.  Returns false if the wait was abandoned.
+__device__ __forceinline__ bool wait_flag(const int* flag, int want, volatile int* abort_flag, int* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (ptx::ld_acquire_gpu(flag) == want) return true;
+    if ((it & 255u) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = ptx::globaltimer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, kDeviceTimeoutCode);
+        return false;
+      }
+    }
+  }
 }
 
 // Bounded mbarrier wait.  Returns false if the wait was abandoned.
@@ -420,7 +522,7 @@ __device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uin
   }
 }
 
-template <int CG, int EPI>
+template <int CG, int EPI, bool SK = false>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
@@ -440,6 +542,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (smem_base & 1023u) {  // the swizzled tiles need a 1024-byte aligned ring: refuse to run otherwise
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
+  }
+  if constexpr (SK) {  // stream-K pieces are parked and finished by the staged epilogue only: refuse anything else
+    if (!p.store_tma || p.sk_ws == nullptr || p.sk_flags == nullptr) {
+      if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+      return;
+    }
   }
   const uint32_t epi_base = smem_base + (uint32_t)p.stages * p.stage_bytes;
   const uint32_t bias_base = epi_base + (uint32_t)(kEpiWarps * p.epi_bufs) * kEpiBufBytes;
@@ -507,13 +615,13 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      int wave = 0;
-      for (int u = unit0; ok && u < p.total_units; u += unit_stride, ++wave) {
-        const WorkUnit w = decode_unit(p, u);
+      UnitWalk<SK> walk(p, unit0, unit_stride);
+      WorkUnit w;
+      while (ok && walk.next(p, w)) {
         // Odd waves walk K downwards: the wave before ended at the top of K, so the operand slabs both waves
         // share (same m-tiles of A, or same n-tiles of B) are met while they are still in L2.  The sum of an
         // output element is then taken in descending k in those tiles, still fixed by (shape, config).
-        const bool k_down = (wave & 1) && p.k_serpentine;
+        const bool k_down = (w.wave & 1) && p.k_serpentine;
         const int m0 = (w.tm * CG + (int)cta_rank) * kTileM;
         // first accumulator column this CTA's B boxes feed, and the W column of every box
         const int col0 = (CG == 2) ? (int)cta_rank * (p.tile_n / 2) : 0;
@@ -590,8 +698,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t acc_phase = 0;
       bool ok = true;
       long long prof_acc_wait = 0, prof_full_wait = 0, prof_first_full = 0;
-      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
-        const WorkUnit w = decode_unit(p, u);
+      UnitWalk<SK> walk(p, unit0, unit_stride);
+      WorkUnit w;
+      while (ok && walk.next(p, w)) {
         long long t0 = prof ? clock64() : 0;
         if (!wait_all(acce_bar(acc), acc_phase ^ 1u)) {
           ok = false;
@@ -671,8 +780,56 @@ __global__ void __launch_bounds__(kThreads, 1)
       long long prof_epi_busy = 0, prof_epi_wait = 0, prof_tiles = 0;
       uint32_t gc = 0;      // chunks this warp has stored so far: buffer = gc % bufs
       uint32_t r_next = 0;  // residual loads have been issued for every chunk counter below this
-      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
-        const WorkUnit w = decode_unit(p, u);
+      UnitWalk<SK> walk(p, unit0, unit_stride);
+      WorkUnit w;
+      // hand the accumulator back to the MMA issuer (of the leader CTA) and move on to the other one
+      // (a relaxed arrival: the barrier orders tensor-memory reads only, which the tcgen05 fences take care of; a
+      // cluster-scope release here waited for the TMA stores in flight, 2500-3600 cycles per tile)
+      auto release_acc = [&]() {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(acce_bar(acc), 0));
+          else ptx::mbar_arrive(acce_bar(acc));
+        }
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      };
+      // stream-K scratch: this CTA's partial tile and the flags of its epilogue warps
+      constexpr int kSkPieceF4 = 8 * kTileM;  // float4 words of one 32-column piece of a CTA's 128 accumulator rows
+      const int sk_pieces = p.tile_n >> 5;
+      float4* const sk_ws4 = reinterpret_cast<float4*>(p.sk_ws);
+      while (ok && walk.next(p, w)) {
+        if constexpr (SK) {
+          if (w.sk_role == 2) {
+            // ---- a later piece of a tile another group finishes: park the raw FP32 accumulator in this CTA's
+            // scratch tile.  Layout [piece][16-byte word j of the thread's 32 columns][row]: consecutive lanes
+            // write consecutive 16-byte words, and the finishing warp reads them back the same way.
+            if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+              ok = false;
+              break;
+            }
+            ptx::tc_fence_after();
+            const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+            float4* const mine = sk_ws4 + (size_t)blockIdx.x * (size_t)(sk_pieces * kSkPieceF4) + (q * 32 + lane);
+            for (int pc = half; pc < sk_pieces; pc += 2) {
+              uint32_t v[32];
+              ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(pc * 32), v);
+              ptx::tmem_wait_ld();
+              float4* dst = mine + (size_t)pc * kSkPieceF4;
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                __stcg(dst + j * kTileM, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+            }
+            release_acc();  // (contains the __syncwarp that orders every lane's stores before lane 0's fence)
+            if (lane == 0) {
+              __threadfence();
+              ptx::st_release_gpu(p.sk_flags + (size_t)blockIdx.x * kEpiWarps + e, 1);
+            }
+            continue;
+          }
+        }
         const int row0 = (w.tm * CG + (int)cta_rank) * kTileM + q * 32;
         const int n_tile0 = w.tn * p.out_cols;
         const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
@@ -735,6 +892,45 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (prof) prof_epi_wait += tb - tw;
         ptx::tc_fence_after();
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+        if constexpr (SK) {
+          // the first piece of a tile: the same warp of the same CTA rank in each of the following groups parks
+          // the rest of the sum; wait until those are complete (they precede everything else those groups do)
+          if (w.sk_role == 1) {
+            int good = 1;
+            if (lane == 0) {
+              for (int pe = 1; pe <= w.sk_peers && good; ++pe)
+                good = wait_flag(p.sk_flags + (size_t)(blockIdx.x + CG * pe) * kEpiWarps + e, 1, abort_p, p.status);
+            }
+            if (!__shfl_sync(0xffffffffu, good, 0)) {
+              ok = false;
+              break;
+            }
+          }
+        }
+        // add the parked partials of accumulator columns [col, col + 32) to v, in group order
+        auto add_peers = [&](uint32_t (&v)[32], int col) {
+          if constexpr (SK) {
+            if (w.sk_role != 1) return;
+            for (int pe = 1; pe <= w.sk_peers; ++pe) {
+              const float4* src = sk_ws4 + (size_t)(blockIdx.x + CG * pe) * (size_t)(sk_pieces * kSkPieceF4) +
+                                  (size_t)(col >> 5) * kSkPieceF4 + (q * 32 + lane);
+#pragma unroll
+              for (int j0 = 0; j0 < 8; j0 += 4) {  // four 16-byte loads in flight per thread
+                float4 t[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) t[j] = __ldcg(src + (j0 + j) * kTileM);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int o = 4 * (j0 + j);
+                  v[o] = __float_as_uint(__uint_as_float(v[o]) + t[j].x);
+                  v[o + 1] = __float_as_uint(__uint_as_float(v[o + 1]) + t[j].y);
+                  v[o + 2] = __float_as_uint(__uint_as_float(v[o + 2]) + t[j].z);
+                  v[o + 3] = __float_as_uint(__uint_as_float(v[o + 3]) + t[j].w);
+                }
+              }
+            }
+          }
+        };
         for (int ci = half; ci < n_chunks; ci += 2) {
           int n_chunk, z;
           if (!chunk_coord(ci, n_chunk, z)) continue;  // uniform across the warp
@@ -760,6 +956,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           }
           ptx::tmem_wait_ld();
+          add_peers(v0, c0);
+          if constexpr (EPI == kEpiSiluGate) add_peers(v1, p.out_cols + c0);
+          else if (pieces == 2) add_peers(v1, c0 + 32);
           // one 32-column piece: fused operation on packed FP32 pairs, rounding, into outw
           auto do_piece = [&](int piece, const uint32_t (&a)[32], const uint32_t (&up)[32]) {
             const int local0 = (ci >> 1) * chunk_cols + piece * 32;  // index among the warp's 128 columns
@@ -810,6 +1009,8 @@ __global__ void __launch_bounds__(kThreads, 1)
               ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(c0 + 32), v0);
               ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c0 + 32), v1);
               ptx::tmem_wait_ld();
+              add_peers(v0, c0 + 32);
+              add_peers(v1, p.out_cols + c0 + 32);
               do_piece(1, v0, v1);
             }
           } else {
@@ -838,21 +1039,17 @@ __global__ void __launch_bounds__(kThreads, 1)
           ++gc;
         }
         if (!ok) break;
-        // hand the accumulator back to the MMA issuer (of the leader CTA)
-        ptx::tc_fence_before();
-        __syncwarp();
-        // (a relaxed arrival: the barrier orders tensor-memory reads only, which the tcgen05 fences take care of; a
-        // cluster-scope release here waited for the TMA stores in flight, 2500-3600 cycles per tile)
-        if (lane == 0) {
-          if constexpr (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(acce_bar(acc), 0));
-          else ptx::mbar_arrive(acce_bar(acc));
+        release_acc();
+        if constexpr (SK) {
+          // the parked partials have been consumed: clear their flags for the next launch (this warp is their
+          // only reader; release_acc's __syncwarp put every lane's reads before this)
+          if (w.sk_role == 1 && lane == 0)
+            for (int pe = 1; pe <= w.sk_peers; ++pe) p.sk_flags[(size_t)(blockIdx.x + CG * pe) * kEpiWarps + e] = 0;
         }
         if (prof) {
           prof_epi_busy += clock64() - tb;
           ++prof_tiles;
         }
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
       }
       if (prof && e == 0 && lane == 0) {
         long long* c = reinterpret_cast<long long*>(p.status + 2);
@@ -872,8 +1069,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else {
       // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
       const bool c_vec = p.c_vec != 0;
-      for (int u = unit0; ok && u < p.total_units; u += unit_stride) {
-        const WorkUnit w = decode_unit(p, u);
+      UnitWalk<false> walk(p, unit0, unit_stride);  // (stream-K always stores through the staged path)
+      WorkUnit w;
+      while (ok && walk.next(p, w)) {
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
           ok = false;
           break;

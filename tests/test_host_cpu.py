@@ -135,3 +135,57 @@ def test_attention_and_block_workloads():
     x, w = wl.make_block_inputs(wl.BlockCase("t", "gpt", 1, 4, 2, 2, 8, 16, 5))
     assert len(w) == 12 and w["w1"].shape == (16, 16) and w["bqkv"].shape == (48,)
     assert [c.name for c in wl.paper_cases()] == ["p3_batched_128x512x2048x1024", "p6_splitk_256x256x524288"]
+
+
+@pytest.mark.parametrize("groups,sk_tiles,k_blocks", [
+    (74, 44, 48), (74, 44 + 74, 12), (148, 1, 2048), (148, 147, 3), (74, 73, 1), (7, 3, 5), (5, 12, 4), (3, 2, 1),
+    (148, 20, 11), (2, 1, 1),
+])
+def test_stream_k_partition_covers_every_k_block_once(libfact, groups, sk_tiles, k_blocks):
+    """The stream-K schedule the kernels walk (fact_stream_k_pieces): runs are contiguous and balanced, every
+    k-block of every tile is in exactly one piece, every tile has exactly one finishing piece, and the pieces it
+    waits for are the first work of the groups right after it."""
+    from paper_2604_26666_b200.binding import stream_k_pieces
+
+    per_group = [stream_k_pieces(groups, sk_tiles, k_blocks, g) for g in range(groups)]
+    lengths = [sum(k1 - k0 for (_, k0, k1, _, _) in ps) for ps in per_group]
+    assert sum(lengths) == sk_tiles * k_blocks
+    assert max(lengths) - min(lengths) <= 1
+    assert lengths == sorted(lengths, reverse=True)  # the longer runs come first
+    covered = {}
+    pos = 0
+    for g, ps in enumerate(per_group):
+        for i, (tile, k0, k1, role, peers) in enumerate(ps):
+            assert 0 <= tile < sk_tiles and 0 <= k0 < k1 <= k_blocks
+            assert tile * k_blocks + k0 == pos, "runs are contiguous in (tile, k) order"
+            pos += k1 - k0
+            for k in range(k0, k1):
+                assert (tile, k) not in covered
+                covered[(tile, k)] = g
+            if role == 0:
+                assert (k0, k1) == (0, k_blocks) and peers == 0
+            elif role == 1:
+                assert k0 == 0 and k1 < k_blocks and peers >= 1
+                assert i == len(ps) - 1, "a run can only end inside a tile with its last piece"
+            else:
+                assert role == 2 and k0 > 0 and peers == 0
+                assert i == 0, "a parked piece is the first thing its group does"
+    assert len(covered) == sk_tiles * k_blocks
+    for tile in range(sk_tiles):
+        owners = sorted({covered[(tile, k)] for k in range(k_blocks)})
+        assert owners == list(range(owners[0], owners[-1] + 1)), "a tile's pieces belong to consecutive groups"
+        first = per_group[owners[0]][-1] if len(owners) > 1 else None
+        if first is not None:
+            assert first[0] == tile and first[3] == 1 and first[4] == len(owners) - 1
+
+
+def test_stream_k_pieces_rejects_bad_arguments(libfact):
+    import ctypes
+
+    n = ctypes.c_int(0)
+    buf = (ctypes.c_int32 * 5)()
+    assert libfact.fact_stream_k_pieces(0, 1, 1, 0, 1, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_stream_k_pieces(4, 1, 0, 0, 1, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_stream_k_pieces(4, 1, 1, 4, 1, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_stream_k_pieces(4, 1, 1, 0, 1, buf, None) == 1
+    assert libfact.fact_stream_k_pieces(4, 1, 8, 3, 0, None, ctypes.byref(n)) == 0 and n.value == 1
