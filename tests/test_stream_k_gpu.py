@@ -192,3 +192,35 @@ def test_stream_k_replays_in_a_cuda_graph(h):
         torch.cuda.synchronize()
         assert h.device_status() == 0
         assert np.array_equal(out.double().cpu().numpy(), oracle_for(ins, case))
+
+
+def test_tuned_stream_k_entry_without_scratch_runs_data_parallel(tmp_path):
+    """A table entry may say stream-K while a caller (a block chain, say) brings no workspace: the library then
+    runs the same tiles data-parallel instead of failing; with an explicit config the missing scratch is an error
+    (test_stream_k_workspace_errors)."""
+    from paper_2604_26666_b200.binding import Handle, lib, _ptr, _ld
+
+    M, N, K = 1280, 1280, 512
+    table = tmp_path / "table.txt"
+    table.write_text(f"0 0 1 0 1 {M} {N} {K} | 128 64 64 0 1 0 -1 0\n")
+    hd = Handle(0, load_table=False)
+    try:
+        hd.tune_cache_load(str(table))
+        assert hd.get_config("gemm", 1, M, N, K, "NONE", "NK", torch.bfloat16).as_dict()["split_k"] == -1
+        assert hd.workspace_bytes("gemm", 1, M, N, K, "NONE", "NK", torch.bfloat16) > 0
+        case = wl.Case("sk_table", "gemm", M, N, K, layout="NK", out="f32", seed=19)
+        ins = small_int_inputs(case, seed=19)
+        A, B = ins.X.cuda(), ins.W.cuda()
+        C = torch.empty(M, N, device="cuda", dtype=torch.bfloat16)
+        s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        rc = lib().fact_gemm(hd._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), 1, _ptr(C), _ld(C), 0, None, None, 0, s)
+        assert rc == 0
+        torch.cuda.synchronize()
+        assert hd.device_status() == 0
+        with_ws = hd.gemm(A, B, layout="NK", out_dtype=torch.bfloat16)  # the binding brings the scratch: stream-K
+        torch.cuda.synchronize()
+        assert hd.device_status() == 0
+        ref = torch.from_numpy(oracle_for(ins, case)).to(torch.bfloat16)  # integers: exact before the BF16 rounding
+        assert torch.equal(C.cpu(), ref) and torch.equal(with_ws.cpu(), ref)
+    finally:
+        hd.close()
