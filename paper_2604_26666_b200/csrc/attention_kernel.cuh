@@ -62,7 +62,8 @@ struct AttnParams {
   int causal;
   float scale_log2;           // softmax scale * log2(e)
   int q_tiles;                // ceil(Tq / 128)
-  int items;                  // B * Hq * q_tiles work items, ordered heaviest query tile first
+  int q_pairs;                // ceil(Tq / 256): the two-tile kernel's unit
+  int items;                  // B * Hq * q_tiles (q_pairs) work items, ordered heaviest query tile first
   uint64_t kmajor_desc;       // UMMA descriptor template, K-major 128B-swizzled tiles (K)
   uint64_t v_desc;            // UMMA descriptor template, V as an N-major operand
   uint32_t idesc_s, idesc_pv;

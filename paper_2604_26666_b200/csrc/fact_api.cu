@@ -18,6 +18,7 @@
 #include "fact.h"
 #include "gemm_kernel.cuh"
 #include "attention_kernel.cuh"
+#include "attention_pair_kernel.cuh"
 #include "norm_kernel.cuh"
 
 // Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
@@ -1031,12 +1032,13 @@ fact_status_t fact_tune_cache_load(fact_handle_t h, const char* path) {
 // ---------------------------------------------------------------------------------------------
 // Fused multi-head attention
 namespace {
-// Rank-4 BF16 tensor map over [B][T][H][D]-like storage, dims ordered (D, H, T, B), box 64 x 1 x 128 x 1.
+// Rank-4 BF16 tensor map over [B][T][H][D]-like storage, dims ordered (D, H, T, B), box 64 x 1 x box_rows x 1.
 fact_status_t encode_map_bthd(fact_handle_t h, CUtensorMap* map, const void* base, long long D, long long H, long long T,
-                              long long B, long long stride_h, long long stride_t, long long stride_b) {
+                              long long B, long long stride_h, long long stride_t, long long stride_b,
+                              int box_rows = kAttnBlockQ) {
   cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
   cuuint64_t strides[3] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2, (cuuint64_t)stride_b * 2};
-  cuuint32_t box[4] = {64, 1, (cuuint32_t)kAttnBlockQ, 1};
+  cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1077,9 +1079,15 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
   if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
   CUtensorMap tq, tk, tv, to;
   auto bs = [&](int64_t s, int64_t fallback) { return (batch > 1 && s > 0) ? s : std::max<int64_t>(fallback, 8); };
+  // Two query tiles per CTA, each a pipeline of its own (keys in blocks of 128 at head_dim 64, of 64 at head_dim
+  // 128), unless the experiment switch (bit 512) asks for the single-tile kernel.
+  const bool pair = !(h->debug_flags & 512);
+  const int block_k = pair ? attn_pair_block_k((int)head_dim) : kAttnBlockK;
   fact_status_t st = encode_map_bthd(h, &tq, Q, head_dim, heads_q, seq_q, batch, q_sh, q_st, bs(q_sb, q_st * seq_q));
-  if (st == FACT_OK) st = encode_map_bthd(h, &tk, K, head_dim, heads_kv, seq_kv, batch, k_sh, k_st, bs(k_sb, k_st * seq_kv));
-  if (st == FACT_OK) st = encode_map_bthd(h, &tv, V, head_dim, heads_kv, seq_kv, batch, v_sh, v_st, bs(v_sb, v_st * seq_kv));
+  if (st == FACT_OK)
+    st = encode_map_bthd(h, &tk, K, head_dim, heads_kv, seq_kv, batch, k_sh, k_st, bs(k_sb, k_st * seq_kv), block_k);
+  if (st == FACT_OK)
+    st = encode_map_bthd(h, &tv, V, head_dim, heads_kv, seq_kv, batch, v_sh, v_st, bs(v_sb, v_st * seq_kv), block_k);
   if (st == FACT_OK) st = encode_map_bthd(h, &to, O, head_dim, heads_q, seq_q, batch, o_sh, o_st, bs(o_sb, o_st * seq_q));
   if (st == FACT_OK) {
     AttnParams p;
@@ -1095,27 +1103,36 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.scale_log2 = (float)(sc * 1.4426950408889634);
     p.q_tiles = (int)((seq_q + kAttnBlockQ - 1) / kAttnBlockQ);
     p.kmajor_desc = smem_desc_template(16, 1024);
-    p.v_desc = smem_desc_template(kAttnBlockK * 128, 1024);  // 64-column chunks of V are one 128-key tile apart
-    p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttnBlockK >> 3) << 17) | ((uint32_t)(kAttnBlockQ >> 4) << 24);
+    p.v_desc = smem_desc_template(block_k * 128, 1024);  // 64-column chunks of V are one block of keys apart
+    p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_k >> 3) << 17) | ((uint32_t)(kAttnBlockQ >> 4) << 24);
     p.idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(head_dim >> 3) << 17) |
                  ((uint32_t)(kAttnBlockQ >> 4) << 24);
     p.status = h->d_status;
     p.debug = h->debug_flags;
-    const long long items = (long long)p.q_tiles * heads_q * batch;
+    p.q_pairs = (p.q_tiles + 1) / 2;
+    const long long items = (long long)(pair ? p.q_pairs : p.q_tiles) * heads_q * batch;
     if (items > 0x7fffffffLL) {
       if (dev != h->device) cudaSetDevice(dev);
       return FACT_ERR_UNSUPPORTED;
     }
     p.items = (int)items;
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
-    const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
+    const int smem = std::max((int)(pair ? attn_pair_smem_bytes(p.D) : attn_smem_bytes(p.D)), kMinSmemRequest);
     if (!(h->configured_mask & (1u << 30))) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fact_attention_pair_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fact_attention_pair_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       cudaFuncAttributes fa, fb;
       if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel<64>);
       if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128>);
+      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_pair_kernel<64>);
+      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_pair_kernel<128>);
       if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
       if (e != cudaSuccess) {
         st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
@@ -1129,7 +1146,9 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      if (pair && head_dim == 64) fact_attention_pair_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      else if (pair) fact_attention_pair_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      else if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       else fact_attention_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
