@@ -46,7 +46,7 @@ __host__ __device__ constexpr uint32_t attn_pair_smem_bytes(int D) {
 }
 
 // How many of every eight key pairs take their exponential on the FMA pipe (0 = all on the special-function unit).
-constexpr int kAttnPolyOf8 = 2;
+constexpr int kAttnPolyOf8 = 1;
 
 // 2^x for a pair of FP32 values, x <= 8 or so, without the special-function unit: x = n + f with n = rint(x)
 // (adding 1.5 * 2^23 leaves n in the low mantissa bits), 2^f on [-0.5, 0.5] by a cubic with relative error
