@@ -364,9 +364,9 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * entry until the first operand stage was ready (the prologue).
  * After a fact_attention launch (same environment variable) the counters are that kernel's: [0] cycles and [1]
  * nanoseconds of the first CTA, [2] a tag of the first device-side wait that gave up (0 if none: barrier index,
- * warp << 8, CTA << 16), [3] cycles softmax warp 0 waited for scores, [4] key blocks it processed, [6] cycles it
- * spent finishing tiles, [7] tiles of that CTA.  The same variable's bits 8, 16, 64 and 128 switch off the
- * attention kernel's softmax arithmetic, its K / V loads, its first and its second products (timing
+ * warp << 8, CTA << 16), [3] cycles the first softmax warp of tile 0 waited for scores, [4] key blocks it
+ * processed, [6] cycles it spent writing finished tiles out, [7] work items of that CTA.  The same variable's bits
+ * 8, 64 and 128 switch off the attention kernel's softmax arithmetic, its first and its second products (timing
  * experiments; the output is then meaningless), like bits 1, 2 and 4 for the GEMM kernel's loads, products
  * and stores. */
 fact_status_t fact_last_kernel_profile(fact_handle_t handle, void* cuda_stream, int64_t counters[8]);

@@ -18,7 +18,6 @@
 #include "fact.h"
 #include "gemm_kernel.cuh"
 #include "attention_kernel.cuh"
-#include "attention_pair_kernel.cuh"
 #include "norm_kernel.cuh"
 
 // Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
@@ -1079,10 +1078,8 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
   if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
   CUtensorMap tq, tk, tv, to;
   auto bs = [&](int64_t s, int64_t fallback) { return (batch > 1 && s > 0) ? s : std::max<int64_t>(fallback, 8); };
-  // Two query tiles per CTA, each a pipeline of its own (keys in blocks of 128 at head_dim 64, of 64 at head_dim
-  // 128), unless the experiment switch (bit 512) asks for the single-tile kernel.
-  const bool pair = !(h->debug_flags & 512);
-  const int block_k = pair ? attn_pair_block_k((int)head_dim) : kAttnBlockK;
+  // keys go in blocks of 128 at head_dim 64 and of 64 at head_dim 128 (the kernel's tensor-memory budget)
+  const int block_k = attn_block_k((int)head_dim);
   fact_status_t st = encode_map_bthd(h, &tq, Q, head_dim, heads_q, seq_q, batch, q_sh, q_st, bs(q_sb, q_st * seq_q));
   if (st == FACT_OK)
     st = encode_map_bthd(h, &tk, K, head_dim, heads_kv, seq_kv, batch, k_sh, k_st, bs(k_sb, k_st * seq_kv), block_k);
@@ -1101,7 +1098,6 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.causal = causal != 0;
     const double sc = scale > 0.f ? (double)scale : 1.0 / std::sqrt((double)head_dim);
     p.scale_log2 = (float)(sc * 1.4426950408889634);
-    p.q_tiles = (int)((seq_q + kAttnBlockQ - 1) / kAttnBlockQ);
     p.kmajor_desc = smem_desc_template(16, 1024);
     p.v_desc = smem_desc_template(block_k * 128, 1024);  // 64-column chunks of V are one block of keys apart
     p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_k >> 3) << 17) | ((uint32_t)(kAttnBlockQ >> 4) << 24);
@@ -1109,30 +1105,22 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
                  ((uint32_t)(kAttnBlockQ >> 4) << 24);
     p.status = h->d_status;
     p.debug = h->debug_flags;
-    p.q_pairs = (p.q_tiles + 1) / 2;
-    const long long items = (long long)(pair ? p.q_pairs : p.q_tiles) * heads_q * batch;
+    p.q_pairs = (int)((seq_q + 2 * kAttnBlockQ - 1) / (2 * kAttnBlockQ));  // an item is two tiles of 128 query rows
+    const long long items = (long long)p.q_pairs * heads_q * batch;
     if (items > 0x7fffffffLL) {
       if (dev != h->device) cudaSetDevice(dev);
       return FACT_ERR_UNSUPPORTED;
     }
     p.items = (int)items;
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
-    const int smem = std::max((int)(pair ? attn_pair_smem_bytes(p.D) : attn_smem_bytes(p.D)), kMinSmemRequest);
+    const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
     if (!(h->configured_mask & (1u << 30))) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(fact_attention_pair_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(fact_attention_pair_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       cudaFuncAttributes fa, fb;
       if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel<64>);
       if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128>);
-      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_pair_kernel<64>);
-      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_pair_kernel<128>);
       if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
       if (e != cudaSuccess) {
         st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
@@ -1146,9 +1134,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      if (pair && head_dim == 64) fact_attention_pair_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
-      else if (pair) fact_attention_pair_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
-      else if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
+      if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       else fact_attention_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
