@@ -92,13 +92,19 @@ typedef enum {
 } fact_blayout_t;
 
 /* Which entry point a workspace / tuning query is about. */
-typedef enum { FACT_OP_GEMM = 0, FACT_OP_GEMM_BATCHED = 1, FACT_OP_GEMM_SPLITK = 2, FACT_OP_LINEAR = 3 } fact_op_t;
+typedef enum {
+  FACT_OP_GEMM = 0,
+  FACT_OP_GEMM_BATCHED = 1,
+  FACT_OP_GEMM_SPLITK = 2,
+  FACT_OP_LINEAR = 3,
+  FACT_OP_LINEAR_FP8 = 4
+} fact_op_t;
 
 /* One kernel configuration.  A zero field means "let the library choose".
  *   tile_m       128 (one CTA per tile) or 256 (a 2-CTA cluster per tile; then cta_group must be 2)
  *   tile_n       accumulator columns per tile, a multiple of 16 in [32, 256] (FACT_B_KN: multiple of 64;
  *                SILU_GATE: multiple of 32, half gate + half up)
- *   tile_k       64 (one 128-byte swizzle row of BF16)
+ *   tile_k       elements of K per pipeline stage: 64 for BF16 operands, 128 for FP8 (one 128-byte swizzle row)
  *   stages       depth of the shared-memory ring, 2..8, limited by 227 KB
  *   cta_group    1 or 2
  *   raster_group G > 0: the scheduler walks groups of G m-tiles (their slab of A/X stays in L2 while the
@@ -218,6 +224,21 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
                           const void* residual, int64_t ldr, void* Y, int64_t ldy, fact_out_t out_type,
                           fact_epilogue_t epilogue, const fact_config_t* cfg, void* workspace,
                           size_t workspace_bytes, void* cuda_stream);
+
+/* Y[M x N_out] = epilogue(scale * X[M x K] . W^T)  with FP8 operands      (Section 3, the pattern table indexed by
+ * rule, data type and architecture; Table 1 lists an FP8 GEMM among the Level-1 kernels the registry holds)
+ * X: FP8 E4M3 [M x K], one byte per element (the OCP "e4m3fn" format: no infinities, S.1111.111 is NaN, largest
+ * magnitude 448); W: FP8 E4M3 [Nw x K] as torch.nn.Linear stores it (Nw = N_out, or 2 * N_out for SILU_GATE).
+ * Products are exact and accumulated in FP32 on the tensor cores (tcgen05.mma.kind::f8f6f4).  `scale` (host
+ * value, finite) multiplies the accumulator before anything else -- the product of the operands' per-tensor
+ * scales; the paper fixes no scaling convention.  bias, residual, Y, out_type, epilogue, cfg and the workspace
+ * are those of fact_linear (bias and residual stay BF16).  ldx and ldw are in elements and must be multiples of
+ * 16 (rows of 16-byte multiples for TMA); X and W 16-byte aligned.  The tuner's key for this entry point is
+ * FACT_OP_LINEAR_FP8 (fact_get_config, fact_workspace_bytes, fact_tune with X, W as A, B and FACT_B_NK). */
+fact_status_t fact_linear_fp8(fact_handle_t handle, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                              const void* W, int64_t ldw, float scale, const void* bias, const void* residual,
+                              int64_t ldr, void* Y, int64_t ldy, fact_out_t out_type, fact_epilogue_t epilogue,
+                              const fact_config_t* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* O = softmax(scale * Q K^T + causal mask) V, fused           (Section 5.2, pattern p1: fused multi-head
  * attention -- causal for the MiniGPT block; grouped queries, 32 query heads over 8 key/value heads of

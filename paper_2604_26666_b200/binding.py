@@ -28,7 +28,7 @@ STATUS_NAMES = {
 EPILOGUES = {"NONE": 0, "BIAS": 1, "BIAS_RELU": 2, "BIAS_GELU_TANH": 3, "SILU_GATE": 4, "BIAS_RESIDUAL": 5}
 LAYOUTS = {"KN": 0, "NK": 1}
 OUT_TYPES = {torch.bfloat16: 0, torch.float32: 1, "bf16": 0, "f32": 1}
-OPS = {"gemm": 0, "gemm_batched": 1, "gemm_splitk": 2, "linear": 3}
+OPS = {"gemm": 0, "gemm_batched": 1, "gemm_splitk": 2, "linear": 3, "linear_fp8": 4}
 
 # every symbol include/fact.h declares
 EXPORTED = [
@@ -37,7 +37,7 @@ EXPORTED = [
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
-    "fact_stream_k_pieces",
+    "fact_stream_k_pieces", "fact_linear_fp8",
 ]
 
 
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
     L.fact_block_workspace_bytes.restype = sz
     L.fact_block_workspace_offsets.argtypes = [POINTER(Block), POINTER(sz)]
     L.fact_block_forward.argtypes = [vp, POINTER(Block), vp, vp, vp, sz, vp]
+    L.fact_linear_fp8.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_float, vp, vp, i64, vp, i64, c_int, c_int, cfgp,
+                                  vp, sz, vp]
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     for name in EXPORTED:
         fn = getattr(L, name)
@@ -388,6 +390,45 @@ class Handle:
                                  _ptr(residual), _ld(residual) if residual is not None else 0, _ptr(out), _ld(out),
                                  OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg), _ptr(ws), nws,
                                  self._stream(stream)), "fact_linear", self._h)
+        return out
+
+    def linear_fp8(self, X, W, scale=1.0, bias=None, residual=None, epilogue="NONE", out=None,
+                   out_dtype=torch.bfloat16, cfg=None, stream=None):
+        """Y = epilogue(scale * X @ W^T)  (fact_linear_fp8).  X [M, K] and W [Nw, K] are FP8 E4M3: torch.float8_e4m3fn
+        tensors, or torch.uint8 tensors holding the codes."""
+        def codes(t, name):
+            if isinstance(t, torch.Tensor) and t.dtype == torch.float8_e4m3fn:
+                t = t.view(torch.uint8)
+            _need(t, name, torch.uint8, 2)
+            return t
+        X, W = codes(X, "X"), codes(W, "W")
+        M, K = X.shape
+        Nw = W.shape[0]
+        if W.shape[1] != K:
+            raise ValueError("inner dimensions differ")
+        if epilogue == "SILU_GATE":
+            if Nw % 2:
+                raise ValueError("SILU_GATE needs an even number of weight rows")
+            N = Nw // 2
+        else:
+            N = Nw
+        if bias is not None:
+            _need(bias, "bias", torch.bfloat16, 1)
+            if bias.shape[0] != N:
+                raise ValueError("bias must have N_out entries")
+        if residual is not None:
+            _need(residual, "residual", torch.bfloat16, 2)
+            if tuple(residual.shape) != (M, N):
+                raise ValueError("residual must be [M, N_out]")
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype, device=X.device)
+        _need(out, "out", out.dtype, 2)
+        nws = self.workspace_bytes("linear_fp8", 1, M, N, K, epilogue, "NK", out.dtype, cfg)
+        ws = self.workspace(nws)
+        _check(lib().fact_linear_fp8(self._h, M, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W), float(scale), _ptr(bias),
+                                     _ptr(residual), _ld(residual) if residual is not None else 0, _ptr(out), _ld(out),
+                                     OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg), _ptr(ws), nws,
+                                     self._stream(stream)), "fact_linear_fp8", self._h)
         return out
 
     def attention(self, q, k, v, causal=True, scale=0.0, out=None, stream=None):

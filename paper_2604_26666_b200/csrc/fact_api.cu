@@ -59,7 +59,11 @@ struct Problem {
   long long ldc, strideC;
   fact_out_t out;
   fact_epilogue_t epi;
+  bool fp8 = false;    // operands are FP8 E4M3 (one byte per element) instead of BF16
+  float alpha = 1.f;   // FP8: the accumulator is multiplied by this before the epilogue
   long long Nw() const { return epi == FACT_EPI_SILU_GATE ? 2 * N_out : N_out; }
+  int k_elems() const { return fp8 ? 2 * kTileK : kTileK; }  // elements of K in a 128-byte row of a stage
+  int op_align() const { return fp8 ? 16 : 8; }              // elements in 16 bytes of an operand
 };
 
 struct Plan {
@@ -157,15 +161,15 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     }
   }
   if (splits_override > 0) c.split_k = splits_override;
-  if (c.tile_k != 0 && c.tile_k != kTileK) return FACT_ERR_UNSUPPORTED;
-  c.tile_k = kTileK;
+  if (c.tile_k != 0 && c.tile_k != q.k_elems()) return FACT_ERR_UNSUPPORTED;
+  c.tile_k = q.k_elems();
   const long long Nw = q.Nw();
   if (c.cta_group == 0 && c.tile_m != 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
   if (c.cta_group == 0 || c.tile_n == 0) {
     // Untuned problem: pick (pair size, tile width) with a small cost model -- waves over the SMs times the
     // cycles of one tile (k-blocks at the tensor-pipe rate of that width, plus a fixed hand-over cost).  A
     // 2-CTA pair halves each CTA's B traffic and wins ties; narrow tiles only pay when wide ones leave SMs idle.
-    const int k_blocks = std::max(1, (int)((q.K + kTileK - 1) / kTileK));
+    const int k_blocks = std::max(1, (int)((q.K + q.k_elems() - 1) / q.k_elems()));
     double best = 1e300;
     int best_cg = 0, best_tn = 0;
     for (int cg = 2; cg >= 1; --cg) {
@@ -219,7 +223,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     const double cost_n = w_bytes + x_bytes * (double)((tiles_n + gn - 1) / gn);
     c.raster_group = (cost_n < cost_m * 0.95) ? -(int)gn : (int)gm;
   }
-  const int k_blocks = (int)((q.K + kTileK - 1) / kTileK);
+  const int k_blocks = (int)((q.K + q.k_elems() - 1) / q.k_elems());
   if (c.split_k == 0) {
     c.split_k = 1;
     if (q.op == FACT_OP_GEMM_SPLITK) {
@@ -265,9 +269,10 @@ fact_status_t validate(const Problem& q) {
     if (q.lda < q.K) return FACT_ERR_INVALID_ARG;
     if (q.ldb < (q.layout == FACT_B_KN ? q.Nw() : q.K)) return FACT_ERR_INVALID_ARG;
     if (!aligned16(q.A) || !aligned16(q.B)) return FACT_ERR_BAD_ALIGNMENT;
-    if (q.lda % 8 || q.ldb % 8) return FACT_ERR_BAD_ALIGNMENT;
+    if (q.lda % q.op_align() || q.ldb % q.op_align()) return FACT_ERR_BAD_ALIGNMENT;
+    if (q.fp8 && q.layout != FACT_B_NK) return FACT_ERR_UNSUPPORTED;  // 8-bit operands are read K-major only
     if (q.batch > 1) {
-      if (q.strideA % 8 || q.strideB % 8) return FACT_ERR_BAD_ALIGNMENT;
+      if (q.strideA % q.op_align() || q.strideB % q.op_align()) return FACT_ERR_BAD_ALIGNMENT;
       if (q.strideA < 0 || q.strideB < 0 || q.strideC < 0) return FACT_ERR_INVALID_ARG;
     }
   }
@@ -286,7 +291,7 @@ int sk_tiles_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
   if (out_cols % (f32 ? 32 : 64) != 0 || (f32 && q.epi == FACT_EPI_BIAS_RESIDUAL) || c.store_mode == 1) return 0;
   const long long tiles = q.batch * ((q.M + c.tile_m - 1) / c.tile_m) * ((q.N_out + out_cols - 1) / out_cols);
   const long long groups = std::max(1, h->sm_count / c.cta_group);
-  const long long k_blocks = (q.K + kTileK - 1) / kTileK;
+  const long long k_blocks = (q.K + q.k_elems() - 1) / q.k_elems();
   long long sk = tiles % groups;
   if (sk == 0) return 0;
   if (c.split_k == -2 && tiles >= sk + groups) sk += groups;
@@ -331,7 +336,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.out_cols = gate ? c.tile_n / 2 : c.tile_n;
   p.tiles_m = (int)((q.M + c.tile_m - 1) / c.tile_m);
   p.tiles_n = (int)((q.N_out + p.out_cols - 1) / p.out_cols);
-  p.k_blocks = (int)((q.K + kTileK - 1) / kTileK);
+  p.k_blocks = (int)((q.K + q.k_elems() - 1) / q.k_elems());
   const int slices = std::max(1, c.split_k);  // (stream-K, split_k < 0, cuts no tile into equal slices)
   p.split_k = slices;
   p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
@@ -376,6 +381,12 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   // N >> 3 @ bit 17, M >> 4 @ bit 24
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_kn << 16) | ((uint32_t)(c.tile_n >> 3) << 17) |
             ((uint32_t)((kTileM * cg) >> 4) << 24);
+  // kind::f8f6f4: format 0 = E4M3 for A and B (bits 7 and 10 clear), K-major both, one instruction per 32 bytes of K
+  if (q.fp8) p.idesc &= ~((1u << 7) | (1u << 10));
+  p.k_elems = q.k_elems();
+  p.fp8 = q.fp8 ? 1 : 0;
+  p.use_alpha = (q.fp8 && q.alpha != 1.f) ? 1 : 0;
+  p.alpha = q.alpha;
   p.tmem_cols = pow2_at_least((uint32_t)(2 * c.tile_n));
   p.C = q.C;
   p.ldc = q.ldc;
@@ -430,13 +441,13 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
 // A rank-3 tensor map (inner, rows, batch) with a (box0 x box1 x 1) box and 128-byte swizzle.
 fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
                          uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1,
-                         bool f32 = false) {
-  const uint64_t esz = f32 ? 4 : 2;
+                         bool f32 = false, bool u8 = false) {
+  const uint64_t esz = f32 ? 4 : (u8 ? 1 : 2);
   cuuint64_t dims[3] = {d0, d1, d2};
   cuuint64_t strides[2] = {stride1_elems * esz, stride2_elems * esz};
   cuuint32_t box[3] = {box0, box1, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = h->encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+  CUresult r = h->encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : (u8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 3,
                          const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -527,6 +538,7 @@ fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan,
   r.R = reinterpret_cast<const __nv_bfloat16*>(q.R);
   r.ldr = q.ldr;
   r.strideR = q.strideR;
+  r.alpha = q.fp8 ? q.alpha : 1.f;
   const long long total = 4LL * r.batch * r.M * ((r.N_out + 3) / 4);  // four threads per group of 4 columns
   const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)h->sm_count * 16);
   fact_splitk_reduce_kernel<<<std::max(1, blocks), 128, 0, stream>>>(r);
@@ -583,8 +595,9 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     memset(tm, 0, sizeof tm);
     const uint64_t batch_dim = (uint64_t)q.batch;
     const uint64_t sA = q.batch > 1 ? (uint64_t)q.strideA : (uint64_t)q.lda * (uint64_t)q.M;
-    st = encode_map(h, &tmA, q.A, (uint64_t)q.K, (uint64_t)q.M, batch_dim, (uint64_t)q.lda, std::max<uint64_t>(sA, 8),
-                    kTileK, kTileM);
+    const uint32_t kbox = (uint32_t)q.k_elems();  // 128 bytes of K
+    st = encode_map(h, &tmA, q.A, (uint64_t)q.K, (uint64_t)q.M, batch_dim, (uint64_t)q.lda, std::max<uint64_t>(sA, 16),
+                    kbox, kTileM, false, q.fp8);
     if (st != FACT_OK) return st;
     if (q.layout == FACT_B_KN) {
       const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.K;
@@ -593,7 +606,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     } else {
       const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.Nw();
       st = encode_map(h, &tmB, q.B, (uint64_t)q.K, (uint64_t)q.Nw(), batch_dim, (uint64_t)q.ldb,
-                      std::max<uint64_t>(sB, 8), kTileK, (uint32_t)plan.p.b_box_n);
+                      std::max<uint64_t>(sB, 16), kbox, (uint32_t)plan.p.b_box_n, false, q.fp8);
     }
     if (st != FACT_OK) return st;
     if (split) {
@@ -653,6 +666,8 @@ Problem make_problem(fact_op_t op, long long batch, long long M, long long N, lo
   q.strideC = sC;
   q.out = out;
   q.epi = epi;
+  q.fp8 = op == FACT_OP_LINEAR_FP8;
+  q.alpha = 1.f;
   return q;
 }
 
@@ -865,6 +880,17 @@ fact_status_t fact_linear(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, 
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
 }
 
+fact_status_t fact_linear_fp8(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                              const void* W, int64_t ldw, float scale, const void* bias, const void* residual,
+                              int64_t ldr, void* Y, int64_t ldy, fact_out_t out, fact_epilogue_t epi,
+                              const fact_config_t* cfg, void* ws, size_t ws_bytes, void* stream) {
+  if (!(scale == scale) || std::isinf(scale)) return FACT_ERR_INVALID_ARG;
+  Problem q = make_problem(FACT_OP_LINEAR_FP8, 1, M, N_out, K, X, ldx, 0, W, ldw, 0, FACT_B_NK, bias, residual, ldr, 0,
+                           Y, ldy, 0, out, epi);
+  q.alpha = scale;
+  return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
 fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
                         int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
                         fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, int64_t strideR,
@@ -885,7 +911,7 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
 
   // Candidate axes: pair size, tile width, ring depth, K slices.
   std::vector<fact_config_t> cands;
-  const int k_blocks = (int)((K + kTileK - 1) / kTileK);
+  const int k_blocks = (int)((K + q.k_elems() - 1) / q.k_elems());
   for (int cg = 1; cg <= 2; ++cg) {
     for (int tn = 32; tn <= 256; tn += 32) {
       if (!tile_ok(q, tn, cg)) continue;
@@ -916,7 +942,7 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
       // short timing run cannot resolve; the model in resolve_config chooses it)
       for (int stg : stage_opts)
         for (int sp : splits) {
-          fact_config_t c = {128 * cg, tn, kTileK, stg, cg, 0, sp, 0};
+          fact_config_t c = {128 * cg, tn, q.k_elems(), stg, cg, 0, sp, 0};
           cands.push_back(c);
         }
     }

@@ -105,6 +105,11 @@ struct GemmParams {
   int fused_reduce;   // 1: after a grid-wide barrier every CTA reduces its share of the output (split-K only)
   int reduce_epi;     // the epilogue the reduction applies
   int* status;        // [0] error word, [2..17] clock / profile counters, [24], [25] grid-barrier counters
+  // 8-bit operands (FP8 E4M3, one byte per element): a k-block is 128 elements, still 128 bytes per row
+  int k_elems;        // elements of K per k-block: 64 (BF16) or 128 (FP8)
+  int fp8;            // 1: tcgen05.mma.kind::f8f6f4, else kind::f16
+  int use_alpha;      // 1: the accumulator is multiplied by alpha before the epilogue (FP8: the operands' scales)
+  float alpha;
   // stream-K (the SK instantiations only): the last `sk_tiles` tiles of the tile list are cut along K into one
   // contiguous run of k-blocks per CTA group; see UnitWalk
   int sk_tiles;       // 0: every tile is data-parallel
@@ -382,6 +387,7 @@ struct ReduceParams {
   const __nv_bfloat16* bias;
   const __nv_bfloat16* R;
   long long ldr, strideR;
+  float alpha;  // the summed accumulator is multiplied by this first (1 unless the operands carry scales)
 };
 
 __device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, float bias, float res) {
@@ -472,7 +478,7 @@ __device__ __forceinline__ void reduce_groups(const ReduceParams& p, long long f
       const float bias = p.bias ? __bfloat162float(p.bias[n + j]) : 0.f;
       const float res =
           (p.epi == kEpiBiasResidual) ? __bfloat162float(p.R[(long long)b * p.strideR + (long long)m * p.ldr + n + j]) : 0.f;
-      const float y = reduce_epilogue(p.epi, av, uv, bias, res);
+      const float y = reduce_epilogue(p.epi, av * p.alpha, uv * p.alpha, bias, res);
       const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n + j;
       if (p.out_f32) reinterpret_cast<float*>(p.C)[off] = y;
       else reinterpret_cast<__nv_bfloat16*>(p.C)[off] = __float2bfloat16_rn(y);
@@ -650,10 +656,10 @@ __global__ void __launch_bounds__(kThreads, 1)
               if constexpr (CG == 2) {
                 if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
                 fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
-                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
+                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * p.k_elems, m0, w.b);
               } else {
                 ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-                ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+                ptx::tma_load_3d(sa, &tmA, fb, kb * p.k_elems, m0, w.b);
               }
             } else {
               if constexpr (CG == 2) fb = ptx::mapa(fb, 0);
@@ -662,11 +668,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (i < p.b_loads) {
                   const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
                   if constexpr (CG == 2) {
-                    if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n_box[i], kb * kTileK, w.b);
-                    else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n_box[i], w.b);
+                    if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b);
+                    else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b);
                   } else {
-                    if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n_box[i], kb * kTileK, w.b);
-                    else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n_box[i], w.b);
+                    if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b);
+                    else ptx::tma_load_3d(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b);
                   }
                 }
               }
@@ -729,8 +735,12 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!(p.debug & 2)) {
 #pragma unroll
               for (int k = 0; k < kTileK / kUmmaK; ++k) {
-                ptx::umma_bf16<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
+                if (p.fp8)
+                  ptx::umma_f8<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
                                    p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+                else
+                  ptx::umma_bf16<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
+                                     p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
               }
             }
             // release the stage (in both CTAs of a pair) once these MMAs have read it
@@ -767,6 +777,14 @@ __global__ void __launch_bounds__(kThreads, 1)
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
+    // FP8 operands: the accumulator times alpha (the product of the operands' scales), before anything else.  Not for
+    // the split-K partial store: there the reduction applies it to the sum.
+    const bool scale_acc = p.use_alpha != 0 && EPI != kEpiPartial;
+    const float alpha = p.alpha;
+    auto scale32 = [&](uint32_t (&v)[32]) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+    };
     if (p.store_tma) {
       // ---- staged: registers -> swizzled shared memory -> TMA tensor store, 32 rows x 128 bytes at a time
       const int bufs = p.epi_bufs;
@@ -959,6 +977,10 @@ __global__ void __launch_bounds__(kThreads, 1)
           add_peers(v0, c0);
           if constexpr (EPI == kEpiSiluGate) add_peers(v1, p.out_cols + c0);
           else if (pieces == 2) add_peers(v1, c0 + 32);
+          if (scale_acc) {
+            scale32(v0);
+            if (EPI == kEpiSiluGate || pieces == 2) scale32(v1);
+          }
           // one 32-column piece: fused operation on packed FP32 pairs, rounding, into outw
           auto do_piece = [&](int piece, const uint32_t (&a)[32], const uint32_t (&up)[32]) {
             const int local0 = (ci >> 1) * chunk_cols + piece * 32;  // index among the warp's 128 columns
@@ -1011,6 +1033,10 @@ __global__ void __launch_bounds__(kThreads, 1)
               ptx::tmem_wait_ld();
               add_peers(v0, c0 + 32);
               add_peers(v1, p.out_cols + c0 + 32);
+              if (scale_acc) {
+                scale32(v0);
+                scale32(v1);
+              }
               do_piece(1, v0, v1);
             }
           } else {
@@ -1093,6 +1119,10 @@ __global__ void __launch_bounds__(kThreads, 1)
           ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
           if constexpr (EPI == kEpiSiluGate) ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)(p.out_cols + c), vu);
           ptx::tmem_wait_ld();
+          if (scale_acc) {
+            scale32(v);
+            if (EPI == kEpiSiluGate) scale32(vu);
+          }
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             const int n = n0 + g * 8;
@@ -1169,6 +1199,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         r.R = p.R;
         r.ldr = p.ldr;
         r.strideR = p.strideR;
+        r.alpha = p.use_alpha ? p.alpha : 1.f;
         reduce_groups(r, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
       }
       __syncthreads();

@@ -294,3 +294,61 @@ def make_block_inputs(case, device="cpu"):
         t = 1.0 + 0.1 * t if "gamma" in name else 0.02 * t
         w[name] = t.to(torch.bfloat16).to(device)
     return x, w
+
+
+# ---------------------------------------------------------------------------------------------
+# FP8 (E4M3) linear layers: the paper's pattern table is indexed by (rule, data type, architecture) and lists
+# an FP8 GEMM among its Level-1 kernels (Section 3, Table 1); it gives no FP8 shapes, so the BF16 shapes are reused.
+@dataclass(frozen=True)
+class Fp8Case:
+    name: str
+    M: int
+    N: int
+    K: int
+    epilogue: str = "NONE"
+    has_bias: bool = False
+    seed: int = 0
+    x_amax: float = 4.0   # activations are scaled so that this many standard deviations reach the format's 448
+    w_std: float = 0.02
+
+    @property
+    def flops(self) -> float:
+        return 2.0 * self.M * self.N * self.K
+
+    @property
+    def algorithmic_bytes(self) -> float:
+        return float(self.M * self.K + self.N * self.K + self.M * self.N * 2 + (self.N * 2 if self.has_bias else 0))
+
+
+def fp8_cases() -> list[Fp8Case]:
+    """The square 8192 problem, and the Llama-shaped and GPT-shaped MLP up-projections of the BF16 configurations."""
+    return [
+        Fp8Case("f8_square_8192", 8192, 8192, 8192, seed=7200),
+        Fp8Case("f8_llama_qkv", 8192, 6144, 4096, seed=7201),
+        Fp8Case("f8_gpt_up_gelu", 16384, 3072, 768, epilogue="BIAS_GELU_TANH", has_bias=True, seed=7202),
+    ]
+
+
+@dataclass
+class Fp8Inputs:
+    X: torch.Tensor                 # uint8 E4M3 codes [M, K]
+    W: torch.Tensor                 # uint8 E4M3 codes [N, K]
+    scale: float                    # the product of the two per-tensor scales
+    bias: Optional[torch.Tensor]    # BF16 [N] or None
+
+
+def make_fp8_inputs(case: Fp8Case) -> Fp8Inputs:
+    """Per-tensor scaled quantisation of N(0,1) activations and N(0, w_std^2) weights, as an FP8 inference stack
+    would store them: x_q = e4m3(x * sx), w_q = e4m3(w * sw) with the scales chosen so that `x_amax` standard
+    deviations map to the format's largest value; the kernel is given 1 / (sx * sw).  Values beyond that clip
+    to +-448 (torch's conversion saturates).  No arithmetic of the method: rounding random numbers to the
+    storage format is input generation."""
+    g = torch.Generator(device="cpu").manual_seed(case.seed)
+    x = torch.randn((case.M, case.K), generator=g, dtype=torch.float32)
+    w = torch.randn((case.N, case.K), generator=g, dtype=torch.float32) * case.w_std
+    bias = torch.randn((case.N,), generator=g, dtype=torch.float32).to(torch.bfloat16) if case.has_bias else None
+    sx = 448.0 / case.x_amax
+    sw = 448.0 / (case.x_amax * case.w_std)
+    xq = (x * sx).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+    wq = (w * sw).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+    return Fp8Inputs(xq, wq, 1.0 / (sx * sw), bias)
