@@ -194,7 +194,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention` or `blocks`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8` or `blocks`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
@@ -236,12 +236,12 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        rows = [] if args.shape in ("attention", "blocks") else per_shape_table(
+        rows = [] if args.shape in ("attention", "blocks", "fp8") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
             side_ref=False, layout=args.layout)
         if args.shape in ("all", "attention"):
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
-        elif args.shape == "blocks":
+        elif args.shape in ("blocks", "fp8"):
             att = []
         else:  # attention shapes can be named like the GEMM shapes
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
@@ -251,7 +251,14 @@ def main():
             blk = block_table(h, dev, stream, flush_l2, peaks)
         elif args.shape == "blocks":  # --warmup / --steps apply, no eager side reference: the form the ncu runs use
             blk = block_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False)
-        print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "gpu_launches": h.launch_count()}))
+        f8 = []
+        if args.shape in ("all", "fp8"):
+            f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps,
+                           side_ref=args.shape == "all")
+        elif names is not None:  # FP8 shapes can be named like the GEMM shapes
+            f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
+                           names=names)
+        print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "fp8": f8, "gpu_launches": h.launch_count()}))
         h.close()
         return 0
 
@@ -340,9 +347,10 @@ def main():
     shapes = []
     if not args.no_shapes and rank == 0:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
-    attention, blocks = [], []
+    attention, blocks, fp8 = [], [], []
     if not args.no_shapes and rank == 0:
         attention = attention_table(h, dev, stream, flush_l2, peaks)
+        fp8 = fp8_table(h, dev, stream, flush_l2, peaks)
         blocks = block_table(h, dev, stream, flush_l2, peaks)
     clocks = sampler.stop()  # sampled from the first warm-up step to the end of the per-shape table
 
@@ -378,6 +386,7 @@ def main():
             "cpu_baseline": cpu,
             "shapes": shapes,
             "attention": attention,
+            "fp8": fp8,
             "blocks": blocks,
         }
         print(json.dumps(line))
@@ -516,6 +525,68 @@ def attention_table(h, dev, stream, flush_l2, peaks, warm=5, iters=20, side_ref=
         })
         assert h.device_status() == 0
         del q, k, v, out
+    return rows
+
+
+def fp8_table(h, dev, stream, flush_l2, peaks, warm=5, iters=20, side_ref=True, names=None):
+    """Time fact_linear_fp8 (FP8 E4M3 operands, BF16 output) on the FP8 shapes, L2 overwritten between launches;
+    torch._scaled_mm (cuBLASLt, matmul only) on the same operands is a side reference.  The peak is the measured
+    BF16 burst peak times the nominal FP8 : BF16 ratio of 2 (there is no measured FP8 figure)."""
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    rows = []
+    peak = 2.0 * peaks["bf16_tflops"]
+    for case in wl.fp8_cases():
+        if names is not None and case.name not in names:
+            continue
+        ins = wl.make_fp8_inputs(case)
+        X, W = ins.X.to(dev), ins.W.to(dev)
+        bias = None if ins.bias is None else ins.bias.to(dev)
+        out = torch.empty((case.M, case.N), dtype=torch.bfloat16, device=dev)
+
+        def call():
+            h.linear_fp8(X, W, ins.scale, bias, epilogue=case.epilogue, out=out)
+
+        def time_it(fn, n):
+            for _ in range(warm):
+                fn()
+            ts = []
+            for _ in range(n):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                ts.append((a, b))
+            torch.cuda.synchronize(dev)
+            return sorted(x.elapsed_time(y) for x, y in ts)
+
+        t = time_it(call, iters)
+        med = t[len(t) // 2]
+        ts = [0.0]
+        if side_ref:
+            try:
+                xs, wt = X.view(torch.float8_e4m3fn), W.view(torch.float8_e4m3fn).t()
+                one = torch.tensor(1.0, device=dev)
+                ts = time_it(lambda: torch._scaled_mm(xs, wt, scale_a=one, scale_b=one, out_dtype=torch.bfloat16), 10)
+            except Exception:  # the side reference is optional
+                ts = [float("nan")]
+        t_tensor = case.flops / (peak * 1e12) * 1e3
+        t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        c = h.get_config("linear_fp8", 1, case.M, case.N, case.K, case.epilogue, "NK", torch.bfloat16).as_dict()
+        rows.append({
+            "name": case.name, "M": case.M, "N": case.N, "K": case.K, "epilogue": case.epilogue, "dtype": "f8e4m3",
+            "us_median": med * 1e3, "us_min": t[0] * 1e3, "tflops": case.flops / (med * 1e-3) / 1e12,
+            "gbs": case.algorithmic_bytes / (med * 1e-3) / 1e9,
+            "bound": "tensor" if t_tensor >= t_hbm else "hbm", "peak_tflops": peak,
+            "peak_source": "2 x measured BF16 burst (nominal FP8 : BF16 ratio)",
+            "roofline_us": max(t_tensor, t_hbm) * 1e3, "roofline_frac": max(t_tensor, t_hbm) / med,
+            "cublaslt_scaled_mm_only_us": ts[len(ts) // 2] * 1e3, "tile": c,
+        })
+        assert h.device_status() == 0
+        del X, W, out
     return rows
 
 

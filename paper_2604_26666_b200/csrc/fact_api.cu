@@ -182,7 +182,11 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
             std::max<long long>(1, q.batch) * ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + out_cols - 1) / out_cols);
         const long long slots = std::max(1, h->sm_count / cg);
         const double waves = (double)((tiles + slots - 1) / slots);
-        const double per_tile = k_blocks * 512.0 * std::max(tn, 96) / 256.0 + 1500.0 + (cg == 1 ? 60.0 * k_blocks : 0.0);
+        // (narrower tiles re-read the A operand from shared memory for less work: measured 0.65 of the full rate at
+        // 128 columns, taken as 0.85 at 192)
+        const double eff = tn >= 256 ? 1.0 : (tn >= 192 ? 0.85 : 0.65);
+        const double per_tile =
+            k_blocks * 512.0 * std::max(tn, 96) / 256.0 / eff + 1500.0 + (cg == 1 ? 60.0 * k_blocks : 0.0);
         const double cost = waves * per_tile;
         if (cost < best * 0.999) {
           best = cost;

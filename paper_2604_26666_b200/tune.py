@@ -3,6 +3,7 @@ write the table that `Handle` loads by default.
 
     python -m paper_2604_26666_b200.tune [--out PATH] [--layout NK|KN|both] [--shapes a,b,...]
     python -m paper_2604_26666_b200.tune --set paper --merge     (the paper's own shapes, added to the table)
+    python -m paper_2604_26666_b200.tune --set fp8 --merge       (the FP8 shapes)
 
 The counterpart of the paper's auto-tuning action (Section 4.2, Action 5): every
 feasible candidate is timed on the device (5 warm-up + 20 timed launches, the
@@ -31,6 +32,12 @@ def tune_case(h: Handle, case: wl.Case, dev: str = "cuda:0"):
     return h.tune(case.op, X, W, layout=case.layout, bias=bias, residual=res, epilogue=case.epilogue, out_dtype=odt)
 
 
+def tune_fp8_case(h: Handle, case: wl.Fp8Case, dev: str = "cuda:0"):
+    ins = wl.make_fp8_inputs(case)
+    bias = None if ins.bias is None else ins.bias.to(dev)
+    return h.tune("linear_fp8", ins.X.to(dev), ins.W.to(dev), layout="NK", bias=bias, epilogue=case.epilogue)
+
+
 def paper_set():
     """The paper's own Level-1 shapes and the four linears of each of its two blocks at the paper's token counts."""
     cases = list(wl.paper_cases())
@@ -55,7 +62,7 @@ def main(argv=None):
     ap.add_argument("--out", default=str(DEFAULT_TABLE))
     ap.add_argument("--layout", default="both", choices=["NK", "KN", "both"])
     ap.add_argument("--shapes", default=None)
-    ap.add_argument("--set", default="benchmark", choices=["benchmark", "paper"])
+    ap.add_argument("--set", default="benchmark", choices=["benchmark", "paper", "fp8"])
     ap.add_argument("--merge", action="store_true", help="start from the table already in --out")
     args = ap.parse_args(argv)
     h = Handle(0, load_table=False)
@@ -64,6 +71,14 @@ def main(argv=None):
     names = None if args.shapes is None else set(args.shapes.split(","))
     seen = set()
     layouts = ["NK", "KN"] if (args.layout == "both" and args.set == "benchmark") else [args.layout if args.layout != "both" else "NK"]
+    if args.set == "fp8":
+        for case in wl.fp8_cases():
+            if names is not None and case.name not in names:
+                continue
+            cfg, ms, n = tune_fp8_case(h, case)
+            print(f"{case.name:32s} NK best {ms * 1e3:9.1f} us  {case.flops / ms / 1e9:8.1f} TFLOP/s  "
+                  f"of {n:3d} candidates: {cfg}", flush=True)
+        layouts = []
     for layout in layouts:
         for case in (wl.benchmark_cases(layout) if args.set == "benchmark" else paper_set()):
             key = (case.name, case.layout)

@@ -22,7 +22,7 @@ def libfact():
 def declared_symbols():
     text = (ROOT / "include" / "fact.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(fact_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(fact_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(libfact):
