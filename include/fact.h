@@ -26,8 +26,8 @@
  *   - Ownership: the caller owns every buffer and the stream.  The library
  *     never allocates or frees device memory on a call path; split-K scratch
  *     is a caller-provided workspace sized by fact_workspace_bytes.  The handle
- *     owns a small device status word, a cache of encoded tensor maps and the
- *     tuner's table.
+ *     owns a small device status area (status word, counters, stream-K flags),
+ *     a 32 KB device table for grouped calls and the tuner's table.
  *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and return; results are valid
  *     in stream order.
@@ -128,8 +128,8 @@ typedef struct {
 } fact_config_t;
 
 /* Create / destroy a handle bound to CUDA device `device`.  fact_create makes
- * that device current, checks for sm_100, allocates the 4-byte device status
- * word and resolves the driver's tensor-map encoder.  These two calls are the
+ * that device current, checks for sm_100, allocates the handle's two small device
+ * buffers and resolves the driver's tensor-map encoder.  These two calls are the
  * only ones that allocate or free device memory. */
 fact_status_t fact_create(fact_handle_t* handle, int device);
 fact_status_t fact_destroy(fact_handle_t handle);
@@ -224,6 +224,24 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
                           const void* residual, int64_t ldr, void* Y, int64_t ldy, fact_out_t out_type,
                           fact_epilogue_t epilogue, const fact_config_t* cfg, void* workspace,
                           size_t workspace_bytes, void* cuda_stream);
+
+/* Grouped linear layer: the rows of X and Y are cut into `groups` consecutive row groups and group g is multiplied
+ * by its own weight matrix,      Y[rows of g, :] = epilogue(X[rows of g, :] . W[g])
+ * (Table 1 lists "Grouped GEMM" among the Level-3 kernels of the registry for both architectures: a list of
+ * products of different sizes in one launch, as a mixture-of-experts layer needs after its tokens have been sorted
+ * by expert).  group_rows: HOST array of `groups` row counts (>= 0, at most 4096 groups); M is their sum.
+ * X: BF16 [M x K], ldx.  W[g]: BF16 at W + g * strideW elements, [Nw x K] (FACT_B_NK) or [K x Nw] (FACT_B_KN), ldw;
+ * strideW a multiple of 8.  bias [N_out] (shared by the groups), residual [M x N_out], Y, out_type, epilogue as in
+ * fact_linear.  One launch: tiles never cross a group boundary (the last tile of a group is ragged), all tiles are
+ * data-parallel, the output is stored by row-predicated register stores (the group table travels to a buffer of
+ * the handle in stream order, so grouped calls through one handle must be stream-ordered with respect to each
+ * other).  cfg: tile shape, pair size and stages only (K slices, stream-K and staged stores are refused with
+ * FACT_ERR_UNSUPPORTED).  groups == 0 or M == 0 is a successful no-op. */
+fact_status_t fact_linear_grouped(fact_handle_t handle, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
+                                  const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
+                                  fact_blayout_t w_layout, const void* bias, const void* residual, int64_t ldr, void* Y,
+                                  int64_t ldy, fact_out_t out_type, fact_epilogue_t epilogue, const fact_config_t* cfg,
+                                  void* cuda_stream);
 
 /* Y[M x N_out] = epilogue(scale * X[M x K] . W^T)  with FP8 operands      (Section 3, the pattern table indexed by
  * rule, data type and architecture; Table 1 lists an FP8 GEMM among the Level-1 kernels the registry holds)

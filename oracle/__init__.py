@@ -200,6 +200,30 @@ def linear(X, W, *, layout="KN", epilogue="NONE", bias=None, residual=None, rows
     return Y if batched else Y[0]
 
 
+def linear_grouped(X, W, group_rows, *, layout="NK", epilogue="NONE", bias=None, residual=None):
+    """Grouped linear layer (the "Grouped GEMM" of the paper's Table 1), written out as its definition: the rows of X
+    are cut into consecutive groups of ``group_rows[g]`` rows and group g is multiplied by ``W[g]``:
+    ``Y[rows of g] = epilogue(X[rows of g] @ W[g])``, one call of ``linear`` per group.
+    X : uint16 [M, K];  W : uint16 [G, Nw, K] ("NK") or [G, K, Nw] ("KN");  bias [N_out] shared by the groups;
+    residual [M, N_out].  Returns float64 [M, N_out]."""
+    X = _bits(X, "X")
+    W = _bits(W, "W")
+    rows = [int(r) for r in group_rows]
+    if W.ndim != 3 or W.shape[0] != len(rows) or sum(rows) != X.shape[0] or min(rows, default=0) < 0:
+        raise ValueError("group_rows must give one non-negative row count per weight matrix and sum to the rows of X")
+    Nw = W.shape[2] if layout == "KN" else W.shape[1]
+    N_out = Nw // 2 if epilogue == "SILU_GATE" else Nw
+    Y = np.empty((X.shape[0], N_out), dtype=np.float64)
+    r0 = 0
+    for g, n in enumerate(rows):
+        if n:
+            res = None if residual is None else np.ascontiguousarray(residual[r0:r0 + n])
+            Y[r0:r0 + n] = linear(np.ascontiguousarray(X[r0:r0 + n]), np.ascontiguousarray(W[g]), layout=layout,
+                                  epilogue=epilogue, bias=bias, residual=res)
+        r0 += n
+    return Y
+
+
 def round_bf16(x: float) -> int:
     """Nearest-even BF16 bit pattern of a double (one rounding)."""
     return int(_load().fact_oracle_round_bf16(float(x)))

@@ -40,6 +40,7 @@ constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the w
                                          // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
 constexpr int kStatusInts = 64;  // status word, clock / profile counters, grid-barrier counters; stream-K flags follow
+constexpr int kMaxGroups = 4096;  // row groups of a grouped GEMM (the handle's device table holds 2 x (kMaxGroups + 1) ints)
 
 // Key of the tuner's table: everything that changes which configuration is best.
 typedef std::tuple<int, int, int, int, long long, long long, long long, long long> TuneKey;
@@ -59,6 +60,8 @@ struct Problem {
   long long ldc, strideC;
   fact_out_t out;
   fact_epilogue_t epi;
+  int groups = 0;                        // > 0: grouped GEMM, A and C rows in consecutive groups, B = W[group]
+  const int64_t* group_rows = nullptr;   // host: rows of each group
   bool fp8 = false;    // operands are FP8 E4M3 (one byte per element) instead of BF16
   float alpha = 1.f;   // FP8: the accumulator is multiplied by this before the epilogue
   long long Nw() const { return epi == FACT_EPI_SILU_GATE ? 2 * N_out : N_out; }
@@ -88,6 +91,7 @@ struct fact_handle_s {
   unsigned configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
+  int* d_groups = nullptr;       // grouped GEMM: m-tile prefix and row offsets of the call in flight
   int* sk_flags() const { return d_status + kStatusInts; }  // stream-K flags: [SM][epilogue warp], 0 between launches
   size_t status_ints() const { return (size_t)kStatusInts + (size_t)sm_count * kEpiWarps; }
 };
@@ -462,11 +466,14 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
   return FACT_OK;
 }
 
-template <int CG, int EPI, bool SK = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false>
 fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                               cudaStream_t stream) {
-  auto kern = fact_gemm_kernel<CG, EPI, SK>;
-  if (!(h->configured_mask & (1u << slot))) {
+  auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED>;
+  if (slot < 0) {  // (no bit left in the handle's mask for these instantiations: set the attribute on every launch)
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+  } else if (!(h->configured_mask & (1u << slot))) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
     h->configured_mask |= (1u << slot);
@@ -522,6 +529,20 @@ fact_status_t launch_epi_sk(fact_handle_t h, int epi, const Plan& plan, const CU
   }
 }
 
+// The grouped instantiations (direct stores, data-parallel tiles).
+template <int CG>
+fact_status_t launch_epi_grouped(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  switch (epi) {
+    case kEpiNone: return launch_instance<CG, kEpiNone, false, true>(h, -1, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias, false, true>(h, -1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, true>(h, -1, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, true>(h, -1, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, true>(h, -1, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, true>(h, -1, plan, tm, stream);
+    default: return FACT_ERR_INVALID_ARG;
+  }
+}
+
 fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan, int splits, const float* ws,
                             cudaStream_t stream) {
   ReduceParams r;
@@ -566,6 +587,38 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
   if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
   if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
 
+  std::vector<int> group_table;
+  if (q.groups > 0) {
+    // Grouped: tiles never cross a group boundary (a group's last m-tile is ragged), every tile is data-parallel and
+    // stored by the row-predicated direct path.  The table -- m-tiles before each group, first row of each group --
+    // goes to the handle's device buffer in stream order.
+    fact_config_t gc = plan.cfg;
+    gc.split_k = 1;
+    gc.store_mode = 1;
+    st = make_plan(h, q, &gc, 0, &plan);
+    if (st != FACT_OK) return st;
+    const int G = q.groups;
+    group_table.resize(2 * (size_t)(G + 1));
+    long long tiles = 0, rows = 0;
+    for (int g = 0; g < G; ++g) {
+      group_table[g] = (int)tiles;
+      group_table[G + 1 + g] = (int)rows;
+      tiles += (q.group_rows[g] + plan.cfg.tile_m - 1) / plan.cfg.tile_m;
+      rows += q.group_rows[g];
+    }
+    group_table[G] = (int)tiles;
+    group_table[2 * G + 1] = (int)rows;
+    const long long units = tiles * plan.p.tiles_n;
+    if (units > 0x7fffffffLL) return FACT_ERR_UNSUPPORTED;
+    plan.p.groups = G;
+    plan.p.grp_tiles = h->d_groups;
+    plan.p.grp_rows = h->d_groups + (G + 1);
+    plan.p.total_units = (int)units;
+    plan.p.strideC = 0;
+    plan.p.strideR = 0;
+    plan.grid = (int)std::min<long long>(std::max(1, h->sm_count / plan.cfg.cta_group), std::max<long long>(units, 1)) *
+                plan.cfg.cta_group;
+  }
   if (plan.cfg.split_k < 0 && (!ws || ws_bytes < plan.ws_bytes) && !user) {
     // a tuned stream-K entry, but this caller brought no scratch: run the tiles data-parallel
     fact_config_t dp = plan.cfg;
@@ -598,18 +651,25 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     CUtensorMap& tmB = tm[1];
     memset(tm, 0, sizeof tm);
     const uint64_t batch_dim = (uint64_t)q.batch;
+    const uint64_t b_batch_dim = q.groups > 0 ? (uint64_t)q.groups : batch_dim;  // grouped: B is W[group]
+    const bool b_strided = q.batch > 1 || q.groups > 0;
+    if (q.groups > 0) {
+      cudaError_t e = cudaMemcpyAsync(h->d_groups, group_table.data(), group_table.size() * sizeof(int),
+                                      cudaMemcpyHostToDevice, stream);  // pageable source: staged before it returns
+      if (e != cudaSuccess) return cuda_fail(h, "cudaMemcpyAsync(group table)", e);
+    }
     const uint64_t sA = q.batch > 1 ? (uint64_t)q.strideA : (uint64_t)q.lda * (uint64_t)q.M;
     const uint32_t kbox = (uint32_t)q.k_elems();  // 128 bytes of K
     st = encode_map(h, &tmA, q.A, (uint64_t)q.K, (uint64_t)q.M, batch_dim, (uint64_t)q.lda, std::max<uint64_t>(sA, 16),
                     kbox, kTileM, false, q.fp8);
     if (st != FACT_OK) return st;
     if (q.layout == FACT_B_KN) {
-      const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.K;
-      st = encode_map(h, &tmB, q.B, (uint64_t)q.Nw(), (uint64_t)q.K, batch_dim, (uint64_t)q.ldb,
+      const uint64_t sB = b_strided ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.K;
+      st = encode_map(h, &tmB, q.B, (uint64_t)q.Nw(), (uint64_t)q.K, b_batch_dim, (uint64_t)q.ldb,
                       std::max<uint64_t>(sB, 8), 64, kTileK);
     } else {
-      const uint64_t sB = q.batch > 1 ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.Nw();
-      st = encode_map(h, &tmB, q.B, (uint64_t)q.K, (uint64_t)q.Nw(), batch_dim, (uint64_t)q.ldb,
+      const uint64_t sB = b_strided ? (uint64_t)q.strideB : (uint64_t)q.ldb * (uint64_t)q.Nw();
+      st = encode_map(h, &tmB, q.B, (uint64_t)q.K, (uint64_t)q.Nw(), b_batch_dim, (uint64_t)q.ldb,
                       std::max<uint64_t>(sB, 16), kbox, (uint32_t)plan.p.b_box_n, false, q.fp8);
     }
     if (st != FACT_OK) return st;
@@ -633,8 +693,10 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       }
     }
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
-    if (stream_k) st = plan.cfg.cta_group == 2 ? launch_epi_sk<2>(h, epi, plan, tm, stream)
-                                               : launch_epi_sk<1>(h, epi, plan, tm, stream);
+    if (q.groups > 0) st = plan.cfg.cta_group == 2 ? launch_epi_grouped<2>(h, epi, plan, tm, stream)
+                                                   : launch_epi_grouped<1>(h, epi, plan, tm, stream);
+    else if (stream_k) st = plan.cfg.cta_group == 2 ? launch_epi_sk<2>(h, epi, plan, tm, stream)
+                                                    : launch_epi_sk<1>(h, epi, plan, tm, stream);
     else if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
     else st = launch_epi<1>(h, epi, plan, tm, stream);
     if (st == FACT_OK && split && !plan.p.fused_reduce)
@@ -725,12 +787,18 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
     delete h;
     return FACT_ERR_CUDA;
   }
+  if (cudaMalloc(&h->d_groups, 2 * (kMaxGroups + 1) * sizeof(int)) != cudaSuccess) {
+    cudaFree(h->d_status);
+    delete h;
+    return FACT_ERR_CUDA;
+  }
   *handle = h;
   return FACT_OK;
 }
 
 fact_status_t fact_destroy(fact_handle_t h) {
   if (!h) return FACT_OK;
+  if (h->d_groups) cudaFree(h->d_groups);
   if (h->d_status) cudaFree(h->d_status);
   delete h;
   return FACT_OK;
@@ -882,6 +950,30 @@ fact_status_t fact_linear(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, 
   Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, 0, layout, bias, residual, ldr, 0, Y,
                            ldy, 0, out, epi);
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_linear_grouped(fact_handle_t h, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
+                                  const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
+                                  fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, void* Y,
+                                  int64_t ldy, fact_out_t out, fact_epilogue_t epi, const fact_config_t* cfg,
+                                  void* stream) {
+  if (!h || groups < 0 || groups > kMaxGroups || (groups > 0 && !group_rows) || strideW < 0) return FACT_ERR_INVALID_ARG;
+  long long M = 0;
+  for (int g = 0; g < groups; ++g) {
+    if (group_rows[g] < 0) return FACT_ERR_INVALID_ARG;
+    M += group_rows[g];
+    if (M > 0x7fffffffLL - 512) return FACT_ERR_INVALID_ARG;
+  }
+  if (groups == 0 || M == 0) return FACT_OK;
+  if (cfg && (cfg->split_k > 1 || cfg->split_k < 0 || cfg->store_mode == 2)) return FACT_ERR_UNSUPPORTED;
+  Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, strideW, layout, bias, residual, ldr, 0, Y,
+                           ldy, 0, out, epi);
+  q.groups = groups;
+  q.group_rows = group_rows;
+  if (strideW % q.op_align()) return FACT_ERR_BAD_ALIGNMENT;
+  const long long w_rows = layout == FACT_B_KN ? K : q.Nw();
+  if (groups > 1 && K > 0 && strideW < w_rows * ldw) return FACT_ERR_INVALID_ARG;  // the groups' weights overlap
+  return run(h, q, cfg, 0, nullptr, 0, stream);
 }
 
 fact_status_t fact_linear_fp8(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,

@@ -105,6 +105,11 @@ struct GemmParams {
   int fused_reduce;   // 1: after a grid-wide barrier every CTA reduces its share of the output (split-K only)
   int reduce_epi;     // the epilogue the reduction applies
   int* status;        // [0] error word, [2..17] clock / profile counters, [24], [25] grid-barrier counters
+  // grouped GEMM (the GROUPED instantiations only): the rows of A and C are cut into `groups` consecutive row
+  // groups, group g multiplies W[g]; see decode_grouped
+  int groups;
+  const int* grp_tiles;   // [groups + 1] m-tiles (of tile_m rows) before each group
+  const int* grp_rows;    // [groups + 1] first row of each group; grp_rows[groups] = M
   // 8-bit operands (FP8 E4M3, one byte per element): a k-block is 128 elements, still 128 bytes per row
   int k_elems;        // elements of K per k-block: 64 (BF16) or 128 (FP8)
   int fp8;            // 1: tcgen05.mma.kind::f8f6f4, else kind::f16
@@ -124,6 +129,8 @@ struct GemmParams {
 
 struct WorkUnit {
   int b, tm, tn, kb_begin, kb_end, split;
+  int m_base;    // grouped: first row of the unit's group (0 otherwise; rows are m_base + tm * tile_m + ...)
+  int m_end;     // grouped: one past the last row of the group (M otherwise)
   int wave;      // ordinal of this data-parallel unit within its CTA (0 for stream-K pieces)
   int sk_role;   // 0: a whole tile; 1: the piece with the tile's first k-block (it finishes the tile); 2: a later piece
   int sk_peers;  // role 1: how many following CTA groups hold the tile's other pieces
@@ -169,6 +176,28 @@ __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
   return w;
 }
 
+// Grouped GEMM: unit u = (global m-tile, n-tile), n-tiles fastest, so that neighbouring CTAs share a slab of A rows
+// and one group's weights.  The group of an m-tile is found by bisection in the prefix table.
+__device__ __forceinline__ WorkUnit decode_grouped(const GemmParams& p, int u) {
+  WorkUnit w;
+  const int mt = u / p.tiles_n;
+  w.tn = u - mt * p.tiles_n;
+  int lo = 0, hi = p.groups;  // invariant: grp_tiles[lo] <= mt < grp_tiles[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(p.grp_tiles + mid) <= mt) lo = mid;
+    else hi = mid;
+  }
+  w.b = lo;
+  w.tm = mt - __ldg(p.grp_tiles + lo);
+  w.m_base = __ldg(p.grp_rows + lo);
+  w.m_end = __ldg(p.grp_rows + lo + 1);
+  w.split = 0;
+  w.kb_begin = 0;
+  w.kb_end = p.k_blocks;
+  return w;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Stream-K partition (host and device share this arithmetic).  The k-block iterations of the stream-K tiles are
 // numbered tile by tile, `k_blocks` per tile, and dealt out in contiguous runs: group c owns
@@ -208,7 +237,7 @@ __host__ __device__ inline SkPiece sk_next_piece(int k_blocks, int len, int rem,
 // A tile's pieces belong to consecutive groups; the group with the first k-block adds the others' FP32
 // partials (in group order) to its own accumulator and applies the epilogue.  Those others meet that piece first
 // of all their work and depend on nobody, so the wait for them cannot be circular.
-template <bool SK>
+template <bool SK, bool GROUPED = false>
 struct UnitWalk {
   int u, stride, wave;
   int sk_pos, sk_end, group;
@@ -224,6 +253,8 @@ struct UnitWalk {
       if (sk_pos < sk_end) {
         const SkPiece pc = sk_next_piece(p.k_blocks, p.sk_len, p.sk_rem, stride, group, sk_pos, sk_end);
         w = decode_unit(p, p.sk_first + pc.tile);
+        w.m_base = 0;
+        w.m_end = p.M;
         w.kb_begin = pc.k0;
         w.kb_end = pc.k1;
         w.wave = 0;
@@ -233,7 +264,13 @@ struct UnitWalk {
       }
     }
     if (u >= p.total_units) return false;
-    w = decode_unit(p, u);
+    if constexpr (GROUPED) {
+      w = decode_grouped(p, u);
+    } else {
+      w = decode_unit(p, u);
+      w.m_base = 0;
+      w.m_end = p.M;
+    }
     w.wave = wave++;
     w.sk_role = 0;
     w.sk_peers = 0;
@@ -528,7 +565,7 @@ __device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uin
   }
 }
 
-template <int CG, int EPI, bool SK = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
@@ -548,6 +585,13 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (smem_base & 1023u) {  // the swizzled tiles need a 1024-byte aligned ring: refuse to run otherwise
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
+  }
+  if constexpr (GROUPED) {  // group boundaries are kept by the row-predicated direct stores only
+    static_assert(!SK && EPI != kEpiPartial, "grouped tiles are data-parallel");
+    if (p.store_tma || p.grp_tiles == nullptr || p.grp_rows == nullptr) {
+      if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+      return;
+    }
   }
   if constexpr (SK) {  // stream-K pieces are parked and finished by the staged epilogue only: refuse anything else
     if (!p.store_tma || p.sk_ws == nullptr || p.sk_flags == nullptr) {
@@ -621,14 +665,15 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      UnitWalk<SK> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         // Odd waves walk K downwards: the wave before ended at the top of K, so the operand slabs both waves
         // share (same m-tiles of A, or same n-tiles of B) are met while they are still in L2.  The sum of an
         // output element is then taken in descending k in those tiles, still fixed by (shape, config).
         const bool k_down = (w.wave & 1) && p.k_serpentine;
-        const int m0 = (w.tm * CG + (int)cta_rank) * kTileM;
+        const int m0 = (GROUPED ? w.m_base : 0) + (w.tm * CG + (int)cta_rank) * kTileM;
+        const int a_batch = GROUPED ? 0 : w.b;  // grouped: A is one matrix, the group selects the weights only
         // first accumulator column this CTA's B boxes feed, and the W column of every box
         const int col0 = (CG == 2) ? (int)cta_rank * (p.tile_n / 2) : 0;
         int n_box[4];
@@ -656,10 +701,10 @@ __global__ void __launch_bounds__(kThreads, 1)
               if constexpr (CG == 2) {
                 if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
                 fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
-                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * p.k_elems, m0, w.b);
+                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * p.k_elems, m0, a_batch);
               } else {
                 ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-                ptx::tma_load_3d(sa, &tmA, fb, kb * p.k_elems, m0, w.b);
+                ptx::tma_load_3d(sa, &tmA, fb, kb * p.k_elems, m0, a_batch);
               }
             } else {
               if constexpr (CG == 2) fb = ptx::mapa(fb, 0);
@@ -704,7 +749,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t acc_phase = 0;
       bool ok = true;
       long long prof_acc_wait = 0, prof_full_wait = 0, prof_first_full = 0;
-      UnitWalk<SK> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         long long t0 = prof ? clock64() : 0;
@@ -798,7 +843,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       long long prof_epi_busy = 0, prof_epi_wait = 0, prof_tiles = 0;
       uint32_t gc = 0;      // chunks this warp has stored so far: buffer = gc % bufs
       uint32_t r_next = 0;  // residual loads have been issued for every chunk counter below this
-      UnitWalk<SK> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
       WorkUnit w;
       // hand the accumulator back to the MMA issuer (of the leader CTA) and move on to the other one
       // (a relaxed arrival: the barrier orders tensor-memory reads only, which the tcgen05 fences take care of; a
@@ -1095,7 +1140,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else {
       // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
       const bool c_vec = p.c_vec != 0;
-      UnitWalk<false> walk(p, unit0, unit_stride);  // (stream-K always stores through the staged path)
+      UnitWalk<false, GROUPED> walk(p, unit0, unit_stride);  // (stream-K always stores through the staged path)
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
@@ -1103,14 +1148,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           break;
         }
         ptx::tc_fence_after();
-        const int row = (w.tm * CG + (int)cta_rank) * kTileM + q * 32 + lane;
-        const bool row_ok = row < p.M;
+        const int row = (GROUPED ? w.m_base : 0) + (w.tm * CG + (int)cta_rank) * kTileM + q * 32 + lane;
+        const bool row_ok = row < (GROUPED ? w.m_end : p.M);
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
         const int n_tile0 = w.tn * p.out_cols;
-        const long long off = (long long)w.b * p.strideC + (long long)row * p.ldc;
+        const long long off = (GROUPED ? 0LL : (long long)w.b * p.strideC) + (long long)row * p.ldc;
         char* c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
         const __nv_bfloat16* r_row = nullptr;
-        if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
+        if constexpr (EPI == kEpiBiasResidual)
+          r_row = p.R + (GROUPED ? 0LL : (long long)w.b * p.strideR) + (long long)row * p.ldr;
         for (int c = half * 32; c < p.out_cols; c += 64) {  // the two warps of a quarter alternate 32-column pieces
           const int n0 = n_tile0 + c;
           if (n0 >= p.N_out) break;  // uniform across the warp

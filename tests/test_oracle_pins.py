@@ -286,3 +286,27 @@ def test_rejects_bad_arguments():
     with pytest.raises(ValueError):
         oracle.linear(x, w, rows=np.array([2]))  # row out of range
     assert oracle.linear(x[:0], w).shape == (0, 6)
+
+
+def test_linear_grouped_is_the_per_group_product():
+    """oracle.linear_grouped against numpy's FP64 matmul group by group (a library routine), with empty groups, and
+    against oracle.linear when there is one group."""
+    rng = np.random.default_rng(11)
+    rows = [5, 0, 17, 1, 0, 9]
+    M, N, K = sum(rows), 12, 40
+    X = rng.integers(0x3C00, 0x4100, size=(M, K)).astype(np.uint16) | (rng.integers(0, 2, size=(M, K)).astype(np.uint16) << 15)
+    W = rng.integers(0x3C00, 0x4100, size=(len(rows), N, K)).astype(np.uint16)
+    bias = rng.integers(0x3C00, 0x4000, size=(N,)).astype(np.uint16)
+    got = oracle.linear_grouped(X, W, rows, layout="NK", epilogue="BIAS", bias=bias)
+    xf, wf, bf = oracle.bf16_to_f64(X), oracle.bf16_to_f64(W), oracle.bf16_to_f64(bias)
+    r0 = 0
+    for g, n in enumerate(rows):
+        ref = xf[r0:r0 + n] @ wf[g].T + bf
+        assert np.allclose(got[r0:r0 + n], ref, rtol=1e-13, atol=0)
+        r0 += n
+    one = oracle.linear_grouped(X, W[:1], [M], layout="NK")
+    assert np.array_equal(one, oracle.linear(X, W[0], layout="NK"))
+    kn = oracle.linear_grouped(X, np.ascontiguousarray(W.transpose(0, 2, 1)), rows, layout="KN", epilogue="BIAS", bias=bias)
+    assert np.array_equal(kn, got)
+    with pytest.raises(ValueError):
+        oracle.linear_grouped(X, W, rows[:-1], layout="NK")
