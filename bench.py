@@ -194,7 +194,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8` or `blocks`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped` or `blocks`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
@@ -236,12 +236,12 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        rows = [] if args.shape in ("attention", "blocks", "fp8") else per_shape_table(
+        rows = [] if args.shape in ("attention", "blocks", "fp8", "grouped") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
             side_ref=False, layout=args.layout)
         if args.shape in ("all", "attention"):
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
-        elif args.shape in ("blocks", "fp8"):
+        elif args.shape in ("blocks", "fp8", "grouped"):
             att = []
         else:  # attention shapes can be named like the GEMM shapes
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
@@ -255,10 +255,15 @@ def main():
         if args.shape in ("all", "fp8"):
             f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps,
                            side_ref=args.shape == "all")
-        elif names is not None:  # FP8 shapes can be named like the GEMM shapes
+        elif names is not None and args.shape != "grouped":  # FP8 shapes can be named like the GEMM shapes
             f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
                            names=names)
-        print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "fp8": f8, "gpu_launches": h.launch_count()}))
+        grp = []
+        if args.shape in ("all", "grouped"):
+            grp = grouped_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps,
+                                side_ref=args.shape == "all")
+        print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "fp8": f8, "grouped": grp,
+                          "gpu_launches": h.launch_count()}))
         h.close()
         return 0
 
@@ -347,10 +352,11 @@ def main():
     shapes = []
     if not args.no_shapes and rank == 0:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
-    attention, blocks, fp8 = [], [], []
+    attention, blocks, fp8, grouped = [], [], [], []
     if not args.no_shapes and rank == 0:
         attention = attention_table(h, dev, stream, flush_l2, peaks)
         fp8 = fp8_table(h, dev, stream, flush_l2, peaks)
+        grouped = grouped_table(h, dev, stream, flush_l2, peaks)
         blocks = block_table(h, dev, stream, flush_l2, peaks)
     clocks = sampler.stop()  # sampled from the first warm-up step to the end of the per-shape table
 
@@ -387,6 +393,7 @@ def main():
             "shapes": shapes,
             "attention": attention,
             "fp8": fp8,
+            "grouped": grouped,
             "blocks": blocks,
         }
         print(json.dumps(line))
@@ -588,6 +595,66 @@ def fp8_table(h, dev, stream, flush_l2, peaks, warm=5, iters=20, side_ref=True, 
         assert h.device_status() == 0
         del X, W, out
     return rows
+
+
+def grouped_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=True, names=None):
+    """Time fact_linear_grouped on mixture-of-experts-shaped problems (uneven, seeded group sizes), L2 overwritten
+    between launches; a loop of torch.matmul calls, one per group (cuBLAS, matmul only), is a side reference."""
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    rows_out = []
+    for case in wl.grouped_cases():
+        if names is not None and case.name not in names:
+            continue
+        rows = wl.grouped_rows(case)
+        X, W = wl.make_grouped_inputs(case, dev)
+        out = torch.empty((case.tokens, case.N), dtype=torch.bfloat16, device=dev)
+        offs = [0]
+        for r in rows:
+            offs.append(offs[-1] + r)
+
+        def call():
+            h.linear_grouped(X, W, rows, epilogue=case.epilogue, out=out)
+
+        def side():
+            for g in range(case.groups):
+                torch.matmul(X[offs[g]:offs[g + 1]], W[g].t())
+
+        def time_it(fn, n):
+            for _ in range(warm):
+                fn()
+            ts = []
+            for _ in range(n):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                ts.append((a, b))
+            torch.cuda.synchronize(dev)
+            return sorted(x.elapsed_time(y) for x, y in ts)
+
+        t = time_it(call, iters)
+        med = t[len(t) // 2]
+        try:
+            ts = time_it(side, 5) if side_ref else [0.0]
+        except Exception:  # the side reference is optional
+            ts = [float("nan")]
+        t_tensor = case.flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        rows_out.append({
+            "name": case.name, "tokens": case.tokens, "groups": case.groups, "N": case.N, "K": case.K,
+            "epilogue": case.epilogue, "rows_min": min(rows), "rows_max": max(rows),
+            "us_median": med * 1e3, "us_min": t[0] * 1e3, "tflops": case.flops / (med * 1e-3) / 1e12,
+            "gbs": case.algorithmic_bytes / (med * 1e-3) / 1e9, "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+            "roofline_us": max(t_tensor, t_hbm) * 1e3, "roofline_frac": max(t_tensor, t_hbm) / med,
+            "torch_matmul_loop_only_us": ts[len(ts) // 2] * 1e3,
+        })
+        assert h.device_status() == 0
+        del X, W, out
+    return rows_out
 
 
 def block_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=True):

@@ -610,6 +610,9 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     group_table[2 * G + 1] = (int)rows;
     const long long units = tiles * plan.p.tiles_n;
     if (units > 0x7fffffffLL) return FACT_ERR_UNSUPPORTED;
+    // slabs of m-tiles whose rows of A fit a 32 MB share of L2
+    plan.p.raster_group = (int)std::max<long long>(
+        1, (32LL << 20) / ((long long)plan.cfg.tile_m * std::max<long long>(q.K, 1) * (q.fp8 ? 1 : 2)));
     plan.p.groups = G;
     plan.p.grp_tiles = h->d_groups;
     plan.p.grp_rows = h->d_groups + (G + 1);

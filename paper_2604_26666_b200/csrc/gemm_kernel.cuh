@@ -176,20 +176,29 @@ __device__ __forceinline__ WorkUnit decode_unit(const GemmParams& p, int u) {
   return w;
 }
 
-// Grouped GEMM: unit u = (global m-tile, n-tile), n-tiles fastest, so that neighbouring CTAs share a slab of A rows
-// and one group's weights.  The group of an m-tile is found by bisection in the prefix table.
+// Grouped GEMM: units are numbered group by group, tiles_n per m-tile.  The group of a unit is found by bisection in
+// the prefix table of m-tiles.  Inside a group the walk takes slabs of `raster_group` m-tiles (their rows of A stay
+// in L2) and, within a slab, the m-tiles fastest: CTAs that run at the same time then share the group's weight
+// columns, which are streamed once per slab.
 __device__ __forceinline__ WorkUnit decode_grouped(const GemmParams& p, int u) {
   WorkUnit w;
   const int mt = u / p.tiles_n;
-  w.tn = u - mt * p.tiles_n;
   int lo = 0, hi = p.groups;  // invariant: grp_tiles[lo] <= mt < grp_tiles[hi]
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (__ldg(p.grp_tiles + mid) <= mt) lo = mid;
     else hi = mid;
   }
+  const int first = __ldg(p.grp_tiles + lo);
+  const int mtiles = __ldg(p.grp_tiles + lo + 1) - first;  // m-tiles of this group (> 0: empty groups own no unit)
+  const int local = u - first * p.tiles_n;
+  const int per_slab = p.raster_group * p.tiles_n;
+  const int slab = local / per_slab;
+  const int rem = local - slab * per_slab;
+  const int height = min(p.raster_group, mtiles - slab * p.raster_group);
+  w.tn = rem / height;
+  w.tm = slab * p.raster_group + (rem - w.tn * height);
   w.b = lo;
-  w.tm = mt - __ldg(p.grp_tiles + lo);
   w.m_base = __ldg(p.grp_rows + lo);
   w.m_end = __ldg(p.grp_rows + lo + 1);
   w.split = 0;

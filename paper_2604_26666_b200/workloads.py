@@ -352,3 +352,56 @@ def make_fp8_inputs(case: Fp8Case) -> Fp8Inputs:
     xq = (x * sx).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
     wq = (w * sw).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
     return Fp8Inputs(xq, wq, 1.0 / (sx * sw), bias)
+
+
+# ---------------------------------------------------------------------------------------------
+# Grouped linear layers ("Grouped GEMM" in the paper's Table 1): the paper gives no shapes; these are the expert
+# projections of a mixture-of-experts layer with the Llama-shaped hidden sizes of configuration 5.
+@dataclass(frozen=True)
+class GroupedCase:
+    name: str
+    tokens: int
+    groups: int
+    N: int
+    K: int
+    epilogue: str = "NONE"
+    seed: int = 0
+
+    @property
+    def n_weight_cols(self) -> int:
+        return 2 * self.N if self.epilogue == "SILU_GATE" else self.N
+
+    @property
+    def flops(self) -> float:
+        return 2.0 * self.tokens * self.n_weight_cols * self.K
+
+    @property
+    def algorithmic_bytes(self) -> float:
+        return 2.0 * (self.tokens * self.K + self.groups * self.n_weight_cols * self.K + self.tokens * self.N)
+
+
+def grouped_cases() -> list[GroupedCase]:
+    return [
+        GroupedCase("g8_moe_up_silu", 16384, 8, 14336, 4096, epilogue="SILU_GATE", seed=7300),
+        GroupedCase("g8_moe_down", 16384, 8, 4096, 14336, seed=7301),
+        GroupedCase("g64_small_experts", 16384, 64, 2048, 2048, seed=7302),
+    ]
+
+
+def grouped_rows(case: GroupedCase) -> list[int]:
+    """Rows per group: every token picks a group uniformly at random (seeded), as a router without load balancing
+    would: the counts are uneven and none is a multiple of the tile height."""
+    g = torch.Generator(device="cpu").manual_seed(case.seed)
+    pick = torch.randint(0, case.groups, (case.tokens,), generator=g)
+    return torch.bincount(pick, minlength=case.groups).tolist()
+
+
+def make_grouped_inputs(case: GroupedCase, device="cpu"):
+    """X ~ N(0,1) [tokens, K], W ~ N(0, 0.02^2) [groups, Nw, K], BF16; drawn on the device when one is given (the
+    weights alone are up to 1.9 GB)."""
+    g = torch.Generator(device=device).manual_seed(case.seed + 1)
+    X = torch.randn((case.tokens, case.K), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    W = torch.empty((case.groups, case.n_weight_cols, case.K), dtype=torch.bfloat16, device=device)
+    for i in range(case.groups):
+        W[i] = (torch.randn((case.n_weight_cols, case.K), generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    return X, W
