@@ -243,6 +243,15 @@ fact_status_t fact_linear_grouped(fact_handle_t handle, int groups, const int64_
                                   int64_t ldy, fact_out_t out_type, fact_epilogue_t epilogue, const fact_config_t* cfg,
                                   void* cuda_stream);
 
+/* The grouped linear layer on FP8 E4M3 operands (Table 1: "FP8 Grouped GEMM"): fact_linear_grouped with the
+ * operand rules of fact_linear_fp8 -- X [M x K] and W[g] [Nw x K] one byte per element, K-major, ldx, ldw and
+ * strideW multiples of 16, one FP32 `scale` for all groups applied to the accumulator before the epilogue. */
+fact_status_t fact_linear_grouped_fp8(fact_handle_t handle, int groups, const int64_t* group_rows, int64_t N_out,
+                                      int64_t K, const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                      int64_t strideW, float scale, const void* bias, const void* residual, int64_t ldr,
+                                      void* Y, int64_t ldy, fact_out_t out_type, fact_epilogue_t epilogue,
+                                      const fact_config_t* cfg, void* cuda_stream);
+
 /* Y[M x N_out] = epilogue(scale * X[M x K] . W^T)  with FP8 operands      (Section 3, the pattern table indexed by
  * rule, data type and architecture; Table 1 lists an FP8 GEMM among the Level-1 kernels the registry holds)
  * X: FP8 E4M3 [M x K], one byte per element (the OCP "e4m3fn" format: no infinities, S.1111.111 is NaN, largest

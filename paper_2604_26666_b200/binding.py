@@ -37,7 +37,7 @@ EXPORTED = [
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
-    "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped",
+    "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
 ]
 
 
@@ -125,6 +125,8 @@ def lib() -> ctypes.CDLL:
                                   vp, sz, vp]
     L.fact_linear_grouped.argtypes = [vp, c_int, POINTER(i64), i64, i64, vp, i64, vp, i64, i64, c_int, vp, vp, i64, vp, i64,
                                       c_int, c_int, cfgp, vp]
+    L.fact_linear_grouped_fp8.argtypes = [vp, c_int, POINTER(i64), i64, i64, vp, i64, vp, i64, i64, c_float, vp, vp, i64, vp,
+                                          i64, c_int, c_int, cfgp, vp]
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     for name in EXPORTED:
         fn = getattr(L, name)
@@ -422,6 +424,35 @@ class Handle:
                                          _ptr(bias), _ptr(residual), _ld(residual) if residual is not None else 0,
                                          _ptr(out), _ld(out), OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg),
                                          self._stream(stream)), "fact_linear_grouped", self._h)
+        return out
+
+    def linear_grouped_fp8(self, X, W, group_rows, scale=1.0, bias=None, epilogue="NONE", out=None,
+                           out_dtype=torch.bfloat16, cfg=None, stream=None):
+        """fact_linear_grouped_fp8: X [M, K] and W [G, Nw, K] are FP8 E4M3 (torch.float8_e4m3fn or uint8 codes)."""
+        def codes(t, name, nd):
+            if isinstance(t, torch.Tensor) and t.dtype == torch.float8_e4m3fn:
+                t = t.view(torch.uint8)
+            _need(t, name, torch.uint8, nd)
+            return t
+        X, W = codes(X, "X", 2), codes(W, "W", 3)
+        rows = [int(r) for r in group_rows]
+        G = len(rows)
+        M, K = X.shape
+        if W.shape[0] != G or sum(rows) != M or W.shape[2] != K:
+            raise ValueError("shapes differ")
+        Nw = W.shape[1]
+        N = Nw // 2 if epilogue == "SILU_GATE" else Nw
+        if bias is not None:
+            _need(bias, "bias", torch.bfloat16, 1)
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype, device=X.device)
+        _need(out, "out", out.dtype, 2)
+        arr = (c_int64 * max(G, 1))(*rows)
+        _check(lib().fact_linear_grouped_fp8(self._h, G, arr, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W),
+                                             int(W.stride(0)) if G > 1 else int(W.shape[1] * W.stride(1)), float(scale),
+                                             _ptr(bias), None, 0, _ptr(out), _ld(out), OUT_TYPES[out.dtype],
+                                             EPILOGUES[epilogue], self._cfg(cfg), self._stream(stream)),
+               "fact_linear_grouped_fp8", self._h)
         return out
 
     def linear_fp8(self, X, W, scale=1.0, bias=None, residual=None, epilogue="NONE", out=None,

@@ -955,12 +955,13 @@ fact_status_t fact_linear(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, 
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
 }
 
-fact_status_t fact_linear_grouped(fact_handle_t h, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
-                                  const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
-                                  fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, void* Y,
-                                  int64_t ldy, fact_out_t out, fact_epilogue_t epi, const fact_config_t* cfg,
-                                  void* stream) {
+static fact_status_t linear_grouped_impl(fact_handle_t h, bool fp8, float scale, int groups, const int64_t* group_rows,
+                                         int64_t N_out, int64_t K, const void* X, int64_t ldx, const void* W,
+                                         int64_t ldw, int64_t strideW, fact_blayout_t layout, const void* bias,
+                                         const void* residual, int64_t ldr, void* Y, int64_t ldy, fact_out_t out,
+                                         fact_epilogue_t epi, const fact_config_t* cfg, void* stream) {
   if (!h || groups < 0 || groups > kMaxGroups || (groups > 0 && !group_rows) || strideW < 0) return FACT_ERR_INVALID_ARG;
+  if (!(scale == scale) || std::isinf(scale)) return FACT_ERR_INVALID_ARG;
   long long M = 0;
   for (int g = 0; g < groups; ++g) {
     if (group_rows[g] < 0) return FACT_ERR_INVALID_ARG;
@@ -969,14 +970,33 @@ fact_status_t fact_linear_grouped(fact_handle_t h, int groups, const int64_t* gr
   }
   if (groups == 0 || M == 0) return FACT_OK;
   if (cfg && (cfg->split_k > 1 || cfg->split_k < 0 || cfg->store_mode == 2)) return FACT_ERR_UNSUPPORTED;
-  Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, strideW, layout, bias, residual, ldr, 0, Y,
-                           ldy, 0, out, epi);
+  Problem q = make_problem(fp8 ? FACT_OP_LINEAR_FP8 : FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, strideW, layout,
+                           bias, residual, ldr, 0, Y, ldy, 0, out, epi);
   q.groups = groups;
   q.group_rows = group_rows;
+  q.alpha = scale;
   if (strideW % q.op_align()) return FACT_ERR_BAD_ALIGNMENT;
   const long long w_rows = layout == FACT_B_KN ? K : q.Nw();
   if (groups > 1 && K > 0 && strideW < w_rows * ldw) return FACT_ERR_INVALID_ARG;  // the groups' weights overlap
   return run(h, q, cfg, 0, nullptr, 0, stream);
+}
+
+fact_status_t fact_linear_grouped(fact_handle_t h, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
+                                  const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
+                                  fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, void* Y,
+                                  int64_t ldy, fact_out_t out, fact_epilogue_t epi, const fact_config_t* cfg,
+                                  void* stream) {
+  return linear_grouped_impl(h, false, 1.f, groups, group_rows, N_out, K, X, ldx, W, ldw, strideW, layout, bias, residual,
+                             ldr, Y, ldy, out, epi, cfg, stream);
+}
+
+fact_status_t fact_linear_grouped_fp8(fact_handle_t h, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
+                                      const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
+                                      float scale, const void* bias, const void* residual, int64_t ldr, void* Y,
+                                      int64_t ldy, fact_out_t out, fact_epilogue_t epi, const fact_config_t* cfg,
+                                      void* stream) {
+  return linear_grouped_impl(h, true, scale, groups, group_rows, N_out, K, X, ldx, W, ldw, strideW, FACT_B_NK, bias,
+                             residual, ldr, Y, ldy, out, epi, cfg, stream);
 }
 
 fact_status_t fact_linear_fp8(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,

@@ -126,3 +126,37 @@ def test_grouped_argument_errors(h):
     assert call(2, [128, 128], cfg=ctypes.byref(Config(store_mode=2))) == 3
     torch.cuda.synchronize()
     assert h.device_status() == 0
+
+
+@pytest.mark.parametrize("epi,cfg", [("NONE", None), ("BIAS_GELU_TANH", dict(tile_n=128, cta_group=2)),
+                                     ("SILU_GATE", dict(tile_n=256, cta_group=1))])
+def test_grouped_fp8_matches_oracle(h, epi, cfg):
+    """FP8 E4M3 operands through the grouped path: the oracle is the FP8 linear oracle, group by group."""
+    from oracle import fp8 as ofp8
+
+    rows = [140, 0, 300, 1, 259]
+    M, N, K = sum(rows), 256, 400
+    Nw = 2 * N if epi == "SILU_GATE" else N
+    g = torch.Generator().manual_seed(41)
+    X = (torch.randn((M, K), generator=g) * 2).to(torch.float8_e4m3fn)
+    W = (torch.randn((len(rows), Nw, K), generator=g) * 0.5).to(torch.float8_e4m3fn)
+    bias = torch.randn((N,), generator=g).to(torch.bfloat16) if epi.startswith("BIAS") else None
+    scale = 0.05
+    out = h.linear_grouped_fp8(X.cuda(), W.cuda(), rows, scale, None if bias is None else bias.cuda(), epilogue=epi, cfg=cfg)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    xc, wc = X.view(torch.uint8).numpy(), W.view(torch.uint8).numpy()
+    ref = np.empty((M, N))
+    r0 = 0
+    for gi, n in enumerate(rows):
+        if n:
+            if epi == "SILU_GATE":
+                acc = ofp8.linear_fp8(xc[r0:r0 + n], wc[gi], scale)
+                gate, up = acc[:, :N], acc[:, N:]
+                ref[r0:r0 + n] = gate / (1.0 + np.exp(-gate)) * up
+            else:
+                ref[r0:r0 + n] = ofp8.linear_fp8(xc[r0:r0 + n], wc[gi], scale,
+                                                 None if bias is None else bias.double().numpy(), epi)
+        r0 += n
+    c, t = gates(ref, to_f64(out), "bf16", epi)
+    assert c <= 1.0 and t <= 1.0, (c, t)
