@@ -193,3 +193,28 @@ def test_error_codes(h):
     with pytest.raises(FactError) as e:
         h.attention(q, k, k, causal=True)
     assert e.value.code == 3  # causal with different lengths
+
+
+def _sweep_cases():
+    rng = np.random.default_rng(2024)
+    cases = []
+    for i in range(28):
+        D = int(rng.choice([64, 128]))
+        causal = bool(rng.integers(0, 2))
+        Hkv = int(rng.integers(1, 4))
+        Hq = Hkv * int(rng.choice([1, 2, 4]))
+        B = int(rng.integers(1, 4))
+        # lengths around the tile (128), item (256) and key-block (64 / 128) borders, and a few larger ones
+        pool = [1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 255, 256, 257, 320, 383, 384, 385, 511, 512, 600, 769]
+        Tq = int(rng.choice(pool))
+        Tk = Tq if causal else int(rng.choice(pool))
+        cases.append((i, B, Tq, Tk, Hq, Hkv, D, causal))
+    return cases
+
+
+@pytest.mark.parametrize("i,B,Tq,Tk,Hq,Hkv,D,causal", _sweep_cases(),
+                         ids=[f"{c[0]}-B{c[1]}-Tq{c[2]}-Tk{c[3]}-H{c[4]}/{c[5]}-D{c[6]}-{'c' if c[7] else 'f'}" for c in _sweep_cases()])
+def test_random_shapes(h, i, B, Tq, Tk, Hq, Hkv, D, causal):
+    """Seeded random shapes: lengths on and around every border the kernel has (tile of 128 query rows, item of two
+    tiles, key blocks of 64 or 128, a second tile wholly past the end), grouped queries, both head sizes."""
+    check(h, rnd((B, Tq, Hq, D), 500 + i), rnd((B, Tk, Hkv, D), 600 + i), rnd((B, Tk, Hkv, D), 700 + i), causal)
