@@ -73,14 +73,19 @@ typedef enum {
  *                   W carries 2*N_out columns: gate columns first, then up columns
  *                                                             (Section 5.2, Llama p2 GEMM 1)
  *   BIAS_RESIDUAL   y = acc + bias[n] + R[m, n]   (bias may be NULL)
- *                                                             (GEMM 2 of both blocks + the residual add) */
+ *                                                             (GEMM 2 of both blocks + the residual add)
+ *   BIAS_SOFTMAX    z = acc[m, :] + bias;  y[m, n] = exp(z[n] - max z) / sum_j exp(z[j] - max z)   (bias may be NULL)
+ *                   the softmax of every output row, inside the tile that holds the row: N_out <= 256, no K split,
+ *                   no stream-K, register stores (FACT_ERR_UNSUPPORTED otherwise)
+ *                                                             (Table 1: the "GEMM-Softmax" fusion) */
 typedef enum {
   FACT_EPI_NONE = 0,
   FACT_EPI_BIAS = 1,
   FACT_EPI_BIAS_RELU = 2,
   FACT_EPI_BIAS_GELU_TANH = 3,
   FACT_EPI_SILU_GATE = 4,
-  FACT_EPI_BIAS_RESIDUAL = 5
+  FACT_EPI_BIAS_RESIDUAL = 5,
+  FACT_EPI_BIAS_SOFTMAX = 6
 } fact_epilogue_t;
 
 typedef enum { FACT_OUT_BF16 = 0, FACT_OUT_F32 = 1 } fact_out_t;

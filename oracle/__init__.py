@@ -200,6 +200,16 @@ def linear(X, W, *, layout="KN", epilogue="NONE", bias=None, residual=None, rows
     return Y if batched else Y[0]
 
 
+def linear_softmax(X, W, *, layout="NK", bias=None, rows=None):
+    """The "GEMM-Softmax" fusion of the paper's Table 1, written out as its definition: ``Z = X @ W (+ bias)`` in
+    FP64 by ``linear``, then the softmax of every row, ``Y[m, n] = exp(Z[m, n] - max_j Z[m, j]) / sum_j exp(Z[m, j] -
+    max_j Z[m, j])`` (subtracting the row maximum changes nothing mathematically and keeps the exponentials finite)."""
+    Z = linear(X, W, layout=layout, epilogue="NONE" if bias is None else "BIAS", bias=bias, rows=rows)
+    Z = Z - Z.max(axis=-1, keepdims=True)
+    E = np.exp(Z)
+    return E / E.sum(axis=-1, keepdims=True)
+
+
 def linear_grouped(X, W, group_rows, *, layout="NK", epilogue="NONE", bias=None, residual=None):
     """Grouped linear layer (the "Grouped GEMM" of the paper's Table 1), written out as its definition: the rows of X
     are cut into consecutive groups of ``group_rows[g]`` rows and group g is multiplied by ``W[g]``:

@@ -25,7 +25,8 @@ STATUS_NAMES = {
     0: "FACT_OK", 1: "FACT_ERR_INVALID_ARG", 2: "FACT_ERR_BAD_ALIGNMENT", 3: "FACT_ERR_UNSUPPORTED",
     4: "FACT_ERR_ARCH", 5: "FACT_ERR_WORKSPACE_TOO_SMALL", 6: "FACT_ERR_CUDA", 7: "FACT_ERR_DEVICE_TIMEOUT",
 }
-EPILOGUES = {"NONE": 0, "BIAS": 1, "BIAS_RELU": 2, "BIAS_GELU_TANH": 3, "SILU_GATE": 4, "BIAS_RESIDUAL": 5}
+EPILOGUES = {"NONE": 0, "BIAS": 1, "BIAS_RELU": 2, "BIAS_GELU_TANH": 3, "SILU_GATE": 4, "BIAS_RESIDUAL": 5,
+             "BIAS_SOFTMAX": 6}
 LAYOUTS = {"KN": 0, "NK": 1}
 OUT_TYPES = {torch.bfloat16: 0, torch.float32: 1, "bf16": 0, "f32": 1}
 OPS = {"gemm": 0, "gemm_batched": 1, "gemm_splitk": 2, "linear": 3, "linear_fp8": 4}

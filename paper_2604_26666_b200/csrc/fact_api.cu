@@ -168,6 +168,23 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.tile_k != 0 && c.tile_k != q.k_elems()) return FACT_ERR_UNSUPPORTED;
   c.tile_k = q.k_elems();
   const long long Nw = q.Nw();
+  if (q.epi == FACT_EPI_BIAS_SOFTMAX) {
+    // the softmax of a row is taken inside one tile: the tile is as wide as the row, tiles are data-parallel and
+    // stored by the direct path
+    if (q.N_out > 256) return FACT_ERR_UNSUPPORTED;
+    const int want = std::max(32, round_up((int)q.N_out, 32));
+    if (c.tile_n != 0 && c.tile_n < want) return FACT_ERR_UNSUPPORTED;
+    if (c.tile_n == 0) {  // the narrowest width the layout and the pair size allow
+      const int cg_try = c.cta_group ? c.cta_group : ((c.tile_m == 256) ? 2 : 1);
+      for (int tn = want; tn <= 256 && c.tile_n == 0; tn += 32)
+        if (tile_ok(q, tn, cg_try)) c.tile_n = tn;
+      if (c.tile_n == 0) return FACT_ERR_UNSUPPORTED;
+      if (c.cta_group == 0) c.cta_group = cg_try;
+    }
+    if (c.split_k > 1 || c.split_k < 0 || c.store_mode == 2) return FACT_ERR_UNSUPPORTED;
+    c.split_k = 1;
+    c.store_mode = 1;
+  }
   if (c.cta_group == 0 && c.tile_m != 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
   if (c.cta_group == 0 || c.tile_n == 0) {
     // Untuned problem: pick (pair size, tile width) with a small cost model -- waves over the SMs times the
@@ -254,7 +271,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 fact_status_t validate(const Problem& q) {
   if (q.batch < 0 || q.M < 0 || q.N_out < 0 || q.K < 0) return FACT_ERR_INVALID_ARG;
-  if (q.epi < FACT_EPI_NONE || q.epi > FACT_EPI_BIAS_RESIDUAL) return FACT_ERR_INVALID_ARG;
+  if (q.epi < FACT_EPI_NONE || q.epi > FACT_EPI_BIAS_SOFTMAX) return FACT_ERR_INVALID_ARG;
   if (q.layout != FACT_B_KN && q.layout != FACT_B_NK) return FACT_ERR_INVALID_ARG;
   if (q.out != FACT_OUT_BF16 && q.out != FACT_OUT_F32) return FACT_ERR_INVALID_ARG;
   if (q.batch == 0 || q.M == 0 || q.N_out == 0) return FACT_OK;
@@ -510,6 +527,7 @@ fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUten
     case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate>(h, base + 4, plan, tm, stream);
     case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual>(h, base + 5, plan, tm, stream);
     case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tm, stream);
+    case kEpiBiasSoftmax: return launch_instance<CG, kEpiBiasSoftmax>(h, base + 7, plan, tm, stream);
     default: return FACT_ERR_INVALID_ARG;
   }
 }
@@ -629,6 +647,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     st = make_plan(h, q, &dp, 0, &plan);
     if (st != FACT_OK) return st;
   }
+  if (q.K == 0 && q.epi == FACT_EPI_BIAS_SOFTMAX) return FACT_ERR_UNSUPPORTED;  // (the stand-alone epilogue has no softmax)
   if (q.K == 0) {  // empty sum: the epilogue of a zero accumulator
     st = launch_reduce(h, q, plan, 0, reinterpret_cast<const float*>(q.C), stream);
   } else {
@@ -970,6 +989,7 @@ static fact_status_t linear_grouped_impl(fact_handle_t h, bool fp8, float scale,
   }
   if (groups == 0 || M == 0) return FACT_OK;
   if (cfg && (cfg->split_k > 1 || cfg->split_k < 0 || cfg->store_mode == 2)) return FACT_ERR_UNSUPPORTED;
+  if (epi == FACT_EPI_BIAS_SOFTMAX) return FACT_ERR_UNSUPPORTED;
   Problem q = make_problem(fp8 ? FACT_OP_LINEAR_FP8 : FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, strideW, layout,
                            bias, residual, ldr, 0, Y, ldy, 0, out, epi);
   q.groups = groups;

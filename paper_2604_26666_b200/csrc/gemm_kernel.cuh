@@ -57,7 +57,8 @@ enum : int {
   kEpiBiasGeluTanh = 3,
   kEpiSiluGate = 4,
   kEpiBiasResidual = 5,
-  kEpiPartial = 6  // raw FP32 accumulator to the split-K workspace
+  kEpiBiasSoftmax = 6,  // softmax over the whole output row (one n-tile per row), direct stores only
+  kEpiPartial = 7       // raw FP32 accumulator to the split-K workspace
 };
 constexpr int kDeviceTimeoutCode = 7;  // FACT_ERR_DEVICE_TIMEOUT
 
@@ -390,7 +391,8 @@ __device__ __forceinline__ float silu_f32(float g) { return __fdividef(g, 1.f + 
 
 template <int EPI>
 constexpr bool epi_has_bias() {
-  return EPI == kEpiBias || EPI == kEpiBiasRelu || EPI == kEpiBiasGeluTanh || EPI == kEpiBiasResidual;
+  return EPI == kEpiBias || EPI == kEpiBiasRelu || EPI == kEpiBiasGeluTanh || EPI == kEpiBiasResidual ||
+         EPI == kEpiBiasSoftmax;
 }
 
 // The fused element-wise operation on 8 consecutive output columns.
@@ -598,6 +600,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   if constexpr (GROUPED) {  // group boundaries are kept by the row-predicated direct stores only
     static_assert(!SK && EPI != kEpiPartial, "grouped tiles are data-parallel");
     if (p.store_tma || p.grp_tiles == nullptr || p.grp_rows == nullptr) {
+      if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+      return;
+    }
+  }
+  if constexpr (EPI == kEpiBiasSoftmax) {  // a row's softmax needs the whole row in one tile and the direct stores
+    if (p.store_tma || p.tiles_n != 1) {
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
       return;
     }
@@ -1149,6 +1157,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else {
       // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
       const bool c_vec = p.c_vec != 0;
+      uint32_t xch_count = 0;  // exchanges with the other warp of the lane quarter so far (row softmax only)
       UnitWalk<false, GROUPED> walk(p, unit0, unit_stride);  // (stream-K always stores through the staged path)
       WorkUnit w;
       while (ok && walk.next(p, w)) {
@@ -1166,6 +1175,85 @@ __global__ void __launch_bounds__(kThreads, 1)
         const __nv_bfloat16* r_row = nullptr;
         if constexpr (EPI == kEpiBiasResidual)
           r_row = p.R + (GROUPED ? 0LL : (long long)w.b * p.strideR) + (long long)row * p.ldr;
+        if constexpr (EPI == kEpiBiasSoftmax) {
+          // ---- y = softmax(acc + bias) over the whole row (the host made the tile as wide as the row).  The two warps
+          // of a lane quarter hold alternate 32-column pieces of every row, so the row maximum and the row sum are
+          // each exchanged once through shared memory, with an mbarrier handshake whose wait is bounded like every
+          // other.  Three passes over tensor memory (maximum, sum, normalise) instead of 128 live registers.
+          const int e_peer = (half ^ 1) * 4 + q;
+          const uint32_t my_slots = epi_base + (uint32_t)(e * p.epi_bufs) * kEpiBufBytes;       // 2 x 32 floats
+          const uint32_t peer_slots = epi_base + (uint32_t)(e_peer * p.epi_bufs) * kEpiBufBytes;
+          auto exchange = [&](float mine, float& theirs) -> bool {
+            const uint32_t slot = (xch_count & 1u) * 128u + (uint32_t)lane * 4u;
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_slots + slot), "f"(mine) : "memory");
+            __syncwarp();
+            // (two barriers in turn: the peer may arrive for the next exchange before this warp has seen this one
+            // complete, which a single one-bit phase could not tell from "not yet")
+            if (lane == 0) ptx::mbar_arrive(res_bar(e_peer, (int)(xch_count & 1u)));
+            if (!wait_bar(res_bar(e, (int)(xch_count & 1u)), (xch_count >> 1) & 1u, abort_p, p.status)) return false;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(theirs) : "r"(peer_slots + slot) : "memory");
+            ++xch_count;
+            return true;
+          };
+          // z = alpha * acc + bias of one 32-column piece, columns past the row's end at -inf
+          auto load_piece = [&](int c, float (&z)[32]) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32b_x32(t_acc + (uint32_t)c, v);
+            ptx::tmem_wait_ld();
+            if (scale_acc) scale32(v);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int n = c + g * 8;
+              float b8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+              if (p.bias != nullptr && n < p.N_out) load_bf16x8(p.bias + n, min(8, p.N_out - n), p.bias_vec != 0, b8);
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                z[g * 8 + j] = (n + j < p.N_out) ? __uint_as_float(v[g * 8 + j]) + b8[j] : -INFINITY;
+            }
+          };
+          float mloc = -INFINITY;
+          for (int c = half * 32; c < p.N_out; c += 64) {
+            float z[32];
+            load_piece(c, z);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mloc = fmaxf(mloc, z[i]);
+          }
+          float mpeer;
+          if (!exchange(mloc, mpeer)) {
+            ok = false;
+            break;
+          }
+          const float m = fmaxf(mloc, mpeer);  // finite: the row has at least one column and column 0 is in a piece
+          float lloc = 0.f;
+          for (int c = half * 32; c < p.N_out; c += 64) {
+            float z[32];
+            load_piece(c, z);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) lloc += __expf(z[i] - m);
+          }
+          float lpeer;
+          if (!exchange(lloc, lpeer)) {
+            ok = false;
+            break;
+          }
+          const float inv = 1.f / (lloc + lpeer);
+          for (int c = half * 32; c < p.N_out; c += 64) {
+            float z[32];
+            load_piece(c, z);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int n = c + g * 8;
+              const int nvalid = min(8, p.N_out - n);
+              if (nvalid > 0 && row_ok && !(p.debug & 4)) {
+                float y[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) y[j] = __expf(z[g * 8 + j] - m) * inv;
+                if (p.out_f32) store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid, c_vec);
+                else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
+              }
+            }
+          }
+        } else
         for (int c = half * 32; c < p.out_cols; c += 64) {  // the two warps of a quarter alternate 32-column pieces
           const int n0 = n_tile0 + c;
           if (n0 >= p.N_out) break;  // uniform across the warp

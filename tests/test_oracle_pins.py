@@ -310,3 +310,27 @@ def test_linear_grouped_is_the_per_group_product():
     assert np.array_equal(kn, got)
     with pytest.raises(ValueError):
         oracle.linear_grouped(X, W, rows[:-1], layout="NK")
+
+
+def test_linear_softmax_pins():
+    """oracle.linear_softmax: rows sum to one, invariance under a shift of the bias, scipy's softmax of the same
+    logits (a library routine), and the two-column closed form (a logistic function of the difference)."""
+    from scipy.special import softmax as scipy_softmax
+
+    rng = np.random.default_rng(12)
+    M, N, K = 9, 21, 33
+    X = rng.integers(0x3C00, 0x4080, size=(M, K)).astype(np.uint16) | (rng.integers(0, 2, size=(M, K)).astype(np.uint16) << 15)
+    W = rng.integers(0x3A00, 0x3F80, size=(N, K)).astype(np.uint16) | (rng.integers(0, 2, size=(N, K)).astype(np.uint16) << 15)
+    bias = rng.integers(0x3C00, 0x4000, size=(N,)).astype(np.uint16)
+    Y = oracle.linear_softmax(X, W, layout="NK", bias=bias)
+    assert np.allclose(Y.sum(axis=1), 1.0, rtol=0, atol=1e-14) and (Y > 0).all()
+    logits = oracle.linear(X, W, layout="NK", epilogue="BIAS", bias=bias)
+    assert np.allclose(Y, scipy_softmax(logits, axis=1), rtol=1e-13, atol=0)
+    shifted = np.array([oracle.round_bf16(v + 2.0) for v in oracle.bf16_to_f64(bias)], dtype=np.uint16)
+    if np.array_equal(oracle.bf16_to_f64(shifted), oracle.bf16_to_f64(bias) + 2.0):  # the shift is exact in BF16 here
+        assert np.allclose(oracle.linear_softmax(X, W, layout="NK", bias=shifted), Y, rtol=1e-12, atol=0)
+    two = oracle.linear_softmax(X, W[:2], layout="NK")
+    z = oracle.linear(X, W[:2], layout="NK")
+    assert np.allclose(two[:, 0], 1.0 / (1.0 + np.exp(z[:, 1] - z[:, 0])), rtol=1e-13, atol=0)
+    one = oracle.linear_softmax(X, W[:1], layout="NK")
+    assert np.array_equal(one, np.ones((M, 1)))
