@@ -61,6 +61,8 @@ enum : int {
   kEpiPartial = 7       // raw FP32 accumulator to the split-K workspace
 };
 constexpr int kDeviceTimeoutCode = 7;  // FACT_ERR_DEVICE_TIMEOUT
+struct FactTrue { static constexpr bool value = true; };    // compile-time tags for code written once and
+struct FactFalse { static constexpr bool value = false; };  // instantiated for both operand formats
 
 struct GemmParams {
   // problem
@@ -759,7 +761,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (cta_rank == 0) {
+    // The operand format is chosen once, outside every loop: whatever the issuing thread does between two
+    // instructions is idle time on the tensor pipe (a warp-uniform `if (p.fp8)` in front of every instruction cost
+    // 16 % of the 8192^3 product: 1.086 M instead of 0.933 M cycles).
+    auto issue_all = [&](auto fp8_tag) {
+      constexpr bool kFp8 = decltype(fp8_tag)::value;
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -797,7 +803,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!(p.debug & 2)) {
 #pragma unroll
               for (int k = 0; k < kTileK / kUmmaK; ++k) {
-                if (p.fp8)
+                if constexpr (kFp8)
                   ptx::umma_f8<CG>(d_tmem, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step),
                                    p.idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
                 else
@@ -828,6 +834,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         c[3] = prof_full_wait;
         c[7] = prof_first_full;  // cycles from kernel entry to the first operand stage being ready
       }
+    };
+    if (cta_rank == 0) {
+      if (p.fp8) issue_all(FactTrue{});
+      else issue_all(FactFalse{});
     }
     __syncwarp();
   } else {
