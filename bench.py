@@ -350,10 +350,12 @@ def main():
 
     # ---------------------------------------------------------------- every shape of the five configurations
     shapes = []
-    if not args.no_shapes and rank == 0:
+    # (single-GPU information: in a multi-rank run every rank but 0 would sit in the process group for minutes)
+    tables = not args.no_shapes and rank == 0 and world == 1
+    if tables:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
     attention, blocks, fp8, grouped = [], [], [], []
-    if not args.no_shapes and rank == 0:
+    if tables:
         attention = attention_table(h, dev, stream, flush_l2, peaks)
         fp8 = fp8_table(h, dev, stream, flush_l2, peaks)
         grouped = grouped_table(h, dev, stream, flush_l2, peaks)
