@@ -240,7 +240,8 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
  * fact_linear.  One launch: tiles never cross a group boundary (the last tile of a group is ragged), all tiles are
  * data-parallel, the output is stored by row-predicated register stores (the group table travels to a buffer of
  * the handle in stream order, so grouped calls through one handle must be stream-ordered with respect to each
- * other).  cfg: tile shape, pair size and stages only (K slices, stream-K and staged stores are refused with
+ * other, and not inside a stream capture: the table is copied from pageable host memory).  cfg: tile shape, pair
+ * size and stages only (K slices, stream-K, staged stores and the row softmax are refused with
  * FACT_ERR_UNSUPPORTED).  groups == 0 or M == 0 is a successful no-op. */
 fact_status_t fact_linear_grouped(fact_handle_t handle, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
                                   const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,
