@@ -307,6 +307,61 @@ typedef enum { FACT_NORM_LAYER = 0, FACT_NORM_RMS = 1 } fact_norm_t;
 fact_status_t fact_norm(fact_handle_t handle, fact_norm_t kind, int64_t M, int64_t C, const void* X, int64_t ldx,
                         const void* gamma, const void* beta, float eps, void* Y, int64_t ldy, void* cuda_stream);
 
+/* A row normalisation between two linear layers without its own pass over the activations (Table 1 lists
+ * "GEMM-LayerNorm-GEMM fusion" among the registry's Level-2 kernels; Section 5.2's blocks have a norm between
+ * the attention output projection and the MLP).  Three pieces:
+ *
+ *  1. the call that PRODUCES the activations also leaves partial sums of every output row:
+ *     row_stats_out[c][m] = (sum, sum of squares) of the stored BF16 values Y[m][64c .. 64c+64), as FP32 pairs,
+ *     [ceil(N_out / 64)][M][2] floats (fact_row_stats computes the same array for a tensor that no call of this
+ *     library produced);
+ *  2. the scale and shift of the normalisation are folded into the next layer's weights once (fact_fold_norm):
+ *     Wf[n][k] = bf16(gamma[k] W[n][k]), colsum[n] = sum_k Wf[n][k], bf[n] = bf16(b[n] + sum_k beta[k] W[n][k]);
+ *  3. the call that CONSUMES them multiplies the raw activations by Wf and corrects the accumulator per row,
+ *         norm(x) . W^T + b  =  rstd[m] * (x . Wf^T)[m][n] - rstd[m] * mean[m] * colsum[n] + bf[n],
+ *     with mean = S1 / K, rstd = 1 / sqrt(S2 / K - mean^2 + eps) (FACT_XNORM_LAYER), or mean = 0 (FACT_XNORM_RMS,
+ *     no colsum), S1, S2 the sums of x_row_stats over the K / 64 chunks; then the epilogue as usual.
+ *
+ * Numerics: x is not centred before the product, so the two terms cancel when |mean| is large against the
+ * standard deviation: the absolute error grows like (|mean| / std) * 2^-8 * |output|.  Residual streams of
+ * pre-norm transformers have |mean| well below std; for data that does not, use fact_norm.
+ *
+ * Limits: fact_linear_ex only (one BF16 product, batch 1); the staged (TMA) store path must be in use (Y 16-byte
+ * aligned, ldy a multiple of 8) and K not sliced (cfg->split_k 0, 1 or negative); row_stats_out needs a BF16
+ * output; FACT_XNORM_LAYER needs N_out a multiple of 64, w_colsum 16-byte aligned, and is not combined with
+ * SILU_GATE (FACT_XNORM_RMS is); BIAS_SOFTMAX takes neither; a stream-K choice (cfg->split_k < 0) is ignored, the tiles run
+ * data-parallel.  FACT_ERR_UNSUPPORTED otherwise. */
+typedef enum { FACT_XNORM_NONE = 0, FACT_XNORM_LAYER = 1, FACT_XNORM_RMS = 2 } fact_xnorm_t;
+typedef struct fact_linear_ext {
+  float* row_stats_out;      /* device, [ceil(N_out / 64)][M][2], or NULL: partial row sums of Y */
+  fact_xnorm_t x_norm;       /* normalisation of X's rows folded into this product */
+  const float* x_row_stats;  /* device, [ceil(K / 64)][M][2]: partial row sums of X (x_norm != NONE) */
+  const float* w_colsum;     /* device, [N_out]: column sums of the folded weights (FACT_XNORM_LAYER) */
+  float eps;                 /* the normalisation's epsilon, >= 0 */
+} fact_linear_ext_t;
+
+/* fact_linear with the extras of fact_linear_ext_t (ext == NULL: exactly fact_linear). */
+fact_status_t fact_linear_ex(fact_handle_t handle, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                             const void* W, int64_t ldw, fact_blayout_t w_layout, const void* bias,
+                             const void* residual, int64_t ldr, void* Y, int64_t ldy, fact_out_t out_type,
+                             fact_epilogue_t epilogue, const fact_linear_ext_t* ext, const fact_config_t* cfg,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* stats[c][m] = (sum, sum of squares) over X[m][64c .. 64c+64) in FP32, [ceil(C / 64)][M][2] floats: the row sums
+ * fact_linear_ex consumes, for an X that came from elsewhere.  X: BF16 [M x C], 16-byte aligned, ldx and C
+ * multiples of 8; stats 8-byte aligned. */
+fact_status_t fact_row_stats(fact_handle_t handle, int64_t M, int64_t C, const void* X, int64_t ldx, float* stats,
+                             void* cuda_stream);
+
+/* Fold a normalisation's gamma [K] (and beta [K], or NULL for an RMS norm) into the weights W [N_w x K] (BF16,
+ * FACT_B_NK layout, ldw) of the linear layer that follows it: writes W_folded [N_w x K] (ldwf; may alias W when
+ * ldwf == ldw), colsum [N_w] FP32 (or NULL), and -- iff beta is given -- bias_folded [N_w] BF16 from bias [N_w]
+ * (or NULL for no bias).  For SILU_GATE pass the stacked gate and up rows, N_w = 2 N_out.  Run once per model;
+ * K a multiple of 8, pointers 16-byte aligned, ldw and ldwf multiples of 8. */
+fact_status_t fact_fold_norm(fact_handle_t handle, int64_t N_w, int64_t K, const void* W, int64_t ldw,
+                             const void* gamma, const void* beta, const void* bias, void* W_folded, int64_t ldwf,
+                             float* colsum, void* bias_folded, void* cuda_stream);
+
 /* One pre-norm transformer block, forward, as a chain of this library's kernels on one stream (Section 5.2:
  * the two Level-3 blocks the paper composes from its attention and MLP patterns):
  *     n1  = norm1(x)

@@ -39,10 +39,19 @@ EXPORTED = [
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
+    "fact_linear_ex", "fact_row_stats", "fact_fold_norm",
 ]
 
 
 NORMS = {"layer": 0, "rms": 1}
+XNORMS = {None: 0, "none": 0, "layer": 1, "rms": 2}
+
+
+class LinearExt(Structure):
+    """Mirror of fact_linear_ext_t."""
+
+    _fields_ = [("row_stats_out", c_void_p), ("x_norm", c_int), ("x_row_stats", c_void_p), ("w_colsum", c_void_p),
+                ("eps", c_float)]
 BLOCK_KINDS = {"gpt": 0, "llama": 1}
 
 
@@ -128,6 +137,10 @@ def lib() -> ctypes.CDLL:
                                       c_int, c_int, cfgp, vp]
     L.fact_linear_grouped_fp8.argtypes = [vp, c_int, POINTER(i64), i64, i64, vp, i64, vp, i64, i64, c_float, vp, vp, i64, vp,
                                           i64, c_int, c_int, cfgp, vp]
+    L.fact_linear_ex.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, vp, i64, vp, i64, c_int, c_int,
+                                 POINTER(LinearExt), cfgp, vp, sz, vp]
+    L.fact_row_stats.argtypes = [vp, i64, i64, vp, i64, vp, vp]
+    L.fact_fold_norm.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     for name in EXPORTED:
         fn = getattr(L, name)
@@ -363,9 +376,12 @@ class Handle:
         return out
 
     def linear(self, X, W, bias=None, residual=None, epilogue="NONE", layout="NK", out=None,
-               out_dtype=torch.bfloat16, cfg=None, stream=None):
+               out_dtype=torch.bfloat16, cfg=None, stream=None, stats_out=None, x_norm=None, x_stats=None,
+               w_colsum=None, eps=1e-5):
         """Y = epilogue(X @ W)  (fact_linear).  layout "NK": W is [Nw, K] (nn.Linear weight); "KN": [K, Nw].
-        For SILU_GATE W carries 2*N_out columns (gate first, then up)."""
+        For SILU_GATE W carries 2*N_out columns (gate first, then up).
+        stats_out (FP32 [ceil(N_out/64), M, 2]) receives partial row sums of Y; x_norm "layer" / "rms" with x_stats
+        (and w_colsum for "layer") folds a normalisation of X's rows into the product (fact_linear_ex)."""
         _need(X, "X", torch.bfloat16, 2)
         _need(W, "W", torch.bfloat16, 2)
         M, K = X.shape
@@ -391,11 +407,61 @@ class Handle:
         _need(out, "out", out.dtype, 2)
         nws = self.workspace_bytes("linear", 1, M, N, K, epilogue, layout, out.dtype, cfg)
         ws = self.workspace(nws)
+        if stats_out is not None or x_norm not in (None, "none") or x_stats is not None or w_colsum is not None:
+            if stats_out is not None:
+                _need(stats_out, "stats_out", torch.float32, 3)
+                if tuple(stats_out.shape) != ((N + 63) // 64, M, 2) or not stats_out.is_contiguous():
+                    raise ValueError("stats_out must be a contiguous [ceil(N_out/64), M, 2]")
+            if x_stats is not None:
+                _need(x_stats, "x_stats", torch.float32, 3)
+                if tuple(x_stats.shape) != ((K + 63) // 64, M, 2) or not x_stats.is_contiguous():
+                    raise ValueError("x_stats must be a contiguous [ceil(K/64), M, 2]")
+            if w_colsum is not None:
+                _need(w_colsum, "w_colsum", torch.float32, 1)
+                if w_colsum.shape[0] != N:
+                    raise ValueError("w_colsum must have N_out entries")
+            ext = LinearExt(_ptr(stats_out), XNORMS[x_norm], _ptr(x_stats), _ptr(w_colsum), float(eps))
+            _check(lib().fact_linear_ex(self._h, M, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W), LAYOUTS[layout],
+                                        _ptr(bias), _ptr(residual), _ld(residual) if residual is not None else 0,
+                                        _ptr(out), _ld(out), OUT_TYPES[out.dtype], EPILOGUES[epilogue],
+                                        ctypes.byref(ext), self._cfg(cfg), _ptr(ws), nws, self._stream(stream)),
+                   "fact_linear_ex", self._h)
+            return out
         _check(lib().fact_linear(self._h, M, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W), LAYOUTS[layout], _ptr(bias),
                                  _ptr(residual), _ld(residual) if residual is not None else 0, _ptr(out), _ld(out),
                                  OUT_TYPES[out.dtype], EPILOGUES[epilogue], self._cfg(cfg), _ptr(ws), nws,
                                  self._stream(stream)), "fact_linear", self._h)
         return out
+
+    def row_stats(self, X, out=None, stream=None):
+        """Partial row sums of X per 64-column chunk: FP32 [ceil(C/64), M, 2] (fact_row_stats)."""
+        _need(X, "X", torch.bfloat16, 2)
+        M, C = X.shape
+        if out is None:
+            out = torch.empty(((C + 63) // 64, M, 2), dtype=torch.float32, device=X.device)
+        _need(out, "out", torch.float32, 3)
+        _check(lib().fact_row_stats(self._h, M, C, _ptr(X), _ld(X), _ptr(out), self._stream(stream)),
+               "fact_row_stats", self._h)
+        return out
+
+    def fold_norm(self, W, gamma, beta=None, bias=None, stream=None):
+        """Fold a normalisation's gamma (and beta) into the [N_w, K] weights of the layer after it (fact_fold_norm).
+        Returns (W_folded, colsum, bias_folded); bias_folded is None without beta."""
+        _need(W, "W", torch.bfloat16, 2)
+        _need(gamma, "gamma", torch.bfloat16, 1)
+        Nw, K = W.shape
+        if gamma.shape[0] != K:
+            raise ValueError("gamma must have K entries")
+        if beta is not None:
+            _need(beta, "beta", torch.bfloat16, 1)
+        if bias is not None:
+            _need(bias, "bias", torch.bfloat16, 1)
+        Wf = torch.empty_like(W)
+        colsum = torch.empty(Nw, dtype=torch.float32, device=W.device)
+        bf = torch.empty(Nw, dtype=torch.bfloat16, device=W.device) if beta is not None else None
+        _check(lib().fact_fold_norm(self._h, Nw, K, _ptr(W), _ld(W), _ptr(gamma), _ptr(beta), _ptr(bias), _ptr(Wf),
+                                    _ld(Wf), _ptr(colsum), _ptr(bf), self._stream(stream)), "fact_fold_norm", self._h)
+        return Wf, colsum, bf
 
     def linear_grouped(self, X, W, group_rows, bias=None, residual=None, epilogue="NONE", layout="NK", out=None,
                        out_dtype=torch.bfloat16, cfg=None, stream=None):

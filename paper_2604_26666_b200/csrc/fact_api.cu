@@ -64,6 +64,11 @@ struct Problem {
   const int64_t* group_rows = nullptr;   // host: rows of each group
   bool fp8 = false;    // operands are FP8 E4M3 (one byte per element) instead of BF16
   float alpha = 1.f;   // FP8: the accumulator is multiplied by this before the epilogue
+  float* stats_out = nullptr;       // partial row sums of the stored output, for a normalisation folded into the next call
+  const float* stats_in = nullptr;  // partial row sums of A from the call that produced it
+  int norm = 0;                     // 0: none; 1: A's rows are layer-normalised over K; 2: RMS-normalised
+  const float* colsum = nullptr;    // norm == 1: sum over k of the folded W[n][k]
+  float norm_eps = 0.f;
   long long Nw() const { return epi == FACT_EPI_SILU_GATE ? 2 * N_out : N_out; }
   int k_elems() const { return fp8 ? 2 * kTileK : kTileK; }  // elements of K in a 128-byte row of a stage
   int op_align() const { return fp8 ? 16 : 8; }              // elements in 16 bytes of an operand
@@ -88,7 +93,7 @@ struct fact_handle_s {
   EncodeTiledFn encode = nullptr;
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
-  unsigned configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
+  unsigned long long configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
   int* d_groups = nullptr;       // grouped GEMM: m-tile prefix and row offsets of the call in flight
@@ -289,6 +294,20 @@ fact_status_t validate(const Problem& q) {
     return FACT_ERR_INVALID_ARG;
   }
   if (q.ldc < q.N_out) return FACT_ERR_INVALID_ARG;
+  if (q.stats_out || q.norm) {
+    if (q.norm < 0 || q.norm > 2) return FACT_ERR_INVALID_ARG;
+    if (q.op != FACT_OP_LINEAR || q.batch != 1 || q.groups > 0 || q.fp8 || q.epi == FACT_EPI_BIAS_SOFTMAX || q.K == 0)
+      return FACT_ERR_UNSUPPORTED;
+    if (q.stats_out && q.out != FACT_OUT_BF16) return FACT_ERR_UNSUPPORTED;  // the sums are over stored BF16 values
+    if (q.norm) {
+      if (!q.stats_in || !(q.norm_eps >= 0.f)) return FACT_ERR_INVALID_ARG;
+      if (q.norm == 1) {
+        if (!q.colsum) return FACT_ERR_INVALID_ARG;
+        if (q.epi == FACT_EPI_SILU_GATE || q.N_out % 64) return FACT_ERR_UNSUPPORTED;
+        if (!aligned16(q.colsum)) return FACT_ERR_BAD_ALIGNMENT;
+      }
+    }
+  }
   if (q.K > 0) {
     if (!q.A || !q.B) return FACT_ERR_INVALID_ARG;
     if (q.lda < q.K) return FACT_ERR_INVALID_ARG;
@@ -436,6 +455,13 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   p.store_tma = (c.store_mode == 1) ? 0 : (can_stage ? 1 : 0);
   p.r_tma = p.store_tma && q.epi == FACT_EPI_BIAS_RESIDUAL && p.r_vec;
   plan->cfg.store_mode = p.store_tma ? 2 : 1;
+  // row sums out and the folded normalisation live in the staged epilogue of an unsliced product
+  if ((q.stats_out || q.norm) && (!p.store_tma || c.split_k > 1)) return FACT_ERR_UNSUPPORTED;
+  p.stats_out = reinterpret_cast<float2*>(q.stats_out);
+  p.stats_in = reinterpret_cast<const float2*>(q.stats_in);
+  p.colsum = q.colsum;
+  p.norm_mode = q.norm;
+  p.norm_eps = q.norm_eps;
   p.status = h->d_status;
   p.debug = h->debug_flags;
   plan->ws_bytes = workspace_for(h, q, c);
@@ -483,17 +509,17 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
   return FACT_OK;
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, bool EXT = false>
 fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                               cudaStream_t stream) {
-  auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED>;
+  auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED, EXT>;
   if (slot < 0) {  // (no bit left in the handle's mask for these instantiations: set the attribute on every launch)
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-  } else if (!(h->configured_mask & (1u << slot))) {
+  } else if (!(h->configured_mask & (1ull << slot))) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-    h->configured_mask |= (1u << slot);
+    h->configured_mask |= (1ull << slot);
   }
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof lc);
@@ -529,6 +555,21 @@ fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUten
     case kEpiPartial: return launch_instance<CG, kEpiPartial>(h, base + 6, plan, tm, stream);
     case kEpiBiasSoftmax: return launch_instance<CG, kEpiBiasSoftmax>(h, base + 7, plan, tm, stream);
     default: return FACT_ERR_INVALID_ARG;
+  }
+}
+
+// The instantiations with row sums out / a folded row normalisation in (staged epilogue, data-parallel tiles).
+template <int CG>
+fact_status_t launch_epi_ext(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  const int base = 32 + (CG - 1) * 8;
+  switch (epi) {
+    case kEpiNone: return launch_instance<CG, kEpiNone, false, false, true>(h, base + 0, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias, false, false, true>(h, base + 1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, false, true>(h, base + 2, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, false, true>(h, base + 3, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, false, true>(h, base + 4, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, false, true>(h, base + 5, plan, tm, stream);
+    default: return FACT_ERR_UNSUPPORTED;
   }
 }
 
@@ -640,6 +681,13 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     plan.grid = (int)std::min<long long>(std::max(1, h->sm_count / plan.cfg.cta_group), std::max<long long>(units, 1)) *
                 plan.cfg.cta_group;
   }
+  if (plan.cfg.split_k < 0 && (q.stats_out || q.norm)) {
+    // the extras live in the data-parallel instantiations: a stream-K choice (the caller's or the table's) is dropped
+    fact_config_t dp = plan.cfg;
+    dp.split_k = 1;
+    st = make_plan(h, q, &dp, 0, &plan);
+    if (st != FACT_OK) return st;
+  }
   if (plan.cfg.split_k < 0 && (!ws || ws_bytes < plan.ws_bytes) && !user) {
     // a tuned stream-K entry, but this caller brought no scratch: run the tiles data-parallel
     fact_config_t dp = plan.cfg;
@@ -717,6 +765,8 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
     if (q.groups > 0) st = plan.cfg.cta_group == 2 ? launch_epi_grouped<2>(h, epi, plan, tm, stream)
                                                    : launch_epi_grouped<1>(h, epi, plan, tm, stream);
+    else if (q.stats_out || q.norm) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2>(h, epi, plan, tm, stream)
+                                                                 : launch_epi_ext<1>(h, epi, plan, tm, stream);
     else if (stream_k) st = plan.cfg.cta_group == 2 ? launch_epi_sk<2>(h, epi, plan, tm, stream)
                                                     : launch_epi_sk<1>(h, epi, plan, tm, stream);
     else if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);
@@ -971,6 +1021,26 @@ fact_status_t fact_linear(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, 
                           const fact_config_t* cfg, void* ws, size_t ws_bytes, void* stream) {
   Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, 0, layout, bias, residual, ldr, 0, Y,
                            ldy, 0, out, epi);
+  return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+fact_status_t fact_linear_ex(fact_handle_t h, int64_t M, int64_t N_out, int64_t K, const void* X, int64_t ldx,
+                             const void* W, int64_t ldw, fact_blayout_t layout, const void* bias, const void* residual,
+                             int64_t ldr, void* Y, int64_t ldy, fact_out_t out, fact_epilogue_t epi,
+                             const fact_linear_ext_t* ext, const fact_config_t* cfg, void* ws, size_t ws_bytes,
+                             void* stream) {
+  Problem q = make_problem(FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, 0, layout, bias, residual, ldr, 0, Y,
+                           ldy, 0, out, epi);
+  if (ext) {
+    if (ext->x_norm != FACT_XNORM_NONE && ext->x_norm != FACT_XNORM_LAYER && ext->x_norm != FACT_XNORM_RMS)
+      return FACT_ERR_INVALID_ARG;
+    q.stats_out = ext->row_stats_out;
+    q.norm = (int)ext->x_norm;
+    q.stats_in = ext->x_row_stats;
+    q.colsum = ext->w_colsum;
+    q.norm_eps = ext->eps;
+    if (q.norm == 0 && (q.stats_in || q.colsum)) return FACT_ERR_INVALID_ARG;
+  }
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
 }
 
@@ -1279,7 +1349,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.items = (int)items;
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
-    if (!(h->configured_mask & (1u << 30))) {
+    if (!(h->configured_mask & (1ull << 30))) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -1295,7 +1365,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
                         std::to_string(kAttnRegsAtLaunch);
         st = FACT_ERR_UNSUPPORTED;
       } else {
-        h->configured_mask |= (1u << 30);
+        h->configured_mask |= (1ull << 30);
       }
     }
     if (st == FACT_OK) {
@@ -1352,6 +1422,64 @@ fact_status_t fact_norm(fact_handle_t h, fact_norm_t kind, int64_t M, int64_t C,
   fact_status_t st = FACT_OK;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) st = cuda_fail(h, "norm launch", e);
+  else h->launches++;
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
+}
+
+fact_status_t fact_row_stats(fact_handle_t h, int64_t M, int64_t C, const void* X, int64_t ldx, float* stats,
+                             void* stream_v) {
+  if (!h || M < 0) return FACT_ERR_INVALID_ARG;
+  if (C < 8 || C % 8) return FACT_ERR_UNSUPPORTED;
+  if (M == 0) return FACT_OK;
+  if (!X || !stats || ldx < C || M > 0x7fffffffLL) return FACT_ERR_INVALID_ARG;
+  if (!aligned16(X) || ldx % 8 || ((uintptr_t)stats & 7u)) return FACT_ERR_BAD_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  const unsigned grid = (unsigned)((M + kNormWarps - 1) / kNormWarps);
+  fact_row_stats_kernel<<<grid, kNormWarps * 32, 0, reinterpret_cast<cudaStream_t>(stream_v)>>>(
+      reinterpret_cast<const __nv_bfloat16*>(X), (long long)M, (int)C, (long long)ldx, reinterpret_cast<float2*>(stats));
+  fact_status_t st = FACT_OK;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) st = cuda_fail(h, "row stats launch", e);
+  else h->launches++;
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
+}
+
+fact_status_t fact_fold_norm(fact_handle_t h, int64_t N_w, int64_t K, const void* W, int64_t ldw, const void* gamma,
+                             const void* beta, const void* bias, void* W_folded, int64_t ldwf, float* colsum,
+                             void* bias_folded, void* stream_v) {
+  if (!h || N_w < 0 || K < 0) return FACT_ERR_INVALID_ARG;
+  if (K % 8) return FACT_ERR_UNSUPPORTED;
+  if (N_w == 0) return FACT_OK;
+  if (!W || !gamma || !W_folded || ldw < K || ldwf < K || N_w > 0x7fffffffLL || K > 0x7fffffffLL)
+    return FACT_ERR_INVALID_ARG;
+  if ((beta != nullptr) != (bias_folded != nullptr)) return FACT_ERR_INVALID_ARG;  // the shift moves into the bias
+  if (!beta && bias) return FACT_ERR_INVALID_ARG;                                   // (without a shift the bias stays as it is)
+  if (!aligned16(W) || !aligned16(W_folded) || !aligned16(gamma) || (beta && !aligned16(beta)) || ldw % 8 || ldwf % 8)
+    return FACT_ERR_BAD_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  FoldParams p;
+  p.W = reinterpret_cast<const __nv_bfloat16*>(W);
+  p.Wf = reinterpret_cast<__nv_bfloat16*>(W_folded);
+  p.gamma = reinterpret_cast<const __nv_bfloat16*>(gamma);
+  p.beta = reinterpret_cast<const __nv_bfloat16*>(beta);
+  p.bias = reinterpret_cast<const __nv_bfloat16*>(bias);
+  p.bias_out = reinterpret_cast<__nv_bfloat16*>(bias_folded);
+  p.colsum = colsum;
+  p.N = (int)N_w;
+  p.K = (int)K;
+  p.ldw = ldw;
+  p.ldwf = ldwf;
+  const unsigned grid = (unsigned)((N_w + kNormWarps - 1) / kNormWarps);
+  fact_fold_norm_kernel<<<grid, kNormWarps * 32, 0, reinterpret_cast<cudaStream_t>(stream_v)>>>(p);
+  fact_status_t st = FACT_OK;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) st = cuda_fail(h, "fold launch", e);
   else h->launches++;
   if (dev != h->device) cudaSetDevice(dev);
   return st;

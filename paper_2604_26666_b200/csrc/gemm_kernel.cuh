@@ -125,6 +125,17 @@ struct GemmParams {
   int sk_len, sk_rem; // group c owns k-block iterations [c * sk_len + min(c, sk_rem), + sk_len + (c < sk_rem))
   float* sk_ws;       // one FP32 accumulator tile per CTA: [gridDim.x][tile_n / 32][8][128] float4
   int* sk_flags;      // [gridDim.x][kEpiWarps]: 1 while that warp's share of the CTA's partial tile is ready
+  // GEMM -> row normalisation -> GEMM without a pass over the activations (the EXT instantiations only: staged
+  // BF16 epilogue of data-parallel tiles).
+  // Producer: stats_out[chunk][row] = (sum, sum of squares) of the row's 64 stored BF16 values of column chunk
+  // `chunk`.  Consumer: the rows of A are to be normalised over K (norm_mode 1: LayerNorm, 2: RMSNorm); the scale
+  // vector is folded into W beforehand, so acc' = rstd[r] * acc - rstd[r] * mean[r] * colsum[n], with mean and
+  // rstd from the K / 64 partial sums of stats_in.
+  float2* stats_out;       // [ceil(N_out / 64)][M] or null
+  const float2* stats_in;  // [ceil(K / 64)][M] or null
+  const float* colsum;     // [N_out]: sum over k of the folded W[n][k] (LayerNorm only)
+  int norm_mode;
+  float norm_eps;
   // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
   // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
   int debug;
@@ -578,7 +589,7 @@ __device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uin
   }
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, bool EXT = false>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
@@ -605,6 +616,16 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
       return;
     }
+  }
+  if constexpr (EXT) {  // row sums out / a folded normalisation in: the staged epilogue of a whole, ungrouped tile
+    static_assert(!SK && !GROUPED && EPI != kEpiPartial && EPI != kEpiBiasSoftmax, "extras: plain data-parallel tiles");
+    if (!p.store_tma || (p.norm_mode != 0 && p.stats_in == nullptr) || (p.norm_mode == 1 && p.colsum == nullptr)) {
+      if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+      return;
+    }
+  } else if (p.norm_mode != 0 || p.stats_out != nullptr) {  // asked of an instantiation that has no code for it
+    if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+    return;
   }
   if constexpr (EPI == kEpiBiasSoftmax) {  // a row's softmax needs the whole row in one tile and the direct stores
     if (p.store_tma || p.tiles_n != 1) {
@@ -978,6 +999,74 @@ __global__ void __launch_bounds__(kThreads, 1)
         // the buffers are a whole main loop old): a load issued only after the first chunk's store leaves most of its
         // latency exposed, 3000 cycles per tile on the 768 -> 768 projection
         if (use_r && bufs == 2 && r_next == gc + 1 && issue_residual(half + 2, gc + 1, true)) r_next = gc + 2;
+        // rows of A normalised over K: this thread's row scale (and scale times mean) from the partial sums the
+        // producing call left, and the column sums of the folded weights for the warp's own 128 columns, four per
+        // lane (lane l holds local columns 4l .. 4l+3) -- all read while the main loop of the tile still runs
+        float nrm_rs = 1.f, nrm_rm = 0.f;
+        float4 nrm_cs = make_float4(0.f, 0.f, 0.f, 0.f);
+        constexpr int kHeldSlots = 16;  // K <= 1024: the partial sums wait in registers until the accumulator is there
+        float2 nrm_held[kHeldSlots];
+        float nrm_s1 = 0.f, nrm_s2 = 0.f;
+        if (EXT && p.norm_mode != 0) {
+          const int row = row0 + lane;
+          const int slots = (p.K + 63) >> 6;
+          const float2* src = p.stats_in + min(row, p.M - 1);  // (rows past M compute a scale nobody stores)
+          if (slots <= kHeldSlots) {
+            // a short main loop leaves these warps no idle time: issue the loads now, add them up after the wait
+            // for the accumulator, so that their trip to L2 is not on the tile's critical path
+#pragma unroll
+            for (int u = 0; u < kHeldSlots; ++u)
+              nrm_held[u] = u < slots ? __ldg(src + (size_t)u * (size_t)p.M) : make_float2(0.f, 0.f);
+          } else {
+            for (int s = 0; s < slots; ++s) {
+              const float2 t = __ldg(src + (size_t)s * (size_t)p.M);
+              nrm_s1 += t.x;
+              nrm_s2 += t.y;
+            }
+          }
+          if (p.norm_mode == 1) {
+            const int local = lane * 4;
+            const int ci = 2 * (local / chunk_cols) + half;
+            const int nc = n_tile0 + ci * chunk_cols + (local % chunk_cols);
+            if (ci < n_chunks && nc < p.N_out) nrm_cs = __ldg(reinterpret_cast<const float4*>(p.colsum + nc));
+          }
+        }
+        auto norm_finish = [&]() {
+          if (((p.K + 63) >> 6) <= kHeldSlots) {
+#pragma unroll
+            for (int u = 0; u < kHeldSlots; ++u) {
+              nrm_s1 += nrm_held[u].x;
+              nrm_s2 += nrm_held[u].y;
+            }
+          }
+          const float inv_k = 1.f / (float)p.K;
+          const float mean = p.norm_mode == 1 ? nrm_s1 * inv_k : 0.f;
+          nrm_rs = rsqrtf(fmaxf(nrm_s2 * inv_k - mean * mean, 0.f) + p.norm_eps);
+          nrm_rm = nrm_rs * mean;
+        };
+        // v <- rstd * v - rstd * mean * colsum  (LayerNorm) or rstd * v (RMSNorm), for the 32 accumulator columns
+        // whose index among the warp's 128 columns starts at local0 (a multiple of 32)
+        auto norm32 = [&](uint32_t (&v)[32], int local0) {
+          const uint64_t rs2 = ptx::pack_f32x2(__float_as_uint(nrm_rs), __float_as_uint(nrm_rs));
+          if (p.norm_mode == 1) {
+            const uint64_t rm2 = ptx::pack_f32x2(__float_as_uint(-nrm_rm), __float_as_uint(-nrm_rm));
+            const int src0 = local0 >> 2;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float cx = __shfl_sync(0xffffffffu, nrm_cs.x, src0 + j), cy = __shfl_sync(0xffffffffu, nrm_cs.y, src0 + j);
+              const float cz = __shfl_sync(0xffffffffu, nrm_cs.z, src0 + j), cw = __shfl_sync(0xffffffffu, nrm_cs.w, src0 + j);
+              const uint64_t t0 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(__float_as_uint(cx), __float_as_uint(cy)));
+              const uint64_t t1 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(__float_as_uint(cz), __float_as_uint(cw)));
+              ptx::unpack_f32x2(ptx::fma_f32x2(rs2, ptx::pack_f32x2(v[4 * j], v[4 * j + 1]), t0), v[4 * j], v[4 * j + 1]);
+              ptx::unpack_f32x2(ptx::fma_f32x2(rs2, ptx::pack_f32x2(v[4 * j + 2], v[4 * j + 3]), t1), v[4 * j + 2],
+                                v[4 * j + 3]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+              ptx::unpack_f32x2(ptx::mul_f32x2(rs2, ptx::pack_f32x2(v[i], v[i + 1])), v[i], v[i + 1]);
+          }
+        };
         long long tw = prof ? clock64() : 0;
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
           ok = false;
@@ -987,6 +1076,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (prof) prof_epi_wait += tb - tw;
         ptx::tc_fence_after();
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
+        if (EXT && p.norm_mode != 0) norm_finish();
         if constexpr (SK) {
           // the first piece of a tile: the same warp of the same CTA rank in each of the following groups parks
           // the rest of the sum; wait until those are complete (they precede everything else those groups do)
@@ -1058,6 +1148,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             scale32(v0);
             if (EPI == kEpiSiluGate || pieces == 2) scale32(v1);
           }
+          if (EXT && p.norm_mode != 0) {  // (gated: RMSNorm only, the column index is not used)
+            norm32(v0, (ci >> 1) * chunk_cols);
+            if (EPI == kEpiSiluGate || pieces == 2) norm32(v1, (ci >> 1) * chunk_cols + 32);
+          }
           // one 32-column piece: fused operation on packed FP32 pairs, rounding, into outw
           auto do_piece = [&](int piece, const uint32_t (&a)[32], const uint32_t (&up)[32]) {
             const int local0 = (ci >> 1) * chunk_cols + piece * 32;  // index among the warp's 128 columns
@@ -1114,11 +1208,32 @@ __global__ void __launch_bounds__(kThreads, 1)
                 scale32(v0);
                 scale32(v1);
               }
+              if (EXT && p.norm_mode != 0) {
+                norm32(v0, 0);
+                norm32(v1, 0);
+              }
               do_piece(1, v0, v1);
             }
           } else {
             do_piece(0, v0, v0);
             if (pieces == 2) do_piece(1, v1, v1);
+          }
+          if (EXT && p.stats_out != nullptr && !f32) {
+            // partial sums of this row's 64 stored values (as rounded), for a normalisation folded into the next product
+            uint64_t sum2 = 0ull, sq2 = 0ull;  // (even columns, odd columns)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const uint64_t y2 = ptx::bf16x2_to_f32x2(outw[i]);
+              sum2 = ptx::add_f32x2(sum2, y2);
+              sq2 = ptx::fma_f32x2(y2, y2, sq2);
+            }
+            uint32_t a0, a1, b0, b1;
+            ptx::unpack_f32x2(sum2, a0, a1);
+            ptx::unpack_f32x2(sq2, b0, b1);
+            const int row = row0 + lane;
+            if (row < p.M)
+              p.stats_out[(size_t)(n_chunk >> 6) * (size_t)p.M + row] =
+                  make_float2(__uint_as_float(a0) + __uint_as_float(a1), __uint_as_float(b0) + __uint_as_float(b1));
           }
           if (!use_r) {
             if (lane == 0) {
