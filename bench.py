@@ -194,7 +194,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped` or `blocks`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped`, `normfold` or `blocks`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     args = ap.parse_args()
@@ -236,12 +236,12 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        rows = [] if args.shape in ("attention", "blocks", "fp8", "grouped") else per_shape_table(
+        rows = [] if args.shape in ("attention", "blocks", "fp8", "grouped", "normfold") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
             side_ref=False, layout=args.layout)
         if args.shape in ("all", "attention"):
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
-        elif args.shape in ("blocks", "fp8", "grouped"):
+        elif args.shape in ("blocks", "fp8", "grouped", "normfold"):
             att = []
         else:  # attention shapes can be named like the GEMM shapes
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
@@ -255,15 +255,18 @@ def main():
         if args.shape in ("all", "fp8"):
             f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps,
                            side_ref=args.shape == "all")
-        elif names is not None and args.shape != "grouped":  # FP8 shapes can be named like the GEMM shapes
+        elif names is not None and args.shape not in ("grouped", "normfold"):  # FP8 shapes can be named like the GEMM shapes
             f8 = fp8_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps, side_ref=False,
                            names=names)
         grp = []
         if args.shape in ("all", "grouped"):
             grp = grouped_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps,
                                 side_ref=args.shape == "all")
+        nfold = []
+        if args.shape in ("all", "normfold"):
+            nfold = norm_fold_table(h, dev, stream, flush_l2, peaks, warm=args.warmup, iters=args.steps)
         print(json.dumps({"shapes": rows, "attention": att, "blocks": blk, "fp8": f8, "grouped": grp,
-                          "gpu_launches": h.launch_count()}))
+                          "norm_fold": nfold, "gpu_launches": h.launch_count()}))
         h.close()
         return 0
 
@@ -354,8 +357,9 @@ def main():
     tables = not args.no_shapes and rank == 0 and world == 1
     if tables:
         shapes = per_shape_table(h, dev, stream, flush_l2, peaks, args.tune)
-    attention, blocks, fp8, grouped = [], [], [], []
+    attention, blocks, fp8, grouped, norm_fold = [], [], [], [], []
     if tables:
+        norm_fold = norm_fold_table(h, dev, stream, flush_l2, peaks)
         attention = attention_table(h, dev, stream, flush_l2, peaks)
         fp8 = fp8_table(h, dev, stream, flush_l2, peaks)
         grouped = grouped_table(h, dev, stream, flush_l2, peaks)
@@ -396,6 +400,7 @@ def main():
             "attention": attention,
             "fp8": fp8,
             "grouped": grouped,
+            "norm_fold": norm_fold,
             "blocks": blocks,
         }
         print(json.dumps(line))
@@ -657,6 +662,85 @@ def grouped_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=Tr
         assert h.device_status() == 0
         del X, W, out
     return rows_out
+
+
+def norm_fold_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10):
+    """Output projection (+ residual) -> row normalisation -> first MLP layer, two ways: three launches (linear,
+    fact_norm, linear) and two (the producer leaves row sums, the consumer corrects its accumulator; the weights are
+    folded once, outside the timed region).  Chain times with L2 overwritten before each chain, and the SM cycles of
+    each product with and without the extras."""
+    import torch
+
+    from paper_2604_26666_b200 import workloads as wl
+
+    rows = []
+    for case in wl.norm_chain_cases():
+        t = wl.make_norm_chain_inputs(case, dev)
+        T, H, F = case.tokens, case.hidden, case.ffn
+        x1 = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
+        n = torch.empty_like(x1)
+        y = torch.empty((T, F), dtype=torch.bfloat16, device=dev)
+        stats = torch.empty((H // 64, T, 2), dtype=torch.float32, device=dev)
+        wf, cs, bf = h.fold_norm(t["w1"], t["gamma"], t.get("beta"), t.get("b1"))
+        colsum = None if case.gated else cs
+
+        def producer(with_sums):
+            h.linear(t["a"], t["wo"], bias=t.get("bo"), residual=t["x0"], epilogue="BIAS_RESIDUAL", out=x1,
+                     stats_out=stats if with_sums else None)
+
+        def consumer(folded):
+            if folded:
+                h.linear(x1, wf, bias=bf, epilogue=case.epilogue, out=y, x_norm=case.kind, x_stats=stats,
+                         w_colsum=colsum)
+            else:
+                h.linear(n, t["w1"], bias=t.get("b1"), epilogue=case.epilogue, out=y)
+
+        def unfused():
+            producer(False)
+            h.norm(x1, t["gamma"], t.get("beta"), kind=case.kind, out=n)
+            consumer(False)
+
+        def fused():
+            producer(True)
+            consumer(True)
+
+        def time_both(f0, f1):  # alternating, so that both see the same clocks
+            for _ in range(warm):
+                f0()
+                f1()
+            ts = ([], [])
+            for _ in range(iters):
+                for k, fn in enumerate((f0, f1)):
+                    flush_l2()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    fn()
+                    b.record(stream)
+                    ts[k].append((a, b))
+            torch.cuda.synchronize(dev)
+            return tuple(sorted(x.elapsed_time(z) for x, z in t) for t in ts)
+
+        def cycles(fn):
+            out = []
+            for _ in range(5):
+                flush_l2()
+                fn()
+                torch.cuda.synchronize(dev)
+                out.append(h.last_kernel_clock()[0])
+            return sorted(out)[2]
+
+        tu, tf = time_both(unfused, fused)
+        unfused()  # leaves n and stats-free x1 for the per-product cycle counts
+        rows.append({
+            "name": case.name, "tokens": T, "hidden": H, "ffn": F, "norm": case.kind, "epilogue": case.epilogue,
+            "us_three_launches": tu[len(tu) // 2] * 1e3, "us_two_launches": tf[len(tf) // 2] * 1e3,
+            "tflops_two_launches": case.flops / (tf[len(tf) // 2] * 1e-3) / 1e12,
+            "producer_cycles": cycles(lambda: producer(False)), "producer_cycles_with_sums": cycles(lambda: producer(True)),
+            "consumer_cycles": cycles(lambda: consumer(False)), "consumer_cycles_folded": cycles(lambda: consumer(True)),
+        })
+        assert h.device_status() == 0
+        del t, x1, n, y, wf
+    return rows
 
 
 def block_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=True):

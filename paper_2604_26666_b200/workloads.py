@@ -405,3 +405,51 @@ def make_grouped_inputs(case: GroupedCase, device="cpu"):
     for i in range(case.groups):
         W[i] = (torch.randn((case.n_weight_cols, case.K), generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
     return X, W
+
+
+# A row normalisation between two linear layers ("GEMM-LayerNorm-GEMM fusion" in the paper's Table 1): the paper
+# gives no shapes; these are the attention output projection -> norm -> first MLP layer of its two blocks
+# (Section 5.2), at the token counts of configurations 4 and 5.
+@dataclass(frozen=True)
+class NormChainCase:
+    name: str
+    tokens: int
+    hidden: int
+    ffn: int
+    kind: str       # "layer": LayerNorm, biases, GELU;  "rms": RMSNorm, no biases, SiLU-gated
+    seed: int = 0
+
+    @property
+    def gated(self) -> bool:
+        return self.kind == "rms"
+
+    @property
+    def epilogue(self) -> str:
+        return "SILU_GATE" if self.gated else "BIAS_GELU_TANH"
+
+    @property
+    def flops(self) -> float:
+        return 2.0 * self.tokens * self.hidden * (self.hidden + (2 if self.gated else 1) * self.ffn)
+
+
+def norm_chain_cases() -> list[NormChainCase]:
+    return [
+        NormChainCase("n_gpt2_out_ln_up", 16384, 768, 3072, "layer", seed=7400),
+        NormChainCase("n_llama_o_rms_gate_up", 8192, 4096, 14336, "rms", seed=7401),
+    ]
+
+
+def make_norm_chain_inputs(case: NormChainCase, device="cpu") -> dict:
+    """Attention output a and block input x0 ~ N(0,1) (x0 with a mean of 0.1: residual streams are not centred),
+    weights ~ N(0, 0.02^2), gamma ~ N(1, 0.1^2), beta and biases ~ N(0, 0.02^2); BF16, seeded, drawn on `device`."""
+    g = torch.Generator(device=device).manual_seed(case.seed)
+
+    def draw(shape, scale, shift=0.0):
+        return (torch.randn(shape, generator=g, device=device, dtype=torch.float32) * scale + shift).to(torch.bfloat16)
+
+    H, F, T = case.hidden, case.ffn, case.tokens
+    t = {"a": draw((T, H), 1.0), "x0": draw((T, H), 1.0, 0.1), "wo": draw((H, H), 0.02), "gamma": draw((H,), 0.1, 1.0),
+         "w1": draw(((2 * F) if case.gated else F, H), 0.02)}
+    if not case.gated:
+        t.update(bo=draw((H,), 0.02), beta=draw((H,), 0.02), b1=draw((F,), 0.02))
+    return t
