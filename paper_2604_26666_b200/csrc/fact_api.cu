@@ -128,7 +128,8 @@ int stage_bytes_for(int tile_n, int cta_group) { return (int)kStageBytesA + (til
 int epi_bufs_for(const Problem& q) { return (q.epi == FACT_EPI_BIAS_RESIDUAL && q.K <= 2048) ? 2 : 1; }
 
 int smem_bytes_for(const Problem& q, int tile_n, int cta_group, int stages) {
-  return stages * stage_bytes_for(tile_n, cta_group) + (int)epi_smem_bytes(epi_bufs_for(q)) + (int)kCtrlSmemBytes;
+  return stages * stage_bytes_for(tile_n, cta_group) + (int)epi_smem_bytes(epi_bufs_for(q)) + (int)kCtrlSmemBytes +
+         (q.norm == 1 ? (int)kNormCsBytes : 0);
 }
 
 int max_stages_for(const Problem& q, int tile_n, int cta_group) {
@@ -509,7 +510,7 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
   return FACT_OK;
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false, bool EXT = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0>
 fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                               cudaStream_t stream) {
   auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED, EXT>;
@@ -558,17 +559,19 @@ fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUten
   }
 }
 
-// The instantiations with row sums out / a folded row normalisation in (staged epilogue, data-parallel tiles).
-template <int CG>
+// The instantiations with row sums out (EXT 1) or a folded row normalisation in, with or without row sums out
+// (EXT 2): staged epilogue, data-parallel tiles.  Two sets, because the consumer's code slows the producer's
+// epilogue down even when it does not run.
+template <int CG, int EXT>
 fact_status_t launch_epi_ext(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
-  const int base = 32 + (CG - 1) * 8;
+  const int base = 32 + (EXT - 1) * 16 + (CG - 1) * 8;
   switch (epi) {
-    case kEpiNone: return launch_instance<CG, kEpiNone, false, false, true>(h, base + 0, plan, tm, stream);
-    case kEpiBias: return launch_instance<CG, kEpiBias, false, false, true>(h, base + 1, plan, tm, stream);
-    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, false, true>(h, base + 2, plan, tm, stream);
-    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, false, true>(h, base + 3, plan, tm, stream);
-    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, false, true>(h, base + 4, plan, tm, stream);
-    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, false, true>(h, base + 5, plan, tm, stream);
+    case kEpiNone: return launch_instance<CG, kEpiNone, false, false, EXT>(h, base + 0, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias, false, false, EXT>(h, base + 1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, false, EXT>(h, base + 2, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, false, EXT>(h, base + 3, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, false, EXT>(h, base + 4, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, false, EXT>(h, base + 5, plan, tm, stream);
     default: return FACT_ERR_UNSUPPORTED;
   }
 }
@@ -765,8 +768,10 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
     if (q.groups > 0) st = plan.cfg.cta_group == 2 ? launch_epi_grouped<2>(h, epi, plan, tm, stream)
                                                    : launch_epi_grouped<1>(h, epi, plan, tm, stream);
-    else if (q.stats_out || q.norm) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2>(h, epi, plan, tm, stream)
-                                                                 : launch_epi_ext<1>(h, epi, plan, tm, stream);
+    else if (q.norm) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 2>(h, epi, plan, tm, stream)
+                                                  : launch_epi_ext<1, 2>(h, epi, plan, tm, stream);
+    else if (q.stats_out) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 1>(h, epi, plan, tm, stream)
+                                                       : launch_epi_ext<1, 1>(h, epi, plan, tm, stream);
     else if (stream_k) st = plan.cfg.cta_group == 2 ? launch_epi_sk<2>(h, epi, plan, tm, stream)
                                                     : launch_epi_sk<1>(h, epi, plan, tm, stream);
     else if (plan.cfg.cta_group == 2) st = launch_epi<2>(h, epi, plan, tm, stream);

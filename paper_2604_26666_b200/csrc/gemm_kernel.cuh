@@ -48,6 +48,8 @@ constexpr uint32_t epi_smem_bytes(int bufs) { return kEpiWarps * ((uint32_t)bufs
 // Shared-memory layout (dynamic, 1024-byte aligned): [stage ring][epilogue staging][bias][mbarriers, flags]
 constexpr int kNumBarriers = 2 * kMaxStages + 4 + kEpiWarps * kEpiMaxBufs;
 constexpr uint32_t kCtrlSmemBytes = kNumBarriers * 8 + 16;
+// folded LayerNorm only: the FP32 column sums of each epilogue warp's 128 columns, behind the control words
+constexpr uint32_t kNormCsBytes = kEpiWarps * 128 * 4;
 
 // Epilogue selector of the kernel: the public enum plus the split-K partial store.
 enum : int {
@@ -589,7 +591,7 @@ __device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uin
   }
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false, bool EXT = false>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0>
 __global__ void __launch_bounds__(kThreads, 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
@@ -617,9 +619,11 @@ __global__ void __launch_bounds__(kThreads, 1)
       return;
     }
   }
-  if constexpr (EXT) {  // row sums out / a folded normalisation in: the staged epilogue of a whole, ungrouped tile
+  if constexpr (EXT != 0) {  // 1: row sums out; 2: a folded normalisation in (and row sums out) -- the staged
+                             // epilogue of a whole, ungrouped tile
     static_assert(!SK && !GROUPED && EPI != kEpiPartial && EPI != kEpiBiasSoftmax, "extras: plain data-parallel tiles");
-    if (!p.store_tma || (p.norm_mode != 0 && p.stats_in == nullptr) || (p.norm_mode == 1 && p.colsum == nullptr)) {
+    if (!p.store_tma || (EXT == 1 && p.norm_mode != 0) || (p.norm_mode != 0 && p.stats_in == nullptr) ||
+        (p.norm_mode == 1 && p.colsum == nullptr)) {
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
       return;
     }
@@ -643,6 +647,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t bias_base = epi_base + (uint32_t)(kEpiWarps * p.epi_bufs) * kEpiBufBytes;
   const uint32_t bar_base = bias_base + kEpiWarps * kEpiBiasBytes;
   const uint32_t ctrl_off = bar_base - smem_base + kNumBarriers * 8;
+  const uint32_t norm_cs_base = bar_base + kCtrlSmemBytes;  // (present only when the host asked for it: norm_mode 1)
   volatile uint32_t* tmem_holder_p = reinterpret_cast<volatile uint32_t*>(smem_raw + ctrl_off);
   volatile int* abort_p = reinterpret_cast<volatile int*>(smem_raw + ctrl_off + 4);
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
@@ -979,6 +984,40 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
           return true;
         };
+        // rows of A normalised over K: this thread's row scale (and scale times mean) come from the partial sums the
+        // producing call left, and the column sums of the folded weights for the warp's own 128 columns go to the
+        // warp's slice of shared memory (lane l fetches local columns 4l .. 4l+3).  Every load is issued here, ahead
+        // of the bias loads below, so that one trip to L2 serves them all; their values are used further down.
+        float nrm_rs = 1.f, nrm_rm = 0.f;
+        const uint32_t nrm_cs_s = norm_cs_base + (uint32_t)e * 512u;  // this warp's slice of the column sums
+        constexpr int kHeldSlots = 16;  // K <= 1024: the partial sums wait in registers until the accumulator is there
+        float2 nrm_held[kHeldSlots];
+        float nrm_s1 = 0.f, nrm_s2 = 0.f;
+        float4 nrm_cs4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (EXT == 2 && p.norm_mode != 0) {
+          const int row = row0 + lane;
+          const int slots = (p.K + 63) >> 6;
+          const float2* src = p.stats_in + min(row, p.M - 1);  // (rows past M compute a scale nobody stores)
+          if (p.norm_mode == 1) {
+            const int local = lane * 4;
+            const int ci = 2 * (local / chunk_cols) + half;
+            const int nc = n_tile0 + ci * chunk_cols + (local % chunk_cols);
+            if (ci < n_chunks && nc < p.N_out) nrm_cs4 = __ldg(reinterpret_cast<const float4*>(p.colsum + nc));
+          }
+          if (slots <= kHeldSlots) {
+            // a short main loop leaves these warps no idle time: the sums are added up only after the wait for the
+            // accumulator
+#pragma unroll
+            for (int u = 0; u < kHeldSlots; ++u)
+              nrm_held[u] = u < slots ? __ldg(src + (size_t)u * (size_t)p.M) : make_float2(0.f, 0.f);
+          } else {
+            for (int s = 0; s < slots; ++s) {
+              const float2 t = __ldg(src + (size_t)s * (size_t)p.M);
+              nrm_s1 += t.x;
+              nrm_s2 += t.y;
+            }
+          }
+        }
         // the bias values of this warp's own chunks, as BF16, into the warp's shared-memory slice
         if constexpr (epi_has_bias<EPI>()) {
           __syncwarp();
@@ -994,43 +1033,17 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
           __syncwarp();
         }
+        if (EXT == 2 && p.norm_mode == 1) {
+          __syncwarp();  // the previous tile's reads of the slice are done
+          ptx::st_shared_v4(nrm_cs_s + (uint32_t)lane * 16u, __float_as_uint(nrm_cs4.x), __float_as_uint(nrm_cs4.y),
+                            __float_as_uint(nrm_cs4.z), __float_as_uint(nrm_cs4.w));
+          __syncwarp();
+        }
         if (use_r && r_next <= gc && issue_residual(half, gc)) r_next = gc + 1;
         // with two buffers the residual tile of this warp's second chunk starts now as well (the stores that last read
         // the buffers are a whole main loop old): a load issued only after the first chunk's store leaves most of its
         // latency exposed, 3000 cycles per tile on the 768 -> 768 projection
         if (use_r && bufs == 2 && r_next == gc + 1 && issue_residual(half + 2, gc + 1, true)) r_next = gc + 2;
-        // rows of A normalised over K: this thread's row scale (and scale times mean) from the partial sums the
-        // producing call left, and the column sums of the folded weights for the warp's own 128 columns, four per
-        // lane (lane l holds local columns 4l .. 4l+3) -- all read while the main loop of the tile still runs
-        float nrm_rs = 1.f, nrm_rm = 0.f;
-        float4 nrm_cs = make_float4(0.f, 0.f, 0.f, 0.f);
-        constexpr int kHeldSlots = 16;  // K <= 1024: the partial sums wait in registers until the accumulator is there
-        float2 nrm_held[kHeldSlots];
-        float nrm_s1 = 0.f, nrm_s2 = 0.f;
-        if (EXT && p.norm_mode != 0) {
-          const int row = row0 + lane;
-          const int slots = (p.K + 63) >> 6;
-          const float2* src = p.stats_in + min(row, p.M - 1);  // (rows past M compute a scale nobody stores)
-          if (slots <= kHeldSlots) {
-            // a short main loop leaves these warps no idle time: issue the loads now, add them up after the wait
-            // for the accumulator, so that their trip to L2 is not on the tile's critical path
-#pragma unroll
-            for (int u = 0; u < kHeldSlots; ++u)
-              nrm_held[u] = u < slots ? __ldg(src + (size_t)u * (size_t)p.M) : make_float2(0.f, 0.f);
-          } else {
-            for (int s = 0; s < slots; ++s) {
-              const float2 t = __ldg(src + (size_t)s * (size_t)p.M);
-              nrm_s1 += t.x;
-              nrm_s2 += t.y;
-            }
-          }
-          if (p.norm_mode == 1) {
-            const int local = lane * 4;
-            const int ci = 2 * (local / chunk_cols) + half;
-            const int nc = n_tile0 + ci * chunk_cols + (local % chunk_cols);
-            if (ci < n_chunks && nc < p.N_out) nrm_cs = __ldg(reinterpret_cast<const float4*>(p.colsum + nc));
-          }
-        }
         auto norm_finish = [&]() {
           if (((p.K + 63) >> 6) <= kHeldSlots) {
 #pragma unroll
@@ -1050,13 +1063,11 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint64_t rs2 = ptx::pack_f32x2(__float_as_uint(nrm_rs), __float_as_uint(nrm_rs));
           if (p.norm_mode == 1) {
             const uint64_t rm2 = ptx::pack_f32x2(__float_as_uint(-nrm_rm), __float_as_uint(-nrm_rm));
-            const int src0 = local0 >> 2;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              const float cx = __shfl_sync(0xffffffffu, nrm_cs.x, src0 + j), cy = __shfl_sync(0xffffffffu, nrm_cs.y, src0 + j);
-              const float cz = __shfl_sync(0xffffffffu, nrm_cs.z, src0 + j), cw = __shfl_sync(0xffffffffu, nrm_cs.w, src0 + j);
-              const uint64_t t0 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(__float_as_uint(cx), __float_as_uint(cy)));
-              const uint64_t t1 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(__float_as_uint(cz), __float_as_uint(cw)));
+              const uint4 c = ptx::ld_shared_v4(nrm_cs_s + (uint32_t)(local0 + 4 * j) * 4u);  // a broadcast read
+              const uint64_t t0 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(c.x, c.y));
+              const uint64_t t1 = ptx::mul_f32x2(rm2, ptx::pack_f32x2(c.z, c.w));
               ptx::unpack_f32x2(ptx::fma_f32x2(rs2, ptx::pack_f32x2(v[4 * j], v[4 * j + 1]), t0), v[4 * j], v[4 * j + 1]);
               ptx::unpack_f32x2(ptx::fma_f32x2(rs2, ptx::pack_f32x2(v[4 * j + 2], v[4 * j + 3]), t1), v[4 * j + 2],
                                 v[4 * j + 3]);
@@ -1076,7 +1087,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (prof) prof_epi_wait += tb - tw;
         ptx::tc_fence_after();
         const uint32_t t_acc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.tile_n);
-        if (EXT && p.norm_mode != 0) norm_finish();
+        if (EXT == 2 && p.norm_mode != 0) norm_finish();
         if constexpr (SK) {
           // the first piece of a tile: the same warp of the same CTA rank in each of the following groups parks
           // the rest of the sum; wait until those are complete (they precede everything else those groups do)
@@ -1148,7 +1159,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             scale32(v0);
             if (EPI == kEpiSiluGate || pieces == 2) scale32(v1);
           }
-          if (EXT && p.norm_mode != 0) {  // (gated: RMSNorm only, the column index is not used)
+          if (EXT == 2 && p.norm_mode != 0) {  // (gated: RMSNorm only, the column index is not used)
             norm32(v0, (ci >> 1) * chunk_cols);
             if (EPI == kEpiSiluGate || pieces == 2) norm32(v1, (ci >> 1) * chunk_cols + 32);
           }
@@ -1208,7 +1219,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 scale32(v0);
                 scale32(v1);
               }
-              if (EXT && p.norm_mode != 0) {
+              if (EXT == 2 && p.norm_mode != 0) {
                 norm32(v0, 0);
                 norm32(v1, 0);
               }
@@ -1218,7 +1229,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             do_piece(0, v0, v0);
             if (pieces == 2) do_piece(1, v1, v1);
           }
-          if (EXT && p.stats_out != nullptr && !f32) {
+          if (EXT != 0 && p.stats_out != nullptr && !f32) {
             // partial sums of this row's 64 stored values (as rounded), for a normalisation folded into the next product
             uint64_t sum2 = 0ull, sq2 = 0ull;  // (even columns, odd columns)
 #pragma unroll
