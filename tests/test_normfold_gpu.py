@@ -76,6 +76,8 @@ PRODUCERS = [
     (1024, 384, 256, "SILU_GATE", dict(tile_n=256)),        # (the default tile, 96 output columns, is not stageable)
     (2048, 2304, 768, "BIAS_RESIDUAL", dict(split_k=-1)),   # a stream-K request is dropped: the tiles run whole
     (4224, 768, 768, "BIAS_RESIDUAL", None),
+    (300, 200, 128, "BIAS_RESIDUAL", None),               # the last chunk holds 8 columns: the others add zeros
+    (5, 64, 72, "BIAS_RELU", None),                       # fewer rows than a warp owns
 ]
 
 
