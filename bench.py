@@ -622,8 +622,13 @@ def grouped_table(h, dev, stream, flush_l2, peaks, warm=3, iters=10, side_ref=Tr
         for r in rows:
             offs.append(offs[-1] + r)
 
+        bias = None
+        if case.epilogue.startswith("BIAS"):
+            gb = torch.Generator(device=dev).manual_seed(case.seed + 2)
+            bias = (torch.randn((case.N,), generator=gb, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+
         def call():
-            h.linear_grouped(X, W, rows, epilogue=case.epilogue, out=out)
+            h.linear_grouped(X, W, rows, bias=bias, epilogue=case.epilogue, out=out)
 
         def side():
             for g in range(case.groups):

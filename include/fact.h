@@ -238,10 +238,12 @@ fact_status_t fact_linear(fact_handle_t handle, int64_t M, int64_t N_out, int64_
  * X: BF16 [M x K], ldx.  W[g]: BF16 at W + g * strideW elements, [Nw x K] (FACT_B_NK) or [K x Nw] (FACT_B_KN), ldw;
  * strideW a multiple of 8.  bias [N_out] (shared by the groups), residual [M x N_out], Y, out_type, epilogue as in
  * fact_linear.  One launch: tiles never cross a group boundary (the last tile of a group is ragged), all tiles are
- * data-parallel, the output is stored by row-predicated register stores (the group table travels to a buffer of
+ * data-parallel, the output is stored by row-predicated 16-byte stores -- staged through shared memory so that
+ * they are whole 128-byte rows when Y is 16-byte aligned with ldy and N_out multiples of 16 bytes, straight from
+ * registers otherwise or with cfg->store_mode == 1 (the group table travels to a buffer of
  * the handle in stream order, so grouped calls through one handle must be stream-ordered with respect to each
  * other, and not inside a stream capture: the table is copied from pageable host memory).  cfg: tile shape, pair
- * size and stages only (K slices, stream-K, staged stores and the row softmax are refused with
+ * size, stages and store mode only (K slices, stream-K and the row softmax are refused with
  * FACT_ERR_UNSUPPORTED).  groups == 0 or M == 0 is a successful no-op. */
 fact_status_t fact_linear_grouped(fact_handle_t handle, int groups, const int64_t* group_rows, int64_t N_out, int64_t K,
                                   const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t strideW,

@@ -656,7 +656,13 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     // goes to the handle's device buffer in stream order.
     fact_config_t gc = plan.cfg;
     gc.split_k = 1;
-    gc.store_mode = 1;
+    // staged through shared memory (then the warp's own row-predicated 16-byte stores) when the output's rows are
+    // whole 16-byte pieces; otherwise straight from registers
+    const bool whole16 = q.N_out % (q.out == FACT_OUT_F32 ? 4 : 8) == 0;
+    if (!whole16 || !plan.p.store_tma) {
+      if (user && user->store_mode == 2) return FACT_ERR_UNSUPPORTED;
+      gc.store_mode = 1;
+    }
     st = make_plan(h, q, &gc, 0, &plan);
     if (st != FACT_OK) return st;
     const int G = q.groups;
@@ -1063,7 +1069,7 @@ static fact_status_t linear_grouped_impl(fact_handle_t h, bool fp8, float scale,
     if (M > 0x7fffffffLL - 512) return FACT_ERR_INVALID_ARG;
   }
   if (groups == 0 || M == 0) return FACT_OK;
-  if (cfg && (cfg->split_k > 1 || cfg->split_k < 0 || cfg->store_mode == 2)) return FACT_ERR_UNSUPPORTED;
+  if (cfg && (cfg->split_k > 1 || cfg->split_k < 0)) return FACT_ERR_UNSUPPORTED;
   if (epi == FACT_EPI_BIAS_SOFTMAX) return FACT_ERR_UNSUPPORTED;
   Problem q = make_problem(fp8 ? FACT_OP_LINEAR_FP8 : FACT_OP_LINEAR, 1, M, N_out, K, X, ldx, 0, W, ldw, strideW, layout,
                            bias, residual, ldr, 0, Y, ldy, 0, out, epi);

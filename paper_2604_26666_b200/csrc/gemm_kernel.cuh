@@ -612,9 +612,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
   }
-  if constexpr (GROUPED) {  // group boundaries are kept by the row-predicated direct stores only
+  if constexpr (GROUPED) {  // (group boundaries are kept by row-predicated stores, staged or direct)
     static_assert(!SK && EPI != kEpiPartial, "grouped tiles are data-parallel");
-    if (p.store_tma || p.grp_tiles == nullptr || p.grp_rows == nullptr) {
+    if (p.grp_tiles == nullptr || p.grp_rows == nullptr) {
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
       return;
     }
@@ -946,7 +946,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             continue;
           }
         }
-        const int row0 = (w.tm * CG + (int)cta_rank) * kTileM + q * 32;
+        const int row0 = (GROUPED ? w.m_base : 0) + (w.tm * CG + (int)cta_rank) * kTileM + q * 32;
         const int n_tile0 = w.tn * p.out_cols;
         const int acc_cols = (EPI == kEpiPartial) ? p.tile_n : p.out_cols;
         const int n_chunks = acc_cols / chunk_cols;
@@ -965,7 +965,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             z = (w.split * p.batch + w.b) * p.ws_planes + plane;
           } else {
             n = n_tile0 + c;
-            z = w.b;
+            z = GROUPED ? 0 : w.b;  // (grouped: w.b selects the weights; the rows of C and R are one matrix)
           }
           return ci < n_chunks && n < p.N_out;
         };
@@ -1259,9 +1259,30 @@ __global__ void __launch_bounds__(kThreads, 1)
                               outw[4 * j + 2], outw[4 * j + 3]);
           ptx::fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) {
-            if (row0 < p.M && !(p.debug & 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
-            ptx::bulk_commit_group();
+          if constexpr (GROUPED) {
+            // A tensor store would run over the end of the group into the next group's rows: the warp writes the
+            // chunk itself, four whole 128-byte rows per instruction (eight lanes a row), rows past the end left out.
+            const int rows_left = w.m_end - row0;  // (<= 0: this warp's rows all lie past the group)
+            const int piece = lane & 7, rsub = lane >> 3;
+            const int elems16 = f32 ? 4 : 8;
+            const int col = n_chunk + piece * elems16;
+            const bool col_ok = col + elems16 <= p.N_out;  // (N_out is a multiple of 16 bytes on this path)
+            uint8_t* const out_b = reinterpret_cast<uint8_t*>(p.C) +
+                                   ((long long)row0 * p.ldc + col) * (long long)(f32 ? 4 : 2);
+            const long long row_bytes = p.ldc * (long long)(f32 ? 4 : 2);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int r = 4 * j + rsub;
+              const uint4 v = ptx::ld_shared_v4(buf + (uint32_t)r * 128u + ((uint32_t)(piece ^ (r & 7)) << 4));
+              if (r < rows_left && col_ok && !(p.debug & 4)) *reinterpret_cast<uint4*>(out_b + r * row_bytes) = v;
+            }
+            ptx::fence_proxy_async_smem();  // (a residual tile may be loaded into this buffer next, by TMA)
+            __syncwarp();
+          } else {
+            if (lane == 0) {
+              if (row0 < p.M && !(p.debug & 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
+              ptx::bulk_commit_group();
+            }
           }
           // with two buffers the next residual tile can start now: its buffer's last store is one chunk old
           if (use_r && bufs == 2 && r_next <= gc + 1 && issue_residual(ci + 2, gc + 1)) r_next = gc + 2;

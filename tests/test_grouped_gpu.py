@@ -60,6 +60,9 @@ CASES = [
     ("silu_gate", [260, 120, 400], 256, 192, "SILU_GATE", "NK", None),
     ("residual", [129, 511, 64], 384, 256, "BIAS_RESIDUAL", "NK", None),
     ("kn_layout", [200, 333, 90], 320, 256, "BIAS", "KN", None),
+    ("direct_stores", [200, 1, 130, 128, 515], 384, 264, "BIAS_RESIDUAL", "NK", dict(store_mode=1)),
+    ("direct_odd_width", [90, 400, 33], 203, 96, "BIAS", "NK", None),     # rows of 406 bytes: registers only
+    ("staged_residual_pairs", [300, 256, 1, 255, 257], 512, 256, "BIAS_RESIDUAL", "NK", dict(tile_n=256, cta_group=2)),
 ]
 
 
@@ -123,7 +126,8 @@ def test_grouped_argument_errors(h):
     assert call(2, [128, 128], stride_w=N * K + 4) == 2   # stride not a multiple of 8 elements
     assert call(2, [128, 128], cfg=ctypes.byref(Config(split_k=2))) == 3
     assert call(2, [128, 128], cfg=ctypes.byref(Config(split_k=-1))) == 3
-    assert call(2, [128, 128], cfg=ctypes.byref(Config(store_mode=2))) == 3
+    assert call(2, [128, 128], cfg=ctypes.byref(Config(store_mode=2))) == 0   # staged: rows of whole 16-byte pieces
+    assert call(2, [128, 128], cfg=ctypes.byref(Config(store_mode=1))) == 0   # straight from registers
     torch.cuda.synchronize()
     assert h.device_status() == 0
 
@@ -160,3 +164,30 @@ def test_grouped_fp8_matches_oracle(h, epi, cfg):
         r0 += n
     c, t = gates(ref, to_f64(out), "bf16", epi)
     assert c <= 1.0 and t <= 1.0, (c, t)
+
+
+def test_grouped_benchmark_shape_sampled_rows(h):
+    """The short-K grouped shape of the benchmark's table at full size, in the configuration the benchmark times
+    (staged stores): rows sampled at every group boundary and in between, each against the oracle."""
+    case = [c for c in wl.grouped_cases() if c.name == "g8_short_k_gelu"][0]
+    rows = wl.grouped_rows(case)
+    X, W = wl.make_grouped_inputs(case, "cuda:0")
+    gb = torch.Generator(device="cuda:0").manual_seed(case.seed + 2)
+    bias = (torch.randn((case.N,), generator=gb, device="cuda:0", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    out = h.linear_grouped(X, W, rows, bias=bias, epilogue=case.epilogue)
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    starts = np.concatenate([[0], np.cumsum(rows)])
+    rng = np.random.default_rng(5)
+    worst_c = worst_t = 0.0
+    Xc, bc = X.cpu(), bias.cpu()
+    for g, n in enumerate(rows):
+        if n == 0:
+            continue
+        local = sorted({0, n - 1, n // 2, *rng.integers(0, n, size=4).tolist()})
+        idx = [int(starts[g]) + r for r in local]
+        ref = oracle.linear(wl.bits(Xc[idx].contiguous()), wl.bits(W[g].cpu()), layout="NK", epilogue=case.epilogue,
+                            bias=wl.bits(bc))
+        c, t = gates(ref, to_f64(out[idx]), "bf16", case.epilogue)
+        worst_c, worst_t = max(worst_c, c), max(worst_t, t)
+    assert worst_c <= 1.0 and worst_t <= 1.0, (worst_c, worst_t)
