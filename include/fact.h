@@ -127,7 +127,11 @@ typedef enum {
  *                (whole waves, K == 0, an output the staged store cannot write) the call is data-parallel.
  *                Stream-K calls through one handle must be stream-ordered with respect to each other (they share
  *                the handle's flags) and must not share a workspace while they overlap.
- *   store_mode   0 = library default, 1 = direct register stores, 2 = shared-memory staged stores */
+ *   store_mode   0 = library default, 1 = direct register stores (any alignment), 2 = shared-memory staged
+ *                tensor stores, 3 = the staged epilogue's arithmetic with every row stored from registers in
+ *                32-byte pieces (Y 32-byte aligned, ldy and N_out multiples of 32 bytes, whole data-parallel
+ *                tiles: no K slices, stream-K, groups or row sums; pays when K is long, FACT_ERR_UNSUPPORTED
+ *                where it cannot run) */
 typedef struct {
   int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode;
 } fact_config_t;

@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <bitset>
 #include <map>
 #include <string>
 #include <tuple>
@@ -93,7 +94,7 @@ struct fact_handle_s {
   EncodeTiledFn encode = nullptr;
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
-  unsigned long long configured_mask = 0;  // kernels whose dynamic shared-memory limit was raised
+  std::bitset<128> configured_mask;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
   int* d_groups = nullptr;       // grouped GEMM: m-tile prefix and row offsets of the call in flight
@@ -268,7 +269,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   }
   if (c.split_k < -2) return FACT_ERR_INVALID_ARG;
   if (c.split_k > 0) c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
-  if (c.store_mode < 0 || c.store_mode > 2) return FACT_ERR_INVALID_ARG;
+  if (c.store_mode < 0 || c.store_mode > 3) return FACT_ERR_INVALID_ARG;
   *out = c;
   return FACT_OK;
 }
@@ -333,7 +334,7 @@ int sk_tiles_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
   const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
   // the pieces are parked and finished by the staged epilogue, which stores whole 128-byte chunks per tile
   const bool f32 = q.out == FACT_OUT_F32;
-  if (out_cols % (f32 ? 32 : 64) != 0 || (f32 && q.epi == FACT_EPI_BIAS_RESIDUAL) || c.store_mode == 1) return 0;
+  if (out_cols % (f32 ? 32 : 64) != 0 || (f32 && q.epi == FACT_EPI_BIAS_RESIDUAL) || c.store_mode == 1 || c.store_mode == 3) return 0;
   const long long tiles = q.batch * ((q.M + c.tile_m - 1) / c.tile_m) * ((q.N_out + out_cols - 1) / out_cols);
   const long long groups = std::max(1, h->sm_count / c.cta_group);
   const long long k_blocks = (q.K + q.k_elems() - 1) / q.k_elems();
@@ -453,9 +454,22 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   const bool can_stage = p.c_vec && (p.out_cols % chunk_cols == 0) &&
                          !(p.out_f32 && q.epi == FACT_EPI_BIAS_RESIDUAL);
   if (c.store_mode == 2 && !can_stage) return FACT_ERR_UNSUPPORTED;
+  const int asked_store = c.store_mode;  // (c aliases plan->cfg, which is rewritten below)
   p.store_tma = (c.store_mode == 1) ? 0 : (can_stage ? 1 : 0);
   p.r_tma = p.store_tma && q.epi == FACT_EPI_BIAS_RESIDUAL && p.r_vec;
   plan->cfg.store_mode = p.store_tma ? 2 : 1;
+  if (asked_store == 3) {
+    // the staged epilogue's arithmetic with each row stored from registers in 32-byte pieces: whole, unsliced,
+    // ungrouped tiles whose output rows are 32-byte aligned multiples of 32 bytes
+    const long long esz = p.out_f32 ? 4 : 2;
+    const bool rows32 = (reinterpret_cast<uintptr_t>(q.C) & 31u) == 0 && (q.ldc * esz) % 32 == 0 &&
+                        (q.N_out * esz) % 32 == 0 && (q.batch <= 1 || (q.strideC * esz) % 32 == 0);
+    if (!can_stage || !rows32 || c.split_k != 1 || q.groups > 0 || q.stats_out || q.norm ||
+        q.epi == FACT_EPI_BIAS_SOFTMAX)
+      return FACT_ERR_UNSUPPORTED;
+    p.row_stores = 1;
+    plan->cfg.store_mode = 3;
+  }
   // row sums out and the folded normalisation live in the staged epilogue of an unsliced product
   if ((q.stats_out || q.norm) && (!p.store_tma || c.split_k > 1)) return FACT_ERR_UNSUPPORTED;
   p.stats_out = reinterpret_cast<float2*>(q.stats_out);
@@ -517,10 +531,10 @@ fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const
   if (slot < 0) {  // (no bit left in the handle's mask for these instantiations: set the attribute on every launch)
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-  } else if (!(h->configured_mask & (1ull << slot))) {
+  } else if (!h->configured_mask.test((size_t)slot)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-    h->configured_mask |= (1ull << slot);
+    h->configured_mask.set((size_t)slot);
   }
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof lc);
@@ -559,8 +573,8 @@ fact_status_t launch_epi(fact_handle_t h, int epi, const Plan& plan, const CUten
   }
 }
 
-// The instantiations with row sums out (EXT 1) or a folded row normalisation in, with or without row sums out
-// (EXT 2): staged epilogue, data-parallel tiles.  Two sets, because the consumer's code slows the producer's
+// The instantiations with row sums out (EXT 1), a folded row normalisation in, with or without row sums out
+// (EXT 2), or rows stored from registers in 32-byte pieces (EXT 3): staged epilogue, data-parallel tiles.  Two sets, because the consumer's code slows the producer's
 // epilogue down even when it does not run.
 template <int CG, int EXT>
 fact_status_t launch_epi_ext(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
@@ -774,6 +788,8 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
     if (q.groups > 0) st = plan.cfg.cta_group == 2 ? launch_epi_grouped<2>(h, epi, plan, tm, stream)
                                                    : launch_epi_grouped<1>(h, epi, plan, tm, stream);
+    else if (plan.p.row_stores && !split) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 3>(h, epi, plan, tm, stream)
+                                                                       : launch_epi_ext<1, 3>(h, epi, plan, tm, stream);
     else if (q.norm) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 2>(h, epi, plan, tm, stream)
                                                   : launch_epi_ext<1, 2>(h, epi, plan, tm, stream);
     else if (q.stats_out) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 1>(h, epi, plan, tm, stream)
@@ -1164,6 +1180,11 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
         for (int sp : splits) {
           fact_config_t c = {128 * cg, tn, q.k_elems(), stg, cg, 0, sp, 0};
           cands.push_back(c);
+          // whole tiles with a long main loop: also with the rows stored from registers (infeasible ones drop out)
+          if (sp == 1 && k_blocks >= 32) {
+            c.store_mode = 3;
+            cands.push_back(c);
+          }
         }
     }
   }
@@ -1360,7 +1381,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     p.items = (int)items;
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
-    if (!(h->configured_mask & (1ull << 30))) {
+    if (!h->configured_mask.test(30)) {
       cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -1376,7 +1397,7 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
                         std::to_string(kAttnRegsAtLaunch);
         st = FACT_ERR_UNSUPPORTED;
       } else {
-        h->configured_mask |= (1ull << 30);
+        h->configured_mask.set(30);
       }
     }
     if (st == FACT_OK) {

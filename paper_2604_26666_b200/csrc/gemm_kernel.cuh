@@ -138,6 +138,9 @@ struct GemmParams {
   const float* colsum;     // [N_out]: sum over k of the folded W[n][k] (LayerNorm only)
   int norm_mode;
   float norm_eps;
+  // EXT = 3 instantiations: the staged epilogue's arithmetic, but every thread stores its own row's 128 bytes of a
+  // chunk straight from registers as four 32-byte stores (no staging traffic through shared memory)
+  int row_stores;
   // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
   // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
   int debug;
@@ -619,15 +622,16 @@ __global__ void __launch_bounds__(kThreads, 1)
       return;
     }
   }
-  if constexpr (EXT != 0) {  // 1: row sums out; 2: a folded normalisation in (and row sums out) -- the staged
-                             // epilogue of a whole, ungrouped tile
+  if constexpr (EXT != 0) {  // 1: row sums out; 2: a folded normalisation in (and row sums out); 3: rows stored
+                             // from registers -- all in the staged epilogue of a whole, ungrouped tile
     static_assert(!SK && !GROUPED && EPI != kEpiPartial && EPI != kEpiBiasSoftmax, "extras: plain data-parallel tiles");
-    if (!p.store_tma || (EXT == 1 && p.norm_mode != 0) || (p.norm_mode != 0 && p.stats_in == nullptr) ||
-        (p.norm_mode == 1 && p.colsum == nullptr)) {
+    if (!p.store_tma || (EXT != 2 && p.norm_mode != 0) || (p.norm_mode != 0 && p.stats_in == nullptr) ||
+        (p.norm_mode == 1 && p.colsum == nullptr) || (EXT == 3) != (p.row_stores != 0) ||
+        (EXT == 3 && p.stats_out != nullptr)) {
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
       return;
     }
-  } else if (p.norm_mode != 0 || p.stats_out != nullptr) {  // asked of an instantiation that has no code for it
+  } else if (p.norm_mode != 0 || p.stats_out != nullptr || p.row_stores != 0) {  // asked of an instantiation that has no code for it
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
   }
@@ -1229,7 +1233,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             do_piece(0, v0, v0);
             if (pieces == 2) do_piece(1, v1, v1);
           }
-          if (EXT != 0 && p.stats_out != nullptr && !f32) {
+          if ((EXT == 1 || EXT == 2) && p.stats_out != nullptr && !f32) {
             // partial sums of this row's 64 stored values (as rounded), for a normalisation folded into the next product
             uint64_t sum2 = 0ull, sq2 = 0ull;  // (even columns, odd columns)
 #pragma unroll
@@ -1245,6 +1249,23 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (row < p.M)
               p.stats_out[(size_t)(n_chunk >> 6) * (size_t)p.M + row] =
                   make_float2(__uint_as_float(a0) + __uint_as_float(a1), __uint_as_float(b0) + __uint_as_float(b1));
+          }
+          if constexpr (EXT == 3) {
+            // The row leaves straight from registers: four 32-byte stores, each a whole sector of its own.  A long
+            // main loop hides their scatter (32 rows per instruction), and the 128 KB per tile that staging writes to
+            // and reads from shared memory no longer compete with the operand reads of the tensor pipe.
+            const int row = row0 + lane;
+            if (row < p.M && !(p.debug & 4)) {
+              uint8_t* dst = reinterpret_cast<uint8_t*>(p.C) +
+                             ((long long)z * p.strideC + (long long)row * p.ldc + n_chunk) * (long long)(f32 ? 4 : 2);
+              const int e32 = f32 ? 8 : 16;  // elements in 32 bytes (N_out is a multiple of it on this path)
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                if (n_chunk + (j + 1) * e32 <= p.N_out) ptx::st_global_v8(dst + 32 * j, &outw[8 * j]);
+            }
+            if (use_r && bufs == 2 && r_next <= gc + 1 && issue_residual(ci + 2, gc + 1)) r_next = gc + 2;
+            ++gc;
+            continue;
           }
           if (!use_r) {
             if (lane == 0) {

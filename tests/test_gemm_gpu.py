@@ -123,6 +123,37 @@ def test_stage_counts(h, stages):
     check_case(h, case, cfg={"tile_n": 128, "stages": stages})
 
 
+ROW_STORE_EPI = ["NONE", "BIAS", "BIAS_RELU", "BIAS_GELU_TANH", "SILU_GATE", "BIAS_RESIDUAL"]
+
+
+@pytest.mark.parametrize("epi", ROW_STORE_EPI)
+@pytest.mark.parametrize("out", ["bf16", "f32"])
+def test_register_row_stores(h, epi, out):
+    """store_mode 3: the staged epilogue's arithmetic, rows stored from registers in 32-byte pieces.  Ragged M, two
+    n-tiles with the second one partly past N, K not a multiple of 64; N a multiple of 32 bytes."""
+    if out == "f32" and epi == "BIAS_RESIDUAL":
+        pytest.skip("an FP32 output with a residual is not stageable")
+    case = mk(f"rs_{epi}", 300, 336, 520, epilogue=epi, layout="NK", out=out, w_scale=0.05)
+    check_case(h, case, cfg={"store_mode": 3, "tile_n": 256, "cta_group": 2})
+    check_case(h, case, cfg={"store_mode": 3, "tile_n": 128, "cta_group": 1})
+
+
+def test_register_row_stores_exact_batched_and_refusals(h):
+    from paper_2604_26666_b200.binding import FactError
+    case = mk("rs_int", 260, 256, 200, epilogue="BIAS_RESIDUAL", layout="KN", out="bf16")
+    bit_exact(h, case, small_int_inputs(case, 11, lo=-2, hi=2), cfg={"store_mode": 3})
+    caseb = mk("rs_batched", 200, 192, 136, op="gemm_batched", layout="NK", batch=3)
+    check_case(h, caseb, cfg={"store_mode": 3})
+    # refusals: rows that are not whole 32-byte pieces, K slices, stream-K
+    for bad_case, cfg in ((mk("rs_n", 128, 200, 128, layout="NK"), {"store_mode": 3}),
+                          (mk("rs_sp", 128, 256, 1024, layout="NK"), {"store_mode": 3, "split_k": 2}),
+                          (mk("rs_sk", 300, 2304, 768, layout="NK"), {"store_mode": 3, "split_k": -1})):
+        with pytest.raises(FactError) as e:
+            run_gpu(h, wl.make_inputs(bad_case), bad_case, cfg=cfg)
+        assert e.value.code == 3
+    assert h.device_status() == 0
+
+
 def test_unaligned_output_and_odd_sizes(h):
     # N odd: rows of C are not 16-byte aligned -> element-wise stores
     for (M, N, K) in [(1, 1, 8), (5, 7, 24), (129, 33, 72), (64, 250, 136)]:
