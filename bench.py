@@ -39,9 +39,8 @@ WORKLOAD = "config 2: square BF16 GEMM 4096^3 + 8192^3, N(0,1)/sqrt(K), seed 1"
 L2_FLUSH_BYTES = 512 << 20
 
 # DRAM traffic per launch of the dominant kernel (8192^3): dram__bytes_read.sum + dram__bytes_write.sum of the
-# ncu capture summarised in profiles/all_shapes_counters.md (916.6 MB + 126.8 MB; it was 1.0745 GB + 127.2 MB in
-# profiles/fact_gemm_kernel_c2_square_8192.md, before every second tile walked K downwards).
-DOMINANT_TRAFFIC_BYTES = 1.0434e9
+# latest ncu capture in profiles/fact_gemm_kernel_c2_square_8192.md (933.4 MB + 126.5 MB, mean of two launches).
+DOMINANT_TRAFFIC_BYTES = 1.0599e9
 
 
 def load_peaks():
