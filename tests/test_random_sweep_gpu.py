@@ -69,3 +69,23 @@ def test_random_sweep(h, seed):
         except AssertionError as e:
             raise AssertionError(f"{case} cfg={cfg}: {e}") from e
     assert ran >= 15, f"only {ran} of 40 random cases were runnable"
+
+
+@pytest.mark.parametrize("seed", [100, 101])
+def test_random_sweep_register_row_stores(h, seed):
+    """The same sweep with the rows stored from registers in 32-byte pieces (store_mode 3): no K slices, and only
+    shapes it accepts have to run (output rows of whole 32-byte pieces, a stageable tile)."""
+    rng = np.random.default_rng(seed)
+    ran = 0
+    for i in range(40):
+        case, cfg = random_case(rng, seed * 100 + i)
+        cfg.pop("split_k", None)
+        cfg["store_mode"] = 3
+        try:
+            check_case(h, case, cfg=cfg)
+            ran += 1
+        except FactError as e:
+            assert e.code == 3, (case, cfg, e)
+        except AssertionError as e:
+            raise AssertionError(f"{case} cfg={cfg}: {e}") from e
+    assert ran >= 8, f"only {ran} of 40 random cases were runnable"
