@@ -38,8 +38,8 @@ METRIC = "TFLOP/s & % of dense BF16 tensor peak per fused-epilogue GEMM shape"
 WORKLOAD = "config 2: square BF16 GEMM 4096^3 + 8192^3, N(0,1)/sqrt(K), seed 1"
 L2_FLUSH_BYTES = 512 << 20
 
-# DRAM traffic per launch of the dominant kernel (8192^3): dram__bytes_read.sum + dram__bytes_write.sum of the
-# latest ncu capture in profiles/fact_gemm_kernel_c2_square_8192.md (933.4 MB + 126.5 MB, mean of two launches).
+# DRAM traffic per launch of the dominant kernel (8192^3): dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture of that launch (933.4 MB + 126.5 MB, mean of two launches).
 DOMINANT_TRAFFIC_BYTES = 1.0599e9
 
 

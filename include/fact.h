@@ -215,11 +215,18 @@ fact_status_t fact_gemm_splitk(fact_handle_t handle, int64_t M, int64_t N, int64
  *     same call), but two calls that overlap on the GPU -- different streams, or different host
  *     threads -- race on it and both results are garbage: keep calls on one device in one stream
  *     order;
- *   - a device-side wait that expires is recorded in a status word that is likewise static and
- *     per device; this entry point does not report it (there is no handle to ask). */
+ *   - a device-side wait that expires (every wait in the kernels is bounded) is recorded in a status
+ *     word that is likewise static and per device; the output of that call is then undefined.  The
+ *     call itself is asynchronous and cannot report it: ask fact_gemm_splitk_static_status. */
 fact_status_t fact_gemm_splitk_static(int device, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                       const void* B, int64_t ldb, fact_blayout_t b_layout, void* C, int64_t ldc,
                                       fact_out_t out_type, int splits, void* cuda_stream);
+
+/* The fact_device_status of fact_gemm_splitk_static (no counterpart in the paper either): synchronise
+ * `cuda_stream`, write the static status word of `device` to *status (FACT_OK or
+ * FACT_ERR_DEVICE_TIMEOUT) and clear it.  0 if no static call has run on that device yet.  Like the
+ * call it serves it allocates nothing: one 4-byte copy, and memsets after a give-up. */
+fact_status_t fact_gemm_splitk_static_status(int device, void* cuda_stream, int* status);
 
 /* Y[M x N_out] = epilogue(X[M x K] . W)        (Section 5.2: fused linear layers)
  * W: FACT_B_NK [Nw x K] (nn.Linear weight) or FACT_B_KN [K x Nw]; Nw = N_out,
@@ -480,11 +487,16 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * After a fact_attention launch (same environment variable) the counters are that kernel's: [0] cycles and [1]
  * nanoseconds of the first CTA, [2] a tag of the first device-side wait that gave up (0 if none: barrier index,
  * warp << 8, CTA << 16), [3] cycles the first softmax warp of tile 0 waited for scores, [4] key blocks it
- * processed, [6] cycles it spent writing finished tiles out, [7] work items of that CTA.  The same variable's bits
- * 8, 64 and 128 switch off the attention kernel's softmax arithmetic, its first and its second products (timing
- * experiments; the output is then meaningless), like bits 1, 2 and 4 for the GEMM kernel's loads, products
- * and stores. */
+ * processed, [6] cycles it spent writing finished tiles out, [7] work items of that CTA.
+ * FACT_DEBUG_FLAGS is read once, by fact_create.  The library as built by default honours two bits, neither of
+ * which changes a result: 256 (these counters) and 2048 (no downward K walk on every second tile).  The
+ * work-skipping experiment switches (1, 2, 4: the GEMM kernel's loads, products, stores; 8, 64, 128: the attention
+ * kernel's softmax arithmetic and its two products), whose output is meaningless, exist only in a library
+ * compiled with -DFACT_EXPERIMENTS; the default build ignores those bits. */
 fact_status_t fact_last_kernel_profile(fact_handle_t handle, void* cuda_stream, int64_t counters[8]);
+
+/* The FACT_DEBUG_FLAGS bits in effect for this handle (0 in normal use; see fact_last_kernel_profile). */
+int fact_debug_flags(fact_handle_t handle);
 
 /* Text of the most recent CUDA runtime/driver failure seen through this handle
  * (the call that returned FACT_ERR_CUDA), "" if none.  Owned by the handle;

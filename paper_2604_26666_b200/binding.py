@@ -39,7 +39,7 @@ EXPORTED = [
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
-    "fact_linear_ex", "fact_row_stats", "fact_fold_norm",
+    "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
 ]
 
 
@@ -142,6 +142,8 @@ def lib() -> ctypes.CDLL:
     L.fact_row_stats.argtypes = [vp, i64, i64, vp, i64, vp, vp]
     L.fact_fold_norm.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
+    L.fact_gemm_splitk_static_status.argtypes = [c_int, vp, POINTER(c_int)]
+    L.fact_debug_flags.argtypes = [vp]
     for name in EXPORTED:
         fn = getattr(L, name)
         if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
@@ -161,15 +163,65 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else c_void_p(t.data_ptr())
 
 
-def _need(t: torch.Tensor, name: str, dtype, ndim):
-    if not isinstance(t, torch.Tensor) or not t.is_cuda:
-        raise TypeError(f"{name} must be a CUDA tensor")
+def _need(t: torch.Tensor, name: str, dtype, ndim, cuda: bool = True):
+    if not isinstance(t, torch.Tensor):
+        raise TypeError(f"{name} must be a tensor")
     if t.dtype != dtype:
         raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
     if t.ndim != ndim:
         raise ValueError(f"{name} must have {ndim} dimensions")
     if t.shape[-1] > 1 and t.stride(-1) != 1:
         raise ValueError(f"{name}: innermost dimension must be contiguous")
+    if cuda and not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+
+
+def _need_out(out: torch.Tensor, shape, like: torch.Tensor, name: str = "out"):
+    """A caller-supplied output must have exactly the result's shape, a supported dtype, and live on the operands'
+    device: the kernels write `shape` elements through its pointer whatever its real size is."""
+    if not isinstance(out, torch.Tensor):
+        raise TypeError(f"{name} must be a tensor")
+    if out.dtype not in (torch.bfloat16, torch.float32):
+        raise TypeError(f"{name} must be bfloat16 or float32, got {out.dtype}")
+    if tuple(out.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(out.shape)}")
+    if out.device != like.device:
+        raise ValueError(f"{name} is on {out.device}, the operands are on {like.device}")
+    if out.shape[-1] > 1 and out.stride(-1) != 1:
+        raise ValueError(f"{name}: innermost dimension must be contiguous")
+    if not out.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+
+
+def _validate_matmul(A, B, out, layout: str, batched: bool = False):
+    """Shape, dtype and device checks of C = A @ B before anything is handed to the library (a mismatch there would
+    be an out-of-bounds device access, not an error code).  Shape errors are reported before the tensors are required
+    to be on a GPU.  Returns (batch, M, N, K)."""
+    nd = 3 if batched else 2
+    _need(A, "A", torch.bfloat16, nd, cuda=False)
+    _need(B, "B", torch.bfloat16, nd, cuda=False)
+    if layout not in LAYOUTS:
+        raise ValueError(f"layout must be one of {sorted(LAYOUTS)}")
+    M, K = A.shape[-2:]
+    N, Kb = (B.shape[-1], B.shape[-2]) if layout == "KN" else (B.shape[-2], B.shape[-1])
+    if Kb != K:
+        raise ValueError(f"inner dimensions differ: A has K = {K}, B has K = {Kb}")
+    batch = A.shape[0] if batched else 1
+    if batched and B.shape[0] != batch:
+        raise ValueError("batch sizes differ")
+    _same_device(A, B)
+    if out is not None:
+        _need_out(out, (batch, M, N) if batched else (M, N), A)
+    for name, t in (("A", A), ("B", B)):
+        if not t.is_cuda:
+            raise TypeError(f"{name} must be a CUDA tensor")
+    return int(batch), int(M), int(N), int(K)
+
+
+def _same_device(*tensors):
+    devs = {t.device for t in tensors if t is not None}
+    if len(devs) > 1:
+        raise ValueError(f"tensors live on different devices: {sorted(str(d) for d in devs)}")
 
 
 def _ld(t: torch.Tensor) -> int:
@@ -195,17 +247,27 @@ def gemm_splitk_static(A, B, out, layout="KN", splits=0, device=None, stream=Non
     """C = A @ B through fact_gemm_splitk_static: no handle, no workspace, no device allocation inside the
     library (its split-K scratch is a fixed 16 MiB array inside the library image).  For callers that may
     not call cudaMalloc; `out` must be preallocated by the caller.  Calls on one device must not overlap."""
-    _need(A, "A", torch.bfloat16, 2)
-    _need(B, "B", torch.bfloat16, 2)
-    _need(out, "out", out.dtype, 2)
-    M, K = A.shape
-    N = B.shape[1] if layout == "KN" else B.shape[0]
+    if out is None:
+        raise TypeError("out must be preallocated by the caller: this entry point exists for callers that cannot allocate")
+    _, M, N, K = _validate_matmul(A, B, out, layout)
     dev = A.device.index if device is None else int(device)
+    if dev != A.device.index:
+        raise ValueError(f"the operands are on cuda:{A.device.index}, the call names device {dev}")
     s = stream if stream is not None else torch.cuda.current_stream(dev)
     _check(lib().fact_gemm_splitk_static(dev, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
                                          _ld(out), OUT_TYPES[out.dtype], int(splits), c_void_p(s.cuda_stream)),
            "fact_gemm_splitk_static")
     return out
+
+
+def gemm_splitk_static_status(device: int = 0, stream=None) -> int:
+    """The device status word of fact_gemm_splitk_static on `device` (0, or 7 after a device-side wait gave up:
+    the output of that call is then undefined); synchronises the stream and clears the word."""
+    s = stream if stream is not None else torch.cuda.current_stream(device)
+    v = c_int(0)
+    _check(lib().fact_gemm_splitk_static_status(int(device), c_void_p(s.cuda_stream), byref(v)),
+           "fact_gemm_splitk_static_status")
+    return int(v.value)
 
 
 class Handle:
@@ -216,6 +278,7 @@ class Handle:
         self.device = int(device)
         _check(lib().fact_create(byref(self._h), self.device), "fact_create")
         self._ws: Optional[torch.Tensor] = None
+        self._ws_streams: dict = {}
         self._ws_cache: dict = {}
         table = _PKG / "tuned_b200.txt"
         if load_table and table.exists():  # the tuner's table for the benchmark shapes, measured on a B200
@@ -235,6 +298,7 @@ class Handle:
     # -- helpers ------------------------------------------------------------------------------
     def _stream(self, stream) -> c_void_p:
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._ws_streams[int(s.cuda_stream)] = s  # kernels on this stream may be using the workspace
         return c_void_p(s.cuda_stream)
 
     def _cfg(self, cfg):
@@ -249,6 +313,11 @@ class Handle:
         if nbytes <= 0:
             return None
         if self._ws is None or self._ws.numel() < nbytes:
+            if self._ws is not None:
+                # kernels launched on other streams than torch's current one may still read the old buffer: tell the
+                # caching allocator, so that it does not hand the block out again before they have finished
+                for s in self._ws_streams.values():
+                    self._ws.record_stream(s)
             self._ws = torch.empty(nbytes, dtype=torch.uint8, device=f"cuda:{self.device}")
         return self._ws
 
@@ -304,6 +373,10 @@ class Handle:
         _check(lib().fact_selftest_wait_timeout(self._h, self._stream(stream), float(limit_ms)),
                "fact_selftest_wait_timeout", self._h)
 
+    def debug_flags(self) -> int:
+        """The FACT_DEBUG_FLAGS bits in effect (0 in normal use; the default build honours diagnostics only)."""
+        return int(lib().fact_debug_flags(self._h))
+
     def launch_count(self) -> int:
         return int(lib().fact_launch_count(self._h))
 
@@ -322,15 +395,9 @@ class Handle:
     # -- compute ------------------------------------------------------------------------------
     def gemm(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
         """C = A @ B  (fact_gemm).  layout "KN": B is [K, N]; "NK": B is [N, K]."""
-        _need(A, "A", torch.bfloat16, 2)
-        _need(B, "B", torch.bfloat16, 2)
-        M, K = A.shape
-        N = B.shape[1] if layout == "KN" else B.shape[0]
-        if (B.shape[0] if layout == "KN" else B.shape[1]) != K:
-            raise ValueError("inner dimensions differ")
+        _, M, N, K = _validate_matmul(A, B, out, layout)
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=A.device)
-        _need(out, "out", out.dtype, 2)
         c = self._cfg(cfg)
         nws = self.workspace_bytes("gemm", 1, M, N, K, "NONE", layout, out.dtype, cfg)
         ws = self.workspace(nws)
@@ -340,15 +407,9 @@ class Handle:
 
     def gemm_batched(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
         """C[b] = A[b] @ B[b]  (fact_gemm_batched)."""
-        _need(A, "A", torch.bfloat16, 3)
-        _need(B, "B", torch.bfloat16, 3)
-        batch, M, K = A.shape
-        N = B.shape[2] if layout == "KN" else B.shape[1]
-        if B.shape[0] != batch or (B.shape[1] if layout == "KN" else B.shape[2]) != K:
-            raise ValueError("shapes differ")
+        batch, M, N, K = _validate_matmul(A, B, out, layout, batched=True)
         if out is None:
             out = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
-        _need(out, "out", out.dtype, 3)
         nws = self.workspace_bytes("gemm_batched", batch, M, N, K, "NONE", layout, out.dtype, cfg)
         ws = self.workspace(nws)
         _check(lib().fact_gemm_batched(self._h, batch, M, N, K, _ptr(A), _ld(A), A.stride(0), _ptr(B), _ld(B),
@@ -359,15 +420,9 @@ class Handle:
 
     def gemm_splitk(self, A, B, layout="KN", out=None, out_dtype=torch.float32, splits=0, cfg=None, stream=None):
         """C = A @ B with K cut into slices and a fixed-order reduction  (fact_gemm_splitk)."""
-        _need(A, "A", torch.bfloat16, 2)
-        _need(B, "B", torch.bfloat16, 2)
-        M, K = A.shape
-        N = B.shape[1] if layout == "KN" else B.shape[0]
-        if (B.shape[0] if layout == "KN" else B.shape[1]) != K:
-            raise ValueError("inner dimensions differ")
+        _, M, N, K = _validate_matmul(A, B, out, layout)
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=A.device)
-        _need(out, "out", out.dtype, 2)
         nws = self.workspace_bytes("gemm_splitk", 1, M, N, K, "NONE", layout, out.dtype, cfg, splits)
         ws = self.workspace(nws)
         _check(lib().fact_gemm_splitk(self._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
@@ -402,9 +457,10 @@ class Handle:
             _need(residual, "residual", torch.bfloat16, 2)
             if tuple(residual.shape) != (M, N):
                 raise ValueError("residual must be [M, N_out]")
+        _same_device(X, W, bias, residual)
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=X.device)
-        _need(out, "out", out.dtype, 2)
+        _need_out(out, (M, N), X)
         nws = self.workspace_bytes("linear", 1, M, N, K, epilogue, layout, out.dtype, cfg)
         ws = self.workspace(nws)
         if stats_out is not None or x_norm not in (None, "none") or x_stats is not None or w_colsum is not None:
@@ -484,7 +540,7 @@ class Handle:
             _need(residual, "residual", torch.bfloat16, 2)
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=X.device)
-        _need(out, "out", out.dtype, 2)
+        _need_out(out, (M, N), X)
         arr = (c_int64 * max(G, 1))(*rows)
         _check(lib().fact_linear_grouped(self._h, G, arr, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W),
                                          int(W.stride(0)) if G > 1 else int(W.shape[1] * W.stride(1)), LAYOUTS[layout],
@@ -513,7 +569,7 @@ class Handle:
             _need(bias, "bias", torch.bfloat16, 1)
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=X.device)
-        _need(out, "out", out.dtype, 2)
+        _need_out(out, (M, N), X)
         arr = (c_int64 * max(G, 1))(*rows)
         _check(lib().fact_linear_grouped_fp8(self._h, G, arr, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W),
                                              int(W.stride(0)) if G > 1 else int(W.shape[1] * W.stride(1)), float(scale),
@@ -552,7 +608,7 @@ class Handle:
                 raise ValueError("residual must be [M, N_out]")
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype, device=X.device)
-        _need(out, "out", out.dtype, 2)
+        _need_out(out, (M, N), X)
         nws = self.workspace_bytes("linear_fp8", 1, M, N, K, epilogue, "NK", out.dtype, cfg)
         ws = self.workspace(nws)
         _check(lib().fact_linear_fp8(self._h, M, N, K, _ptr(X), _ld(X), _ptr(W), _ld(W), float(scale), _ptr(bias),
@@ -571,7 +627,7 @@ class Handle:
         _, Tk, Hkv, _ = k.shape
         if out is None:
             out = torch.empty((B, Tq, Hq, D), dtype=torch.bfloat16, device=q.device)
-        _need(out, "out", torch.bfloat16, 4)
+        _need_out(out, (B, Tq, Hq, D), q)
         st = lambda t: (int(t.stride(0)), int(t.stride(1)), int(t.stride(2)))
         _check(lib().fact_attention(self._h, B, Tq, Tk, Hq, Hkv, D, _ptr(q), *st(q), _ptr(k), *st(k), _ptr(v), *st(v),
                                     _ptr(out), *st(out), 1 if causal else 0, float(scale), self._stream(stream)),

@@ -1,6 +1,10 @@
 """Build libfact.so in-tree with nvcc for sm_100a (no JIT cache, no pip install).
 
     python -m paper_2604_26666_b200.build [--force] [--verbose]
+
+FACT_EXPERIMENTS=1 in the environment adds -DFACT_EXPERIMENTS: a library for timing experiments whose kernels
+honour the work-skipping FACT_DEBUG_FLAGS bits (loads, products or stores left out; results are garbage).
+The default build has no such code.
 """
 from __future__ import annotations
 
@@ -32,11 +36,15 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
+def _flags() -> list:
+    return NVCC_FLAGS + (["-DFACT_EXPERIMENTS"] if os.environ.get("FACT_EXPERIMENTS") == "1" else [])
+
+
 def source_hash() -> str:
     h = hashlib.sha1()
     for f in [CSRC / s for s in SOURCES + HEADERS] + [ROOT / "include" / "fact.h"]:
         h.update(f.read_bytes())
-    h.update(" ".join(NVCC_FLAGS).encode())
+    h.update(" ".join(_flags()).encode())
     return h.hexdigest()
 
 
@@ -47,7 +55,7 @@ def is_current() -> bool:
 def build(force: bool = False, verbose: bool = False) -> Path:
     if is_current() and not force:
         return LIB
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", str(ROOT / "include"), "-I", str(CSRC)]
+    cmd = [_nvcc(), *_flags(), "-I", str(ROOT / "include"), "-I", str(CSRC)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [str(CSRC / s) for s in SOURCES]

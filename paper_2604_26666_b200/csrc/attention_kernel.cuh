@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       const uint32_t tmem_o = tmem_base + (uint32_t)t * 256u + kColO;
       const uint32_t q_addr = q_s0 + (uint32_t)t * tile_bytes;
       const uint64_t qdesc0 = p.kmajor_desc | (uint64_t)((q_addr >> 4) & 0x3fffu);
-      const bool skip_s = (p.debug & 64) != 0, skip_pv = (p.debug & 128) != 0;  // experiment switches, 0 in normal use
+      const bool skip_s = FACT_SKIP(p, 64), skip_pv = FACT_SKIP(p, 128);  // experiment switches, 0 in normal use
       int g = 0;   // key blocks of the items so far (the producer's numbering)
       int gt = 0;  // blocks this tile has processed
       bool ok = true;
@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(bar(S_READ + t));
-        if (p.debug & 8) {  // experiment switch: no softmax arithmetic, the barrier protocol only
+        if (FACT_SKIP(p, 8)) {  // experiment switch: no softmax arithmetic, the barrier protocol only
           if (gt > 0) ok = wait_all(bar(PV_DONE + t), (uint32_t)(gt - 1) & 1u);
           if (!ok) break;
           __syncwarp();

@@ -26,8 +26,9 @@
 // 16 MiB until the process exits.  In host code these names are only stand-ins for the device symbols; the
 // device addresses the kernels get come from cudaGetSymbolAddress (see static_setup below).
 constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
+constexpr int kStaticStatusInts = 64;  // the words a split-K launch touches: error word, clock stamps, grid-barrier counters
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-static __device__ __align__(256) int g_static_status[32];
+static __device__ __align__(256) int g_static_status[kStaticStatusInts];
 
 namespace {
 
@@ -41,6 +42,7 @@ constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the w
                                          // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
 constexpr int kStatusInts = 64;  // status word, clock / profile counters, grid-barrier counters; stream-K flags follow
+constexpr int kDiagnosticFlags = 256 | 2048;  // FACT_DEBUG_FLAGS bits that leave results intact: cycle counters, no K serpentine
 constexpr int kMaxGroups = 4096;  // row groups of a grouped GEMM (the handle's device table holds 2 x (kMaxGroups + 1) ints)
 
 // Key of the tuner's table: everything that changes which configuration is best.
@@ -77,6 +79,7 @@ struct Problem {
 
 struct Plan {
   fact_config_t cfg;
+  bool from_table = false;  // cfg came from the tuner's table: its store mode and K slices are hints, not demands
   int smem_bytes;
   int grid;
   size_t ws_bytes;
@@ -96,7 +99,8 @@ struct fact_handle_s {
   std::map<TuneKey, fact_config_t> table;
   std::bitset<128> configured_mask;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
-  int debug_flags = 0;           // FACT_DEBUG_FLAGS: kernel experiment switches, 0 in normal use
+  int debug_flags = 0;           // FACT_DEBUG_FLAGS: diagnostics (256 cycle counters, 2048 no K serpentine); the
+                                 // work-skipping experiment switches only in a -DFACT_EXPERIMENTS build
   int* d_groups = nullptr;       // grouped GEMM: m-tile prefix and row offsets of the call in flight
   int* sk_flags() const { return d_status + kStatusInts; }  // stream-K flags: [SM][epilogue warp], 0 between launches
   size_t status_ints() const { return (size_t)kStatusInts + (size_t)sm_count * kEpiWarps; }
@@ -159,7 +163,7 @@ bool tile_ok(const Problem& q, int tile_n, int cg) {
 
 // Fill every zero field of `cfg`.  Returns FACT_ERR_UNSUPPORTED for a combination the kernels cannot run.
 fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_config_t* user, int splits_override,
-                             fact_config_t* out) {
+                             fact_config_t* out, bool* from_table_out = nullptr) {
   fact_config_t c;
   memset(&c, 0, sizeof c);
   bool from_table = false;
@@ -271,6 +275,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.split_k > 0) c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
   if (c.store_mode < 0 || c.store_mode > 3) return FACT_ERR_INVALID_ARG;
   *out = c;
+  if (from_table_out) *from_table_out = from_table;
   return FACT_OK;
 }
 
@@ -366,7 +371,7 @@ uint64_t smem_desc_template(uint32_t lbo_bytes, uint32_t sbo_bytes) {
 
 fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* user, int splits_override,
                         Plan* plan) {
-  fact_status_t st = resolve_config(h, q, user, splits_override, &plan->cfg);
+  fact_status_t st = resolve_config(h, q, user, splits_override, &plan->cfg, &plan->from_table);
   if (st != FACT_OK) return st;
   const fact_config_t& c = plan->cfg;
   GemmParams& p = plan->p;
@@ -453,6 +458,15 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   const int chunk_cols = p.out_f32 ? 32 : 64;
   const bool can_stage = p.c_vec && (p.out_cols % chunk_cols == 0) &&
                          !(p.out_f32 && q.epi == FACT_EPI_BIAS_RESIDUAL);
+  // The table is keyed on the shape alone, so what it says about the store path is a hint: this call's output may
+  // be less aligned than the one the entry was tuned on.  Only a caller's own configuration is refused.
+  const long long esz_c = p.out_f32 ? 4 : 2;
+  const bool rows32 = (reinterpret_cast<uintptr_t>(q.C) & 31u) == 0 && (q.ldc * esz_c) % 32 == 0 &&
+                      (q.N_out * esz_c) % 32 == 0 && (q.batch <= 1 || (q.strideC * esz_c) % 32 == 0);
+  const bool can_rows32 = can_stage && rows32 && c.split_k == 1 && q.groups == 0 && !q.stats_out && !q.norm &&
+                          q.epi != FACT_EPI_BIAS_SOFTMAX;
+  if (plan->from_table && ((c.store_mode == 2 && !can_stage) || (c.store_mode == 3 && !can_rows32)))
+    plan->cfg.store_mode = 0;
   if (c.store_mode == 2 && !can_stage) return FACT_ERR_UNSUPPORTED;
   const int asked_store = c.store_mode;  // (c aliases plan->cfg, which is rewritten below)
   p.store_tma = (c.store_mode == 1) ? 0 : (can_stage ? 1 : 0);
@@ -461,12 +475,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   if (asked_store == 3) {
     // the staged epilogue's arithmetic with each row stored from registers in 32-byte pieces: whole, unsliced,
     // ungrouped tiles whose output rows are 32-byte aligned multiples of 32 bytes
-    const long long esz = p.out_f32 ? 4 : 2;
-    const bool rows32 = (reinterpret_cast<uintptr_t>(q.C) & 31u) == 0 && (q.ldc * esz) % 32 == 0 &&
-                        (q.N_out * esz) % 32 == 0 && (q.batch <= 1 || (q.strideC * esz) % 32 == 0);
-    if (!can_stage || !rows32 || c.split_k != 1 || q.groups > 0 || q.stats_out || q.norm ||
-        q.epi == FACT_EPI_BIAS_SOFTMAX)
-      return FACT_ERR_UNSUPPORTED;
+    if (!can_rows32) return FACT_ERR_UNSUPPORTED;
     p.row_stores = 1;
     plan->cfg.store_mode = 3;
   }
@@ -718,6 +727,15 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     st = make_plan(h, q, &dp, 0, &plan);
     if (st != FACT_OK) return st;
   }
+  if (plan.cfg.split_k > 1 && plan.from_table && splits_override == 0 && q.op != FACT_OP_GEMM_SPLITK &&
+      (!ws || ws_bytes < plan.ws_bytes || !aligned16(ws))) {
+    // a tuned entry with K slices, but this caller brought no (or too little) scratch: one slice
+    fact_config_t dp = plan.cfg;
+    dp.split_k = 1;
+    dp.store_mode = 0;
+    st = make_plan(h, q, &dp, 0, &plan);
+    if (st != FACT_OK) return st;
+  }
   if (q.K == 0 && q.epi == FACT_EPI_BIAS_SOFTMAX) return FACT_ERR_UNSUPPORTED;  // (the stand-alone epilogue has no softmax)
   if (q.K == 0) {  // empty sum: the epilogue of a zero accumulator
     st = launch_reduce(h, q, plan, 0, reinterpret_cast<const float*>(q.C), stream);
@@ -873,6 +891,9 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
   h->cc_major = prop.major;
   h->cc_minor = prop.minor;
   if (const char* dbg = getenv("FACT_DEBUG_FLAGS")) h->debug_flags = atoi(dbg);
+#ifndef FACT_EXPERIMENTS
+  h->debug_flags &= kDiagnosticFlags;  // the work-skipping switches do not exist in this build
+#endif
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -1681,5 +1702,32 @@ fact_status_t fact_gemm_splitk_static(int device, int64_t M, int64_t N, int64_t 
   if (prev != device) cudaSetDevice(prev);
   return rc;
 }
+
+fact_status_t fact_gemm_splitk_static_status(int device, void* stream, int* status) {
+  if (device < 0 || device >= kMaxStaticDevices || !status) return FACT_ERR_INVALID_ARG;
+  StaticDeviceState* st = &g_static_state[device];
+  *status = 0;
+  if (!st->ready) return FACT_OK;  // no call has run on this device yet
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) return FACT_ERR_CUDA;
+  // read (and, after a give-up, clear) the static status word and the grid-barrier counters: a stream
+  // synchronisation, one 4-byte copy and memsets -- nothing allocates
+  fact_status_t rc = FACT_OK;
+  int v = 0;
+  int* word = st->handle.d_status;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess ||
+      cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      (v != 0 && (cudaMemset(word, 0, sizeof(int)) != cudaSuccess ||
+                  cudaMemset(word + 24, 0, 2 * sizeof(int)) != cudaSuccess))) {
+    cudaGetLastError();
+    rc = FACT_ERR_CUDA;
+  }
+  *status = v;
+  if (prev != device) cudaSetDevice(prev);
+  return rc;
+}
+
+int fact_debug_flags(fact_handle_t h) { return h ? h->debug_flags : 0; }
 
 }  // extern "C"

@@ -26,6 +26,15 @@
 
 #include "ptx.cuh"
 
+// Work-skipping experiment switches (loads, products or stores left out to isolate one ceiling; the results are
+// garbage) exist only in a -DFACT_EXPERIMENTS build.  In the ordinary build the tests are the constant 0 and the
+// compiler drops the code behind them.
+#ifdef FACT_EXPERIMENTS
+#define FACT_SKIP(p, bit) (((p).debug & (bit)) != 0)
+#else
+#define FACT_SKIP(p, bit) false
+#endif
+
 namespace fact {
 
 constexpr int kMaxStages = 8;
@@ -141,8 +150,9 @@ struct GemmParams {
   // EXT = 3 instantiations: the staged epilogue's arithmetic, but every thread stores its own row's 128 bytes of a
   // chunk straight from registers as four 32-byte stores (no staging traffic through shared memory)
   int row_stores;
-  // experiment switches (0 in normal use): 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA;
-  // 4 = epilogue skips its global stores.  They isolate the feed, issue and store ceilings; results are garbage.
+  // bit 256: the first CTA counts where its cycles go (fact_last_kernel_profile).  In a -DFACT_EXPERIMENTS build
+  // also the work-skipping switches: 1 = no loads, MMA on stale shared memory; 2 = loads only, no MMA; 4 = the
+  // epilogue skips its global stores (they isolate the feed, issue and store ceilings; results are garbage).
   int debug;
 };
 
@@ -710,7 +720,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------ TMA producers
     // Warp 0 loads the A tiles (and posts the expected byte count), warp 6 the B boxes.
     const bool do_a = warp == 0;
-    if (!(p.debug & 1)) {
+    if (!FACT_SKIP(p, 1)) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -815,7 +825,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tile_n);
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
           if (prof) t0 = clock64();
-          if (!(p.debug & 1) && !wait_all(full_bar(stage), phase)) {
+          if (!FACT_SKIP(p, 1) && !wait_all(full_bar(stage), phase)) {
             ok = false;
             break;
           }
@@ -830,7 +840,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint64_t adesc = p.a_desc | (uint64_t)((sa >> 4) & 0x3fffu);
           const uint64_t bdesc = p.b_desc | (uint64_t)((sb >> 4) & 0x3fffu);
           if (ptx::elect_one()) {
-            if (!(p.debug & 2)) {
+            if (!FACT_SKIP(p, 2)) {
 #pragma unroll
               for (int k = 0; k < kTileK / kUmmaK; ++k) {
                 if constexpr (kFp8)
@@ -1255,7 +1265,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // main loop hides their scatter (32 rows per instruction), and the 128 KB per tile that staging writes to
             // and reads from shared memory no longer compete with the operand reads of the tensor pipe.
             const int row = row0 + lane;
-            if (row < p.M && !(p.debug & 4)) {
+            if (row < p.M && !FACT_SKIP(p, 4)) {
               uint8_t* dst = reinterpret_cast<uint8_t*>(p.C) +
                              ((long long)z * p.strideC + (long long)row * p.ldc + n_chunk) * (long long)(f32 ? 4 : 2);
               const int e32 = f32 ? 8 : 16;  // elements in 32 bytes (N_out is a multiple of it on this path)
@@ -1295,13 +1305,13 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int j = 0; j < 8; ++j) {
               const int r = 4 * j + rsub;
               const uint4 v = ptx::ld_shared_v4(buf + (uint32_t)r * 128u + ((uint32_t)(piece ^ (r & 7)) << 4));
-              if (r < rows_left && col_ok && !(p.debug & 4)) *reinterpret_cast<uint4*>(out_b + r * row_bytes) = v;
+              if (r < rows_left && col_ok && !FACT_SKIP(p, 4)) *reinterpret_cast<uint4*>(out_b + r * row_bytes) = v;
             }
             ptx::fence_proxy_async_smem();  // (a residual tile may be loaded into this buffer next, by TMA)
             __syncwarp();
           } else {
             if (lane == 0) {
-              if (row0 < p.M && !(p.debug & 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
+              if (row0 < p.M && !FACT_SKIP(p, 4)) ptx::tma_store_3d(&tmC, buf, n_chunk, row0, z);
               ptx::bulk_commit_group();
             }
           }
@@ -1427,7 +1437,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int g = 0; g < 4; ++g) {
               const int n = c + g * 8;
               const int nvalid = min(8, p.N_out - n);
-              if (nvalid > 0 && row_ok && !(p.debug & 4)) {
+              if (nvalid > 0 && row_ok && !FACT_SKIP(p, 4)) {
                 float y[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) y[j] = __expf(z[g * 8 + j] - m) * inv;
@@ -1464,7 +1474,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (row_ok) load_bf16x8(r_row + n, nvalid, p.r_vec != 0, res);
               }
               apply_epilogue8<EPI>(&v[g * 8], &vu[g * 8], bias, res, y);
-              if (row_ok && !(p.debug & 4)) {
+              if (row_ok && !FACT_SKIP(p, 4)) {
                 if (p.out_f32) store_f32x8(reinterpret_cast<float*>(c_row) + n, y, nvalid, c_vec);
                 else store_bf16x8(reinterpret_cast<__nv_bfloat16*>(c_row) + n, y, nvalid, c_vec);
               }

@@ -1,11 +1,11 @@
 """Parity of the five benchmark configurations at their full sizes, in the launch
 configuration bench.py times (the handle's tuned table / default choice).
 
-The small configuration (config 1) and the batched / split-K shapes are compared
-element by element.  For the large shapes the oracle computes a stratified sample of
-output rows (first/last rows, tile borders, random rows: every column of each), and a
-Freivalds-style product check covers every element of the linear epilogues:
-    Y x  ==  X (W x) + (bias . x) + R x        for random +-1 vectors x, in FP64.
+Every shape is compared element by element, over the whole output, with the FP64
+oracle (5.1 TFLOP of oracle work in all: about half a minute on 16 host cores).  The
+linear epilogues also get a Freivalds-style product check in FP64,
+    Y x  ==  X (W x) + (bias . x) + R x        for random +-1 vectors x,
+which is independent of the oracle's loops.
 """
 import numpy as np
 import pytest
@@ -13,7 +13,7 @@ import torch
 
 import oracle
 from paper_2604_26666_b200 import workloads as wl
-from tests.helpers import check_case, gates, oracle_for, run_gpu, stratified_rows, to_f64
+from tests.helpers import check_case, gates, oracle_for, run_gpu, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -110,22 +110,23 @@ def freivalds(ins, case, got, n_vec=2, seed=0):
     return worst
 
 
-LINEAR_SAMPLED = ["c2_square_4096", "c2_square_8192", "c4_qkv", "c4_out_proj", "c4_mlp_up_gelu", "c4_mlp_down",
-                  "c5_qkv", "c5_o_proj", "c5_gate_up_silu", "c5_down"]
+FULL_SIZE = ["c2_square_4096", "c2_square_8192", "c4_qkv", "c4_out_proj", "c4_mlp_up_gelu", "c4_mlp_down",
+             "c5_qkv", "c5_o_proj", "c5_gate_up_silu", "c5_down"]
 
 
-@pytest.mark.parametrize("name", LINEAR_SAMPLED)
-def test_full_size_sampled_rows(h, name):
+@pytest.mark.parametrize("name", FULL_SIZE)
+def test_full_size_elementwise(h, name):
+    """The whole output of every large benchmark shape against the oracle: every CTA tile, every lane quarter,
+    every column chunk, in the configuration the handle's table (or default choice) runs."""
     case = (CASES_KN if name.startswith("c2") else CASES)[name]
     ins = wl.make_inputs(case)
     got = run_gpu(h, ins, case)
     torch.cuda.synchronize()
     assert h.device_status() == 0
-    n_rows = 48 if case.flops > 5e11 else 96
-    rows = stratified_rows(case.M, n_rows, seed=case.seed, tile=256)
-    ref = oracle_for(ins, case, rows=rows)
-    g = to_f64(got)[rows]
-    assert np.isfinite(to_f64(got)).all()
+    ref = oracle_for(ins, case)
+    g = to_f64(got)
+    assert g.shape == ref.shape == (case.M, case.N)
+    assert np.isfinite(g).all()
     c, t = gates(ref, g, case.out, case.epilogue)
     assert c <= 1.0, f"{name}: contract gate ratio {c:.3f}"
     assert t <= 1.0, f"{name}: tight gate ratio {t:.3f}"
@@ -136,7 +137,5 @@ def test_full_size_sampled_rows(h, name):
 
 @pytest.mark.parametrize("name", ["c4_qkv", "c4_mlp_down", "c5_o_proj"])
 def test_full_size_kn_layout(h, name):
-    """The same linears with the weight stored [K x N]."""
-    case = CASES_KN[name]
-    rows = stratified_rows(case.M, 32, seed=1, tile=256)
-    check_case(h, case, rows=rows)
+    """The same linears with the weight stored [K x N], whole output."""
+    check_case(h, CASES_KN[name])

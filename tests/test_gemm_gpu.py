@@ -176,6 +176,65 @@ def test_strided_operands(h):
     assert (Cbig[:, N:] == 0).all(), "wrote outside the N columns"
 
 
+def test_table_entries_are_hints_for_less_aligned_outputs(h, tmp_path):
+    """The tuner's table is keyed on the shape alone.  An entry that asks for staged tensor stores, 32-byte register
+    row stores or K slices must not turn a call with a less aligned output, or without scratch, into an error: the
+    library falls back to a store path (one K slice) that can run, and the result is still the oracle's."""
+    from paper_2604_26666_b200.binding import Handle, lib
+    import ctypes
+
+    M, N, K = 384, 320, 2048 + 64
+    path = tmp_path / "hints.txt"
+    # op LINEAR(3) epilogue BIAS(1) layout NK(1) out BF16(0): staged stores; op GEMM(0): register row stores (mode 3);
+    # op LINEAR with BIAS_RELU(2): 4 K slices
+    path.write_text(f"3 1 1 0 1 {M} {N} {K} | 128 64 64 4 1 0 1 2\n"
+                    f"0 0 0 0 1 {M} {N} {K} | 128 64 64 4 1 0 1 3\n"
+                    f"3 2 1 0 1 {M} {N} {K} | 128 64 64 4 1 0 4 2\n")
+    h2 = Handle(0, load_table=False)
+    h2.tune_cache_load(str(path))
+    dev = "cuda:0"
+    # (a) staged entry, output with ldc = N + 2: rows are not 16-byte multiples
+    case = mk("hint_staged", M, N, K, epilogue="BIAS", layout="NK")
+    ins = wl.make_inputs(case)
+    big = torch.zeros(M, N + 2, dtype=torch.bfloat16, device=dev)
+    out = big[:, :N]
+    h2.linear(ins.X.to(dev), ins.W.to(dev), bias=ins.bias.to(dev), epilogue="BIAS", layout="NK", out=out)
+    torch.cuda.synchronize()
+    assert h2.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", "BIAS")
+    assert c <= 1 and t <= 1, (c, t)
+    assert (big[:, N:] == 0).all()
+    # (b) register-row-store entry, output 16-byte but not 32-byte aligned
+    case = mk("hint_rows32", M, N, K, op="gemm", layout="KN")
+    ins = wl.make_inputs(case)
+    flat = torch.zeros(M * N + 8, dtype=torch.bfloat16, device=dev)
+    out = flat[8:].view(M, N)
+    assert out.data_ptr() % 32 == 16
+    h2.gemm(ins.X.to(dev), ins.W.to(dev), layout="KN", out=out)
+    torch.cuda.synchronize()
+    assert h2.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", "NONE")
+    assert c <= 1 and t <= 1, (c, t)
+    assert (flat[:8] == 0).all()
+    # (c) an entry with K slices, called through the raw C ABI without any workspace
+    case = mk("hint_split", M, N, K, epilogue="BIAS_RELU", layout="NK")
+    ins = wl.make_inputs(case)
+    X, W, b = ins.X.to(dev), ins.W.to(dev), ins.bias.to(dev)
+    out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    vp = ctypes.c_void_p
+    rc = lib().fact_linear(h2._h, M, N, K, vp(X.data_ptr()), K, vp(W.data_ptr()), K, 1, vp(b.data_ptr()), None, 0,
+                           vp(out.data_ptr()), N, 0, 2, None, None, 0, vp(torch.cuda.current_stream(0).cuda_stream))
+    assert rc == 0, rc
+    torch.cuda.synchronize()
+    assert h2.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", "BIAS_RELU")
+    assert c <= 1 and t <= 1, (c, t)
+    # a caller's own configuration is still refused where it cannot run
+    with pytest.raises(Exception):
+        h2.linear(X, W, bias=b, epilogue="BIAS_RELU", layout="NK", out=big[:, :N], cfg={"store_mode": 2})
+    h2.close()
+
+
 # ------------------------------------------------------------------ batched and split-K
 @pytest.mark.parametrize("layout", ["KN", "NK"])
 def test_batched(h, layout):

@@ -189,3 +189,52 @@ def test_stream_k_pieces_rejects_bad_arguments(libfact):
     assert libfact.fact_stream_k_pieces(4, 1, 1, 4, 1, buf, ctypes.byref(n)) == 1
     assert libfact.fact_stream_k_pieces(4, 1, 1, 0, 1, buf, None) == 1
     assert libfact.fact_stream_k_pieces(4, 1, 8, 3, 0, None, ctypes.byref(n)) == 0 and n.value == 1
+
+
+def test_binding_rejects_mismatched_shapes_without_launching_anything():
+    """A Python shape mistake must be a ValueError, not an out-of-bounds device access: the binding checks inner
+    dimensions, the output's shape and the devices before it hands a pointer to the library.  CPU tensors reach
+    the shape checks (the CUDA requirement comes last), so nothing can launch here."""
+    import torch
+
+    from paper_2604_26666_b200 import binding as bd
+
+    bf, f32 = torch.bfloat16, torch.float32
+    A = torch.zeros(64, 128, dtype=bf)
+    with pytest.raises(ValueError, match="inner dimensions"):
+        bd._validate_matmul(A, torch.zeros(120, 96, dtype=bf), None, "KN")
+    with pytest.raises(ValueError, match="inner dimensions"):
+        bd._validate_matmul(A, torch.zeros(96, 120, dtype=bf), None, "NK")
+    with pytest.raises(ValueError, match="shape"):  # too small an output would be written past its end
+        bd._validate_matmul(A, torch.zeros(128, 96, dtype=bf), torch.zeros(32, 96, dtype=f32), "KN")
+    with pytest.raises(ValueError, match="shape"):
+        bd._validate_matmul(torch.zeros(2, 64, 128, dtype=bf), torch.zeros(2, 128, 96, dtype=bf),
+                            torch.zeros(64, 96, dtype=bf), "KN", batched=True)
+    with pytest.raises(ValueError, match="batch"):
+        bd._validate_matmul(torch.zeros(2, 64, 128, dtype=bf), torch.zeros(3, 128, 96, dtype=bf), None, "KN", batched=True)
+    with pytest.raises(TypeError):  # wrong operand dtype
+        bd._validate_matmul(A.float(), torch.zeros(128, 96, dtype=bf), None, "KN")
+    with pytest.raises(ValueError, match="operands are on"):
+        bd._need_out(torch.zeros(64, 96, dtype=f32, device="meta"), (64, 96), A)
+    with pytest.raises(ValueError, match="contiguous"):
+        bd._need_out(torch.zeros(96, 64, dtype=f32).t(), (64, 96), A)
+    # consistent shapes pass the shape checks and stop at the CUDA requirement
+    with pytest.raises(TypeError, match="CUDA"):
+        bd._validate_matmul(A, torch.zeros(128, 96, dtype=bf), torch.zeros(64, 96, dtype=f32), "KN")
+    # the allocation-free entry point goes through the same checks before it calls the library
+    with pytest.raises(ValueError, match="inner dimensions"):
+        bd.gemm_splitk_static(A, torch.zeros(120, 96, dtype=bf), torch.zeros(64, 96, dtype=f32))
+    with pytest.raises(ValueError, match="shape"):
+        bd.gemm_splitk_static(A, torch.zeros(128, 96, dtype=bf), torch.zeros(64, 90, dtype=f32))
+    with pytest.raises(TypeError):
+        bd.gemm_splitk_static(A, torch.zeros(128, 96, dtype=bf), None)
+
+
+def test_static_status_query_without_a_device(libfact):
+    from ctypes import byref, c_int
+
+    v = c_int(5)
+    assert libfact.fact_gemm_splitk_static_status(0, None, byref(v)) == 0 and v.value == 0  # no call has run yet
+    assert libfact.fact_gemm_splitk_static_status(-1, None, byref(v)) == 1
+    assert libfact.fact_gemm_splitk_static_status(0, None, None) == 1
+    assert libfact.fact_debug_flags(None) == 0
