@@ -215,6 +215,8 @@ def main():
     torch.cuda.set_device(dev)
     dist = dist_util.init("nccl", dev)
     h = Handle(local_rank)
+    if h.debug_flags() & ~(256 | 2048):  # only a -DFACT_EXPERIMENTS build honours the work-skipping switches
+        raise SystemExit("bench.py refuses to run with work-skipping FACT_DEBUG_FLAGS bits set")
     peaks = load_peaks()
     stream = torch.cuda.current_stream(dev)
 
@@ -392,7 +394,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": e2e_wall_ms / e2e_steps,
                     "api": "HostGemmPipeline (pinned host in, pinned host out, copies overlapped with kernels)"},
-            "gpu_launches": launches,
+            "gpu_launches": launches, "debug_flags": h.debug_flags(),
             "clocks": dict(clocks, sm_mhz_in_dominant_kernel=(1e3 * k_cycles / k_ns if k_ns else None)),
             "cpu_baseline": cpu,
             "shapes": shapes,
@@ -407,6 +409,65 @@ def main():
         dist.destroy_process_group()
     h.close()
     return 0
+
+
+SHORT_SHAPE_US = 120.0  # shapes whose single cold launch is shorter than this are (also) timed back to back
+
+
+def back_to_back_us(call_set, case, X, W, bias, res, out, h, dev, stream, reps=5, min_launches=20):
+    """Microseconds per launch of `case`, from N >= 20 launches back to back between one event pair, rotating through
+    R copies of the operands and outputs with R x footprint > 2 x L2 (so no launch finds its data in L2).  Median of
+    `reps` such trains.  call_set "side": the cuBLAS matmul-only side reference on the same buffers."""
+    import torch
+
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    foot = max(1.0, case.algorithmic_bytes)
+    R = int(min(512, max(2, -(-2 * l2 // int(foot)) + 1)))
+    sets = []
+    for _ in range(R):
+        sets.append((X.clone(), W.clone(), None if bias is None else bias.clone(),
+                     None if res is None else res.clone(), torch.empty_like(out)))
+    n = R * max(1, -(-min_launches // R))
+
+    def one(s):
+        Xs, Ws, bs, rs, os_ = s
+        if call_set == "side":
+            if case.batch > 1:
+                torch.bmm(Xs, Ws if case.layout == "KN" else Ws.transpose(1, 2))
+            else:
+                torch.matmul(Xs, Ws if case.layout == "KN" else Ws.t())
+        elif case.op == "gemm":
+            h.gemm(Xs, Ws, layout=case.layout, out=os_)
+        elif case.op == "gemm_batched":
+            h.gemm_batched(Xs, Ws, layout=case.layout, out=os_)
+        elif case.op == "gemm_splitk":
+            h.gemm_splitk(Xs, Ws, layout=case.layout, out=os_)
+        else:
+            h.linear(Xs, Ws, bias=bs, residual=rs, epilogue=case.epilogue, layout=case.layout, out=os_)
+
+    for s in sets:  # warm-up: every set once (also sizes the workspace)
+        one(s)
+    torch.cuda.synchronize(dev)
+    # The train is replayed from a CUDA graph: issued from Python, a launch costs the host more than these kernels
+    # take, and the figure would be the interpreter's launch rate.
+    graph = torch.cuda.CUDAGraph()
+    side_stream = torch.cuda.Stream(dev)
+    with torch.cuda.graph(graph, stream=side_stream):
+        for i in range(n):
+            one(sets[i % R])  # (inside the capture torch's current stream is the capturing stream)
+    graph.replay()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        a.record(stream)
+        graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize(dev)
+        ts.append(a.elapsed_time(b) / n)
+    del graph
+    del sets
+    return sorted(ts)[len(ts) // 2] * 1e3
 
 
 def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, iters=20, side_ref=True, layout="NK"):
@@ -470,16 +531,37 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
         bound = "tensor" if t_tensor >= t_hbm else "hbm"
         cfg = h.get_config(case.op, case.batch, case.M, case.N, case.K, case.epilogue, case.layout, odt).as_dict()
-        rows.append({
+        row = {
             "name": case.name, "config": case.config, "op": case.op, "epilogue": case.epilogue,
             "layout": case.layout, "batch": case.batch, "M": case.M, "N": case.N, "K": case.K, "out": case.out,
             "us_median": med * 1e3, "us_min": t[0] * 1e3, "us_hot_l2_median": t_hot[len(t_hot) // 2] * 1e3,
-            "tflops": case.flops / (med * 1e-3) / 1e12, "gbs": case.algorithmic_bytes / (med * 1e-3) / 1e9,
-            "pct_of_bf16_peak_burst": 100 * case.flops / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "bound": bound, "roofline_us": max(t_tensor, t_hbm) * 1e3,
-            "roofline_frac": max(t_tensor, t_hbm) / med,
             "cublas_matmul_only_us": t_side[len(t_side) // 2] * 1e3, "tile": cfg,
+        }
+        # Shapes of the order of 100 us and below: an event pair around ONE launch that follows the L2-flush kernels
+        # also times the launch itself (10-12 us on this part), so the figure that counts for them is N launches back
+        # to back between one event pair, rotating through R sets of operands and outputs whose total exceeds twice
+        # the L2 -- every launch still finds its data in DRAM, and the cost per launch is the stream time it adds.
+        t_use = med
+        if med * 1e3 < SHORT_SHAPE_US:
+            t_b2b = back_to_back_us(call_set=None, case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev,
+                                    stream=stream) * 1e-3
+            row["us_back_to_back_cold"] = t_b2b * 1e3
+            row["timing"] = "back-to-back launches over rotating buffer sets (total > 2 x L2), per launch"
+            if side_ref:
+                row["cublas_matmul_only_back_to_back_us"] = back_to_back_us(
+                    call_set="side", case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev, stream=stream)
+            t_use = t_b2b
+        else:
+            row["timing"] = "one launch per event pair after an L2 flush, median"
+        row.update({
+            "us": t_use * 1e3, "tflops": case.flops / (t_use * 1e-3) / 1e12,
+            "gbs": case.algorithmic_bytes / (t_use * 1e-3) / 1e9,
+            "pct_of_bf16_peak_burst": 100 * case.flops / (t_use * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "roofline_frac": max(t_tensor, t_hbm) / t_use,
+            "roofline_frac_single_launch": max(t_tensor, t_hbm) / med,
         })
+        rows.append(row)
         del X, W, out
     return rows
 

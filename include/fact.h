@@ -138,8 +138,9 @@ typedef struct {
 
 /* Create / destroy a handle bound to CUDA device `device`.  fact_create makes
  * that device current, checks for sm_100, allocates the handle's two small device
- * buffers and resolves the driver's tensor-map encoder.  These two calls are the
- * only ones that allocate or free device memory. */
+ * buffers and resolves the driver's tensor-map encoder.  These two calls and the tuner
+ * (fact_tune, which is off the per-call path) are the only ones that allocate or free
+ * device memory. */
 fact_status_t fact_create(fact_handle_t* handle, int device);
 fact_status_t fact_destroy(fact_handle_t handle);
 
@@ -421,22 +422,74 @@ fact_status_t fact_get_config(fact_handle_t handle, fact_op_t op, int64_t batch,
                               fact_epilogue_t epilogue, fact_blayout_t b_layout, fact_out_t out_type,
                               fact_config_t* cfg_out);
 
-/* On-device tile-configuration search for one problem (Section 4.2, Action 5
- * "auto-tuning": sweep tile shapes, pipeline depth, cluster size and grid
- * schedule, time every feasible candidate, keep the best).  Runs on the given
- * device buffers (outputs are overwritten), times each feasible candidate with
- * CUDA events (`warmup` + `iters` launches; 0 = 5 and 20, the paper's
- * protocol in Section 5.1), synchronises the stream, stores the winner in the
- * handle's table and returns it.  Candidates over the shared-memory or TMEM
- * budget are skipped on the host and never launched.  `workspace` must be
- * large enough for every split-K candidate the search is allowed to try:
- * candidates that need more are skipped. */
+/* On-device tile-configuration search for one problem (Section 4.2, Actions 4 and 5: every candidate is
+ * verified, then benchmarked; the sweep covers tile shapes, pipeline depth, cluster size, grid schedule and
+ * store path, and the best verified candidate is kept).  Runs on the given device buffers (the output is
+ * overwritten; it ends holding the winner's result), synchronises the stream, stores the winner in the
+ * handle's table and returns it.
+ *   - Feasibility: candidates over the shared-memory or TMEM budget, or that the kernels cannot run on this
+ *     problem, are rejected on the host and never launched; candidates that need more than `workspace_bytes`
+ *     of scratch are skipped.  (The paper's sweep launches them and records the failures, Section 5.1.)
+ *   - Verify gate: the library's default configuration is run once and a dense FP32 copy of its output kept;
+ *     before a candidate is timed, its output (written over NaNs) is compared with that copy element by
+ *     element on the device, tolerance 2^-7 |ref| + 1e-3 mean|ref| for BF16 outputs and 2e-4 (|ref| +
+ *     mean|ref|) for FP32 outputs -- what two correct FP32-accumulated results in different summation orders
+ *     can differ by, far below what a dropped k-block or a misplaced tile changes.  A candidate outside it
+ *     is recorded as FACT_TUNE_VERIFY_FAILED, is never timed and can never win.
+ *   - Timing: `warmup` + `iters` launches per candidate (0 = 5 and 20, the paper's protocol in Section 5.1),
+ *     CUDA events, each candidate ranked by its time relative to the default configuration timed right
+ *     before and after it (the clock of a power-limited part drifts over a sweep); the four fastest are
+ *     timed three more times in alternation.  Warm L2 by default: launches back to back.
+ * fact_tune_ex takes options (NULL = the defaults of fact_tune):
+ *   cold_l2       1: a buffer twice the size of L2 is overwritten before every timed launch and every launch
+ *                 is timed by an event pair of its own -- the protocol of a benchmark that flushes L2
+ *   verify        0 switches the verify gate off (default 1)
+ *   inject_fault  index (in sweep order) of a candidate whose verification is run against a deliberately
+ *                 wrong reference, -1 for none: the gate's own test -- that candidate must come back
+ *                 FACT_TUNE_VERIFY_FAILED although its output is right
+ *   records       caller's array of max_records entries (may be NULL): one per candidate in sweep order --
+ *                 the configuration as resolved, what happened to it, its time per launch (ms), that time
+ *                 relative to the default configuration's, and worst |cand - ref| / tolerance; *n_records
+ *                 receives the number of candidates (which may exceed max_records)
+ * This is the one compute-path call that allocates: for its own duration it holds the FP32 reference copy
+ * (4 bytes per output element), its events and, in cold mode, the L2-sized buffer.  It returns
+ * FACT_ERR_UNSUPPORTED when the residual aliases the output (every candidate would read its predecessor's
+ * result) and when no candidate could be timed. */
+typedef enum {
+  FACT_TUNE_TIMED = 0,         /* verified and timed */
+  FACT_TUNE_INFEASIBLE = 1,    /* rejected on the host (budget / unsupported combination): never launched */
+  FACT_TUNE_NO_WORKSPACE = 2,  /* needs more scratch than the caller passed: never launched */
+  FACT_TUNE_LAUNCH_FAILED = 3, /* a launch returned an error or a device-side wait gave up */
+  FACT_TUNE_VERIFY_FAILED = 4  /* output differs from the reference configuration's: never timed */
+} fact_tune_outcome_t;
+typedef struct {
+  fact_config_t cfg;
+  int status;        /* fact_tune_outcome_t */
+  float ms;          /* per launch in the sweep; < 0 if not timed */
+  float rel;         /* ms relative to the default configuration's; < 0 if not timed */
+  float verify_err;  /* worst |candidate - reference| / tolerance; < 0 if not verified */
+} fact_tune_record_t;
+typedef struct {
+  int cold_l2;
+  int verify;
+  int inject_fault;
+  fact_tune_record_t* records;
+  int max_records;
+  int* n_records;
+} fact_tune_opts_t;
 fact_status_t fact_tune(fact_handle_t handle, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
                         const void* A, int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
                         fact_blayout_t b_layout, const void* bias, const void* residual, int64_t ldr,
                         int64_t strideR, void* C, int64_t ldc, int64_t strideC, fact_out_t out_type,
                         fact_epilogue_t epilogue, void* workspace, size_t workspace_bytes, int warmup, int iters,
                         void* cuda_stream, fact_config_t* best, double* best_ms, int* n_tried);
+fact_status_t fact_tune_ex(fact_handle_t handle, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                           const void* A, int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                           fact_blayout_t b_layout, const void* bias, const void* residual, int64_t ldr,
+                           int64_t strideR, void* C, int64_t ldc, int64_t strideC, fact_out_t out_type,
+                           fact_epilogue_t epilogue, void* workspace, size_t workspace_bytes, int warmup, int iters,
+                           void* cuda_stream, const fact_tune_opts_t* opts, fact_config_t* best, double* best_ms,
+                           int* n_tried);
 
 /* Persist / restore the tuner's table as a text file (one line per problem
  * key; host path).  Loading merges into the handle's table. */

@@ -40,6 +40,7 @@ EXPORTED = [
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
     "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
+    "fact_tune_ex",
 ]
 
 
@@ -65,6 +66,9 @@ class Block(Structure):
                                          "norm2_beta", "w1", "b1", "w2", "b2")])
 
 
+TUNE_OUTCOMES = {0: "timed", 1: "infeasible", 2: "no_workspace", 3: "launch_failed", 4: "verify_failed"}
+
+
 class FactError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -82,6 +86,23 @@ class Config(Structure):
 
     def __repr__(self):
         return "Config(" + ", ".join(f"{k}={v}" for k, v in self.as_dict().items()) + ")"
+
+
+class TuneRecord(Structure):
+    """Mirror of fact_tune_record_t: what the tuner did with one candidate."""
+
+    _fields_ = [("cfg", Config), ("status", c_int), ("ms", c_float), ("rel", c_float), ("verify_err", c_float)]
+
+    def as_dict(self):
+        return {"cfg": self.cfg.as_dict(), "outcome": TUNE_OUTCOMES.get(int(self.status), int(self.status)),
+                "ms": float(self.ms), "rel": float(self.rel), "verify_err": float(self.verify_err)}
+
+
+class TuneOpts(Structure):
+    """Mirror of fact_tune_opts_t."""
+
+    _fields_ = [("cold_l2", c_int), ("verify", c_int), ("inject_fault", c_int), ("records", POINTER(TuneRecord)),
+                ("max_records", c_int), ("n_records", POINTER(c_int))]
 
 
 _lib = None
@@ -115,6 +136,9 @@ def lib() -> ctypes.CDLL:
     L.fact_get_config.argtypes = [vp, c_int, i64, i64, i64, i64, c_int, c_int, c_int, cfgp]
     L.fact_tune.argtypes = [vp, c_int, i64, i64, i64, i64, vp, i64, i64, vp, i64, i64, c_int, vp, vp, i64, i64, vp,
                             i64, i64, c_int, c_int, vp, sz, c_int, c_int, vp, cfgp, POINTER(c_double), POINTER(c_int)]
+    L.fact_tune_ex.argtypes = [vp, c_int, i64, i64, i64, i64, vp, i64, i64, vp, i64, i64, c_int, vp, vp, i64, i64, vp,
+                               i64, i64, c_int, c_int, vp, sz, c_int, c_int, vp, POINTER(TuneOpts), cfgp,
+                               POINTER(c_double), POINTER(c_int)]
     L.fact_tune_cache_save.argtypes = [vp, c_char_p]
     L.fact_tune_cache_load.argtypes = [vp, c_char_p]
     L.fact_device_status.argtypes = [vp, vp, POINTER(c_int)]
@@ -691,9 +715,11 @@ class Handle:
         return out
 
     def tune(self, op, A, B, layout="KN", bias=None, residual=None, epilogue="NONE", out=None,
-             out_dtype=torch.bfloat16, workspace_bytes=256 << 20, warmup=0, iters=0, stream=None):
-        """Search tile configurations for this problem on the device (fact_tune).
-        Returns (Config, best_ms, n_tried)."""
+             out_dtype=torch.bfloat16, workspace_bytes=256 << 20, warmup=0, iters=0, stream=None, cold_l2=False,
+             verify=True, inject_fault=-1, records=False):
+        """Search tile configurations for this problem on the device (fact_tune_ex): every candidate is verified
+        against the default configuration's output, then timed (cold_l2: with L2 overwritten before each launch).
+        Returns (Config, best_ms, n_tried), plus the per-candidate records (a list of dicts) with records=True."""
         batched = A.ndim == 3
         batch = A.shape[0] if batched else 1
         M, K = A.shape[-2:]
@@ -701,14 +727,21 @@ class Handle:
         N = Nw // 2 if epilogue == "SILU_GATE" else Nw
         if out is None:
             out = torch.empty(((batch, M, N) if batched else (M, N)), dtype=out_dtype, device=A.device)
+        _need_out(out, (batch, M, N) if batched else (M, N), A)
         ws = self.workspace(workspace_bytes)
         best, ms, n = Config(), c_double(0.0), c_int(0)
         self._ws_cache.clear()
-        _check(lib().fact_tune(self._h, OPS[op], batch, M, N, K, _ptr(A), _ld(A), A.stride(0) if batched else 0,
-                               _ptr(B), _ld(B), B.stride(0) if batched else 0, LAYOUTS[layout], _ptr(bias),
-                               _ptr(residual), _ld(residual) if residual is not None else 0,
-                               residual.stride(0) if (residual is not None and batched) else 0, _ptr(out), _ld(out),
-                               out.stride(0) if batched else 0, OUT_TYPES[out.dtype], EPILOGUES[epilogue], _ptr(ws),
-                               ws.numel() if ws is not None else 0, warmup, iters, self._stream(stream), byref(best),
-                               byref(ms), byref(n)), "fact_tune", self._h)
+        cap = 512
+        recs = (TuneRecord * cap)()
+        n_recs = c_int(0)
+        opts = TuneOpts(1 if cold_l2 else 0, 1 if verify else 0, int(inject_fault), recs, cap, ctypes.pointer(n_recs))
+        _check(lib().fact_tune_ex(self._h, OPS[op], batch, M, N, K, _ptr(A), _ld(A), A.stride(0) if batched else 0,
+                                  _ptr(B), _ld(B), B.stride(0) if batched else 0, LAYOUTS[layout], _ptr(bias),
+                                  _ptr(residual), _ld(residual) if residual is not None else 0,
+                                  residual.stride(0) if (residual is not None and batched) else 0, _ptr(out), _ld(out),
+                                  out.stride(0) if batched else 0, OUT_TYPES[out.dtype], EPILOGUES[epilogue], _ptr(ws),
+                                  ws.numel() if ws is not None else 0, warmup, iters, self._stream(stream),
+                                  byref(opts), byref(best), byref(ms), byref(n)), "fact_tune_ex", self._h)
+        if records:
+            return best, float(ms.value), int(n.value), [recs[i].as_dict() for i in range(min(cap, n_recs.value))]
         return best, float(ms.value), int(n.value)

@@ -20,6 +20,7 @@
 #include "gemm_kernel.cuh"
 #include "attention_kernel.cuh"
 #include "norm_kernel.cuh"
+#include "tune_kernels.cuh"
 
 // Storage of fact_gemm_splitk_static: split-K scratch and a status word that live in the library's own
 // device image, so that entry point never has to allocate.  Every GPU that loads the library holds these
@@ -1148,25 +1149,81 @@ fact_status_t fact_linear_fp8(fact_handle_t h, int64_t M, int64_t N_out, int64_t
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
 }
 
-fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
-                        int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
-                        fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, int64_t strideR,
-                        void* C, int64_t ldc, int64_t strideC, fact_out_t out, fact_epilogue_t epi, void* ws,
-                        size_t ws_bytes, int warmup, int iters, void* stream_v, fact_config_t* best, double* best_ms,
-                        int* n_tried) {
+fact_status_t fact_tune_ex(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K,
+                           const void* A, int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                           fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr,
+                           int64_t strideR, void* C, int64_t ldc, int64_t strideC, fact_out_t out, fact_epilogue_t epi,
+                           void* ws, size_t ws_bytes, int warmup, int iters, void* stream_v,
+                           const fact_tune_opts_t* opts, fact_config_t* best, double* best_ms, int* n_tried) {
   if (!h || !best) return FACT_ERR_INVALID_ARG;
   Problem q = make_problem(op, batch, M, N, K, A, lda, strideA, B, ldb, strideB, layout, bias, residual, ldr, strideR,
                            C, ldc, strideC, out, epi);
   fact_status_t st = validate(q);
   if (st != FACT_OK) return st;
   if (q.batch == 0 || q.M == 0 || q.N_out == 0 || q.K == 0) return resolve_config(h, q, nullptr, 0, best);
+  if (q.R && q.R == q.C) return FACT_ERR_UNSUPPORTED;  // every candidate would read the previous one's output
   if (warmup <= 0) warmup = 5;
   if (iters <= 0) iters = 20;
+  const bool verify = !opts || opts->verify != 0;
+  const bool cold = opts && opts->cold_l2 != 0;
+  const int inject = opts ? opts->inject_fault : -1;
+  fact_tune_record_t* recs = opts ? opts->records : nullptr;
+  const int max_recs = (opts && recs) ? opts->max_records : 0;
+  int n_recs = 0;
+  auto record = [&](const fact_config_t& c, int status, double ms, double rel, double verr) -> int {
+    const int at = n_recs++;
+    if (at < max_recs) {
+      recs[at].cfg = c;
+      recs[at].status = status;
+      recs[at].ms = (float)ms;
+      recs[at].rel = (float)rel;
+      recs[at].verify_err = (float)verr;
+    }
+    return at;
+  };
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
-  cudaEvent_t e0, e1;
-  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return FACT_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
 
-  // Candidate axes: pair size, tile width, ring depth, K slices.
+  // The tuner is off the per-call path and owns what it needs for the length of this call: event pairs, a dense FP32
+  // copy of the reference output for the verify gate, a buffer larger than L2 for the cold-L2 mode.
+  const int n_ev = cold ? iters : 1;
+  std::vector<cudaEvent_t> ev0((size_t)n_ev), ev1((size_t)n_ev);
+  float* d_ref = nullptr;
+  double* d_sum = nullptr;       // [0] sum |ref|, then two 32-bit result words behind it
+  unsigned char* d_flush = nullptr;
+  size_t flush_bytes = 0;
+  bool setup_ok = true;
+  for (int i = 0; i < n_ev; ++i)
+    setup_ok = setup_ok && cudaEventCreate(&ev0[(size_t)i]) == cudaSuccess && cudaEventCreate(&ev1[(size_t)i]) == cudaSuccess;
+  const long long out_elems = (long long)q.batch * q.M * q.N_out;
+  if (verify)
+    setup_ok = setup_ok && cudaMalloc(&d_ref, (size_t)out_elems * sizeof(float)) == cudaSuccess &&
+               cudaMalloc(&d_sum, 2 * sizeof(double)) == cudaSuccess;
+  if (cold) {
+    int l2 = 0;
+    cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, h->device);
+    flush_bytes = std::max<size_t>((size_t)256 << 20, 2 * (size_t)std::max(l2, 0));
+    setup_ok = setup_ok && cudaMalloc(&d_flush, flush_bytes) == cudaSuccess;
+  }
+  auto cleanup = [&]() {
+    for (int i = 0; i < n_ev; ++i) {
+      cudaEventDestroy(ev0[(size_t)i]);
+      cudaEventDestroy(ev1[(size_t)i]);
+    }
+    if (d_ref) cudaFree(d_ref);
+    if (d_sum) cudaFree(d_sum);
+    if (d_flush) cudaFree(d_flush);
+    if (dev != h->device) cudaSetDevice(dev);
+  };
+  if (!setup_ok) {
+    cudaGetLastError();
+    cleanup();
+    return FACT_ERR_CUDA;
+  }
+
+  // Candidate axes: pair size, tile width, ring depth, K slices / stream-K, store path.
   std::vector<fact_config_t> cands;
   const int k_blocks = (int)((K + q.k_elems() - 1) / q.k_elems());
   for (int cg = 1; cg <= 2; ++cg) {
@@ -1209,75 +1266,180 @@ fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M,
         }
     }
   }
-  // Time `c` over `n` launches; a negative result means the candidate failed.
+  // Time `c` over `n` launches (per launch, ms); a negative result means the candidate failed.  Warm L2: the launches
+  // run back to back between one event pair.  Cold L2: a buffer twice the size of L2 is overwritten before each
+  // launch and every launch has an event pair of its own (what a benchmark that flushes L2 between launches sees).
   auto time_cfg = [&](const fact_config_t& c, int n_warm, int n) -> double {
     bool ok = true;
     for (int i = 0; i < n_warm && ok; ++i) ok = run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
     if (!ok) return -1.0;
-    cudaEventRecord(e0, stream);
-    for (int i = 0; i < n && ok; ++i) ok = run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
-    cudaEventRecord(e1, stream);
+    n = cold ? std::min(n, n_ev) : n;
+    if (cold) {
+      for (int i = 0; i < n && ok; ++i) {
+        ok = cudaMemsetAsync(d_flush, i & 0xff, flush_bytes, stream) == cudaSuccess;
+        cudaEventRecord(ev0[(size_t)i], stream);
+        ok = ok && run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
+        cudaEventRecord(ev1[(size_t)i], stream);
+      }
+    } else {
+      cudaEventRecord(ev0[0], stream);
+      for (int i = 0; i < n && ok; ++i) ok = run(h, q, &c, 0, ws, ws_bytes, stream_v) == FACT_OK;
+      cudaEventRecord(ev1[0], stream);
+    }
     int dev_status = 0;
     if (fact_device_status(h, stream_v, &dev_status) != FACT_OK || dev_status != 0 || !ok) return -1.0;
-    float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) return -1.0;
-    return (double)ms / n;
+    double total = 0.0;
+    for (int i = 0; i < (cold ? n : 1); ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ev0[(size_t)i], ev1[(size_t)i]) != cudaSuccess) return -1.0;
+      total += ms;
+    }
+    return total / n;
   };
-  // Sweep: every feasible candidate once.  A sweep lasts seconds on a power-limited part whose clock drifts, so
-  // a candidate is ranked by its time RELATIVE to the library's default configuration timed right before and after.
+  // The reference: the library's default configuration, never a previously tuned entry.
   fact_config_t ref_c;
   {
-    auto saved = h->table;  // the default must not be a previously tuned entry
+    auto saved = h->table;
     h->table.erase(make_key(q));
     const fact_status_t rs = resolve_config(h, q, nullptr, 0, &ref_c);
     h->table = saved;
     if (rs != FACT_OK || workspace_for(h, q, ref_c) > ws_bytes) {
-      cudaEventDestroy(e0);
-      cudaEventDestroy(e1);
+      cleanup();
       return rs != FACT_OK ? rs : FACT_ERR_WORKSPACE_TOO_SMALL;
     }
   }
+  // Verify gate.  The reference configuration's output is kept as a dense FP32 copy; a candidate's output must agree
+  // with it element by element to within what two correct results can differ by: both are FP32 sums of the same
+  // products in different orders (accumulation noise ~ sqrt(K) 2^-24 of the output scale), each rounded once to the
+  // output type (one BF16 ulp = 2^-8 relative when they straddle a rounding boundary).
+  TuneViewParams view;
+  view.C = C;
+  view.ldc = ldc;
+  view.strideC = strideC;
+  view.batch = (int)q.batch;
+  view.M = (int)q.M;
+  view.N = (int)q.N_out;
+  view.f32 = out == FACT_OUT_F32;
+  const int vgrid = (int)std::min<long long>((out_elems + 255) / 256, (long long)h->sm_count * 8);
+  float floor_abs = 0.f;
+  const float rel_tol = view.f32 ? 2e-4f : 0.0078125f;  // 2^-7 for BF16 outputs
+  unsigned int* d_result = verify ? reinterpret_cast<unsigned int*>(d_sum + 1) : nullptr;
+  if (verify) {
+    bool ok = cudaMemsetAsync(d_sum, 0, 2 * sizeof(double), stream) == cudaSuccess;
+    fact_tune_poison_kernel<<<vgrid, 256, 0, stream>>>(view);
+    ok = ok && run(h, q, &ref_c, 0, ws, ws_bytes, stream_v) == FACT_OK;
+    fact_tune_snapshot_kernel<<<vgrid, 256, 0, stream>>>(view, d_ref, d_sum);
+    double abs_sum = 0.0;
+    int dev_status = 0;
+    ok = ok && cudaGetLastError() == cudaSuccess && fact_device_status(h, stream_v, &dev_status) == FACT_OK &&
+         dev_status == 0 && cudaMemcpy(&abs_sum, d_sum, sizeof(double), cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (!ok || !(abs_sum == abs_sum)) {  // the reference itself failed to run, or produced NaNs
+      cudaGetLastError();
+      cleanup();
+      return FACT_ERR_CUDA;
+    }
+    const double mean_abs = abs_sum / (double)out_elems;
+    floor_abs = (float)((view.f32 ? 2e-4 : 1e-3) * mean_abs + 1e-30);
+  }
+  // worst |candidate - reference| / tolerance over the whole output; negative if the check itself failed
+  auto verify_cfg = [&](const fact_config_t& c, bool perturb) -> double {
+    fact_tune_poison_kernel<<<vgrid, 256, 0, stream>>>(view);
+    if (run(h, q, &c, 0, ws, ws_bytes, stream_v) != FACT_OK) return -1.0;
+    if (cudaMemsetAsync(d_result, 0, 2 * sizeof(unsigned int), stream) != cudaSuccess) return -1.0;
+    fact_tune_compare_kernel<<<vgrid, 256, 0, stream>>>(view, d_ref, rel_tol, floor_abs, perturb ? 1 : 0, d_result);
+    unsigned int res[2] = {0u, 0u};
+    int dev_status = 0;
+    if (cudaGetLastError() != cudaSuccess || fact_device_status(h, stream_v, &dev_status) != FACT_OK ||
+        dev_status != 0 || cudaMemcpy(res, d_result, sizeof res, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return -1.0;
+    float worst;
+    memcpy(&worst, &res[1], sizeof worst);
+    return res[0] != 0 ? std::max(1.0000001, (double)worst) : (double)worst;
+  };
+
+  // Sweep: every feasible candidate once.  A sweep lasts seconds on a power-limited part whose clock drifts, so
+  // a candidate is ranked by its time RELATIVE to the reference configuration timed right before and after.
   const int ref_iters = std::max(3, iters / 4);
-  std::vector<std::pair<double, fact_config_t>> timed;  // (relative time, configuration)
+  struct Timed {
+    double rel;
+    fact_config_t cfg;
+    int rec;
+  };
+  std::vector<Timed> timed;
   double t_ref = time_cfg(ref_c, warmup, ref_iters);
+  int cand_index = 0;
   for (const fact_config_t& c : cands) {
+    const int my_index = cand_index++;
     Plan plan;
-    if (make_plan(h, q, &c, 0, &plan) != FACT_OK) continue;  // over budget: never launched
-    if (plan.ws_bytes > ws_bytes) continue;
+    if (make_plan(h, q, &c, 0, &plan) != FACT_OK) {  // over a budget, or a combination the kernels cannot run
+      record(c, FACT_TUNE_INFEASIBLE, -1.0, -1.0, -1.0);
+      continue;
+    }
+    if (plan.ws_bytes > ws_bytes) {
+      record(plan.cfg, FACT_TUNE_NO_WORKSPACE, -1.0, -1.0, -1.0);
+      continue;
+    }
+    double verr = 0.0;
+    if (verify) {
+      verr = verify_cfg(c, my_index == inject);
+      if (verr < 0.0) {
+        record(plan.cfg, FACT_TUNE_LAUNCH_FAILED, -1.0, -1.0, -1.0);
+        continue;
+      }
+      if (verr > 1.0) {  // wrong numbers: recorded, never timed, never eligible
+        record(plan.cfg, FACT_TUNE_VERIFY_FAILED, -1.0, -1.0, verr);
+        continue;
+      }
+    }
     const double t = time_cfg(c, warmup, iters);
     const double t_ref_after = time_cfg(ref_c, 1, ref_iters);
-    if (t >= 0 && t_ref > 0 && t_ref_after > 0) timed.push_back(std::make_pair(2.0 * t / (t_ref + t_ref_after), plan.cfg));
+    if (t >= 0 && t_ref > 0 && t_ref_after > 0) {
+      const double rel = 2.0 * t / (t_ref + t_ref_after);
+      timed.push_back({rel, plan.cfg, record(plan.cfg, FACT_TUNE_TIMED, t, rel, verr)});
+    } else {
+      record(plan.cfg, FACT_TUNE_LAUNCH_FAILED, -1.0, -1.0, verr);
+    }
     if (t_ref_after > 0) t_ref = t_ref_after;
   }
   const int tried = (int)timed.size();
-  std::sort(timed.begin(), timed.end(),
-            [](const std::pair<double, fact_config_t>& x, const std::pair<double, fact_config_t>& y) {
-              return x.first < y.first;
-            });
+  std::sort(timed.begin(), timed.end(), [](const Timed& x, const Timed& y) { return x.rel < y.rel; });
   // Play-off: the few fastest candidates are timed again in alternation and ranked by their best round.
   double best_t = 1e30;
   fact_config_t best_c;
   memset(&best_c, 0, sizeof best_c);
   const int finalists = std::min(tried, 4);
-  std::vector<double> best_round(finalists, 1e30);
+  std::vector<double> best_round((size_t)finalists, 1e30);
   for (int round = 0; round < 3; ++round)
     for (int i = 0; i < finalists; ++i) {
-      const double t = time_cfg(timed[i].second, 2, iters);
-      if (t >= 0) best_round[i] = std::min(best_round[i], t);
+      const double t = time_cfg(timed[(size_t)i].cfg, 2, iters);
+      if (t >= 0) best_round[(size_t)i] = std::min(best_round[(size_t)i], t);
     }
   for (int i = 0; i < finalists; ++i)
-    if (best_round[i] < best_t) {
-      best_t = best_round[i];
-      best_c = timed[i].second;
+    if (best_round[(size_t)i] < best_t) {
+      best_t = best_round[(size_t)i];
+      best_c = timed[(size_t)i].cfg;
     }
-  cudaEventDestroy(e0);
-  cudaEventDestroy(e1);
+  // the caller's output ends as the winner's (or, with nothing timed, the reference's) result
+  if (tried > 0) run(h, q, &best_c, 0, ws, ws_bytes, stream_v);
+  cudaStreamSynchronize(stream);
+  cleanup();
+  if (opts && opts->n_records) *opts->n_records = n_recs;
   if (n_tried) *n_tried = tried;
   if (tried == 0) return FACT_ERR_UNSUPPORTED;
   h->table[make_key(q)] = best_c;
   *best = best_c;
   if (best_ms) *best_ms = best_t;
   return FACT_OK;
+}
+
+fact_status_t fact_tune(fact_handle_t h, fact_op_t op, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
+                        int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                        fact_blayout_t layout, const void* bias, const void* residual, int64_t ldr, int64_t strideR,
+                        void* C, int64_t ldc, int64_t strideC, fact_out_t out, fact_epilogue_t epi, void* ws,
+                        size_t ws_bytes, int warmup, int iters, void* stream_v, fact_config_t* best, double* best_ms,
+                        int* n_tried) {
+  return fact_tune_ex(h, op, batch, M, N, K, A, lda, strideA, B, ldb, strideB, layout, bias, residual, ldr, strideR, C,
+                      ldc, strideC, out, epi, ws, ws_bytes, warmup, iters, stream_v, nullptr, best, best_ms, n_tried);
 }
 
 fact_status_t fact_tune_cache_save(fact_handle_t h, const char* path) {

@@ -353,3 +353,40 @@ def test_tuner_returns_a_runnable_config_and_the_table_round_trips(h, tmp_path):
     assert {k: after[k] for k in ("tile_n", "cta_group", "stages")} == {k: d[k] for k in ("tile_n", "cta_group", "stages")}
     assert isinstance(before, dict)
     h2.close()
+
+
+def test_tuner_verifies_before_it_times_and_records_every_candidate(h):
+    """Section 4.2: verify, then benchmark.  Every candidate's output is compared on the device with the default
+    configuration's before it is timed; the record says what happened to each.  The gate itself is tested by letting
+    one candidate (a correct one) be compared with a deliberately wrong reference: it must be rejected, untimed."""
+    case = mk("tune_gate", 640, 384, 1024 + 64, epilogue="BIAS_GELU_TANH", layout="NK")
+    ins = wl.make_inputs(case)
+    dev = "cuda:0"
+    X, W, b = ins.X.to(dev), ins.W.to(dev), ins.bias.to(dev)
+    out = torch.empty(case.M, case.N, dtype=torch.bfloat16, device=dev)
+    cfg, ms, n, recs = h.tune("linear", X, W, layout="NK", bias=b, epilogue=case.epilogue, out=out, warmup=1, iters=3,
+                              records=True)
+    outcomes = [r["outcome"] for r in recs]
+    assert n == outcomes.count("timed") and n >= 4
+    assert "verify_failed" not in outcomes and "launch_failed" not in outcomes
+    assert all(0 <= r["verify_err"] <= 1 and r["ms"] > 0 and r["rel"] > 0 for r in recs if r["outcome"] == "timed")
+    assert all(r["ms"] < 0 for r in recs if r["outcome"] != "timed")
+    # the output is left holding the winner's result: the oracle's, within the gates
+    torch.cuda.synchronize()
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", case.epilogue)
+    assert c <= 1 and t <= 1, (c, t)
+    # the gate's own test: the k-th feasible candidate is checked against a wrong reference
+    k = outcomes.index("timed")
+    cfg2, ms2, n2, recs2 = h.tune("linear", X, W, layout="NK", bias=b, epilogue=case.epilogue, out=out, warmup=1,
+                                  iters=3, records=True, inject_fault=k)
+    assert recs2[k]["outcome"] == "verify_failed" and recs2[k]["verify_err"] > 1 and recs2[k]["ms"] < 0
+    assert n2 == n - 1 and [r["outcome"] for i, r in enumerate(recs2) if i != k] == \
+           [o for i, o in enumerate(outcomes) if i != k]
+    # cold-L2 timing and FP32 output through the same gate
+    case3 = mk("tune_gate_f32", 256, 256, 8192, op="gemm_splitk", layout="KN", out="f32", x_dist="uniform",
+               w_dist="uniform")
+    ins3 = wl.make_inputs(case3)
+    cfg3, ms3, n3, recs3 = h.tune("gemm_splitk", ins3.X.to(dev), ins3.W.to(dev), layout="KN",
+                                  out_dtype=torch.float32, warmup=1, iters=3, cold_l2=True, records=True)
+    assert n3 >= 2 and "verify_failed" not in [r["outcome"] for r in recs3]
+    check_case(h, case3, ins=ins3)  # runs with the tuned entry
