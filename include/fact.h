@@ -131,9 +131,19 @@ typedef enum {
  *                tensor stores, 3 = the staged epilogue's arithmetic with every row stored from registers in
  *                32-byte pieces (Y 32-byte aligned, ldy and N_out multiples of 32 bytes, whole data-parallel
  *                tiles: no K slices, stream-K, groups or row sums; pays when K is long, FACT_ERR_UNSUPPORTED
- *                where it cannot run) */
+ *                where it cannot run)
+ *   schedule     how data-parallel tiles reach the CTAs (the grid-level policy of Section 4.2, Action 2): 0 = the
+ *                library's choice, 1 = static: a persistent grid of one CTA group per SM (pair of SMs), group g
+ *                takes tiles g, g + G, g + 2G, ...; 2 = dynamic: the grid has one cluster per tile, the clusters
+ *                that get an SM keep it and obtain further tiles by cancelling the launch of clusters that have
+ *                not started (clusterlaunchcontrol; a twelfth warp per CTA keeps one request in flight ahead of
+ *                the tile in progress), so a CTA group that falls behind simply takes fewer tiles.  Which group
+ *                computes a tile never changes a value: every tile is summed by one group in the same order.
+ *                Dynamic scheduling serves whole tiles only (no K slices, stream-K, row sums, folded
+ *                normalisation, register row stores or row softmax: FACT_ERR_UNSUPPORTED with those), and is
+ *                the static schedule when all tiles fit one wave. */
 typedef struct {
-  int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode;
+  int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode, schedule;
 } fact_config_t;
 
 /* Create / destroy a handle bound to CUDA device `device`.  fact_create makes

@@ -79,7 +79,7 @@ class Config(Structure):
     """Mirror of fact_config_t; zero fields mean "library's choice"."""
 
     _fields_ = [(n, c_int) for n in
-                ("tile_m", "tile_n", "tile_k", "stages", "cta_group", "raster_group", "split_k", "store_mode")]
+                ("tile_m", "tile_n", "tile_k", "stages", "cta_group", "raster_group", "split_k", "store_mode", "schedule")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

@@ -189,6 +189,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder_p;
+  // the set-up above may overlap the tail of the previous kernel in the stream; global memory only from here on
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
 
   // Items are numbered with the query position as the slow index, heaviest first (the late rows of a causal
   // problem), so neighbouring CTAs work on query heads that share K and V.

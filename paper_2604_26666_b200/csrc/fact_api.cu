@@ -14,6 +14,7 @@
 #include <map>
 #include <string>
 #include <tuple>
+#include <utility>
 #include <vector>
 
 #include "fact.h"
@@ -43,7 +44,8 @@ constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the w
                                          // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
 constexpr int kStatusInts = 64;  // status word, clock / profile counters, grid-barrier counters; stream-K flags follow
-constexpr int kDiagnosticFlags = 256 | 2048;  // FACT_DEBUG_FLAGS bits that leave results intact: cycle counters, no K serpentine
+constexpr int kDiagnosticFlags = 256 | 2048 | 4096;  // FACT_DEBUG_FLAGS bits that leave results intact: cycle counters,
+                                                      // no K serpentine, no programmatic dependent launch
 constexpr int kMaxGroups = 4096;  // row groups of a grouped GEMM (the handle's device table holds 2 x (kMaxGroups + 1) ints)
 
 // Key of the tuner's table: everything that changes which configuration is best.
@@ -81,6 +83,7 @@ struct Problem {
 struct Plan {
   fact_config_t cfg;
   bool from_table = false;  // cfg came from the tuner's table: its store mode and K slices are hints, not demands
+  bool dynamic = false;     // tiles are handed out through cluster launch control (one cluster of the grid per tile)
   int smem_bytes;
   int grid;
   size_t ws_bytes;
@@ -98,7 +101,7 @@ struct fact_handle_s {
   EncodeTiledFn encode = nullptr;
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
-  std::bitset<128> configured_mask;  // kernels whose dynamic shared-memory limit was raised
+  std::bitset<192> configured_mask;  // kernels whose dynamic shared-memory limit was raised
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: diagnostics (256 cycle counters, 2048 no K serpentine); the
                                  // work-skipping experiment switches only in a -DFACT_EXPERIMENTS build
@@ -119,6 +122,38 @@ fact_status_t cuda_fail(fact_handle_t h, const char* where, cudaError_t e) {
   return FACT_ERR_CUDA;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the stream
+// is still running (its own griddepcontrol.wait holds it before its first global-memory access), so its set-up --
+// barrier initialisation, tensor-memory allocation, descriptor prefetch -- overlaps the predecessor's tail.
+// Every kernel launched this way executes griddepcontrol.wait before it touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(fact_handle_t h, void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                       cudaStream_t stream, int cluster, Args&&... args) {
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3(grid, 1, 1);
+  lc.blockDim = dim3(block, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (!(h->debug_flags & 4096)) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  lc.attrs = attr;
+  lc.numAttrs = n;
+  return cudaLaunchKernelEx(&lc, kern, std::forward<Args>(args)...);
+}
+
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 uint32_t pow2_at_least(uint32_t x) {
   uint32_t r = 32;
@@ -133,9 +168,10 @@ int stage_bytes_for(int tile_n, int cta_group) { return (int)kStageBytesA + (til
 // into, but only short main loops (small K) have no slack to hide that load behind.
 int epi_bufs_for(const Problem& q) { return (q.epi == FACT_EPI_BIAS_RESIDUAL && q.K <= 2048) ? 2 : 1; }
 
+// (the dynamic scheduler's ring is counted for every configuration: 192 bytes never cost a stage)
 int smem_bytes_for(const Problem& q, int tile_n, int cta_group, int stages) {
   return stages * stage_bytes_for(tile_n, cta_group) + (int)epi_smem_bytes(epi_bufs_for(q)) + (int)kCtrlSmemBytes +
-         (q.norm == 1 ? (int)kNormCsBytes : 0);
+         (q.norm == 1 ? (int)kNormCsBytes : (int)kSchedSmemBytes);
 }
 
 int max_stages_for(const Problem& q, int tile_n, int cta_group) {
@@ -160,6 +196,53 @@ bool tile_ok(const Problem& q, int tile_n, int cg) {
     if (gate && (tile_n / 2) % 64) return false;
   }
   return true;
+}
+
+// Raster model: which tiles run at the same time decides the DRAM traffic, and on a power-limited part every extra
+// gigabyte costs SM clock.  All CTA groups walk K in step, so what one wave of `slots` concurrent tiles fetches is
+// the union of its operand slabs: with groups of G tiles of one dimension (the raster walks those fastest) a wave
+// covers G slabs of that operand and ceil(slots / G) slabs of the other.  Between waves the G slabs of the grouped
+// operand are wanted again and the others are new; what survives in L2 is what the streamed slabs of two waves
+// leave of an effective capacity of 55 MB -- the figure that reproduces the measured DRAM reads (8192^3, 256 x 256
+// tiles: 1.04 GB with groups of 8 m-tiles, 1.00 GB with 12, 0.96 GB with 16; the Llama down projection: 1.43 GB with
+// groups of 4 n-tiles, 1.01 GB with 8; nominal L2 126 MB on two dies).  Returns G > 0 for groups of m-tiles, G < 0
+// for groups of n-tiles.
+int raster_model(fact_handle_t h, const Problem& q, const fact_config_t& c) {
+  const double l2_eff = 55.0 * 1024 * 1024;
+  const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
+  const long long tiles_m = std::max<long long>(1, (q.M + c.tile_m - 1) / c.tile_m);
+  const long long tiles_n = std::max<long long>(1, (q.N_out + out_cols - 1) / out_cols);
+  const double esz = q.fp8 ? 1.0 : 2.0;
+  const double slab_m = esz * c.tile_m * (double)std::max<long long>(q.K, 1);  // rows of X of one m-tile
+  const double slab_n = esz * c.tile_n * (double)std::max<long long>(q.K, 1);  // columns of W of one n-tile
+  const double slots = std::max(1, h->sm_count / std::max(1, c.cta_group));
+  double best = 1e300;
+  int best_g = (int)tiles_m;
+  for (int dir = 0; dir < 2; ++dir) {
+    const long long n_grouped = dir == 0 ? tiles_m : tiles_n, n_other = dir == 0 ? tiles_n : tiles_m;
+    const double slab_g = dir == 0 ? slab_m : slab_n, slab_o = dir == 0 ? slab_n : slab_m;
+    // DRAM bytes of the waves that work through one group of `gs` tiles of the grouped dimension
+    auto group_bytes = [&](double gs) {
+      // (a wave that straddles two groups touches the slabs of both: on average slots / (2 x tiles per group) more;
+      // a group smaller than a wave: the wave spans several groups and every slab of the other operand)
+      const double straddle = 1.0 + std::min(1.0, slots / (2.0 * gs * (double)n_other));
+      const double kept = std::max(gs, slots / (double)n_other) * slab_g * straddle;                     // wanted again
+      const double streamed = std::min<double>((double)n_other, std::ceil(slots / gs)) * slab_o;        // new per wave
+      const double survive = std::max(0.0, std::min(1.0, (l2_eff - 2.0 * streamed) / kept));
+      const double group_waves = gs * (double)n_other / slots;
+      // what survives is fetched once per group, the rest once per wave
+      return group_waves * (streamed + (1.0 - survive) * kept) + survive * gs * slab_g;
+    };
+    for (long long g = 1; g <= n_grouped; ++g) {
+      const long long full = n_grouped / g, rem = n_grouped % g;
+      const double total = (double)full * group_bytes((double)g) + (rem ? group_bytes((double)rem) : 0.0);
+      if (total < best * 0.999) {
+        best = total;
+        best_g = dir == 0 ? (int)g : -(int)g;
+      }
+    }
+  }
+  return best_g;
 }
 
 // Fill every zero field of `cfg`.  Returns FACT_ERR_UNSUPPORTED for a combination the kernels cannot run.
@@ -243,23 +326,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.stages == 0) c.stages = smax;
   if (from_table && c.stages > smax) c.stages = smax;  // a table written when the other buffers were smaller
   if (c.stages < 2 || c.stages > smax) return FACT_ERR_UNSUPPORTED;
-  if (c.raster_group == 0) {
-    // Raster model.  With a group of G m-tiles the CTAs walk the n-tiles of that group; the group's slab of X
-    // (G * tile_m rows * K) is reused from L2 by every n-tile if it fits there, and W is streamed once per group:
-    // DRAM bytes = X + W * ceil(tiles_m / G).  Grouping n-tiles instead (a negative raster_group) keeps a slab
-    // of W resident and streams X once per group.  G is the largest group whose slab stays within a 32 MB share
-    // of L2; the direction with fewer modelled bytes wins.  (DRAM traffic is not the bound of these kernels, but
-    // on a power-limited part every extra gigabyte costs SM clock: 18 % of run time on the gate/up projection.)
-    const double slab_budget = 32.0 * 1024 * 1024;
-    const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
-    const long long tiles_m = (q.M + c.tile_m - 1) / c.tile_m, tiles_n = (q.N_out + out_cols - 1) / out_cols;
-    const double x_bytes = 2.0 * q.M * q.K, w_bytes = 2.0 * q.Nw() * q.K;
-    const long long gm = std::max<long long>(1, std::min<long long>(tiles_m, (long long)(slab_budget / (2.0 * c.tile_m * std::max<long long>(q.K, 1)))));
-    const long long gn = std::max<long long>(1, std::min<long long>(tiles_n, (long long)(slab_budget / (2.0 * c.tile_n * std::max<long long>(q.K, 1)))));
-    const double cost_m = x_bytes + w_bytes * (double)((tiles_m + gm - 1) / gm);
-    const double cost_n = w_bytes + x_bytes * (double)((tiles_n + gn - 1) / gn);
-    c.raster_group = (cost_n < cost_m * 0.95) ? -(int)gn : (int)gm;
-  }
+  if (c.raster_group == 0) c.raster_group = raster_model(h, q, c);
   const int k_blocks = (int)((q.K + q.k_elems() - 1) / q.k_elems());
   if (c.split_k == 0) {
     c.split_k = 1;
@@ -275,6 +342,8 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.split_k < -2) return FACT_ERR_INVALID_ARG;
   if (c.split_k > 0) c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
   if (c.store_mode < 0 || c.store_mode > 3) return FACT_ERR_INVALID_ARG;
+  if (c.schedule < 0 || c.schedule > 2) return FACT_ERR_INVALID_ARG;
+  if (c.schedule == 0) c.schedule = 1;
   *out = c;
   if (from_table_out) *from_table_out = from_table;
   return FACT_OK;
@@ -495,6 +564,20 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   if (plan->smem_bytes > kSmemBudget || kSmemBudget > h->max_smem) return FACT_ERR_UNSUPPORTED;
   const int slots = std::max(1, h->sm_count / cg);
   plan->grid = (int)std::min<long long>(slots, units) * cg;
+  plan->dynamic = false;
+  if (c.schedule == 2) {
+    // whole data-parallel tiles through the ordinary epilogues only; a table entry tuned on another call's
+    // circumstances falls back to the static schedule, a caller's own request is refused
+    const bool can = c.split_k == 1 && !p.row_stores && !q.stats_out && !q.norm && q.epi != FACT_EPI_BIAS_SOFTMAX &&
+                     units * cg <= 0x7fffffffLL;
+    if (!can && !plan->from_table) return FACT_ERR_UNSUPPORTED;
+    if (can && units > slots) {  // (one wave or less: every cluster has an SM at once, nothing to hand out)
+      plan->dynamic = true;
+      plan->grid = (int)(units * cg);
+    } else if (!can) {
+      plan->cfg.schedule = 1;
+    }
+  }
   if (c.split_k < 0) {
     // Stream-K: the staged epilogue parks and finishes the pieces, so an output it cannot store is data-parallel.
     const int sk = p.store_tma ? sk_tiles_for(h, q, c) : 0;
@@ -534,10 +617,10 @@ fact_status_t encode_map(fact_handle_t h, CUtensorMap* map, const void* base, ui
   return FACT_OK;
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0>
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0, bool DYN = false>
 fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                               cudaStream_t stream) {
-  auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED, EXT>;
+  auto kern = fact_gemm_kernel<CG, EPI, SK, GROUPED, EXT, DYN>;
   if (slot < 0) {  // (no bit left in the handle's mask for these instantiations: set the attribute on every launch)
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
@@ -546,22 +629,8 @@ fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
     h->configured_mask.set((size_t)slot);
   }
-  cudaLaunchConfig_t lc;
-  memset(&lc, 0, sizeof lc);
-  lc.gridDim = dim3((unsigned)plan.grid, 1, 1);
-  lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = (size_t)plan.smem_bytes;
-  lc.stream = stream;
-  cudaLaunchAttribute attr[1];
-  if (CG == 2) {
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-  }
-  cudaError_t e = cudaLaunchKernelEx(&lc, kern, tm[0], tm[1], tm[2], tm[3], plan.p);
+  cudaError_t e = launch_pdl(h, kern, (unsigned)plan.grid, (unsigned)(kThreads + (DYN ? 32 : 0)),
+                             (size_t)plan.smem_bytes, stream, CG, tm[0], tm[1], tm[2], tm[3], plan.p);
   if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx", e);
   h->launches++;
   return FACT_OK;
@@ -615,16 +684,17 @@ fact_status_t launch_epi_sk(fact_handle_t h, int epi, const Plan& plan, const CU
   }
 }
 
-// The grouped instantiations (direct stores, data-parallel tiles).
-template <int CG>
-fact_status_t launch_epi_grouped(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+// The grouped instantiations (data-parallel tiles), and the dynamically scheduled ones, grouped or not.
+template <int CG, bool GROUPED, bool DYN>
+fact_status_t launch_epi_dp(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  const int base = 80 + (GROUPED ? 32 : 0) + (DYN ? 16 : 0) + (CG - 1) * 8;
   switch (epi) {
-    case kEpiNone: return launch_instance<CG, kEpiNone, false, true>(h, -1, plan, tm, stream);
-    case kEpiBias: return launch_instance<CG, kEpiBias, false, true>(h, -1, plan, tm, stream);
-    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, true>(h, -1, plan, tm, stream);
-    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, true>(h, -1, plan, tm, stream);
-    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, true>(h, -1, plan, tm, stream);
-    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, true>(h, -1, plan, tm, stream);
+    case kEpiNone: return launch_instance<CG, kEpiNone, false, GROUPED, 0, DYN>(h, base + 0, plan, tm, stream);
+    case kEpiBias: return launch_instance<CG, kEpiBias, false, GROUPED, 0, DYN>(h, base + 1, plan, tm, stream);
+    case kEpiBiasRelu: return launch_instance<CG, kEpiBiasRelu, false, GROUPED, 0, DYN>(h, base + 2, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_instance<CG, kEpiBiasGeluTanh, false, GROUPED, 0, DYN>(h, base + 3, plan, tm, stream);
+    case kEpiSiluGate: return launch_instance<CG, kEpiSiluGate, false, GROUPED, 0, DYN>(h, base + 4, plan, tm, stream);
+    case kEpiBiasResidual: return launch_instance<CG, kEpiBiasResidual, false, GROUPED, 0, DYN>(h, base + 5, plan, tm, stream);
     default: return FACT_ERR_INVALID_ARG;
   }
 }
@@ -652,8 +722,7 @@ fact_status_t launch_reduce(fact_handle_t h, const Problem& q, const Plan& plan,
   r.alpha = q.fp8 ? q.alpha : 1.f;
   const long long total = 4LL * r.batch * r.M * ((r.N_out + 3) / 4);  // four threads per group of 4 columns
   const int blocks = (int)std::min<long long>((total + 127) / 128, (long long)h->sm_count * 16);
-  fact_splitk_reduce_kernel<<<std::max(1, blocks), 128, 0, stream>>>(r);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(h, fact_splitk_reduce_kernel, (unsigned)std::max(1, blocks), 128u, 0, stream, 1, r);
   if (e != cudaSuccess) return cuda_fail(h, "split-K reduce launch", e);
   h->launches++;
   return FACT_OK;
@@ -711,8 +780,10 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     plan.p.total_units = (int)units;
     plan.p.strideC = 0;
     plan.p.strideR = 0;
-    plan.grid = (int)std::min<long long>(std::max(1, h->sm_count / plan.cfg.cta_group), std::max<long long>(units, 1)) *
-                plan.cfg.cta_group;
+    const long long g_slots = std::max(1, h->sm_count / plan.cfg.cta_group);
+    plan.grid = (int)std::min<long long>(g_slots, std::max<long long>(units, 1)) * plan.cfg.cta_group;
+    plan.dynamic = plan.cfg.schedule == 2 && units > g_slots && units * plan.cfg.cta_group <= 0x7fffffffLL;
+    if (plan.dynamic) plan.grid = (int)(units * plan.cfg.cta_group);
   }
   if (plan.cfg.split_k < 0 && (q.stats_out || q.norm)) {
     // the extras live in the data-parallel instantiations: a stream-K choice (the caller's or the table's) is dropped
@@ -805,8 +876,13 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       }
     }
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
-    if (q.groups > 0) st = plan.cfg.cta_group == 2 ? launch_epi_grouped<2>(h, epi, plan, tm, stream)
-                                                   : launch_epi_grouped<1>(h, epi, plan, tm, stream);
+    const bool two = plan.cfg.cta_group == 2;
+    if (q.groups > 0 && plan.dynamic) st = two ? launch_epi_dp<2, true, true>(h, epi, plan, tm, stream)
+                                               : launch_epi_dp<1, true, true>(h, epi, plan, tm, stream);
+    else if (q.groups > 0) st = two ? launch_epi_dp<2, true, false>(h, epi, plan, tm, stream)
+                                    : launch_epi_dp<1, true, false>(h, epi, plan, tm, stream);
+    else if (plan.dynamic) st = two ? launch_epi_dp<2, false, true>(h, epi, plan, tm, stream)
+                                    : launch_epi_dp<1, false, true>(h, epi, plan, tm, stream);
     else if (plan.p.row_stores && !split) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 3>(h, epi, plan, tm, stream)
                                                                        : launch_epi_ext<1, 3>(h, epi, plan, tm, stream);
     else if (q.norm) st = plan.cfg.cta_group == 2 ? launch_epi_ext<2, 2>(h, epi, plan, tm, stream)
@@ -1256,11 +1332,17 @@ fact_status_t fact_tune_ex(fact_handle_t h, fact_op_t op, int64_t batch, int64_t
       // short timing run cannot resolve; the model in resolve_config chooses it)
       for (int stg : stage_opts)
         for (int sp : splits) {
-          fact_config_t c = {128 * cg, tn, q.k_elems(), stg, cg, 0, sp, 0};
+          fact_config_t c = {128 * cg, tn, q.k_elems(), stg, cg, 0, sp, 0, 0};
           cands.push_back(c);
           // whole tiles with a long main loop: also with the rows stored from registers (infeasible ones drop out)
           if (sp == 1 && k_blocks >= 32) {
             c.store_mode = 3;
+            cands.push_back(c);
+            c.store_mode = 0;
+          }
+          // more than one wave of whole tiles: also handed out dynamically
+          if (sp == 1 && tiles > slots && stg == smax) {
+            c.schedule = 2;
             cands.push_back(c);
           }
         }
@@ -1446,13 +1528,13 @@ fact_status_t fact_tune_cache_save(fact_handle_t h, const char* path) {
   if (!h || !path) return FACT_ERR_INVALID_ARG;
   FILE* f = fopen(path, "w");
   if (!f) return FACT_ERR_INVALID_ARG;
-  fprintf(f, "# libfact tuner table v1: op epilogue layout out batch M N K | tile_m tile_n tile_k stages cta_group raster_group split_k store_mode\n");
+  fprintf(f, "# libfact tuner table v2: op epilogue layout out batch M N K | tile_m tile_n tile_k stages cta_group raster_group split_k store_mode schedule\n");
   for (const auto& kv : h->table) {
     const TuneKey& k = kv.first;
     const fact_config_t& c = kv.second;
-    fprintf(f, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d\n", std::get<0>(k), std::get<1>(k),
+    fprintf(f, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d %d\n", std::get<0>(k), std::get<1>(k),
             std::get<2>(k), std::get<3>(k), std::get<4>(k), std::get<5>(k), std::get<6>(k), std::get<7>(k), c.tile_m,
-            c.tile_n, c.tile_k, c.stages, c.cta_group, c.raster_group, c.split_k, c.store_mode);
+            c.tile_n, c.tile_k, c.stages, c.cta_group, c.raster_group, c.split_k, c.store_mode, c.schedule);
   }
   fclose(f);
   return FACT_OK;
@@ -1468,9 +1550,11 @@ fact_status_t fact_tune_cache_load(fact_handle_t h, const char* path) {
     int op, epi, lay, out;
     long long b, M, N, K;
     fact_config_t c;
-    if (sscanf(line, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d", &op, &epi, &lay, &out, &b, &M, &N, &K,
-               &c.tile_m, &c.tile_n, &c.tile_k, &c.stages, &c.cta_group, &c.raster_group, &c.split_k,
-               &c.store_mode) != 16)
+    memset(&c, 0, sizeof c);
+    // (the ninth configuration field is absent from tables written before the schedule field existed)
+    if (sscanf(line, "%d %d %d %d %lld %lld %lld %lld | %d %d %d %d %d %d %d %d %d", &op, &epi, &lay, &out, &b, &M, &N,
+               &K, &c.tile_m, &c.tile_n, &c.tile_k, &c.stages, &c.cta_group, &c.raster_group, &c.split_k,
+               &c.store_mode, &c.schedule) < 16)
       continue;
     h->table[TuneKey(op, epi, lay, out, b, M, N, K)] = c;
   }
@@ -1584,9 +1668,10 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      if (head_dim == 64) fact_attention_kernel<64><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
-      else fact_attention_kernel<128><<<(unsigned)ctas, kAttnThreads, smem, stream>>>(tq, tk, tv, to, p);
-      cudaError_t e = cudaGetLastError();
+      cudaError_t e = head_dim == 64 ? launch_pdl(h, fact_attention_kernel<64>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                                  (size_t)smem, stream, 1, tq, tk, tv, to, p)
+                                     : launch_pdl(h, fact_attention_kernel<128>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                                  (size_t)smem, stream, 1, tq, tk, tv, to, p);
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
       else h->launches++;
     }
@@ -1624,18 +1709,18 @@ fact_status_t fact_norm(fact_handle_t h, fact_norm_t kind, int64_t M, int64_t C,
   const int threads = kNormWarps * 32;
   const bool rms = kind == FACT_NORM_RMS;
   // a lane keeps ceil(C / 256) 16-byte chunks of its row in registers
+  cudaError_t e;
   if (C <= 1024) {
-    if (rms) fact_norm_kernel<4, true><<<grid, threads, 0, stream>>>(p);
-    else fact_norm_kernel<4, false><<<grid, threads, 0, stream>>>(p);
+    e = rms ? launch_pdl(h, fact_norm_kernel<4, true>, grid, (unsigned)threads, 0, stream, 1, p)
+            : launch_pdl(h, fact_norm_kernel<4, false>, grid, (unsigned)threads, 0, stream, 1, p);
   } else if (C <= 4096) {
-    if (rms) fact_norm_kernel<16, true><<<grid, threads, 0, stream>>>(p);
-    else fact_norm_kernel<16, false><<<grid, threads, 0, stream>>>(p);
+    e = rms ? launch_pdl(h, fact_norm_kernel<16, true>, grid, (unsigned)threads, 0, stream, 1, p)
+            : launch_pdl(h, fact_norm_kernel<16, false>, grid, (unsigned)threads, 0, stream, 1, p);
   } else {
-    if (rms) fact_norm_kernel<32, true><<<grid, threads, 0, stream>>>(p);
-    else fact_norm_kernel<32, false><<<grid, threads, 0, stream>>>(p);
+    e = rms ? launch_pdl(h, fact_norm_kernel<32, true>, grid, (unsigned)threads, 0, stream, 1, p)
+            : launch_pdl(h, fact_norm_kernel<32, false>, grid, (unsigned)threads, 0, stream, 1, p);
   }
   fact_status_t st = FACT_OK;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) st = cuda_fail(h, "norm launch", e);
   else h->launches++;
   if (dev != h->device) cudaSetDevice(dev);

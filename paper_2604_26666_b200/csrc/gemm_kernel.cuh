@@ -59,6 +59,15 @@ constexpr int kNumBarriers = 2 * kMaxStages + 4 + kEpiWarps * kEpiMaxBufs;
 constexpr uint32_t kCtrlSmemBytes = kNumBarriers * 8 + 16;
 // folded LayerNorm only: the FP32 column sums of each epilogue warp's 128 columns, behind the control words
 constexpr uint32_t kNormCsBytes = kEpiWarps * 128 * 4;
+// Dynamic tile scheduling (the DYN instantiations only), behind the control words of the leader CTA: a ring of
+// kSchedDepth unit numbers that a twelfth warp obtains by cancelling the launch of clusters that have not started
+// (clusterlaunchcontrol) and every other warp of the CTA group consumes.  Per slot: the 16-byte answer, the unit
+// number, and three mbarriers (answer arrived / unit published / unit consumed by everyone).
+constexpr int kSchedDepth = 4;
+constexpr int kSchedConsumers = 11;  // warps per CTA that walk the tile list: 2 producers, MMA, 8 epilogue
+constexpr uint32_t kSchedRespOff = 0, kSchedUnitOff = 16 * kSchedDepth, kSchedBarOff = kSchedUnitOff + 4 * kSchedDepth;
+constexpr uint32_t kSchedSmemBytes = kSchedBarOff + 3 * 8 * kSchedDepth;
+static_assert(kSchedBarOff % 8 == 0, "mbarriers are 8-byte aligned");
 
 // Epilogue selector of the kernel: the public enum plus the split-K partial store.
 enum : int {
@@ -275,16 +284,61 @@ __host__ __device__ inline SkPiece sk_next_piece(int k_blocks, int len, int rem,
 // A tile's pieces belong to consecutive groups; the group with the first k-block adds the others' FP32
 // partials (in group order) to its own accumulator and applies the epilogue.  Those others meet that piece first
 // of all their work and depend on nobody, so the wait for them cannot be circular.
-template <bool SK, bool GROUPED = false>
+// What a warp needs to take unit numbers from the dynamic scheduler's ring (DYN instantiations).
+struct SchedCtx {
+  uint32_t unit_full0;    // this CTA's "unit published" barriers (the scheduler of the leader CTA arrives on both CTAs')
+  uint32_t unit_empty0;   // the leader CTA's "unit consumed" barriers, as a shared::cluster address
+  uint32_t unit_ring0;    // the leader CTA's unit numbers, as a shared::cluster address
+  volatile int* abort_flag;
+  int* status;
+};
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                         unsigned long long limit_ns);
+__device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status);
+
+template <bool SK, bool GROUPED = false, bool DYN = false, int CG = 1>
 struct UnitWalk {
   int u, stride, wave;
   int sk_pos, sk_end, group;
-  __device__ __forceinline__ UnitWalk(const GemmParams& p, int unit0, int unit_stride)
-      : u(unit0), stride(unit_stride), wave(0), sk_pos(0), sk_end(0), group(unit0) {
+  int slot;
+  uint32_t phase;
+  const SchedCtx* sc;
+  __device__ __forceinline__ UnitWalk(const GemmParams& p, int unit0, int unit_stride, const SchedCtx* sched = nullptr)
+      : u(unit0), stride(unit_stride), wave(0), sk_pos(0), sk_end(0), group(unit0), slot(0), phase(0), sc(sched) {
     if constexpr (SK) {
       sk_pos = sk_group_begin(p.sk_len, p.sk_rem, unit0);
       sk_end = sk_group_begin(p.sk_len, p.sk_rem, unit0 + 1);
     }
+  }
+  // DYN: the number of the next unit from the scheduler's ring (warp-uniform; -1: no more, or the wait was given up).
+  // The first unit of a CTA group is its own cluster's; the others come in the order the scheduler obtained them.
+  __device__ __forceinline__ int next_dynamic() {
+    if (wave == 0) return u;
+    const uint32_t fb = sc->unit_full0 + 8u * (uint32_t)slot;
+    bool ok;
+    if constexpr (CG == 2) ok = wait_bar_cluster(fb, phase, sc->abort_flag, sc->status);
+    else ok = wait_bar(fb, phase, sc->abort_flag, sc->status, kWaitLimitNs);
+    int v = -1;
+    if ((threadIdx.x & 31) == 0 && ok) {
+      if constexpr (CG == 2) v = ptx::ld_shared_cluster_s32(sc->unit_ring0 + 4u * (uint32_t)slot);
+      else asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(sc->unit_ring0 + 4u * (uint32_t)slot) : "memory");
+    }
+    // (the shuffle cannot issue before the load has returned, and the arrival below is issued after the shuffle: the
+    // slot is not handed back to the scheduler before its value has been read)
+    v = __shfl_sync(0xffffffffu, v, 0);
+    ok = __all_sync(0xffffffffu, ok) != 0;
+    if (!ok) return -1;
+    if ((threadIdx.x & 31) == 0) {
+      const uint32_t eb = sc->unit_empty0 + 8u * (uint32_t)slot;
+      if constexpr (CG == 2) ptx::mbar_arrive_cluster_relaxed(eb);
+      else ptx::mbar_arrive(eb);
+    }
+    if (++slot == kSchedDepth) {
+      slot = 0;
+      phase ^= 1u;
+    }
+    return v;
   }
   __device__ __forceinline__ bool next(const GemmParams& p, WorkUnit& w) {
     if constexpr (SK) {
@@ -301,7 +355,12 @@ struct UnitWalk {
         return true;
       }
     }
-    if (u >= p.total_units) return false;
+    if constexpr (DYN) {
+      u = next_dynamic();
+      if (u < 0 || u >= p.total_units) return false;
+    } else {
+      if (u >= p.total_units) return false;
+    }
     if constexpr (GROUPED) {
       w = decode_grouped(p, u);
     } else {
@@ -312,7 +371,7 @@ struct UnitWalk {
     w.wave = wave++;
     w.sk_role = 0;
     w.sk_peers = 0;
-    u += stride;
+    if constexpr (!DYN) u += stride;
     return true;
   }
 };
@@ -338,7 +397,7 @@ __device__ __forceinline__ bool wait_flag(const int* flag, int want, volatile in
 
 // Bounded mbarrier wait.  Returns false if the wait was abandoned.
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                         unsigned long long limit_ns = kWaitLimitNs) {
+                                         unsigned long long limit_ns) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -349,6 +408,30 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
       if (t0 == 0) {
         t0 = now;
       } else if (now - t0 > limit_ns) {
+        *abort_flag = 1;
+        atomicExch(status, kDeviceTimeoutCode);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  return wait_bar(bar, parity, abort_flag, status, kWaitLimitNs);
+}
+
+// The same wait with cluster-scope acquire: for a barrier the peer CTA arrives on after writing data this CTA reads.
+__device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (ptx::mbar_try_wait_cluster(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (ptx::mbar_try_wait_cluster(bar, parity)) return true;
+    if ((it & 1023u) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = ptx::globaltimer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitNs) {
         *abort_flag = 1;
         atomicExch(status, kDeviceTimeoutCode);
         return false;
@@ -563,6 +646,8 @@ __device__ __forceinline__ void reduce_groups(const ReduceParams& p, long long f
 }
 
 __global__ void __launch_bounds__(128) fact_splitk_reduce_kernel(const ReduceParams p) {
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
   reduce_groups(p, blockIdx.x * (long long)blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
 }
 
@@ -604,13 +689,12 @@ __device__ __forceinline__ uint64_t epilogue_pair(uint64_t acc, uint64_t up, uin
   }
 }
 
-template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int CG, int EPI, bool SK = false, bool GROUPED = false, int EXT = 0, bool DYN = false>
+__global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
     fact_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmR,
                      const GemmParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  const long long t_entry = clock64();
 
   // The warp index is made provably warp-uniform (a shuffle result), and the producer / MMA roles
   // run their loops with all 32 lanes converged, electing one lane only for the instruction that
@@ -645,6 +729,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
   }
+  if constexpr (DYN) {  // dynamic scheduling hands out whole data-parallel tiles, one cluster of the grid per tile
+    static_assert(!SK && EXT == 0 && EPI != kEpiPartial, "dynamic scheduling: plain data-parallel tiles");
+    if ((int)(gridDim.x / CG) != p.total_units || p.split_k != 1) {
+      if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
+      return;
+    }
+  }
   if constexpr (EPI == kEpiBiasSoftmax) {  // a row's softmax needs the whole row in one tile and the direct stores
     if (p.store_tma || p.tiles_n != 1) {
       if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
@@ -672,6 +763,28 @@ __global__ void __launch_bounds__(kThreads, 1)
     return bar_base + 8u * (uint32_t)(2 * kMaxStages + 4 + e * kEpiMaxBufs + b);
   };
 
+  // dynamic scheduler's ring (DYN only; the host reserved the bytes): answers, unit numbers, barriers
+  const uint32_t sched_base = bar_base + kCtrlSmemBytes;
+  auto clc_bar = [&](int s) { return sched_base + kSchedBarOff + 8u * (uint32_t)s; };
+  auto unit_full_bar = [&](int s) { return sched_base + kSchedBarOff + 8u * (uint32_t)(kSchedDepth + s); };
+  auto unit_empty_bar = [&](int s) { return sched_base + kSchedBarOff + 8u * (uint32_t)(2 * kSchedDepth + s); };
+  SchedCtx sched_ctx;
+  if constexpr (DYN) {
+    sched_ctx.unit_full0 = unit_full_bar(0);
+    sched_ctx.unit_empty0 = (CG == 2) ? ptx::mapa(unit_empty_bar(0), 0) : unit_empty_bar(0);
+    sched_ctx.unit_ring0 = (CG == 2) ? ptx::mapa(sched_base + kSchedUnitOff, 0) : sched_base + kSchedUnitOff;
+    sched_ctx.abort_flag = abort_p;
+    sched_ctx.status = p.status;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + 3 * kSchedDepth) {
+      const int i = (int)threadIdx.x - 64;
+      // answer arrived: the requesting thread; unit published: the scheduler; unit consumed: every walking warp of
+      // the CTA group
+      ptx::mbar_init(sched_base + kSchedBarOff + 8u * (uint32_t)i, i >= 2 * kSchedDepth ? kSchedConsumers * CG : 1);
+      ptx::fence_mbar_init();
+    }
+  }
+  const SchedCtx* const sched = DYN ? &sched_ctx : nullptr;
+
   // One thread per mbarrier: serial initialisation by a single thread costs about a thousand cycles of prologue.
   if (threadIdx.x < kNumBarriers) {
     const int i = (int)threadIdx.x;
@@ -698,6 +811,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder_p;
+  // Everything above touched shared and tensor memory only and may overlap the tail of the kernel before this one
+  // in the stream; from here on global memory is read and written.  The successor may set itself up likewise.
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+  const long long t_go = clock64();
 
   // CTA 0 stamps the SM cycle counter and the nanosecond timer around its work (status[2..5]):
   // their ratio is the SM clock this launch really ran at.
@@ -724,13 +842,15 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         // Odd waves walk K downwards: the wave before ended at the top of K, so the operand slabs both waves
         // share (same m-tiles of A, or same n-tiles of B) are met while they are still in L2.  The sum of an
         // output element is then taken in descending k in those tiles, still fixed by (shape, config).
-        const bool k_down = (w.wave & 1) && p.k_serpentine;
+        // (not with dynamic scheduling: which tiles a CTA gets, and so the parity of their count, is not fixed there,
+        // and the order of a sum must not depend on it)
+        const bool k_down = !DYN && (w.wave & 1) && p.k_serpentine;
         const int m0 = (GROUPED ? w.m_base : 0) + (w.tm * CG + (int)cta_rank) * kTileM;
         const int a_batch = GROUPED ? 0 : w.b;  // grouped: A is one matrix, the group selects the weights only
         // first accumulator column this CTA's B boxes feed, and the W column of every box
@@ -812,7 +932,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t acc_phase = 0;
       bool ok = true;
       long long prof_acc_wait = 0, prof_full_wait = 0, prof_first_full = 0;
-      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         long long t0 = prof ? clock64() : 0;
@@ -832,7 +952,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (prof) {
             const long long now = clock64();
             prof_full_wait += now - t0;
-            if (prof_first_full == 0) prof_first_full = now - t_entry;
+            if (prof_first_full == 0) prof_first_full = now - t_go;
           }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
@@ -852,7 +972,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               }
             }
             // release the stage (in both CTAs of a pair) once these MMAs have read it
-            if constexpr (CG == 2) ptx::umma_commit_pair(empty_bar(stage), 0x3);
+            if constexpr (CG == 2) ptx::umma_commit_pair(empty_bar(stage));
             else ptx::umma_commit<CG>(empty_bar(stage));
           }
           if (++stage == p.stages) {
@@ -862,7 +982,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (!ok) break;
         if (ptx::elect_one()) {
-          if constexpr (CG == 2) ptx::umma_commit_pair(accf_bar(acc), 0x3);
+          if constexpr (CG == 2) ptx::umma_commit_pair(accf_bar(acc));
           else ptx::umma_commit<CG>(accf_bar(acc));
         }
         acc ^= 1;
@@ -872,12 +992,57 @@ __global__ void __launch_bounds__(kThreads, 1)
         long long* c = reinterpret_cast<long long*>(p.status + 2);
         c[2] = prof_acc_wait;
         c[3] = prof_full_wait;
-        c[7] = prof_first_full;  // cycles from kernel entry to the first operand stage being ready
+        c[7] = prof_first_full;  // cycles from "may touch global memory" to the first operand stage being ready
       }
     };
     if (cta_rank == 0) {
       if (p.fp8) issue_all(FactTrue{});
       else issue_all(FactFalse{});
+    } else if constexpr (DYN) {
+      // the peer's MMA warp issues nothing, but it is one of the warps the scheduler counts: it walks the list
+      UnitWalk<SK, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);
+      WorkUnit w;
+      while (walk.next(p, w)) {
+      }
+    }
+    __syncwarp();
+  } else if (DYN && warp == kThreads / 32) {
+    // ------------------------------------------------------------ dynamic tile scheduler (twelfth warp, DYN only)
+    // Obtains the CTA group's further units by cancelling the launch of clusters of this grid that have not started:
+    // the group then owes that cluster's tile.  One request is always in flight ahead of the consumers, so the next
+    // unit is known before the current tile ends.  The first answer that says "nothing left" is published as -1 and
+    // ends every walk; no request follows it.
+    if (cta_rank == 0) {
+      int slot = 0;
+      uint32_t phase = 0;
+      for (bool more = true; more;) {
+        if (!wait_all(unit_empty_bar(slot), phase ^ 1u)) break;  // every walking warp has read the slot's last value
+        const uint32_t resp = sched_base + kSchedRespOff + 16u * (uint32_t)slot;
+        if (ptx::elect_one()) {
+          ptx::mbar_arrive_expect_tx(clc_bar(slot), 16);
+          ptx::clc_try_cancel(resp, clc_bar(slot));
+        }
+        if (!wait_all(clc_bar(slot), phase)) break;
+        int unit = -1;
+        if (lane == 0) {
+          const int x = ptx::clc_query_ctaid_x(resp);
+          unit = x < 0 ? -1 : x / CG;
+          ptx::fence_proxy_async_smem();  // the answer was written through the async proxy and will be again
+          asm volatile("st.shared.s32 [%0], %1;" ::"r"(sched_base + kSchedUnitOff + 4u * (uint32_t)slot), "r"(unit)
+                       : "memory");
+        }
+        unit = __shfl_sync(0xffffffffu, unit, 0);
+        __syncwarp();
+        if (lane == 0) {
+          ptx::mbar_arrive(unit_full_bar(slot));
+          if constexpr (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(unit_full_bar(slot), 1));  // (release, cluster scope)
+        }
+        more = unit >= 0;
+        if (++slot == kSchedDepth) {
+          slot = 0;
+          phase ^= 1u;
+        }
+      }
     }
     __syncwarp();
   } else {
@@ -910,7 +1075,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       long long prof_epi_busy = 0, prof_epi_wait = 0, prof_tiles = 0;
       uint32_t gc = 0;      // chunks this warp has stored so far: buffer = gc % bufs
       uint32_t r_next = 0;  // residual loads have been issued for every chunk counter below this
-      UnitWalk<SK, GROUPED> walk(p, unit0, unit_stride);
+      UnitWalk<SK, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);
       WorkUnit w;
       // hand the accumulator back to the MMA issuer (of the leader CTA) and move on to the other one
       // (a relaxed arrival: the barrier orders tensor-memory reads only, which the tcgen05 fences take care of; a
@@ -1351,7 +1516,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // ---- direct: each thread stores its own row from registers (any alignment, any leading dimension)
       const bool c_vec = p.c_vec != 0;
       uint32_t xch_count = 0;  // exchanges with the other warp of the lane quarter so far (row softmax only)
-      UnitWalk<false, GROUPED> walk(p, unit0, unit_stride);  // (stream-K always stores through the staged path)
+      UnitWalk<false, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);  // (stream-K always stores through the staged path)
       WorkUnit w;
       while (ok && walk.next(p, w)) {
         if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
