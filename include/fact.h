@@ -442,14 +442,17 @@ fact_status_t fact_get_config(fact_handle_t handle, fact_op_t op, int64_t batch,
  *     of scratch are skipped.  (The paper's sweep launches them and records the failures, Section 5.1.)
  *   - Verify gate: the library's default configuration is run once and a dense FP32 copy of its output kept;
  *     before a candidate is timed, its output (written over NaNs) is compared with that copy element by
- *     element on the device, tolerance 2^-7 |ref| + 1e-3 mean|ref| for BF16 outputs and 2e-4 (|ref| +
- *     mean|ref|) for FP32 outputs -- what two correct FP32-accumulated results in different summation orders
- *     can differ by, far below what a dropped k-block or a misplaced tile changes.  A candidate outside it
- *     is recorded as FACT_TUNE_VERIFY_FAILED, is never timed and can never win.
+ *     element on the device, tolerance 2^-7 |ref| + 1e-3 mean|ref| for BF16 outputs and 1e-3 (|ref| +
+ *     mean|ref|) for FP32 outputs -- above what two correct FP32-accumulated results in different summation
+ *     orders differ by (one BF16 ulp; for FP32 outputs half the stated tolerance: a single 131072-term
+ *     accumulator and a sliced sum of the same products differ by 3.4e-4), far below what a dropped k-block or
+ *     a misplaced tile changes.  A candidate outside it is recorded as FACT_TUNE_VERIFY_FAILED, is never
+ *     timed and can never win.
  *   - Timing: `warmup` + `iters` launches per candidate (0 = 5 and 20, the paper's protocol in Section 5.1),
- *     CUDA events, each candidate ranked by its time relative to the default configuration timed right
- *     before and after it (the clock of a power-limited part drifts over a sweep); the four fastest are
- *     timed three more times in alternation.  Warm L2 by default: launches back to back.
+ *     CUDA events, each time multiplied by the SM clock the kernel itself measured (a time in cycles: the
+ *     clock of a power-limited part drifts by more than candidates differ) and ranked relative to the default
+ *     configuration timed right before and after; the five fastest are timed five more times in alternation
+ *     and the best median wins.  Warm L2 by default: launches back to back.
  * fact_tune_ex takes options (NULL = the defaults of fact_tune):
  *   cold_l2       1: a buffer twice the size of L2 is overwritten before every timed launch and every launch
  *                 is timed by an event pair of its own -- the protocol of a benchmark that flushes L2
@@ -557,6 +560,11 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * kernel's softmax arithmetic and its two products), whose output is meaningless, exist only in a library
  * compiled with -DFACT_EXPERIMENTS; the default build ignores those bits. */
 fact_status_t fact_last_kernel_profile(fact_handle_t handle, void* cuda_stream, int64_t counters[8]);
+
+/* Diagnostic (FACT_DEBUG_FLAGS=256 only, else 0): nanoseconds from the moment the first CTA of the most recent
+ * GEMM launch was allowed to touch global memory to the moment its last CTA left -- the kernel's span over all CTAs,
+ * without the launch and completion latencies an event pair around one launch also contains. */
+fact_status_t fact_last_kernel_span(fact_handle_t handle, void* cuda_stream, int64_t* nanoseconds);
 
 /* The FACT_DEBUG_FLAGS bits in effect for this handle (0 in normal use; see fact_last_kernel_profile). */
 int fact_debug_flags(fact_handle_t handle);

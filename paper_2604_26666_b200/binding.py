@@ -40,7 +40,7 @@ EXPORTED = [
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
     "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
-    "fact_tune_ex",
+    "fact_tune_ex", "fact_last_kernel_span",
 ]
 
 
@@ -168,6 +168,7 @@ def lib() -> ctypes.CDLL:
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     L.fact_gemm_splitk_static_status.argtypes = [c_int, vp, POINTER(c_int)]
     L.fact_debug_flags.argtypes = [vp]
+    L.fact_last_kernel_span.argtypes = [vp, vp, POINTER(i64)]
     for name in EXPORTED:
         fn = getattr(L, name)
         if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
@@ -391,6 +392,12 @@ class Handle:
         arr = (c_int64 * 8)()
         _check(lib().fact_last_kernel_profile(self._h, self._stream(stream), arr), "fact_last_kernel_profile")
         return [int(x) for x in arr]
+
+    def last_kernel_span(self, stream=None) -> int:
+        """Nanoseconds from the first CTA's start to the last CTA's end of the last GEMM launch (FACT_DEBUG_FLAGS=256)."""
+        v = c_int64(0)
+        _check(lib().fact_last_kernel_span(self._h, self._stream(stream), byref(v)), "fact_last_kernel_span")
+        return int(v.value)
 
     def selftest_wait_timeout(self, limit_ms: float = 5.0, stream=None):
         """Run the bounded-wait self-test (fact_selftest_wait_timeout); raises unless the wait gave up cleanly."""

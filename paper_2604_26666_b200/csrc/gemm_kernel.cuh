@@ -560,7 +560,7 @@ __device__ __forceinline__ float reduce_epilogue(int epi, float a, float up, flo
   }
 }
 
-constexpr int kReduceBatch = 8;  // loads in flight per thread and round trip (32 slices)
+constexpr int kReduceBatch = 10;  // loads in flight per thread and round trip: 40 slices (the 37 of a 148-SM part in one trip)
 
 // Four adjacent lanes share one group of 4 output columns: lane q of the quad adds slices q, q+4, q+8, ...
 // in ascending order, then the four sums are combined as (s0 + s1) + (s2 + s3).  The order of every
@@ -825,8 +825,11 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
     t_clk0 = clock64();
     t_ns0 = ptx::globaltimer_ns();
   }
-  // With debug bit 256 the first CTA also counts where its cycles go (status[2..]: see fact_last_kernel_profile).
+  // With debug bit 256 the first CTA also counts where its cycles go (status[2..]: see fact_last_kernel_profile), and
+  // every CTA stamps the nanosecond timer on its way in and out (status[40..43]: earliest start, latest end).
   const bool prof = (p.debug & 256) && blockIdx.x == 0;
+  if ((p.debug & 256) && threadIdx.x == 0)
+    atomicMin(reinterpret_cast<unsigned long long*>(p.status + 40), (unsigned long long)ptx::globaltimer_ns());
   const int unit0 = (int)(blockIdx.x / CG);
   const int unit_stride = (int)(gridDim.x / CG);
   // a bounded wait whose verdict is warp-uniform
@@ -1727,6 +1730,8 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
     stamp[0] = clock64() - t_clk0;
     stamp[1] = (long long)(ptx::globaltimer_ns() - t_ns0);
   }
+  if ((p.debug & 256) && threadIdx.x == 0)
+    atomicMax(reinterpret_cast<unsigned long long*>(p.status + 42), (unsigned long long)ptx::globaltimer_ns());
   if constexpr (CG == 2) {  // neither CTA may free tensor memory or exit while its peer still uses it
     ptx::cluster_arrive();
     ptx::cluster_wait();
