@@ -39,8 +39,8 @@ WORKLOAD = "config 2: square BF16 GEMM 4096^3 + 8192^3, N(0,1)/sqrt(K), seed 1"
 L2_FLUSH_BYTES = 512 << 20
 
 # DRAM traffic per launch of the dominant kernel (8192^3): dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture of that launch (933.4 MB + 126.5 MB, mean of two launches).
-DOMINANT_TRAFFIC_BYTES = 1.0599e9
+# capture of that launch (877.0 MB + 128.6 MB, mean of two launches).
+DOMINANT_TRAFFIC_BYTES = 1.0056e9
 
 
 def load_peaks():
@@ -196,6 +196,8 @@ def main():
                     help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped`, `normfold` or `blocks`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
+    ap.add_argument("--no-trains", action="store_true",
+                    help="with --shape: skip the back-to-back launch trains of the short shapes (the profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -239,7 +241,7 @@ def main():
         names = None if args.shape == "all" else args.shape.split(",")
         rows = [] if args.shape in ("attention", "blocks", "fp8", "grouped", "normfold") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
-            side_ref=False, layout=args.layout)
+            side_ref=False, layout=args.layout, trains=not args.no_trains)
         if args.shape in ("all", "attention"):
             att = attention_table(h, dev, stream, flush_l2, peaks, warm=args.warmup)
         elif args.shape in ("blocks", "fp8", "grouped", "normfold"):
@@ -318,8 +320,9 @@ def main():
     achieved = dom_case.flops / (dom_avg_ms * 1e-3) / 1e12
 
     # ---------------------------------------------------------------- end to end: host buffers in, host result out
-    # Through the package's host-buffer front end (HostGemmPipeline): every step copies its inputs from pinned
-    # host memory and its results back to pinned host memory; copies of neighbouring problems overlap the kernels.
+    # Through the library's host-buffer entry point (fact_gemm_host over the C ABI): every step hands it pinned host
+    # operands and a pinned host result; the call copies in, multiplies and copies out on the handle's three streams,
+    # and the copies of neighbouring problems overlap the kernels (two device scratch buffers per shape, in turn).
     from paper_2604_26666_b200.pipeline import HostGemmPipeline
 
     host_outs = [torch.empty((c.M, c.N), dtype=torch.bfloat16).pin_memory() for c in cases]
@@ -328,19 +331,19 @@ def main():
 
     def e2e_step():
         for c, hi, ho in zip(cases, host_inputs, host_outs):
-            pipe.submit(hi.X, hi.W, ho)
+            pipe.submit(hi.X, hi.W, ho, stream=stream)
 
     e2e_step()
-    pipe.finish()
+    pipe.finish(stream)
     barrier()
     t_wall0 = time.perf_counter()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(pipe.s_in)
+    e0.record(stream)
     pipe.h2d_bytes = pipe.d2h_bytes = 0
     for _ in range(e2e_steps):
         e2e_step()
-    e1.record(pipe.s_out)
-    pipe.finish()
+    e1.record(stream)  # (the stream waits for every call's copy-out)
+    pipe.finish(stream)
     barrier()
     e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1), dist, dev)
     e2e_wall_ms = (time.perf_counter() - t_wall0) * 1e3
@@ -393,7 +396,8 @@ def main():
                          "traffic": DOMINANT_TRAFFIC_BYTES, "algorithmic_bytes": dom_case.algorithmic_bytes},
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": e2e_wall_ms / e2e_steps,
-                    "api": "HostGemmPipeline (pinned host in, pinned host out, copies overlapped with kernels)"},
+                    "api": "fact_gemm_host over the C ABI (pinned host in, pinned host out; copy-in, product and "
+                           "copy-out on the handle's three streams, two device scratch buffers per shape)"},
             "gpu_launches": launches, "debug_flags": h.debug_flags(),
             "clocks": dict(clocks, sm_mhz_in_dominant_kernel=(1e3 * k_cycles / k_ns if k_ns else None)),
             "cpu_baseline": cpu,
@@ -470,7 +474,8 @@ def back_to_back_us(call_set, case, X, W, bias, res, out, h, dev, stream, reps=5
     return sorted(ts)[len(ts) // 2] * 1e3
 
 
-def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, iters=20, side_ref=True, layout="NK"):
+def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, iters=20, side_ref=True, layout="NK",
+                    trains=True):
     """Time every benchmark shape alone (5 warm-up + 20 timed launches, L2 overwritten between launches)."""
     import torch
 
@@ -523,6 +528,18 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
             torch.cuda.synchronize(dev)
             return sorted(x.elapsed_time(y) for x, y in ts)
 
+        def kernel_span_us(n=7):
+            """The kernel's own clock: microseconds and SM MHz of the first CTA's span in a cold launch, median of n
+            (fact_last_kernel_clock; no launch or completion latency in it)."""
+            spans = []
+            for _ in range(n):
+                flush_l2()
+                call()
+                cyc, ns = h.last_kernel_clock()
+                spans.append((ns * 1e-3, 1e3 * cyc / ns if ns else 0.0))
+            spans.sort()
+            return spans[len(spans) // 2]
+
         t = time_it(call)
         t_hot = time_it(call, cold=False) if side_ref else t
         t_side = time_it(side, iters=10) if side_ref else [0.0]
@@ -531,7 +548,10 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
         bound = "tensor" if t_tensor >= t_hbm else "hbm"
         cfg = h.get_config(case.op, case.batch, case.M, case.N, case.K, case.epilogue, case.layout, odt).as_dict()
+        span_us, span_mhz = kernel_span_us()
         row = {
+            "us_kernel_span_first_cta": span_us, "sm_mhz_in_kernel": span_mhz,
+            "roofline_frac_of_kernel_span": max(t_tensor, t_hbm) * 1e3 / span_us if span_us else None,
             "name": case.name, "config": case.config, "op": case.op, "epilogue": case.epilogue,
             "layout": case.layout, "batch": case.batch, "M": case.M, "N": case.N, "K": case.K, "out": case.out,
             "us_median": med * 1e3, "us_min": t[0] * 1e3, "us_hot_l2_median": t_hot[len(t_hot) // 2] * 1e3,
@@ -543,7 +563,7 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         # to back between one event pair, rotating through R sets of operands and outputs whose total exceeds twice
         # the L2 -- every launch still finds its data in DRAM, and the cost per launch is the stream time it adds.
         t_use = med
-        if med * 1e3 < SHORT_SHAPE_US:
+        if med * 1e3 < SHORT_SHAPE_US and trains:
             t_b2b = back_to_back_us(call_set=None, case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev,
                                     stream=stream) * 1e-3
             row["us_back_to_back_cold"] = t_b2b * 1e3

@@ -40,7 +40,7 @@ EXPORTED = [
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
     "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
-    "fact_tune_ex", "fact_last_kernel_span",
+    "fact_tune_ex", "fact_last_kernel_span", "fact_gemm_host", "fact_gemm_host_scratch_bytes",
 ]
 
 
@@ -169,9 +169,13 @@ def lib() -> ctypes.CDLL:
     L.fact_gemm_splitk_static_status.argtypes = [c_int, vp, POINTER(c_int)]
     L.fact_debug_flags.argtypes = [vp]
     L.fact_last_kernel_span.argtypes = [vp, vp, POINTER(i64)]
+    L.fact_gemm_host_scratch_bytes.argtypes = [i64, i64, i64, c_int]
+    L.fact_gemm_host_scratch_bytes.restype = sz
+    L.fact_gemm_host.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, cfgp, vp, sz, vp]
     for name in EXPORTED:
         fn = getattr(L, name)
-        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
+        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes",
+                        "fact_gemm_host_scratch_bytes"):
             fn.restype = c_int
     _lib = L
     return L
@@ -435,6 +439,38 @@ class Handle:
         _check(lib().fact_gemm(self._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
                                _ld(out), OUT_TYPES[out.dtype], c, _ptr(ws), nws, self._stream(stream)), "fact_gemm", self._h)
         return out
+
+    def gemm_host(self, A, B, out, scratch, layout="KN", cfg=None, stream=None):
+        """C = A @ B for HOST tensors (fact_gemm_host): A, B BF16 CPU tensors (pinned for asynchronous copies), `out`
+        a BF16 or FP32 CPU tensor, `scratch` a device uint8 tensor of at least gemm_host_scratch_bytes(...) bytes.
+        Enqueues copy-in, product and copy-out on the handle's own three streams; `out` is valid once `stream`
+        (default: torch's current stream) has been synchronised.  Give consecutive calls different scratch tensors
+        and their copies overlap each other's products."""
+        nd = 2
+        _need(A, "A", torch.bfloat16, nd, cuda=False)
+        _need(B, "B", torch.bfloat16, nd, cuda=False)
+        if A.is_cuda or B.is_cuda or out.is_cuda:
+            raise TypeError("gemm_host takes host tensors; use gemm for device tensors")
+        M, K = A.shape
+        N, Kb = (B.shape[1], B.shape[0]) if layout == "KN" else (B.shape[0], B.shape[1])
+        if Kb != K:
+            raise ValueError(f"inner dimensions differ: A has K = {K}, B has K = {Kb}")
+        if out.dtype not in (torch.bfloat16, torch.float32) or tuple(out.shape) != (M, N):
+            raise ValueError(f"out must be a bfloat16 or float32 host tensor of shape {(M, N)}")
+        if out.shape[-1] > 1 and out.stride(-1) != 1:
+            raise ValueError("out: innermost dimension must be contiguous")
+        need = self.gemm_host_scratch_bytes(M, N, K, out.dtype)
+        if not (isinstance(scratch, torch.Tensor) and scratch.is_cuda and scratch.dtype == torch.uint8
+                and scratch.is_contiguous() and scratch.numel() >= need and scratch.device.index == self.device):
+            raise ValueError(f"scratch must be a contiguous uint8 tensor of at least {need} bytes on cuda:{self.device}")
+        _check(lib().fact_gemm_host(self._h, M, N, K, _ptr(A), _ld(A), _ptr(B), _ld(B), LAYOUTS[layout], _ptr(out),
+                                    _ld(out), OUT_TYPES[out.dtype], self._cfg(cfg), _ptr(scratch), scratch.numel(),
+                                    self._stream(stream)), "fact_gemm_host", self._h)
+        return out
+
+    @staticmethod
+    def gemm_host_scratch_bytes(M, N, K, out_dtype=torch.bfloat16) -> int:
+        return int(lib().fact_gemm_host_scratch_bytes(M, N, K, OUT_TYPES[out_dtype]))
 
     def gemm_batched(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
         """C[b] = A[b] @ B[b]  (fact_gemm_batched)."""

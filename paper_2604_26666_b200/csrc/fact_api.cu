@@ -106,6 +106,12 @@ struct fact_handle_s {
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: diagnostics (256 cycle counters, 2048 no K serpentine); the
                                  // work-skipping experiment switches only in a -DFACT_EXPERIMENTS build
   int* d_groups = nullptr;       // grouped GEMM: m-tile prefix and row offsets of the call in flight
+  // fact_gemm_host: copy-in, compute and copy-out streams and a ring of events, created by its first call
+  cudaStream_t host_streams[3] = {nullptr, nullptr, nullptr};
+  static constexpr int kHostEvents = 16;
+  cudaEvent_t host_events[kHostEvents] = {};
+  int host_event_next = 0;
+  std::map<const void*, cudaEvent_t> scratch_busy;  // device scratch -> "the call that last used it has copied out"
   int* sk_flags() const { return d_status + kStatusInts; }  // stream-K flags: [SM][epilogue warp], 0 between launches
   size_t status_ints() const { return (size_t)kStatusInts + (size_t)sm_count * kEpiWarps; }
 };
@@ -999,6 +1005,14 @@ fact_status_t fact_create(fact_handle_t* handle, int device) {
 
 fact_status_t fact_destroy(fact_handle_t h) {
   if (!h) return FACT_OK;
+  for (cudaStream_t st : h->host_streams)
+    if (st) {
+      cudaStreamSynchronize(st);
+      cudaStreamDestroy(st);
+    }
+  for (cudaEvent_t e : h->host_events)
+    if (e) cudaEventDestroy(e);
+  for (auto& kv : h->scratch_busy) cudaEventDestroy(kv.second);
   if (h->d_groups) cudaFree(h->d_groups);
   if (h->d_status) cudaFree(h->d_status);
   delete h;
@@ -1132,6 +1146,103 @@ fact_status_t fact_gemm(fact_handle_t h, int64_t M, int64_t N, int64_t K, const 
   Problem q = make_problem(FACT_OP_GEMM, 1, M, N, K, A, lda, 0, B, ldb, 0, layout, nullptr, nullptr, 0, 0, C, ldc, 0,
                            out, FACT_EPI_NONE);
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
+}
+
+size_t fact_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K, fact_out_t out) {
+  if (M < 0 || N < 0 || K < 0) return 0;
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  auto up8 = [](int64_t v) { return (size_t)((v + 7) / 8 * 8); };  // device rows are padded to whole 16-byte pieces
+  return up((size_t)M * up8(K) * 2) + up(std::max(up8(K) * (size_t)N, up8(N) * (size_t)K) * 2) +
+         up((size_t)M * N * (out == FACT_OUT_F32 ? 4 : 2));
+}
+
+fact_status_t fact_gemm_host(fact_handle_t h, int64_t M, int64_t N, int64_t K, const void* A_host, int64_t lda,
+                             const void* B_host, int64_t ldb, fact_blayout_t layout, void* C_host, int64_t ldc,
+                             fact_out_t out, const fact_config_t* cfg, void* scratch, size_t scratch_bytes,
+                             void* stream_v) {
+  if (!h || M < 0 || N < 0 || K < 0) return FACT_ERR_INVALID_ARG;
+  if (layout != FACT_B_KN && layout != FACT_B_NK) return FACT_ERR_INVALID_ARG;
+  if (out != FACT_OUT_BF16 && out != FACT_OUT_F32) return FACT_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return FACT_OK;
+  const int64_t b_rows = layout == FACT_B_KN ? K : N, b_cols = layout == FACT_B_KN ? N : K;
+  if (!C_host || ldc < N || (K > 0 && (!A_host || !B_host || lda < K || ldb < b_cols))) return FACT_ERR_INVALID_ARG;
+  if (!scratch || scratch_bytes < fact_gemm_host_scratch_bytes(M, N, K, out)) return FACT_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(scratch) & 255u) return FACT_ERR_BAD_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  auto fail = [&](const char* where, cudaError_t e) {
+    const fact_status_t r = cuda_fail(h, where, e);
+    if (dev != h->device) cudaSetDevice(dev);
+    return r;
+  };
+  if (!h->host_streams[0]) {  // first call: the three streams and the event ring (no device memory)
+    for (int i = 0; i < 3; ++i) {
+      cudaError_t e = cudaStreamCreateWithFlags(&h->host_streams[i], cudaStreamNonBlocking);
+      if (e != cudaSuccess) return fail("cudaStreamCreate (fact_gemm_host)", e);
+    }
+    for (int i = 0; i < fact_handle_s::kHostEvents; ++i) {
+      cudaError_t e = cudaEventCreateWithFlags(&h->host_events[i], cudaEventDisableTiming);
+      if (e != cudaSuccess) return fail("cudaEventCreate (fact_gemm_host)", e);
+    }
+  }
+  auto next_event = [&]() {
+    cudaEvent_t e = h->host_events[h->host_event_next];
+    h->host_event_next = (h->host_event_next + 1) % fact_handle_s::kHostEvents;
+    return e;
+  };
+  cudaStream_t caller = reinterpret_cast<cudaStream_t>(stream_v);
+  cudaStream_t s_in = h->host_streams[0], s_mm = h->host_streams[1], s_out = h->host_streams[2];
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  auto up8 = [](int64_t v) { return (size_t)((v + 7) / 8 * 8); };
+  const size_t esz_c = out == FACT_OUT_F32 ? 4 : 2;
+  const size_t lda_dev = up8(K), ldb_dev = up8(b_cols);  // operand rows padded to whole 16-byte pieces (TMA)
+  uint8_t* dA = reinterpret_cast<uint8_t*>(scratch);
+  uint8_t* dB = dA + up((size_t)M * lda_dev * 2);
+  uint8_t* dC = dB + up(std::max(up8(K) * (size_t)N, up8(N) * (size_t)K) * 2);
+  cudaError_t e;
+  // what the caller's stream has enqueued so far comes first; so does the copy-out of the call that last used this
+  // scratch (a wait captures the event's most recent record, so the ring may wrap)
+  cudaEvent_t ev_entry = next_event();
+  if ((e = cudaEventRecord(ev_entry, caller)) != cudaSuccess) return fail("cudaEventRecord", e);
+  if ((e = cudaStreamWaitEvent(s_in, ev_entry, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
+  auto busy = h->scratch_busy.find(scratch);
+  if (busy == h->scratch_busy.end()) {  // first use of this scratch: an event of its own
+    cudaEvent_t ne;
+    if ((e = cudaEventCreateWithFlags(&ne, cudaEventDisableTiming)) != cudaSuccess) return fail("cudaEventCreate", e);
+    busy = h->scratch_busy.emplace(scratch, ne).first;
+  } else if ((e = cudaStreamWaitEvent(s_in, busy->second, 0)) != cudaSuccess) {
+    return fail("cudaStreamWaitEvent", e);
+  }
+  if (K > 0) {
+    if ((e = cudaMemcpy2DAsync(dA, lda_dev * 2, A_host, (size_t)lda * 2, (size_t)K * 2, (size_t)M,
+                               cudaMemcpyHostToDevice, s_in)) != cudaSuccess)
+      return fail("cudaMemcpy2DAsync(A)", e);
+    if ((e = cudaMemcpy2DAsync(dB, ldb_dev * 2, B_host, (size_t)ldb * 2, (size_t)b_cols * 2, (size_t)b_rows,
+                               cudaMemcpyHostToDevice, s_in)) != cudaSuccess)
+      return fail("cudaMemcpy2DAsync(B)", e);
+  }
+  cudaEvent_t ev_loaded = next_event();
+  if ((e = cudaEventRecord(ev_loaded, s_in)) != cudaSuccess) return fail("cudaEventRecord", e);
+  if ((e = cudaStreamWaitEvent(s_mm, ev_loaded, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
+  Problem q = make_problem(FACT_OP_GEMM, 1, M, N, K, dA, (long long)lda_dev, 0, dB, (long long)ldb_dev, 0, layout, nullptr,
+                           nullptr, 0, 0, dC, N, 0, out, FACT_EPI_NONE);
+  const fact_status_t st = run(h, q, cfg, 0, nullptr, 0, s_mm);  // (a table entry that wants scratch of its own runs without)
+  if (st != FACT_OK) {
+    if (dev != h->device) cudaSetDevice(dev);
+    return st;
+  }
+  cudaEvent_t ev_done = next_event();
+  if ((e = cudaEventRecord(ev_done, s_mm)) != cudaSuccess) return fail("cudaEventRecord", e);
+  if ((e = cudaStreamWaitEvent(s_out, ev_done, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
+  if ((e = cudaMemcpy2DAsync(C_host, (size_t)ldc * esz_c, dC, (size_t)N * esz_c, (size_t)N * esz_c, (size_t)M,
+                             cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
+    return fail("cudaMemcpy2DAsync(C)", e);
+  cudaEvent_t ev_out = busy->second;
+  if ((e = cudaEventRecord(ev_out, s_out)) != cudaSuccess) return fail("cudaEventRecord", e);
+  if ((e = cudaStreamWaitEvent(caller, ev_out, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
+  if (dev != h->device) cudaSetDevice(dev);
+  return FACT_OK;
 }
 
 fact_status_t fact_gemm_batched(fact_handle_t h, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,
