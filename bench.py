@@ -342,7 +342,8 @@ def main():
     pipe.h2d_bytes = pipe.d2h_bytes = 0
     for _ in range(e2e_steps):
         e2e_step()
-    e1.record(stream)  # (the stream waits for every call's copy-out)
+    h.gemm_host_wait(stream)  # the stream waits for every call's copy-out
+    e1.record(stream)
     pipe.finish(stream)
     barrier()
     e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1), dist, dev)

@@ -178,22 +178,29 @@ fact_status_t fact_gemm(fact_handle_t handle, int64_t M, int64_t N, int64_t K, c
 /* C = A . B for operands and a result that live in HOST memory -- the call a caller without device-resident data
  * makes (the drop-in replacement of the paper's problem statement, Section 3, for tensors that have not been
  * moved yet).  A, B, C are host pointers (row-major, leading dimensions in elements, same layouts and output
- * types as fact_gemm); `device_scratch` is device memory of at least fact_gemm_host_scratch_bytes(M, N, K,
- * out_type) bytes, 256-byte aligned, owned by the caller.  The call enqueues and returns: a copy of A and B to the
+ * types as fact_gemm); `device_scratch` is device memory of at least fact_gemm_host_scratch_bytes(...) bytes
+ * (the dense device copies of A, B and C, plus the workspace the product's configuration wants), 256-byte
+ * aligned, owned by the caller.  The call enqueues and returns: a copy of A and B to the
  * scratch on the handle's copy-in stream, the product on its compute stream, the copy of C back on its copy-out
- * stream, chained by events.  It is ordered after everything enqueued on `cuda_stream` before the call, and
- * `cuda_stream` is made to wait for the copy-out, so C_host is valid once `cuda_stream` reaches that point
- * (synchronise it before reading C on the host).  Consecutive calls overlap -- the copy-in of one runs during the
- * product of the one before and the copy-out of the one before that -- provided they are given different
- * scratch buffers; a call waits for the copy-out of the last call that used the same scratch.  The copies are
+ * stream, chained by events.  It is ordered after everything enqueued on `cuda_stream` before the call.
+ * fact_gemm_host_wait(handle, stream) makes `stream` wait for the copy-out of every host-buffer call made so far:
+ * C_host is valid once that stream reaches that point (synchronise it before reading C on the host; the wait is
+ * a call of its own so that a train of products does not serialise on the caller's stream).  Consecutive calls
+ * overlap -- the copy-in of one runs during the product of the one before and the copy-out of the one before that
+ * -- provided they are given different scratch buffers; a call waits for the copy-out of the last call that used
+ * the same scratch.  The copies are
  * asynchronous only for page-locked host memory.  The first call through a handle creates the three streams
- * and the events (no device memory).  Product configuration as in fact_gemm with cfg (NULL = the library's choice;
- * a tuned entry that wants K slices or stream-K runs without them: there is no workspace). */
-size_t fact_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K, fact_out_t out_type);
+ * and the events (no device memory).  Product configuration as in fact_gemm with cfg (NULL = the library's choice);
+ * a scratch that holds the operands but not the configuration's workspace makes a tuned entry run without K slices
+ * or stream-K, and a caller's own such configuration fail with FACT_ERR_WORKSPACE_TOO_SMALL. */
+fact_status_t fact_gemm_host_scratch_bytes(fact_handle_t handle, int64_t M, int64_t N, int64_t K,
+                                           fact_blayout_t b_layout, fact_out_t out_type, const fact_config_t* cfg,
+                                           size_t* bytes);
 fact_status_t fact_gemm_host(fact_handle_t handle, int64_t M, int64_t N, int64_t K, const void* A_host, int64_t lda,
                              const void* B_host, int64_t ldb, fact_blayout_t b_layout, void* C_host, int64_t ldc,
                              fact_out_t out_type, const fact_config_t* cfg, void* device_scratch,
                              size_t device_scratch_bytes, void* cuda_stream);
+fact_status_t fact_gemm_host_wait(fact_handle_t handle, void* cuda_stream);
 
 /* C[b] = A[b] . B[b] for b in [0, batch)      (Section 5.1, Problem 3: batched)
  * Batch b of an operand starts stride* elements after batch b-1. */

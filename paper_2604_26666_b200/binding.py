@@ -41,6 +41,7 @@ EXPORTED = [
     "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
     "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
     "fact_tune_ex", "fact_last_kernel_span", "fact_gemm_host", "fact_gemm_host_scratch_bytes",
+    "fact_gemm_host_wait",
 ]
 
 
@@ -169,13 +170,12 @@ def lib() -> ctypes.CDLL:
     L.fact_gemm_splitk_static_status.argtypes = [c_int, vp, POINTER(c_int)]
     L.fact_debug_flags.argtypes = [vp]
     L.fact_last_kernel_span.argtypes = [vp, vp, POINTER(i64)]
-    L.fact_gemm_host_scratch_bytes.argtypes = [i64, i64, i64, c_int]
-    L.fact_gemm_host_scratch_bytes.restype = sz
+    L.fact_gemm_host_scratch_bytes.argtypes = [vp, i64, i64, i64, c_int, c_int, cfgp, POINTER(sz)]
+    L.fact_gemm_host_wait.argtypes = [vp, vp]
     L.fact_gemm_host.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, c_int, vp, i64, c_int, cfgp, vp, sz, vp]
     for name in EXPORTED:
         fn = getattr(L, name)
-        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes",
-                        "fact_gemm_host_scratch_bytes"):
+        if name not in ("fact_status_string", "fact_launch_count", "fact_last_error", "fact_block_workspace_bytes"):
             fn.restype = c_int
     _lib = L
     return L
@@ -443,9 +443,9 @@ class Handle:
     def gemm_host(self, A, B, out, scratch, layout="KN", cfg=None, stream=None):
         """C = A @ B for HOST tensors (fact_gemm_host): A, B BF16 CPU tensors (pinned for asynchronous copies), `out`
         a BF16 or FP32 CPU tensor, `scratch` a device uint8 tensor of at least gemm_host_scratch_bytes(...) bytes.
-        Enqueues copy-in, product and copy-out on the handle's own three streams; `out` is valid once `stream`
-        (default: torch's current stream) has been synchronised.  Give consecutive calls different scratch tensors
-        and their copies overlap each other's products."""
+        Enqueues copy-in, product and copy-out on the handle's own three streams; `out` is valid after
+        gemm_host_wait() and a synchronisation of that stream.  Give consecutive calls different scratch tensors and
+        their copies overlap each other's products."""
         nd = 2
         _need(A, "A", torch.bfloat16, nd, cuda=False)
         _need(B, "B", torch.bfloat16, nd, cuda=False)
@@ -459,7 +459,7 @@ class Handle:
             raise ValueError(f"out must be a bfloat16 or float32 host tensor of shape {(M, N)}")
         if out.shape[-1] > 1 and out.stride(-1) != 1:
             raise ValueError("out: innermost dimension must be contiguous")
-        need = self.gemm_host_scratch_bytes(M, N, K, out.dtype)
+        need = self.gemm_host_scratch_bytes(M, N, K, out.dtype, layout, cfg)
         if not (isinstance(scratch, torch.Tensor) and scratch.is_cuda and scratch.dtype == torch.uint8
                 and scratch.is_contiguous() and scratch.numel() >= need and scratch.device.index == self.device):
             raise ValueError(f"scratch must be a contiguous uint8 tensor of at least {need} bytes on cuda:{self.device}")
@@ -468,9 +468,16 @@ class Handle:
                                     self._stream(stream)), "fact_gemm_host", self._h)
         return out
 
-    @staticmethod
-    def gemm_host_scratch_bytes(M, N, K, out_dtype=torch.bfloat16) -> int:
-        return int(lib().fact_gemm_host_scratch_bytes(M, N, K, OUT_TYPES[out_dtype]))
+    def gemm_host_wait(self, stream=None):
+        """Make `stream` (default: torch's current stream) wait for the copy-out of every gemm_host call so far."""
+        _check(lib().fact_gemm_host_wait(self._h, self._stream(stream)), "fact_gemm_host_wait", self._h)
+
+    def gemm_host_scratch_bytes(self, M, N, K, out_dtype=torch.bfloat16, layout="KN", cfg=None) -> int:
+        """Device scratch a gemm_host call of this shape needs: the operands' device copies and the product's workspace."""
+        n = c_size_t(0)
+        _check(lib().fact_gemm_host_scratch_bytes(self._h, M, N, K, LAYOUTS[layout], OUT_TYPES[out_dtype],
+                                                  self._cfg(cfg), byref(n)), "fact_gemm_host_scratch_bytes")
+        return int(n.value)
 
     def gemm_batched(self, A, B, layout="KN", out=None, out_dtype=torch.bfloat16, cfg=None, stream=None):
         """C[b] = A[b] @ B[b]  (fact_gemm_batched)."""

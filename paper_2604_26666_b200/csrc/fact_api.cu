@@ -1148,12 +1148,26 @@ fact_status_t fact_gemm(fact_handle_t h, int64_t M, int64_t N, int64_t K, const 
   return run(h, q, cfg, 0, ws, ws_bytes, stream);
 }
 
-size_t fact_gemm_host_scratch_bytes(int64_t M, int64_t N, int64_t K, fact_out_t out) {
-  if (M < 0 || N < 0 || K < 0) return 0;
+namespace {
+// Device copies of A, B and C of a host-buffer product (operand rows padded to whole 16-byte pieces), each on a
+// 256-byte boundary; the product's own workspace, if its configuration wants one, follows.
+size_t host_gemm_operand_bytes(int64_t M, int64_t N, int64_t K, fact_out_t out) {
   auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
-  auto up8 = [](int64_t v) { return (size_t)((v + 7) / 8 * 8); };  // device rows are padded to whole 16-byte pieces
+  auto up8 = [](int64_t v) { return (size_t)((v + 7) / 8 * 8); };
   return up((size_t)M * up8(K) * 2) + up(std::max(up8(K) * (size_t)N, up8(N) * (size_t)K) * 2) +
          up((size_t)M * N * (out == FACT_OUT_F32 ? 4 : 2));
+}
+}  // namespace
+
+fact_status_t fact_gemm_host_scratch_bytes(fact_handle_t h, int64_t M, int64_t N, int64_t K, fact_blayout_t layout,
+                                           fact_out_t out, const fact_config_t* cfg, size_t* bytes) {
+  if (!h || !bytes || M < 0 || N < 0 || K < 0) return FACT_ERR_INVALID_ARG;
+  Problem q = shape_only(FACT_OP_GEMM, 1, M, N, K, FACT_EPI_NONE, layout, out);
+  fact_config_t c;
+  const fact_status_t st = resolve_config(h, q, cfg, 0, &c);
+  if (st != FACT_OK) return st;
+  *bytes = host_gemm_operand_bytes(M, N, K, out) + workspace_for(h, q, c);
+  return FACT_OK;
 }
 
 fact_status_t fact_gemm_host(fact_handle_t h, int64_t M, int64_t N, int64_t K, const void* A_host, int64_t lda,
@@ -1166,7 +1180,8 @@ fact_status_t fact_gemm_host(fact_handle_t h, int64_t M, int64_t N, int64_t K, c
   if (M == 0 || N == 0) return FACT_OK;
   const int64_t b_rows = layout == FACT_B_KN ? K : N, b_cols = layout == FACT_B_KN ? N : K;
   if (!C_host || ldc < N || (K > 0 && (!A_host || !B_host || lda < K || ldb < b_cols))) return FACT_ERR_INVALID_ARG;
-  if (!scratch || scratch_bytes < fact_gemm_host_scratch_bytes(M, N, K, out)) return FACT_ERR_WORKSPACE_TOO_SMALL;
+  const size_t operand_bytes = host_gemm_operand_bytes(M, N, K, out);
+  if (!scratch || scratch_bytes < operand_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
   if (reinterpret_cast<uintptr_t>(scratch) & 255u) return FACT_ERR_BAD_ALIGNMENT;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
@@ -1214,20 +1229,29 @@ fact_status_t fact_gemm_host(fact_handle_t h, int64_t M, int64_t N, int64_t K, c
   } else if ((e = cudaStreamWaitEvent(s_in, busy->second, 0)) != cudaSuccess) {
     return fail("cudaStreamWaitEvent", e);
   }
+  // one flat copy where source and destination rows are back to back, a pitched copy otherwise
+  auto copy_rows = [](void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, size_t rows,
+                      cudaMemcpyKind kind, cudaStream_t st) {
+    if (dpitch == width && spitch == width) return cudaMemcpyAsync(dst, src, width * rows, kind, st);
+    return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, rows, kind, st);
+  };
   if (K > 0) {
-    if ((e = cudaMemcpy2DAsync(dA, lda_dev * 2, A_host, (size_t)lda * 2, (size_t)K * 2, (size_t)M,
-                               cudaMemcpyHostToDevice, s_in)) != cudaSuccess)
-      return fail("cudaMemcpy2DAsync(A)", e);
-    if ((e = cudaMemcpy2DAsync(dB, ldb_dev * 2, B_host, (size_t)ldb * 2, (size_t)b_cols * 2, (size_t)b_rows,
-                               cudaMemcpyHostToDevice, s_in)) != cudaSuccess)
-      return fail("cudaMemcpy2DAsync(B)", e);
+    if ((e = copy_rows(dA, lda_dev * 2, A_host, (size_t)lda * 2, (size_t)K * 2, (size_t)M, cudaMemcpyHostToDevice,
+                       s_in)) != cudaSuccess)
+      return fail("copy of A to the device", e);
+    if ((e = copy_rows(dB, ldb_dev * 2, B_host, (size_t)ldb * 2, (size_t)b_cols * 2, (size_t)b_rows,
+                       cudaMemcpyHostToDevice, s_in)) != cudaSuccess)
+      return fail("copy of B to the device", e);
   }
   cudaEvent_t ev_loaded = next_event();
   if ((e = cudaEventRecord(ev_loaded, s_in)) != cudaSuccess) return fail("cudaEventRecord", e);
   if ((e = cudaStreamWaitEvent(s_mm, ev_loaded, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
   Problem q = make_problem(FACT_OP_GEMM, 1, M, N, K, dA, (long long)lda_dev, 0, dB, (long long)ldb_dev, 0, layout, nullptr,
                            nullptr, 0, 0, dC, N, 0, out, FACT_EPI_NONE);
-  const fact_status_t st = run(h, q, cfg, 0, nullptr, 0, s_mm);  // (a table entry that wants scratch of its own runs without)
+  // what is left of the scratch behind the operands is the product's workspace (K slices, stream-K); a tuned entry
+  // that wants more than there is runs without
+  const fact_status_t st = run(h, q, cfg, 0, scratch_bytes > operand_bytes ? dA + operand_bytes : nullptr,
+                               scratch_bytes - operand_bytes, s_mm);
   if (st != FACT_OK) {
     if (dev != h->device) cudaSetDevice(dev);
     return st;
@@ -1235,14 +1259,29 @@ fact_status_t fact_gemm_host(fact_handle_t h, int64_t M, int64_t N, int64_t K, c
   cudaEvent_t ev_done = next_event();
   if ((e = cudaEventRecord(ev_done, s_mm)) != cudaSuccess) return fail("cudaEventRecord", e);
   if ((e = cudaStreamWaitEvent(s_out, ev_done, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
-  if ((e = cudaMemcpy2DAsync(C_host, (size_t)ldc * esz_c, dC, (size_t)N * esz_c, (size_t)N * esz_c, (size_t)M,
-                             cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
-    return fail("cudaMemcpy2DAsync(C)", e);
+  if ((e = copy_rows(C_host, (size_t)ldc * esz_c, dC, (size_t)N * esz_c, (size_t)N * esz_c, (size_t)M,
+                     cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
+    return fail("copy of C to the host", e);
   cudaEvent_t ev_out = busy->second;
   if ((e = cudaEventRecord(ev_out, s_out)) != cudaSuccess) return fail("cudaEventRecord", e);
-  if ((e = cudaStreamWaitEvent(caller, ev_out, 0)) != cudaSuccess) return fail("cudaStreamWaitEvent", e);
   if (dev != h->device) cudaSetDevice(dev);
   return FACT_OK;
+}
+
+fact_status_t fact_gemm_host_wait(fact_handle_t h, void* stream_v) {
+  if (!h) return FACT_ERR_INVALID_ARG;
+  if (!h->host_streams[2]) return FACT_OK;  // no host-buffer call has run
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
+  if (dev != h->device && cudaSetDevice(h->device) != cudaSuccess) return FACT_ERR_CUDA;
+  cudaEvent_t ev = h->host_events[h->host_event_next];
+  h->host_event_next = (h->host_event_next + 1) % fact_handle_s::kHostEvents;
+  fact_status_t st = FACT_OK;
+  cudaError_t e = cudaEventRecord(ev, h->host_streams[2]);  // copy-outs complete in the order they were enqueued
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(reinterpret_cast<cudaStream_t>(stream_v), ev, 0);
+  if (e != cudaSuccess) st = cuda_fail(h, "fact_gemm_host_wait", e);
+  if (dev != h->device) cudaSetDevice(dev);
+  return st;
 }
 
 fact_status_t fact_gemm_batched(fact_handle_t h, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A,

@@ -33,7 +33,7 @@ class HostGemmPipeline:
         self.out_dtype = out_dtype
         self.scratch = {}
         for (M, N, K) in set(shapes):
-            nbytes = h.gemm_host_scratch_bytes(M, N, K, out_dtype)
+            nbytes = h.gemm_host_scratch_bytes(M, N, K, out_dtype, layout)
             self.scratch[(M, N, K)] = [torch.empty(nbytes, dtype=torch.uint8, device=self.dev) for _ in range(depth)]
         self.turn = {k: 0 for k in self.scratch}
         self.h2d_bytes = 0
@@ -54,4 +54,5 @@ class HostGemmPipeline:
     def finish(self, stream=None):
         """Block until every submitted problem's result is in host memory."""
         s = stream if stream is not None else torch.cuda.current_stream(self.dev)
+        self.h.gemm_host_wait(s)
         s.synchronize()

@@ -52,9 +52,10 @@ def test_gemm_host_entry_point_layouts_strides_and_errors():
     A, W = Abig[:, :K], Wbig[:, :K]
     Cbig = torch.zeros(M, N + 8, dtype=torch.float32).pin_memory()
     C = Cbig[:, :N]
-    scratch = torch.empty(h.gemm_host_scratch_bytes(M, N, K, torch.float32), dtype=torch.uint8, device="cuda:0")
+    scratch = torch.empty(h.gemm_host_scratch_bytes(M, N, K, torch.float32, "NK"), dtype=torch.uint8, device="cuda:0")
     for _ in range(3):  # the same scratch again and again: each call waits for the copy-out of the one before
         h.gemm_host(A, W, C, scratch, layout="NK")
+    h.gemm_host_wait()
     torch.cuda.current_stream(0).synchronize()
     assert h.device_status() == 0
     ref = oracle.linear(wl.bits(Abig)[:, :K], wl.bits(Wbig)[:, :K], layout="NK")
