@@ -563,18 +563,25 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         # also times the launch itself (10-12 us on this part), so the figure that counts for them is N launches back
         # to back between one event pair, rotating through R sets of operands and outputs whose total exceeds twice
         # the L2 -- every launch still finds its data in DRAM, and the cost per launch is the stream time it adds.
-        t_use = med
+        # Which time the roofline fraction uses: an HBM-bound shape (and the latency-bound 512^3) the train -- every
+        # launch cold, write-back of the previous output included, no launch latency -- against the measured copy
+        # bandwidth; a tensor-bound shape the single cold launch against the burst peak (a kernel timed alone), with
+        # the train against the sustained peak (a kernel timed inside a long run) reported beside it.
+        t_use, used_train = med, False
         if med * 1e3 < SHORT_SHAPE_US and trains:
             t_b2b = back_to_back_us(call_set=None, case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev,
                                     stream=stream) * 1e-3
             row["us_back_to_back_cold"] = t_b2b * 1e3
-            row["timing"] = "back-to-back launches over rotating buffer sets (total > 2 x L2), per launch"
             if side_ref:
                 row["cublas_matmul_only_back_to_back_us"] = back_to_back_us(
                     call_set="side", case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev, stream=stream)
-            t_use = t_b2b
-        else:
-            row["timing"] = "one launch per event pair after an L2 flush, median"
+            t_tensor_sustained = case.flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+            row["roofline_frac_train"] = (t_hbm if bound == "hbm" else t_tensor_sustained) / t_b2b
+            row["roofline_train_peak"] = "measured copy bandwidth" if bound == "hbm" else "measured sustained BF16 peak"
+            if bound == "hbm":
+                t_use, used_train = t_b2b, True
+        row["timing"] = ("back-to-back launches over rotating buffer sets (total > 2 x L2), per launch"
+                         if used_train else "one launch per event pair after an L2 flush, median")
         row.update({
             "us": t_use * 1e3, "tflops": case.flops / (t_use * 1e-3) / 1e12,
             "gbs": case.algorithmic_bytes / (t_use * 1e-3) / 1e9,
