@@ -549,10 +549,7 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         t_hbm = case.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
         bound = "tensor" if t_tensor >= t_hbm else "hbm"
         cfg = h.get_config(case.op, case.batch, case.M, case.N, case.K, case.epilogue, case.layout, odt).as_dict()
-        span_us, span_mhz = kernel_span_us()
         row = {
-            "us_kernel_span_first_cta": span_us, "sm_mhz_in_kernel": span_mhz,
-            "roofline_frac_of_kernel_span": max(t_tensor, t_hbm) * 1e3 / span_us if span_us else None,
             "name": case.name, "config": case.config, "op": case.op, "epilogue": case.epilogue,
             "layout": case.layout, "batch": case.batch, "M": case.M, "N": case.N, "K": case.K, "out": case.out,
             "us_median": med * 1e3, "us_min": t[0] * 1e3, "us_hot_l2_median": t_hot[len(t_hot) // 2] * 1e3,
@@ -568,6 +565,11 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
         # bandwidth; a tensor-bound shape the single cold launch against the burst peak (a kernel timed alone), with
         # the train against the sustained peak (a kernel timed inside a long run) reported beside it.
         t_use, used_train = med, False
+        if med * 1e3 < SHORT_SHAPE_US:
+            # (short launches only: there the event pair's fixed 7-10 us are a large part of the figure)
+            span_us, span_mhz = kernel_span_us()
+            row.update({"us_kernel_span_first_cta": span_us, "sm_mhz_in_kernel": span_mhz,
+                        "roofline_frac_of_kernel_span": max(t_tensor, t_hbm) * 1e3 / span_us if span_us else None})
         if med * 1e3 < SHORT_SHAPE_US and trains:
             t_b2b = back_to_back_us(call_set=None, case=case, X=X, W=W, bias=bias, res=res, out=out, h=h, dev=dev,
                                     stream=stream) * 1e-3
