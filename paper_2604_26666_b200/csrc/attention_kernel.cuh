@@ -191,7 +191,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const uint32_t tmem_base = *tmem_holder_p;
   // the set-up above may overlap the tail of the previous kernel in the stream; global memory only from here on
   ptx::grid_dependency_wait();
-  ptx::grid_launch_dependents();
 
   // Items are numbered with the query position as the slow index, heaviest first (the late rows of a causal
   // problem), so neighbouring CTAs work on query heads that share K and V.
@@ -564,6 +563,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   }
 
   // ------------------------------------------------------------ teardown
+  ptx::grid_launch_dependents();  // this CTA's items are done: the next kernel of the stream may move in behind it
   if (*abort_p) {
     const unsigned long long tw = ptx::globaltimer_ns();
     while (ptx::globaltimer_ns() - tw < 200000ull) {

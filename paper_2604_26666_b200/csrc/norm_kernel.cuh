@@ -51,8 +51,8 @@ __device__ __forceinline__ float norm_warp_sum(float v) {
 
 template <int CH, bool RMS>
 __global__ void __launch_bounds__(kNormWarps * 32, (CH <= 16) ? 2 : 1) fact_norm_kernel(const NormParams p) {
-  ptx::grid_dependency_wait();  // (launched with programmatic stream serialization: see ptx.cuh)
-  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();  // (launched with programmatic stream serialization: see ptx.cuh; the successor is
+                                // released when this grid's CTAs exit)
   const int lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * kNormWarps + (threadIdx.x >> 5);
   if (row >= p.M) return;

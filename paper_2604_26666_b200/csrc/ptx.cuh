@@ -34,7 +34,8 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 // stream is still running.  grid_dependency_wait blocks until that predecessor has completed and its memory
 // operations are visible (a no-op for an ordinary launch); nothing that reads or writes global memory may come
 // before it.  grid_launch_dependents lets the successor's CTAs be scheduled as soon as every CTA of this grid has
-// executed it (or exited) -- they still wait, in their own grid_dependency_wait, for this grid to complete.
+// executed it (or exited) -- they still wait, in their own grid_dependency_wait, for this grid to complete.  The
+// kernels say it when a CTA's work is done, not earlier (see the GEMM kernel's teardown).
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
