@@ -107,3 +107,28 @@ def test_dynamic_schedule_refusals_and_fallbacks(h):
     # a single wave: nothing to hand out, the static grid runs
     small = mk("dyn_one_wave", 300, 200, 128)
     check_case(h, small, cfg={"tile_m": 128, "tile_n": 64, "cta_group": 1, "schedule": 2})
+
+
+def test_dynamic_schedule_in_a_cuda_graph_and_back_to_back(h):
+    """A dynamically scheduled launch can be captured and replayed, and launches that follow one another on a stream
+    (each is allowed to move onto the SMs while its predecessor's last CTAs leave) give the same bits every time."""
+    case = mk("dyn_graph", 2048, 1024, 520, epilogue="BIAS_RELU")
+    ins = wl.make_inputs(case)
+    dev = "cuda:0"
+    X, W, b = ins.X.to(dev), ins.W.to(dev), ins.bias.to(dev)
+    cfg = {"tile_m": 256, "tile_n": 64, "cta_group": 2, "schedule": 2}
+    first = h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", cfg=cfg)
+    torch.cuda.synchronize()
+    out = torch.empty_like(first)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream(dev)):
+        for _ in range(4):  # four launches back to back inside the graph
+            h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", out=out, cfg=cfg)
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, first)
+    assert h.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", case.epilogue)
+    assert c <= 1 and t <= 1, (c, t)
