@@ -472,9 +472,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         const uint64_t scale2 = ptx::pack_f32x2(__float_as_uint(p.scale_log2), __float_as_uint(p.scale_log2));
         const uint64_t negm2 = ptx::pack_f32x2(__float_as_uint(-m_use), __float_as_uint(-m_use));
         uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
+        uint32_t pw[BK / 64][32];
 #pragma unroll
         for (int hh = 0; hh < BK / 64; ++hh) {  // 64 keys = 32 columns of BF16 pairs at a time
-          uint32_t pw[32];
 #pragma unroll
           for (int c = 0; c < 2; ++c)
 #pragma unroll
@@ -493,17 +493,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
               sum2[pr & 3] = ptx::add_f32x2(sum2[pr & 3], p2);
               uint32_t p0, p1;
               ptx::unpack_f32x2(p2, p0, p1);
-              pw[pr] = pack_bf16x2(__uint_as_float(p0), __uint_as_float(p1));
+              pw[hh][pr] = pack_bf16x2(__uint_as_float(p0), __uint_as_float(p1));
             }
-          // the probabilities of the block before must have been consumed before these overwrite them
-          if (hh == 0 && gt > 0 && !pv_waited) {
-            ok = wait_all(bar(PV_DONE + t), (uint32_t)(gt - 1) & 1u);
-            if (!ok) break;
-          }
-          // lane = row, column c holds keys 2c and 2c + 1
-          ptx::tmem_st_32x32b_x32(p_addr + (uint32_t)hh * 32u, pw);
         }
-        if (!ok) break;
+        // the probabilities of the block before must have been consumed before these overwrite them
+        if (gt > 0 && !pv_waited) {
+          ok = wait_all(bar(PV_DONE + t), (uint32_t)(gt - 1) & 1u);
+          if (!ok) break;
+        }
+        // lane = row, column c holds keys 2c and 2c + 1
+#pragma unroll
+        for (int hh = 0; hh < BK / 64; ++hh) ptx::tmem_st_32x32b_x32(p_addr + (uint32_t)hh * 32u, pw[hh]);
         {
           const uint64_t st = ptx::add_f32x2(ptx::add_f32x2(sum2[0], sum2[1]), ptx::add_f32x2(sum2[2], sum2[3]));
           uint32_t lo, hi;
