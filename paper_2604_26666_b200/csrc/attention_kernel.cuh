@@ -408,9 +408,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           ++prof_blocks;
         }
         ptx::tc_fence_after();
-        uint32_t s[BK / 32][32];
+        uint32_t s64[BK / 64][64];
 #pragma unroll
-        for (int c = 0; c < BK / 32; ++c) ptx::tmem_ld_32x32b_x32(s_addr + (uint32_t)c * 32u, s[c]);
+        for (int c = 0; c < BK / 64; ++c) ptx::tmem_ld_32x32b_x64(s_addr + (uint32_t)c * 64u, s64[c]);
+        uint32_t (&s)[BK / 32][32] = *reinterpret_cast<uint32_t (*)[BK / 32][32]>(&s64[0][0]);
         ptx::tmem_wait_ld();
         // the scores are in registers: the next block's may overwrite them
         ptx::tc_fence_before();
@@ -502,8 +503,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           if (!ok) break;
         }
         // lane = row, column c holds keys 2c and 2c + 1
-#pragma unroll
-        for (int hh = 0; hh < BK / 64; ++hh) ptx::tmem_st_32x32b_x32(p_addr + (uint32_t)hh * 32u, pw[hh]);
+        if constexpr (BK == 128) {
+          ptx::tmem_st_32x32b_x64(p_addr, *reinterpret_cast<uint32_t (*)[64]>(&pw[0][0]));
+        } else {
+          ptx::tmem_st_32x32b_x32(p_addr, pw[0]);
+        }
         {
           const uint64_t st = ptx::add_f32x2(ptx::add_f32x2(sum2[0], sum2[1]), ptx::add_f32x2(sum2[2], sum2[3]));
           uint32_t lo, hi;
