@@ -511,6 +511,24 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
             else:
                 torch.matmul(X, W if case.layout == "KN" else W.t())
 
+        def side_same_op():
+            # the same fused operation composed from PyTorch's own operators (eager; cuBLASLt's bias epilogue where
+            # F.linear uses it): what the fusion is worth, next to the bare product above
+            import torch.nn.functional as F
+            wt = W.t() if case.layout == "KN" else W  # [N, K]
+            if case.epilogue == "SILU_GATE":
+                y = F.linear(X, wt)
+                n = y.shape[-1] // 2
+                return F.silu(y[:, :n]) * y[:, n:]
+            y = F.linear(X, wt, bias)
+            if case.epilogue == "BIAS_RELU":
+                return torch.relu(y)
+            if case.epilogue == "BIAS_GELU_TANH":
+                return F.gelu(y, approximate="tanh")
+            if case.epilogue == "BIAS_RESIDUAL":
+                return y + res
+            return y
+
         if tune:
             h.tune(case.op, X, W, layout=case.layout, bias=bias, residual=res, epilogue=case.epilogue, out=out)
 
@@ -556,6 +574,9 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
             "bound": bound, "roofline_us": max(t_tensor, t_hbm) * 1e3,
             "cublas_matmul_only_us": t_side[len(t_side) // 2] * 1e3, "tile": cfg,
         }
+        if side_ref and case.op == "linear" and case.epilogue != "NONE":
+            t_same = time_it(side_same_op, iters=10)
+            row["torch_eager_same_op_us"] = t_same[len(t_same) // 2] * 1e3
         # Shapes of the order of 100 us and below: an event pair around ONE launch that follows the L2-flush kernels
         # also times the launch itself (10-12 us on this part), so the figure that counts for them is N launches back
         # to back between one event pair, rotating through R sets of operands and outputs whose total exceeds twice
