@@ -1,0 +1,104 @@
+"""Seeded sweep over shapes x epilogues x kernel configurations (Section 4.2: every candidate is verified).
+
+Each case draws a ragged problem size, an epilogue, a layout, an output type and a configuration from the space the
+tuner sweeps (tile width, stage count, CTA pairs, raster group, K slices or stream-K, store mode, schedule), runs it
+through the C ABI and compares the whole output with the FP64 oracle.  The inputs are small integers, so every
+product and every partial sum is exact in FP32 whatever the order of the additions: NONE / BIAS / ReLU / residual
+outputs must match the oracle bit for bit for every schedule, GELU and SiLU go through the gates.  A combination
+the library refuses as infeasible for the problem is relaxed knob by knob until it runs.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_26666_b200 import workloads as wl
+from tests.helpers import gates, oracle_for, run_gpu, small_int_inputs, to_f64
+
+pytestmark = pytest.mark.gpu
+
+EPILOGUES = ["NONE", "BIAS", "BIAS_RELU", "BIAS_GELU_TANH", "SILU_GATE", "BIAS_RESIDUAL"]
+EXACT = {"NONE", "BIAS", "BIAS_RELU", "BIAS_RESIDUAL"}
+N_CASES = 160
+
+
+def _draw(i):
+    rng = np.random.default_rng(9000 + i)
+    epi = EPILOGUES[int(rng.integers(0, len(EPILOGUES)))]
+    layout = "KN" if rng.integers(0, 2) else "NK"
+    out = "f32" if rng.integers(0, 4) == 0 else "bf16"
+    M = int(rng.choice([1, 40, 128, 200, 256, 392, 520, 777, 1024]))
+    N = 8 * int(rng.integers(1, 130))          # row pitches stay multiples of 16 bytes
+    K = 8 * int(rng.integers(1, 200))
+    if rng.integers(0, 5) == 0:
+        K = 64 * int(rng.integers(20, 70))     # long enough for slices and stream-K runs
+    cfg = {}
+    if rng.integers(0, 4):
+        cfg["cta_group"] = int(rng.choice([1, 2]))
+    if rng.integers(0, 3):
+        widths = [64, 128, 192, 256] if layout == "KN" else [32, 64, 96, 128, 160, 192, 256]
+        cfg["tile_n"] = int(rng.choice(widths))
+    if rng.integers(0, 2):
+        cfg["stages"] = int(rng.integers(2, 7))
+    if rng.integers(0, 2):
+        cfg["raster_group"] = int(rng.choice([-8, -3, -1, 1, 2, 5, 16]))
+    cfg["split_k"] = int(rng.choice([1, 1, 1, 2, 3, 5, -1, -2]))
+    cfg["store_mode"] = int(rng.choice([0, 0, 1, 2, 3]))
+    cfg["schedule"] = int(rng.choice([0, 1, 2]))
+    return epi, layout, out, M, N, K, cfg
+
+
+@pytest.fixture(scope="module")
+def h():
+    from paper_2604_26666_b200.binding import Handle
+    hd = Handle(0)
+    yield hd
+    hd.close()
+
+
+def test_seeded_sweep_of_shapes_epilogues_and_configurations(h):
+    from paper_2604_26666_b200.binding import FactError
+
+    ran, refused = 0, []
+    for i in range(N_CASES):
+        epi, layout, out, M, N, K, cfg = _draw(i)
+        has_bias = epi in ("BIAS", "BIAS_RELU", "BIAS_GELU_TANH", "BIAS_RESIDUAL")
+        case = wl.Case(f"fuzz{i}", "linear", M, N, K, epilogue=epi, layout=layout, out=out, has_bias=has_bias,
+                       has_residual=epi == "BIAS_RESIDUAL", seed=9000 + i)
+        ins = small_int_inputs(case, 9000 + i, lo=-2, hi=2)
+        tag = f"case {i}: {epi} {layout} {out} {M}x{N}x{K} {cfg}"
+        # A combination the library refuses as infeasible for this problem (refused before any launch) is relaxed one
+        # knob at a time, the most special first, until it is accepted.
+        got = None
+        for drop in (None, "schedule", "store_mode", "split_k", "tile_n", "cta_group", "stages", "raster_group"):
+            if drop is not None:
+                if drop not in cfg:
+                    continue
+                cfg = {k: v for k, v in cfg.items() if k != drop}
+            try:
+                got = run_gpu(h, ins, case, cfg=cfg)
+                break
+            except FactError as e:
+                assert e.code in (1, 3, 5), (tag, cfg, e)
+                refused.append((i, drop, e.code))
+        assert got is not None, f"{tag}: refused even with the library's own configuration"
+        tag += f" -> ran as {cfg}"
+        torch.cuda.synchronize()
+        assert h.device_status() == 0, tag
+        ref = oracle_for(ins, case)
+        g = to_f64(got)
+        assert g.shape == ref.shape and np.isfinite(g).all(), tag
+        if epi in EXACT:
+            if out == "bf16":
+                want = np.vectorize(oracle.round_bf16, otypes=[np.uint16])(ref)
+                bad = np.argwhere(wl.bits(got.cpu().contiguous()) != want)
+            else:
+                bad = np.argwhere(g != ref)
+            assert len(bad) == 0, f"{tag}: {len(bad)} of {ref.size} elements differ, first at {bad[:4].tolist()}"
+        else:
+            c, t = gates(ref, g, out, epi)
+            assert c <= 1.0 and t <= 1.0, (tag, c, t)
+        ran += 1
+    assert ran == N_CASES
+    # most draws keep most of their knobs: the sweep is not a sweep of the default configuration
+    assert len(refused) < 2 * N_CASES, refused
