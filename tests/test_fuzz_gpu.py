@@ -102,3 +102,37 @@ def test_seeded_sweep_of_shapes_epilogues_and_configurations(h):
     assert ran == N_CASES
     # most draws keep most of their knobs: the sweep is not a sweep of the default configuration
     assert len(refused) < 2 * N_CASES, refused
+
+
+def test_seeded_sweep_of_batched_and_sliced_products(h):
+    """The same for the batched product and for the K-sliced product with a caller's slice count."""
+    for i in range(48):
+        rng = np.random.default_rng(9500 + i)
+        layout = "KN" if rng.integers(0, 2) else "NK"
+        out = "f32" if rng.integers(0, 2) else "bf16"
+        M = int(rng.choice([8, 130, 256, 300, 512]))
+        N = 8 * int(rng.integers(1, 70))
+        batched = bool(rng.integers(0, 2))
+        if batched:
+            K = 8 * int(rng.integers(1, 120))
+            case = wl.Case(f"fuzzb{i}", "gemm_batched", M, N, K, batch=int(rng.choice([2, 3, 5])), layout=layout, out=out,
+                           seed=9500 + i)
+            splits = 0
+        else:
+            K = 64 * int(rng.integers(4, 120)) + 8 * int(rng.integers(0, 8))
+            case = wl.Case(f"fuzzs{i}", "gemm_splitk", M, N, K, layout=layout, out=out, seed=9500 + i)
+            splits = int(rng.choice([0, 2, 3, 7, 12, 33]))
+        ins = small_int_inputs(case, 9500 + i, lo=-2, hi=2)
+        got = run_gpu(h, ins, case, splits=splits)
+        torch.cuda.synchronize()
+        tag = f"case {i}: {case.op} {layout} {out} batch {case.batch} {M}x{N}x{K} splits {splits}"
+        assert h.device_status() == 0, tag
+        ref = oracle_for(ins, case)
+        g = to_f64(got)
+        assert g.shape == ref.shape, tag
+        if out == "bf16":
+            want = np.vectorize(oracle.round_bf16, otypes=[np.uint16])(ref)
+            bad = np.argwhere(wl.bits(got.cpu().contiguous()) != want)
+        else:
+            bad = np.argwhere(g != ref)
+        assert len(bad) == 0, f"{tag}: {len(bad)} of {ref.size} elements differ, first at {bad[:4].tolist()}"
