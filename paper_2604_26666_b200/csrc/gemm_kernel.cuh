@@ -645,9 +645,96 @@ __device__ __forceinline__ void reduce_groups(const ReduceParams& p, long long f
   }
 }
 
+// The same sums for a few slices of a large output: one thread adds every slice of 8 adjacent columns of a row,
+// with all its loads in flight at once, and stores 16 (BF16) or 32 (FP32) bytes.  (The quads above keep one round
+// trip to L2 per 32 outputs of a warp, which a 16384 x 768 output with two slices pays 400 000 times over: 445 us.)
+// Same association as the quads -- s_q = slices q, q + 4 in ascending order, then (s0 + s1) + (s2 + s3) -- so the
+// two walks agree bit for bit and either may serve a call.
+constexpr int kReduceWideSlices = 8;
+__device__ __forceinline__ bool reduce_wide_applies(const ReduceParams& p) {
+  return p.splits <= kReduceWideSlices && p.epi != kEpiSiluGate && (p.ws_ld & 7) == 0;
+}
+__device__ __forceinline__ void reduce_wide(const ReduceParams& p, long long first, long long stride) {
+  const long long groups_per_row = (p.N_out + 7) / 8;
+  const long long total = (long long)p.batch * p.M * groups_per_row;
+  const long long plane_stride = (long long)p.M * p.ws_ld;
+  const long long slice_stride = (long long)p.batch * p.planes * plane_stride;
+  const size_t esz = p.out_f32 ? 4 : 2;
+  const bool c_vec = (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 && ((p.ldc * esz) & 15) == 0 && ((p.strideC * esz) & 15) == 0;
+  const bool r_vec = p.R != nullptr && (reinterpret_cast<uintptr_t>(p.R) & 15) == 0 && (p.ldr & 7) == 0 && (p.strideR & 7) == 0;
+  const bool b_vec = p.bias != nullptr && (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
+  for (long long i = first; i < total; i += stride) {
+    int gcol, m, b;
+    if (total < 0x7fffffffLL) {
+      const unsigned iu = (unsigned)i, gpr = (unsigned)groups_per_row;
+      const unsigned rmu = iu / gpr;
+      gcol = (int)(iu - rmu * gpr);
+      b = (int)(rmu / (unsigned)p.M);
+      m = (int)(rmu - (unsigned)b * (unsigned)p.M);
+    } else {
+      gcol = (int)(i % groups_per_row);
+      const long long rm = i / groups_per_row;
+      m = (int)(rm % p.M);
+      b = (int)(rm / p.M);
+    }
+    const int n = gcol * 8;
+    const int nvalid = min(8, p.N_out - n);
+    const float* base = p.ws + ((long long)b * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
+    float4 v[kReduceWideSlices][2];
+#pragma unroll
+    for (int sl = 0; sl < kReduceWideSlices; ++sl)
+      if (sl < p.splits) {  // (ws_ld is a multiple of 8 here: both loads stay inside the row's padding)
+        const float4* ps = reinterpret_cast<const float4*>(base + (long long)sl * slice_stride);
+        v[sl][0] = __ldcg(ps);
+        v[sl][1] = __ldcg(ps + 1);
+      }
+    float acc[4][8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[q][j] = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < kReduceWideSlices; ++sl)
+      if (sl < p.splits) {
+        const int q = sl & 3;
+        acc[q][0] += v[sl][0].x; acc[q][1] += v[sl][0].y; acc[q][2] += v[sl][0].z; acc[q][3] += v[sl][0].w;
+        acc[q][4] += v[sl][1].x; acc[q][5] += v[sl][1].y; acc[q][6] += v[sl][1].z; acc[q][7] += v[sl][1].w;
+      }
+    float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (p.bias != nullptr) load_bf16x8(p.bias + n, nvalid, b_vec, bias);
+    if (p.epi == kEpiBiasResidual)
+      load_bf16x8(p.R + (long long)b * p.strideR + (long long)m * p.ldr + n, nvalid, r_vec, res);
+    float y[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float tot = (acc[0][j] + acc[1][j]) + (acc[2][j] + acc[3][j]);
+      y[j] = reduce_epilogue(p.epi, tot * p.alpha, 0.f, bias[j], res[j]);
+    }
+    const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n;
+    if (p.out_f32) {
+      float* dst = reinterpret_cast<float*>(p.C) + off;
+      if (c_vec && nvalid == 8) {
+        reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
+        reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (j < nvalid) dst[j] = y[j];
+      }
+    } else {
+      store_bf16x8(reinterpret_cast<__nv_bfloat16*>(p.C) + off, y, nvalid, c_vec);
+    }
+  }
+}
+
+__device__ __forceinline__ void reduce_slices(const ReduceParams& p, long long first, long long stride) {
+  if (reduce_wide_applies(p)) reduce_wide(p, first, stride);
+  else reduce_groups(p, first, stride);
+}
+
 __global__ void __launch_bounds__(128) fact_splitk_reduce_kernel(const ReduceParams p) {
   ptx::grid_dependency_wait();  // (the successor is released when this grid's CTAs exit)
-  reduce_groups(p, blockIdx.x * (long long)blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+  reduce_slices(p, blockIdx.x * (long long)blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
 }
 
 // The fused element-wise operation on two adjacent output columns, as packed FP32 pairs
@@ -1702,7 +1789,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
         r.ldr = p.ldr;
         r.strideR = p.strideR;
         r.alpha = p.use_alpha ? p.alpha : 1.f;
-        reduce_groups(r, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
+        reduce_slices(r, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x);
       }
       __syncthreads();
       // the last CTA to leave resets both counters for the next launch
