@@ -268,6 +268,32 @@ def test_splitk_with_epilogue_through_linear(h):
         check_case(h, case, cfg={"split_k": 5})
 
 
+@pytest.mark.parametrize("out", ["bf16", "f32"])
+def test_few_slices_take_the_wide_reduction_and_keep_every_bit(h, out):
+    """With eight slices or fewer one thread adds all slices of 8 adjacent columns (vector or element-wise stores, a
+    ragged last group); with more, four lanes share a group of 4.  Integer inputs: both must equal the oracle bit for
+    bit, for aligned and unaligned outputs, with bias and residual."""
+    for (M, N, K, epi) in [(200, 136, 2048, "BIAS_RESIDUAL"), (130, 102, 1024, "BIAS_RELU"), (64, 1030, 512, "BIAS")]:
+        case = mk(f"wide_{N}_{epi}", M, N, K, epilogue=epi, layout="NK", out=out)
+        ins = small_int_inputs(case, 21, lo=-2, hi=2)
+        ref = oracle_for(ins, case)
+        for splits in (2, 3, 8, 9):
+            for pad in (0, 3):  # pad 3: rows of the output are not 16-byte aligned
+                dt = torch.float32 if out == "f32" else torch.bfloat16
+                big = torch.full((M, N + pad), -7.0, dtype=dt, device="cuda")
+                got = run_gpu(h, ins, case, cfg={"split_k": splits}, out=big[:, :N])
+                torch.cuda.synchronize()
+                assert h.device_status() == 0
+                if out == "bf16":
+                    want = np.vectorize(oracle.round_bf16, otypes=[np.uint16])(ref)
+                    bad = np.argwhere(wl.bits(got.cpu().contiguous()) != want)
+                else:
+                    bad = np.argwhere(got.cpu().double().numpy() != ref)
+                assert len(bad) == 0, (case.name, splits, pad, len(bad), bad[:4].tolist())
+                if pad:
+                    assert (big[:, N:] == -7.0).all(), "wrote outside the N columns"
+
+
 # ------------------------------------------------------------------ degenerate sizes
 def test_empty_and_k_zero(h):
     dev = "cuda:0"
