@@ -127,6 +127,11 @@ typedef enum {
  *                (whole waves, K == 0, an output the staged store cannot write) the call is data-parallel.
  *                Stream-K calls through one handle must be stream-ordered with respect to each other (they share
  *                the handle's flags) and must not share a workspace while they overlap.
+ *                0 (the library's choice) is one slice, except for an untuned fact_gemm / fact_linear whose tiles
+ *                are few and whose K is long (say 256 x 4096 x 14336): there the library's cost model may take
+ *                the K slices that fill the SMs in one wave, if the call brings the workspace that
+ *                fact_workspace_bytes reports for it -- without it the same call runs in one slice, like a table
+ *                entry.  The two differ in the order of the FP32 additions, not in anything else.
  *   store_mode   0 = library default, 1 = direct register stores (any alignment), 2 = shared-memory staged
  *                tensor stores, 3 = the staged epilogue's arithmetic with every row stored from registers in
  *                32-byte pieces (Y 32-byte aligned, ldy and N_out multiples of 32 bytes, whole data-parallel

@@ -305,11 +305,47 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     c.store_mode = 1;
   }
   if (c.cta_group == 0 && c.tile_m != 0) c.cta_group = (c.tile_m == 256) ? 2 : 1;
+  // The cost model of an untuned problem, in SM cycles: waves over the SMs times the cycles of one tile (k-blocks at
+  // the tensor-pipe rate of that width, plus a fixed hand-over cost).  A 2-CTA pair halves each CTA's B traffic and
+  // wins ties; narrow tiles only pay when wide ones leave SMs idle.  Where the tiles are few and K is long, K slices
+  // that fill the SMs in one wave are weighed against the reduction they need (a barrier, and the partial planes
+  // through L2): a 256 x 4096 x 14336 product is 16 wide tiles of 224 k-blocks, or four times as many of 56.
+  const int k_blocks_all = std::max(1, (int)((q.K + q.k_elems() - 1) / q.k_elems()));
+  const bool may_slice = c.split_k == 0 && (q.op == FACT_OP_GEMM || q.op == FACT_OP_LINEAR) && q.batch == 1 &&
+                         q.groups == 0 && !q.fp8 && !q.stats_out && !q.norm && q.epi != FACT_EPI_BIAS_SOFTMAX;
+  auto model = [&](int cg, int tn, int* slices_out) -> double {
+    const int out_cols = q.epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
+    const long long tiles =
+        std::max<long long>(1, q.batch) * ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + out_cols - 1) / out_cols);
+    const long long slots = std::max(1, h->sm_count / cg);
+    // (narrower tiles re-read the A operand from shared memory for less work: measured 0.65 of the full rate at
+    // 128 columns, taken as 0.85 at 192)
+    const double eff = tn >= 256 ? 1.0 : (tn >= 192 ? 0.85 : 0.65);
+    auto per_tile = [&](double kb) {
+      return kb * 512.0 * std::max(tn, 96) / 256.0 / eff + 1500.0 + (cg == 1 ? 60.0 * kb : 0.0);
+    };
+    double best_cost = (double)((tiles + slots - 1) / slots) * per_tile(k_blocks_all);
+    int best_s = 1;
+    if (may_slice) {
+      const double plane_bytes = (double)q.M * (double)round_up((int)q.N_out, 4) * 4.0 * ws_planes_for(q);
+      for (int s2 = 2; tiles * s2 <= slots && k_blocks_all / s2 >= 4; ++s2) {
+        if (plane_bytes * s2 > 64.0 * 1024 * 1024) break;  // scratch a caller would not expect to be asked for
+        const double kb = std::ceil((double)k_blocks_all / s2);
+        // measured on the part: the partial stores, the grid barrier and the reduction cost 8-12 us even for a
+        // 256 x 256 output (256 x 256 x 32768: 108 us in one slice, 65 / 43 / 31 in 2 / 4 / 8), and the planes
+        // travel at about 900 bytes a cycle (two 1536 x 1536 planes: 21k cycles)
+        const double cost = per_tile(kb) + 18000.0 + plane_bytes * s2 / 900.0;
+        if (cost < best_cost * 0.8) {  // (slices must win clearly: they cost scratch and a second rounding order)
+          best_cost = cost;
+          best_s = s2;
+        }
+      }
+    }
+    if (slices_out) *slices_out = best_s;
+    return best_cost;
+  };
+  int model_slices = 1;
   if (c.cta_group == 0 || c.tile_n == 0) {
-    // Untuned problem: pick (pair size, tile width) with a small cost model -- waves over the SMs times the
-    // cycles of one tile (k-blocks at the tensor-pipe rate of that width, plus a fixed hand-over cost).  A
-    // 2-CTA pair halves each CTA's B traffic and wins ties; narrow tiles only pay when wide ones leave SMs idle.
-    const int k_blocks = std::max(1, (int)((q.K + q.k_elems() - 1) / q.k_elems()));
     double best = 1e300;
     int best_cg = 0, best_tn = 0;
     for (int cg = 2; cg >= 1; --cg) {
@@ -317,30 +353,25 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
       for (int tn = 256; tn >= 64; tn -= 64) {
         if (c.tile_n != 0 && c.tile_n != tn) continue;
         if (!tile_ok(q, tn, cg) || max_stages_for(q, tn, cg) < 2) continue;
-        const int out_cols = q.epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
-        const long long tiles =
-            std::max<long long>(1, q.batch) * ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + out_cols - 1) / out_cols);
-        const long long slots = std::max(1, h->sm_count / cg);
-        const double waves = (double)((tiles + slots - 1) / slots);
-        // (narrower tiles re-read the A operand from shared memory for less work: measured 0.65 of the full rate at
-        // 128 columns, taken as 0.85 at 192)
-        const double eff = tn >= 256 ? 1.0 : (tn >= 192 ? 0.85 : 0.65);
-        const double per_tile =
-            k_blocks * 512.0 * std::max(tn, 96) / 256.0 / eff + 1500.0 + (cg == 1 ? 60.0 * k_blocks : 0.0);
-        const double cost = waves * per_tile;
+        int sl = 1;
+        const double cost = model(cg, tn, &sl);
         if (cost < best * 0.999) {
           best = cost;
           best_cg = cg;
           best_tn = tn;
+          model_slices = sl;
         }
       }
     }
     if (best_cg == 0) {  // nothing in the 64-column grid fits (a user-chosen odd width): keep what was asked
       best_cg = c.cta_group ? c.cta_group : 1;
       best_tn = c.tile_n ? c.tile_n : 64;
+      model_slices = 1;
     }
     c.cta_group = best_cg;
     c.tile_n = best_tn;
+  } else if (may_slice && !from_table && tile_ok(q, c.tile_n, c.cta_group)) {
+    (void)model(c.cta_group, c.tile_n, &model_slices);
   }
   if (c.tile_m == 0) c.tile_m = 128 * c.cta_group;
   if (c.tile_m != 128 * c.cta_group) return FACT_ERR_UNSUPPORTED;
@@ -353,7 +384,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.raster_group == 0) c.raster_group = raster_model(h, q, c);
   const int k_blocks = (int)((q.K + q.k_elems() - 1) / q.k_elems());
   if (c.split_k == 0) {
-    c.split_k = 1;
+    c.split_k = may_slice ? model_slices : 1;
     if (q.op == FACT_OP_GEMM_SPLITK) {
       const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
       const long long tiles = q.batch * ((q.M + c.tile_m - 1) / c.tile_m) * ((q.N_out + out_cols - 1) / out_cols);
@@ -837,12 +868,17 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     st = make_plan(h, q, &dp, 0, &plan);
     if (st != FACT_OK) return st;
   }
-  if (plan.cfg.split_k > 1 && plan.from_table && splits_override == 0 && q.op != FACT_OP_GEMM_SPLITK &&
-      (!ws || ws_bytes < plan.ws_bytes || !aligned16(ws))) {
-    // a tuned entry with K slices, but this caller brought no (or too little) scratch: one slice
+  if (plan.cfg.split_k > 1 && (plan.from_table || !user || user->split_k == 0) && splits_override == 0 &&
+      q.op != FACT_OP_GEMM_SPLITK && (!ws || ws_bytes < plan.ws_bytes || !aligned16(ws))) {
+    // K slices from the tuner's table or the library's own model, but this caller brought no (or too little)
+    // scratch: one slice
     fact_config_t dp = plan.cfg;
+    if (!plan.from_table) {  // the model's choice: choose the tiles again, for one slice
+      memset(&dp, 0, sizeof dp);
+      if (user) dp = *user;
+    }
     dp.split_k = 1;
-    dp.store_mode = 0;
+    dp.store_mode = plan.from_table ? 0 : dp.store_mode;
     st = make_plan(h, q, &dp, 0, &plan);
     if (st != FACT_OK) return st;
   }

@@ -654,7 +654,9 @@ constexpr int kReduceWideSlices = 8;
 __device__ __forceinline__ bool reduce_wide_applies(const ReduceParams& p) {
   return p.splits <= kReduceWideSlices && p.epi != kEpiSiluGate && (p.ws_ld & 7) == 0;
 }
-__device__ __forceinline__ void reduce_wide(const ReduceParams& p, long long first, long long stride) {
+// G groups per trip, each with up to S slices: G * S * 2 16-byte loads in flight per thread.
+template <int G, int S>
+__device__ __forceinline__ void reduce_wide_gs(const ReduceParams& p, long long first, long long stride) {
   const long long groups_per_row = (p.N_out + 7) / 8;
   const long long total = (long long)p.batch * p.M * groups_per_row;
   const long long plane_stride = (long long)p.M * p.ws_ld;
@@ -663,68 +665,85 @@ __device__ __forceinline__ void reduce_wide(const ReduceParams& p, long long fir
   const bool c_vec = (reinterpret_cast<uintptr_t>(p.C) & 15) == 0 && ((p.ldc * esz) & 15) == 0 && ((p.strideC * esz) & 15) == 0;
   const bool r_vec = p.R != nullptr && (reinterpret_cast<uintptr_t>(p.R) & 15) == 0 && (p.ldr & 7) == 0 && (p.strideR & 7) == 0;
   const bool b_vec = p.bias != nullptr && (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0;
-  for (long long i = first; i < total; i += stride) {
-    int gcol, m, b;
-    if (total < 0x7fffffffLL) {
-      const unsigned iu = (unsigned)i, gpr = (unsigned)groups_per_row;
-      const unsigned rmu = iu / gpr;
-      gcol = (int)(iu - rmu * gpr);
-      b = (int)(rmu / (unsigned)p.M);
-      m = (int)(rmu - (unsigned)b * (unsigned)p.M);
-    } else {
-      gcol = (int)(i % groups_per_row);
-      const long long rm = i / groups_per_row;
-      m = (int)(rm % p.M);
-      b = (int)(rm / p.M);
-    }
-    const int n = gcol * 8;
-    const int nvalid = min(8, p.N_out - n);
-    const float* base = p.ws + ((long long)b * p.planes) * plane_stride + (long long)m * p.ws_ld + n;
-    float4 v[kReduceWideSlices][2];
+  for (long long i0 = first; i0 < total; i0 += stride * G) {
+    int n[G], m[G], b[G];
+    bool valid[G];
+    float4 v[G][S][2];
 #pragma unroll
-    for (int sl = 0; sl < kReduceWideSlices; ++sl)
-      if (sl < p.splits) {  // (ws_ld is a multiple of 8 here: both loads stay inside the row's padding)
-        const float4* ps = reinterpret_cast<const float4*>(base + (long long)sl * slice_stride);
-        v[sl][0] = __ldcg(ps);
-        v[sl][1] = __ldcg(ps + 1);
-      }
-    float acc[4][8];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[q][j] = 0.f;
-#pragma unroll
-    for (int sl = 0; sl < kReduceWideSlices; ++sl)
-      if (sl < p.splits) {
-        const int q = sl & 3;
-        acc[q][0] += v[sl][0].x; acc[q][1] += v[sl][0].y; acc[q][2] += v[sl][0].z; acc[q][3] += v[sl][0].w;
-        acc[q][4] += v[sl][1].x; acc[q][5] += v[sl][1].y; acc[q][6] += v[sl][1].z; acc[q][7] += v[sl][1].w;
-      }
-    float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (p.bias != nullptr) load_bf16x8(p.bias + n, nvalid, b_vec, bias);
-    if (p.epi == kEpiBiasResidual)
-      load_bf16x8(p.R + (long long)b * p.strideR + (long long)m * p.ldr + n, nvalid, r_vec, res);
-    float y[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float tot = (acc[0][j] + acc[1][j]) + (acc[2][j] + acc[3][j]);
-      y[j] = reduce_epilogue(p.epi, tot * p.alpha, 0.f, bias[j], res[j]);
-    }
-    const long long off = (long long)b * p.strideC + (long long)m * p.ldc + n;
-    if (p.out_f32) {
-      float* dst = reinterpret_cast<float*>(p.C) + off;
-      if (c_vec && nvalid == 8) {
-        reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
-        reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+    for (int g = 0; g < G; ++g) {
+      const long long i = i0 + (long long)g * stride;
+      valid[g] = i < total;
+      const long long ii = valid[g] ? i : 0;
+      int gcol;
+      if (total < 0x7fffffffLL) {
+        const unsigned iu = (unsigned)ii, gpr = (unsigned)groups_per_row;
+        const unsigned rmu = iu / gpr;
+        gcol = (int)(iu - rmu * gpr);
+        b[g] = (int)(rmu / (unsigned)p.M);
+        m[g] = (int)(rmu - (unsigned)b[g] * (unsigned)p.M);
       } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (j < nvalid) dst[j] = y[j];
+        gcol = (int)(ii % groups_per_row);
+        const long long rm = ii / groups_per_row;
+        m[g] = (int)(rm % p.M);
+        b[g] = (int)(rm / p.M);
       }
-    } else {
-      store_bf16x8(reinterpret_cast<__nv_bfloat16*>(p.C) + off, y, nvalid, c_vec);
+      n[g] = gcol * 8;
+      const float* base = p.ws + ((long long)b[g] * p.planes) * plane_stride + (long long)m[g] * p.ws_ld + n[g];
+#pragma unroll
+      for (int sl = 0; sl < S; ++sl)
+        if (valid[g] && sl < p.splits) {  // (ws_ld is a multiple of 8 here: both loads stay inside the row's padding)
+          const float4* ps = reinterpret_cast<const float4*>(base + (long long)sl * slice_stride);
+          v[g][sl][0] = __ldcg(ps);
+          v[g][sl][1] = __ldcg(ps + 1);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      if (!valid[g]) continue;
+      const int nvalid = min(8, p.N_out - n[g]);
+      float acc[4][8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[q][j] = 0.f;
+#pragma unroll
+      for (int sl = 0; sl < S; ++sl)
+        if (sl < p.splits) {
+          const int q = sl & 3;
+          acc[q][0] += v[g][sl][0].x; acc[q][1] += v[g][sl][0].y; acc[q][2] += v[g][sl][0].z; acc[q][3] += v[g][sl][0].w;
+          acc[q][4] += v[g][sl][1].x; acc[q][5] += v[g][sl][1].y; acc[q][6] += v[g][sl][1].z; acc[q][7] += v[g][sl][1].w;
+        }
+      float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, res[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (p.bias != nullptr) load_bf16x8(p.bias + n[g], nvalid, b_vec, bias);
+      if (p.epi == kEpiBiasResidual)
+        load_bf16x8(p.R + (long long)b[g] * p.strideR + (long long)m[g] * p.ldr + n[g], nvalid, r_vec, res);
+      float y[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float tot = (acc[0][j] + acc[1][j]) + (acc[2][j] + acc[3][j]);
+        y[j] = reduce_epilogue(p.epi, tot * p.alpha, 0.f, bias[j], res[j]);
+      }
+      const long long off = (long long)b[g] * p.strideC + (long long)m[g] * p.ldc + n[g];
+      if (p.out_f32) {
+        float* dst = reinterpret_cast<float*>(p.C) + off;
+        if (c_vec && nvalid == 8) {
+          reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
+          reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (j < nvalid) dst[j] = y[j];
+        }
+      } else {
+        store_bf16x8(reinterpret_cast<__nv_bfloat16*>(p.C) + off, y, nvalid, c_vec);
+      }
     }
   }
+}
+__device__ __forceinline__ void reduce_wide(const ReduceParams& p, long long first, long long stride) {
+  if (p.splits <= 2) reduce_wide_gs<4, 2>(p, first, stride);
+  else if (p.splits <= 4) reduce_wide_gs<2, 4>(p, first, stride);
+  else reduce_wide_gs<1, kReduceWideSlices>(p, first, stride);
 }
 
 __device__ __forceinline__ void reduce_slices(const ReduceParams& p, long long first, long long stride) {

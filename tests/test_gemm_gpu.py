@@ -294,6 +294,34 @@ def test_few_slices_take_the_wide_reduction_and_keep_every_bit(h, out):
                     assert (big[:, N:] == -7.0).all(), "wrote outside the N columns"
 
 
+def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
+    """The library's own choice for an untuned product of few tiles and long K is K slices (Section 4.2, Action 2:
+    the grid-level policy is a design choice) -- with the workspace the binding brings; the same call through the C
+    ABI without a workspace runs in one slice.  Both are checked against the oracle."""
+    import ctypes
+
+    from paper_2604_26666_b200.binding import lib
+
+    case = mk("few_tiles_long_k", 256, 512, 16384, op="gemm", layout="NK")
+    cfg = h.get_config("gemm", 1, case.M, case.N, case.K, "NONE", "NK", torch.bfloat16).as_dict()
+    assert cfg["split_k"] > 1, cfg
+    assert h.workspace_bytes("gemm", 1, case.M, case.N, case.K, "NONE", "NK", torch.bfloat16) > 0
+    ins = wl.make_inputs(case)
+    check_case(h, case, ins=ins)
+    # an explicit single slice is respected, and a short K is never sliced
+    assert h.get_config("gemm", 1, 256, 512, 512, "NONE", "NK", torch.bfloat16).as_dict()["split_k"] == 1
+    X, W = ins.X.cuda(), ins.W.cuda()
+    out = torch.full((case.M, case.N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    rc = lib().fact_gemm(h._h, case.M, case.N, case.K, ctypes.c_void_p(X.data_ptr()), X.stride(0),
+                         ctypes.c_void_p(W.data_ptr()), W.stride(0), 1, ctypes.c_void_p(out.data_ptr()), out.stride(0), 0,
+                         None, None, 0, None)
+    assert rc == 0, rc
+    torch.cuda.synchronize()
+    assert h.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out), "bf16", "NONE")
+    assert c <= 1.0 and t <= 1.0, (c, t)
+
+
 # ------------------------------------------------------------------ degenerate sizes
 def test_empty_and_k_zero(h):
     dev = "cuda:0"
