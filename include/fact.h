@@ -131,7 +131,8 @@ typedef enum {
  *                are few and whose K is long (say 256 x 4096 x 14336): there the library's cost model may take
  *                the K slices that fill the SMs in one wave, if the call brings the workspace that
  *                fact_workspace_bytes reports for it -- without it the same call runs in one slice, like a table
- *                entry.  The two differ in the order of the FP32 additions, not in anything else.
+ *                entry -- or 2 / 4 / 8 slices as a cluster (schedule 3), which needs no workspace.  The choices
+ *                differ in the order of the FP32 additions, not in anything else.
  *   store_mode   0 = library default, 1 = direct register stores (any alignment), 2 = shared-memory staged
  *                tensor stores, 3 = the staged epilogue's arithmetic with every row stored from registers in
  *                32-byte pieces (Y 32-byte aligned, ldy and N_out multiples of 32 bytes, whole data-parallel
@@ -146,7 +147,18 @@ typedef enum {
  *                computes a tile never changes a value: every tile is summed by one group in the same order.
  *                Dynamic scheduling serves whole tiles only (no K slices, stream-K, row sums, folded
  *                normalisation, register row stores or row softmax: FACT_ERR_UNSUPPORTED with those), and is
- *                the static schedule when all tiles fit one wave. */
+ *                the static schedule when all tiles fit one wave.
+ *                3 = the K slices of a tile as one thread-block cluster (the K-sliced regime of Section 5.2,
+ *                Problem 6, for products of few tiles and long K): split_k = 2, 4 or 8 CTAs share a 128-row tile
+ *                (tile_m 128, cta_group 1, tile_n a multiple of 32 * split_k), each multiplies its slice of K with
+ *                its own loads and its own accumulator -- no operand is loaded twice, nothing is multicast -- and
+ *                the slices are added up through distributed shared memory: CTA r sends block j of its
+ *                accumulator's columns to CTA j, which adds the blocks in the order of the workspace reduction
+ *                (same bits as the same split_k through a workspace), applies the epilogue and stores.  No
+ *                workspace, no partial planes in global memory, no grid-wide barrier.  Column-wise epilogues on
+ *                BF16 operands (not SILU_GATE, row softmax, 8-bit operands, groups, row sums or a folded
+ *                normalisation: FACT_ERR_UNSUPPORTED).  An untuned fact_gemm / fact_linear may take this schedule
+ *                on its own (see split_k). */
 typedef struct {
   int tile_m, tile_n, tile_k, stages, cta_group, raster_group, split_k, store_mode, schedule;
 } fact_config_t;

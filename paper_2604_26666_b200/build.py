@@ -21,7 +21,7 @@ LIB = PKG / "libfact.so"
 STAMP = PKG / "libfact.so.srchash"
 
 SOURCES = ["fact_api.cu"]
-HEADERS = ["gemm_kernel.cuh", "attention_kernel.cuh", "norm_kernel.cuh", "tune_kernels.cuh", "ptx.cuh"]
+HEADERS = ["gemm_kernel.cuh", "kcluster_kernel.cuh", "attention_kernel.cuh", "norm_kernel.cuh", "tune_kernels.cuh", "ptx.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

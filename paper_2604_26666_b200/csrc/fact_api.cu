@@ -19,6 +19,7 @@
 
 #include "fact.h"
 #include "gemm_kernel.cuh"
+#include "kcluster_kernel.cuh"
 #include "attention_kernel.cuh"
 #include "norm_kernel.cuh"
 #include "tune_kernels.cuh"
@@ -84,6 +85,7 @@ struct Plan {
   fact_config_t cfg;
   bool from_table = false;  // cfg came from the tuner's table: its store mode and K slices are hints, not demands
   bool dynamic = false;     // tiles are handed out through cluster launch control (one cluster of the grid per tile)
+  bool kcluster = false;    // the K slices of a tile run as one cluster and are added up through shared memory
   int smem_bytes;
   int grid;
   size_t ws_bytes;
@@ -102,6 +104,7 @@ struct fact_handle_s {
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
   std::bitset<192> configured_mask;  // kernels whose dynamic shared-memory limit was raised
+  int kc_clusters[3] = {0, 0, 0};    // clusters of 2 / 4 / 8 CTAs of the K-slice kernel the device holds at once
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: diagnostics (256 cycle counters, 2048 no K serpentine); the
                                  // work-skipping experiment switches only in a -DFACT_EXPERIMENTS build
@@ -231,6 +234,37 @@ bool tile_ok(const Problem& q, int tile_n, int cg) {
 // tiles: 1.04 GB with groups of 8 m-tiles, 1.00 GB with 12, 0.96 GB with 16; the Llama down projection: 1.43 GB with
 // groups of 4 n-tiles, 1.01 GB with 8; nominal L2 126 MB on two dies).  Returns G > 0 for groups of m-tiles, G < 0
 // for groups of n-tiles.
+// How many clusters of `slices` CTAs of the K-slice kernel are resident at once (a cluster needs its SMs inside one
+// GPC, so this is less than SMs / slices); asked of the runtime once per cluster size.
+int kc_max_clusters(fact_handle_t h, int slices) {
+  const int idx = slices == 2 ? 0 : (slices == 4 ? 1 : 2);
+  if (h->kc_clusters[idx] == 0) {
+    int n = 0, dev = -1;
+    const bool switched = cudaGetDevice(&dev) == cudaSuccess && dev != h->device && cudaSetDevice(h->device) == cudaSuccess;
+    auto kern = fact_gemm_kcluster_kernel<kEpiNone>;
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3((unsigned)(slices * h->sm_count), 1, 1);
+    lc.blockDim = dim3((unsigned)kKcThreads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)kSmemBudget;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)slices;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, kern, &lc) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = std::max(1, (h->sm_count / slices) * 3 / 4);  // (what GPCs of 16 usable SMs out of 18 or 20 would hold)
+    }
+    if (switched) cudaSetDevice(dev);
+    h->kc_clusters[idx] = n;
+  }
+  return h->kc_clusters[idx];
+}
+
 int raster_model(fact_handle_t h, const Problem& q, const fact_config_t& c) {
   const double l2_eff = 55.0 * 1024 * 1024;
   const int out_cols = q.epi == FACT_EPI_SILU_GATE ? c.tile_n / 2 : c.tile_n;
@@ -311,16 +345,18 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   // that fill the SMs in one wave are weighed against the reduction they need (a barrier, and the partial planes
   // through L2): a 256 x 4096 x 14336 product is 16 wide tiles of 224 k-blocks, or four times as many of 56.
   const int k_blocks_all = std::max(1, (int)((q.K + q.k_elems() - 1) / q.k_elems()));
+  const bool gate_epi = q.epi == FACT_EPI_SILU_GATE;
   const bool may_slice = c.split_k == 0 && (q.op == FACT_OP_GEMM || q.op == FACT_OP_LINEAR) && q.batch == 1 &&
                          q.groups == 0 && !q.fp8 && !q.stats_out && !q.norm && q.epi != FACT_EPI_BIAS_SOFTMAX;
-  auto model = [&](int cg, int tn, int* slices_out) -> double {
+  auto model = [&](int cg, int tn, int* slices_out, bool calibrated = false) -> double {
     const int out_cols = q.epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
     const long long tiles =
         std::max<long long>(1, q.batch) * ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + out_cols - 1) / out_cols);
     const long long slots = std::max(1, h->sm_count / cg);
-    // (narrower tiles re-read the A operand from shared memory for less work: measured 0.65 of the full rate at
-    // 128 columns, taken as 0.85 at 192)
-    const double eff = tn >= 256 ? 1.0 : (tn >= 192 ? 0.85 : 0.65);
+    // (narrower tiles re-read the A operand from shared memory for less work: 0.65 of the full rate at 128 columns,
+    // taken as 0.85 at 192, rank the widths against each other; timed on untuned shapes a k-block costs 450 cycles
+    // at 128 columns and 420 at 64 -- 0.57 and 0.45 -- which is what the comparison with the cluster schedule uses)
+    const double eff = tn >= 256 ? 1.0 : (tn >= 192 ? 0.85 : (!calibrated ? 0.65 : (tn >= 128 ? 0.57 : 0.45)));
     auto per_tile = [&](double kb) {
       return kb * 512.0 * std::max(tn, 96) / 256.0 / eff + 1500.0 + (cg == 1 ? 60.0 * kb : 0.0);
     };
@@ -370,6 +406,37 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     }
     c.cta_group = best_cg;
     c.tile_n = best_tn;
+    // K slices as a cluster (schedule 3: no workspace, no grid barrier): one wave of clusters of 2 / 4 / 8 CTAs on
+    // 128-row tiles.  Per k-block 400 / 450 / 1000 cycles at 64 / 128 / 256 columns, never faster than the operands
+    // stream from DRAM, plus 10k cycles (13k at 256 columns) for the exchange, the epilogue and a cold start --
+    // fitted to 66 timed (shape, slices, width) combinations, within a few percent where the cluster schedule wins.
+    if (may_slice && c.schedule == 0 && !gate_epi && (user == nullptr || user->cta_group == 0 || user->cta_group == 1) &&
+        (user == nullptr || user->tile_n == 0) && (user == nullptr || user->tile_m == 0 || user->tile_m == 128)) {
+      const double hbm = ((double)q.M + (double)Nw) * (double)q.K * 2.0 / 3686.0 * 1.15;
+      double best_kc = 1e300;
+      int kc_s = 0, kc_tn = 0;
+      for (int sl = 2; sl <= 8; sl *= 2)
+        for (int tn = 64; tn <= 256; tn *= 2) {
+          if (tn % (32 * sl) || !tile_ok(q, tn, 1) || max_stages_for(q, tn, 1) < 2 || k_blocks_all < 4 * sl) continue;
+          const long long tiles = ((q.M + 127) / 128) * ((q.N_out + tn - 1) / tn);
+          if (tiles > kc_max_clusters(h, sl)) continue;
+          const double per_kb = tn == 64 ? 400.0 : (tn == 128 ? 450.0 : 1000.0);
+          const double cost = std::max(std::ceil((double)k_blocks_all / sl) * per_kb, hbm) + (tn == 256 ? 13000.0 : 10000.0);
+          if (cost < best_kc) {
+            best_kc = cost;
+            kc_s = sl;
+            kc_tn = tn;
+          }
+        }
+      int unused = 1;
+      const double best_timed = best_cg != 0 ? model(best_cg, best_tn, &unused, true) : best;
+      if (kc_s != 0 && best_kc < 0.92 * best_timed) {
+        c.cta_group = 1;
+        c.tile_n = kc_tn;
+        c.split_k = kc_s;
+        c.schedule = 3;
+      }
+    }
   } else if (may_slice && !from_table && tile_ok(q, c.tile_n, c.cta_group)) {
     (void)model(c.cta_group, c.tile_n, &model_slices);
   }
@@ -397,7 +464,7 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   if (c.split_k < -2) return FACT_ERR_INVALID_ARG;
   if (c.split_k > 0) c.split_k = std::max(1, std::min(c.split_k, std::max(1, k_blocks)));
   if (c.store_mode < 0 || c.store_mode > 3) return FACT_ERR_INVALID_ARG;
-  if (c.schedule < 0 || c.schedule > 2) return FACT_ERR_INVALID_ARG;
+  if (c.schedule < 0 || c.schedule > 3) return FACT_ERR_INVALID_ARG;
   if (c.schedule == 0) c.schedule = 1;
   *out = c;
   if (from_table_out) *from_table_out = from_table;
@@ -476,6 +543,7 @@ int sk_tiles_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
 }
 
 size_t workspace_for(fact_handle_t h, const Problem& q, const fact_config_t& c) {
+  if (c.schedule == 3) return 0;  // K slices as a cluster: the partial sums never leave the SMs
   if (c.split_k < 0) {  // stream-K: one FP32 accumulator tile per CTA
     if (sk_tiles_for(h, q, c) == 0) return 0;
     const size_t ctas = (size_t)std::max(1, h->sm_count / c.cta_group) * (size_t)c.cta_group;
@@ -633,6 +701,20 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
       plan->cfg.schedule = 1;
     }
   }
+  if (c.schedule == 3) {
+    // K slices as a cluster: 128-row tiles, 2 / 4 / 8 slices, every CTA finishes tile_n / slices columns (whole
+    // 32-column pieces), column-wise epilogues on BF16 operands; every slice has at least one k-block
+    const bool can = cg == 1 && (c.split_k == 2 || c.split_k == 4 || c.split_k == 8) && c.tile_n % (32 * c.split_k) == 0 &&
+                     !gate && q.epi != FACT_EPI_BIAS_SOFTMAX && !q.fp8 && q.groups == 0 && !q.stats_out && !q.norm &&
+                     p.k_blocks >= c.split_k && units <= 0x7fffffffLL;
+    if (!can) return FACT_ERR_UNSUPPORTED;
+    plan->kcluster = true;
+    plan->ws_bytes = 0;
+    plan->smem_bytes = std::max((int)kc_smem_bytes(c.tile_n, c.split_k, c.stages, p.stage_bytes), kMinSmemRequest);
+    if (plan->smem_bytes > kSmemBudget) return FACT_ERR_UNSUPPORTED;
+    const long long tiles = units / c.split_k;
+    plan->grid = (int)std::min<long long>(tiles, kc_max_clusters(h, c.split_k)) * c.split_k;
+  }
   if (c.split_k < 0) {
     // Stream-K: the staged epilogue parks and finishes the pieces, so an output it cannot store is data-parallel.
     const int sk = p.store_tma ? sk_tiles_for(h, q, c) : 0;
@@ -703,6 +785,33 @@ fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const
   if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx", e);
   h->launches++;
   return FACT_OK;
+}
+
+template <int EPI>
+fact_status_t launch_kcluster_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
+                                       cudaStream_t stream) {
+  auto kern = fact_gemm_kcluster_kernel<EPI>;
+  if (!h->configured_mask.test((size_t)slot)) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+    h->configured_mask.set((size_t)slot);
+  }
+  cudaError_t e = launch_pdl(h, kern, (unsigned)plan.grid, (unsigned)kKcThreads, (size_t)plan.smem_bytes, stream,
+                             plan.cfg.split_k, tm[0], tm[1], plan.p);
+  if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx (K slices as a cluster)", e);
+  h->launches++;
+  return FACT_OK;
+}
+
+fact_status_t launch_kcluster(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  switch (epi) {
+    case kEpiNone: return launch_kcluster_instance<kEpiNone>(h, 150, plan, tm, stream);
+    case kEpiBias: return launch_kcluster_instance<kEpiBias>(h, 151, plan, tm, stream);
+    case kEpiBiasRelu: return launch_kcluster_instance<kEpiBiasRelu>(h, 152, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_kcluster_instance<kEpiBiasGeluTanh>(h, 153, plan, tm, stream);
+    case kEpiBiasResidual: return launch_kcluster_instance<kEpiBiasResidual>(h, 154, plan, tm, stream);
+    default: return FACT_ERR_UNSUPPORTED;
+  }
 }
 
 template <int CG>
@@ -806,6 +915,14 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
   Plan plan;
   st = make_plan(h, q, user, splits_override, &plan);
+  if (st == FACT_ERR_UNSUPPORTED && plan.from_table && plan.cfg.schedule == 3) {
+    // a table entry with K slices as a cluster, tuned on a plain call of this shape: this call (row sums, a folded
+    // normalisation) takes the library's own choice instead
+    fact_config_t none;
+    memset(&none, 0, sizeof none);
+    none.split_k = 1;
+    st = make_plan(h, q, &none, 0, &plan);
+  }
   if (st != FACT_OK) return st;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return FACT_ERR_CUDA;
@@ -868,7 +985,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     st = make_plan(h, q, &dp, 0, &plan);
     if (st != FACT_OK) return st;
   }
-  if (plan.cfg.split_k > 1 && (plan.from_table || !user || user->split_k == 0) && splits_override == 0 &&
+  if (plan.cfg.split_k > 1 && !plan.kcluster && (plan.from_table || !user || user->split_k == 0) && splits_override == 0 &&
       q.op != FACT_OP_GEMM_SPLITK && (!ws || ws_bytes < plan.ws_bytes || !aligned16(ws))) {
     // K slices from the tuner's table or the library's own model, but this caller brought no (or too little)
     // scratch: one slice
@@ -886,7 +1003,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
   if (q.K == 0) {  // empty sum: the epilogue of a zero accumulator
     st = launch_reduce(h, q, plan, 0, reinterpret_cast<const float*>(q.C), stream);
   } else {
-    const bool split = plan.cfg.split_k > 1;
+    const bool split = plan.cfg.split_k > 1 && !plan.kcluster;
     const bool stream_k = plan.cfg.split_k < 0;
     if (stream_k) {
       if (!ws || ws_bytes < plan.ws_bytes) return FACT_ERR_WORKSPACE_TOO_SMALL;
@@ -940,7 +1057,7 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       st = encode_map(h, &tm[2], ws, (uint64_t)plan.p.ws_ld, (uint64_t)q.M, planes, (uint64_t)plan.p.ws_ld,
                       (uint64_t)plan.p.ws_ld * (uint64_t)q.M, 32, 32, true);
       if (st != FACT_OK) return st;
-    } else if (plan.p.store_tma) {
+    } else if (plan.p.store_tma && !plan.kcluster) {
       const bool f32 = q.out == FACT_OUT_F32;
       const uint64_t sC = q.batch > 1 ? (uint64_t)q.strideC : (uint64_t)q.ldc * (uint64_t)q.M;
       st = encode_map(h, &tm[2], q.C, (uint64_t)q.N_out, (uint64_t)q.M, batch_dim, (uint64_t)q.ldc,
@@ -955,7 +1072,8 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
     }
     const int epi = split ? (int)kEpiPartial : (int)q.epi;
     const bool two = plan.cfg.cta_group == 2;
-    if (q.groups > 0 && plan.dynamic) st = two ? launch_epi_dp<2, true, true>(h, epi, plan, tm, stream)
+    if (plan.kcluster) st = launch_kcluster(h, epi, plan, tm, stream);
+    else if (q.groups > 0 && plan.dynamic) st = two ? launch_epi_dp<2, true, true>(h, epi, plan, tm, stream)
                                                : launch_epi_dp<1, true, true>(h, epi, plan, tm, stream);
     else if (q.groups > 0) st = two ? launch_epi_dp<2, true, false>(h, epi, plan, tm, stream)
                                     : launch_epi_dp<1, true, false>(h, epi, plan, tm, stream);
@@ -1579,6 +1697,18 @@ fact_status_t fact_tune_ex(fact_handle_t h, fact_op_t op, int64_t batch, int64_t
         }
     }
   }
+  // K slices as a cluster (schedule 3): up to two waves of clusters of 2 / 4 / 8 CTAs (make_plan refuses what the
+  // kernel cannot run: gated or row-softmax epilogues, 8-bit operands, groups)
+  for (int sl = 2; sl <= 8; sl *= 2)
+    for (int tn = 64; tn <= 256; tn *= 2) {
+      if (tn % (32 * sl) || !tile_ok(q, tn, 1) || k_blocks < 2 * sl) continue;
+      const int smax = max_stages_for(q, tn, 1);
+      if (smax < 2) continue;
+      const long long tiles = batch * ((M + 127) / 128) * ((N + tn - 1) / tn);
+      if (tiles > 2LL * kc_max_clusters(h, sl)) continue;
+      fact_config_t c = {128, tn, q.k_elems(), smax, 1, 0, sl, 0, 3};
+      cands.push_back(c);
+    }
   // Time `c` over `n` launches (per launch, ms); a negative result means the candidate failed.  Warm L2: the launches
   // run back to back between one event pair.  Cold L2: a buffer twice the size of L2 is overwritten before each
   // launch and every launch has an event pair of its own (what a benchmark that flushes L2 between launches sees).

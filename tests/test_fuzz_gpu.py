@@ -1,7 +1,8 @@
 """Seeded sweep over shapes x epilogues x kernel configurations (Section 4.2: every candidate is verified).
 
 Each case draws a ragged problem size, an epilogue, a layout, an output type and a configuration from the space the
-tuner sweeps (tile width, stage count, CTA pairs, raster group, K slices or stream-K, store mode, schedule), runs it
+tuner sweeps (tile width, stage count, CTA pairs, raster group, K slices or stream-K, store mode, schedule -- static,
+dynamic, or the K slices of a tile as one cluster), runs it
 through the C ABI and compares the whole output with the FP64 oracle.  The inputs are small integers, so every
 product and every partial sum is exact in FP32 whatever the order of the additions: NONE / BIAS / ReLU / residual
 outputs must match the oracle bit for bit for every schedule, GELU and SiLU go through the gates.  A combination
@@ -45,6 +46,12 @@ def _draw(i):
     cfg["split_k"] = int(rng.choice([1, 1, 1, 2, 3, 5, -1, -2]))
     cfg["store_mode"] = int(rng.choice([0, 0, 1, 2, 3]))
     cfg["schedule"] = int(rng.choice([0, 1, 2]))
+    if rng.integers(0, 4) == 0:
+        # K slices as a cluster, added up through distributed shared memory
+        cfg = {"cta_group": 1, "tile_n": int(rng.choice([64, 128, 256])), "split_k": int(rng.choice([2, 4, 8])),
+               "schedule": 3}
+        if rng.integers(0, 2):
+            cfg["stages"] = int(rng.integers(2, 5))
     return epi, layout, out, M, N, K, cfg
 
 

@@ -294,6 +294,38 @@ def test_few_slices_take_the_wide_reduction_and_keep_every_bit(h, out):
                     assert (big[:, N:] == -7.0).all(), "wrote outside the N columns"
 
 
+@pytest.mark.parametrize("layout", ["KN", "NK"])
+@pytest.mark.parametrize("slices,tile_n", [(2, 64), (2, 128), (4, 128), (2, 256), (4, 256), (8, 256)])
+def test_k_slices_as_a_cluster_are_exact_and_equal_the_workspace_reduction(h, layout, slices, tile_n):
+    """schedule 3: the K slices of a tile run as one cluster and are added up through distributed shared memory, in
+    the order of the workspace reduction.  Integer inputs: bit-exact against the oracle, for every epilogue the
+    schedule serves, several tiles per cluster (more tiles than clusters), ragged M, N and K, FP32 and BF16 outputs;
+    random inputs: the same bits as the same number of slices through the workspace."""
+    from paper_2604_26666_b200.binding import FactError
+
+    kc = {"cta_group": 1, "tile_n": tile_n, "split_k": slices, "schedule": 3}
+    for (M, N, K, epi, out) in [(200, 520, 1096, "BIAS_RESIDUAL", "bf16"), (130, 264, 2048, "BIAS_RELU", "f32"),
+                                (128 * 40 + 8, 512, 1024, "NONE", "bf16")]:
+        case = mk(f"kc_{slices}_{tile_n}_{epi}", M, N, K, epilogue=epi, layout=layout, out=out)
+        bit_exact(h, case, small_int_inputs(case, 31, lo=-2, hi=2), cfg=kc)
+    case = mk(f"kc_rand_{slices}_{tile_n}", 300, 520, 4096, epilogue="BIAS_GELU_TANH", layout=layout)
+    ins = wl.make_inputs(case)
+    check_case(h, case, ins=ins, cfg=kc)
+    a = run_gpu(h, ins, case, cfg=kc)
+    b = run_gpu(h, ins, case, cfg={"cta_group": 1, "tile_n": tile_n, "split_k": slices})
+    torch.cuda.synchronize()
+    assert torch.equal(a, b), "cluster and workspace reductions of the same slices differ"
+    assert h.workspace_bytes("linear", 1, 300, 520, 4096, "BIAS_GELU_TANH", layout, torch.bfloat16, kc) == 0
+    # what the schedule does not serve is refused before any launch
+    gate = mk("kc_gate", 128, 256, 1024, epilogue="SILU_GATE", layout=layout)
+    with pytest.raises(FactError):
+        run_gpu(h, wl.make_inputs(gate), gate, cfg=kc)
+    for bad in ({"cta_group": 2}, {"split_k": 3}, {"tile_n": 96}):
+        with pytest.raises(FactError):
+            run_gpu(h, ins, case, cfg={**kc, **bad})
+    assert h.device_status() == 0
+
+
 def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
     """The library's own choice for an untuned product of few tiles and long K is K slices (Section 4.2, Action 2:
     the grid-level policy is a design choice) -- with the workspace the binding brings; the same call through the C
@@ -305,7 +337,8 @@ def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
     case = mk("few_tiles_long_k", 256, 512, 16384, op="gemm", layout="NK")
     cfg = h.get_config("gemm", 1, case.M, case.N, case.K, "NONE", "NK", torch.bfloat16).as_dict()
     assert cfg["split_k"] > 1, cfg
-    assert h.workspace_bytes("gemm", 1, case.M, case.N, case.K, "NONE", "NK", torch.bfloat16) > 0
+    # (slices through the workspace, or -- schedule 3 -- as a cluster, which needs none)
+    assert (h.workspace_bytes("gemm", 1, case.M, case.N, case.K, "NONE", "NK", torch.bfloat16) > 0) != (cfg["schedule"] == 3)
     ins = wl.make_inputs(case)
     check_case(h, case, ins=ins)
     # an explicit single slice is respected, and a short K is never sliced
