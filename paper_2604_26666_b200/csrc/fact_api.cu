@@ -1017,7 +1017,10 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
       plan.p.store_tma = 1;  // partials always go through the staged path: the workspace layout is the library's
       plan.p.r_tma = 0;
       plan.p.ws = reinterpret_cast<const float*>(ws);
-      plan.p.fused_reduce = 1;  // the grid never exceeds the SM count, so the barrier in the kernel's tail is safe
+      // the reduction runs in the kernel's tail (the grid never exceeds the SM count, so the barrier there is safe)
+      // unless the slices are few enough for the wide walk of the stand-alone reduction kernel
+      plan.p.fused_reduce = !(plan.cfg.split_k <= kReduceWideSlices && q.epi != FACT_EPI_SILU_GATE &&
+                              (plan.p.ws_ld & 7) == 0);
       plan.p.reduce_epi = (int)q.epi;
     }
     if (h->debug_flags & 256) {  // the all-CTA span stamps start from "no start yet" / "no end yet"
