@@ -193,7 +193,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tune", action="store_true", help="run the on-device tuner for every shape first")
     ap.add_argument("--shape", default=None,
-                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped`, `normfold` or `blocks`): "
+                    help="time only this benchmark shape (a name from the `shapes` table, `all`, `attention`, `fp8`, `grouped`, `normfold`, `blocks` or `untuned`): "
                          "--warmup/--steps launches, no side reference; the small command used for profiling")
     ap.add_argument("--layout", default="NK", choices=["NK", "KN"], help="weight layout of the config 4/5 linears")
     ap.add_argument("--no-trains", action="store_true",
@@ -239,6 +239,11 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
+        if args.shape == "untuned":
+            print(json.dumps({"untuned": untuned_table(h, dev, stream, flush_l2, warm=args.warmup, iters=max(args.steps, 9)),
+                              "gpu_launches": h.launch_count()}))
+            h.close()
+            return 0
         rows = [] if args.shape in ("attention", "blocks", "fp8", "grouped", "normfold") else per_shape_table(
             h, dev, stream, flush_l2, peaks, args.tune, names=names, warm=args.warmup, iters=args.steps,
             side_ref=False, layout=args.layout, trains=not args.no_trains)
@@ -613,6 +618,52 @@ def per_shape_table(h, dev, stream, flush_l2, peaks, tune, names=None, warm=5, i
             "roofline_frac_single_launch": max(t_tensor, t_hbm) / med,
         })
         rows.append(row)
+        del X, W, out
+    return rows
+
+
+UNTUNED_SHAPES = [(1024, 1024, 1024), (2048, 2048, 2048), (2048, 8192, 1024), (8192, 1024, 4096), (16, 4096, 4096),
+                  (64, 8192, 8192), (128, 14336, 4096), (256, 4096, 14336), (1000, 1000, 1000), (4096, 128, 4096),
+                  (8192, 64, 8192), (1536, 1536, 6144), (512, 512, 8192), (512, 2048, 16384), (1024, 1024, 8192),
+                  (256, 256, 32768), (128, 4096, 8192), (2048, 512, 4096), (768, 768, 3072), (32, 14336, 4096),
+                  (4096, 4096, 512), (8192, 8192, 128)]
+
+
+def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9):
+    """Shapes the tuner's table does not know (`--shape untuned`): the library's own choice of configuration (its cost
+    model: data-parallel tiles, K slices through a workspace, or K slices as a cluster), the same call held to one
+    slice, and `torch.matmul`; single launches after an L2 flush, mean of the middle of `iters` runs."""
+    import torch
+
+    def time_it(fn):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize(dev)
+            ts.append(a.elapsed_time(b) * 1e3)
+        ts.sort()
+        mid = ts[len(ts) // 4: len(ts) - len(ts) // 4]
+        return sum(mid) / len(mid)
+
+    rows = []
+    g = torch.Generator(device="cpu").manual_seed(77)
+    for (M, N, K) in UNTUNED_SHAPES:
+        X = torch.randn(M, K, generator=g).to(torch.bfloat16).to(dev)
+        W = (torch.randn(N, K, generator=g) * K ** -0.5).to(torch.bfloat16).to(dev)
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        cfg = h.get_config("gemm", 1, M, N, K, "NONE", "NK", torch.bfloat16).as_dict()
+        rows.append({
+            "M": M, "N": N, "K": K, "config": cfg,
+            "us": time_it(lambda: h.gemm(X, W, layout="NK", out=out)),
+            "us_one_slice": time_it(lambda: h.gemm(X, W, layout="NK", out=out, cfg={"split_k": 1})),
+            "torch_matmul_us": time_it(lambda: torch.matmul(X, W.t(), out=out)),
+        })
         del X, W, out
     return rows
 
