@@ -151,7 +151,7 @@ typedef enum {
  *                3 = the K slices of a tile as one thread-block cluster (the K-sliced regime of Section 5.2,
  *                Problem 6, for products of few tiles and long K): split_k = 2, 4 or 8 CTAs share a 128-row tile
  *                (tile_m 128, cta_group 1, tile_n a multiple of 32 * split_k), each multiplies its slice of K with
- *                its own loads and its own accumulator -- no operand is loaded twice, every CTA issues only its own plain loads -- and
+ *                its own plain loads and its own accumulator -- no operand is loaded twice -- and
  *                the slices are added up through distributed shared memory: CTA r sends block j of its
  *                accumulator's columns to CTA j, which adds the blocks in the order of the workspace reduction
  *                (same bits as the same split_k through a workspace), applies the epilogue and stores.  No

@@ -3,8 +3,8 @@
 // For products of few tiles and long K (Section 5.2, Problem 6: the K-sliced / stream-K regime).  A cluster of S CTAs
 // (S = 2, 4 or 8) owns one 128 x tile_n output tile at a time; CTA r of the cluster multiplies the r-th slice of K
 // with its own TMA ring and its own FP32 accumulator in tensor memory -- the slices share no operand, so nothing is
-// loaded twice and every CTA issues only its own plain loads.  When the S accumulators are complete, CTA r sends the j-th block of
-// tile_n / S columns of its accumulator to CTA j (plain vector stores to the peer's shared memory), CTA j adds the
+// loaded twice and every CTA issues only its own plain loads.  When the S accumulators are complete, CTA r sends the
+// j-th block of tile_n / S columns of its accumulator to CTA j (vector stores to the peer's shared memory), CTA j adds the
 // S blocks it received in a fixed order, applies the epilogue and stores its columns of the tile.  No partial planes
 // in global memory, no workspace, no grid-wide barrier: the clusters of a launch do not depend on one another, so
 // the grid may be larger than what is resident.
