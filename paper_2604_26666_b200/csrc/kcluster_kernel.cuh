@@ -21,10 +21,13 @@
 namespace fact {
 
 constexpr int kKcThreads = 192;
-constexpr int kKcPad = 4;  // floats of padding per received row: consecutive rows start 4 banks apart
 
+// What a CTA receives: from each of the S senders its block of tile_n / S columns of 128 rows, kept as
+// [sender][group of 4 columns][row] 16-byte pieces -- the 32 lanes of a warp (32 rows) write, and later read, 512
+// contiguous bytes per instruction.  (Row-major blocks made every lane's 16 bytes a transaction of its own: 1000-1300
+// cycles per 32-column piece sent instead of 300.)
 __host__ __device__ constexpr uint32_t kc_exchange_bytes(int tile_n, int slices) {
-  return (uint32_t)slices * kTileM * (uint32_t)(tile_n / slices + kKcPad) * 4u;
+  return (uint32_t)tile_n * kTileM * 4u + 0u * (uint32_t)slices;
 }
 __host__ __device__ constexpr uint32_t kc_smem_bytes(int tile_n, int slices, int stages, uint32_t stage_bytes) {
   const uint32_t ring = (uint32_t)stages * stage_bytes, xch = kc_exchange_bytes(tile_n, slices);
@@ -93,6 +96,13 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder_p;
   ptx::grid_dependency_wait();  // set-up above overlaps the tail of the kernel before; global memory from here on
+  // With debug bit 256 the first CTA stamps its first tile's milestones, in SM cycles from here (status[2..17], read by
+  // fact_last_kernel_profile): [0] whole kernel, [1] the same in nanoseconds, [2] first operand stage ready,
+  // [3] accumulator complete, [4] every peer's complete, [5] blocks sent, [6] blocks received, [7] tile stored.
+  const bool prof = (p.debug & 256) && blockIdx.x == 0;
+  const long long t_go = clock64();
+  const unsigned long long ns_go = prof ? ptx::globaltimer_ns() : 0ull;
+  long long* const prof_c = reinterpret_cast<long long*>(p.status + 2);
 
   const int cluster_id = (int)(blockIdx.x / (unsigned)S);
   const int n_clusters = (int)(gridDim.x / (unsigned)S);
@@ -157,6 +167,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
           ok = false;
           break;
         }
+        if (prof && it == 0 && kb == w.kb_begin && lane == 0) prof_c[2] = clock64() - t_go;
         ptx::tc_fence_after();
         const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
         const uint32_t sb = sa + kStageBytesA;
@@ -182,9 +193,9 @@ __global__ void __launch_bounds__(kKcThreads, 1)
     // ------------------------------------------------------------ exchange and epilogue: one accumulator row per thread
     const int q = warp & 3;  // the TMEM lane quarter this warp may read
     const int row_in_tile = q * 32 + lane;
-    const uint32_t row_stride = (uint32_t)(cb + kKcPad) * 4u;                   // bytes between received rows
-    const uint32_t block_stride = (uint32_t)kTileM * row_stride;                // ... between the blocks of two senders
-    const uint32_t my_slot = smem_base + rank * block_stride + (uint32_t)row_in_tile * row_stride;  // where a peer keeps MY block
+    const uint32_t chunk_stride = (uint32_t)kTileM * 16u;                   // bytes between two 4-column groups
+    const uint32_t block_stride = (uint32_t)(cb >> 2) * chunk_stride;       // ... between the blocks of two senders
+    const uint32_t my_slot = smem_base + rank * block_stride + (uint32_t)row_in_tile * 16u;  // where a peer keeps MY block
     const bool c_vec = p.c_vec != 0;
     bool ok = true;
     int it = 0;
@@ -198,40 +209,62 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         break;
       }
       ptx::tc_fence_after();
+      const bool stamp = prof && it == 0 && warp == 2 && lane == 0;
+      if (stamp) prof_c[3] = clock64() - t_go;
       if (warp == 2) {
-        if (lane < S) ptx::mbar_arrive_cluster(ptx::mapa(peers_bar, (uint32_t)lane));
+        // (a relaxed arrival: it publishes no data, it says that this CTA's products have stopped reading its ring,
+        // which this thread has just observed through the accumulator's barrier)
+        if (lane < S) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(peers_bar, (uint32_t)lane));
         __syncwarp();
       }
       if (!wait_bar_cluster(peers_bar, par, abort_p, p.status)) {
         ok = false;
         break;
       }
+      if (stamp) prof_c[4] = clock64() - t_go;
       // ---- send: 32 accumulator columns at a time, starting with the block of the next CTA round the cluster so
       // that the S senders do not all write to the same receiver at once
       const int pieces = p.tile_n >> 5;
       const int per_owner = cb >> 5;
-      for (int i = 0; i < pieces; ++i) {
+      auto piece_of = [&](int i) {
         int pc = i + ((int)rank + 1) * per_owner;
         if (pc >= pieces) pc -= pieces;
         if (pc >= pieces) pc -= pieces;  // ((rank + 1) * per_owner may equal pieces)
+        return pc;
+      };
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      auto send = [&](int pc, const uint32_t (&v)[32]) {
         const int owner = pc / per_owner;
         const int col = (pc - owner * per_owner) << 5;  // first column inside the owner's block
-        uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(pc << 5), v);
-        ptx::tmem_wait_ld();
-        const uint32_t dst = ptx::mapa(my_slot + (uint32_t)col * 4u, (uint32_t)owner);
+        const uint32_t dst = ptx::mapa(my_slot + (uint32_t)(col >> 2) * chunk_stride, (uint32_t)owner);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) st_shared_cluster_v4(dst + 16u * (uint32_t)j, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        for (int j = 0; j < 8; ++j)
+          st_shared_cluster_v4(dst + chunk_stride * (uint32_t)j, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      };
+      // two pieces per trip: the second piece's tensor-memory load is in flight while the first is sent
+      for (int i = 0; i < pieces; i += 2) {
+        uint32_t v0[32], v1[32];
+        const int pc0 = piece_of(i), pc1 = i + 1 < pieces ? piece_of(i + 1) : 0;
+        ptx::tmem_ld_32x32b_x32(t_row + (uint32_t)(pc0 << 5), v0);
+        ptx::tmem_wait_ld();
+        if (i + 1 < pieces) ptx::tmem_ld_32x32b_x32(t_row + (uint32_t)(pc1 << 5), v1);
+        send(pc0, v0);
+        if (i + 1 < pieces) {
+          ptx::tmem_wait_ld();
+          send(pc1, v1);
+        }
       }
       ptx::tc_fence_before();
       __syncwarp();  // every lane's stores are ordered before lane 0's releasing arrivals
       if (lane < S) ptx::mbar_arrive_cluster(ptx::mapa(xfull_bar, (uint32_t)lane));
+      if (stamp) prof_c[5] = clock64() - t_go;
       // ---- receive: add the S blocks of this CTA's columns in the order of the workspace reduction, apply the
       // epilogue, store
       if (!wait_bar_cluster(xfull_bar, par, abort_p, p.status)) {
         ok = false;
         break;
       }
+      if (stamp) prof_c[6] = clock64() - t_go;
       const int row = w.tm * kTileM + row_in_tile;
       const bool row_ok = row < p.M;
       const int n_block0 = w.tn * p.tile_n + (int)rank * cb;
@@ -239,7 +272,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       char* c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
       const __nv_bfloat16* r_row = nullptr;
       if constexpr (EPI == kEpiBiasResidual) r_row = p.R + (long long)w.b * p.strideR + (long long)row * p.ldr;
-      const uint32_t mine = smem_base + (uint32_t)row_in_tile * row_stride;
+      const uint32_t mine = smem_base + (uint32_t)row_in_tile * 16u;
       for (int c = 0; c < cb; c += 8) {
         const int n = n_block0 + c;
         const int nvalid = min(8, p.N_out - n);
@@ -252,8 +285,8 @@ __global__ void __launch_bounds__(kKcThreads, 1)
 #pragma unroll
         for (int s = 0; s < 8; ++s)
           if (s < S) {
-            const uint4 lo = ptx::ld_shared_v4(mine + (uint32_t)s * block_stride + (uint32_t)c * 4u);
-            const uint4 hi = ptx::ld_shared_v4(mine + (uint32_t)s * block_stride + (uint32_t)c * 4u + 16u);
+            const uint4 lo = ptx::ld_shared_v4(mine + (uint32_t)s * block_stride + (uint32_t)(c >> 2) * chunk_stride);
+            const uint4 hi = ptx::ld_shared_v4(mine + (uint32_t)s * block_stride + (uint32_t)((c >> 2) + 1) * chunk_stride);
             const int a = s & 3;
             acc[a][0] += __uint_as_float(lo.x); acc[a][1] += __uint_as_float(lo.y);
             acc[a][2] += __uint_as_float(lo.z); acc[a][3] += __uint_as_float(lo.w);
@@ -282,6 +315,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(xdone_bar);
+      if (stamp) prof_c[7] = clock64() - t_go;
     }
     __syncwarp();
   }
@@ -297,6 +331,10 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   __syncthreads();
   ptx::cluster_arrive();  // no CTA leaves while a peer may still write to its shared memory or arrive on its barriers
   ptx::cluster_wait();
+  if (prof && threadIdx.x == 0) {
+    prof_c[0] = clock64() - t_go;
+    prof_c[1] = (long long)(ptx::globaltimer_ns() - ns_go);
+  }
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc<1>(tmem_base, p.tmem_cols);
