@@ -598,6 +598,10 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * nanoseconds of the first CTA, [2] a tag of the first device-side wait that gave up (0 if none: barrier index,
  * warp << 8, CTA << 16), [3] cycles the first softmax warp of tile 0 waited for scores, [4] key blocks it
  * processed, [6] cycles it spent writing finished tiles out, [7] work items of that CTA.
+ * After a launch with K slices as a cluster (schedule 3) they are the milestones of the first CTA's first tile, in
+ * cycles from the moment the kernel may touch global memory: [0] end of the kernel and [1] the same in nanoseconds,
+ * [2] first operand stage ready, [3] accumulator complete, [4] every peer's accumulator complete, [5] column blocks
+ * sent, [6] column blocks received, [7] tile stored.
  * FACT_DEBUG_FLAGS is read once, by fact_create.  The library as built by default honours two bits, neither of
  * which changes a result: 256 (these counters) and 2048 (no downward K walk on every second tile).  The
  * work-skipping experiment switches (1, 2, 4: the GEMM kernel's loads, products, stores; 8, 64, 128: the attention
