@@ -239,8 +239,13 @@ def main():
     # (the handle has already loaded the package's tuned table for the benchmark shapes)
     if args.shape is not None:
         names = None if args.shape == "all" else args.shape.split(",")
-        if args.shape == "untuned":
-            print(json.dumps({"untuned": untuned_table(h, dev, stream, flush_l2, warm=args.warmup, iters=max(args.steps, 9)),
+        if args.shape == "untuned" or args.shape.startswith("untuned:"):
+            # `untuned:1024x1024x8192[,MxNxK...]` times only those shapes (the small command used for profiling)
+            only = None
+            if ":" in args.shape:
+                only = [tuple(int(v) for v in t.split("x")) for t in args.shape.split(":", 1)[1].split(",")]
+            print(json.dumps({"untuned": untuned_table(h, dev, stream, flush_l2, warm=args.warmup, iters=max(args.steps, 3),
+                                                       shapes=only),
                               "gpu_launches": h.launch_count()}))
             h.close()
             return 0
@@ -629,7 +634,7 @@ UNTUNED_SHAPES = [(1024, 1024, 1024), (2048, 2048, 2048), (2048, 8192, 1024), (8
                   (4096, 4096, 512), (8192, 8192, 128)]
 
 
-def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9):
+def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9, shapes=None):
     """Shapes the tuner's table does not know (`--shape untuned`): the library's own choice of configuration (its cost
     model: data-parallel tiles, K slices through a workspace, or K slices as a cluster), the same call held to one
     slice, and `torch.matmul`; single launches after an L2 flush, mean of the middle of `iters` runs."""
@@ -653,7 +658,7 @@ def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9):
 
     rows = []
     g = torch.Generator(device="cpu").manual_seed(77)
-    for (M, N, K) in UNTUNED_SHAPES:
+    for (M, N, K) in (shapes or UNTUNED_SHAPES):
         X = torch.randn(M, K, generator=g).to(torch.bfloat16).to(dev)
         W = (torch.randn(N, K, generator=g) * K ** -0.5).to(torch.bfloat16).to(dev)
         out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
