@@ -326,6 +326,16 @@ def test_k_slices_as_a_cluster_are_exact_and_equal_the_workspace_reduction(h, la
     assert h.device_status() == 0
 
 
+def test_k_slices_as_a_cluster_serve_the_batched_and_the_sliced_entry_points(h):
+    kc = {"cta_group": 1, "tile_n": 128, "split_k": 4, "schedule": 3}
+    for layout in ("KN", "NK"):
+        case = mk("kc_batched", 200, 264, 1536, op="gemm_batched", batch=5, layout=layout, out="f32")
+        bit_exact(h, case, small_int_inputs(case, 41, lo=-2, hi=2), cfg=kc)
+        case = mk("kc_splitk_op", 256, 256, 8192 + 64, op="gemm_splitk", layout=layout, out="f32")
+        bit_exact(h, case, small_int_inputs(case, 42, lo=-2, hi=2), cfg=kc, splits=4)
+    assert h.device_status() == 0
+
+
 def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
     """The library's own choice for an untuned product of few tiles and long K is K slices (Section 4.2, Action 2:
     the grid-level policy is a design choice) -- with the workspace the binding brings; the same call through the C
