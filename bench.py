@@ -245,7 +245,7 @@ def main():
             if ":" in args.shape:
                 only = [tuple(int(v) for v in t.split("x")) for t in args.shape.split(":", 1)[1].split(",")]
             print(json.dumps({"untuned": untuned_table(h, dev, stream, flush_l2, warm=args.warmup, iters=max(args.steps, 3),
-                                                       shapes=only),
+                                                       shapes=only, tune=args.tune),
                               "gpu_launches": h.launch_count()}))
             h.close()
             return 0
@@ -634,7 +634,7 @@ UNTUNED_SHAPES = [(1024, 1024, 1024), (2048, 2048, 2048), (2048, 8192, 1024), (8
                   (4096, 4096, 512), (8192, 8192, 128)]
 
 
-def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9, shapes=None):
+def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9, shapes=None, tune=False):
     """Shapes the tuner's table does not know (`--shape untuned`): the library's own choice of configuration (its cost
     model: data-parallel tiles, K slices through a workspace, or K slices as a cluster), the same call held to one
     slice, and `torch.matmul`; single launches after an L2 flush, mean of the middle of `iters` runs."""
@@ -669,6 +669,10 @@ def untuned_table(h, dev, stream, flush_l2, warm=3, iters=9, shapes=None):
             "us_one_slice": time_it(lambda: h.gemm(X, W, layout="NK", out=out, cfg={"split_k": 1})),
             "torch_matmul_us": time_it(lambda: torch.matmul(X, W.t(), out=out)),
         })
+        if tune:  # (--tune: what the on-device tuner finds for the shape, timed the same way)
+            best, _, n_tried = h.tune("gemm", X, W, layout="NK", out=out, cold_l2=True)
+            rows[-1].update({"tuned_config": best.as_dict(), "tuned_candidates": n_tried,
+                             "us_tuned": time_it(lambda: h.gemm(X, W, layout="NK", out=out))})
         del X, W, out
     return rows
 
