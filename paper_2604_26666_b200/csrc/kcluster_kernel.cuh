@@ -110,6 +110,9 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
     return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_p, p.status)) != 0;
   };
+  auto wait_all_cluster = [&](uint32_t bar, uint32_t parity) -> bool {  // ... for barriers the peers arrive on
+    return __all_sync(0xffffffffu, wait_bar_cluster(bar, parity, abort_p, p.status)) != 0;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -204,7 +207,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       const uint32_t par = (uint32_t)it & 1u;
       // ---- this CTA's slice is complete: tell every CTA of the cluster, then wait until all of them are (their
       // rings are then idle and may receive blocks)
-      if (!wait_bar(accf_bar, par, abort_p, p.status)) {
+      if (!wait_all(accf_bar, par)) {  // (every verdict is warp-uniform: what follows is warp-wide)
         ok = false;
         break;
       }
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         if (lane < S) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(peers_bar, (uint32_t)lane));
         __syncwarp();
       }
-      if (!wait_bar_cluster(peers_bar, par, abort_p, p.status)) {
+      if (!wait_all_cluster(peers_bar, par)) {
         ok = false;
         break;
       }
@@ -260,7 +263,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       if (stamp) prof_c[5] = clock64() - t_go;
       // ---- receive: add the S blocks of this CTA's columns in the order of the workspace reduction, apply the
       // epilogue, store
-      if (!wait_bar_cluster(xfull_bar, par, abort_p, p.status)) {
+      if (!wait_all_cluster(xfull_bar, par)) {
         ok = false;
         break;
       }
