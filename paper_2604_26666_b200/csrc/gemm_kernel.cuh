@@ -1207,7 +1207,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
             // ---- a later piece of a tile another group finishes: park the raw FP32 accumulator in this CTA's
             // scratch tile.  Layout [piece][16-byte word j of the thread's 32 columns][row]: consecutive lanes
             // write consecutive 16-byte words, and the finishing warp reads them back the same way.
-            if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+            if (!wait_all(accf_bar(acc), acc_phase)) {  // (a warp-uniform verdict: what follows is warp-wide)
               ok = false;
               break;
             }
@@ -1365,7 +1365,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
           }
         };
         long long tw = prof ? clock64() : 0;
-        if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+        if (!wait_all(accf_bar(acc), acc_phase)) {  // (a warp-uniform verdict: what follows is warp-wide)
           ok = false;
           break;
         }
@@ -1432,7 +1432,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
           }
           if (use_r) {
             if (r_next <= gc && issue_residual(ci, gc)) r_next = gc + 1;
-            if (!wait_bar(res_bar(e, (int)(gc % bufs)), (gc / bufs) & 1u, abort_p, p.status)) {
+            if (!wait_all(res_bar(e, (int)(gc % bufs)), (gc / bufs) & 1u)) {
               ok = false;
               break;
             }
@@ -1626,7 +1626,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
       UnitWalk<false, GROUPED, DYN, CG> walk(p, unit0, unit_stride, sched);  // (stream-K always stores through the staged path)
       WorkUnit w;
       while (ok && walk.next(p, w)) {
-        if (!wait_bar(accf_bar(acc), acc_phase, abort_p, p.status)) {
+        if (!wait_all(accf_bar(acc), acc_phase)) {  // (a warp-uniform verdict: what follows is warp-wide)
           ok = false;
           break;
         }
@@ -1655,7 +1655,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
             // (two barriers in turn: the peer may arrive for the next exchange before this warp has seen this one
             // complete, which a single one-bit phase could not tell from "not yet")
             if (lane == 0) ptx::mbar_arrive(res_bar(e_peer, (int)(xch_count & 1u)));
-            if (!wait_bar(res_bar(e, (int)(xch_count & 1u)), (xch_count >> 1) & 1u, abort_p, p.status)) return false;
+            if (!wait_all(res_bar(e, (int)(xch_count & 1u)), (xch_count >> 1) & 1u)) return false;
             asm volatile("ld.shared.f32 %0, [%1];" : "=f"(theirs) : "r"(peer_slots + slot) : "memory");
             ++xch_count;
             return true;
