@@ -336,6 +336,34 @@ def test_k_slices_as_a_cluster_serve_the_batched_and_the_sliced_entry_points(h):
     assert h.device_status() == 0
 
 
+def test_k_slices_as_a_cluster_in_a_cuda_graph_and_back_to_back(h):
+    """Cluster launches can be captured and replayed, and launches that follow one another on a stream (each may move
+    onto the SMs while its predecessor's last CTAs leave) -- of the cluster kernel and of the persistent kernel in
+    turn -- give the same bits every time."""
+    case = mk("kc_graph", 384, 512, 4096, epilogue="BIAS_RELU", layout="NK")
+    ins = wl.make_inputs(case)
+    X, W, b = ins.X.cuda(), ins.W.cuda(), ins.bias.cuda()
+    kc = {"cta_group": 1, "tile_n": 128, "split_k": 4, "schedule": 3}
+    first_kc = h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", cfg=kc)
+    first_dp = h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", cfg={"split_k": 1})
+    torch.cuda.synchronize()
+    out_kc, out_dp = torch.empty_like(first_kc), torch.empty_like(first_dp)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream("cuda:0")):
+        for _ in range(3):
+            h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", out=out_kc, cfg=kc)
+            h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", out=out_dp, cfg={"split_k": 1})
+    for _ in range(3):
+        out_kc.zero_()
+        out_dp.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out_kc, first_kc) and torch.equal(out_dp, first_dp)
+    assert h.device_status() == 0
+    c, t = gates(oracle_for(ins, case), to_f64(out_kc), "bf16", case.epilogue)
+    assert c <= 1 and t <= 1, (c, t)
+
+
 def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
     """The library's own choice for an untuned product of few tiles and long K is K slices (Section 4.2, Action 2:
     the grid-level policy is a design choice) -- with the workspace the binding brings; the same call through the C
