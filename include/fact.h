@@ -127,7 +127,8 @@ typedef enum {
  *                (whole waves, K == 0, an output the staged store cannot write) the call is data-parallel.
  *                Stream-K calls through one handle must be stream-ordered with respect to each other (they share
  *                the handle's flags) and must not share a workspace while they overlap.
- *                0 (the library's choice) is one slice, except for an untuned fact_gemm / fact_linear whose tiles
+ *                0 (the library's choice) is one slice, except for an untuned fact_gemm / fact_linear (and for
+ *                fact_gemm_splitk called with splits = 0, whose choice is always the library's) whose tiles
  *                are few and whose K is long (say 256 x 4096 x 14336): there the library's cost model may take
  *                the K slices that fill the SMs in one wave, if the call brings the workspace that
  *                fact_workspace_bytes reports for it -- without it the same call runs in one slice, like a table

@@ -346,7 +346,8 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
   // through L2): a 256 x 4096 x 14336 product is 16 wide tiles of 224 k-blocks, or four times as many of 56.
   const int k_blocks_all = std::max(1, (int)((q.K + q.k_elems() - 1) / q.k_elems()));
   const bool gate_epi = q.epi == FACT_EPI_SILU_GATE;
-  const bool may_slice = c.split_k == 0 && (q.op == FACT_OP_GEMM || q.op == FACT_OP_LINEAR) && q.batch == 1 &&
+  const bool may_slice = c.split_k == 0 &&
+                         (q.op == FACT_OP_GEMM || q.op == FACT_OP_LINEAR || q.op == FACT_OP_GEMM_SPLITK) && q.batch == 1 &&
                          q.groups == 0 && !q.fp8 && !q.stats_out && !q.norm && q.epi != FACT_EPI_BIAS_SOFTMAX;
   auto model = [&](int cg, int tn, int* slices_out, bool calibrated = false) -> double {
     const int out_cols = q.epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
