@@ -151,10 +151,11 @@ typedef enum {
  *                the static schedule when all tiles fit one wave.
  *                3 = the K slices of a tile as one thread-block cluster (the K-sliced regime of Section 5.2,
  *                Problem 6, for products of few tiles and long K): split_k = 2, 4 or 8 CTAs share a 128-row tile
- *                (tile_m 128, cta_group 1, tile_n a multiple of 32 * split_k), each multiplies its slice of K with
- *                its own plain loads and its own accumulator -- no operand is loaded twice -- and
- *                the slices are added up through distributed shared memory: CTA r sends block j of its
- *                accumulator's columns to CTA j, which adds the blocks in the order of the workspace reduction
+ *                (tile_m 128, cta_group 1), or split_k = 2 or 4 CTA pairs share a 256-row tile (tile_m 256,
+ *                cta_group 2; a cluster holds at most 8 CTAs); tile_n is a multiple of 32 * split_k.  Each slice
+ *                multiplies its part of K with its own plain loads and its own accumulator -- no operand is
+ *                loaded twice -- and the slices are added up through distributed shared memory: slice r sends
+ *                block j of its accumulator's columns to slice j, which adds the blocks in the order of the workspace reduction
  *                (same bits as the same split_k through a workspace), applies the epilogue and stores.  No
  *                workspace, no partial planes in global memory, no grid-wide barrier.  Column-wise epilogues on
  *                BF16 operands (not SILU_GATE, row softmax, 8-bit operands, groups, row sums or a folded

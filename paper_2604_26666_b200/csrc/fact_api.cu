@@ -104,7 +104,8 @@ struct fact_handle_s {
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
   std::bitset<192> configured_mask;  // kernels whose dynamic shared-memory limit was raised
-  int kc_clusters[3] = {0, 0, 0};    // clusters of 2 / 4 / 8 CTAs of the K-slice kernel the device holds at once
+  int kc_clusters[6] = {0, 0, 0, 0, 0, 0};  // clusters of 2 / 4 / 8 CTAs of the K-slice kernel (single CTAs, pairs) the
+                                            // device holds at once
   std::string last_error;        // text of the most recent CUDA failure
   int debug_flags = 0;           // FACT_DEBUG_FLAGS: diagnostics (256 cycle counters, 2048 no K serpentine); the
                                  // work-skipping experiment switches only in a -DFACT_EXPERIMENTS build
@@ -236,20 +237,21 @@ bool tile_ok(const Problem& q, int tile_n, int cg) {
 // for groups of n-tiles.
 // How many clusters of `slices` CTAs of the K-slice kernel are resident at once (a cluster needs its SMs inside one
 // GPC, so this is less than SMs / slices); asked of the runtime once per cluster size.
-int kc_max_clusters(fact_handle_t h, int slices) {
-  const int idx = slices == 2 ? 0 : (slices == 4 ? 1 : 2);
+int kc_max_clusters(fact_handle_t h, int slices, int cg = 1) {
+  const int ctas = slices * cg;  // CTAs per cluster: 2, 4 or 8
+  const int idx = (ctas == 2 ? 0 : (ctas == 4 ? 1 : 2)) + 3 * (cg - 1);
   if (h->kc_clusters[idx] == 0) {
     int n = 0, dev = -1;
     const bool switched = cudaGetDevice(&dev) == cudaSuccess && dev != h->device && cudaSetDevice(h->device) == cudaSuccess;
-    auto kern = fact_gemm_kcluster_kernel<kEpiNone>;
+    auto kern = cg == 2 ? fact_gemm_kcluster_kernel<kEpiNone, 2> : fact_gemm_kcluster_kernel<kEpiNone, 1>;
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof lc);
-    lc.gridDim = dim3((unsigned)(slices * h->sm_count), 1, 1);
+    lc.gridDim = dim3((unsigned)(ctas * h->sm_count), 1, 1);
     lc.blockDim = dim3((unsigned)kKcThreads, 1, 1);
     lc.dynamicSmemBytes = (size_t)kSmemBudget;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)slices;
+    attr[0].val.clusterDim.x = (unsigned)ctas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
@@ -257,7 +259,7 @@ int kc_max_clusters(fact_handle_t h, int slices) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
         cudaOccupancyMaxActiveClusters(&n, kern, &lc) != cudaSuccess || n <= 0) {
       cudaGetLastError();
-      n = std::max(1, (h->sm_count / slices) * 3 / 4);  // (what GPCs of 16 usable SMs out of 18 or 20 would hold)
+      n = std::max(1, (h->sm_count / ctas) * 3 / 4);  // (what GPCs of 16 usable SMs out of 18 or 20 would hold)
     }
     if (switched) cudaSetDevice(dev);
     h->kc_clusters[idx] = n;
@@ -407,32 +409,38 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
     }
     c.cta_group = best_cg;
     c.tile_n = best_tn;
-    // K slices as a cluster (schedule 3: no workspace, no grid barrier): one wave of clusters of 2 / 4 / 8 CTAs on
-    // 128-row tiles.  Per k-block 400 / 450 / 1000 cycles at 64 / 128 / 256 columns, never faster than the operands
-    // stream from DRAM, plus 10k cycles (13k at 256 columns) for the exchange, the epilogue and a cold start --
-    // fitted to 66 timed (shape, slices, width) combinations, within a few percent where the cluster schedule wins.
-    if (may_slice && c.schedule == 0 && !gate_epi && (user == nullptr || user->cta_group == 0 || user->cta_group == 1) &&
-        (user == nullptr || user->tile_n == 0) && (user == nullptr || user->tile_m == 0 || user->tile_m == 128)) {
+    // K slices as a cluster (schedule 3: no workspace, no grid barrier): one wave of clusters of at most 8 CTAs, the
+    // slices single CTAs on 128-row tiles or pairs on 256-row tiles.  Per k-block 400 / 450 / 1000 cycles at 64 / 128 /
+    // 256 columns (pairs: 400 / 400 / 880), never faster than the operands stream from DRAM, plus 10k cycles (13k at
+    // 256 columns) for the exchange, the epilogue and a cold start -- fitted to 66 timed (shape, slices, width)
+    // combinations of single CTAs, within a few percent where the cluster schedule wins; pairs timed on 19 shapes.
+    if (may_slice && c.schedule == 0 && !gate_epi && (user == nullptr || user->tile_n == 0)) {
       const double hbm = ((double)q.M + (double)Nw) * (double)q.K * 2.0 / 3686.0 * 1.15;
       double best_kc = 1e300;
-      int kc_s = 0, kc_tn = 0;
-      for (int sl = 2; sl <= 8; sl *= 2)
-        for (int tn = 64; tn <= 256; tn *= 2) {
-          if (tn % (32 * sl) || !tile_ok(q, tn, 1) || max_stages_for(q, tn, 1) < 2 || k_blocks_all < 4 * sl) continue;
-          const long long tiles = ((q.M + 127) / 128) * ((q.N_out + tn - 1) / tn);
-          if (tiles > kc_max_clusters(h, sl)) continue;
-          const double per_kb = tn == 64 ? 400.0 : (tn == 128 ? 450.0 : 1000.0);
-          const double cost = std::max(std::ceil((double)k_blocks_all / sl) * per_kb, hbm) + (tn == 256 ? 13000.0 : 10000.0);
-          if (cost < best_kc) {
-            best_kc = cost;
-            kc_s = sl;
-            kc_tn = tn;
+      int kc_s = 0, kc_tn = 0, kc_cg = 0;
+      for (int cg = 1; cg <= 2; ++cg) {
+        if (user != nullptr && user->cta_group != 0 && user->cta_group != cg) continue;
+        if (user != nullptr && user->tile_m != 0 && user->tile_m != 128 * cg) continue;
+        for (int sl = 2; sl * cg <= 8; sl *= 2)
+          for (int tn = 64; tn <= 256; tn *= 2) {
+            if (tn % (32 * sl) || !tile_ok(q, tn, cg) || max_stages_for(q, tn, cg) < 2 || k_blocks_all < 4 * sl) continue;
+            const long long tiles = ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + tn - 1) / tn);
+            if (tiles > kc_max_clusters(h, sl, cg)) continue;
+            const double per_kb = cg == 1 ? (tn == 64 ? 400.0 : (tn == 128 ? 450.0 : 1000.0)) : (tn == 256 ? 880.0 : 400.0);
+            const double cost =
+                std::max(std::ceil((double)k_blocks_all / sl) * per_kb, hbm) + (tn == 256 ? 13000.0 : 10000.0);
+            if (cost < best_kc * 0.999) {
+              best_kc = cost;
+              kc_s = sl;
+              kc_tn = tn;
+              kc_cg = cg;
+            }
           }
-        }
+      }
       int unused = 1;
       const double best_timed = best_cg != 0 ? model(best_cg, best_tn, &unused, true) : best;
       if (kc_s != 0 && best_kc < 0.92 * best_timed) {
-        c.cta_group = 1;
+        c.cta_group = kc_cg;
         c.tile_n = kc_tn;
         c.split_k = kc_s;
         c.schedule = 3;
@@ -703,9 +711,11 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
     }
   }
   if (c.schedule == 3) {
-    // K slices as a cluster: 128-row tiles, 2 / 4 / 8 slices, every CTA finishes tile_n / slices columns (whole
-    // 32-column pieces), column-wise epilogues on BF16 operands; every slice has at least one k-block
-    const bool can = cg == 1 && (c.split_k == 2 || c.split_k == 4 || c.split_k == 8) && c.tile_n % (32 * c.split_k) == 0 &&
+    // K slices as a cluster: 2 / 4 / 8 slices of single CTAs (128-row tiles) or 2 / 4 of pairs (256-row tiles), at
+    // most 8 CTAs; every CTA finishes tile_n / slices columns (whole 32-column pieces); column-wise epilogues on
+    // BF16 operands; every slice has at least one k-block
+    const bool can = (c.split_k == 2 || c.split_k == 4 || c.split_k == 8) && c.split_k * cg <= 8 &&
+                     c.tile_n % (32 * c.split_k) == 0 &&
                      !gate && q.epi != FACT_EPI_BIAS_SOFTMAX && !q.fp8 && q.groups == 0 && !q.stats_out && !q.norm &&
                      p.k_blocks >= c.split_k && units <= 0x7fffffffLL;
     if (!can) return FACT_ERR_UNSUPPORTED;
@@ -714,7 +724,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
     plan->smem_bytes = std::max((int)kc_smem_bytes(c.tile_n, c.split_k, c.stages, p.stage_bytes), kMinSmemRequest);
     if (plan->smem_bytes > kSmemBudget) return FACT_ERR_UNSUPPORTED;
     const long long tiles = units / c.split_k;
-    plan->grid = (int)std::min<long long>(tiles, kc_max_clusters(h, c.split_k)) * c.split_k;
+    plan->grid = (int)std::min<long long>(tiles, kc_max_clusters(h, c.split_k, cg)) * c.split_k * cg;
   }
   if (c.split_k < 0) {
     // Stream-K: the staged epilogue parks and finishes the pieces, so an output it cannot store is data-parallel.
@@ -788,29 +798,39 @@ fact_status_t launch_instance(fact_handle_t h, int slot, const Plan& plan, const
   return FACT_OK;
 }
 
-template <int EPI>
+template <int EPI, int CG>
 fact_status_t launch_kcluster_instance(fact_handle_t h, int slot, const Plan& plan, const CUtensorMap* tm,
                                        cudaStream_t stream) {
-  auto kern = fact_gemm_kcluster_kernel<EPI>;
+  auto kern = fact_gemm_kcluster_kernel<EPI, CG>;
   if (!h->configured_mask.test((size_t)slot)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e != cudaSuccess) return cuda_fail(h, "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
     h->configured_mask.set((size_t)slot);
   }
   cudaError_t e = launch_pdl(h, kern, (unsigned)plan.grid, (unsigned)kKcThreads, (size_t)plan.smem_bytes, stream,
-                             plan.cfg.split_k, tm[0], tm[1], plan.p);
+                             plan.cfg.split_k * CG, tm[0], tm[1], plan.p);
   if (e != cudaSuccess) return cuda_fail(h, "cudaLaunchKernelEx (K slices as a cluster)", e);
   h->launches++;
   return FACT_OK;
 }
 
 fact_status_t launch_kcluster(fact_handle_t h, int epi, const Plan& plan, const CUtensorMap* tm, cudaStream_t stream) {
+  if (plan.cfg.cta_group == 2) {
+    switch (epi) {
+      case kEpiNone: return launch_kcluster_instance<kEpiNone, 2>(h, 160, plan, tm, stream);
+      case kEpiBias: return launch_kcluster_instance<kEpiBias, 2>(h, 161, plan, tm, stream);
+      case kEpiBiasRelu: return launch_kcluster_instance<kEpiBiasRelu, 2>(h, 162, plan, tm, stream);
+      case kEpiBiasGeluTanh: return launch_kcluster_instance<kEpiBiasGeluTanh, 2>(h, 163, plan, tm, stream);
+      case kEpiBiasResidual: return launch_kcluster_instance<kEpiBiasResidual, 2>(h, 164, plan, tm, stream);
+      default: return FACT_ERR_UNSUPPORTED;
+    }
+  }
   switch (epi) {
-    case kEpiNone: return launch_kcluster_instance<kEpiNone>(h, 150, plan, tm, stream);
-    case kEpiBias: return launch_kcluster_instance<kEpiBias>(h, 151, plan, tm, stream);
-    case kEpiBiasRelu: return launch_kcluster_instance<kEpiBiasRelu>(h, 152, plan, tm, stream);
-    case kEpiBiasGeluTanh: return launch_kcluster_instance<kEpiBiasGeluTanh>(h, 153, plan, tm, stream);
-    case kEpiBiasResidual: return launch_kcluster_instance<kEpiBiasResidual>(h, 154, plan, tm, stream);
+    case kEpiNone: return launch_kcluster_instance<kEpiNone, 1>(h, 150, plan, tm, stream);
+    case kEpiBias: return launch_kcluster_instance<kEpiBias, 1>(h, 151, plan, tm, stream);
+    case kEpiBiasRelu: return launch_kcluster_instance<kEpiBiasRelu, 1>(h, 152, plan, tm, stream);
+    case kEpiBiasGeluTanh: return launch_kcluster_instance<kEpiBiasGeluTanh, 1>(h, 153, plan, tm, stream);
+    case kEpiBiasResidual: return launch_kcluster_instance<kEpiBiasResidual, 1>(h, 154, plan, tm, stream);
     default: return FACT_ERR_UNSUPPORTED;
   }
 }
@@ -1701,18 +1721,19 @@ fact_status_t fact_tune_ex(fact_handle_t h, fact_op_t op, int64_t batch, int64_t
         }
     }
   }
-  // K slices as a cluster (schedule 3): up to two waves of clusters of 2 / 4 / 8 CTAs (make_plan refuses what the
-  // kernel cannot run: gated or row-softmax epilogues, 8-bit operands, groups)
-  for (int sl = 2; sl <= 8; sl *= 2)
-    for (int tn = 64; tn <= 256; tn *= 2) {
-      if (tn % (32 * sl) || !tile_ok(q, tn, 1) || k_blocks < 2 * sl) continue;
-      const int smax = max_stages_for(q, tn, 1);
-      if (smax < 2) continue;
-      const long long tiles = batch * ((M + 127) / 128) * ((N + tn - 1) / tn);
-      if (tiles > 2LL * kc_max_clusters(h, sl)) continue;
-      fact_config_t c = {128, tn, q.k_elems(), smax, 1, 0, sl, 0, 3};
-      cands.push_back(c);
-    }
+  // K slices as a cluster (schedule 3): up to two waves of clusters of at most 8 CTAs, the slices single CTAs or pairs
+  // (make_plan refuses what the kernel cannot run: gated or row-softmax epilogues, 8-bit operands, groups)
+  for (int cg = 1; cg <= 2; ++cg)
+    for (int sl = 2; sl * cg <= 8; sl *= 2)
+      for (int tn = 64; tn <= 256; tn *= 2) {
+        if (tn % (32 * sl) || !tile_ok(q, tn, cg) || k_blocks < 2 * sl) continue;
+        const int smax = max_stages_for(q, tn, cg);
+        if (smax < 2) continue;
+        const long long tiles = batch * ((M + 128 * cg - 1) / (128 * cg)) * ((N + tn - 1) / tn);
+        if (tiles > 2LL * kc_max_clusters(h, sl, cg)) continue;
+        fact_config_t c = {128 * cg, tn, q.k_elems(), smax, cg, 0, sl, 0, 3};
+        cands.push_back(c);
+      }
   // Time `c` over `n` launches (per launch, ms); a negative result means the candidate failed.  Warm L2: the launches
   // run back to back between one event pair.  Cold L2: a buffer twice the size of L2 is overwritten before each
   // launch and every launch has an event pair of its own (what a benchmark that flushes L2 between launches sees).

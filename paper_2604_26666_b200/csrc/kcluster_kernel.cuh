@@ -31,7 +31,7 @@ __host__ __device__ constexpr uint32_t kc_exchange_bytes(int tile_n, int slices)
 }
 __host__ __device__ constexpr uint32_t kc_smem_bytes(int tile_n, int slices, int stages, uint32_t stage_bytes) {
   const uint32_t ring = (uint32_t)stages * stage_bytes, xch = kc_exchange_bytes(tile_n, slices);
-  return (ring > xch ? ring : xch) + (2 * kMaxStages + 4) * 8 + 16;
+  return (ring > xch ? ring : xch) + (2 * kMaxStages + 5) * 8 + 16;
 }
 
 __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
@@ -39,7 +39,7 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint
                : "memory");
 }
 
-template <int EPI>
+template <int EPI, int CG>
 __global__ void __launch_bounds__(kKcThreads, 1)
     fact_gemm_kcluster_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                               const GemmParams p) {
@@ -48,13 +48,16 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   const uint32_t smem_base = ptx::smem_u32(smem_raw);
-  const int S = p.split_k;                      // CTAs per cluster = K slices per tile
+  const int S = p.split_k;                      // K slices per tile; the cluster has S CTAs (CG == 1) or S pairs
   const uint32_t rank = ptx::cluster_ctarank();
+  const uint32_t half = rank % (uint32_t)CG;     // which CTA of its pair: the first (the leader) issues the pair's products
+  const uint32_t kr = rank / (uint32_t)CG;       // the slice of K this CTA (pair) multiplies
+  const uint32_t leader = rank - half;
   const int cb = p.tile_n / S;                  // accumulator columns each CTA finishes (a multiple of 32)
   const uint32_t ring_bytes = (uint32_t)p.stages * p.stage_bytes;
   const uint32_t xch_bytes = kc_exchange_bytes(p.tile_n, S);
   const uint32_t bar_base = smem_base + (ring_bytes > xch_bytes ? ring_bytes : xch_bytes);
-  const uint32_t ctrl_off = bar_base - smem_base + (2 * kMaxStages + 4) * 8;
+  const uint32_t ctrl_off = bar_base - smem_base + (2 * kMaxStages + 5) * 8;
   volatile uint32_t* tmem_holder_p = reinterpret_cast<volatile uint32_t*>(smem_raw + ctrl_off);
   volatile int* abort_p = reinterpret_cast<volatile int*>(smem_raw + ctrl_off + 4);
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
@@ -63,19 +66,22 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   const uint32_t peers_bar = bar_base + 8u * (uint32_t)(2 * kMaxStages + 1);  // ... and so is every peer's: S arrivals
   const uint32_t xfull_bar = bar_base + 8u * (uint32_t)(2 * kMaxStages + 2);  // all S blocks have arrived: 4 S arrivals
   const uint32_t xdone_bar = bar_base + 8u * (uint32_t)(2 * kMaxStages + 3);  // ... and have been added up: 4 arrivals
+  const uint32_t mdone_bar = bar_base + 8u * (uint32_t)(2 * kMaxStages + 4);  // the same for every CTA of the pair (the
+                                                                              // leader's products write both): 4 CG
   // A launch this kernel cannot serve is refused by every CTA alike, before any barrier exists.
-  const bool refuse = (smem_base & 1023u) || S < 2 || S > 8 || (int)ptx::cluster_nctarank() != S || cb * S != p.tile_n ||
+  const bool refuse = (smem_base & 1023u) || S < 2 || S * CG > 8 || (int)ptx::cluster_nctarank() != S * CG || cb * S != p.tile_n ||
                       (cb & 31) || p.k_base < 1 || p.gate;
   if (refuse) {
     if (threadIdx.x == 0) atomicExch(p.status, kDeviceTimeoutCode);
     return;
   }
-  if (threadIdx.x < 2 * kMaxStages + 4) {
+  if (threadIdx.x < 2 * kMaxStages + 5) {
     const int i = (int)threadIdx.x;
     uint32_t count = 1;
     if (i == 2 * kMaxStages + 1) count = (uint32_t)S;
     if (i == 2 * kMaxStages + 2) count = 4u * (uint32_t)S;
     if (i == 2 * kMaxStages + 3) count = 4u;
+    if (i == 2 * kMaxStages + 4) count = 4u * (uint32_t)CG;
     ptx::mbar_init(bar_base + 8u * (uint32_t)i, count);
     if (i == 0) *abort_p = 0;
     ptx::fence_mbar_init();
@@ -86,8 +92,8 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   }
   if (warp == 1) {
     __syncwarp();
-    ptx::tmem_alloc<1>(smem_base + ctrl_off, p.tmem_cols);
-    ptx::tmem_relinquish<1>();
+    ptx::tmem_alloc<CG>(smem_base + ctrl_off, p.tmem_cols);
+    ptx::tmem_relinquish<CG>();
   }
   ptx::tc_fence_before();
   __syncthreads();
@@ -104,8 +110,8 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   const unsigned long long ns_go = prof ? ptx::globaltimer_ns() : 0ull;
   long long* const prof_c = reinterpret_cast<long long*>(p.status + 2);
 
-  const int cluster_id = (int)(blockIdx.x / (unsigned)S);
-  const int n_clusters = (int)(gridDim.x / (unsigned)S);
+  const int cluster_id = (int)(blockIdx.x / (unsigned)(S * CG));
+  const int n_clusters = (int)(gridDim.x / (unsigned)(S * CG));
   const int tiles = p.total_units / S;  // (units are numbered tile-major, slice-minor)
   auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
     return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_p, p.status)) != 0;
@@ -121,11 +127,12 @@ __global__ void __launch_bounds__(kKcThreads, 1)
     bool ok = true;
     int it = 0;
     for (int tile = cluster_id; ok && tile < tiles; tile += n_clusters, ++it) {
-      const WorkUnit w = decode_unit(p, tile * S + (int)rank);
+      const WorkUnit w = decode_unit(p, tile * S + (int)kr);
       // the ring doubles as the exchange buffer: the blocks of the tile before must have been added up
       if (it > 0) ok = wait_all(xdone_bar, (uint32_t)(it - 1) & 1u);
       if (!ok) break;
-      const int m0 = w.tm * kTileM;
+      const int m0 = (w.tm * CG + (int)half) * kTileM;
+      const int col0 = (int)half * (p.tile_n / CG);  // a pair's CTAs load one half of the B tile each
       for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
         if (!wait_all(empty_bar(stage), phase ^ 1u)) {
           ok = false;
@@ -133,17 +140,27 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         }
         const uint32_t sa = smem_base + (uint32_t)stage * p.stage_bytes;
         const uint32_t sb = sa + kStageBytesA;
-        const uint32_t fb = full_bar(stage);
+        uint32_t fb = full_bar(stage);
         if (ptx::elect_one()) {
-          ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-          ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+          if (half == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);  // (the bytes of both CTAs of a pair)
+          if constexpr (CG == 2) {
+            fb = ptx::mapa(fb, leader);  // both CTAs' loads complete on the leader's barrier
+            ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
+          } else {
+            ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+          }
 #pragma unroll
           for (int i = 0; i < 4; ++i)
             if (i < p.b_loads) {
-              const int n = w.tn * p.tile_n + i * p.b_box_n;
+              const int n = w.tn * p.tile_n + col0 + i * p.b_box_n;
               const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
-              if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n, kb * kTileK, w.b);
-              else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n, w.b);
+              if constexpr (CG == 2) {
+                if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n, kb * kTileK, w.b);
+                else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n, w.b);
+              } else {
+                if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n, kb * kTileK, w.b);
+                else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n, w.b);
+              }
             }
         }
         if (++stage == p.stages) {
@@ -153,16 +170,20 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 && half == 0) {
+    // ------------------------------------------------------------ MMA issuer (of the pair's leader)
+    auto commit = [&](uint32_t b) {  // to this CTA's barrier and, for a pair, to the peer's at the same offset
+      ptx::umma_commit<CG>(b);
+      if constexpr (CG == 2) ptx::umma_commit<2>(ptx::mapa(b, rank + 1));
+    };
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     int it = 0;
     for (int tile = cluster_id; ok && tile < tiles; tile += n_clusters, ++it) {
-      const WorkUnit w = decode_unit(p, tile * S + (int)rank);
-      // the accumulator of the tile before must have been read (its blocks are added up only after that)
-      if (it > 0) ok = wait_all(xdone_bar, (uint32_t)(it - 1) & 1u);
+      const WorkUnit w = decode_unit(p, tile * S + (int)kr);
+      // the accumulators of the tile before must have been read (their blocks are added up only after that)
+      if (it > 0) ok = wait_all_cluster(mdone_bar, (uint32_t)(it - 1) & 1u);
       if (!ok) break;
       ptx::tc_fence_after();
       for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
@@ -179,9 +200,9 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         if (ptx::elect_one()) {
 #pragma unroll
           for (int k = 0; k < kTileK / kUmmaK; ++k)
-            ptx::umma_bf16<1>(tmem_base, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step), p.idesc,
-                              (kb > w.kb_begin || k > 0) ? 1u : 0u);
-          ptx::umma_commit<1>(empty_bar(stage));
+            ptx::umma_bf16<CG>(tmem_base, adesc + (uint64_t)(k * p.a_k_step), bdesc + (uint64_t)(k * p.b_k_step), p.idesc,
+                               (kb > w.kb_begin || k > 0) ? 1u : 0u);
+          commit(empty_bar(stage));
         }
         if (++stage == p.stages) {
           stage = 0;
@@ -189,21 +210,21 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         }
       }
       if (!ok) break;
-      if (ptx::elect_one()) ptx::umma_commit<1>(accf_bar);
+      if (ptx::elect_one()) commit(accf_bar);
     }
     __syncwarp();
-  } else {
+  } else if (warp >= 2) {
     // ------------------------------------------------------------ exchange and epilogue: one accumulator row per thread
     const int q = warp & 3;  // the TMEM lane quarter this warp may read
     const int row_in_tile = q * 32 + lane;
     const uint32_t chunk_stride = (uint32_t)kTileM * 16u;                   // bytes between two 4-column groups
     const uint32_t block_stride = (uint32_t)(cb >> 2) * chunk_stride;       // ... between the blocks of two senders
-    const uint32_t my_slot = smem_base + rank * block_stride + (uint32_t)row_in_tile * 16u;  // where a peer keeps MY block
+    const uint32_t my_slot = smem_base + kr * block_stride + (uint32_t)row_in_tile * 16u;  // where a peer keeps MY block
     const bool c_vec = p.c_vec != 0;
     bool ok = true;
     int it = 0;
     for (int tile = cluster_id; ok && tile < tiles; tile += n_clusters, ++it) {
-      const WorkUnit w = decode_unit(p, tile * S + (int)rank);
+      const WorkUnit w = decode_unit(p, tile * S + (int)kr);
       const uint32_t par = (uint32_t)it & 1u;
       // ---- this CTA's slice is complete: tell every CTA of the cluster, then wait until all of them are (their
       // rings are then idle and may receive blocks)
@@ -217,7 +238,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       if (warp == 2) {
         // (a relaxed arrival: it publishes no data, it says that this CTA's products have stopped reading its ring,
         // which this thread has just observed through the accumulator's barrier)
-        if (lane < S) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(peers_bar, (uint32_t)lane));
+        if (lane < S) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(peers_bar, (uint32_t)lane * CG + half));
         __syncwarp();
       }
       if (!wait_all_cluster(peers_bar, par)) {
@@ -230,16 +251,16 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       const int pieces = p.tile_n >> 5;
       const int per_owner = cb >> 5;
       auto piece_of = [&](int i) {
-        int pc = i + ((int)rank + 1) * per_owner;
+        int pc = i + ((int)kr + 1) * per_owner;
         if (pc >= pieces) pc -= pieces;
-        if (pc >= pieces) pc -= pieces;  // ((rank + 1) * per_owner may equal pieces)
+        if (pc >= pieces) pc -= pieces;  // ((kr + 1) * per_owner may equal pieces)
         return pc;
       };
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
       auto send = [&](int pc, const uint32_t (&v)[32]) {
         const int owner = pc / per_owner;
         const int col = (pc - owner * per_owner) << 5;  // first column inside the owner's block
-        const uint32_t dst = ptx::mapa(my_slot + (uint32_t)(col >> 2) * chunk_stride, (uint32_t)owner);
+        const uint32_t dst = ptx::mapa(my_slot + (uint32_t)(col >> 2) * chunk_stride, (uint32_t)owner * CG + half);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           st_shared_cluster_v4(dst + chunk_stride * (uint32_t)j, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -259,7 +280,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       }
       ptx::tc_fence_before();
       __syncwarp();  // every lane's stores are ordered before lane 0's releasing arrivals
-      if (lane < S) ptx::mbar_arrive_cluster(ptx::mapa(xfull_bar, (uint32_t)lane));
+      if (lane < S) ptx::mbar_arrive_cluster(ptx::mapa(xfull_bar, (uint32_t)lane * CG + half));
       if (stamp) prof_c[5] = clock64() - t_go;
       // ---- receive: add the S blocks of this CTA's columns in the order of the workspace reduction, apply the
       // epilogue, store
@@ -268,9 +289,9 @@ __global__ void __launch_bounds__(kKcThreads, 1)
         break;
       }
       if (stamp) prof_c[6] = clock64() - t_go;
-      const int row = w.tm * kTileM + row_in_tile;
+      const int row = (w.tm * CG + (int)half) * kTileM + row_in_tile;
       const bool row_ok = row < p.M;
-      const int n_block0 = w.tn * p.tile_n + (int)rank * cb;
+      const int n_block0 = w.tn * p.tile_n + (int)kr * cb;
       const long long off = (long long)w.b * p.strideC + (long long)row * p.ldc;
       char* c_row = reinterpret_cast<char*>(p.C) + off * (p.out_f32 ? 4 : 2);
       const __nv_bfloat16* r_row = nullptr;
@@ -316,8 +337,12 @@ __global__ void __launch_bounds__(kKcThreads, 1)
       }
       // the next tile's operands arrive in this memory through the asynchronous proxy
       ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(xdone_bar);
+      if (lane == 0) {
+        ptx::mbar_arrive(xdone_bar);
+        ptx::mbar_arrive_cluster_relaxed(ptx::mapa(mdone_bar, leader));  // (orders tensor-memory reads: the fences do)
+      }
       if (stamp) prof_c[7] = clock64() - t_go;
     }
     __syncwarp();
@@ -340,7 +365,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
   }
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc<1>(tmem_base, p.tmem_cols);
+    ptx::tmem_dealloc<CG>(tmem_base, p.tmem_cols);
   }
 }
 

@@ -50,8 +50,8 @@ def _draw(i):
     cfg["schedule"] = int(rng.choice([0, 1, 2]))
     if rng.integers(0, 4) == 0:
         # K slices as a cluster, added up through distributed shared memory
-        cfg = {"cta_group": 1, "tile_n": int(rng.choice([64, 128, 256])), "split_k": int(rng.choice([2, 4, 8])),
-               "schedule": 3}
+        cfg = {"cta_group": int(rng.choice([1, 2])), "tile_n": int(rng.choice([64, 128, 256])),
+               "split_k": int(rng.choice([2, 4, 8])), "schedule": 3}
         if rng.integers(0, 2):
             cfg["stages"] = int(rng.integers(2, 5))
     return epi, layout, out, M, N, K, cfg

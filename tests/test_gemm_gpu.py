@@ -295,24 +295,32 @@ def test_few_slices_take_the_wide_reduction_and_keep_every_bit(h, out):
 
 
 @pytest.mark.parametrize("layout", ["KN", "NK"])
-@pytest.mark.parametrize("slices,tile_n", [(2, 64), (2, 128), (4, 128), (2, 256), (4, 256), (8, 256)])
-def test_k_slices_as_a_cluster_are_exact_and_equal_the_workspace_reduction(h, layout, slices, tile_n):
-    """schedule 3: the K slices of a tile run as one cluster and are added up through distributed shared memory, in
+@pytest.mark.parametrize("pair,slices,tile_n", [(1, 2, 64), (1, 2, 128), (1, 4, 128), (1, 2, 256), (1, 4, 256), (1, 8, 256),
+                                                (2, 2, 64), (2, 2, 128), (2, 4, 128), (2, 2, 256), (2, 4, 256)])
+def test_k_slices_as_a_cluster_are_exact_and_equal_the_workspace_reduction(h, layout, pair, slices, tile_n):
+    """schedule 3: the K slices of a tile run as one cluster (each slice a CTA on a 128-row tile, or a CTA pair on a
+    256-row tile) and are added up through distributed shared memory, in
     the order of the workspace reduction.  Integer inputs: bit-exact against the oracle, for every epilogue the
     schedule serves, several tiles per cluster (more tiles than clusters), ragged M, N and K, FP32 and BF16 outputs;
     random inputs: the same bits as the same number of slices through the workspace."""
     from paper_2604_26666_b200.binding import FactError
 
-    kc = {"cta_group": 1, "tile_n": tile_n, "split_k": slices, "schedule": 3}
+    kc = {"cta_group": pair, "tile_n": tile_n, "split_k": slices, "schedule": 3}
+    if pair == 2 and tile_n == 64 and layout == "KN":
+        # (each CTA of a pair loads half the tile's columns of B; a [K, N] operand has no 32-column box)
+        case = mk("kc_pair_kn_64", 256, 256, 1024, layout=layout)
+        with pytest.raises(FactError):
+            run_gpu(h, wl.make_inputs(case), case, cfg=kc)
+        return
     for (M, N, K, epi, out) in [(200, 520, 1096, "BIAS_RESIDUAL", "bf16"), (130, 264, 2048, "BIAS_RELU", "f32"),
                                 (128 * 40 + 8, 512, 1024, "NONE", "bf16")]:
-        case = mk(f"kc_{slices}_{tile_n}_{epi}", M, N, K, epilogue=epi, layout=layout, out=out)
+        case = mk(f"kc_{pair}_{slices}_{tile_n}_{epi}", M, N, K, epilogue=epi, layout=layout, out=out)
         bit_exact(h, case, small_int_inputs(case, 31, lo=-2, hi=2), cfg=kc)
-    case = mk(f"kc_rand_{slices}_{tile_n}", 300, 520, 4096, epilogue="BIAS_GELU_TANH", layout=layout)
+    case = mk(f"kc_rand_{pair}_{slices}_{tile_n}", 300, 520, 4096, epilogue="BIAS_GELU_TANH", layout=layout)
     ins = wl.make_inputs(case)
     check_case(h, case, ins=ins, cfg=kc)
     a = run_gpu(h, ins, case, cfg=kc)
-    b = run_gpu(h, ins, case, cfg={"cta_group": 1, "tile_n": tile_n, "split_k": slices})
+    b = run_gpu(h, ins, case, cfg={"cta_group": pair, "tile_n": tile_n, "split_k": slices})
     torch.cuda.synchronize()
     assert torch.equal(a, b), "cluster and workspace reductions of the same slices differ"
     assert h.workspace_bytes("linear", 1, 300, 520, 4096, "BIAS_GELU_TANH", layout, torch.bfloat16, kc) == 0
@@ -320,14 +328,16 @@ def test_k_slices_as_a_cluster_are_exact_and_equal_the_workspace_reduction(h, la
     gate = mk("kc_gate", 128, 256, 1024, epilogue="SILU_GATE", layout=layout)
     with pytest.raises(FactError):
         run_gpu(h, wl.make_inputs(gate), gate, cfg=kc)
-    for bad in ({"cta_group": 2}, {"split_k": 3}, {"tile_n": 96}):
+    # (a cluster holds at most 8 CTAs: 8 slices of pairs would be 16)
+    for bad in ({"cta_group": 2, "split_k": 8, "tile_n": 256}, {"split_k": 3}, {"tile_n": 96}):
         with pytest.raises(FactError):
             run_gpu(h, ins, case, cfg={**kc, **bad})
     assert h.device_status() == 0
 
 
-def test_k_slices_as_a_cluster_serve_the_batched_and_the_sliced_entry_points(h):
-    kc = {"cta_group": 1, "tile_n": 128, "split_k": 4, "schedule": 3}
+@pytest.mark.parametrize("pair", [1, 2])
+def test_k_slices_as_a_cluster_serve_the_batched_and_the_sliced_entry_points(h, pair):
+    kc = {"cta_group": pair, "tile_n": 128, "split_k": 4, "schedule": 3}
     for layout in ("KN", "NK"):
         case = mk("kc_batched", 200, 264, 1536, op="gemm_batched", batch=5, layout=layout, out="f32")
         bit_exact(h, case, small_int_inputs(case, 41, lo=-2, hi=2), cfg=kc)
@@ -336,14 +346,15 @@ def test_k_slices_as_a_cluster_serve_the_batched_and_the_sliced_entry_points(h):
     assert h.device_status() == 0
 
 
-def test_k_slices_as_a_cluster_in_a_cuda_graph_and_back_to_back(h):
+@pytest.mark.parametrize("pair", [1, 2])
+def test_k_slices_as_a_cluster_in_a_cuda_graph_and_back_to_back(h, pair):
     """Cluster launches can be captured and replayed, and launches that follow one another on a stream (each may move
     onto the SMs while its predecessor's last CTAs leave) -- of the cluster kernel and of the persistent kernel in
     turn -- give the same bits every time."""
     case = mk("kc_graph", 384, 512, 4096, epilogue="BIAS_RELU", layout="NK")
     ins = wl.make_inputs(case)
     X, W, b = ins.X.cuda(), ins.W.cuda(), ins.bias.cuda()
-    kc = {"cta_group": 1, "tile_n": 128, "split_k": 4, "schedule": 3}
+    kc = {"cta_group": pair, "tile_n": 128, "split_k": 4, "schedule": 3}
     first_kc = h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", cfg=kc)
     first_dp = h.linear(X, W, bias=b, epilogue=case.epilogue, layout="NK", cfg={"split_k": 1})
     torch.cuda.synchronize()
