@@ -604,8 +604,9 @@ fact_status_t fact_last_kernel_clock(fact_handle_t handle, void* cuda_stream, in
  * cycles from the moment the kernel may touch global memory: [0] end of the kernel and [1] the same in nanoseconds,
  * [2] first operand stage ready, [3] accumulator complete, [4] every peer's accumulator complete, [5] column blocks
  * sent, [6] column blocks received, [7] tile stored.
- * FACT_DEBUG_FLAGS is read once, by fact_create.  The library as built by default honours two bits, neither of
- * which changes a result: 256 (these counters) and 2048 (no downward K walk on every second tile).  The
+ * FACT_DEBUG_FLAGS is read once, by fact_create.  The library as built by default honours four bits, none of
+ * which changes a result: 256 (these counters), 2048 (no downward K walk on every second tile), 4096 (no
+ * programmatic dependent launch) and 8192 (operand loads without the evict-last L2 policy).  The
  * work-skipping experiment switches (1, 2, 4: the GEMM kernel's loads, products, stores; 8, 64, 128: the attention
  * kernel's softmax arithmetic and its two products), whose output is meaningless, exist only in a library
  * compiled with -DFACT_EXPERIMENTS; the default build ignores those bits. */

@@ -45,8 +45,9 @@ constexpr int kSmemBudget = 227 * 1024;  // dynamic shared memory per CTA: the w
                                          // shared memory is used; the kernel checks the 1024-byte alignment of its base)
 constexpr int kMinSmemRequest = 120 * 1024;  // > half an SM: one CTA per SM, so TMEM allocation never blocks
 constexpr int kStatusInts = 64;  // status word, clock / profile counters, grid-barrier counters; stream-K flags follow
-constexpr int kDiagnosticFlags = 256 | 2048 | 4096;  // FACT_DEBUG_FLAGS bits that leave results intact: cycle counters,
-                                                      // no K serpentine, no programmatic dependent launch
+constexpr int kDiagnosticFlags = 256 | 2048 | 4096 | 8192;  // FACT_DEBUG_FLAGS bits that leave results intact: cycle
+                                                             // counters, no K serpentine, no programmatic dependent
+                                                             // launch, no L2 eviction priority on operand loads
 constexpr int kMaxGroups = 4096;  // row groups of a grouped GEMM (the handle's device table holds 2 x (kMaxGroups + 1) ints)
 
 // Key of the tuner's table: everything that changes which configuration is best.
@@ -593,6 +594,7 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   const int slices = std::max(1, c.split_k);  // (stream-K, split_k < 0, cuts no tile into equal slices)
   p.split_k = slices;
   p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
+  p.l2_keep_operands = (h->debug_flags & 8192) ? 0 : 1;
   p.k_base = p.k_blocks / slices;
   p.k_rem = p.k_blocks % slices;
   p.raster_along_n = c.raster_group < 0;

@@ -93,6 +93,7 @@ struct GemmParams {
   int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
   int raster_along_n; // 1: the raster groups n-tiles (a slab of W stays in L2), 0: m-tiles (a slab of X)
   int k_serpentine;   // 1: every second tile of a CTA walks K downwards (L2 reuse between waves)
+  int l2_keep_operands;  // 1: the operand loads ask L2 to evict their lines last (ptx::l2_policy)
   int k_base, k_rem;  // k_blocks = split_k * k_base + k_rem: slice s covers k_base (+1 if s < k_rem) k-blocks
   int total_units;   // batch * tiles_m * tiles_n * split_k
   // B operand loads issued by ONE CTA per stage
@@ -946,6 +947,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
     // Warp 0 loads the A tiles (and posts the expected byte count), warp 6 the B boxes.
     const bool do_a = warp == 0;
     if (!FACT_SKIP(p, 1)) {
+      const uint64_t pol = ptx::l2_policy(p.l2_keep_operands != 0);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -987,10 +989,10 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
               if constexpr (CG == 2) {
                 if (cta_rank == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
                 fb = ptx::mapa(fb, 0);  // both CTAs' loads complete on the leader's barrier
-                ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * p.k_elems, m0, a_batch);
+                ptx::tma_load_3d_cg2_hint(sa, &tmA, fb, kb * p.k_elems, m0, a_batch, pol);
               } else {
                 ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);
-                ptx::tma_load_3d(sa, &tmA, fb, kb * p.k_elems, m0, a_batch);
+                ptx::tma_load_3d_hint(sa, &tmA, fb, kb * p.k_elems, m0, a_batch, pol);
               }
             } else {
               if constexpr (CG == 2) fb = ptx::mapa(fb, 0);
@@ -999,11 +1001,11 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
                 if (i < p.b_loads) {
                   const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
                   if constexpr (CG == 2) {
-                    if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b);
-                    else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b);
+                    if (p.b_kn) ptx::tma_load_3d_cg2_hint(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b, pol);
+                    else ptx::tma_load_3d_cg2_hint(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b, pol);
                   } else {
-                    if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b);
-                    else ptx::tma_load_3d(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b);
+                    if (p.b_kn) ptx::tma_load_3d_hint(dst, &tmB, fb, n_box[i], kb * p.k_elems, w.b, pol);
+                    else ptx::tma_load_3d_hint(dst, &tmB, fb, kb * p.k_elems, n_box[i], w.b, pol);
                   }
                 }
               }
