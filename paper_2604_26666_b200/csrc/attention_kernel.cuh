@@ -240,6 +240,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       // ------------------------------------------------------------ TMA producer
       int g = 0;  // key blocks loaded so far
       bool ok = true;
+      // keys and values are read again by every query tile of their head (and of the heads that share them)
+      const uint64_t keep = ptx::l2_policy((p.debug & 8192) == 0);
       for (int n = 0; ok && n < n_items; ++n) {
         const AttnItem it = item_of(n);
         for (int t = 0; ok && t < 2; ++t) {
@@ -259,14 +261,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           if (ptx::elect_one()) {
             ptx::mbar_arrive_expect_tx(bar(K_FULL + s), kv_bytes);
             for (int c = 0; c < chunks; ++c)
-              ptx::tma_load_4d(k_s0 + s * kv_bytes + c * kv_chunk, &tmK, bar(K_FULL + s), c * 64, it.kvh, j * BK, it.b);
+              ptx::tma_load_4d_hint(k_s0 + s * kv_bytes + c * kv_chunk, &tmK, bar(K_FULL + s), c * 64, it.kvh, j * BK, it.b,
+                                    keep);
           }
           ok = wait_all(bar(V_EMPTY + s), par);
           if (!ok) break;
           if (ptx::elect_one()) {
             ptx::mbar_arrive_expect_tx(bar(V_FULL + s), kv_bytes);
             for (int c = 0; c < chunks; ++c)
-              ptx::tma_load_4d(v_s0 + s * kv_bytes + c * kv_chunk, &tmV, bar(V_FULL + s), c * 64, it.kvh, j * BK, it.b);
+              ptx::tma_load_4d_hint(v_s0 + s * kv_bytes + c * kv_chunk, &tmV, bar(V_FULL + s), c * 64, it.kvh, j * BK, it.b,
+                                    keep);
           }
         }
       }
