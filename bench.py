@@ -217,7 +217,7 @@ def main():
     torch.cuda.set_device(dev)
     dist = dist_util.init("nccl", dev)
     h = Handle(local_rank)
-    if h.debug_flags() & ~(256 | 2048 | 4096):  # only a -DFACT_EXPERIMENTS build honours the work-skipping switches
+    if h.debug_flags() & ~(256 | 2048 | 4096 | 8192):  # only a -DFACT_EXPERIMENTS build honours the work-skipping switches
         raise SystemExit("bench.py refuses to run with work-skipping FACT_DEBUG_FLAGS bits set")
     peaks = load_peaks()
     stream = torch.cuda.current_stream(dev)

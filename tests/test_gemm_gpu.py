@@ -404,6 +404,32 @@ def test_untuned_few_tiles_long_k_takes_k_slices_when_it_has_the_scratch(h):
     assert c <= 1.0 and t <= 1.0, (c, t)
 
 
+def test_diagnostic_switches_change_no_bit(h, monkeypatch):
+    """FACT_DEBUG_FLAGS (read once, when a handle is created): without the downward K walk of every second tile the
+    sums of those tiles are taken in the other order, which integer inputs do not see; without programmatic dependent
+    launch and without the L2 eviction priority of the operand loads nothing about the arithmetic changes at all, so
+    random inputs give the same bits.  The default build masks every other bit."""
+    from paper_2604_26666_b200.binding import Handle
+
+    case = mk("diag", 1100, 1032, 2048 + 72, epilogue="BIAS_GELU_TANH", layout="NK")
+    ins = wl.make_inputs(case)
+    ints = small_int_inputs(case, 77, lo=-2, hi=2)
+    want = run_gpu(h, ins, case).clone()
+    want_int = run_gpu(h, ints, case).clone()
+    for flags in (2048, 4096, 8192, 4096 | 8192, 1 | 2 | 4):
+        monkeypatch.setenv("FACT_DEBUG_FLAGS", str(flags))
+        h2 = Handle(0)
+        try:
+            assert h2.debug_flags() == (flags & (256 | 2048 | 4096 | 8192))
+            if not flags & 2048:
+                assert torch.equal(run_gpu(h2, ins, case), want), flags
+            assert torch.equal(run_gpu(h2, ints, case), want_int), flags
+            torch.cuda.synchronize()
+            assert h2.device_status() == 0
+        finally:
+            h2.close()
+
+
 # ------------------------------------------------------------------ degenerate sizes
 def test_empty_and_k_zero(h):
     dev = "cuda:0"
