@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       int g = 0;  // key blocks loaded so far
       bool ok = true;
       // keys and values are read again by every query tile of their head (and of the heads that share them)
-      const uint64_t keep = ptx::l2_policy((p.debug & 8192) == 0);
+      const uint64_t keep = ptx::l2_policy((p.debug & 8192) ? 0 : 2);
       for (int n = 0; ok && n < n_items; ++n) {
         const AttnItem it = item_of(n);
         for (int t = 0; ok && t < 2; ++t) {

@@ -594,7 +594,10 @@ fact_status_t make_plan(fact_handle_t h, const Problem& q, const fact_config_t* 
   const int slices = std::max(1, c.split_k);  // (stream-K, split_k < 0, cuts no tile into equal slices)
   p.split_k = slices;
   p.k_serpentine = (h->debug_flags & 2048) ? 0 : 1;
-  p.l2_keep_operands = (h->debug_flags & 8192) ? 0 : 1;
+  // L2 eviction priority of the operand loads: last where tiles share operand slabs (whole tiles, K slices as a
+  // cluster), first where K slices through the workspace stream every operand byte past once or twice and what must
+  // stay in L2 are the partial planes the tail of the launch reads back
+  p.l2_keep_operands = (h->debug_flags & 8192) ? 0 : (slices > 1 && c.schedule != 3 ? 1 : 2);
   p.k_base = p.k_blocks / slices;
   p.k_rem = p.k_blocks % slices;
   p.raster_along_n = c.raster_group < 0;

@@ -93,7 +93,7 @@ struct GemmParams {
   int tiles_m, tiles_n, k_blocks, split_k, raster_group, stages;
   int raster_along_n; // 1: the raster groups n-tiles (a slab of W stays in L2), 0: m-tiles (a slab of X)
   int k_serpentine;   // 1: every second tile of a CTA walks K downwards (L2 reuse between waves)
-  int l2_keep_operands;  // 1: the operand loads ask L2 to evict their lines last (ptx::l2_policy)
+  int l2_keep_operands;  // L2 eviction priority of the operand loads (ptx::l2_policy)
   int k_base, k_rem;  // k_blocks = split_k * k_base + k_rem: slice s covers k_base (+1 if s < k_rem) k-blocks
   int total_units;   // batch * tiles_m * tiles_n * split_k
   // B operand loads issued by ONE CTA per stage
@@ -947,7 +947,7 @@ __global__ void __launch_bounds__(kThreads + (DYN ? 32 : 0), 1)
     // Warp 0 loads the A tiles (and posts the expected byte count), warp 6 the B boxes.
     const bool do_a = warp == 0;
     if (!FACT_SKIP(p, 1)) {
-      const uint64_t pol = ptx::l2_policy(p.l2_keep_operands != 0);
+      const uint64_t pol = ptx::l2_policy(p.l2_keep_operands);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;

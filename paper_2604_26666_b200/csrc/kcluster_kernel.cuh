@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(kKcThreads, 1)
     uint32_t phase = 0;
     bool ok = true;
     int it = 0;
+    const uint64_t pol = ptx::l2_policy(p.l2_keep_operands);
     for (int tile = cluster_id; ok && tile < tiles; tile += n_clusters, ++it) {
       const WorkUnit w = decode_unit(p, tile * S + (int)kr);
       // the ring doubles as the exchange buffer: the blocks of the tile before must have been added up
@@ -145,9 +146,9 @@ __global__ void __launch_bounds__(kKcThreads, 1)
           if (half == 0) ptx::mbar_arrive_expect_tx(fb, p.tx_bytes);  // (the bytes of both CTAs of a pair)
           if constexpr (CG == 2) {
             fb = ptx::mapa(fb, leader);  // both CTAs' loads complete on the leader's barrier
-            ptx::tma_load_3d_cg2(sa, &tmA, fb, kb * kTileK, m0, w.b);
+            ptx::tma_load_3d_cg2_hint(sa, &tmA, fb, kb * kTileK, m0, w.b, pol);
           } else {
-            ptx::tma_load_3d(sa, &tmA, fb, kb * kTileK, m0, w.b);
+            ptx::tma_load_3d_hint(sa, &tmA, fb, kb * kTileK, m0, w.b, pol);
           }
 #pragma unroll
           for (int i = 0; i < 4; ++i)
@@ -155,11 +156,11 @@ __global__ void __launch_bounds__(kKcThreads, 1)
               const int n = w.tn * p.tile_n + col0 + i * p.b_box_n;
               const uint32_t dst = sb + (uint32_t)i * p.b_box_bytes;
               if constexpr (CG == 2) {
-                if (p.b_kn) ptx::tma_load_3d_cg2(dst, &tmB, fb, n, kb * kTileK, w.b);
-                else ptx::tma_load_3d_cg2(dst, &tmB, fb, kb * kTileK, n, w.b);
+                if (p.b_kn) ptx::tma_load_3d_cg2_hint(dst, &tmB, fb, n, kb * kTileK, w.b, pol);
+                else ptx::tma_load_3d_cg2_hint(dst, &tmB, fb, kb * kTileK, n, w.b, pol);
               } else {
-                if (p.b_kn) ptx::tma_load_3d(dst, &tmB, fb, n, kb * kTileK, w.b);
-                else ptx::tma_load_3d(dst, &tmB, fb, kb * kTileK, n, w.b);
+                if (p.b_kn) ptx::tma_load_3d_hint(dst, &tmB, fb, n, kb * kTileK, w.b, pol);
+                else ptx::tma_load_3d_hint(dst, &tmB, fb, kb * kTileK, n, w.b, pol);
               }
             }
         }

@@ -164,11 +164,13 @@ __device__ __forceinline__ void tma_load_3d_cg2(uint32_t dst, const void* tmap, 
       : "memory");
 }
 
-// An L2 eviction priority for the lines a load brings in: evicted last (operand slabs, which other CTAs and the next
-// waves want again, outlive the output lines written meanwhile) or the normal priority.
-__device__ __forceinline__ uint64_t l2_policy(bool evict_last) {
+// An L2 eviction priority for the lines a load brings in: 2 = evicted last (operand slabs, which other CTAs and the
+// next waves want again, outlive the output lines written meanwhile), 1 = evicted first (operands met once, so that
+// what the launch writes and reads back stays), 0 = the normal priority.
+__device__ __forceinline__ uint64_t l2_policy(int kind) {
   uint64_t pol;
-  if (evict_last) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  else if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
