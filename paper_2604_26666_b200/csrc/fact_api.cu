@@ -354,8 +354,14 @@ fact_status_t resolve_config(fact_handle_t h, const Problem& q, const fact_confi
                          q.groups == 0 && !q.fp8 && !q.stats_out && !q.norm && q.epi != FACT_EPI_BIAS_SOFTMAX;
   auto model = [&](int cg, int tn, int* slices_out, bool calibrated = false) -> double {
     const int out_cols = q.epi == FACT_EPI_SILU_GATE ? tn / 2 : tn;
-    const long long tiles =
-        std::max<long long>(1, q.batch) * ((q.M + 128 * cg - 1) / (128 * cg)) * ((q.N_out + out_cols - 1) / out_cols);
+    // (a grouped problem's m-tiles are counted group by group: every group ends in a ragged tile of its own, and
+    // 64 groups of 222-291 rows are 1.5 pair tiles of 256 rows each but 2.5 single tiles of 128)
+    long long m_tiles = (q.M + 128 * cg - 1) / (128 * cg);
+    if (q.groups > 0 && q.group_rows != nullptr) {
+      m_tiles = 0;
+      for (int g = 0; g < q.groups; ++g) m_tiles += (q.group_rows[g] + 128 * cg - 1) / (128 * cg);
+    }
+    const long long tiles = std::max<long long>(1, q.batch) * m_tiles * ((q.N_out + out_cols - 1) / out_cols);
     const long long slots = std::max(1, h->sm_count / cg);
     // (narrower tiles re-read the A operand from shared memory for less work: 0.65 of the full rate at 128 columns,
     // taken as 0.85 at 192, rank the widths against each other; timed on untuned shapes a k-block costs 450 cycles
