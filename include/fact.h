@@ -569,6 +569,16 @@ fact_status_t fact_device_status(fact_handle_t handle, void* cuda_stream, int* s
  * fact_device_status reports (and clears) the timeout; the context stays usable. */
 fact_status_t fact_selftest_wait_timeout(fact_handle_t handle, void* cuda_stream, double limit_ms);
 
+/* Diagnostic, host arithmetic only (no device is touched): the items CTA `cta` of `ctas` works through in a causal
+ * fact_attention call of few rounds (more items than CTAs, fewer than 16 per CTA, at most 8192 items; other calls
+ * deal the items out in closed form inside the kernel).  An item is 256 query rows of one (batch, head); item idx
+ * is head idx % batch_heads and the (idx / batch_heads)-th pair of tiles counted from the END of the sequence, so
+ * items come heaviest first.  The host gives each item, in that order, to the CTA whose items so far see the fewest
+ * key blocks (plus a fixed cost per item; the lower CTA on a tie) and hands the list to the kernel as a parameter.
+ * Writes at most max_items item numbers and their count to *n_items.  FACT_ERR_UNSUPPORTED above 8192 items. */
+fact_status_t fact_attention_deal(int ctas, int64_t batch_heads, int64_t seq, int head_dim, int cta, int max_items,
+                                  int32_t* items, int* n_items);
+
 /* Diagnostic, host arithmetic only (no device is touched): the stream-K schedule of one CTA group.  With
  * `sk_tiles` tiles of `k_blocks` k-blocks each shared out over `groups` CTA groups, writes the pieces group
  * `group` processes, in its order, as rows of five ints -- tile (index among the stream-K tiles), first k-block,

@@ -38,7 +38,7 @@ EXPORTED = [
     "fact_tune_cache_load", "fact_device_status", "fact_launch_count", "fact_device_info", "fact_last_error",
     "fact_last_kernel_clock", "fact_gemm_splitk_static", "fact_last_kernel_profile", "fact_selftest_wait_timeout",
     "fact_attention", "fact_norm", "fact_block_workspace_bytes", "fact_block_workspace_offsets", "fact_block_forward",
-    "fact_stream_k_pieces", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
+    "fact_stream_k_pieces", "fact_attention_deal", "fact_linear_fp8", "fact_linear_grouped", "fact_linear_grouped_fp8",
     "fact_linear_ex", "fact_row_stats", "fact_fold_norm", "fact_gemm_splitk_static_status", "fact_debug_flags",
     "fact_tune_ex", "fact_last_kernel_span", "fact_gemm_host", "fact_gemm_host_scratch_bytes",
     "fact_gemm_host_wait",
@@ -167,6 +167,7 @@ def lib() -> ctypes.CDLL:
     L.fact_row_stats.argtypes = [vp, i64, i64, vp, i64, vp, vp]
     L.fact_fold_norm.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
     L.fact_stream_k_pieces.argtypes = [c_int, i64, i64, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
+    L.fact_attention_deal.argtypes = [c_int, i64, i64, c_int, c_int, c_int, POINTER(ctypes.c_int32), POINTER(c_int)]
     L.fact_gemm_splitk_static_status.argtypes = [c_int, vp, POINTER(c_int)]
     L.fact_debug_flags.argtypes = [vp]
     L.fact_last_kernel_span.argtypes = [vp, vp, POINTER(i64)]
@@ -269,6 +270,18 @@ def stream_k_pieces(groups: int, sk_tiles: int, k_blocks: int, group: int):
                "fact_stream_k_pieces")
         if n.value <= cap:
             return [tuple(buf[5 * i: 5 * i + 5]) for i in range(n.value)]
+        cap = n.value
+
+
+def attention_deal(ctas: int, batch_heads: int, seq: int, head_dim: int, cta: int):
+    """The items one CTA of a causal attention call takes (fact_attention_deal; host arithmetic, no device needed)."""
+    cap = 64
+    while True:
+        buf = (ctypes.c_int32 * cap)()
+        n = c_int(0)
+        _check(lib().fact_attention_deal(ctas, batch_heads, seq, head_dim, cta, cap, buf, byref(n)), "fact_attention_deal")
+        if n.value <= cap:
+            return list(buf[: n.value])
         cap = n.value
 
 

@@ -112,11 +112,32 @@ struct AttnItem {
   int nbi;       // key blocks the item loads
 };
 
-template <int HD>  // head_dim: 64 or 128
+// Which items a CTA works through, decided on the host for causal problems of few rounds: the items in order of
+// weight (key blocks they see), each given to the CTA that has the least so far.  list[off[c] .. off[c + 1]) are CTA
+// c's items.  Travels as a kernel parameter, so no call shares it with another.
+constexpr int kAttnDealItems = 8192;
+constexpr int kAttnDealCtas = 256;
+struct AttnDeal {
+  uint16_t off[kAttnDealCtas + 1];
+  uint16_t list[kAttnDealItems];
+};
+struct AttnNoDeal {
+  int unused;
+};
+template <bool DEAL>
+struct AttnDealArg {
+  using type = AttnNoDeal;
+};
+template <>
+struct AttnDealArg<true> {
+  using type = AttnDeal;
+};
+
+template <int HD, bool DEAL = false>  // head_dim: 64 or 128; DEAL: the items come from the host's list
 __global__ void __launch_bounds__(kAttnThreads, 1)
     fact_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                               const AttnParams p) {
+                               const AttnParams p, const __grid_constant__ typename AttnDealArg<DEAL>::type deal) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
@@ -201,11 +222,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const int G = (int)gridDim.x;
   const int full_rounds = p.items / G, tail = p.items - full_rounds * G;
   auto pos_in_round = [&](int n) { return (n & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x; };
-  const int n_items = full_rounds + (pos_in_round(full_rounds) < tail ? 1 : 0);
+  int n_items = full_rounds + (pos_in_round(full_rounds) < tail ? 1 : 0);
+  int deal_first = 0;
+  if constexpr (DEAL) {
+    deal_first = deal.off[blockIdx.x];
+    n_items = (int)deal.off[blockIdx.x + 1] - deal_first;
+  }
   const int kv_blocks_all = (p.Tk + BK - 1) / BK;
   const int bh_count = p.B * p.Hq;
   auto item_of = [&](int n) -> AttnItem {
-    const int idx = n * G + pos_in_round(n);
+    int idx = n * G + pos_in_round(n);
+    if constexpr (DEAL) idx = deal.list[deal_first + n];
     const int qr = idx / bh_count;
     const int bh = idx - qr * bh_count;
     const int qp = p.causal ? (p.q_pairs - 1 - qr) : qr;

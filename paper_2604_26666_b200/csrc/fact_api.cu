@@ -6,12 +6,15 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <array>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <bitset>
 #include <map>
+#include <memory>
+#include <queue>
 #include <string>
 #include <tuple>
 #include <utility>
@@ -105,6 +108,8 @@ struct fact_handle_s {
   long long launches = 0;
   std::map<TuneKey, fact_config_t> table;
   std::bitset<192> configured_mask;  // kernels whose dynamic shared-memory limit was raised
+  std::unique_ptr<AttnDeal> attn_deal;         // the host's deal of the last causal attention shape (see fact_attention)
+  std::array<long long, 6> attn_deal_key{};
   int kc_clusters[6] = {0, 0, 0, 0, 0, 0};  // clusters of 2 / 4 / 8 CTAs of the K-slice kernel (single CTAs, pairs) the
                                             // device holds at once
   std::string last_error;        // text of the most recent CUDA failure
@@ -1131,6 +1136,34 @@ fact_status_t run(fact_handle_t h, const Problem& q, const fact_config_t* user, 
   return st;
 }
 
+// Which items of a causal attention problem every CTA takes: the items in order of weight (the key blocks an item's
+// later tile sees, plus about one block of fixed cost), each given to the CTA that has the least so far (the lower
+// CTA on a tie, so the first round is CTA c <- item c).  Item idx is (query pair qr = idx / bh counted from the
+// end of the sequence, head idx % bh), the kernel's own numbering.
+void build_attention_deal(int G, long long bh, int q_pairs, int bk, long long seq_kv, AttnDeal& d) {
+  const int items = (int)(bh * q_pairs);
+  const int kv_blocks = (int)((seq_kv + bk - 1) / bk);
+  std::vector<std::vector<uint16_t>> mine((size_t)G);
+  using Slot = std::pair<double, int>;  // (load, CTA)
+  std::priority_queue<Slot, std::vector<Slot>, std::greater<Slot>> heap;
+  for (int c = 0; c < G; ++c) heap.push({0.0, c});
+  for (int idx = 0; idx < items; ++idx) {
+    const int qp = q_pairs - 1 - (int)(idx / bh);
+    const int nb1 = std::min(kv_blocks, (qp * 2 * kAttnBlockQ + 2 * kAttnBlockQ - 1) / bk + 1);
+    const double w = nb1 + (bk == 128 ? 1.0 : 2.0);
+    const Slot s = heap.top();
+    heap.pop();
+    mine[(size_t)s.second].push_back((uint16_t)idx);
+    heap.push({s.first + w, s.second});
+  }
+  int pos = 0;
+  for (int c = 0; c < G; ++c) {
+    d.off[c] = (uint16_t)pos;
+    for (uint16_t v : mine[(size_t)c]) d.list[pos++] = v;
+  }
+  d.off[G] = (uint16_t)pos;
+}
+
 Problem make_problem(fact_op_t op, long long batch, long long M, long long N, long long K, const void* A,
                      long long lda, long long sA, const void* B, long long ldb, long long sB, fact_blayout_t layout,
                      const void* bias, const void* R, long long ldr, long long sR, void* C, long long ldc,
@@ -1246,6 +1279,21 @@ fact_status_t fact_device_info(fact_handle_t h, int* sm_count, int* max_smem, in
   if (max_smem) *max_smem = h->max_smem;
   if (cc_major) *cc_major = h->cc_major;
   if (cc_minor) *cc_minor = h->cc_minor;
+  return FACT_OK;
+}
+
+fact_status_t fact_attention_deal(int ctas, int64_t batch_heads, int64_t seq, int head_dim, int cta, int max_items,
+                                  int32_t* items, int* n_items) {
+  if (ctas < 1 || ctas > kAttnDealCtas || batch_heads < 1 || seq < 1 || (head_dim != 64 && head_dim != 128) || cta < 0 ||
+      cta >= ctas || max_items < 0 || !n_items || (max_items > 0 && !items))
+    return FACT_ERR_INVALID_ARG;
+  const long long q_pairs = (seq + 2 * kAttnBlockQ - 1) / (2 * kAttnBlockQ);
+  if (batch_heads * q_pairs > kAttnDealItems) return FACT_ERR_UNSUPPORTED;
+  std::unique_ptr<AttnDeal> d(new AttnDeal());
+  build_attention_deal(ctas, batch_heads, (int)q_pairs, head_dim == 64 ? 128 : 64, seq, *d);
+  const int n = (int)d->off[cta + 1] - (int)d->off[cta];
+  *n_items = n;
+  for (int i = 0; i < n && i < max_items; ++i) items[i] = d->list[d->off[cta] + i];
   return FACT_OK;
 }
 
@@ -2072,12 +2120,20 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
     const long long ctas = std::min<long long>(p.items, h->sm_count);  // persistent: one CTA per SM
     const int smem = std::max((int)attn_smem_bytes(p.D), kMinSmemRequest);
     if (!h->configured_mask.test(30)) {
-      cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      cudaError_t e = cudaFuncSetAttribute(fact_attention_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(fact_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        e = cudaFuncSetAttribute(fact_attention_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fact_attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fact_attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
       cudaFuncAttributes fa, fb;
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel<64>);
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128>);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fact_attention_kernel<64, false>);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128, false>);
+      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<64, true>);
+      if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, fact_attention_kernel<128, true>);
       if (e == cudaSuccess) fa.numRegs = std::min(fa.numRegs, fb.numRegs);
       if (e != cudaSuccess) {
         st = cuda_fail(h, "cudaFuncSetAttribute(attention)", e);
@@ -2091,10 +2147,33 @@ fact_status_t fact_attention(fact_handle_t h, int64_t batch, int64_t seq_q, int6
       }
     }
     if (st == FACT_OK) {
-      cudaError_t e = head_dim == 64 ? launch_pdl(h, fact_attention_kernel<64>, (unsigned)ctas, (unsigned)kAttnThreads,
-                                                  (size_t)smem, stream, 1, tq, tk, tv, to, p)
-                                     : launch_pdl(h, fact_attention_kernel<128>, (unsigned)ctas, (unsigned)kAttnThreads,
-                                                  (size_t)smem, stream, 1, tq, tk, tv, to, p);
+      // Causal problems of few rounds: the closed-form deal (round by round, every second round reversed) leaves some
+      // CTAs up to 10 % more key blocks than the mean (16 x 12 heads x 1024 tokens: 28 block-times against 25.9), so
+      // the host deals the items out itself -- heaviest first, each to the CTA with the least so far -- and hands the
+      // list to the kernel as a parameter.  The list is kept for the next call of the same shape.
+      const int bk = head_dim == 64 ? 128 : 64;
+      const bool deal = causal != 0 && p.items > ctas && p.items <= kAttnDealItems && ctas <= kAttnDealCtas &&
+                        p.items < 16 * ctas;
+      if (deal) {
+        const std::array<long long, 6> key = {(long long)batch * heads_q, (long long)p.q_pairs, (long long)bk, (long long)seq_kv, (long long)ctas, (long long)seq_q};
+        if (!h->attn_deal || h->attn_deal_key != key) {
+          if (!h->attn_deal) h->attn_deal.reset(new AttnDeal());
+          build_attention_deal((int)ctas, batch * heads_q, p.q_pairs, bk, seq_kv, *h->attn_deal);
+          h->attn_deal_key = key;
+        }
+      }
+      const AttnNoDeal none = {0};
+      cudaError_t e;
+      if (deal)
+        e = head_dim == 64 ? launch_pdl(h, fact_attention_kernel<64, true>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                        (size_t)smem, stream, 1, tq, tk, tv, to, p, *h->attn_deal)
+                           : launch_pdl(h, fact_attention_kernel<128, true>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                        (size_t)smem, stream, 1, tq, tk, tv, to, p, *h->attn_deal);
+      else
+        e = head_dim == 64 ? launch_pdl(h, fact_attention_kernel<64, false>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                        (size_t)smem, stream, 1, tq, tk, tv, to, p, none)
+                           : launch_pdl(h, fact_attention_kernel<128, false>, (unsigned)ctas, (unsigned)kAttnThreads,
+                                        (size_t)smem, stream, 1, tq, tk, tv, to, p, none);
       if (e != cudaSuccess) st = cuda_fail(h, "attention launch", e);
       else h->launches++;
     }

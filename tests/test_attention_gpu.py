@@ -144,6 +144,12 @@ def test_many_ragged_tiles_per_cta(h, causal):
     B, T, Hq, Hkv, D = 40, 333, 8, 2, 64
     q, k, v = rnd((B, T, Hq, D), 31), rnd((B, T, Hkv, D), 32), rnd((B, T, Hkv, D), 33)
     check(h, q, k, v, causal)
+    # 384 items of four different weights at head_dim 128: causal, the host deals them out (fact_attention_deal) and
+    # the kernel walks the list it was handed; the same rows must come out as for any other order
+    B, T, Hq, Hkv, D = 6, 1000, 16, 4, 128
+    q, k, v = rnd((B, T, Hq, D), 131), rnd((B, T, Hkv, D), 132), rnd((B, T, Hkv, D), 133)
+    rows = np.array(sorted({0, 1, 127, 128, 255, 256, 500, 767, 768, 998, 999}), dtype=np.int64)
+    check(h, q, k, v, causal, rows=rows)
 
 
 def test_long_sequence_sampled_rows(h):

@@ -238,3 +238,45 @@ def test_static_status_query_without_a_device(libfact):
     assert libfact.fact_gemm_splitk_static_status(-1, None, byref(v)) == 1
     assert libfact.fact_gemm_splitk_static_status(0, None, None) == 1
     assert libfact.fact_debug_flags(None) == 0
+
+
+@pytest.mark.parametrize("ctas,bh,seq,hd", [(148, 192, 1024, 64), (148, 128, 2048, 128), (148, 20, 4000, 64),
+                                            (7, 5, 1500, 128), (148, 149, 300, 64), (3, 1, 2048, 64)])
+def test_attention_deal_gives_every_item_to_one_cta_and_balances_the_key_blocks(libfact, ctas, bh, seq, hd):
+    """The host's deal of a causal attention problem (fact_attention_deal): every item goes to exactly one CTA, the
+    first round is CTA c <- item c, and no CTA carries more than the mean plus one item's weight (what giving every
+    item, heaviest first, to the CTA with the least so far guarantees)."""
+    from paper_2604_26666_b200.binding import attention_deal
+
+    bk = 128 if hd == 64 else 64
+    q_pairs = (seq + 255) // 256
+    items = bh * q_pairs
+    kv_blocks = (seq + bk - 1) // bk
+
+    def weight(idx):
+        qp = q_pairs - 1 - idx // bh
+        return min(kv_blocks, (qp * 256 + 255) // bk + 1) + (1.0 if bk == 128 else 2.0)
+
+    per_cta = [attention_deal(ctas, bh, seq, hd, c) for c in range(ctas)]
+    seen = sorted(i for lst in per_cta for i in lst)
+    assert seen == list(range(items))
+    for c in range(min(ctas, items)):
+        assert per_cta[c][0] == c
+    loads = [sum(weight(i) for i in lst) for lst in per_cta]
+    mean = sum(loads) / ctas
+    assert max(loads) <= mean + weight(0) + 1e-9
+    # heaviest first inside every CTA
+    for lst in per_cta:
+        assert lst == sorted(lst)
+
+
+def test_attention_deal_argument_errors(libfact):
+    import ctypes
+
+    n = ctypes.c_int(0)
+    buf = (ctypes.c_int32 * 4)()
+    assert libfact.fact_attention_deal(0, 4, 512, 64, 0, 4, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_attention_deal(4, 4, 512, 96, 0, 4, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_attention_deal(4, 4, 512, 64, 4, 4, buf, ctypes.byref(n)) == 1
+    assert libfact.fact_attention_deal(4, 4, 512, 64, 0, 4, buf, None) == 1
+    assert libfact.fact_attention_deal(148, 10000, 512, 64, 0, 4, buf, ctypes.byref(n)) == 3  # more than 8192 items
