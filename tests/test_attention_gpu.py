@@ -183,6 +183,39 @@ def test_repeated_calls_are_bitwise_identical(h):
     assert h.device_status() == 0
 
 
+def test_host_dealt_causal_calls_in_a_cuda_graph_and_between_other_shapes(h):
+    """A causal problem whose items the host deals out (the list travels as a kernel parameter, so a captured launch
+    keeps its own copy): replayed from a CUDA graph, and interleaved with another dealt shape and a shape that is
+    not dealt, every call gives the bits of its first run."""
+    dev = "cuda:0"
+    shapes = [(16, 1024, 12, 12, 64), (6, 1000, 16, 4, 128), (2, 300, 4, 4, 64)]
+    ins, first = [], []
+    for i, (B, T, Hq, Hkv, D) in enumerate(shapes):
+        q, k, v = (rnd((B, T, Hq, D), 50 + i).to(dev), rnd((B, T, Hkv, D), 60 + i).to(dev),
+                   rnd((B, T, Hkv, D), 70 + i).to(dev))
+        ins.append((q, k, v))
+        first.append(h.attention(q, k, v, causal=True).clone())
+    for _ in range(2):
+        for (q, k, v), want in zip(ins, first):
+            assert torch.equal(h.attention(q, k, v, causal=True), want)
+    outs = [torch.empty_like(f) for f in first]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream(dev)):
+        for (q, k, v), o in zip(ins, outs):
+            h.attention(q, k, v, causal=True, out=o)
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for o, want in zip(outs, first):
+            assert torch.equal(o, want)
+    assert h.device_status() == 0
+    rows = np.array([0, 127, 128, 511, 512, 1023], dtype=np.int64)
+    c, t = attention_gates(ins[0][0].cpu(), ins[0][1].cpu(), ins[0][2].cpu(), True, to_f64(first[0])[:, rows], rows=rows)
+    assert c <= 1.0 and t <= 1.0, (c, t)
+
+
 def test_error_codes(h):
     from paper_2604_26666_b200.binding import FactError
     dev = "cuda:0"
